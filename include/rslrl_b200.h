@@ -1,0 +1,242 @@
+/*
+ * rslrl_b200 -- C ABI of the PPO learn-iteration hot path on one NVIDIA B200 (sm_100a).
+ *
+ * The paper (RSL-RL: A Learning Library for Robotics Research) describes the loop in its
+ * section "Implementation Details": a Runner alternates environment stepping with agent
+ * learning; the Algorithm is PPO (section "Features / Algorithms", after Schulman et al.
+ * 2017) on MLP Networks; observations come in groups that are routed to different modules
+ * (actor vs. privileged critic); environments use same-step reset and episodic time-outs
+ * are handled properly; section "Auxiliary Techniques" adds mirrored-state augmentation with
+ * an optional symmetry loss.  One learn iteration through this library is
+ *
+ *     for t in 0..T-1:   rslrl_act(obs_t)  ->  actions;   simulator steps;   rslrl_record_step(r, done, timeout)
+ *     rslrl_gae(obs_T);   rslrl_ppo_update();
+ *
+ * Conventions
+ *   - "d_" pointers are DEVICE pointers, "h_" pointers are HOST pointers.  Buffers passed in
+ *     by the caller need the natural alignment of their element type (4 bytes for float)
+ *     unless a call says otherwise, and must stay valid until the context's stream has
+ *     executed the call.  Buffers owned by the library are 16-byte aligned.
+ *   - All calls enqueue on the CUDA stream given to rslrl_create and return without a host
+ *     synchronisation unless stated.  A context is not thread-safe.
+ *   - Every function returns an rslrl_status; nothing throws, aborts or traps the device.
+ *     Argument errors are found on the host before anything is launched.
+ *     rslrl_last_error gives a human-readable message for the last failure of a context.
+ *   - The library owns the context, the rollout storage, the parameters, the optimiser state
+ *     and all scratch memory; it allocates them in rslrl_create and nowhere else.
+ */
+#ifndef RSLRL_B200_H
+#define RSLRL_B200_H
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef enum {
+    RSLRL_OK = 0,
+    RSLRL_ERR_INVALID_ARG = 1,   /* null pointer, negative size, unknown enum value           */
+    RSLRL_ERR_SHAPE = 2,         /* e.g. T*N not divisible by the number of minibatches       */
+    RSLRL_ERR_ALIGNMENT = 3,     /* a pointer does not have the alignment the call requires   */
+    RSLRL_ERR_STATE = 4,         /* call order: act/record after T steps, gae before T steps  */
+    RSLRL_ERR_UNSUPPORTED = 5,   /* a size beyond a documented limit                          */
+    RSLRL_ERR_CUDA = 6,          /* a CUDA runtime call failed; see rslrl_last_error          */
+    RSLRL_ERR_NONFINITE = 7,     /* a loss or gradient norm was not finite                    */
+    RSLRL_ERR_TIMEOUT = 8        /* a bounded wait inside a kernel ran out; results invalid   */
+} rslrl_status;
+
+/* Arithmetic of the hidden-layer matrix products.  Accumulation, bias, ELU, losses, master
+ * weights, gradients and Adam are FP32 in every mode. */
+typedef enum {
+    RSLRL_FP32 = 0,              /* FP32 operands on the FP32 pipes                           */
+    RSLRL_TF32 = 1,              /* TF32 operands on the tensor cores                         */
+    RSLRL_BF16 = 2               /* BF16 operands on the tensor cores                         */
+} rslrl_precision;
+
+#define RSLRL_MAX_HIDDEN 8
+
+/* Networks (paper: "Network architectures used by the algorithm"; MLPs, ELU hidden
+ * activations, linear heads; diagonal Gaussian policy with a learned state-independent
+ * log-std). */
+typedef struct {
+    int32_t num_envs;                         /* N                                             */
+    int32_t num_steps;                        /* T                                             */
+    int32_t actor_obs_dim;                    /* D_a                                           */
+    int32_t critic_obs_dim;                   /* D_c                                           */
+    int32_t num_actions;                      /* A  (1..64)                                    */
+    int32_t shared_obs;                       /* 1: actor and critic read the same observation
+                                                 (D_a == D_c); stored once                     */
+    int32_t num_actor_hidden;                 /* 1..RSLRL_MAX_HIDDEN                           */
+    int32_t actor_hidden[RSLRL_MAX_HIDDEN];
+    int32_t num_critic_hidden;
+    int32_t critic_hidden[RSLRL_MAX_HIDDEN];
+    float   elu_alpha;                        /* 1.0                                           */
+    int32_t precision;                        /* rslrl_precision                               */
+} rslrl_model_cfg;
+
+/* PPO hyper-parameters (Schulman et al. 2017, as named by the paper's "Algorithms"). */
+typedef struct {
+    float   gamma, lam;                       /* discount, GAE lambda                          */
+    float   clip;                             /* surrogate clip range c                        */
+    float   value_clip;                       /* value clip range c_v                          */
+    float   value_coef;                       /* k_v                                           */
+    float   entropy_coef;                     /* k_e                                           */
+    int32_t use_clipped_value_loss;
+    int32_t epochs, minibatches;              /* E, M; T*N must be divisible by M              */
+    float   lr, lr_min, lr_max, lr_factor;    /* initial step size and the adaptive rule       */
+    float   desired_kl;
+    int32_t adaptive_lr;
+    float   max_grad_norm;
+    float   adam_b1, adam_b2, adam_eps;
+    int32_t normalize_adv;                    /* normalise advantages inside rslrl_gae         */
+    int32_t adv_std_unbiased;                 /* 1: divide the variance by B-1, 0: by B        */
+    float   adv_eps;
+    /* Symmetry augmentation (paper: "Auxiliary Techniques").  (S x)[i] = sign[i]*x[perm[i]].
+     * HOST pointers, copied by rslrl_create; ignored when sym_enable == 0. */
+    int32_t sym_enable;
+    float   sym_coef;
+    const int32_t *h_sym_obs_perm;  const float *h_sym_obs_sign;    /* [D_a] */
+    const int32_t *h_sym_cobs_perm; const float *h_sym_cobs_sign;   /* [D_c] */
+    const int32_t *h_sym_act_perm;  const float *h_sym_act_sign;    /* [A]   */
+    uint64_t seed;                            /* keys the sampling noise and the shuffles      */
+} rslrl_ppo_cfg;
+
+/* Structure-of-arrays rollout storage (DEVICE pointers, owned by the context).  Every base
+ * pointer is 16-byte aligned and every row stride is a multiple of 4 floats.  [t][n] arrays
+ * are t-major so that consecutive environments are consecutive in memory. */
+typedef struct {
+    int32_t T, N;
+    int32_t step;                             /* transitions recorded so far in this rollout   */
+    int32_t obs_a_stride, obs_c_stride, act_stride;   /* row strides in floats                 */
+    float  *obs_actor;                        /* [T][N][obs_a_stride]                          */
+    float  *obs_critic;                       /* [T][N][obs_c_stride]; == obs_actor if shared  */
+    float  *actions;                          /* [T][N][act_stride]                            */
+    float  *mu;                               /* [T][N][act_stride]   policy mean at act time  */
+    float  *sigma;                            /* [T][act_stride]      policy std  at act time  */
+    float  *logp, *values, *rewards, *returns, *advantages;         /* [T][N]                  */
+    uint8_t *dones, *timeouts;                /* [T][N] 0/1                                    */
+} rslrl_storage;
+
+/* Scalars of one rslrl_ppo_update call (means over its E*M minibatch steps, except where
+ * stated). */
+typedef struct {
+    float   surrogate, value_loss, entropy, sym_loss, kl;
+    float   first_surrogate, first_value_loss, first_kl, first_sym_loss;  /* first minibatch  */
+    float   first_grad_norm, last_grad_norm;
+    float   lr;                               /* learning rate after the call                  */
+    int32_t steps;                            /* optimiser steps taken (E*M)                   */
+    int32_t nonfinite;                        /* 1 if any loss / grad norm was not finite      */
+} rslrl_update_stats;
+
+typedef struct rslrl_ctx rslrl_ctx;
+
+/* Number of FP32 parameters of the model, in the flat order
+ *   actor  W1[in][out], b1, ..., Wout, bout, log_std[A],  critic W1, b1, ..., Wout, bout
+ * with every W row-major [fan_in][fan_out].  Returns 0 on an invalid configuration. */
+size_t rslrl_num_params(const rslrl_model_cfg *model);
+
+/* Create a context on the current CUDA device.  `cuda_stream` is a cudaStream_t (NULL = the
+ * legacy default stream).  Allocates storage, parameters (zero; log_std zero), optimiser state
+ * and scratch.  Synchronises the stream once. */
+rslrl_status rslrl_create(const rslrl_model_cfg *model, const rslrl_ppo_cfg *ppo,
+                          void *cuda_stream, rslrl_ctx **out);
+rslrl_status rslrl_destroy(rslrl_ctx *ctx);
+const char  *rslrl_last_error(const rslrl_ctx *ctx);   /* ctx may be NULL: last create error  */
+
+/* Borrowed view of the storage; pointers stay valid until rslrl_destroy. */
+rslrl_status rslrl_storage_view(rslrl_ctx *ctx, rslrl_storage *out);
+
+/* Parameters, last pre-clip gradient, Adam moments: HOST flat arrays of rslrl_num_params
+ * floats.  These calls synchronise the stream. */
+rslrl_status rslrl_set_params(rslrl_ctx *ctx, const float *h_flat, size_t n);
+rslrl_status rslrl_get_params(rslrl_ctx *ctx, float *h_flat, size_t n);
+rslrl_status rslrl_get_grads(rslrl_ctx *ctx, float *h_flat, size_t n);
+rslrl_status rslrl_get_adam(rslrl_ctx *ctx, float *h_m, float *h_v, size_t n);
+rslrl_status rslrl_set_adam(rslrl_ctx *ctx, const float *h_m, const float *h_v, size_t n);
+
+/* Optimiser / counter state for checkpoint and resume.  set takes effect immediately. */
+typedef struct {
+    float    lr;                 /* current learning rate                                     */
+    int32_t  adam_step;          /* optimiser steps taken so far                              */
+    uint32_t global_step;        /* rslrl_act calls so far (indexes the sampling noise)       */
+    uint32_t iteration;          /* rslrl_ppo_update calls so far (indexes the shuffles)      */
+} rslrl_counters;
+rslrl_status rslrl_get_counters(rslrl_ctx *ctx, rslrl_counters *out);
+rslrl_status rslrl_set_counters(rslrl_ctx *ctx, const rslrl_counters *in);
+
+/* (1) PPO rollout step (paper: "Algorithms", stochastic on-policy PPO; observation groups
+ * routed to actor and critic).  For every environment n: mu = actor(o_a), V = critic(o_c),
+ * a = mu + exp(log_std) * eps, eps ~ N(0,1) from Philox-4x32-10 keyed by the seed with counter
+ * (n, global_step, action quad, 1), and the Gaussian log-density of a.  Writes row `step` of
+ * the storage (observations, actions, mu, sigma, logp, values) and, if d_actions_out is not
+ * NULL, the actions to d_actions_out[N][act_stride].
+ *   d_actor_obs  [N][actor_obs_dim]  float32, dense rows (device)
+ *   d_critic_obs [N][critic_obs_dim] float32 (device); with shared_obs it may be NULL or equal
+ *                to d_actor_obs.
+ * RSLRL_ERR_STATE if T steps were already taken in this rollout. */
+rslrl_status rslrl_act(rslrl_ctx *ctx, const float *d_actor_obs, const float *d_critic_obs,
+                       float *d_actions_out);
+
+/* Record the simulator's answer to the last rslrl_act: rewards[N] float32, dones[N] and
+ * timeouts[N] bytes (0/1; a time-out is also a done) -- device pointers.  Advances `step`. */
+rslrl_status rslrl_record_step(rslrl_ctx *ctx, const float *d_rewards, const uint8_t *d_dones,
+                               const uint8_t *d_timeouts);
+
+/* (2) Returns and advantages (paper: "Implementation Details": proper handling of episodic
+ * time-outs under same-step reset).  V_T = critic(o_T); reverse scan over t with A_T = 0:
+ *     r~ = r_t + gamma V_t timeout_t;  delta = r~ + gamma V_{t+1} (1-done_t) - V_t
+ *     A_t = delta + gamma lam (1-done_t) A_{t+1};   R_t = A_t + V_t
+ * then, if normalize_adv, A <- (A - mean) / (std + adv_eps) over all T*N transitions.
+ *   d_last_critic_obs [N][critic_obs_dim] float32 (device): the observation after the last step.
+ * RSLRL_ERR_STATE unless exactly T steps were recorded. */
+rslrl_status rslrl_gae(rslrl_ctx *ctx, const float *d_last_critic_obs);
+
+/* (3) The minibatch PPO update (paper: "Algorithms" PPO; "Auxiliary Techniques" symmetry).
+ * For E epochs: shuffle the T*N transitions with a keyed bijection, cut into M minibatches;
+ * per minibatch: gather (plus mirrored copies when sym_enable), actor/critic forward, clipped
+ * surrogate + clipped value loss - entropy bonus (+ symmetry loss), backward, KL(old||new) ->
+ * adaptive learning rate, global grad-norm clip, Adam.  Starts a new rollout (step = 0).
+ * If h_stats is not NULL the call synchronises the stream and fills it; otherwise it only
+ * enqueues.  RSLRL_ERR_STATE unless rslrl_gae ran on this rollout. */
+rslrl_status rslrl_ppo_update(rslrl_ctx *ctx, rslrl_update_stats *h_stats);
+
+/* Variant of rslrl_ppo_update that stops after `max_steps` minibatch steps (tests compare the
+ * state after exactly one optimiser step).  max_steps <= 0 means all E*M steps. */
+rslrl_status rslrl_ppo_update_steps(rslrl_ctx *ctx, int32_t max_steps, rslrl_update_stats *h_stats);
+
+/* Host-buffer variants of the per-step calls: the same work with the host<->device copies
+ * inside the call (pinned host memory makes them asynchronous).  h_actions_out[N][A] dense;
+ * when it is not NULL the call waits for the actions. */
+rslrl_status rslrl_act_host(rslrl_ctx *ctx, const float *h_actor_obs, const float *h_critic_obs,
+                            float *h_actions_out);
+rslrl_status rslrl_record_step_host(rslrl_ctx *ctx, const float *h_rewards, const uint8_t *h_dones,
+                                    const uint8_t *h_timeouts);
+rslrl_status rslrl_gae_host(rslrl_ctx *ctx, const float *h_last_critic_obs);
+
+/* Stand-alone pieces of the path on caller-owned DEVICE buffers (used for size sweeps and
+ * roofline measurements; same kernels as the context calls).
+ *
+ * rslrl_gae_scan: the reverse scan and normalisation of (2) on [T][N] arrays, V_T given.
+ *   d_scratch: at least rslrl_gae_scratch_bytes(T, N) bytes of device memory; d_advantages and
+ *   d_scratch must be 16-byte aligned.
+ * rslrl_minibatch_indices: row indices of minibatch k of `epoch` (the keyed Feistel shuffle of
+ *   B = T*N rows cut into M chunks): d_rows_out[B/M] int32. */
+size_t       rslrl_gae_scratch_bytes(int32_t T, int32_t N);
+rslrl_status rslrl_gae_scan(const float *d_rewards, const float *d_values, const uint8_t *d_dones,
+                            const uint8_t *d_timeouts, const float *d_last_values,
+                            float *d_returns, float *d_advantages, int32_t T, int32_t N,
+                            float gamma, float lam, int32_t normalize, int32_t unbiased,
+                            float adv_eps, void *d_scratch, void *cuda_stream);
+rslrl_status rslrl_minibatch_indices(uint64_t seed, uint32_t iteration, uint32_t epoch,
+                                     int32_t batch, int32_t minibatches, int32_t k,
+                                     int32_t *d_rows_out, void *cuda_stream);
+
+/* Number of kernels this library has launched in the current process (all contexts). */
+uint64_t     rslrl_kernel_launch_count(void);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* RSLRL_B200_H */

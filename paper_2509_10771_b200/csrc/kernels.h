@@ -1,0 +1,169 @@
+// Host-side launchers of the rslrl_b200 kernels (internal; the public boundary is
+// include/rslrl_b200.h).  Every launcher enqueues on `stream` and returns the CUDA status of
+// the launch.
+#pragma once
+#include <cuda_runtime.h>
+#include <cuda_bf16.h>
+#include <stdint.h>
+
+namespace rslrl {
+
+void count_launch(int n = 1);
+
+// ------------------------------------------------------------------------- SIMT FP32 GEMM
+// C[M x N] = op(A)[M x K] * op(B)[K x N] followed by an epilogue.  Leading dimensions are
+// multiples of 4 floats and base pointers 16-byte aligned.
+enum GemmEpilogue {
+    EPI_BIAS_ELU = 0,   // C = ELU(acc + bias[n]); columns [N, Cn) are written as 0
+    EPI_BIAS = 1,       // C = acc + bias[n]
+    EPI_DELU = 2,       // C = acc * ELU'(aux[m][n])        (aux = stored post-activation)
+    EPI_PLAIN = 3       // C = acc                           (split partial of a weight gradient)
+};
+
+struct GemmProblem {
+    const float* A; const float* B; float* C;
+    const float* bias; const float* aux;
+    int lda, ldb, ldc, ldaux;
+    int M, N, K;
+    int Cn;                 // columns written per row (N <= Cn <= ldc)
+    int splits;             // the K range is cut into `splits` chunks of `kchunk`
+    int kchunk;
+    long long split_stride; // distance in floats between the C of consecutive splits
+};
+
+struct GemmBatch {
+    GemmProblem p[2];
+    int count;
+    float alpha;            // ELU alpha
+};
+
+// transA: A(m,k) = A[k*lda + m] instead of A[m*lda + k]; transB: B(k,n) = B[n*ldb + k].
+cudaError_t launch_sgemm(const GemmBatch& b, bool transA, bool transB, int epilogue,
+                         cudaStream_t stream);
+
+// Column sums of X[rows][ld] over a split of the rows: out[s * split_stride + n].
+constexpr int kMaxColsum = 16;
+struct ColsumProblem { const void* X; float* out; int rows, n, ld; };
+struct ColsumBatch { ColsumProblem p[kMaxColsum]; int count; int splits; long long split_stride; int is_bf16; };
+cudaError_t launch_colsum(const ColsumBatch& b, cudaStream_t stream);
+
+// ------------------------------------------------------------------------- rollout kernels
+// dst[n][dst_ld] <- src[n][dim] (zero padded), optionally a second destination in bf16.
+cudaError_t launch_pad_rows(const float* src, int dim, float* dst, int dst_ld,
+                            __nv_bfloat16* dst16, int dst16_ld, int rows, cudaStream_t stream);
+
+struct HeadParams {                 // final linear layers of actor and critic
+    const float* Wa; const float* ba; int ldwa;      // [n_a][ldwa], ldwa = round4(A)
+    const float* Wc; const float* bc; int ldwc;      // [n_c][ldwc], ldwc = 4
+    const float* log_std;
+    int n_a, n_c, A;                                  // widths of the last hidden layers
+};
+
+struct ActOut {
+    float* actions; float* mu; float* sigma; float* logp; float* values;   // storage row t
+    float* actions_out;                                                    // may be null
+    int act_stride;
+};
+// Head + Gaussian sample + log-density for N rows; hidden activations are float or bf16.
+cudaError_t launch_act_head(const void* Ha, int ldha, const void* Hc, int ldhc, bool bf16_act,
+                            const HeadParams& hp, const ActOut& out, int N, uint64_t seed,
+                            uint32_t global_step, cudaStream_t stream);
+// Critic head only: values[N].
+cudaError_t launch_value_head(const void* Hc, int ldhc, bool bf16_act, const HeadParams& hp,
+                              float* values, int N, cudaStream_t stream);
+
+cudaError_t launch_record_step(const float* rew, const uint8_t* dones, const uint8_t* timeouts,
+                               float* s_rew, uint8_t* s_dones, uint8_t* s_timeouts, int N,
+                               cudaStream_t stream);
+
+// GAE reverse scan + block moments; then normalisation.  scratch: 3 floats per scan block.
+int gae_scan_blocks(int N);
+cudaError_t launch_gae(const float* rewards, const float* values, const uint8_t* dones,
+                       const uint8_t* timeouts, const float* last_values, float* returns,
+                       float* advantages, int T, int N, float gamma, float lam, int normalize,
+                       int unbiased, float adv_eps, float* scratch, cudaStream_t stream);
+
+// ------------------------------------------------------------------------- update kernels
+struct SymTables {                  // device pointers; null when symmetry is off
+    const int* obs_perm; const float* obs_sign;
+    const int* cobs_perm; const float* cobs_sign;
+    const int* act_perm; const float* act_sign;
+};
+
+struct GatherArgs {
+    // storage
+    const float* obs_a; const float* obs_c; const float* actions; const float* mu;
+    const float* sigma; const float* logp; const float* values; const float* returns;
+    const float* adv;
+    int N, sa, sc, as, Da, Dc, A;
+    int shared_obs;
+    // minibatch destination (rows [0,Bmb) originals, [Bmb,2Bmb) mirrored when sym)
+    float* x_a; float* x_c; int ldxa, ldxc;                 // fp32 (null in bf16 mode)
+    __nv_bfloat16* x_a16; __nv_bfloat16* x_c16; int ldxa16, ldxc16;
+    float* act_mb; float* mu_old; float* sigma_old;         // [R][as], [Bmb][as], [Bmb][as]
+    float* logp_old; float* v_old; float* ret; float* adv_mb;   // [Bmb]
+    int* rows_out;                                          // [Bmb] source indices (may be null)
+    int Bmb; int sym;
+    SymTables st;
+    uint32_t seed_lo, seed_hi, iteration, epoch, batch, first;   // first = k * Bmb
+};
+cudaError_t launch_gather(const GatherArgs& a, cudaStream_t stream);
+cudaError_t launch_perm_rows(uint64_t seed, uint32_t iteration, uint32_t epoch, uint32_t batch,
+                             uint32_t first, int count, int* rows_out, cudaStream_t stream);
+
+struct LossHyper {
+    float clip, value_clip, value_coef, entropy_coef, sym_coef, alpha;
+    int use_clipped_value_loss;
+};
+
+// Slots of the loss sums; slot LS_COUNT holds the policy entropy.
+enum { LS_SURR = 0, LS_VALUE = 1, LS_KL = 2, LS_SYM = 3, LS_COUNT = 4 };
+
+struct HeadLossArgs {
+    const void* Ha; const void* Hc; int ldha, ldhc; int bf16_act;
+    HeadParams hp;
+    const float* act_mb; const float* mu_old; const float* sigma_old; int as;
+    const float* logp_old; const float* v_old; const float* ret; const float* adv;
+    const float* act_sign; const int* act_perm;       // mirror of actions (null when sym off)
+    int Bmb; int sym;
+    LossHyper h;
+    // outputs
+    float* dmu; int lddmu;          // [R][round4(A)]   fp32
+    float* dv;                      // [R][4]  column 0 = dL/dV, columns 1..3 zero
+    __nv_bfloat16* dmu16; int lddmu16; __nv_bfloat16* dv16; int lddv16;   // bf16 twins (may be null)
+    void* dZa; void* dZc; int lddza, lddzc;           // dL/dz of the last hidden layers
+    float* block_partials;          // [blocks][head_partial_stride()]  (losses, db_head, dlog_std)
+    float* mu_out; float* v_out;    // optional copies of mu [R][as] and V [R] (may be null)
+};
+int head_loss_blocks(int Bmb);
+int head_partial_stride();
+cudaError_t launch_head_loss(const HeadLossArgs& a, cudaStream_t stream);
+// Sums the head_loss block partials: loss sums -> loss_sums[0..LS_COUNT), entropy ->
+// loss_sums[LS_COUNT], head-bias and log_std gradients -> split 0 of the gradient partials.
+cudaError_t launch_head_finalize(const float* block_partials, int nblocks, float* partials0, int off_ba,
+                                 int off_logstd, int off_bc, int A, float entropy_coef,
+                                 const float* log_std, float* loss_sums, cudaStream_t stream);
+
+struct ReduceArgs {
+    const float* partials; int splits; long long split_stride;   // gradient partials [splits][P]
+    float* grad; int P;                                            // padded device layout
+    float* sumsq_partials;          // [reduce_blocks(P)]
+};
+int reduce_blocks(int P);
+cudaError_t launch_reduce(const ReduceArgs& a, cudaStream_t stream);
+
+struct AdamArgs {
+    float* param; float* m; float* v; const float* grad; int P;
+    const float* sumsq_partials; int nsumsq;
+    const float* loss_sums;
+    float inv_rows_all, inv_rows_orig, inv_sym;      // 1/R, 1/Bmb, 1/(Bmb*A)
+    float* lr_io;                   // [2] double-buffered learning rate
+    int* step_io;                   // [2] double-buffered optimiser step count
+    int parity;                     // which slot is current
+    float lr_min, lr_max, lr_factor, desired_kl; int adaptive;
+    float max_norm, b1, b2, eps;
+    float* stats_row;               // [8]: surr, value, entropy, sym, kl, grad_norm, lr, nonfinite
+};
+cudaError_t launch_adam(const AdamArgs& a, cudaStream_t stream);
+
+}  // namespace rslrl
