@@ -1,0 +1,730 @@
+// Tensor-core engine: the hidden-layer products of act, forward and backward as grouped,
+// persistent tcgen05 GEMM kernels.  Operands are BF16 tiles staged in shared memory by TMA
+// (128-byte swizzle), accumulators are FP32 in tensor memory (two buffers, so the epilogue of
+// one tile overlaps the main loop of the next), and the epilogues fuse bias+ELU (forward),
+// the ELU derivative (data gradient) or the split-partial store (weight gradient).
+//
+// Warp roles in a CTA of 320 threads: warp 0 = TMA producer, warp 1 = MMA issuer and owner of
+// the tensor-memory allocation, warps 2..9 = epilogue (each reads its quarter of the 128
+// accumulator lanes and half of the tile's columns).
+//
+// Every wait on an mbarrier is bounded in time; on expiry the CTA raises an error flag that
+// the host reads, drains its own asynchronous work, frees its tensor memory and returns.
+#include "umma.h"
+
+#include <cuda.h>
+#include <algorithm>
+#include <cstring>
+#include <vector>
+
+namespace rslrl {
+
+namespace {
+
+constexpr int kStages = 4;
+constexpr int BLOCK_M = 128;
+constexpr int BLOCK_K = 64;                      // bf16 elements = one 128-byte swizzle row
+constexpr int UMMA_K = 16;
+constexpr int kMaxBN = 256;
+constexpr int kEpiWarps = 8;
+constexpr int kThreads = 32 * (2 + kEpiWarps);
+constexpr uint32_t kStageA = BLOCK_M * BLOCK_K * 2;      // 16 KiB
+constexpr uint32_t kStageB = kMaxBN * BLOCK_K * 2;       // 32 KiB
+constexpr uint32_t kTmemCols = 512;                      // two accumulator buffers of 256 columns
+constexpr int kMaxProblems = 8;
+constexpr size_t kSmemBytes = 1024 + kStages * (kStageA + kStageB) + 256;
+constexpr unsigned long long kWaitLimitNs = 2000000000ull;   // 2 s
+
+enum TcMode { TC_FWD = 0, TC_DGRAD = 1, TC_WGRAD = 2 };
+
+struct TcProblem {
+    int m_extent, n_extent;        // rows / columns of D that exist (stores are clipped to them)
+    int m_tiles, n_tiles, bn;
+    int kblocks;                   // k-blocks of 64 along the contraction
+    int splits, kb_per_split;      // weight gradient: the contraction is cut into splits
+    int item_begin;
+    const float* bias; int bias_n;
+    __nv_bfloat16* out16; int ld_out;
+    const __nv_bfloat16* aux16; int ld_aux;
+    float* out32; int ld_out32; long long split_stride;
+};
+
+struct TcParams {
+    CUtensorMap tmA[kMaxProblems];
+    CUtensorMap tmB[kMaxProblems];
+    TcProblem p[kMaxProblems];
+    int count, total_items;
+    float alpha;
+    int* error;
+};
+
+// ------------------------------------------------------------------------------ PTX wrappers
+__device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
+
+__device__ __forceinline__ void mbar_init(uint64_t* bar, uint32_t count) {
+    asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(smem_u32(bar)), "r"(count));
+}
+__device__ __forceinline__ void mbar_expect_tx(uint64_t* bar, uint32_t bytes) {
+    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(smem_u32(bar)), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ void mbar_arrive(uint64_t* bar) {
+    asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(smem_u32(bar)) : "memory");
+}
+__device__ __forceinline__ bool mbar_try_wait(uint64_t* bar, uint32_t parity) {
+    uint32_t ok;
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+        "selp.b32 %0, 1, 0, p;\n\t}"
+        : "=r"(ok) : "r"(smem_u32(bar)), "r"(parity) : "memory");
+    return ok != 0;
+}
+__device__ __forceinline__ unsigned long long global_ns() {
+    unsigned long long t;
+    asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
+    return t;
+}
+// Bounded wait.  Returns false when the wait ran out of time or another role gave up.
+__device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity, volatile int* abort_flag, int* error, int code) {
+    if (mbar_try_wait(bar, parity)) return true;
+    const unsigned long long t0 = global_ns();
+    while (true) {
+        if (mbar_try_wait(bar, parity)) return true;
+        if (*abort_flag) return false;
+        if (global_ns() - t0 > kWaitLimitNs) {
+            *abort_flag = 1;
+            atomicExch(error, code);
+            return false;
+        }
+    }
+}
+
+__device__ __forceinline__ void tma_load_2d(void* smem_dst, const CUtensorMap* tm, int x, int y, uint64_t* bar) {
+    asm volatile(
+        "cp.async.bulk.tensor.2d.shared::cluster.global.tile.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];"
+        ::"r"(smem_u32(smem_dst)), "l"(tm), "r"(x), "r"(y), "r"(smem_u32(bar)) : "memory");
+}
+__device__ __forceinline__ void tma_prefetch_desc(const CUtensorMap* tm) {
+    asm volatile("prefetch.tensormap [%0];" ::"l"(tm) : "memory");
+}
+
+__device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
+__device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
+
+__device__ __forceinline__ void tmem_alloc(uint32_t* slot, uint32_t cols) {
+    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(slot)), "r"(cols) : "memory");
+    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+}
+__device__ __forceinline__ void tmem_dealloc(uint32_t addr, uint32_t cols) {
+    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(addr), "r"(cols) : "memory");
+}
+// D[tmem] (+)= A[smem] * B[smem]
+__device__ __forceinline__ void umma_bf16(uint32_t d_tmem, uint64_t a_desc, uint64_t b_desc, uint32_t idesc, uint32_t accumulate) {
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "setp.ne.b32 p, %4, 0;\n\t"
+        "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}"
+        ::"r"(d_tmem), "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(accumulate) : "memory");
+}
+// The mbarrier gets one arrival when all tcgen05 operations issued so far by this thread are done.
+__device__ __forceinline__ void umma_commit(uint64_t* bar) {
+    asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(smem_u32(bar)) : "memory");
+}
+__device__ __forceinline__ void tmem_ld32(uint32_t taddr, uint32_t (&r)[32]) {
+    asm volatile(
+        "tcgen05.ld.sync.aligned.32x32b.x32.b32 "
+        "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, "
+        "%16, %17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31}, [%32];"
+        : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]),
+          "=r"(r[8]), "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15]),
+          "=r"(r[16]), "=r"(r[17]), "=r"(r[18]), "=r"(r[19]), "=r"(r[20]), "=r"(r[21]), "=r"(r[22]), "=r"(r[23]),
+          "=r"(r[24]), "=r"(r[25]), "=r"(r[26]), "=r"(r[27]), "=r"(r[28]), "=r"(r[29]), "=r"(r[30]), "=r"(r[31])
+        : "r"(taddr) : "memory");
+    asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
+}
+
+// Shared-memory matrix descriptor, 128-byte swizzle.  Byte offsets are encoded in 16-byte units.
+//   K-major tile (rows of 128 bytes along the contraction): groups of 8 rows are 1024 bytes
+//     apart (stride offset); the leading offset is not used by swizzled K-major layouts.
+//   MN-major tile (rows of 128 bytes along M/N, one row per contraction index): consecutive
+//     blocks of 64 M/N elements are `lead_bytes` apart, groups of 8 contraction rows 1024 bytes.
+__device__ __forceinline__ uint64_t smem_desc(uint32_t addr, uint32_t lead_bytes, uint32_t stride_bytes) {
+    uint64_t d = 0;
+    d |= (uint64_t)((addr >> 4) & 0x3FFFu);
+    d |= (uint64_t)((lead_bytes >> 4) & 0x3FFFu) << 16;
+    d |= (uint64_t)((stride_bytes >> 4) & 0x3FFFu) << 32;
+    d |= 1ull << 46;                 // descriptor version of this architecture
+    d |= 2ull << 61;                 // 128-byte swizzle
+    return d;
+}
+
+// Instruction descriptor: BF16 x BF16 -> FP32, M = 128, N = bn; major bits: 0 = K-major, 1 = MN-major.
+__device__ __forceinline__ uint32_t instr_desc(int bn, int a_mn_major, int b_mn_major) {
+    return (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)a_mn_major << 15) | ((uint32_t)b_mn_major << 16) |
+           ((uint32_t)(bn >> 3) << 17) | ((uint32_t)(BLOCK_M >> 4) << 24);
+}
+
+struct Item { int prob, m0, n0, kb0, kb1, split; };
+
+__device__ __forceinline__ Item decode_item(const TcParams& P, int item) {
+    int pi = 0;
+#pragma unroll 1
+    for (int i = 1; i < P.count; ++i)
+        if (item >= P.p[i].item_begin) pi = i;
+    const TcProblem& p = P.p[pi];
+    const int local = item - p.item_begin;
+    const int per_split = p.m_tiles * p.n_tiles;
+    Item it;
+    it.prob = pi;
+    it.split = local / per_split;
+    const int rem = local - it.split * per_split;
+    it.m0 = (rem / p.n_tiles) * BLOCK_M;
+    it.n0 = (rem % p.n_tiles) * p.bn;
+    it.kb0 = it.split * p.kb_per_split;
+    it.kb1 = min(p.kblocks, it.kb0 + p.kb_per_split);
+    return it;
+}
+
+__device__ __forceinline__ float elu_fast(float z, float alpha) { return z > 0.f ? z : alpha * (__expf(z) - 1.0f); }
+
+template <int MODE>
+__global__ void __launch_bounds__(kThreads, 1) tc_gemm_kernel(const __grid_constant__ TcParams P) {
+    extern __shared__ uint8_t smem_raw[];
+    uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
+    uint8_t* sA = smem;
+    uint8_t* sB = smem + kStages * kStageA;
+    uint64_t* full = reinterpret_cast<uint64_t*>(sB + kStages * kStageB);
+    uint64_t* empty = full + kStages;
+    uint64_t* tfull = empty + kStages;
+    uint64_t* tempty = tfull + 2;
+    uint64_t* drain = tempty + 2;
+    uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(drain + 1);
+    volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
+
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    if (threadIdx.x == 0) {
+        for (int s = 0; s < kStages; ++s) { mbar_init(&full[s], 1); mbar_init(&empty[s], 1); }
+        for (int b = 0; b < 2; ++b) { mbar_init(&tfull[b], 1); mbar_init(&tempty[b], kEpiWarps); }
+        mbar_init(drain, 1);
+        *abort_flag = 0;
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+        asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+    }
+    if (warp == 1) tmem_alloc(tmem_slot, kTmemCols);
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    const uint32_t tmem_base = *tmem_slot;
+
+    if (warp == 0) {
+        // ================================ TMA producer =================================
+        if (lane == 0) {
+            for (int i = 0; i < P.count; ++i) { tma_prefetch_desc(&P.tmA[i]); tma_prefetch_desc(&P.tmB[i]); }
+            int stage = 0; uint32_t phase = 0;
+            uint32_t issued_mask = 0, issued_parity = 0;
+            bool ok = true;
+            for (int item = blockIdx.x; ok && item < P.total_items; item += gridDim.x) {
+                const Item it = decode_item(P, item);
+                const TcProblem& p = P.p[it.prob];
+                const uint32_t bytes = (uint32_t)(BLOCK_M + p.bn) * BLOCK_K * 2;
+                for (int kb = it.kb0; kb < it.kb1; ++kb) {
+                    if (!mbar_wait(&empty[stage], phase ^ 1u, abort_flag, P.error, 1)) { ok = false; break; }
+                    mbar_expect_tx(&full[stage], bytes);
+                    uint8_t* a_dst = sA + stage * kStageA;
+                    uint8_t* b_dst = sB + stage * kStageB;
+                    if (MODE == TC_WGRAD) {
+                        // operands are [row][feature] with the feature contiguous: boxes of
+                        // 64 features x 64 rows, one 8 KiB block per 64 features
+                        for (int i = 0; i < 2; ++i)
+                            tma_load_2d(a_dst + i * 8192, &P.tmA[it.prob], it.m0 + 64 * i, kb * BLOCK_K, &full[stage]);
+                        for (int j = 0; j < p.bn / 64; ++j)
+                            tma_load_2d(b_dst + j * 8192, &P.tmB[it.prob], it.n0 + 64 * j, kb * BLOCK_K, &full[stage]);
+                    } else {
+                        tma_load_2d(a_dst, &P.tmA[it.prob], kb * BLOCK_K, it.m0, &full[stage]);
+                        tma_load_2d(b_dst, &P.tmB[it.prob], kb * BLOCK_K, it.n0, &full[stage]);
+                    }
+                    issued_mask |= 1u << stage;
+                    issued_parity = (issued_parity & ~(1u << stage)) | (phase << stage);
+                    if (++stage == kStages) { stage = 0; phase ^= 1u; }
+                }
+            }
+            if (!ok) {
+                // let the copies already issued land before the CTA's shared memory goes away
+                for (int s = 0; s < kStages; ++s) {
+                    if (!(issued_mask & (1u << s))) continue;
+                    const unsigned long long t0 = global_ns();
+                    while (!mbar_try_wait(&full[s], (issued_parity >> s) & 1u) && global_ns() - t0 < kWaitLimitNs) {}
+                }
+            }
+        }
+    } else if (warp == 1) {
+        // ================================ MMA issuer ===================================
+        if (lane == 0) {
+            int stage = 0; uint32_t phase = 0;
+            bool ok = true;
+            int local = 0;
+            for (int item = blockIdx.x; ok && item < P.total_items; item += gridDim.x, ++local) {
+                const Item it = decode_item(P, item);
+                const TcProblem& p = P.p[it.prob];
+                const int buf = local & 1;
+                const uint32_t use = (uint32_t)(local >> 1);
+                if (!mbar_wait(&tempty[buf], (use & 1u) ^ 1u, abort_flag, P.error, 2)) { ok = false; break; }
+                tc_fence_after();
+                const uint32_t d_tmem = tmem_base + (uint32_t)buf * kMaxBN;
+                const uint32_t idesc = instr_desc(p.bn, MODE == TC_WGRAD, MODE == TC_WGRAD);
+                for (int kb = it.kb0; kb < it.kb1; ++kb) {
+                    if (!mbar_wait(&full[stage], phase, abort_flag, P.error, 3)) { ok = false; break; }
+                    tc_fence_after();
+                    const uint32_t a_addr = smem_u32(sA + stage * kStageA);
+                    const uint32_t b_addr = smem_u32(sB + stage * kStageB);
+#pragma unroll
+                    for (int k = 0; k < BLOCK_K / UMMA_K; ++k) {
+                        uint64_t da, db;
+                        if (MODE == TC_WGRAD) {
+                            da = smem_desc(a_addr + k * (UMMA_K * 128), 8192, 1024);
+                            db = smem_desc(b_addr + k * (UMMA_K * 128), 8192, 1024);
+                        } else {
+                            da = smem_desc(a_addr + k * (UMMA_K * 2), 16, 1024);
+                            db = smem_desc(b_addr + k * (UMMA_K * 2), 16, 1024);
+                        }
+                        umma_bf16(d_tmem, da, db, idesc, (kb > it.kb0 || k > 0) ? 1u : 0u);
+                    }
+                    umma_commit(&empty[stage]);       // frees the stage once these MMAs have read it
+                    if (++stage == kStages) { stage = 0; phase ^= 1u; }
+                }
+                if (ok) umma_commit(&tfull[buf]);     // accumulator complete
+            }
+            if (!ok) {
+                umma_commit(drain);
+                const unsigned long long t0 = global_ns();
+                while (!mbar_try_wait(drain, 0) && global_ns() - t0 < kWaitLimitNs) {}
+            }
+        }
+    } else {
+        // ================================ epilogue =====================================
+        const int q = warp & 3;                    // accumulator lanes 32q .. 32q+31
+        const int half = (warp - 2) >> 2;          // which half of the tile's columns
+        bool ok = true;
+        int local = 0;
+        for (int item = blockIdx.x; ok && item < P.total_items; item += gridDim.x, ++local) {
+            const Item it = decode_item(P, item);
+            const TcProblem& p = P.p[it.prob];
+            const int buf = local & 1;
+            const uint32_t use = (uint32_t)(local >> 1);
+            if (!mbar_wait(&tfull[buf], use & 1u, abort_flag, P.error, 4)) { ok = false; break; }
+            tc_fence_after();
+            const int row = it.m0 + 32 * q + lane;
+            const int chunks = p.bn / 32;
+            const int c_begin = half * (chunks / 2), c_end = (half + 1) * (chunks / 2);
+            for (int c = c_begin; c < c_end; ++c) {
+                uint32_t acc[32];
+                tmem_ld32(tmem_base + ((uint32_t)(32 * q) << 16) + (uint32_t)(buf * kMaxBN + 32 * c), acc);
+                const int col = it.n0 + 32 * c;
+                if (row >= p.m_extent || col >= p.n_extent) continue;
+                if (MODE == TC_FWD) {
+                    uint32_t packed[16];
+#pragma unroll
+                    for (int j = 0; j < 32; j += 2) {
+                        const float b0 = (col + j < p.bias_n) ? __ldg(p.bias + col + j) : 0.f;
+                        const float b1 = (col + j + 1 < p.bias_n) ? __ldg(p.bias + col + j + 1) : 0.f;
+                        const float v0 = elu_fast(__uint_as_float(acc[j]) + b0, P.alpha);
+                        const float v1 = elu_fast(__uint_as_float(acc[j + 1]) + b1, P.alpha);
+                        __nv_bfloat162 h2 = __floats2bfloat162_rn(v0, v1);
+                        packed[j / 2] = *reinterpret_cast<uint32_t*>(&h2);
+                    }
+                    uint4* dst = reinterpret_cast<uint4*>(p.out16 + (size_t)row * p.ld_out + col);
+#pragma unroll
+                    for (int g = 0; g < 4; ++g) dst[g] = make_uint4(packed[4 * g], packed[4 * g + 1], packed[4 * g + 2], packed[4 * g + 3]);
+                } else if (MODE == TC_DGRAD) {
+                    const uint4* hsrc = reinterpret_cast<const uint4*>(p.aux16 + (size_t)row * p.ld_aux + col);
+                    uint4* dst = reinterpret_cast<uint4*>(p.out16 + (size_t)row * p.ld_out + col);
+#pragma unroll
+                    for (int g = 0; g < 4; ++g) {
+                        const uint4 hv = __ldg(hsrc + g);
+                        const uint32_t hw[4] = {hv.x, hv.y, hv.z, hv.w};
+                        uint32_t o[4];
+#pragma unroll
+                        for (int e = 0; e < 4; ++e) {
+                            const __nv_bfloat162 h2 = *reinterpret_cast<const __nv_bfloat162*>(&hw[e]);
+                            const float h0 = __low2float(h2), h1 = __high2float(h2);
+                            const float v0 = __uint_as_float(acc[8 * g + 2 * e]) * (h0 > 0.f ? 1.0f : h0 + P.alpha);
+                            const float v1 = __uint_as_float(acc[8 * g + 2 * e + 1]) * (h1 > 0.f ? 1.0f : h1 + P.alpha);
+                            __nv_bfloat162 r2 = __floats2bfloat162_rn(v0, v1);
+                            o[e] = *reinterpret_cast<uint32_t*>(&r2);
+                        }
+                        dst[g] = make_uint4(o[0], o[1], o[2], o[3]);
+                    }
+                } else {
+                    float* dst = p.out32 + (size_t)it.split * p.split_stride + (size_t)row * p.ld_out32 + col;
+#pragma unroll
+                    for (int g = 0; g < 8; ++g)
+                        if (col + 4 * g < p.n_extent)
+                            *reinterpret_cast<float4*>(dst + 4 * g) =
+                                make_float4(__uint_as_float(acc[4 * g]), __uint_as_float(acc[4 * g + 1]),
+                                            __uint_as_float(acc[4 * g + 2]), __uint_as_float(acc[4 * g + 3]));
+                }
+            }
+            tc_fence_before();
+            __syncwarp();
+            if (lane == 0) mbar_arrive(&tempty[buf]);
+        }
+    }
+    tc_fence_before();
+    __syncthreads();
+    if (warp == 1) {
+        tc_fence_after();
+        tmem_dealloc(tmem_base, kTmemCols);
+    }
+}
+
+// ------------------------------------------------------------------------- small kernels
+struct CvtEntry {
+    const float* src; int in, out, ld_src;      // FP32 master W[in][ld_src]
+    __nv_bfloat16* wt; int ld_wt;               // [out][ld_wt]  (contraction = in)   forward operand
+    __nv_bfloat16* wn; int ld_wn;               // [in][ld_wn]   (contraction = out)  data-gradient operand, may be null
+};
+
+__global__ void convert_weights_kernel(const CvtEntry* __restrict__ table) {
+    const CvtEntry e = table[blockIdx.y];
+    const int total = e.in * e.out;
+    for (int idx = blockIdx.x * blockDim.x + threadIdx.x; idx < total; idx += gridDim.x * blockDim.x) {
+        const int i = idx / e.out, o = idx - i * e.out;
+        const __nv_bfloat16 v = __float2bfloat16_rn(e.src[(size_t)i * e.ld_src + o]);
+        e.wt[(size_t)o * e.ld_wt + i] = v;
+        if (e.wn) e.wn[(size_t)i * e.ld_wn + o] = v;
+    }
+}
+
+// ------------------------------------------------------------------------------- host side
+typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
+                                  const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
+                                  CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+EncodeTiledFn get_encode_fn() {
+    static EncodeTiledFn fn = nullptr;
+    if (fn) return fn;
+    void* p = nullptr;
+    cudaDriverEntryPointQueryResult qres;
+    if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &p, cudaEnableDefault, &qres) != cudaSuccess ||
+        qres != cudaDriverEntryPointSuccess)
+        return nullptr;
+    fn = reinterpret_cast<EncodeTiledFn>(p);
+    return fn;
+}
+
+// 2-D BF16 tensor [rows][cols] with row stride ld (elements); box = box_cols x box_rows, 128-byte swizzle.
+bool make_tmap(CUtensorMap* tm, const void* base, int rows, int cols, int ld, int box_cols, int box_rows) {
+    EncodeTiledFn fn = get_encode_fn();
+    if (!fn) return false;
+    const cuuint64_t dims[2] = {(cuuint64_t)cols, (cuuint64_t)rows};
+    const cuuint64_t strides[1] = {(cuuint64_t)ld * 2};
+    const cuuint32_t box[2] = {(cuuint32_t)box_cols, (cuuint32_t)box_rows};
+    const cuuint32_t estr[2] = {1, 1};
+    return fn(tm, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(base), dims, strides, box, estr,
+              CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+              CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
+inline int round_up(int x, int m) { return (x + m - 1) / m * m; }
+inline int pick_bn(int width) { return std::min(kMaxBN, width); }   // widths are multiples of 64
+
+}  // namespace
+
+struct UmmaEngine {
+    UmmaSetup s;
+    int nh[2];                                   // hidden layers per net
+    int kp[2];                                   // padded observation width
+    int pw[2][kMaxLayers];                       // padded hidden widths
+    std::vector<void*> allocs;
+    __nv_bfloat16 *obs16_act[2] = {}, *h_act[2][kMaxLayers] = {};
+    __nv_bfloat16 *x16[2] = {}, *h[2][kMaxLayers] = {}, *dz[2][kMaxLayers] = {};
+    __nv_bfloat16 *dmu16 = nullptr, *dv16 = nullptr;
+    __nv_bfloat16 *wt[2][kMaxLayers] = {}, *wn[2][kMaxLayers] = {};
+    CvtEntry* cvt_dev = nullptr; int n_cvt = 0; int cvt_max = 0;
+    int* error_dev = nullptr;
+    int num_sms = 148;
+    std::vector<TcParams> act_fwd, act_fwd_critic, upd_fwd, upd_dgrad, upd_wgrad;
+    ColsumBatch colsum{};
+};
+
+namespace {
+
+template <typename T>
+bool ealloc(UmmaEngine* e, T** p, size_t count) {
+    void* q = nullptr;
+    const size_t bytes = std::max<size_t>(count, 1) * sizeof(T);
+    if (cudaMalloc(&q, bytes) != cudaSuccess) return false;
+    e->allocs.push_back(q);
+    if (cudaMemsetAsync(q, 0, bytes, e->s.stream) != cudaSuccess) return false;
+    *p = reinterpret_cast<T*>(q);
+    return true;
+}
+
+void finish_params(TcParams& P, float alpha, int* error) {
+    int items = 0;
+    for (int i = 0; i < P.count; ++i) {
+        P.p[i].item_begin = items;
+        items += P.p[i].m_tiles * P.p[i].n_tiles * P.p[i].splits;
+    }
+    P.total_items = items;
+    P.alpha = alpha;
+    P.error = error;
+}
+
+// D[rows x width_out] = A[rows x k] * B[width_out x k]^T, both operands contraction-major.
+bool add_rowmajor_problem(TcParams& P, const __nv_bfloat16* A, int rows, int k, const __nv_bfloat16* B, int width_out) {
+    const int i = P.count;
+    TcProblem& p = P.p[i];
+    memset(&p, 0, sizeof p);
+    p.bn = pick_bn(width_out);
+    p.m_extent = rows; p.n_extent = width_out;
+    p.m_tiles = (rows + BLOCK_M - 1) / BLOCK_M;
+    p.n_tiles = (width_out + p.bn - 1) / p.bn;
+    p.kblocks = k / BLOCK_K; p.splits = 1; p.kb_per_split = p.kblocks;
+    if (!make_tmap(&P.tmA[i], A, rows, k, k, BLOCK_K, BLOCK_M)) return false;
+    if (!make_tmap(&P.tmB[i], B, width_out, k, k, BLOCK_K, p.bn)) return false;
+    P.count++;
+    return true;
+}
+
+template <int MODE>
+cudaError_t launch_tc(const TcParams& P, int num_sms, cudaStream_t s) {
+    if (P.total_items == 0) return cudaSuccess;
+    const int grid = std::min(P.total_items, num_sms);
+    tc_gemm_kernel<MODE><<<grid, kThreads, kSmemBytes, s>>>(P);
+    count_launch();
+    return cudaGetLastError();
+}
+
+}  // namespace
+
+int umma_wgrad_tiles(const UmmaSetup& s) {
+    int tiles = 0;
+    for (int ni = 0; ni < 2; ++ni) {
+        const int nh = s.nl[ni] - 1;
+        for (int l = 0; l <= nh; ++l) {
+            const int wa = round_up(l == 0 ? s.in_dim[ni] : s.out[ni][l - 1], 64);
+            const int wb = l == nh ? 64 : round_up(s.out[ni][l], 64);
+            tiles += ((wa + BLOCK_M - 1) / BLOCK_M) * ((wb + pick_bn(wb) - 1) / pick_bn(wb));
+        }
+    }
+    return tiles;
+}
+
+UmmaEngine* umma_create(const UmmaSetup& s, std::string* err) {
+    auto failmsg = [&](const char* m) { if (err) *err = m; return (UmmaEngine*)nullptr; };
+    if (s.model.precision != RSLRL_BF16) return failmsg("only the BF16 tensor-core mode is available");
+    if (!get_encode_fn()) return failmsg("cuTensorMapEncodeTiled is not available from the driver");
+    int dev = 0; cudaDeviceProp prop;
+    if (cudaGetDevice(&dev) != cudaSuccess || cudaGetDeviceProperties(&prop, dev) != cudaSuccess) return failmsg("no CUDA device");
+    if (prop.major != 10) return failmsg("the tensor-core mode needs an sm_100 device");
+    if (cudaFuncSetAttribute(tc_gemm_kernel<TC_FWD>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kSmemBytes) != cudaSuccess ||
+        cudaFuncSetAttribute(tc_gemm_kernel<TC_DGRAD>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kSmemBytes) != cudaSuccess ||
+        cudaFuncSetAttribute(tc_gemm_kernel<TC_WGRAD>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kSmemBytes) != cudaSuccess)
+        return failmsg("could not reserve shared memory for the tensor-core kernels");
+    UmmaEngine* e = new UmmaEngine();
+    e->s = s;
+    e->num_sms = prop.multiProcessorCount;
+    auto bail = [&](const char* m) { if (err) *err = m; umma_destroy(e); return (UmmaEngine*)nullptr; };
+    const int N = s.N, R = s.R;
+    if (!ealloc(e, &e->error_dev, 1)) return bail("allocation failed");
+    for (int ni = 0; ni < 2; ++ni) {
+        e->nh[ni] = s.nl[ni] - 1;
+        e->kp[ni] = round_up(s.in_dim[ni], 64);
+        for (int l = 0; l < e->nh[ni]; ++l) e->pw[ni][l] = round_up(s.out[ni][l], 64);
+    }
+    const bool shared = s.model.shared_obs != 0;
+    for (int ni = 0; ni < 2; ++ni) {
+        if (ni == 1 && shared) { e->obs16_act[1] = e->obs16_act[0]; e->x16[1] = e->x16[0]; }
+        else {
+            if (!ealloc(e, &e->obs16_act[ni], (size_t)N * e->kp[ni])) return bail("allocation failed");
+            if (!ealloc(e, &e->x16[ni], (size_t)R * e->kp[ni])) return bail("allocation failed");
+        }
+        for (int l = 0; l < e->nh[ni]; ++l) {
+            const int kin = l == 0 ? e->kp[ni] : e->pw[ni][l - 1];
+            if (!ealloc(e, &e->h_act[ni][l], (size_t)N * e->pw[ni][l]) || !ealloc(e, &e->h[ni][l], (size_t)R * e->pw[ni][l]) ||
+                !ealloc(e, &e->dz[ni][l], (size_t)R * e->pw[ni][l]) || !ealloc(e, &e->wt[ni][l], (size_t)e->pw[ni][l] * kin))
+                return bail("allocation failed");
+            if (l > 0 && !ealloc(e, &e->wn[ni][l], (size_t)e->pw[ni][l - 1] * e->pw[ni][l])) return bail("allocation failed");
+        }
+    }
+    if (!ealloc(e, &e->dmu16, (size_t)R * 64) || !ealloc(e, &e->dv16, (size_t)R * 64)) return bail("allocation failed");
+
+    // weight conversion table
+    std::vector<CvtEntry> table;
+    for (int ni = 0; ni < 2; ++ni)
+        for (int l = 0; l < e->nh[ni]; ++l) {
+            CvtEntry c{};
+            c.src = s.param + s.w_off[ni][l]; c.in = s.in[ni][l]; c.out = s.out[ni][l]; c.ld_src = s.out_p[ni][l];
+            c.wt = e->wt[ni][l]; c.ld_wt = l == 0 ? e->kp[ni] : e->pw[ni][l - 1];
+            c.wn = l > 0 ? e->wn[ni][l] : nullptr; c.ld_wn = e->pw[ni][l];
+            table.push_back(c);
+            e->cvt_max = std::max(e->cvt_max, c.in * c.out);
+        }
+    e->n_cvt = (int)table.size();
+    if (!ealloc(e, &e->cvt_dev, table.size())) return bail("allocation failed");
+    if (cudaMemcpyAsync(e->cvt_dev, table.data(), table.size() * sizeof(CvtEntry), cudaMemcpyHostToDevice, s.stream) != cudaSuccess ||
+        cudaStreamSynchronize(s.stream) != cudaSuccess)
+        return bail("copy of the conversion table failed");
+
+    const float alpha = s.model.elu_alpha;
+    const int maxh = std::max(e->nh[0], e->nh[1]);
+    // ---- forward launches (act rows and update rows), one per hidden layer index -----------
+    auto build_fwd = [&](std::vector<TcParams>& out, int rows, bool actor, bool critic, bool act_buffers) -> bool {
+        for (int l = 0; l < maxh; ++l) {
+            TcParams P; memset(&P, 0, sizeof P);
+            for (int ni = 0; ni < 2; ++ni) {
+                if ((ni == 0 && !actor) || (ni == 1 && !critic) || l >= e->nh[ni]) continue;
+                const __nv_bfloat16* in = l == 0 ? (act_buffers ? e->obs16_act[ni] : e->x16[ni])
+                                                 : (act_buffers ? e->h_act[ni][l - 1] : e->h[ni][l - 1]);
+                const int k = l == 0 ? e->kp[ni] : e->pw[ni][l - 1];
+                if (!add_rowmajor_problem(P, in, rows, k, e->wt[ni][l], e->pw[ni][l])) return false;
+                TcProblem& p = P.p[P.count - 1];
+                p.bias = s.param + s.b_off[ni][l]; p.bias_n = s.out[ni][l];
+                p.out16 = act_buffers ? e->h_act[ni][l] : e->h[ni][l]; p.ld_out = e->pw[ni][l];
+            }
+            finish_params(P, alpha, e->error_dev);
+            out.push_back(P);
+        }
+        return true;
+    };
+    if (!build_fwd(e->act_fwd, N, true, true, true) || !build_fwd(e->act_fwd_critic, N, false, true, true) ||
+        !build_fwd(e->upd_fwd, R, true, true, false))
+        return bail("tensor map encoding failed");
+    // ---- data-gradient launches: step b produces dZ of hidden layer nh-2-b -------------------
+    for (int b = 0; b + 1 < maxh; ++b) {
+        TcParams P; memset(&P, 0, sizeof P);
+        for (int ni = 0; ni < 2; ++ni) {
+            const int l = e->nh[ni] - 1 - b;
+            if (l < 1) continue;
+            if (!add_rowmajor_problem(P, e->dz[ni][l], R, e->pw[ni][l], e->wn[ni][l], e->pw[ni][l - 1]))
+                return bail("tensor map encoding failed");
+            TcProblem& p = P.p[P.count - 1];
+            p.out16 = e->dz[ni][l - 1]; p.ld_out = e->pw[ni][l - 1];
+            p.aux16 = e->h[ni][l - 1]; p.ld_aux = e->pw[ni][l - 1];
+        }
+        finish_params(P, alpha, e->error_dev);
+        e->upd_dgrad.push_back(P);
+    }
+    // ---- weight-gradient problems (all layers of both nets, heads included) ------------------
+    {
+        const int kblocks = (R + BLOCK_K - 1) / BLOCK_K;
+        const int kb_per_split = (kblocks + s.splits - 1) / s.splits;
+        const int splits_eff = (kblocks + kb_per_split - 1) / kb_per_split;
+        TcParams P; memset(&P, 0, sizeof P);
+        auto flush = [&]() { if (P.count) { finish_params(P, alpha, e->error_dev); e->upd_wgrad.push_back(P); memset(&P, 0, sizeof P); } };
+        for (int ni = 0; ni < 2; ++ni)
+            for (int l = 0; l <= e->nh[ni]; ++l) {
+                const bool head = l == e->nh[ni];
+                const __nv_bfloat16* A = l == 0 ? e->x16[ni] : e->h[ni][l - 1];
+                const int wa = l == 0 ? e->kp[ni] : e->pw[ni][l - 1];
+                const __nv_bfloat16* B = head ? (ni == 0 ? e->dmu16 : e->dv16) : e->dz[ni][l];
+                const int wb = head ? 64 : e->pw[ni][l];
+                if (P.count == kMaxProblems) flush();
+                const int i = P.count;
+                TcProblem& p = P.p[i];
+                p.bn = pick_bn(wb);
+                p.m_extent = s.in[ni][l]; p.n_extent = s.out_p[ni][l];
+                p.m_tiles = (wa + BLOCK_M - 1) / BLOCK_M; p.n_tiles = (wb + p.bn - 1) / p.bn;
+                p.kblocks = kblocks; p.splits = splits_eff; p.kb_per_split = kb_per_split;
+                p.out32 = s.partials + s.w_off[ni][l]; p.ld_out32 = s.out_p[ni][l]; p.split_stride = s.P_dev;
+                if (!make_tmap(&P.tmA[i], A, R, wa, wa, 64, BLOCK_K) || !make_tmap(&P.tmB[i], B, R, wb, wb, 64, BLOCK_K))
+                    return bail("tensor map encoding failed");
+                P.count++;
+            }
+        flush();
+    }
+    // ---- bias gradients of the hidden layers: column sums of dZ -------------------------------
+    e->colsum.count = 0; e->colsum.splits = s.splits; e->colsum.split_stride = s.P_dev; e->colsum.is_bf16 = 1;
+    for (int ni = 0; ni < 2; ++ni)
+        for (int l = 0; l < e->nh[ni]; ++l) {
+            if (e->colsum.count == kMaxColsum) return bail("too many layers for the bias-gradient launch");
+            ColsumProblem& q = e->colsum.p[e->colsum.count++];
+            q.X = e->dz[ni][l]; q.out = s.partials + s.b_off[ni][l]; q.rows = R; q.n = s.out[ni][l]; q.ld = e->pw[ni][l];
+        }
+    if (cudaStreamSynchronize(s.stream) != cudaSuccess) return bail("stream synchronisation failed");
+    return e;
+}
+
+void umma_destroy(UmmaEngine* e) {
+    if (!e) return;
+    for (void* p : e->allocs) cudaFree(p);
+    delete e;
+}
+
+cudaError_t umma_refresh_weights(UmmaEngine* e) {
+    dim3 grid(std::max(1, std::min(64, (e->cvt_max + 255) / 256)), e->n_cvt);
+    convert_weights_kernel<<<grid, 256, 0, e->s.stream>>>(e->cvt_dev);
+    count_launch();
+    return cudaGetLastError();
+}
+
+cudaError_t umma_act_forward(UmmaEngine* e, const float* d_obs_a, const float* d_obs_c, float* store_a, float* store_c,
+                             int sa, int sc, bool do_actor, const void** ha, int* ldha, const void** hc, int* ldhc) {
+    const UmmaSetup& s = e->s;
+    cudaError_t err;
+    const bool shared = s.model.shared_obs != 0;
+    if (do_actor) {
+        err = launch_pad_rows(d_obs_a, s.in_dim[0], store_a, sa, e->obs16_act[0], e->kp[0], s.N, s.stream);
+        if (err != cudaSuccess) return err;
+        if (!shared) {
+            err = launch_pad_rows(d_obs_c, s.in_dim[1], store_c, sc, e->obs16_act[1], e->kp[1], s.N, s.stream);
+            if (err != cudaSuccess) return err;
+        }
+    } else {
+        err = launch_pad_rows(d_obs_c, s.in_dim[1], nullptr, 0, e->obs16_act[1], e->kp[1], s.N, s.stream);
+        if (err != cudaSuccess) return err;
+    }
+    const std::vector<TcParams>& seq = do_actor ? e->act_fwd : e->act_fwd_critic;
+    for (const TcParams& P : seq) {
+        err = launch_tc<TC_FWD>(P, e->num_sms, s.stream);
+        if (err != cudaSuccess) return err;
+    }
+    *ha = e->h_act[0][e->nh[0] - 1]; *ldha = e->pw[0][e->nh[0] - 1];
+    *hc = e->h_act[1][e->nh[1] - 1]; *ldhc = e->pw[1][e->nh[1] - 1];
+    return cudaSuccess;
+}
+
+void umma_gather_targets(UmmaEngine* e, GatherArgs* g) {
+    g->x_a = nullptr; g->x_c = nullptr;
+    g->x_a16 = e->x16[0]; g->ldxa16 = e->kp[0];
+    g->x_c16 = e->x16[1]; g->ldxc16 = e->kp[1];
+}
+
+cudaError_t umma_update_forward(UmmaEngine* e) {
+    for (const TcParams& P : e->upd_fwd) {
+        cudaError_t err = launch_tc<TC_FWD>(P, e->num_sms, e->s.stream);
+        if (err != cudaSuccess) return err;
+    }
+    return cudaSuccess;
+}
+
+void umma_head_loss_targets(UmmaEngine* e, HeadLossArgs* a) {
+    a->Ha = e->h[0][e->nh[0] - 1]; a->ldha = e->pw[0][e->nh[0] - 1];
+    a->Hc = e->h[1][e->nh[1] - 1]; a->ldhc = e->pw[1][e->nh[1] - 1];
+    a->bf16_act = 1;
+    a->dZa = e->dz[0][e->nh[0] - 1]; a->lddza = a->ldha;
+    a->dZc = e->dz[1][e->nh[1] - 1]; a->lddzc = a->ldhc;
+    a->dmu16 = e->dmu16; a->lddmu16 = 64; a->dv16 = e->dv16; a->lddv16 = 64;
+}
+
+cudaError_t umma_update_backward(UmmaEngine* e) {
+    cudaError_t err;
+    for (const TcParams& P : e->upd_dgrad) {
+        err = launch_tc<TC_DGRAD>(P, e->num_sms, e->s.stream);
+        if (err != cudaSuccess) return err;
+    }
+    for (const TcParams& P : e->upd_wgrad) {
+        err = launch_tc<TC_WGRAD>(P, e->num_sms, e->s.stream);
+        if (err != cudaSuccess) return err;
+    }
+    return launch_colsum(e->colsum, e->s.stream);
+}
+
+cudaError_t umma_read_error(UmmaEngine* e, int* host_code) {
+    cudaError_t err = cudaMemcpyAsync(host_code, e->error_dev, sizeof(int), cudaMemcpyDeviceToHost, e->s.stream);
+    if (err != cudaSuccess) return err;
+    return cudaStreamSynchronize(e->s.stream);
+}
+
+}  // namespace rslrl

@@ -1,0 +1,48 @@
+// Tensor-core engine (RSLRL_BF16): hidden-layer products of act, forward and backward on
+// tcgen05 tiles fed by TMA, with FP32 accumulation in tensor memory.
+#pragma once
+#include "../../include/rslrl_b200.h"
+#include "common.cuh"
+#include "kernels.h"
+#include <string>
+
+namespace rslrl {
+
+struct UmmaSetup {
+    rslrl_model_cfg model;
+    int N, Bmb, R;                 // rollout rows per act call, minibatch rows, rows incl. mirrored
+    cudaStream_t stream;
+    float* param; int P_dev;       // FP32 master parameters (padded device layout)
+    float* partials; int splits;   // weight-gradient partials [splits][P_dev]
+    int nl[2], in_dim[2];          // layers per net (head included), observation widths
+    int in[2][kMaxLayers], out[2][kMaxLayers], out_p[2][kMaxLayers];
+    size_t w_off[2][kMaxLayers], b_off[2][kMaxLayers];
+};
+
+struct UmmaEngine;
+
+UmmaEngine* umma_create(const UmmaSetup& s, std::string* err);
+void umma_destroy(UmmaEngine* e);
+// Number of 128-row x <=256-column output tiles of all weight gradients (for choosing splits).
+int umma_wgrad_tiles(const UmmaSetup& s);
+// Re-derive the low-precision operand copies of the weights from the FP32 masters.
+cudaError_t umma_refresh_weights(UmmaEngine* e);
+// Hidden layers on N rollout rows.  d_obs_* are dense [N][dim] FP32 rows; when store_* is not
+// null the padded FP32 copy of the observations is also written there (row strides sa / sc).
+// Returns the last hidden activations of both nets (actor's only when do_actor).
+cudaError_t umma_act_forward(UmmaEngine* e, const float* d_obs_a, const float* d_obs_c, float* store_a,
+                             float* store_c, int sa, int sc, bool do_actor, const void** ha, int* ldha,
+                             const void** hc, int* ldhc);
+// Point the gather at the engine's minibatch input buffers.
+void umma_gather_targets(UmmaEngine* e, GatherArgs* g);
+cudaError_t umma_update_forward(UmmaEngine* e);
+// Point the head/loss kernel at the engine's last hidden activations and dZ buffers.
+void umma_head_loss_targets(UmmaEngine* e, HeadLossArgs* a);
+// Data gradients, weight-gradient partials and bias-gradient partials of all hidden layers
+// and heads, from the dZ / d_head buffers the head/loss kernel filled.
+cudaError_t umma_update_backward(UmmaEngine* e);
+// Synchronises the stream and returns the device error code (0 = none; otherwise the role
+// whose bounded wait expired).
+cudaError_t umma_read_error(UmmaEngine* e, int* host_code);
+
+}  // namespace rslrl
