@@ -1,0 +1,58 @@
+"""The C-ABI library loads and exports every symbol the public header declares (no GPU needed)."""
+import ctypes
+import os
+import re
+
+ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+
+
+def declared_functions():
+    text = open(os.path.join(ROOT, "include", "rslrl_b200.h")).read()
+    text = re.sub(r"/\*.*?\*/", "", text, flags=re.S)
+    return sorted(set(re.findall(r"\b(rslrl_[a-z_0-9]+)\s*\(", text)))
+
+
+def test_header_declares_the_path():
+    names = declared_functions()
+    for must in ("rslrl_create", "rslrl_destroy", "rslrl_act", "rslrl_record_step", "rslrl_gae", "rslrl_ppo_update"):
+        assert must in names
+
+
+def test_library_exports_every_declared_symbol():
+    from paper_2509_10771_b200 import binding, build
+    build.build()
+    lib = ctypes.CDLL(binding.LIB_PATH)
+    for name in declared_functions():
+        assert hasattr(lib, name), f"{name} is declared in include/rslrl_b200.h but not exported"
+    assert sorted(binding.EXPORTS) == declared_functions()
+
+
+def test_binding_structs_match_header_sizes():
+    from paper_2509_10771_b200 import binding
+    assert ctypes.sizeof(binding.ModelCfg) == 4 * (6 + 1 + 8 + 1 + 8 + 1 + 1)
+    assert ctypes.sizeof(binding.Counters) == 16
+    assert ctypes.sizeof(binding.UpdateStats) == 4 * 14
+    assert ctypes.sizeof(binding.Storage) == 4 * 6 + 8 * 12
+    assert binding.PpoCfg.seed.offset % 8 == 0
+
+
+def test_num_params_and_config_validation_without_a_device():
+    from paper_2509_10771_b200 import binding, build, workloads as WL
+    build.build()
+    lib = binding.load_library()
+    for w in WL.CONFIGS:
+        mc = binding.model_cfg(w)
+        assert lib.rslrl_num_params(ctypes.byref(mc)) == w.num_params()
+    bad = binding.model_cfg(WL.TINY)
+    bad.num_actions = 0
+    assert lib.rslrl_num_params(ctypes.byref(bad)) == 0
+    # argument errors are reported before any CUDA call
+    handle = ctypes.c_void_p()
+    pc = binding.ppo_cfg(WL.TINY)
+    assert lib.rslrl_create(ctypes.byref(bad), ctypes.byref(pc), None, ctypes.byref(handle)) == 1
+    assert b"num_actions" in lib.rslrl_last_error(None)
+    pc.minibatches = 7
+    assert lib.rslrl_create(ctypes.byref(binding.model_cfg(WL.TINY)), ctypes.byref(pc), None, ctypes.byref(handle)) == 2
+    assert lib.rslrl_gae_scan(None, None, None, None, None, None, None, 0, 0, 0.99, 0.95, 1, 1, 1e-8, None, None) == 0
+    assert lib.rslrl_gae_scan(None, None, None, None, None, None, None, 4, 4, 0.99, 0.95, 1, 1, 1e-8, None, None) == 1
+    assert lib.rslrl_minibatch_indices(0, 0, 0, 10, 3, 0, None, None) == 2
