@@ -236,6 +236,14 @@ rslrl_status rslrl_minibatch_indices(uint64_t seed, uint32_t iteration, uint32_t
 /* Number of kernels this library has launched in the current process (all contexts). */
 uint64_t     rslrl_kernel_launch_count(void);
 
+/* Per-kernel timing for roofline reports.  While enabled, every kernel launch of the library
+ * is bracketed by a pair of CUDA events on its stream (this slows the host side down; leave
+ * it off when measuring throughput).  rslrl_profile_report waits for the recorded launches,
+ * writes one line "family launches total_ms" per kernel family into h_text (NUL-terminated,
+ * RSLRL_ERR_UNSUPPORTED if capacity is too small) and forgets them. */
+rslrl_status rslrl_profile_enable(int32_t on);
+rslrl_status rslrl_profile_report(char *h_text, size_t capacity);
+
 #ifdef __cplusplus
 }
 #endif

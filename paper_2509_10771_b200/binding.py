@@ -81,7 +81,7 @@ EXPORTS = [
     "rslrl_get_counters", "rslrl_set_counters", "rslrl_act", "rslrl_record_step", "rslrl_gae",
     "rslrl_ppo_update", "rslrl_ppo_update_steps", "rslrl_act_host", "rslrl_record_step_host",
     "rslrl_gae_host", "rslrl_gae_scratch_bytes", "rslrl_gae_scan", "rslrl_minibatch_indices",
-    "rslrl_kernel_launch_count",
+    "rslrl_kernel_launch_count", "rslrl_profile_enable", "rslrl_profile_report",
 ]
 
 _lib = None
@@ -122,6 +122,8 @@ def load_library() -> C.CDLL:
         "rslrl_gae_scan": (i32, [vp, vp, vp, vp, vp, vp, vp, i32, i32, f32, f32, i32, i32, f32, vp, vp]),
         "rslrl_minibatch_indices": (i32, [u64, u32, u32, i32, i32, i32, vp, vp]),
         "rslrl_kernel_launch_count": (u64, []),
+        "rslrl_profile_enable": (i32, [i32]),
+        "rslrl_profile_report": (i32, [C.c_char_p, sz]),
     }
     for name, (res, args) in sig.items():
         fn = getattr(lib, name)
@@ -306,3 +308,20 @@ def minibatch_indices(seed: int, iteration: int, epoch: int, batch: int, minibat
 
 def kernel_launch_count() -> int:
     return int(load_library().rslrl_kernel_launch_count())
+
+
+def profile_enable(on: bool):
+    load_library().rslrl_profile_enable(int(on))
+
+
+def profile_report() -> Dict[str, Dict[str, float]]:
+    """{kernel family: {"launches": n, "ms": total}} of the launches recorded since the last report."""
+    buf = C.create_string_buffer(1 << 16)
+    st = load_library().rslrl_profile_report(buf, len(buf))
+    if st != 0:
+        raise RslrlError(st, "rslrl_profile_report")
+    out = {}
+    for line in buf.value.decode().splitlines():
+        name, n, ms = line.split()
+        out[name] = {"launches": int(n), "ms": float(ms)}
+    return out

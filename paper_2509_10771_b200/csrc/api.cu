@@ -14,11 +14,6 @@
 #include <string>
 #include <vector>
 
-namespace rslrl {
-static std::atomic<uint64_t> g_launches{0};
-void count_launch(int n) { g_launches.fetch_add((uint64_t)n, std::memory_order_relaxed); }
-}  // namespace rslrl
-
 using namespace rslrl;
 
 namespace {
@@ -317,8 +312,6 @@ size_t rslrl_num_params(const rslrl_model_cfg* m) {
 }
 
 const char* rslrl_last_error(const rslrl_ctx* c) { return c ? c->err.c_str() : g_create_error.c_str(); }
-
-uint64_t rslrl_kernel_launch_count(void) { return g_launches.load(); }
 
 rslrl_status rslrl_destroy(rslrl_ctx* c) {
     if (!c) return RSLRL_ERR_INVALID_ARG;

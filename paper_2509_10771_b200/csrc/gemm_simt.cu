@@ -203,16 +203,16 @@ cudaError_t launch_tiles(const GemmBatch& b, bool ta, bool tb, int epi, cudaStre
         sp = std::max(sp, b.p[i].splits);
     }
     dim3 grid(nt, mt, sp * b.count);
-#define RSLRL_SGEMM_CASE(TA_, TB_, EPI_)                                                  \
+#define RSLRL_SGEMM_CASE(TA_, TB_, EPI_, NAME_)                                                \
     if (ta == TA_ && tb == TB_ && epi == EPI_) {                                          \
+        LaunchScope scope_(NAME_, s);                                                     \
         sgemm_kernel<BM, BN, TA_, TB_, EPI_><<<grid, NT, 0, s>>>(b);                      \
-        count_launch();                                                                   \
         return cudaGetLastError();                                                        \
     }
-    RSLRL_SGEMM_CASE(false, false, EPI_BIAS_ELU)
-    RSLRL_SGEMM_CASE(false, false, EPI_BIAS)
-    RSLRL_SGEMM_CASE(false, true, EPI_DELU)
-    RSLRL_SGEMM_CASE(true, false, EPI_PLAIN)
+    RSLRL_SGEMM_CASE(false, false, EPI_BIAS_ELU, "sgemm_fwd")
+    RSLRL_SGEMM_CASE(false, false, EPI_BIAS, "sgemm_fwd_linear")
+    RSLRL_SGEMM_CASE(false, true, EPI_DELU, "sgemm_dgrad")
+    RSLRL_SGEMM_CASE(true, false, EPI_PLAIN, "sgemm_wgrad")
 #undef RSLRL_SGEMM_CASE
     return cudaErrorInvalidValue;
 }
@@ -258,9 +258,9 @@ cudaError_t launch_colsum(const ColsumBatch& b, cudaStream_t s) {
     int nmax = 0;
     for (int i = 0; i < b.count; ++i) nmax = std::max(nmax, b.p[i].n);
     dim3 grid((nmax + 127) / 128, b.splits, b.count);
+    LaunchScope scope_("colsum", s);
     if (b.is_bf16) colsum_kernel<__nv_bfloat16><<<grid, 128, 0, s>>>(b);
     else colsum_kernel<float><<<grid, 128, 0, s>>>(b);
-    count_launch();
     return cudaGetLastError();
 }
 

@@ -8,7 +8,13 @@
 
 namespace rslrl {
 
-void count_launch(int n = 1);
+// Counts one kernel launch; while profiling is on it also brackets the launch with CUDA events
+// on `stream` so that the time of every kernel family can be reported.
+struct LaunchScope {
+    LaunchScope(const char* name, cudaStream_t stream);
+    ~LaunchScope();
+    const char* name; cudaStream_t stream; int slot;
+};
 
 // ------------------------------------------------------------------------- SIMT FP32 GEMM
 // C[M x N] = op(A)[M x K] * op(B)[K x N] followed by an epilogue.  Leading dimensions are

@@ -265,8 +265,8 @@ cudaError_t launch_pad_rows(const float* src, int dim, float* dst, int dst_ld, _
     const int ld = std::max(dst ? dst_ld : 0, dst16 ? dst16_ld : 0);
     const long long total = (long long)rows * ld;
     const int blocks = (int)std::min((total + 255) / 256, (long long)(148 * 16));
+    LaunchScope scope_("pad_rows", s);
     pad_rows_kernel<<<blocks, 256, 0, s>>>(src, dim, dst, dst_ld, dst16, dst16_ld, rows);
-    count_launch();
     return cudaGetLastError();
 }
 
@@ -275,32 +275,32 @@ cudaError_t launch_act_head(const void* Ha, int ldha, const void* Hc, int ldhc, 
                             uint32_t global_step, cudaStream_t s) {
     const int blocks = (N * 32 + 255) / 256;
     const uint32_t lo = (uint32_t)seed, hi = (uint32_t)(seed >> 32);
+    LaunchScope scope_("act_head", s);
     if (bf16_act)
         act_head_kernel<__nv_bfloat16><<<blocks, 256, 0, s>>>(
             (const __nv_bfloat16*)Ha, ldha, (const __nv_bfloat16*)Hc, ldhc, hp, out, N, lo, hi, global_step);
     else
         act_head_kernel<float><<<blocks, 256, 0, s>>>((const float*)Ha, ldha, (const float*)Hc, ldhc,
                                                       hp, out, N, lo, hi, global_step);
-    count_launch();
     return cudaGetLastError();
 }
 
 cudaError_t launch_value_head(const void* Hc, int ldhc, bool bf16_act, const HeadParams& hp,
                               float* values, int N, cudaStream_t s) {
     const int blocks = (N * 32 + 255) / 256;
+    LaunchScope scope_("value_head", s);
     if (bf16_act)
         value_head_kernel<__nv_bfloat16><<<blocks, 256, 0, s>>>((const __nv_bfloat16*)Hc, ldhc, hp, values, N);
     else
         value_head_kernel<float><<<blocks, 256, 0, s>>>((const float*)Hc, ldhc, hp, values, N);
-    count_launch();
     return cudaGetLastError();
 }
 
 cudaError_t launch_record_step(const float* rew, const uint8_t* dones, const uint8_t* timeouts,
                                float* s_rew, uint8_t* s_dones, uint8_t* s_timeouts, int N,
                                cudaStream_t s) {
+    LaunchScope scope_("record_step", s);
     record_step_kernel<<<(N + 255) / 256, 256, 0, s>>>(rew, dones, timeouts, s_rew, s_dones, s_timeouts, N);
-    count_launch();
     return cudaGetLastError();
 }
 
@@ -312,15 +312,18 @@ cudaError_t launch_gae(const float* rewards, const float* values, const uint8_t*
                        int unbiased, float adv_eps, float* scratch, cudaStream_t s) {
     if (T <= 0 || N <= 0) return cudaSuccess;
     const int blocks = gae_scan_blocks(N);
-    gae_scan_kernel<<<blocks, kGaeThreads, 0, s>>>(rewards, values, dones, timeouts, last_values,
-                                                   returns, advantages, T, N, gamma, lam, scratch);
-    count_launch();
-    cudaError_t e = cudaGetLastError();
+    cudaError_t e;
+    {
+        LaunchScope scope_("gae_scan", s);
+        gae_scan_kernel<<<blocks, kGaeThreads, 0, s>>>(rewards, values, dones, timeouts, last_values,
+                                                       returns, advantages, T, N, gamma, lam, scratch);
+        e = cudaGetLastError();
+    }
     if (e != cudaSuccess || !normalize) return e;
     const long long total = (long long)T * N;
     const int nb = (int)std::min((total / 4 + 255) / 256 + 1, (long long)(148 * 8));
+    LaunchScope scope_("gae_normalize", s);
     gae_normalize_kernel<<<nb, 256, 0, s>>>(advantages, total, scratch, blocks, unbiased, adv_eps);
-    count_launch();
     return cudaGetLastError();
 }
 

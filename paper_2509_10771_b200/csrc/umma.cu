@@ -491,8 +491,8 @@ template <int MODE>
 cudaError_t launch_tc(const TcParams& P, int num_sms, cudaStream_t s) {
     if (P.total_items == 0) return cudaSuccess;
     const int grid = std::min(P.total_items, num_sms);
+    LaunchScope scope_(MODE == TC_FWD ? "tc_gemm_fwd" : MODE == TC_DGRAD ? "tc_gemm_dgrad" : "tc_gemm_wgrad", s);
     tc_gemm_kernel<MODE><<<grid, kThreads, kSmemBytes, s>>>(P);
-    count_launch();
     return cudaGetLastError();
 }
 
@@ -654,8 +654,8 @@ void umma_destroy(UmmaEngine* e) {
 
 cudaError_t umma_refresh_weights(UmmaEngine* e) {
     dim3 grid(std::max(1, std::min(64, (e->cvt_max + 255) / 256)), e->n_cvt);
+    LaunchScope scope_("convert_weights", e->s.stream);
     convert_weights_kernel<<<grid, 256, 0, e->s.stream>>>(e->cvt_dev);
-    count_launch();
     return cudaGetLastError();
 }
 

@@ -446,9 +446,9 @@ __global__ void __launch_bounds__(kAdamThreads) adam_kernel(const AdamArgs a) {
 cudaError_t launch_gather(const GatherArgs& a, cudaStream_t s) {
     if (a.Bmb <= 0) return cudaSuccess;
     const int blocks = std::min((a.Bmb + 7) / 8, 148 * 8);
+    LaunchScope scope_("gather", s);
     if (a.x_a16) gather_kernel<true><<<blocks, 256, 0, s>>>(a);
     else gather_kernel<false><<<blocks, 256, 0, s>>>(a);
-    count_launch();
     return cudaGetLastError();
 }
 
@@ -456,8 +456,8 @@ cudaError_t launch_perm_rows(uint64_t seed, uint32_t iteration, uint32_t epoch, 
                              uint32_t first, int count, int* rows_out, cudaStream_t s) {
     if (count <= 0) return cudaSuccess;
     PermKey pk{(uint32_t)seed, (uint32_t)(seed >> 32), iteration, epoch, batch, feistel_half_bits(batch)};
+    LaunchScope scope_("perm_rows", s);
     perm_rows_kernel<<<(count + 255) / 256, 256, 0, s>>>(pk, first, count, rows_out);
-    count_launch();
     return cudaGetLastError();
 }
 
@@ -468,6 +468,7 @@ cudaError_t launch_head_loss(const HeadLossArgs& a, cudaStream_t s) {
     const int blocks = head_loss_blocks(a.Bmb);
     const size_t smem = sizeof(float) * ((size_t)a.hp.n_a * (a.hp.ldwa + 1) + (size_t)a.hp.n_c * 2 +
                                          (size_t)kHLWarps * kPartialStride);
+    LaunchScope scope_("head_loss", s);
     cudaError_t e;
     if (a.bf16_act) {
         e = cudaFuncSetAttribute(head_loss_kernel<__nv_bfloat16>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
@@ -478,31 +479,30 @@ cudaError_t launch_head_loss(const HeadLossArgs& a, cudaStream_t s) {
         if (e != cudaSuccess) return e;
         head_loss_kernel<float><<<blocks, kHLThreads, smem, s>>>(a);
     }
-    count_launch();
     return cudaGetLastError();
 }
 
 cudaError_t launch_head_finalize(const float* block_partials, int nblocks, float* partials0, int off_ba,
                                  int off_logstd, int off_bc, int A, float entropy_coef,
                                  const float* log_std, float* loss_sums, cudaStream_t s) {
+    LaunchScope scope_("head_finalize", s);
     head_finalize_kernel<<<1, 256, 0, s>>>(block_partials, nblocks, partials0, off_ba, off_logstd, off_bc, A,
                                            entropy_coef, log_std, loss_sums);
-    count_launch();
     return cudaGetLastError();
 }
 
 int reduce_blocks(int P) { return (P + kRedThreads * kRedPerThread - 1) / (kRedThreads * kRedPerThread); }
 
 cudaError_t launch_reduce(const ReduceArgs& a, cudaStream_t s) {
+    LaunchScope scope_("grad_reduce", s);
     reduce_kernel<<<reduce_blocks(a.P), kRedThreads, 0, s>>>(a);
-    count_launch();
     return cudaGetLastError();
 }
 
 cudaError_t launch_adam(const AdamArgs& a, cudaStream_t s) {
     const int blocks = std::max(1, std::min((a.P / 4 + kAdamThreads - 1) / kAdamThreads, 148 * 4));
+    LaunchScope scope_("adam", s);
     adam_kernel<<<blocks, kAdamThreads, 0, s>>>(a);
-    count_launch();
     return cudaGetLastError();
 }
 
