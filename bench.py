@@ -1,0 +1,352 @@
+#!/usr/bin/env python
+"""Benchmark of the PPO learn-iteration hot path (rollout inference + GAE + PPO update).
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--impl ours|reference]
+
+One "step" is one whole learn iteration over one rollout of synthetic data:
+T x (rslrl_act + rslrl_record_step), rslrl_gae, rslrl_ppo_update (E x M minibatch steps).
+The metric is transitions/s = T * N_envs * K / time.  Rank 0 prints ONE JSON line.
+
+  value   inputs already resident in device memory when the timed region starts
+  e2e     the same iteration through the host-buffer entry points (pinned host memory,
+          host<->device copies inside the timed region)
+  roofline  the kernel family with the largest share of device time, from a separate pass of
+          the same K steps with one CUDA event pair per launch
+  cpu_baseline  the FP64 oracle, as it stands, on the host cores, on a bounded sample
+
+With --gpus N > 1 (launched by torch.distributed.run) every rank runs an independent replica
+of the workload on its own GPU: the path has no inter-GPU exchange ("replicas only").
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import statistics
+import subprocess
+import sys
+import time
+
+import numpy as np
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+sys.path.insert(0, ROOT)
+
+from paper_2509_10771_b200 import workloads as WL  # noqa: E402
+
+METRIC = "PPO learn-iteration transitions/s"
+UNIT = "transitions/s"
+WORKLOAD = WL.ROUGH                       # rough-terrain locomotion shape: the config the metric is quoted on
+PRECISION = WL.PRECISION_BF16
+ORACLE_SAMPLE_ENVS = 512                  # bounded sample for the CPU baseline: 512 of the 4096 environments
+
+
+def read_peaks():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        d = json.load(open(path))
+        return {"hbm_gbs": d["hbm_gbs"], "bf16_tflops": d["bf16_tflops"],
+                "bf16_tflops_sustained": d.get("bf16_tflops_sustained", d["bf16_tflops"]), "source": "measured"}
+    return {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0, "source": "fallback"}
+
+
+# ------------------------------------------------------------------------------------------
+# algorithmic work per learn iteration (real layer widths, no padding)
+# ------------------------------------------------------------------------------------------
+def hidden_flops_per_row(w, net):
+    return sum(2 * i * o for i, o in w.layer_dims(net)[:-1])
+
+
+def family_flops(w):
+    """FLOPs of one learn iteration attributed to the three tensor-core kernel families."""
+    T, N = w.num_steps, w.num_envs
+    steps = w.epochs * w.minibatches
+    R = w.minibatch_rows * (2 if w.sym_enable else 1)
+    fa, fc = hidden_flops_per_row(w, "actor"), hidden_flops_per_row(w, "critic")
+    fwd = T * N * (fa + fc) + N * fc + steps * R * (fa + fc)
+    dgrad = steps * R * sum(2 * i * o for net in ("actor", "critic") for i, o in w.layer_dims(net)[1:-1])
+    wgrad = steps * R * sum(2 * i * o for net in ("actor", "critic") for i, o in w.layer_dims(net))
+    return {"tc_gemm_fwd": fwd, "tc_gemm_dgrad": dgrad, "tc_gemm_wgrad": wgrad}
+
+
+def iteration_flops(w):
+    T, N = w.num_steps, w.num_envs
+    steps = w.epochs * w.minibatches
+    R = w.minibatch_rows * (2 if w.sym_enable else 1)
+    full = sum(2 * i * o for net in ("actor", "critic") for i, o in w.layer_dims(net))
+    first = sum(2 * i * o for net in ("actor", "critic") for i, o in w.layer_dims(net)[:1])
+    return T * N * full + steps * R * (3 * full - first)
+
+
+# ------------------------------------------------------------------------------------------
+# the oracle arm (CPU baseline and --impl reference)
+# ------------------------------------------------------------------------------------------
+def oracle_iteration_seconds(w, repeats=1):
+    from oracle import ppo_oracle as O
+    dims = (w.layer_dims("actor"), w.layer_dims("critic"), w.num_actions)
+    theta = WL.make_params(w).astype(np.float64)
+    inputs = WL.make_rollout_inputs(w)
+    mir = WL.make_mirror(w) if w.sym_enable else None
+    state = O.OptimState(theta, w.lr)
+    times = []
+    for it in range(repeats):
+        t0 = time.perf_counter()
+        storage = O.rollout(state.theta, dims, inputs, w, seed=w.seed, first_global_step=it * w.num_steps)
+        O.ppo_update(state, dims, storage, w, seed=w.seed, iteration=it, sym=mir)
+        times.append(time.perf_counter() - t0)
+    return times
+
+
+def blas_threads():
+    try:
+        from threadpoolctl import threadpool_info
+        n = [p.get("num_threads", 0) for p in threadpool_info() if p.get("user_api") == "blas"]
+        return max(n) if n else os.cpu_count()
+    except Exception:
+        return os.cpu_count()
+
+
+def run_reference(args, rank):
+    if rank != 0:
+        return
+    w = WORKLOAD.scaled(ORACLE_SAMPLE_ENVS)
+    times = oracle_iteration_seconds(w, repeats=args.warmup + args.steps)[args.warmup:]
+    total = sum(times)
+    value = w.batch * len(times) / total
+    sample = (f"{ORACLE_SAMPLE_ENVS} of the {WORKLOAD.num_envs} environments of {WORKLOAD.name}, whole learn "
+              f"iterations (T={w.num_steps}, E={w.epochs}, M={w.minibatches}), numpy float64")
+    line = {
+        "impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus,
+        "steps": args.steps, "warmup": args.warmup, "ms_per_step": 1e3 * total / len(times),
+        "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+        "config": {"workload": WORKLOAD.name, "sample": sample},
+        "cpu_baseline": {"value": value, "unit": UNIT, "cores": blas_threads(), "kind": "oracle", "sample": sample},
+        "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+        "gpu_launches": 0,
+    }
+    print(json.dumps(line), flush=True)
+
+
+# ------------------------------------------------------------------------------------------
+# clocks
+# ------------------------------------------------------------------------------------------
+class ClockSampler:
+    QUERY = ("index,clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,"
+             "clocks_event_reasons.hw_slowdown,clocks_event_reasons.hw_thermal_slowdown,"
+             "clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, device_index):
+        self.proc = None
+        self.idx = device_index
+
+    def start(self):
+        try:
+            self.proc = subprocess.Popen(["nvidia-smi", f"--query-gpu={self.QUERY}", "--format=csv,noheader,nounits",
+                                          "-lms", "100", "-i", str(self.idx)], stdout=subprocess.PIPE,
+                                         stderr=subprocess.DEVNULL, text=True)
+        except Exception:
+            self.proc = None
+
+    def stop(self):
+        if self.proc is None:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
+        self.proc.terminate()
+        try:
+            out, _ = self.proc.communicate(timeout=5)
+        except Exception:
+            self.proc.kill()
+            out = ""
+        sm, smax, reasons = [], [], set()
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        for line in out.splitlines():
+            f = [x.strip() for x in line.split(",")]
+            if len(f) < 9:
+                continue
+            try:
+                sm.append(float(f[1])); smax.append(float(f[2]))
+            except ValueError:
+                continue
+            for name, val in zip(names, f[5:9]):
+                if val.lower().startswith("active"):
+                    reasons.add(name)
+        return {"sm_mhz": statistics.median(sm) if sm else None, "sm_max_mhz": max(smax) if smax else None,
+                "samples": len(sm), "reasons": sorted(reasons)}
+
+
+# ------------------------------------------------------------------------------------------
+def run_ours(args, rank, world, local_rank):
+    import torch
+    import torch.distributed as dist
+    from paper_2509_10771_b200 import binding, build
+
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device: the path has no CPU fallback")
+    torch.cuda.set_device(local_rank)
+    if world > 1:
+        dist.init_process_group("nccl", device_id=torch.device("cuda", local_rank))
+    if rank == 0:
+        build.build()
+    if world > 1:
+        dist.barrier()
+
+    w = WORKLOAD
+    T, N, A = w.num_steps, w.num_envs, w.num_actions
+    inputs = WL.make_rollout_inputs(w, seed=rank)          # every replica draws its own rollout
+    theta = WL.make_params(w, seed=rank)
+    dev = torch.device("cuda", local_rank)
+    stream = torch.cuda.current_stream()
+    ctx = binding.Context(w, precision=PRECISION, stream=stream.cuda_stream)
+    ctx.set_params(theta)
+
+    d_obs = torch.from_numpy(inputs["obs_actor"]).to(dev)
+    d_rew = torch.from_numpy(inputs["rewards"]).to(dev)
+    d_done = torch.from_numpy(inputs["dones"]).to(dev)
+    d_to = torch.from_numpy(inputs["timeouts"]).to(dev)
+    flush_buf = torch.empty(256 << 20, dtype=torch.uint8, device=dev)      # 2x the 126 MB L2
+
+    def iteration_device():
+        for t in range(T):
+            ctx.act(d_obs[t])
+            ctx.record_step(d_rew[t], d_done[t], d_to[t])
+        ctx.gae(d_obs[T])
+        ctx.ppo_update(want_stats=False)
+
+    h_obs = torch.from_numpy(inputs["obs_actor"]).pin_memory()
+    h_rew = torch.from_numpy(inputs["rewards"]).pin_memory()
+    h_done = torch.from_numpy(inputs["dones"]).pin_memory()
+    h_to = torch.from_numpy(inputs["timeouts"]).pin_memory()
+    h_act = torch.empty((N, A), dtype=torch.float32).pin_memory()
+    np_obs, np_rew, np_done, np_to, np_act = (x.numpy() for x in (h_obs, h_rew, h_done, h_to, h_act))
+
+    def iteration_host():
+        for t in range(T):
+            ctx.act_host(np_obs[t], None, np_act)          # H2D obs, D2H actions (waits for them)
+            ctx.record_step_host(np_rew[t], np_done[t], np_to[t])
+        ctx.gae_host(np_obs[T])
+        return ctx.ppo_update(want_stats=True)             # D2H of the update's scalars
+
+    h2d = T * (N * w.actor_obs_dim * 4 + N * 4 + 2 * N) + N * w.critic_obs_dim * 4
+    d2h = T * N * A * 4 + w.epochs * w.minibatches * 8 * 4
+
+    def barrier():
+        torch.cuda.synchronize()
+        if world > 1:
+            dist.barrier()
+            torch.cuda.synchronize()
+
+    def timed(fn, steps):
+        """Sum of per-step device times (CUDA events on the launching stream); L2 flushed between steps."""
+        evs = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(steps)]
+        barrier()
+        for a, b in evs:
+            flush_buf.zero_()
+            a.record(stream)
+            fn()
+            b.record(stream)
+        barrier()
+        return sum(a.elapsed_time(b) for a, b in evs)      # ms
+
+    for _ in range(max(args.warmup, 3)):
+        iteration_device()
+    torch.cuda.synchronize()
+
+    try:
+        gpu_id = "GPU-" + str(torch.cuda.get_device_properties(local_rank).uuid)
+    except Exception:
+        gpu_id = str(local_rank)
+    sampler = ClockSampler(gpu_id)
+    launches0 = binding.kernel_launch_count()
+    sampler.start()
+    ms_total = timed(iteration_device, args.steps)
+    clocks = sampler.stop()
+    launches = binding.kernel_launch_count() - launches0
+
+    iteration_host()
+    ms_e2e = timed(iteration_host, args.steps)
+
+    # per-kernel pass: the same K steps with one event pair per launch
+    binding.profile_enable(True)
+    binding.profile_report()
+    for _ in range(args.steps):
+        flush_buf.zero_()
+        iteration_device()
+    torch.cuda.synchronize()
+    prof = binding.profile_report()
+    binding.profile_enable(False)
+
+    if world > 1:
+        t = torch.tensor([ms_total, ms_e2e], dtype=torch.float64, device=dev)
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        ms_total, ms_e2e = t.tolist()
+    if rank != 0:
+        if world > 1:
+            dist.destroy_process_group()
+        return
+
+    peaks = read_peaks()
+    transitions = T * N * args.steps * world
+    value = transitions / (ms_total * 1e-3)
+    e2e_value = transitions / (ms_e2e * 1e-3)
+
+    total_prof_ms = sum(v["ms"] for v in prof.values()) or 1.0
+    shares = {k: {"launches": v["launches"], "ms": round(v["ms"], 3), "share": round(v["ms"] / total_prof_ms, 4)}
+              for k, v in sorted(prof.items(), key=lambda kv: -kv[1]["ms"])}
+    fam_flops = family_flops(w)
+    tc = {k: v for k, v in prof.items() if k in fam_flops}
+    top = max(tc, key=lambda k: tc[k]["ms"])
+    achieved = fam_flops[top] * args.steps / (tc[top]["ms"] * 1e-3) / 1e12
+    peak = peaks["bf16_tflops_sustained"]
+    roofline = {"bound": "tensor", "kernel": top, "achieved": achieved, "peak": peak, "unit": "TFLOP/s",
+                "frac": achieved / peak, "traffic": None, "peak_source": f"bf16 sustained, {peaks['source']}",
+                "avg_launch_us": 1e3 * tc[top]["ms"] / tc[top]["launches"],
+                "families": {k: {"tflops": fam_flops[k] * args.steps / (tc[k]["ms"] * 1e-3) / 1e12,
+                                 "frac": fam_flops[k] * args.steps / (tc[k]["ms"] * 1e-3) / 1e12 / peak} for k in tc},
+                "timing": "one CUDA event pair per launch, separate pass over the same K steps"}
+
+    ws = WORKLOAD.scaled(ORACLE_SAMPLE_ENVS)
+    o_times = oracle_iteration_seconds(ws, repeats=1)
+    sample = (f"one whole learn iteration on {ORACLE_SAMPLE_ENVS} of the {w.num_envs} environments of {w.name} "
+              f"(T={w.num_steps}, E={w.epochs}, M={w.minibatches}), numpy float64")
+    cpu = {"value": ws.batch / o_times[0], "unit": UNIT, "cores": blas_threads(), "kind": "oracle", "sample": sample}
+
+    line = {
+        "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": max(args.warmup, 3),
+        "ms_per_step": ms_total / args.steps, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+        "dtype": "bf16", "data": "synthetic",
+        "config": {"workload": w.name, "num_envs": N, "num_steps": T, "obs_dim": w.actor_obs_dim, "actions": A,
+                   "hidden": list(w.actor_hidden), "epochs": w.epochs, "minibatches": w.minibatches,
+                   "precision": "bf16 operands, fp32 accumulate", "l2": "256 MiB buffer written between timed steps",
+                   "parallelism": "replicas only" if world > 1 else "1 gpu"},
+        "clocks": clocks,
+        "e2e": {"value": e2e_value, "unit": UNIT, "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h,
+                "ms_per_step": ms_e2e / args.steps},
+        "gpu_launches": int(launches),
+        "roofline": roofline,
+        "iteration_tflops": iteration_flops(w) * args.steps * world / (ms_total * 1e-3) / 1e12,
+        "kernel_shares": shares,
+        "cpu_baseline": cpu,
+    }
+    print(json.dumps(line), flush=True)
+    ctx.destroy()
+    if world > 1:
+        dist.destroy_process_group()
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=10)
+    ap.add_argument("--warmup", type=int, default=3)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    args = ap.parse_args()
+    rank = int(os.environ.get("RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    local_rank = int(os.environ.get("LOCAL_RANK", "0"))
+    if args.impl == "reference":
+        run_reference(args, rank)
+    else:
+        run_ours(args, rank, world, local_rank)
+
+
+if __name__ == "__main__":
+    main()
