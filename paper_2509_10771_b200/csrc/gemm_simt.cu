@@ -228,28 +228,54 @@ cudaError_t launch_sgemm(const GemmBatch& b, bool ta, bool tb, int epi, cudaStre
 }
 
 // ---------------------------------------------------------------------------------------
-// Column sums over a split of the rows (bias gradients).  grid = (ceil(n/128), splits, count),
-// 128 threads = 128 columns, coalesced across columns.
+// Column sums over a split of the rows (bias gradients).  grid = (ceil(n/32), splits, count);
+// a block of 1024 threads covers 32 columns (16 column pairs) with 64 row lanes, so that the
+// whole machine is busy even when there are only a few splits.  The 64 row-lane partials of a
+// column are added in a fixed order: the result does not depend on scheduling.
 // ---------------------------------------------------------------------------------------
 namespace {
+constexpr int kCsPairs = 16, kCsLanes = 64;
+
+__device__ __forceinline__ float2 load_pair(const float* p) { return *reinterpret_cast<const float2*>(p); }
+__device__ __forceinline__ float2 load_pair(const __nv_bfloat16* p) {
+    return __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162*>(p));
+}
+
 template <typename T>
-__global__ void colsum_kernel(const ColsumBatch b) {
+__global__ void __launch_bounds__(kCsPairs * kCsLanes) colsum_kernel(const ColsumBatch b) {
     const ColsumProblem& p = b.p[blockIdx.z];
-    const int n = blockIdx.x * blockDim.x + threadIdx.x;
-    if (n >= p.n) return;
+    __shared__ float2 part[kCsLanes][kCsPairs];
+    const int pair = threadIdx.x % kCsPairs, rl = threadIdx.x / kCsPairs;
+    const int n = blockIdx.x * (2 * kCsPairs) + 2 * pair;      // leading dimensions are even
+    if (blockIdx.x * (2 * kCsPairs) >= p.n) return;
     const int chunk = (p.rows + b.splits - 1) / b.splits;
     const int r0 = blockIdx.y * chunk, r1 = min(p.rows, r0 + chunk);
     const T* X = reinterpret_cast<const T*>(p.X);
-    float s0 = 0.f, s1 = 0.f, s2 = 0.f, s3 = 0.f;
-    int r = r0;
-    for (; r + 3 < r1; r += 4) {
-        s0 += to_float(X[(size_t)r * p.ld + n]);
-        s1 += to_float(X[(size_t)(r + 1) * p.ld + n]);
-        s2 += to_float(X[(size_t)(r + 2) * p.ld + n]);
-        s3 += to_float(X[(size_t)(r + 3) * p.ld + n]);
+    float2 s0 = make_float2(0.f, 0.f), s1 = s0, s2 = s0, s3 = s0;
+    if (n < p.ld) {
+        int r = r0 + rl;
+        for (; r + 3 * kCsLanes < r1; r += 4 * kCsLanes) {
+            const float2 a0 = load_pair(X + (size_t)r * p.ld + n);
+            const float2 a1 = load_pair(X + (size_t)(r + kCsLanes) * p.ld + n);
+            const float2 a2 = load_pair(X + (size_t)(r + 2 * kCsLanes) * p.ld + n);
+            const float2 a3 = load_pair(X + (size_t)(r + 3 * kCsLanes) * p.ld + n);
+            s0.x += a0.x; s0.y += a0.y; s1.x += a1.x; s1.y += a1.y;
+            s2.x += a2.x; s2.y += a2.y; s3.x += a3.x; s3.y += a3.y;
+        }
+        for (; r < r1; r += kCsLanes) {
+            const float2 a0 = load_pair(X + (size_t)r * p.ld + n);
+            s0.x += a0.x; s0.y += a0.y;
+        }
     }
-    for (; r < r1; ++r) s0 += to_float(X[(size_t)r * p.ld + n]);
-    p.out[(size_t)blockIdx.y * b.split_stride + n] = (s0 + s1) + (s2 + s3);
+    part[rl][pair] = make_float2((s0.x + s1.x) + (s2.x + s3.x), (s0.y + s1.y) + (s2.y + s3.y));
+    __syncthreads();
+    if (threadIdx.x < 2 * kCsPairs) {
+        const int c = threadIdx.x;                 // column within the block
+        float t = 0.f;
+        for (int l = 0; l < kCsLanes; ++l) t += (c & 1) ? part[l][c >> 1].y : part[l][c >> 1].x;
+        const int col = blockIdx.x * (2 * kCsPairs) + c;
+        if (col < p.n) p.out[(size_t)blockIdx.y * b.split_stride + col] = t;
+    }
 }
 }  // namespace
 
@@ -257,10 +283,10 @@ cudaError_t launch_colsum(const ColsumBatch& b, cudaStream_t s) {
     if (b.count <= 0) return cudaSuccess;
     int nmax = 0;
     for (int i = 0; i < b.count; ++i) nmax = std::max(nmax, b.p[i].n);
-    dim3 grid((nmax + 127) / 128, b.splits, b.count);
+    dim3 grid((nmax + 2 * kCsPairs - 1) / (2 * kCsPairs), b.splits, b.count);
     LaunchScope scope_("colsum", s);
-    if (b.is_bf16) colsum_kernel<__nv_bfloat16><<<grid, 128, 0, s>>>(b);
-    else colsum_kernel<float><<<grid, 128, 0, s>>>(b);
+    if (b.is_bf16) colsum_kernel<__nv_bfloat16><<<grid, kCsPairs * kCsLanes, 0, s>>>(b);
+    else colsum_kernel<float><<<grid, kCsPairs * kCsLanes, 0, s>>>(b);
     return cudaGetLastError();
 }
 

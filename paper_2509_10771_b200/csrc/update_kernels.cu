@@ -323,23 +323,21 @@ __global__ void __launch_bounds__(256) head_finalize_kernel(const float* __restr
         for (int i = 0; i < A; ++i) ent += 0.5f + kHalfLog2Pi + log_std[i];
         loss_sums[LS_COUNT] = ent;
     }
-    for (int e = threadIdx.x; e < kPartialStride; e += blockDim.x) {
+    // one warp per entry: lane l adds blocks l, l+32, ... in order, then a fixed shuffle tree
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5, nwarps = blockDim.x >> 5;
+    for (int e = warp; e < kPartialStride; e += nwarps) {
         if (e >= 5 && e < 8) continue;
-        // four interleaved accumulators, fixed association
-        float s0 = 0.f, s1 = 0.f, s2 = 0.f, s3 = 0.f;
-        int b = 0;
-        for (; b + 3 < nblocks; b += 4) {
-            s0 += block_partials[(size_t)b * kPartialStride + e];
-            s1 += block_partials[(size_t)(b + 1) * kPartialStride + e];
-            s2 += block_partials[(size_t)(b + 2) * kPartialStride + e];
-            s3 += block_partials[(size_t)(b + 3) * kPartialStride + e];
-        }
-        for (; b < nblocks; ++b) s0 += block_partials[(size_t)b * kPartialStride + e];
-        const float s = (s0 + s1) + (s2 + s3);
+        if (e >= 8 && e < 8 + kMaxActions && e - 8 >= A) continue;
+        if (e >= 8 + kMaxActions && e - 8 - kMaxActions >= A) continue;
+        float s = 0.f;
+        for (int b = lane; b < nblocks; b += 32) s += block_partials[(size_t)b * kPartialStride + e];
+#pragma unroll
+        for (int o = 16; o > 0; o >>= 1) s += __shfl_down_sync(0xffffffffu, s, o);
+        if (lane != 0) continue;
         if (e < LS_COUNT) loss_sums[e] = s;
         else if (e == 4) partials0[off_bc] = s;
-        else if (e < 8 + kMaxActions) { if (e - 8 < A) partials0[off_ba + e - 8] = s; }
-        else { const int i = e - 8 - kMaxActions; if (i < A) partials0[off_logstd + i] = s - entropy_coef; }
+        else if (e < 8 + kMaxActions) partials0[off_ba + e - 8] = s;
+        else partials0[off_logstd + e - 8 - kMaxActions] = s - entropy_coef;
     }
 }
 
