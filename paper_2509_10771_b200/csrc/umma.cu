@@ -4,9 +4,9 @@
 // one tile overlaps the main loop of the next), and the epilogues fuse bias+ELU (forward),
 // the ELU derivative (data gradient) or the split-partial store (weight gradient).
 //
-// Warp roles in a CTA of 320 threads: warp 0 = TMA producer, warp 1 = MMA issuer and owner of
-// the tensor-memory allocation, warps 2..9 = epilogue (each reads its quarter of the 128
-// accumulator lanes and half of the tile's columns).
+// Warp roles in a CTA of 576 threads: warp 0 = TMA producer, warp 1 = MMA issuer and owner of
+// the tensor-memory allocation, warps 2..17 = epilogue (each reads its quarter of the 128
+// accumulator lanes and every fourth 32-column chunk of the tile).
 //
 // Every wait on an mbarrier is bounded in time; on expiry the CTA raises an error flag that
 // the host reads, drains its own asynchronous work, frees its tensor memory and returns.
@@ -26,7 +26,7 @@ constexpr int BLOCK_M = 128;
 constexpr int BLOCK_K = 64;                      // bf16 elements = one 128-byte swizzle row
 constexpr int UMMA_K = 16;
 constexpr int kMaxBN = 256;
-constexpr int kEpiWarps = 8;
+constexpr int kEpiWarps = 16;
 constexpr int kThreads = 32 * (2 + kEpiWarps);
 constexpr uint32_t kStageA = BLOCK_M * BLOCK_K * 2;      // 16 KiB
 constexpr uint32_t kStageB = kMaxBN * BLOCK_K * 2;       // 32 KiB
@@ -185,7 +185,11 @@ __device__ __forceinline__ Item decode_item(const TcParams& P, int item) {
     return it;
 }
 
-__device__ __forceinline__ float elu_fast(float z, float alpha) { return z > 0.f ? z : alpha * (__expf(z) - 1.0f); }
+// Branch-free ELU; the exponential is the fast hardware one, which is ample for a BF16 result.
+__device__ __forceinline__ float elu_fast(float z, float alpha) {
+    const float e = alpha * (__expf(fminf(z, 0.f)) - 1.0f);
+    return z > 0.f ? z : e;
+}
 
 template <int MODE>
 __global__ void __launch_bounds__(kThreads, 1) tc_gemm_kernel(const __grid_constant__ TcParams P) {
@@ -303,7 +307,7 @@ __global__ void __launch_bounds__(kThreads, 1) tc_gemm_kernel(const __grid_const
     } else {
         // ================================ epilogue =====================================
         const int q = warp & 3;                    // accumulator lanes 32q .. 32q+31
-        const int half = (warp - 2) >> 2;          // which half of the tile's columns
+        const int group = (warp - 2) >> 2;         // handles chunks group, group + 4, ...
         bool ok = true;
         int local = 0;
         for (int item = blockIdx.x; ok && item < P.total_items; item += gridDim.x, ++local) {
@@ -311,36 +315,55 @@ __global__ void __launch_bounds__(kThreads, 1) tc_gemm_kernel(const __grid_const
             const TcProblem& p = P.p[it.prob];
             const int buf = local & 1;
             const uint32_t use = (uint32_t)(local >> 1);
-            if (!mbar_wait(&tfull[buf], use & 1u, abort_flag, P.error, 4)) { ok = false; break; }
-            tc_fence_after();
             const int row = it.m0 + 32 * q + lane;
             const int chunks = p.bn / 32;
-            const int c_begin = half * (chunks / 2), c_end = (half + 1) * (chunks / 2);
-            for (int c = c_begin; c < c_end; ++c) {
+            // data gradient: fetch the stored post-activations of this thread's chunks before
+            // waiting for the accumulator, so that the loads overlap the main loop
+            uint4 haux[2][4];
+            if (MODE == TC_DGRAD) {
+#pragma unroll
+                for (int ci = 0; ci < 2; ++ci) {
+                    const int col = it.n0 + 32 * (group + 4 * ci);
+                    if (group + 4 * ci < chunks && row < p.m_extent && col < p.n_extent) {
+                        const uint4* hsrc = reinterpret_cast<const uint4*>(p.aux16 + (size_t)row * p.ld_aux + col);
+#pragma unroll
+                        for (int g = 0; g < 4; ++g) haux[ci][g] = __ldg(hsrc + g);
+                    }
+                }
+            }
+            if (!mbar_wait(&tfull[buf], use & 1u, abort_flag, P.error, 4)) { ok = false; break; }
+            tc_fence_after();
+#pragma unroll
+            for (int ci = 0; ci < 2; ++ci) {
+                const int c = group + 4 * ci;
+                if (c >= chunks) break;                       // uniform across the warp
                 uint32_t acc[32];
                 tmem_ld32(tmem_base + ((uint32_t)(32 * q) << 16) + (uint32_t)(buf * kMaxBN + 32 * c), acc);
                 const int col = it.n0 + 32 * c;
                 if (row >= p.m_extent || col >= p.n_extent) continue;
                 if (MODE == TC_FWD) {
-                    uint32_t packed[16];
-#pragma unroll
-                    for (int j = 0; j < 32; j += 2) {
-                        const float b0 = (col + j < p.bias_n) ? __ldg(p.bias + col + j) : 0.f;
-                        const float b1 = (col + j + 1 < p.bias_n) ? __ldg(p.bias + col + j + 1) : 0.f;
-                        const float v0 = elu_fast(__uint_as_float(acc[j]) + b0, P.alpha);
-                        const float v1 = elu_fast(__uint_as_float(acc[j + 1]) + b1, P.alpha);
-                        __nv_bfloat162 h2 = __floats2bfloat162_rn(v0, v1);
-                        packed[j / 2] = *reinterpret_cast<uint32_t*>(&h2);
-                    }
-                    uint4* dst = reinterpret_cast<uint4*>(p.out16 + (size_t)row * p.ld_out + col);
-#pragma unroll
-                    for (int g = 0; g < 4; ++g) dst[g] = make_uint4(packed[4 * g], packed[4 * g + 1], packed[4 * g + 2], packed[4 * g + 3]);
-                } else if (MODE == TC_DGRAD) {
-                    const uint4* hsrc = reinterpret_cast<const uint4*>(p.aux16 + (size_t)row * p.ld_aux + col);
+                    // p.bias is zero-padded to the padded width: no bounds checks
+                    const float4* b4 = reinterpret_cast<const float4*>(p.bias + col);
                     uint4* dst = reinterpret_cast<uint4*>(p.out16 + (size_t)row * p.ld_out + col);
 #pragma unroll
                     for (int g = 0; g < 4; ++g) {
-                        const uint4 hv = __ldg(hsrc + g);
+                        const float4 ba = __ldg(b4 + 2 * g), bb = __ldg(b4 + 2 * g + 1);
+                        const float bv[8] = {ba.x, ba.y, ba.z, ba.w, bb.x, bb.y, bb.z, bb.w};
+                        uint32_t o[4];
+#pragma unroll
+                        for (int e = 0; e < 4; ++e) {
+                            const float v0 = elu_fast(__uint_as_float(acc[8 * g + 2 * e]) + bv[2 * e], P.alpha);
+                            const float v1 = elu_fast(__uint_as_float(acc[8 * g + 2 * e + 1]) + bv[2 * e + 1], P.alpha);
+                            __nv_bfloat162 h2 = __floats2bfloat162_rn(v0, v1);
+                            o[e] = *reinterpret_cast<uint32_t*>(&h2);
+                        }
+                        dst[g] = make_uint4(o[0], o[1], o[2], o[3]);
+                    }
+                } else if (MODE == TC_DGRAD) {
+                    uint4* dst = reinterpret_cast<uint4*>(p.out16 + (size_t)row * p.ld_out + col);
+#pragma unroll
+                    for (int g = 0; g < 4; ++g) {
+                        const uint4 hv = haux[ci][g];
                         const uint32_t hw[4] = {hv.x, hv.y, hv.z, hv.w};
                         uint32_t o[4];
 #pragma unroll
@@ -379,6 +402,7 @@ __global__ void __launch_bounds__(kThreads, 1) tc_gemm_kernel(const __grid_const
 
 // ------------------------------------------------------------------------- small kernels
 struct CvtEntry {
+    const float* bsrc; float* bdst;             // bias -> zero-padded FP32 copy
     const float* src; int in, out, ld_src;      // FP32 master W[in][ld_src]
     __nv_bfloat16* wt; int ld_wt;               // [out][ld_wt]  (contraction = in)   forward operand
     __nv_bfloat16* wn; int ld_wn;               // [in][ld_wn]   (contraction = out)  data-gradient operand, may be null
@@ -387,6 +411,7 @@ struct CvtEntry {
 __global__ void convert_weights_kernel(const CvtEntry* __restrict__ table) {
     const CvtEntry e = table[blockIdx.y];
     const int total = e.in * e.out;
+    for (int o = blockIdx.x * blockDim.x + threadIdx.x; o < e.out; o += gridDim.x * blockDim.x) e.bdst[o] = e.bsrc[o];
     for (int idx = blockIdx.x * blockDim.x + threadIdx.x; idx < total; idx += gridDim.x * blockDim.x) {
         const int i = idx / e.out, o = idx - i * e.out;
         const __nv_bfloat16 v = __float2bfloat16_rn(e.src[(size_t)i * e.ld_src + o]);
@@ -440,6 +465,7 @@ struct UmmaEngine {
     __nv_bfloat16 *x16[2] = {}, *h[2][kMaxLayers] = {}, *dz[2][kMaxLayers] = {};
     __nv_bfloat16 *dmu16 = nullptr, *dv16 = nullptr;
     __nv_bfloat16 *wt[2][kMaxLayers] = {}, *wn[2][kMaxLayers] = {};
+    float* bias_pad[2][kMaxLayers] = {};         // [pw] zero-padded copies of the hidden biases
     CvtEntry* cvt_dev = nullptr; int n_cvt = 0; int cvt_max = 0;
     int* error_dev = nullptr;
     int num_sms = 148;
@@ -543,7 +569,8 @@ UmmaEngine* umma_create(const UmmaSetup& s, std::string* err) {
         for (int l = 0; l < e->nh[ni]; ++l) {
             const int kin = l == 0 ? e->kp[ni] : e->pw[ni][l - 1];
             if (!ealloc(e, &e->h_act[ni][l], (size_t)N * e->pw[ni][l]) || !ealloc(e, &e->h[ni][l], (size_t)R * e->pw[ni][l]) ||
-                !ealloc(e, &e->dz[ni][l], (size_t)R * e->pw[ni][l]) || !ealloc(e, &e->wt[ni][l], (size_t)e->pw[ni][l] * kin))
+                !ealloc(e, &e->dz[ni][l], (size_t)R * e->pw[ni][l]) || !ealloc(e, &e->wt[ni][l], (size_t)e->pw[ni][l] * kin) ||
+                !ealloc(e, &e->bias_pad[ni][l], (size_t)e->pw[ni][l]))
                 return bail("allocation failed");
             if (l > 0 && !ealloc(e, &e->wn[ni][l], (size_t)e->pw[ni][l - 1] * e->pw[ni][l])) return bail("allocation failed");
         }
@@ -555,6 +582,7 @@ UmmaEngine* umma_create(const UmmaSetup& s, std::string* err) {
     for (int ni = 0; ni < 2; ++ni)
         for (int l = 0; l < e->nh[ni]; ++l) {
             CvtEntry c{};
+            c.bsrc = s.param + s.b_off[ni][l]; c.bdst = e->bias_pad[ni][l];
             c.src = s.param + s.w_off[ni][l]; c.in = s.in[ni][l]; c.out = s.out[ni][l]; c.ld_src = s.out_p[ni][l];
             c.wt = e->wt[ni][l]; c.ld_wt = l == 0 ? e->kp[ni] : e->pw[ni][l - 1];
             c.wn = l > 0 ? e->wn[ni][l] : nullptr; c.ld_wn = e->pw[ni][l];
@@ -580,7 +608,7 @@ UmmaEngine* umma_create(const UmmaSetup& s, std::string* err) {
                 const int k = l == 0 ? e->kp[ni] : e->pw[ni][l - 1];
                 if (!add_rowmajor_problem(P, in, rows, k, e->wt[ni][l], e->pw[ni][l])) return false;
                 TcProblem& p = P.p[P.count - 1];
-                p.bias = s.param + s.b_off[ni][l]; p.bias_n = s.out[ni][l];
+                p.bias = e->bias_pad[ni][l]; p.bias_n = e->pw[ni][l];
                 p.out16 = act_buffers ? e->h_act[ni][l] : e->h[ni][l]; p.ld_out = e->pw[ni][l];
             }
             finish_params(P, alpha, e->error_dev);
