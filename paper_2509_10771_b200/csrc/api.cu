@@ -128,7 +128,7 @@ void build_net(Net& n, int in_dim, const int32_t* hidden, int nh, int out_dim, s
         L.b_off = dev_off; dev_off += L.out_p;
         L.w_flat = flat_off; flat_off += (size_t)L.in * L.out;
         L.b_flat = flat_off; flat_off += L.out;
-        n.hid_ld[l] = L.out_p;
+        n.hid_ld[l] = round_up(L.out, 8);      // activation rows are walked in 32-byte pieces
         in = L.out;
     }
 }

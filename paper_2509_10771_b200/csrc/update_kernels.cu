@@ -12,8 +12,9 @@ namespace {
 constexpr float kHalfLog2Pi = 0.91893853320467274178f;
 
 // =======================================================================================
-// Gather.  One warp per minibatch row: the warp resolves the source transition through the
-// Feistel shuffle, then streams the row (float4 per lane) into the minibatch buffers.
+// Gather.  A block takes 32 minibatch rows: one warp resolves their source transitions through
+// the Feistel shuffle (one row per lane), then all warps stream the rows into the minibatch
+// buffers.
 // =======================================================================================
 template <bool BF16>
 __device__ __forceinline__ void copy_obs_row(const float* __restrict__ src, int dim, int ld_src,
@@ -44,48 +45,65 @@ __device__ __forceinline__ void copy_obs_row(const float* __restrict__ src, int 
     }
 }
 
+constexpr int kGatherRows = 32;      // minibatch rows per block
+
 template <bool BF16>
 __global__ void __launch_bounds__(256) gather_kernel(const GatherArgs a) {
-    const int lane = threadIdx.x & 31;
-    const int warps = (gridDim.x * blockDim.x) >> 5;
+    __shared__ uint32_t s_src[kGatherRows];
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
     PermKey pk{a.seed_lo, a.seed_hi, a.iteration, a.epoch, a.batch, feistel_half_bits(a.batch)};
-    for (int j = (blockIdx.x * blockDim.x + threadIdx.x) >> 5; j < a.Bmb; j += warps) {
-        const uint32_t src = feistel_permute(pk, a.first + (uint32_t)j);
-        const int t = (int)(src / (uint32_t)a.N);
-        if (lane == 0) {
-            if (a.rows_out) a.rows_out[j] = (int)src;
-            a.logp_old[j] = a.logp[src];
-            a.v_old[j] = a.values[src];
-            a.ret[j] = a.returns[src];
-            a.adv_mb[j] = a.adv[src];
+    for (int j0 = blockIdx.x * kGatherRows; j0 < a.Bmb; j0 += gridDim.x * kGatherRows) {
+        // Phase 1: warp 0 resolves the source transition of the block's rows, one row per lane
+        // (the shuffle costs a few hundred integer instructions: once per row, not per lane),
+        // and moves the per-row scalars.
+        if (warp == 0) {
+            const int jm = j0 + lane;
+            if (jm < a.Bmb) {
+                const uint32_t src = feistel_permute(pk, a.first + (uint32_t)jm);
+                s_src[lane] = src;
+                if (a.rows_out) a.rows_out[jm] = (int)src;
+                a.logp_old[jm] = a.logp[src];
+                a.v_old[jm] = a.values[src];
+                a.ret[jm] = a.returns[src];
+                a.adv_mb[jm] = a.adv[src];
+            }
         }
-        const float* oa = a.obs_a + (size_t)src * a.sa;
-        const int ldxa = BF16 ? a.ldxa16 : a.ldxa;
-        copy_obs_row<BF16>(oa, a.Da, a.sa, a.x_a ? a.x_a + (size_t)j * ldxa : nullptr,
-                           a.x_a16 ? a.x_a16 + (size_t)j * ldxa : nullptr, ldxa, nullptr, nullptr, lane);
-        if (a.sym)
-            copy_obs_row<BF16>(oa, a.Da, a.sa, a.x_a ? a.x_a + (size_t)(j + a.Bmb) * ldxa : nullptr,
-                               a.x_a16 ? a.x_a16 + (size_t)(j + a.Bmb) * ldxa : nullptr, ldxa,
-                               a.st.obs_perm, a.st.obs_sign, lane);
-        if (!a.shared_obs) {
-            const float* oc = a.obs_c + (size_t)src * a.sc;
-            const int ldxc = BF16 ? a.ldxc16 : a.ldxc;
-            copy_obs_row<BF16>(oc, a.Dc, a.sc, a.x_c ? a.x_c + (size_t)j * ldxc : nullptr,
-                               a.x_c16 ? a.x_c16 + (size_t)j * ldxc : nullptr, ldxc, nullptr, nullptr, lane);
+        __syncthreads();
+        // Phase 2: each warp streams its share of the rows (float4 per lane).
+        const int nrows = min(kGatherRows, a.Bmb - j0);
+        for (int rr = warp; rr < nrows; rr += 8) {
+            const int j = j0 + rr;
+            const uint32_t src = s_src[rr];
+            const int t = (int)(src / (uint32_t)a.N);
+            const float* oa = a.obs_a + (size_t)src * a.sa;
+            const int ldxa = BF16 ? a.ldxa16 : a.ldxa;
+            copy_obs_row<BF16>(oa, a.Da, a.sa, a.x_a ? a.x_a + (size_t)j * ldxa : nullptr,
+                               a.x_a16 ? a.x_a16 + (size_t)j * ldxa : nullptr, ldxa, nullptr, nullptr, lane);
             if (a.sym)
-                copy_obs_row<BF16>(oc, a.Dc, a.sc, a.x_c ? a.x_c + (size_t)(j + a.Bmb) * ldxc : nullptr,
-                                   a.x_c16 ? a.x_c16 + (size_t)(j + a.Bmb) * ldxc : nullptr, ldxc,
-                                   a.st.cobs_perm, a.st.cobs_sign, lane);
+                copy_obs_row<BF16>(oa, a.Da, a.sa, a.x_a ? a.x_a + (size_t)(j + a.Bmb) * ldxa : nullptr,
+                                   a.x_a16 ? a.x_a16 + (size_t)(j + a.Bmb) * ldxa : nullptr, ldxa,
+                                   a.st.obs_perm, a.st.obs_sign, lane);
+            if (!a.shared_obs) {
+                const float* oc = a.obs_c + (size_t)src * a.sc;
+                const int ldxc = BF16 ? a.ldxc16 : a.ldxc;
+                copy_obs_row<BF16>(oc, a.Dc, a.sc, a.x_c ? a.x_c + (size_t)j * ldxc : nullptr,
+                                   a.x_c16 ? a.x_c16 + (size_t)j * ldxc : nullptr, ldxc, nullptr, nullptr, lane);
+                if (a.sym)
+                    copy_obs_row<BF16>(oc, a.Dc, a.sc, a.x_c ? a.x_c + (size_t)(j + a.Bmb) * ldxc : nullptr,
+                                       a.x_c16 ? a.x_c16 + (size_t)(j + a.Bmb) * ldxc : nullptr, ldxc,
+                                       a.st.cobs_perm, a.st.cobs_sign, lane);
+            }
+            const float* act = a.actions + (size_t)src * a.as;
+            for (int c = lane; c < a.as; c += 32) {
+                a.act_mb[(size_t)j * a.as + c] = act[c];
+                a.mu_old[(size_t)j * a.as + c] = a.mu[(size_t)src * a.as + c];
+                a.sigma_old[(size_t)j * a.as + c] = a.sigma[(size_t)t * a.as + c];
+                if (a.sym)
+                    a.act_mb[(size_t)(j + a.Bmb) * a.as + c] =
+                        c < a.A ? a.st.act_sign[c] * act[a.st.act_perm[c]] : 0.f;
+            }
         }
-        const float* act = a.actions + (size_t)src * a.as;
-        for (int c = lane; c < a.as; c += 32) {
-            a.act_mb[(size_t)j * a.as + c] = act[c];
-            a.mu_old[(size_t)j * a.as + c] = a.mu[(size_t)src * a.as + c];
-            a.sigma_old[(size_t)j * a.as + c] = a.sigma[(size_t)t * a.as + c];
-            if (a.sym)
-                a.act_mb[(size_t)(j + a.Bmb) * a.as + c] =
-                    c < a.A ? a.st.act_sign[c] * act[a.st.act_perm[c]] : 0.f;
-        }
+        __syncthreads();
     }
 }
 
@@ -95,143 +113,153 @@ __global__ void perm_rows_kernel(PermKey pk, uint32_t first, int count, int* __r
 }
 
 // =======================================================================================
-// Head + loss.  One warp per minibatch row (and its mirrored twin).  Lane i owns action i
-// (and i + 32): policy mean, log-density terms, dL/dmu.  The hidden row is read coalesced.
+// Head + loss.  One thread per minibatch row (and its mirrored twin): the thread walks the row
+// of last-hidden activations in 16-byte pieces against head weights broadcast from shared
+// memory, finishes the PPO loss terms of the row, and walks the row again to emit dL/dz of the
+// last hidden layers.  No cross-lane traffic until the block-level sums at the end.
+// NP = number of 16-action passes (actions are padded to 16 * NP in registers).
 // =======================================================================================
-constexpr int kHLThreads = 256;
-constexpr int kHLWarps = kHLThreads / 32;
+constexpr int kHLThreads = 128;
 constexpr int kPartialStride = 8 + 2 * kMaxActions;   // [0..3] loss sums, [4] db_critic, [8..) db_actor, dlog_std
 
-template <typename T>
-__device__ __forceinline__ void head_fwd(const T* __restrict__ h, int n, const float* __restrict__ Ws,
-                                         int ldws, const float* __restrict__ bias, int nout,
-                                         float& out_lo, float& out_hi) {
-    const int lane = threadIdx.x & 31;
-    out_lo = 0.f; out_hi = 0.f;
-    for (int o0 = 0; o0 < nout; o0 += 8) {
-        float acc[8];
+__device__ __forceinline__ void load8(const float* p, float (&h)[8]) {
+    const float4 a = *reinterpret_cast<const float4*>(p), b = *reinterpret_cast<const float4*>(p + 4);
+    h[0] = a.x; h[1] = a.y; h[2] = a.z; h[3] = a.w; h[4] = b.x; h[5] = b.y; h[6] = b.z; h[7] = b.w;
+}
+__device__ __forceinline__ void load8(const __nv_bfloat16* p, float (&h)[8]) {
+    const uint4 v = *reinterpret_cast<const uint4*>(p);
+    const uint32_t w[4] = {v.x, v.y, v.z, v.w};
 #pragma unroll
-        for (int q = 0; q < 8; ++q) acc[q] = 0.f;
-        for (int k = lane; k < n; k += 32) {
-            const float hv = to_float(h[k]);
-            const float* w = Ws + k * ldws + o0;
-#pragma unroll
-            for (int q = 0; q < 8; ++q)
-                if (o0 + q < nout) acc[q] = fmaf(hv, w[q], acc[q]);
-        }
-#pragma unroll
-        for (int q = 0; q < 8; ++q) {
-            const int o = o0 + q;
-            if (o < nout) {
-                const float val = warp_sum(acc[q]) + bias[o];
-                if (lane == (o & 31)) { if (o < 32) out_lo = val; else out_hi = val; }
-            }
-        }
+    for (int e = 0; e < 4; ++e) {
+        const __nv_bfloat162 h2 = *reinterpret_cast<const __nv_bfloat162*>(&w[e]);
+        h[2 * e] = __low2float(h2); h[2 * e + 1] = __high2float(h2);
     }
 }
-
-// dZ[k] = ELU'(h[k]) * sum_i d_i W[k][i] for the lane's k = lane, lane+32, ...
-template <typename T>
-__device__ __forceinline__ void head_bwd(const T* __restrict__ h, int n, const float* __restrict__ Ws,
-                                         int ldws, int nout, float d_lo, float d_hi, float alpha,
-                                         T* __restrict__ dz, int ld_out_pad) {
-    const int lane = threadIdx.x & 31;
-    for (int k0 = 0; k0 < ld_out_pad; k0 += 128) {
-        float acc[4] = {0.f, 0.f, 0.f, 0.f};
-        for (int i = 0; i < nout; ++i) {
-            const float d = __shfl_sync(0xffffffffu, i < 32 ? d_lo : d_hi, i & 31);
+__device__ __forceinline__ void store8(float* p, const float (&v)[8]) {
+    *reinterpret_cast<float4*>(p) = make_float4(v[0], v[1], v[2], v[3]);
+    *reinterpret_cast<float4*>(p + 4) = make_float4(v[4], v[5], v[6], v[7]);
+}
+__device__ __forceinline__ void store8(__nv_bfloat16* p, const float (&v)[8]) {
+    uint32_t w[4];
 #pragma unroll
-            for (int q = 0; q < 4; ++q) {
-                const int k = k0 + lane + 32 * q;
-                if (k < n) acc[q] = fmaf(d, Ws[k * ldws + i], acc[q]);
-            }
-        }
-#pragma unroll
-        for (int q = 0; q < 4; ++q) {
-            const int k = k0 + lane + 32 * q;
-            if (k < ld_out_pad) {
-                float v = 0.f;
-                if (k < n) v = acc[q] * elu_grad_from_h(to_float(h[k]), alpha);
-                dz[k] = from_float<T>(v);
-            }
-        }
+    for (int e = 0; e < 4; ++e) {
+        __nv_bfloat162 h2 = __floats2bfloat162_rn(v[2 * e], v[2 * e + 1]);
+        w[e] = *reinterpret_cast<uint32_t*>(&h2);
     }
+    *reinterpret_cast<uint4*>(p) = make_uint4(w[0], w[1], w[2], w[3]);
 }
 
-template <typename T>
+// Block-wide sum in a fixed order: shuffle tree inside each warp, then warp 0 adds the warps.
+__device__ __forceinline__ float block_sum(float v, float* scratch /* [warps] */) {
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) v += __shfl_down_sync(0xffffffffu, v, o);
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    __syncthreads();
+    if (lane == 0) scratch[warp] = v;
+    __syncthreads();
+    float t = 0.f;
+    for (int w = 0; w < kHLThreads / 32; ++w) t += scratch[w];
+    return t;
+}
+
+template <typename T, int NP>
 __global__ void __launch_bounds__(kHLThreads) head_loss_kernel(const HeadLossArgs a) {
+    constexpr int AP = 16 * NP;
     extern __shared__ float smem[];
     const HeadParams& hp = a.hp;
-    const int ldwa_s = hp.ldwa + 1, ldwc_s = 2;       // odd / tiny strides: no bank conflicts
-    float* Wa_s = smem;                                // [n_a][ldwa_s]
-    float* Wc_s = Wa_s + hp.n_a * ldwa_s;              // [n_c][2]
-    float* red = Wc_s + hp.n_c * ldwc_s;               // [kHLWarps][kPartialStride]
-    for (int e = threadIdx.x; e < hp.n_a * hp.ldwa; e += kHLThreads) {
-        const int k = e / hp.ldwa, i = e % hp.ldwa;
-        Wa_s[k * ldwa_s + i] = hp.Wa[e];
+    const int A = hp.A;
+    float* Wa_s = smem;                                 // [n_a][AP], zero padded
+    float* Wc_s = Wa_s + hp.n_a * AP;                   // [n_c]
+    float* mu_s = Wc_s + ((hp.n_c + 3) & ~3);           // [threads][AP + 1]  policy mean of the original row
+    float* red = mu_s + kHLThreads * (AP + 1);          // [warps]
+    for (int e = threadIdx.x; e < hp.n_a * AP; e += kHLThreads) {
+        const int k = e / AP, i = e % AP;
+        Wa_s[e] = i < A ? hp.Wa[(size_t)k * hp.ldwa + i] : 0.f;
     }
-    for (int k = threadIdx.x; k < hp.n_c; k += kHLThreads) Wc_s[k * ldwc_s] = hp.Wc[(size_t)k * hp.ldwc];
+    for (int k = threadIdx.x; k < hp.n_c; k += kHLThreads) Wc_s[k] = hp.Wc[(size_t)k * hp.ldwc];
     __syncthreads();
 
-    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
-    const int A = hp.A;
+    const int j = blockIdx.x * kHLThreads + threadIdx.x;
+    const bool live = j < a.Bmb;
     const int R = a.sym ? 2 * a.Bmb : a.Bmb;
     const float inv_R = 1.0f / (float)R;
     const float inv_sym = 1.0f / ((float)a.Bmb * (float)A);
-    // per-lane constants of actions i = lane, lane + 32
-    float ls[2], inv_var[2];
-    int aperm[2]; float asign[2];
-#pragma unroll
-    for (int hf = 0; hf < 2; ++hf) {
-        const int i = lane + 32 * hf;
-        ls[hf] = i < A ? hp.log_std[i] : 0.f;
-        const float sg = expf(ls[hf]);
-        inv_var[hf] = 1.0f / (sg * sg);
-        aperm[hf] = (a.sym && i < A) ? a.act_perm[i] : i;
-        asign[hf] = (a.sym && i < A) ? a.act_sign[i] : 1.f;
-    }
     float s_surr = 0.f, s_val = 0.f, s_kl = 0.f, s_sym = 0.f, s_dbc = 0.f;
-    float s_dba[2] = {0.f, 0.f}, s_dls[2] = {0.f, 0.f};
+    float s_dba[AP], s_dls[AP];
+#pragma unroll
+    for (int i = 0; i < AP; ++i) { s_dba[i] = 0.f; s_dls[i] = 0.f; }
 
-    const int warps_total = gridDim.x * kHLWarps;
-    for (int j = blockIdx.x * kHLWarps + warp; j < a.Bmb; j += warps_total) {
+    if (live) {
         const float logp_old = a.logp_old[j], v_old = a.v_old[j], ret = a.ret[j], adv = a.adv[j];
-        float mu_orig[2] = {0.f, 0.f};
+        float* mu_mine = mu_s + threadIdx.x * (AP + 1);
         for (int copy = 0; copy < (a.sym ? 2 : 1); ++copy) {
             const int r = j + copy * a.Bmb;
             const T* ha = reinterpret_cast<const T*>(a.Ha) + (size_t)r * a.ldha;
             const T* hc = reinterpret_cast<const T*>(a.Hc) + (size_t)r * a.ldhc;
-            float mu[2], v, unused;
-            head_fwd(ha, hp.n_a, Wa_s, ldwa_s, hp.ba, A, mu[0], mu[1]);
-            head_fwd(hc, hp.n_c, Wc_s, ldwc_s, hp.bc, 1, v, unused);
-            v = __shfl_sync(0xffffffffu, v, 0);
-            // ---- log-density, KL -------------------------------------------------------
-            float act[2], lp = 0.f, kl = 0.f;
+            // ---- heads ------------------------------------------------------------------
+            float mu[AP];
 #pragma unroll
-            for (int hf = 0; hf < 2; ++hf) {
-                const int i = lane + 32 * hf;
-                act[hf] = 0.f;
-                if (i < A) {
-                    act[hf] = a.act_mb[(size_t)r * a.as + i];
-                    const float d = act[hf] - mu[hf];
-                    lp += -(d * d) * 0.5f * inv_var[hf] - ls[hf] - kHalfLog2Pi;
-                    if (copy == 0) {
-                        const float so = a.sigma_old[(size_t)j * a.as + i];
-                        const float dm = a.mu_old[(size_t)j * a.as + i] - mu[hf];
-                        kl += (ls[hf] - logf(so)) + (so * so + dm * dm) * 0.5f * inv_var[hf] - 0.5f;
+            for (int i = 0; i < AP; ++i) mu[i] = i < A ? hp.ba[i] : 0.f;
+            for (int k0 = 0; k0 < hp.n_a; k0 += 8) {       // row strides are multiples of 8
+                float h[8];
+                load8(ha + k0, h);
+#pragma unroll
+                for (int kk = 0; kk < 8; ++kk) {
+                    if (k0 + kk < hp.n_a) {
+                        const float4* w4 = reinterpret_cast<const float4*>(Wa_s + (k0 + kk) * AP);
+#pragma unroll
+                        for (int i4 = 0; i4 < AP / 4; ++i4) {
+                            const float4 w = w4[i4];
+                            mu[4 * i4] = fmaf(h[kk], w.x, mu[4 * i4]); mu[4 * i4 + 1] = fmaf(h[kk], w.y, mu[4 * i4 + 1]);
+                            mu[4 * i4 + 2] = fmaf(h[kk], w.z, mu[4 * i4 + 2]); mu[4 * i4 + 3] = fmaf(h[kk], w.w, mu[4 * i4 + 3]);
+                        }
                     }
                 }
             }
-            lp = warp_sum(lp);
-            if (copy == 0) s_kl += warp_sum(kl);
-            // ---- surrogate ------------------------------------------------------------
+            float v = hp.bc[0];
+            {
+                float v1 = 0.f, v2 = 0.f, v3 = 0.f;
+                for (int k0 = 0; k0 < hp.n_c; k0 += 8) {
+                    float h[8];
+                    load8(hc + k0, h);
+#pragma unroll
+                    for (int kk = 0; kk < 8; kk += 4) {
+                        if (k0 + kk < hp.n_c) v = fmaf(h[kk], Wc_s[k0 + kk], v);
+                        if (k0 + kk + 1 < hp.n_c) v1 = fmaf(h[kk + 1], Wc_s[k0 + kk + 1], v1);
+                        if (k0 + kk + 2 < hp.n_c) v2 = fmaf(h[kk + 2], Wc_s[k0 + kk + 2], v2);
+                        if (k0 + kk + 3 < hp.n_c) v3 = fmaf(h[kk + 3], Wc_s[k0 + kk + 3], v3);
+                    }
+                }
+                v += (v1 + v2) + v3;
+            }
+            // ---- log-density, KL ---------------------------------------------------------
+            float dmu[AP];
+            float lp = 0.f, kl = 0.f;
+#pragma unroll
+            for (int i = 0; i < AP; ++i) {
+                dmu[i] = 0.f;
+                if (i < A) {
+                    const float ls = hp.log_std[i];
+                    const float iv = __expf(-2.0f * ls);              // 1 / sigma^2
+                    const float d = a.act_mb[(size_t)r * a.as + i] - mu[i];
+                    lp += -(d * d) * 0.5f * iv - ls - kHalfLog2Pi;
+                    dmu[i] = d * iv;                                    // d logp / d mu_i
+                    if (copy == 0) {
+                        const float so = a.sigma_old[(size_t)j * a.as + i];
+                        const float dm = a.mu_old[(size_t)j * a.as + i] - mu[i];
+                        kl += (ls - logf(so)) + (so * so + dm * dm) * 0.5f * iv - 0.5f;
+                    }
+                }
+            }
+            if (copy == 0) s_kl += kl;
+            // ---- surrogate ---------------------------------------------------------------
             const float ratio = expf(lp - logp_old);
             const float s1 = -adv * ratio;
             const float s2 = -adv * fminf(fmaxf(ratio, 1.0f - a.h.clip), 1.0f + a.h.clip);
             s_surr += fmaxf(s1, s2);
             const bool inside = ratio >= 1.0f - a.h.clip && ratio <= 1.0f + a.h.clip;
             const float dlogp = (inside || s1 > s2) ? s1 * inv_R : 0.f;
-            // ---- value ----------------------------------------------------------------
+            // ---- value -------------------------------------------------------------------
             float dv;
             const float e1 = (v - ret) * (v - ret);
             if (a.h.use_clipped_value_loss) {
@@ -245,65 +273,104 @@ __global__ void __launch_bounds__(kHLThreads) head_loss_kernel(const HeadLossArg
                 dv = 2.0f * (v - ret);
             }
             dv *= a.h.value_coef * inv_R;
-            // ---- dL/dmu, dL/dlog_std, symmetry -----------------------------------------
-            float dmu[2];
-#pragma unroll
-            for (int hf = 0; hf < 2; ++hf) {
-                const int i = lane + 32 * hf;
-                dmu[hf] = 0.f;
-                float tgt_src = 0.f;
-                if (copy == 1) {
-                    // target_i = sign_i * mu_orig[perm_i]; every lane takes part in the shuffle
-                    const int p = aperm[hf];
-                    const float lo = __shfl_sync(0xffffffffu, mu_orig[0], p & 31);
-                    const float hi = __shfl_sync(0xffffffffu, mu_orig[1], p & 31);
-                    tgt_src = p < 32 ? lo : hi;
-                }
-                if (i < A) {
-                    const float d = act[hf] - mu[hf];
-                    dmu[hf] = dlogp * d * inv_var[hf];
-                    s_dls[hf] += dlogp * (d * d * inv_var[hf] - 1.0f);
-                    if (copy == 1) {
-                        const float diff = mu[hf] - asign[hf] * tgt_src;
-                        s_sym += diff * diff;            // summed over lanes at the end
-                        dmu[hf] += a.h.sym_coef * 2.0f * diff * inv_sym;
-                    }
-                    s_dba[hf] += dmu[hf];
-                }
-            }
-            if (copy == 0) { mu_orig[0] = mu[0]; mu_orig[1] = mu[1]; }
             s_dbc += dv;
-            // ---- outputs ---------------------------------------------------------------
-            for (int hf = 0; hf < 2; ++hf) {
-                const int i = lane + 32 * hf;
-                if (i < a.lddmu) a.dmu[(size_t)r * a.lddmu + i] = dmu[hf];
-                if (a.dmu16 && i < a.lddmu16) a.dmu16[(size_t)r * a.lddmu16 + i] = __float2bfloat16_rn(dmu[hf]);
-                if (a.mu_out && i < a.as) a.mu_out[(size_t)r * a.as + i] = mu[hf];
+            // ---- dL/dmu, dL/dlog_std, symmetry -------------------------------------------
+#pragma unroll
+            for (int i = 0; i < AP; ++i) {
+                if (i < A) {
+                    const float ls = hp.log_std[i];
+                    const float var = __expf(2.0f * ls);
+                    const float dlp_dmu = dmu[i];                       // (a - mu) / sigma^2
+                    s_dls[i] += dlogp * (dlp_dmu * dlp_dmu * var - 1.0f);
+                    float g = dlogp * dlp_dmu;
+                    if (copy == 1) {
+                        const float diff = mu[i] - a.act_sign[i] * mu_mine[a.act_perm[i]];
+                        s_sym += diff * diff;
+                        g += a.h.sym_coef * 2.0f * diff * inv_sym;
+                    }
+                    dmu[i] = g;
+                    s_dba[i] += g;
+                }
             }
-            if (lane < 4) a.dv[(size_t)r * 4 + lane] = lane == 0 ? dv : 0.f;
-            if (a.dv16 && lane < a.lddv16) a.dv16[(size_t)r * a.lddv16 + lane] = __float2bfloat16_rn(lane == 0 ? dv : 0.f);
-            if (a.v_out && lane == 0) a.v_out[r] = v;
-            head_bwd(ha, hp.n_a, Wa_s, ldwa_s, A, dmu[0], dmu[1], a.h.alpha,
-                     reinterpret_cast<T*>(a.dZa) + (size_t)r * a.lddza, a.lddza);
-            head_bwd(hc, hp.n_c, Wc_s, ldwc_s, 1, dv, 0.f, a.h.alpha,
-                     reinterpret_cast<T*>(a.dZc) + (size_t)r * a.lddzc, a.lddzc);
+            if (copy == 0 && a.sym) {
+#pragma unroll
+                for (int i = 0; i < AP; ++i) mu_mine[i] = mu[i];
+            }
+            // ---- outputs -------------------------------------------------------------------
+            for (int i = 0; i < a.lddmu; i += 4) {
+                float4 o;
+                o.x = dmu[0]; o.y = 0.f; o.z = 0.f; o.w = 0.f;
+#pragma unroll
+                for (int q = 0; q < AP; q += 4)
+                    if (q == i) o = make_float4(dmu[q], dmu[q + 1], dmu[q + 2], dmu[q + 3]);
+                *reinterpret_cast<float4*>(a.dmu + (size_t)r * a.lddmu + i) = o;
+            }
+            *reinterpret_cast<float4*>(a.dv + (size_t)r * 4) = make_float4(dv, 0.f, 0.f, 0.f);
+            if (a.dmu16) {
+#pragma unroll
+                for (int q = 0; q < AP; q += 8) {
+                    if (q < a.lddmu16) {
+                        const float o8[8] = {dmu[q], dmu[q + 1], dmu[q + 2], dmu[q + 3], dmu[q + 4], dmu[q + 5], dmu[q + 6], dmu[q + 7]};
+                        store8(a.dmu16 + (size_t)r * a.lddmu16 + q, o8);
+                    }
+                }
+                const float d8[8] = {dv, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f};
+                store8(a.dv16 + (size_t)r * a.lddv16, d8);
+            }
+            if (a.mu_out) for (int i = 0; i < A; ++i) {
+                float m = 0.f;
+#pragma unroll
+                for (int q = 0; q < AP; ++q) if (q == i) m = mu[q];
+                a.mu_out[(size_t)r * a.as + i] = m;
+            }
+            if (a.v_out) a.v_out[r] = v;
+            // ---- dL/dz of the last hidden layers --------------------------------------------
+            T* dza = reinterpret_cast<T*>(a.dZa) + (size_t)r * a.lddza;
+            for (int k0 = 0; k0 < a.lddza; k0 += 8) {
+                float h[8], o[8];
+                if (k0 < hp.n_a) load8(ha + k0, h);
+#pragma unroll
+                for (int kk = 0; kk < 8; ++kk) {
+                    float acc = 0.f;
+                    if (k0 + kk < hp.n_a) {
+                        const float4* w4 = reinterpret_cast<const float4*>(Wa_s + (k0 + kk) * AP);
+#pragma unroll
+                        for (int i4 = 0; i4 < AP / 4; ++i4) {
+                            const float4 w = w4[i4];
+                            acc = fmaf(dmu[4 * i4], w.x, acc); acc = fmaf(dmu[4 * i4 + 1], w.y, acc);
+                            acc = fmaf(dmu[4 * i4 + 2], w.z, acc); acc = fmaf(dmu[4 * i4 + 3], w.w, acc);
+                        }
+                        acc *= elu_grad_from_h(h[kk], a.h.alpha);
+                    }
+                    o[kk] = acc;
+                }
+                store8(dza + k0, o);
+            }
+            T* dzc = reinterpret_cast<T*>(a.dZc) + (size_t)r * a.lddzc;
+            for (int k0 = 0; k0 < a.lddzc; k0 += 8) {
+                float h[8], o[8];
+                if (k0 < hp.n_c) load8(hc + k0, h);
+#pragma unroll
+                for (int kk = 0; kk < 8; ++kk)
+                    o[kk] = k0 + kk < hp.n_c ? dv * Wc_s[k0 + kk] * elu_grad_from_h(h[kk], a.h.alpha) : 0.f;
+                store8(dzc + k0, o);
+            }
         }
     }
-    // ---- block partials (fixed order over the warps) --------------------------------------
-    s_sym = warp_sum(s_sym);
-    float* my = red + warp * kPartialStride;
-    if (lane == 0) {
-        my[LS_SURR] = s_surr; my[LS_VALUE] = s_val; my[LS_KL] = s_kl; my[LS_SYM] = s_sym;
-        my[4] = s_dbc;
-    }
-    my[8 + lane] = s_dba[0]; my[8 + 32 + lane] = s_dba[1];
-    my[8 + kMaxActions + lane] = s_dls[0]; my[8 + kMaxActions + 32 + lane] = s_dls[1];
-    __syncthreads();
-    for (int e = threadIdx.x; e < kPartialStride; e += kHLThreads) {
-        if (e >= 5 && e < 8) continue;
-        float s = 0.f;
-        for (int w = 0; w < kHLWarps; ++w) s += red[w * kPartialStride + e];
-        a.block_partials[(size_t)blockIdx.x * kPartialStride + e] = s;
+    // ---- block partials (fixed order) ----------------------------------------------------------
+    float* out = a.block_partials + (size_t)blockIdx.x * kPartialStride;
+    float t;
+    t = block_sum(s_surr, red); if (threadIdx.x == 0) out[LS_SURR] = t;
+    t = block_sum(s_val, red);  if (threadIdx.x == 0) out[LS_VALUE] = t;
+    t = block_sum(s_kl, red);   if (threadIdx.x == 0) out[LS_KL] = t;
+    t = block_sum(s_sym, red);  if (threadIdx.x == 0) out[LS_SYM] = t;
+    t = block_sum(s_dbc, red);  if (threadIdx.x == 0) out[4] = t;
+#pragma unroll
+    for (int i = 0; i < AP; ++i) {
+        if (i < A) {                                    // uniform across the block
+            t = block_sum(s_dba[i], red); if (threadIdx.x == 0) out[8 + i] = t;
+            t = block_sum(s_dls[i], red); if (threadIdx.x == 0) out[8 + kMaxActions + i] = t;
+        }
     }
 }
 
@@ -459,25 +526,35 @@ cudaError_t launch_perm_rows(uint64_t seed, uint32_t iteration, uint32_t epoch, 
     return cudaGetLastError();
 }
 
-int head_loss_blocks(int Bmb) { return std::max(1, std::min((Bmb + kHLWarps - 1) / kHLWarps, 148 * 4)); }
+int head_loss_blocks(int Bmb) { return std::max(1, (Bmb + kHLThreads - 1) / kHLThreads); }
 int head_partial_stride() { return kPartialStride; }
 
-cudaError_t launch_head_loss(const HeadLossArgs& a, cudaStream_t s) {
-    const int blocks = head_loss_blocks(a.Bmb);
-    const size_t smem = sizeof(float) * ((size_t)a.hp.n_a * (a.hp.ldwa + 1) + (size_t)a.hp.n_c * 2 +
-                                         (size_t)kHLWarps * kPartialStride);
+namespace {
+template <typename T, int NP>
+cudaError_t launch_head_loss_t(const HeadLossArgs& a, cudaStream_t s) {
+    const int AP = 16 * NP;
+    const size_t smem = sizeof(float) * ((size_t)a.hp.n_a * AP + ((a.hp.n_c + 3) & ~3) + (size_t)kHLThreads * (AP + 1) +
+                                         kHLThreads / 32);
+    cudaError_t e = cudaFuncSetAttribute(head_loss_kernel<T, NP>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+    if (e != cudaSuccess) return e;
     LaunchScope scope_("head_loss", s);
-    cudaError_t e;
-    if (a.bf16_act) {
-        e = cudaFuncSetAttribute(head_loss_kernel<__nv_bfloat16>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
-        if (e != cudaSuccess) return e;
-        head_loss_kernel<__nv_bfloat16><<<blocks, kHLThreads, smem, s>>>(a);
-    } else {
-        e = cudaFuncSetAttribute(head_loss_kernel<float>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
-        if (e != cudaSuccess) return e;
-        head_loss_kernel<float><<<blocks, kHLThreads, smem, s>>>(a);
-    }
+    head_loss_kernel<T, NP><<<head_loss_blocks(a.Bmb), kHLThreads, smem, s>>>(a);
     return cudaGetLastError();
+}
+template <typename T>
+cudaError_t launch_head_loss_np(const HeadLossArgs& a, cudaStream_t s) {
+    const int np = (a.hp.A + 15) / 16;
+    if (np == 1) return launch_head_loss_t<T, 1>(a, s);
+    if (np == 2) return launch_head_loss_t<T, 2>(a, s);
+    if (np == 3) return launch_head_loss_t<T, 3>(a, s);
+    return launch_head_loss_t<T, 4>(a, s);
+}
+}  // namespace
+
+cudaError_t launch_head_loss(const HeadLossArgs& a, cudaStream_t s) {
+    // row strides of the hidden activations must allow 16-byte pieces
+    if ((a.ldha % 8) || (a.ldhc % 8) || (a.lddza % 8) || (a.lddzc % 8)) return cudaErrorInvalidValue;
+    return a.bf16_act ? launch_head_loss_np<__nv_bfloat16>(a, s) : launch_head_loss_np<float>(a, s);
 }
 
 cudaError_t launch_head_finalize(const float* block_partials, int nblocks, float* partials0, int off_ba,
