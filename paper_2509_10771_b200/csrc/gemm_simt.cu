@@ -228,52 +228,54 @@ cudaError_t launch_sgemm(const GemmBatch& b, bool ta, bool tb, int epi, cudaStre
 }
 
 // ---------------------------------------------------------------------------------------
-// Column sums over a split of the rows (bias gradients).  grid = (ceil(n/32), splits, count);
-// a block of 1024 threads covers 32 columns (16 column pairs) with 64 row lanes, so that the
+// Column sums over a split of the rows (bias gradients).  grid = (ceil(n/64), splits, count);
+// a block of 1024 threads covers 64 columns (16 column quads) with 64 row lanes, so that the
 // whole machine is busy even when there are only a few splits.  The 64 row-lane partials of a
 // column are added in a fixed order: the result does not depend on scheduling.
 // ---------------------------------------------------------------------------------------
 namespace {
-constexpr int kCsPairs = 16, kCsLanes = 64;
+constexpr int kCsQuads = 16, kCsLanes = 64, kCsCols = 4 * kCsQuads;
 
-__device__ __forceinline__ float2 load_pair(const float* p) { return *reinterpret_cast<const float2*>(p); }
-__device__ __forceinline__ float2 load_pair(const __nv_bfloat16* p) {
-    return __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162*>(p));
+__device__ __forceinline__ float4 load_quad(const float* p) { return *reinterpret_cast<const float4*>(p); }
+__device__ __forceinline__ float4 load_quad(const __nv_bfloat16* p) {
+    const uint2 v = *reinterpret_cast<const uint2*>(p);
+    const float2 a = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162*>(&v.x));
+    const float2 b = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162*>(&v.y));
+    return make_float4(a.x, a.y, b.x, b.y);
 }
+__device__ __forceinline__ void add4(float4& s, const float4 a) { s.x += a.x; s.y += a.y; s.z += a.z; s.w += a.w; }
 
 template <typename T>
-__global__ void __launch_bounds__(kCsPairs * kCsLanes) colsum_kernel(const ColsumBatch b) {
+__global__ void __launch_bounds__(kCsQuads * kCsLanes) colsum_kernel(const ColsumBatch b) {
     const ColsumProblem& p = b.p[blockIdx.z];
-    __shared__ float2 part[kCsLanes][kCsPairs];
-    const int pair = threadIdx.x % kCsPairs, rl = threadIdx.x / kCsPairs;
-    const int n = blockIdx.x * (2 * kCsPairs) + 2 * pair;      // leading dimensions are even
-    if (blockIdx.x * (2 * kCsPairs) >= p.n) return;
+    __shared__ float4 part[kCsLanes][kCsQuads];
+    if (blockIdx.x * kCsCols >= p.n) return;
+    const int quad = threadIdx.x % kCsQuads, rl = threadIdx.x / kCsQuads;
+    const int n = blockIdx.x * kCsCols + 4 * quad;             // leading dimensions are multiples of 4
     const int chunk = (p.rows + b.splits - 1) / b.splits;
     const int r0 = blockIdx.y * chunk, r1 = min(p.rows, r0 + chunk);
     const T* X = reinterpret_cast<const T*>(p.X);
-    float2 s0 = make_float2(0.f, 0.f), s1 = s0, s2 = s0, s3 = s0;
+    float4 s0 = make_float4(0.f, 0.f, 0.f, 0.f), s1 = s0, s2 = s0, s3 = s0;
     if (n < p.ld) {
         int r = r0 + rl;
         for (; r + 3 * kCsLanes < r1; r += 4 * kCsLanes) {
-            const float2 a0 = load_pair(X + (size_t)r * p.ld + n);
-            const float2 a1 = load_pair(X + (size_t)(r + kCsLanes) * p.ld + n);
-            const float2 a2 = load_pair(X + (size_t)(r + 2 * kCsLanes) * p.ld + n);
-            const float2 a3 = load_pair(X + (size_t)(r + 3 * kCsLanes) * p.ld + n);
-            s0.x += a0.x; s0.y += a0.y; s1.x += a1.x; s1.y += a1.y;
-            s2.x += a2.x; s2.y += a2.y; s3.x += a3.x; s3.y += a3.y;
+            const float4 a0 = load_quad(X + (size_t)r * p.ld + n);
+            const float4 a1 = load_quad(X + (size_t)(r + kCsLanes) * p.ld + n);
+            const float4 a2 = load_quad(X + (size_t)(r + 2 * kCsLanes) * p.ld + n);
+            const float4 a3 = load_quad(X + (size_t)(r + 3 * kCsLanes) * p.ld + n);
+            add4(s0, a0); add4(s1, a1); add4(s2, a2); add4(s3, a3);
         }
-        for (; r < r1; r += kCsLanes) {
-            const float2 a0 = load_pair(X + (size_t)r * p.ld + n);
-            s0.x += a0.x; s0.y += a0.y;
-        }
+        for (; r < r1; r += kCsLanes) add4(s0, load_quad(X + (size_t)r * p.ld + n));
     }
-    part[rl][pair] = make_float2((s0.x + s1.x) + (s2.x + s3.x), (s0.y + s1.y) + (s2.y + s3.y));
+    part[rl][quad] = make_float4((s0.x + s1.x) + (s2.x + s3.x), (s0.y + s1.y) + (s2.y + s3.y),
+                                 (s0.z + s1.z) + (s2.z + s3.z), (s0.w + s1.w) + (s2.w + s3.w));
     __syncthreads();
-    if (threadIdx.x < 2 * kCsPairs) {
+    if (threadIdx.x < kCsCols) {
         const int c = threadIdx.x;                 // column within the block
+        const float* flat = reinterpret_cast<const float*>(&part[0][0]);
         float t = 0.f;
-        for (int l = 0; l < kCsLanes; ++l) t += (c & 1) ? part[l][c >> 1].y : part[l][c >> 1].x;
-        const int col = blockIdx.x * (2 * kCsPairs) + c;
+        for (int l = 0; l < kCsLanes; ++l) t += flat[l * kCsCols + c];
+        const int col = blockIdx.x * kCsCols + c;
         if (col < p.n) p.out[(size_t)blockIdx.y * b.split_stride + col] = t;
     }
 }
@@ -283,10 +285,10 @@ cudaError_t launch_colsum(const ColsumBatch& b, cudaStream_t s) {
     if (b.count <= 0) return cudaSuccess;
     int nmax = 0;
     for (int i = 0; i < b.count; ++i) nmax = std::max(nmax, b.p[i].n);
-    dim3 grid((nmax + 2 * kCsPairs - 1) / (2 * kCsPairs), b.splits, b.count);
+    dim3 grid((nmax + kCsCols - 1) / kCsCols, b.splits, b.count);
     LaunchScope scope_("colsum", s);
-    if (b.is_bf16) colsum_kernel<__nv_bfloat16><<<grid, kCsPairs * kCsLanes, 0, s>>>(b);
-    else colsum_kernel<float><<<grid, kCsPairs * kCsLanes, 0, s>>>(b);
+    if (b.is_bf16) colsum_kernel<__nv_bfloat16><<<grid, kCsQuads * kCsLanes, 0, s>>>(b);
+    else colsum_kernel<float><<<grid, kCsQuads * kCsLanes, 0, s>>>(b);
     return cudaGetLastError();
 }
 

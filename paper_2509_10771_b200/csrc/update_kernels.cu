@@ -149,6 +149,39 @@ __device__ __forceinline__ void store8(__nv_bfloat16* p, const float (&v)[8]) {
     *reinterpret_cast<uint4*>(p) = make_uint4(w[0], w[1], w[2], w[3]);
 }
 
+// A block of kRowPieces consecutive 16-byte pieces of an activation row, fetched with all loads
+// in flight at once (the row walk is latency bound otherwise; longer blocks bloat the unrolled
+// code past the instruction cache).
+constexpr int kRowPieces = 4;
+template <typename T>
+struct RowBlock {
+    static constexpr int EPV = 16 / (int)sizeof(T);     // elements per piece
+    static constexpr int N = kRowPieces * EPV;          // elements per block
+    uint4 v[kRowPieces];
+    __device__ __forceinline__ void load(const T* row, int k0, int ld) {
+#pragma unroll
+        for (int i = 0; i < kRowPieces; ++i)
+            if (k0 + i * EPV < ld) v[i] = *reinterpret_cast<const uint4*>(row + k0 + i * EPV);
+    }
+    __device__ __forceinline__ void unpack(int i, float (&h)[EPV]) const {
+        if (sizeof(T) == 4) {
+            h[0] = __uint_as_float(v[i].x); h[1] = __uint_as_float(v[i].y);
+            h[2] = __uint_as_float(v[i].z); h[3] = __uint_as_float(v[i].w);
+        } else {
+            const uint32_t w[4] = {v[i].x, v[i].y, v[i].z, v[i].w};
+#pragma unroll
+            for (int e = 0; e < 4; ++e) {
+                const __nv_bfloat162 h2 = *reinterpret_cast<const __nv_bfloat162*>(&w[e]);
+                h[(2 * e) % EPV] = __low2float(h2); h[(2 * e + 1) % EPV] = __high2float(h2);
+            }
+        }
+    }
+};
+__device__ __forceinline__ void store_piece(float* p, const float (&o)[4]) {
+    *reinterpret_cast<float4*>(p) = make_float4(o[0], o[1], o[2], o[3]);
+}
+__device__ __forceinline__ void store_piece(__nv_bfloat16* p, const float (&o)[8]) { store8(p, o); }
+
 // Block-wide sum in a fixed order: shuffle tree inside each warp, then warp 0 adds the warps.
 __device__ __forceinline__ float block_sum(float v, float* scratch /* [warps] */) {
 #pragma unroll
@@ -200,18 +233,26 @@ __global__ void __launch_bounds__(kHLThreads) head_loss_kernel(const HeadLossArg
             float mu[AP];
 #pragma unroll
             for (int i = 0; i < AP; ++i) mu[i] = i < A ? hp.ba[i] : 0.f;
-            for (int k0 = 0; k0 < hp.n_a; k0 += 8) {       // row strides are multiples of 8
-                float h[8];
-                load8(ha + k0, h);
+            constexpr int EPV = RowBlock<T>::EPV;
+            RowBlock<T> blk;
+            for (int k0 = 0; k0 < hp.n_a; k0 += RowBlock<T>::N) {   // row strides are multiples of 8
+                blk.load(ha, k0, a.ldha);
 #pragma unroll
-                for (int kk = 0; kk < 8; ++kk) {
-                    if (k0 + kk < hp.n_a) {
-                        const float4* w4 = reinterpret_cast<const float4*>(Wa_s + (k0 + kk) * AP);
+                for (int pi = 0; pi < kRowPieces; ++pi) {
+                    if (k0 + pi * EPV >= hp.n_a) break;
+                    float h[EPV];
+                    blk.unpack(pi, h);
 #pragma unroll
-                        for (int i4 = 0; i4 < AP / 4; ++i4) {
-                            const float4 w = w4[i4];
-                            mu[4 * i4] = fmaf(h[kk], w.x, mu[4 * i4]); mu[4 * i4 + 1] = fmaf(h[kk], w.y, mu[4 * i4 + 1]);
-                            mu[4 * i4 + 2] = fmaf(h[kk], w.z, mu[4 * i4 + 2]); mu[4 * i4 + 3] = fmaf(h[kk], w.w, mu[4 * i4 + 3]);
+                    for (int kk = 0; kk < EPV; ++kk) {
+                        const int k = k0 + pi * EPV + kk;
+                        if (k < hp.n_a) {
+                            const float4* w4 = reinterpret_cast<const float4*>(Wa_s + k * AP);
+#pragma unroll
+                            for (int i4 = 0; i4 < AP / 4; ++i4) {
+                                const float4 w = w4[i4];
+                                mu[4 * i4] = fmaf(h[kk], w.x, mu[4 * i4]); mu[4 * i4 + 1] = fmaf(h[kk], w.y, mu[4 * i4 + 1]);
+                                mu[4 * i4 + 2] = fmaf(h[kk], w.z, mu[4 * i4 + 2]); mu[4 * i4 + 3] = fmaf(h[kk], w.w, mu[4 * i4 + 3]);
+                            }
                         }
                     }
                 }
@@ -219,15 +260,21 @@ __global__ void __launch_bounds__(kHLThreads) head_loss_kernel(const HeadLossArg
             float v = hp.bc[0];
             {
                 float v1 = 0.f, v2 = 0.f, v3 = 0.f;
-                for (int k0 = 0; k0 < hp.n_c; k0 += 8) {
-                    float h[8];
-                    load8(hc + k0, h);
+                for (int k0 = 0; k0 < hp.n_c; k0 += RowBlock<T>::N) {
+                    blk.load(hc, k0, a.ldhc);
 #pragma unroll
-                    for (int kk = 0; kk < 8; kk += 4) {
-                        if (k0 + kk < hp.n_c) v = fmaf(h[kk], Wc_s[k0 + kk], v);
-                        if (k0 + kk + 1 < hp.n_c) v1 = fmaf(h[kk + 1], Wc_s[k0 + kk + 1], v1);
-                        if (k0 + kk + 2 < hp.n_c) v2 = fmaf(h[kk + 2], Wc_s[k0 + kk + 2], v2);
-                        if (k0 + kk + 3 < hp.n_c) v3 = fmaf(h[kk + 3], Wc_s[k0 + kk + 3], v3);
+                    for (int pi = 0; pi < kRowPieces; ++pi) {
+                        if (k0 + pi * EPV >= hp.n_c) break;
+                        float h[EPV];
+                        blk.unpack(pi, h);
+#pragma unroll
+                        for (int kk = 0; kk < EPV; kk += 4) {
+                            const int k = k0 + pi * EPV + kk;
+                            if (k < hp.n_c) v = fmaf(h[kk], Wc_s[k], v);
+                            if (k + 1 < hp.n_c) v1 = fmaf(h[kk + 1], Wc_s[k + 1], v1);
+                            if (k + 2 < hp.n_c) v2 = fmaf(h[kk + 2], Wc_s[k + 2], v2);
+                            if (k + 3 < hp.n_c) v3 = fmaf(h[kk + 3], Wc_s[k + 3], v3);
+                        }
                     }
                 }
                 v += (v1 + v2) + v3;
@@ -326,34 +373,48 @@ __global__ void __launch_bounds__(kHLThreads) head_loss_kernel(const HeadLossArg
             if (a.v_out) a.v_out[r] = v;
             // ---- dL/dz of the last hidden layers --------------------------------------------
             T* dza = reinterpret_cast<T*>(a.dZa) + (size_t)r * a.lddza;
-            for (int k0 = 0; k0 < a.lddza; k0 += 8) {
-                float h[8], o[8];
-                if (k0 < hp.n_a) load8(ha + k0, h);
+            for (int k0 = 0; k0 < a.lddza; k0 += RowBlock<T>::N) {
+                blk.load(ha, k0, min(a.ldha, a.lddza));
 #pragma unroll
-                for (int kk = 0; kk < 8; ++kk) {
-                    float acc = 0.f;
-                    if (k0 + kk < hp.n_a) {
-                        const float4* w4 = reinterpret_cast<const float4*>(Wa_s + (k0 + kk) * AP);
+                for (int pi = 0; pi < kRowPieces; ++pi) {
+                    if (k0 + pi * EPV >= a.lddza) break;
+                    float h[EPV], o[EPV];
+                    blk.unpack(pi, h);
 #pragma unroll
-                        for (int i4 = 0; i4 < AP / 4; ++i4) {
-                            const float4 w = w4[i4];
-                            acc = fmaf(dmu[4 * i4], w.x, acc); acc = fmaf(dmu[4 * i4 + 1], w.y, acc);
-                            acc = fmaf(dmu[4 * i4 + 2], w.z, acc); acc = fmaf(dmu[4 * i4 + 3], w.w, acc);
+                    for (int kk = 0; kk < EPV; ++kk) {
+                        const int k = k0 + pi * EPV + kk;
+                        float acc = 0.f;
+                        if (k < hp.n_a) {
+                            const float4* w4 = reinterpret_cast<const float4*>(Wa_s + k * AP);
+                            float acc1 = 0.f;
+#pragma unroll
+                            for (int i4 = 0; i4 < AP / 4; ++i4) {
+                                const float4 w = w4[i4];
+                                acc = fmaf(dmu[4 * i4], w.x, acc); acc1 = fmaf(dmu[4 * i4 + 1], w.y, acc1);
+                                acc = fmaf(dmu[4 * i4 + 2], w.z, acc); acc1 = fmaf(dmu[4 * i4 + 3], w.w, acc1);
+                            }
+                            acc = (acc + acc1) * elu_grad_from_h(h[kk], a.h.alpha);
                         }
-                        acc *= elu_grad_from_h(h[kk], a.h.alpha);
+                        o[kk] = acc;
                     }
-                    o[kk] = acc;
+                    store_piece(dza + k0 + pi * EPV, o);
                 }
-                store8(dza + k0, o);
             }
             T* dzc = reinterpret_cast<T*>(a.dZc) + (size_t)r * a.lddzc;
-            for (int k0 = 0; k0 < a.lddzc; k0 += 8) {
-                float h[8], o[8];
-                if (k0 < hp.n_c) load8(hc + k0, h);
+            for (int k0 = 0; k0 < a.lddzc; k0 += RowBlock<T>::N) {
+                blk.load(hc, k0, min(a.ldhc, a.lddzc));
 #pragma unroll
-                for (int kk = 0; kk < 8; ++kk)
-                    o[kk] = k0 + kk < hp.n_c ? dv * Wc_s[k0 + kk] * elu_grad_from_h(h[kk], a.h.alpha) : 0.f;
-                store8(dzc + k0, o);
+                for (int pi = 0; pi < kRowPieces; ++pi) {
+                    if (k0 + pi * EPV >= a.lddzc) break;
+                    float h[EPV], o[EPV];
+                    blk.unpack(pi, h);
+#pragma unroll
+                    for (int kk = 0; kk < EPV; ++kk) {
+                        const int k = k0 + pi * EPV + kk;
+                        o[kk] = k < hp.n_c ? dv * Wc_s[k] * elu_grad_from_h(h[kk], a.h.alpha) : 0.f;
+                    }
+                    store_piece(dzc + k0 + pi * EPV, o);
+                }
             }
         }
     }
