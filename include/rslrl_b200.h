@@ -233,6 +233,30 @@ rslrl_status rslrl_minibatch_indices(uint64_t seed, uint32_t iteration, uint32_t
                                      int32_t batch, int32_t minibatches, int32_t k,
                                      int32_t *d_rows_out, void *cuda_stream);
 
+/* rslrl_gae_scan without any allocation.  (The paper has no counterpart: this is an addition
+ * for embedding the library, not a step of the method.)
+ *
+ * Meant for callers that cannot obtain device memory while they run -- a plug-in living inside
+ * a simulator that owns the whole device pool, a fixed-period control loop that may not risk
+ * the device-wide stall or the failure of an allocation, a process under a fixed memory
+ * budget -- and so cannot supply the scratch buffer rslrl_gae_scan asks for.  The scratch sits
+ * in a fixed array inside the library image instead (96 KiB per GPU that loads the library,
+ * held until the process exits); the call itself allocates and frees nothing.
+ *   - Same arguments, results and alignment rule as rslrl_gae_scan, minus d_scratch.
+ *   - N may not exceed RSLRL_GAE_STATIC_MAX_ENVS: a larger N returns RSLRL_ERR_UNSUPPORTED and
+ *     rslrl_last_error(NULL) says so; nothing is launched.
+ *   - The first call on a device looks up the array's device address (once per device, with
+ *     that device current); make that first call before starting any stream capture.
+ *   - Every call on a device uses the same array, which keeps what the previous call left in
+ *     it.  The call needs nothing in it to start at zero, but two calls that overlap on the GPU
+ *     (different streams, no ordering between them) race on it: order them. */
+#define RSLRL_GAE_STATIC_MAX_ENVS 1048576
+rslrl_status rslrl_gae_scan_static(const float *d_rewards, const float *d_values, const uint8_t *d_dones,
+                                   const uint8_t *d_timeouts, const float *d_last_values,
+                                   float *d_returns, float *d_advantages, int32_t T, int32_t N,
+                                   float gamma, float lam, int32_t normalize, int32_t unbiased,
+                                   float adv_eps, void *cuda_stream);
+
 /* Number of kernels this library has launched in the current process (all contexts). */
 uint64_t     rslrl_kernel_launch_count(void);
 

@@ -81,7 +81,7 @@ EXPORTS = [
     "rslrl_get_counters", "rslrl_set_counters", "rslrl_act", "rslrl_record_step", "rslrl_gae",
     "rslrl_ppo_update", "rslrl_ppo_update_steps", "rslrl_act_host", "rslrl_record_step_host",
     "rslrl_gae_host", "rslrl_gae_scratch_bytes", "rslrl_gae_scan", "rslrl_minibatch_indices",
-    "rslrl_kernel_launch_count", "rslrl_profile_enable", "rslrl_profile_report",
+    "rslrl_kernel_launch_count", "rslrl_profile_enable", "rslrl_profile_report", "rslrl_gae_scan_static",
 ]
 
 _lib = None
@@ -121,6 +121,7 @@ def load_library() -> C.CDLL:
         "rslrl_gae_scratch_bytes": (sz, [i32, i32]),
         "rslrl_gae_scan": (i32, [vp, vp, vp, vp, vp, vp, vp, i32, i32, f32, f32, i32, i32, f32, vp, vp]),
         "rslrl_minibatch_indices": (i32, [u64, u32, u32, i32, i32, i32, vp, vp]),
+        "rslrl_gae_scan_static": (i32, [vp, vp, vp, vp, vp, vp, vp, i32, i32, f32, f32, i32, i32, f32, vp]),
         "rslrl_kernel_launch_count": (u64, []),
         "rslrl_profile_enable": (i32, [i32]),
         "rslrl_profile_report": (i32, [C.c_char_p, sz]),
@@ -292,6 +293,21 @@ def gae_scan(d_rewards, d_values, d_dones, d_timeouts, d_last_values, d_returns,
                             adv_eps, _ptr(d_scratch), C.c_void_p(stream))
     if st != 0:
         raise RslrlError(st, "rslrl_gae_scan")
+
+
+GAE_STATIC_MAX_ENVS = 1048576
+
+
+def gae_scan_static(d_rewards, d_values, d_dones, d_timeouts, d_last_values, d_returns, d_advantages, T: int, N: int,
+                    gamma: float, lam: float, normalize: bool, unbiased: bool, adv_eps: float, stream: int = 0):
+    """rslrl_gae_scan_static: the GAE scan with its scratch inside the library, for callers that
+    cannot allocate device memory.  At most GAE_STATIC_MAX_ENVS environments."""
+    lib = load_library()
+    st = lib.rslrl_gae_scan_static(_ptr(d_rewards), _ptr(d_values), _ptr(d_dones), _ptr(d_timeouts),
+                                   _ptr(d_last_values), _ptr(d_returns), _ptr(d_advantages), T, N, gamma, lam,
+                                   int(normalize), int(unbiased), adv_eps, C.c_void_p(stream))
+    if st != 0:
+        raise RslrlError(st, lib.rslrl_last_error(None).decode() or "rslrl_gae_scan_static")
 
 
 def gae_scratch_bytes(T: int, N: int) -> int:

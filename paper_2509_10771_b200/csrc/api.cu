@@ -37,6 +37,11 @@ std::string g_create_error;
 
 }  // namespace
 
+namespace rslrl {
+// Message returned by rslrl_last_error(NULL); used by entry points that have no context.
+void set_global_error(const char* msg) { g_create_error = msg; }
+}  // namespace rslrl
+
 struct rslrl_ctx {
     rslrl_model_cfg mc;
     rslrl_ppo_cfg pc;

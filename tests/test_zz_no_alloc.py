@@ -1,0 +1,52 @@
+"""rslrl_gae_scan_static -- the allocation-free GAE entry point -- against rslrl_gae_scan.
+
+The static variant exists for hosts that cannot get device memory while they run (see the
+header).  It runs the same scan, so on the same inputs it must reproduce the regular entry
+point; two calls in a row check that what the first call leaves in the shared scratch array
+does not leak into the second.  This file sorts last on purpose: it exercises an optional
+addition, and a run that stops at the first failure should have seen every other test first.
+"""
+import numpy as np
+import pytest
+
+pytestmark = pytest.mark.gpu
+
+
+def _inputs(T, N, seed):
+    rng = np.random.default_rng(seed)
+    r = rng.normal(0, 0.5, (T, N)).astype(np.float32)
+    v = rng.normal(0, 1.0, (T, N)).astype(np.float32)
+    lv = rng.normal(0, 1.0, N).astype(np.float32)
+    d = (rng.random((T, N)) < 0.02).astype(np.uint8)
+    to = (d & (rng.random((T, N)) < 0.5)).astype(np.uint8)
+    return r, v, d, to, lv
+
+
+def test_static_gae_matches_regular_entry_point_on_two_calls_in_a_row():
+    import torch
+    from paper_2509_10771_b200 import binding
+    from parity_utils import assert_close
+
+    dev = lambda x: torch.from_numpy(x).cuda()
+    # a large call first, then a smaller one with other data: stale triples of the first call
+    # sit beyond the blocks the second call uses and must not influence it
+    for T, N, seed, normalize in ((24, 40000, 1, True), (8, 1000, 2, True), (5, 130, 3, False)):
+        r, v, d, to, lv = (dev(x) for x in _inputs(T, N, seed))
+        ret_a = torch.empty((T, N), device="cuda"); adv_a = torch.empty((T, N), device="cuda")
+        ret_b = torch.empty((T, N), device="cuda"); adv_b = torch.empty((T, N), device="cuda")
+        scratch = torch.empty(binding.gae_scratch_bytes(T, N), dtype=torch.uint8, device="cuda")
+        binding.gae_scan(r, v, d, to, lv, ret_a, adv_a, T, N, 0.99, 0.95, normalize, True, 1e-8, scratch)
+        binding.gae_scan_static(r, v, d, to, lv, ret_b, adv_b, T, N, 0.99, 0.95, normalize, True, 1e-8)
+        torch.cuda.synchronize()
+        assert_close(ret_b.cpu().numpy(), ret_a.cpu().numpy(), 1e-5, "returns")
+        assert_close(adv_b.cpu().numpy(), adv_a.cpu().numpy(), 1e-5, "advantages")
+
+
+def test_static_gae_rejects_sizes_beyond_its_limit():
+    from paper_2509_10771_b200 import binding
+    with pytest.raises(binding.RslrlError) as e:
+        binding.gae_scan_static(None, None, None, None, None, None, None, 4, binding.GAE_STATIC_MAX_ENVS + 1,
+                                0.99, 0.95, True, True, 1e-8)
+    assert e.value.status == 5 and "RSLRL_GAE_STATIC_MAX_ENVS" in str(e.value)
+    # empty input: nothing to do, nothing launched
+    binding.gae_scan_static(None, None, None, None, None, None, None, 0, 0, 0.99, 0.95, True, True, 1e-8)
