@@ -32,7 +32,8 @@ constexpr uint32_t kStageA = BLOCK_M * BLOCK_K * 2;      // 16 KiB
 constexpr uint32_t kStageB = kMaxBN * BLOCK_K * 2;       // 32 KiB
 constexpr uint32_t kTmemCols = 512;                      // two accumulator buffers of 256 columns
 constexpr int kMaxProblems = 8;
-constexpr size_t kSmemBytes = 1024 + kStages * (kStageA + kStageB) + 256;
+constexpr uint32_t kStageOut = 32 * 32 * 2;              // 2 KiB staging per epilogue warp (32 rows x 32 bf16)
+constexpr size_t kSmemBytes = 1024 + kStages * (kStageA + kStageB) + kEpiWarps * kStageOut + 256;
 constexpr unsigned long long kWaitLimitNs = 2000000000ull;   // 2 s
 
 enum TcMode { TC_FWD = 0, TC_DGRAD = 1, TC_WGRAD = 2 };
@@ -52,6 +53,7 @@ struct TcProblem {
 struct TcParams {
     CUtensorMap tmA[kMaxProblems];
     CUtensorMap tmB[kMaxProblems];
+    CUtensorMap tmOut[kMaxProblems];   // BF16 output, boxes of 32 columns x 32 rows, 64-byte swizzle
     TcProblem p[kMaxProblems];
     int count, total_items;
     float alpha;
@@ -104,6 +106,16 @@ __device__ __forceinline__ void tma_load_2d(void* smem_dst, const CUtensorMap* t
         "cp.async.bulk.tensor.2d.shared::cluster.global.tile.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];"
         ::"r"(smem_u32(smem_dst)), "l"(tm), "r"(x), "r"(y), "r"(smem_u32(bar)) : "memory");
 }
+// Shared -> global tile store, tracked by the issuing thread's bulk async-group.
+__device__ __forceinline__ void tma_store_2d(const CUtensorMap* tm, const void* smem_src, int x, int y) {
+    asm volatile("cp.async.bulk.tensor.2d.global.shared::cta.bulk_group [%0, {%2, %3}], [%1];"
+                 ::"l"(tm), "r"(smem_u32(smem_src)), "r"(x), "r"(y) : "memory");
+    asm volatile("cp.async.bulk.commit_group;" ::: "memory");
+}
+__device__ __forceinline__ void tma_store_wait_read() { asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory"); }
+__device__ __forceinline__ void tma_store_wait_all() { asm volatile("cp.async.bulk.wait_group 0;" ::: "memory"); }
+__device__ __forceinline__ void fence_async_smem() { asm volatile("fence.proxy.async.shared::cta;" ::: "memory"); }
+
 __device__ __forceinline__ void tma_prefetch_desc(const CUtensorMap* tm) {
     asm volatile("prefetch.tensormap [%0];" ::"l"(tm) : "memory");
 }
@@ -197,7 +209,8 @@ __global__ void __launch_bounds__(kThreads, 1) tc_gemm_kernel(const __grid_const
     uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
     uint8_t* sA = smem;
     uint8_t* sB = smem + kStages * kStageA;
-    uint64_t* full = reinterpret_cast<uint64_t*>(sB + kStages * kStageB);
+    uint8_t* sOut = sB + kStages * kStageB;                 // kEpiWarps staging buffers, 1 KiB aligned
+    uint64_t* full = reinterpret_cast<uint64_t*>(sOut + kEpiWarps * kStageOut);
     uint64_t* empty = full + kStages;
     uint64_t* tfull = empty + kStages;
     uint64_t* tempty = tfull + 2;
@@ -308,6 +321,11 @@ __global__ void __launch_bounds__(kThreads, 1) tc_gemm_kernel(const __grid_const
         // ================================ epilogue =====================================
         const int q = warp & 3;                    // accumulator lanes 32q .. 32q+31
         const int group = (warp - 2) >> 2;         // handles chunks group, group + 4, ...
+        // BF16 results leave through a 32 x 32 staging tile per warp and a TMA store: lane r
+        // writes row r as four 16-byte pieces, piece j at (j ^ ((r >> 1) & 3)) (64-byte swizzle,
+        // conflict-free), then one lane hands the tile to the copy engine.
+        uint8_t* stage_row = sOut + (warp - 2) * kStageOut + lane * 64;
+        const int sw = (lane >> 1) & 3;
         bool ok = true;
         int local = 0;
         for (int item = blockIdx.x; ok && item < P.total_items; item += gridDim.x, ++local) {
@@ -319,7 +337,7 @@ __global__ void __launch_bounds__(kThreads, 1) tc_gemm_kernel(const __grid_const
             const int chunks = p.bn / 32;
             // data gradient: fetch the stored post-activations of this thread's chunks before
             // waiting for the accumulator, so that the loads overlap the main loop
-            uint4 haux[2][4];
+            uint4 haux[2][4] = {};
             if (MODE == TC_DGRAD) {
 #pragma unroll
                 for (int ci = 0; ci < 2; ++ci) {
@@ -340,11 +358,15 @@ __global__ void __launch_bounds__(kThreads, 1) tc_gemm_kernel(const __grid_const
                 uint32_t acc[32];
                 tmem_ld32(tmem_base + ((uint32_t)(32 * q) << 16) + (uint32_t)(buf * kMaxBN + 32 * c), acc);
                 const int col = it.n0 + 32 * c;
-                if (row >= p.m_extent || col >= p.n_extent) continue;
+                if (col >= p.n_extent) continue;              // uniform across the warp
+                if (MODE != TC_WGRAD) {
+                    // the previous tile must have left the staging buffer before it is rewritten
+                    if (lane == 0) tma_store_wait_read();
+                    __syncwarp();
+                }
                 if (MODE == TC_FWD) {
                     // p.bias is zero-padded to the padded width: no bounds checks
                     const float4* b4 = reinterpret_cast<const float4*>(p.bias + col);
-                    uint4* dst = reinterpret_cast<uint4*>(p.out16 + (size_t)row * p.ld_out + col);
 #pragma unroll
                     for (int g = 0; g < 4; ++g) {
                         const float4 ba = __ldg(b4 + 2 * g), bb = __ldg(b4 + 2 * g + 1);
@@ -357,10 +379,9 @@ __global__ void __launch_bounds__(kThreads, 1) tc_gemm_kernel(const __grid_const
                             __nv_bfloat162 h2 = __floats2bfloat162_rn(v0, v1);
                             o[e] = *reinterpret_cast<uint32_t*>(&h2);
                         }
-                        dst[g] = make_uint4(o[0], o[1], o[2], o[3]);
+                        *reinterpret_cast<uint4*>(stage_row + ((g ^ sw) << 4)) = make_uint4(o[0], o[1], o[2], o[3]);
                     }
                 } else if (MODE == TC_DGRAD) {
-                    uint4* dst = reinterpret_cast<uint4*>(p.out16 + (size_t)row * p.ld_out + col);
 #pragma unroll
                     for (int g = 0; g < 4; ++g) {
                         const uint4 hv = haux[ci][g];
@@ -375,9 +396,9 @@ __global__ void __launch_bounds__(kThreads, 1) tc_gemm_kernel(const __grid_const
                             __nv_bfloat162 r2 = __floats2bfloat162_rn(v0, v1);
                             o[e] = *reinterpret_cast<uint32_t*>(&r2);
                         }
-                        dst[g] = make_uint4(o[0], o[1], o[2], o[3]);
+                        *reinterpret_cast<uint4*>(stage_row + ((g ^ sw) << 4)) = make_uint4(o[0], o[1], o[2], o[3]);
                     }
-                } else {
+                } else if (row < p.m_extent) {
                     float* dst = p.out32 + (size_t)it.split * p.split_stride + (size_t)row * p.ld_out32 + col;
 #pragma unroll
                     for (int g = 0; g < 8; ++g)
@@ -386,11 +407,19 @@ __global__ void __launch_bounds__(kThreads, 1) tc_gemm_kernel(const __grid_const
                                 make_float4(__uint_as_float(acc[4 * g]), __uint_as_float(acc[4 * g + 1]),
                                             __uint_as_float(acc[4 * g + 2]), __uint_as_float(acc[4 * g + 3]));
                 }
+                if (MODE != TC_WGRAD) {
+                    fence_async_smem();                       // staging writes -> visible to the copy engine
+                    __syncwarp();
+                    // rows at or beyond the tensor's extent are clipped by the store itself
+                    if (lane == 0 && it.m0 + 32 * q < p.m_extent)
+                        tma_store_2d(&P.tmOut[it.prob], sOut + (warp - 2) * kStageOut, col, it.m0 + 32 * q);
+                }
             }
             tc_fence_before();
             __syncwarp();
             if (lane == 0) mbar_arrive(&tempty[buf]);
         }
+        if (MODE != TC_WGRAD && lane == 0) tma_store_wait_all();   // stores done before the CTA retires
     }
     tc_fence_before();
     __syncthreads();
@@ -437,8 +466,9 @@ EncodeTiledFn get_encode_fn() {
     return fn;
 }
 
-// 2-D BF16 tensor [rows][cols] with row stride ld (elements); box = box_cols x box_rows, 128-byte swizzle.
-bool make_tmap(CUtensorMap* tm, const void* base, int rows, int cols, int ld, int box_cols, int box_rows) {
+// 2-D BF16 tensor [rows][cols] with row stride ld (elements); box = box_cols x box_rows.
+bool make_tmap(CUtensorMap* tm, const void* base, int rows, int cols, int ld, int box_cols, int box_rows,
+               CUtensorMapSwizzle swizzle = CU_TENSOR_MAP_SWIZZLE_128B) {
     EncodeTiledFn fn = get_encode_fn();
     if (!fn) return false;
     const cuuint64_t dims[2] = {(cuuint64_t)cols, (cuuint64_t)rows};
@@ -446,7 +476,7 @@ bool make_tmap(CUtensorMap* tm, const void* base, int rows, int cols, int ld, in
     const cuuint32_t box[2] = {(cuuint32_t)box_cols, (cuuint32_t)box_rows};
     const cuuint32_t estr[2] = {1, 1};
     return fn(tm, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(base), dims, strides, box, estr,
-              CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+              CU_TENSOR_MAP_INTERLEAVE_NONE, swizzle, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
               CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
@@ -610,6 +640,8 @@ UmmaEngine* umma_create(const UmmaSetup& s, std::string* err) {
                 TcProblem& p = P.p[P.count - 1];
                 p.bias = e->bias_pad[ni][l]; p.bias_n = e->pw[ni][l];
                 p.out16 = act_buffers ? e->h_act[ni][l] : e->h[ni][l]; p.ld_out = e->pw[ni][l];
+                if (!make_tmap(&P.tmOut[P.count - 1], p.out16, rows, e->pw[ni][l], e->pw[ni][l], 32, 32, CU_TENSOR_MAP_SWIZZLE_64B))
+                    return false;
             }
             finish_params(P, alpha, e->error_dev);
             out.push_back(P);
@@ -630,6 +662,8 @@ UmmaEngine* umma_create(const UmmaSetup& s, std::string* err) {
             TcProblem& p = P.p[P.count - 1];
             p.out16 = e->dz[ni][l - 1]; p.ld_out = e->pw[ni][l - 1];
             p.aux16 = e->h[ni][l - 1]; p.ld_aux = e->pw[ni][l - 1];
+            if (!make_tmap(&P.tmOut[P.count - 1], p.out16, R, e->pw[ni][l - 1], e->pw[ni][l - 1], 32, 32, CU_TENSOR_MAP_SWIZZLE_64B))
+                return bail("tensor map encoding failed");
         }
         finish_params(P, alpha, e->error_dev);
         e->upd_dgrad.push_back(P);
