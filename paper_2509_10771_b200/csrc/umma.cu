@@ -21,7 +21,9 @@ namespace rslrl {
 
 namespace {
 
-constexpr int kStages = 4;
+// Forward and data gradient: 3 pipeline stages + a 4 KiB result tile per epilogue warp;
+// weight gradient (long contraction, FP32 results stored from registers): 4 stages.
+__host__ __device__ constexpr int stages_of(int mode) { return mode == 2 ? 4 : 3; }
 constexpr int BLOCK_M = 128;
 constexpr int BLOCK_K = 64;                      // bf16 elements = one 128-byte swizzle row
 constexpr int UMMA_K = 16;
@@ -32,8 +34,10 @@ constexpr uint32_t kStageA = BLOCK_M * BLOCK_K * 2;      // 16 KiB
 constexpr uint32_t kStageB = kMaxBN * BLOCK_K * 2;       // 32 KiB
 constexpr uint32_t kTmemCols = 512;                      // two accumulator buffers of 256 columns
 constexpr int kMaxProblems = 8;
-constexpr uint32_t kStageOut = 32 * 32 * 2;              // 2 KiB staging per epilogue warp (32 rows x 32 bf16)
-constexpr size_t kSmemBytes = 1024 + kStages * (kStageA + kStageB) + kEpiWarps * kStageOut + 256;
+constexpr uint32_t kStageOut = 32 * 64 * 2;              // 4 KiB result tile per epilogue warp (32 rows x 64 bf16)
+__host__ __device__ constexpr size_t smem_bytes_of(int mode) {
+    return 1024 + (size_t)stages_of(mode) * (kStageA + kStageB) + (mode == 2 ? 0 : kEpiWarps * kStageOut) + 512;
+}
 constexpr unsigned long long kWaitLimitNs = 2000000000ull;   // 2 s
 
 enum TcMode { TC_FWD = 0, TC_DGRAD = 1, TC_WGRAD = 2 };
@@ -53,7 +57,8 @@ struct TcProblem {
 struct TcParams {
     CUtensorMap tmA[kMaxProblems];
     CUtensorMap tmB[kMaxProblems];
-    CUtensorMap tmOut[kMaxProblems];   // BF16 output, boxes of 32 columns x 32 rows, 64-byte swizzle
+    CUtensorMap tmOut[kMaxProblems];   // BF16 output, boxes of 64 columns x 32 rows, 128-byte swizzle
+    CUtensorMap tmAux[kMaxProblems];   // data gradient: stored post-activations, same boxes
     TcProblem p[kMaxProblems];
     int count, total_items;
     float alpha;
@@ -205,17 +210,19 @@ __device__ __forceinline__ float elu_fast(float z, float alpha) {
 
 template <int MODE>
 __global__ void __launch_bounds__(kThreads, 1) tc_gemm_kernel(const __grid_constant__ TcParams P) {
+    constexpr int kStages = stages_of(MODE);
     extern __shared__ uint8_t smem_raw[];
     uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
     uint8_t* sA = smem;
     uint8_t* sB = smem + kStages * kStageA;
-    uint8_t* sOut = sB + kStages * kStageB;                 // kEpiWarps staging buffers, 1 KiB aligned
-    uint64_t* full = reinterpret_cast<uint64_t*>(sOut + kEpiWarps * kStageOut);
+    uint8_t* sOut = sB + kStages * kStageB;                 // kEpiWarps result tiles, 1 KiB aligned
+    uint64_t* full = reinterpret_cast<uint64_t*>(sOut + (MODE == TC_WGRAD ? 0 : kEpiWarps * kStageOut));
     uint64_t* empty = full + kStages;
     uint64_t* tfull = empty + kStages;
     uint64_t* tempty = tfull + 2;
     uint64_t* drain = tempty + 2;
-    uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(drain + 1);
+    uint64_t* auxbar = drain + 1;                           // one per epilogue warp
+    uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(auxbar + kEpiWarps);
     volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
@@ -223,6 +230,7 @@ __global__ void __launch_bounds__(kThreads, 1) tc_gemm_kernel(const __grid_const
         for (int s = 0; s < kStages; ++s) { mbar_init(&full[s], 1); mbar_init(&empty[s], 1); }
         for (int b = 0; b < 2; ++b) { mbar_init(&tfull[b], 1); mbar_init(&tempty[b], kEpiWarps); }
         mbar_init(drain, 1);
+        for (int w = 0; w < kEpiWarps; ++w) mbar_init(&auxbar[w], 1);
         *abort_flag = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
         asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
@@ -320,12 +328,17 @@ __global__ void __launch_bounds__(kThreads, 1) tc_gemm_kernel(const __grid_const
     } else {
         // ================================ epilogue =====================================
         const int q = warp & 3;                    // accumulator lanes 32q .. 32q+31
-        const int group = (warp - 2) >> 2;         // handles chunks group, group + 4, ...
-        // BF16 results leave through a 32 x 32 staging tile per warp and a TMA store: lane r
-        // writes row r as four 16-byte pieces, piece j at (j ^ ((r >> 1) & 3)) (64-byte swizzle,
-        // conflict-free), then one lane hands the tile to the copy engine.
-        uint8_t* stage_row = sOut + (warp - 2) * kStageOut + lane * 64;
-        const int sw = (lane >> 1) & 3;
+        const int group = (warp - 2) >> 2;         // handles the 64 columns [64 group, 64 group + 64) of the tile
+        // BF16 results leave through a 32 x 64 tile per warp and one TMA store per work item:
+        // lane r owns row r (128 bytes = eight 16-byte pieces), piece j is kept at j ^ (r & 7)
+        // (the 128-byte swizzle of the tensor map; conflict-free for the warp).  For the data
+        // gradient the same tile first receives the stored post-activations by TMA load.
+        uint8_t* tile = sOut + (warp - 2) * kStageOut;
+        uint8_t* tile_row = tile + lane * 128;
+        const int sw = lane & 7;
+        uint64_t* my_aux = &auxbar[warp - 2];
+        uint32_t aux_phase = 0;
+        bool aux_pending = false;
         bool ok = true;
         int local = 0;
         for (int item = blockIdx.x; ok && item < P.total_items; item += gridDim.x, ++local) {
@@ -335,35 +348,34 @@ __global__ void __launch_bounds__(kThreads, 1) tc_gemm_kernel(const __grid_const
             const uint32_t use = (uint32_t)(local >> 1);
             const int row = it.m0 + 32 * q + lane;
             const int chunks = p.bn / 32;
-            // data gradient: fetch the stored post-activations of this thread's chunks before
-            // waiting for the accumulator, so that the loads overlap the main loop
-            uint4 haux[2][4] = {};
-            if (MODE == TC_DGRAD) {
-#pragma unroll
-                for (int ci = 0; ci < 2; ++ci) {
-                    const int col = it.n0 + 32 * (group + 4 * ci);
-                    if (group + 4 * ci < chunks && row < p.m_extent && col < p.n_extent) {
-                        const uint4* hsrc = reinterpret_cast<const uint4*>(p.aux16 + (size_t)row * p.ld_aux + col);
-#pragma unroll
-                        for (int g = 0; g < 4; ++g) haux[ci][g] = __ldg(hsrc + g);
+            const int col0 = it.n0 + 64 * group;                          // first column of this warp
+            const bool active = 2 * group < chunks && col0 < p.n_extent;  // uniform across the warp
+            if (MODE != TC_WGRAD && active) {
+                // the previous item's store must have read the tile before it is reused
+                if (lane == 0) {
+                    tma_store_wait_read();
+                    if (MODE == TC_DGRAD) {
+                        mbar_expect_tx(my_aux, kStageOut);
+                        tma_load_2d(tile, &P.tmAux[it.prob], col0, it.m0 + 32 * q, my_aux);
                     }
                 }
+                if (MODE == TC_DGRAD) aux_pending = true;
+                __syncwarp();
             }
             if (!mbar_wait(&tfull[buf], use & 1u, abort_flag, P.error, 4)) { ok = false; break; }
             tc_fence_after();
+            if (MODE == TC_DGRAD && active) {
+                if (!mbar_wait(my_aux, aux_phase, abort_flag, P.error, 5)) { ok = false; break; }
+                aux_phase ^= 1u;
+                aux_pending = false;
+            }
 #pragma unroll
             for (int ci = 0; ci < 2; ++ci) {
-                const int c = group + 4 * ci;
-                if (c >= chunks) break;                       // uniform across the warp
+                if (!active) break;
+                const int c = 2 * group + ci;
                 uint32_t acc[32];
                 tmem_ld32(tmem_base + ((uint32_t)(32 * q) << 16) + (uint32_t)(buf * kMaxBN + 32 * c), acc);
                 const int col = it.n0 + 32 * c;
-                if (col >= p.n_extent) continue;              // uniform across the warp
-                if (MODE != TC_WGRAD) {
-                    // the previous tile must have left the staging buffer before it is rewritten
-                    if (lane == 0) tma_store_wait_read();
-                    __syncwarp();
-                }
                 if (MODE == TC_FWD) {
                     // p.bias is zero-padded to the padded width: no bounds checks
                     const float4* b4 = reinterpret_cast<const float4*>(p.bias + col);
@@ -379,12 +391,13 @@ __global__ void __launch_bounds__(kThreads, 1) tc_gemm_kernel(const __grid_const
                             __nv_bfloat162 h2 = __floats2bfloat162_rn(v0, v1);
                             o[e] = *reinterpret_cast<uint32_t*>(&h2);
                         }
-                        *reinterpret_cast<uint4*>(stage_row + ((g ^ sw) << 4)) = make_uint4(o[0], o[1], o[2], o[3]);
+                        *reinterpret_cast<uint4*>(tile_row + (((4 * ci + g) ^ sw) << 4)) = make_uint4(o[0], o[1], o[2], o[3]);
                     }
                 } else if (MODE == TC_DGRAD) {
 #pragma unroll
                     for (int g = 0; g < 4; ++g) {
-                        const uint4 hv = haux[ci][g];
+                        uint4* piece = reinterpret_cast<uint4*>(tile_row + (((4 * ci + g) ^ sw) << 4));
+                        const uint4 hv = *piece;
                         const uint32_t hw[4] = {hv.x, hv.y, hv.z, hv.w};
                         uint32_t o[4];
 #pragma unroll
@@ -396,7 +409,7 @@ __global__ void __launch_bounds__(kThreads, 1) tc_gemm_kernel(const __grid_const
                             __nv_bfloat162 r2 = __floats2bfloat162_rn(v0, v1);
                             o[e] = *reinterpret_cast<uint32_t*>(&r2);
                         }
-                        *reinterpret_cast<uint4*>(stage_row + ((g ^ sw) << 4)) = make_uint4(o[0], o[1], o[2], o[3]);
+                        *piece = make_uint4(o[0], o[1], o[2], o[3]);
                     }
                 } else if (row < p.m_extent) {
                     float* dst = p.out32 + (size_t)it.split * p.split_stride + (size_t)row * p.ld_out32 + col;
@@ -407,19 +420,26 @@ __global__ void __launch_bounds__(kThreads, 1) tc_gemm_kernel(const __grid_const
                                 make_float4(__uint_as_float(acc[4 * g]), __uint_as_float(acc[4 * g + 1]),
                                             __uint_as_float(acc[4 * g + 2]), __uint_as_float(acc[4 * g + 3]));
                 }
-                if (MODE != TC_WGRAD) {
-                    fence_async_smem();                       // staging writes -> visible to the copy engine
-                    __syncwarp();
-                    // rows at or beyond the tensor's extent are clipped by the store itself
-                    if (lane == 0 && it.m0 + 32 * q < p.m_extent)
-                        tma_store_2d(&P.tmOut[it.prob], sOut + (warp - 2) * kStageOut, col, it.m0 + 32 * q);
-                }
             }
+            // the accumulator has been read: hand the tensor-memory buffer back first
             tc_fence_before();
             __syncwarp();
             if (lane == 0) mbar_arrive(&tempty[buf]);
+            if (MODE != TC_WGRAD && active) {
+                fence_async_smem();                           // tile writes -> visible to the copy engine
+                __syncwarp();
+                // rows at or beyond the tensor's extent are clipped by the store itself
+                if (lane == 0 && it.m0 + 32 * q < p.m_extent)
+                    tma_store_2d(&P.tmOut[it.prob], tile, col0, it.m0 + 32 * q);
+            }
         }
-        if (MODE != TC_WGRAD && lane == 0) tma_store_wait_all();   // stores done before the CTA retires
+        if (MODE != TC_WGRAD && lane == 0) {
+            if (aux_pending) {      // gave up with a load in flight: let it land first
+                const unsigned long long t0 = global_ns();
+                while (!mbar_try_wait(my_aux, aux_phase) && global_ns() - t0 < kWaitLimitNs) {}
+            }
+            tma_store_wait_all();   // stores done before the CTA retires
+        }
     }
     tc_fence_before();
     __syncthreads();
@@ -548,7 +568,7 @@ cudaError_t launch_tc(const TcParams& P, int num_sms, cudaStream_t s) {
     if (P.total_items == 0) return cudaSuccess;
     const int grid = std::min(P.total_items, num_sms);
     LaunchScope scope_(MODE == TC_FWD ? "tc_gemm_fwd" : MODE == TC_DGRAD ? "tc_gemm_dgrad" : "tc_gemm_wgrad", s);
-    tc_gemm_kernel<MODE><<<grid, kThreads, kSmemBytes, s>>>(P);
+    tc_gemm_kernel<MODE><<<grid, kThreads, smem_bytes_of(MODE), s>>>(P);
     return cudaGetLastError();
 }
 
@@ -574,9 +594,9 @@ UmmaEngine* umma_create(const UmmaSetup& s, std::string* err) {
     int dev = 0; cudaDeviceProp prop;
     if (cudaGetDevice(&dev) != cudaSuccess || cudaGetDeviceProperties(&prop, dev) != cudaSuccess) return failmsg("no CUDA device");
     if (prop.major != 10) return failmsg("the tensor-core mode needs an sm_100 device");
-    if (cudaFuncSetAttribute(tc_gemm_kernel<TC_FWD>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kSmemBytes) != cudaSuccess ||
-        cudaFuncSetAttribute(tc_gemm_kernel<TC_DGRAD>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kSmemBytes) != cudaSuccess ||
-        cudaFuncSetAttribute(tc_gemm_kernel<TC_WGRAD>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kSmemBytes) != cudaSuccess)
+    if (cudaFuncSetAttribute(tc_gemm_kernel<TC_FWD>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem_bytes_of(TC_FWD)) != cudaSuccess ||
+        cudaFuncSetAttribute(tc_gemm_kernel<TC_DGRAD>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem_bytes_of(TC_DGRAD)) != cudaSuccess ||
+        cudaFuncSetAttribute(tc_gemm_kernel<TC_WGRAD>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem_bytes_of(TC_WGRAD)) != cudaSuccess)
         return failmsg("could not reserve shared memory for the tensor-core kernels");
     UmmaEngine* e = new UmmaEngine();
     e->s = s;
@@ -640,8 +660,7 @@ UmmaEngine* umma_create(const UmmaSetup& s, std::string* err) {
                 TcProblem& p = P.p[P.count - 1];
                 p.bias = e->bias_pad[ni][l]; p.bias_n = e->pw[ni][l];
                 p.out16 = act_buffers ? e->h_act[ni][l] : e->h[ni][l]; p.ld_out = e->pw[ni][l];
-                if (!make_tmap(&P.tmOut[P.count - 1], p.out16, rows, e->pw[ni][l], e->pw[ni][l], 32, 32, CU_TENSOR_MAP_SWIZZLE_64B))
-                    return false;
+                if (!make_tmap(&P.tmOut[P.count - 1], p.out16, rows, e->pw[ni][l], e->pw[ni][l], 64, 32)) return false;
             }
             finish_params(P, alpha, e->error_dev);
             out.push_back(P);
@@ -662,7 +681,8 @@ UmmaEngine* umma_create(const UmmaSetup& s, std::string* err) {
             TcProblem& p = P.p[P.count - 1];
             p.out16 = e->dz[ni][l - 1]; p.ld_out = e->pw[ni][l - 1];
             p.aux16 = e->h[ni][l - 1]; p.ld_aux = e->pw[ni][l - 1];
-            if (!make_tmap(&P.tmOut[P.count - 1], p.out16, R, e->pw[ni][l - 1], e->pw[ni][l - 1], 32, 32, CU_TENSOR_MAP_SWIZZLE_64B))
+            if (!make_tmap(&P.tmOut[P.count - 1], p.out16, R, e->pw[ni][l - 1], e->pw[ni][l - 1], 64, 32) ||
+                !make_tmap(&P.tmAux[P.count - 1], p.aux16, R, e->pw[ni][l - 1], e->pw[ni][l - 1], 64, 32))
                 return bail("tensor map encoding failed");
         }
         finish_params(P, alpha, e->error_dev);
