@@ -71,6 +71,7 @@ struct rslrl_ctx {
     void* up_h[2][kMaxLayers] = {};
     void* up_dz[2][kMaxLayers] = {};
     float *dmu = nullptr, *dv = nullptr; int lddmu = 0;
+    int* perm = nullptr;                  // [T*N] shuffle of the current epoch
     float *partials = nullptr, *block_partials = nullptr, *sumsq_partials = nullptr, *loss_sums = nullptr;
     float* stats_dev = nullptr; float* stats_host = nullptr; int max_stat_rows = 0;
     SymTables sym{};
@@ -398,6 +399,7 @@ rslrl_status rslrl_create(const rslrl_model_cfg* m, const rslrl_ppo_cfg* p, void
     A_(c->act_mb, (size_t)c->R * as); A_(c->mu_old, (size_t)c->Bmb * as); A_(c->sigma_old, (size_t)c->Bmb * as);
     A_(c->logp_old, c->Bmb); A_(c->v_old, c->Bmb); A_(c->ret_mb, c->Bmb); A_(c->adv_mb, c->Bmb);
     A_(c->dmu, (size_t)c->R * as); A_(c->dv, (size_t)c->R * 4);
+    A_(c->perm, (size_t)B);
     A_(c->partials, (size_t)c->splits * c->P_dev);
     A_(c->block_partials, (size_t)head_loss_blocks(c->Bmb) * head_partial_stride());
     A_(c->sumsq_partials, reduce_blocks(c->P_dev)); A_(c->loss_sums, 8);
@@ -613,10 +615,9 @@ rslrl_status rslrl_ppo_update_steps(rslrl_ctx* c, int32_t max_steps, rslrl_updat
             if (c->umma) umma_gather_targets(c->umma, &g);
             g.act_mb = c->act_mb; g.mu_old = c->mu_old; g.sigma_old = c->sigma_old;
             g.logp_old = c->logp_old; g.v_old = c->v_old; g.ret = c->ret_mb; g.adv_mb = c->adv_mb;
-            g.rows_out = nullptr; g.Bmb = c->Bmb; g.sym = pc.sym_enable; g.st = c->sym;
-            g.seed_lo = (uint32_t)pc.seed; g.seed_hi = (uint32_t)(pc.seed >> 32);
-            g.iteration = c->iteration; g.epoch = (uint32_t)e; g.batch = (uint32_t)(T * N);
-            g.first = (uint32_t)k * (uint32_t)c->Bmb;
+            g.rows = c->perm + (size_t)k * c->Bmb; g.Bmb = c->Bmb; g.sym = pc.sym_enable; g.st = c->sym;
+            if (k == 0)   // the epoch's shuffle, resolved once for all of its minibatches
+                CU(c, launch_perm_rows(pc.seed, c->iteration, (uint32_t)e, (uint32_t)(T * N), 0u, T * N, c->perm, c->stream));
             CU(c, launch_gather(g, c->stream));
             // ---- forward ----------------------------------------------------------------
             HeadLossArgs hl{};
@@ -642,9 +643,6 @@ rslrl_status rslrl_ppo_update_steps(rslrl_ctx* c, int32_t max_steps, rslrl_updat
             hl.dmu = c->dmu; hl.lddmu = c->lddmu; hl.dv = c->dv;
             hl.block_partials = c->block_partials; hl.mu_out = nullptr; hl.v_out = nullptr;
             CU(c, launch_head_loss(hl, c->stream));
-            CU(c, launch_head_finalize(c->block_partials, head_loss_blocks(c->Bmb), c->partials, (int)ha.b_off,
-                                       (int)c->logstd_off, (int)hc.b_off, A, pc.entropy_coef,
-                                       c->param + c->logstd_off, c->loss_sums, c->stream));
             // ---- backward ---------------------------------------------------------------
             if (c->prec == RSLRL_FP32) TRY(backward_fp32(c));
             else CU(c, umma_update_backward(c->umma));
@@ -652,6 +650,9 @@ rslrl_status rslrl_ppo_update_steps(rslrl_ctx* c, int32_t max_steps, rslrl_updat
             ReduceArgs r{};
             r.partials = c->partials; r.splits = c->splits; r.split_stride = c->P_dev;
             r.grad = c->grad; r.P = c->P_dev; r.sumsq_partials = c->sumsq_partials;
+            r.block_partials = c->block_partials; r.nblocks = head_loss_blocks(c->Bmb);
+            r.off_ba = (int)ha.b_off; r.off_logstd = (int)c->logstd_off; r.off_bc = (int)hc.b_off; r.A = A;
+            r.entropy_coef = pc.entropy_coef; r.log_std = c->param + c->logstd_off; r.loss_sums = c->loss_sums;
             CU(c, launch_reduce(r, c->stream));
             AdamArgs ad{};
             ad.param = c->param; ad.m = c->adam_m; ad.v = c->adam_v; ad.grad = c->grad; ad.P = c->P_dev;
@@ -663,9 +664,9 @@ rslrl_status rslrl_ppo_update_steps(rslrl_ctx* c, int32_t max_steps, rslrl_updat
             ad.adaptive = pc.adaptive_lr; ad.max_norm = pc.max_grad_norm;
             ad.b1 = pc.adam_b1; ad.b2 = pc.adam_b2; ad.eps = pc.adam_eps;
             ad.stats_row = c->stats_dev + (size_t)done_steps * 8;
+            if (c->umma) umma_fill_cvt(c->umma, &ad);
             CU(c, launch_adam(ad, c->stream));
             c->parity ^= 1;
-            if (c->umma) CU(c, umma_refresh_weights(c->umma));
         }
     }
     c->iteration++;

@@ -108,10 +108,9 @@ struct GatherArgs {
     __nv_bfloat16* x_a16; __nv_bfloat16* x_c16; int ldxa16, ldxc16;
     float* act_mb; float* mu_old; float* sigma_old;         // [R][as], [Bmb][as], [Bmb][as]
     float* logp_old; float* v_old; float* ret; float* adv_mb;   // [Bmb]
-    int* rows_out;                                          // [Bmb] source indices (may be null)
+    const int* rows;                                        // [Bmb] source transition of every minibatch row
     int Bmb; int sym;
     SymTables st;
-    uint32_t seed_lo, seed_hi, iteration, epoch, batch, first;   // first = k * Bmb
 };
 cudaError_t launch_gather(const GatherArgs& a, cudaStream_t stream);
 cudaError_t launch_perm_rows(uint64_t seed, uint32_t iteration, uint32_t epoch, uint32_t batch,
@@ -144,19 +143,28 @@ struct HeadLossArgs {
 int head_loss_blocks(int Bmb);
 int head_partial_stride();
 cudaError_t launch_head_loss(const HeadLossArgs& a, cudaStream_t stream);
-// Sums the head_loss block partials: loss sums -> loss_sums[0..LS_COUNT), entropy ->
-// loss_sums[LS_COUNT], head-bias and log_std gradients -> split 0 of the gradient partials.
-cudaError_t launch_head_finalize(const float* block_partials, int nblocks, float* partials0, int off_ba,
-                                 int off_logstd, int off_bc, int A, float entropy_coef,
-                                 const float* log_std, float* loss_sums, cudaStream_t stream);
 
 struct ReduceArgs {
     const float* partials; int splits; long long split_stride;   // gradient partials [splits][P]
     float* grad; int P;                                            // padded device layout
     float* sumsq_partials;          // [reduce_blocks(P)]
+    // head_loss block partials: the head-bias and log_std gradients and the loss sums are
+    // finished here (loss sums -> loss_sums[0..LS_COUNT), entropy -> loss_sums[LS_COUNT])
+    const float* block_partials; int nblocks;
+    int off_ba, off_logstd, off_bc, A;
+    float entropy_coef; const float* log_std; float* loss_sums;
 };
 int reduce_blocks(int P);
 cudaError_t launch_reduce(const ReduceArgs& a, cudaStream_t stream);
+
+// One hidden layer's low-precision operand copies (see the tensor-core engine).
+struct CvtRange {
+    int w_off, b_off, in, out, out_p;          // location in the padded FP32 parameter vector
+    __nv_bfloat16* wt; int ld_wt;               // [out][ld_wt]
+    __nv_bfloat16* wn; int ld_wn;               // [in][ld_wn], may be null
+    float* bias_pad;                            // [>= out] zero-padded FP32 bias copy
+};
+constexpr int kMaxCvt = 16;
 
 struct AdamArgs {
     float* param; float* m; float* v; const float* grad; int P;
@@ -169,6 +177,8 @@ struct AdamArgs {
     float lr_min, lr_max, lr_factor, desired_kl; int adaptive;
     float max_norm, b1, b2, eps;
     float* stats_row;               // [8]: surr, value, entropy, sym, kl, grad_norm, lr, nonfinite
+    // BF16 mode: the operand copies of the weights are refreshed by the same pass
+    int n_cvt; CvtRange cvt[kMaxCvt];
 };
 cudaError_t launch_adam(const AdamArgs& a, cudaStream_t stream);
 

@@ -734,6 +734,20 @@ void umma_destroy(UmmaEngine* e) {
     delete e;
 }
 
+void umma_fill_cvt(UmmaEngine* e, AdamArgs* a) {
+    const UmmaSetup& s = e->s;
+    a->n_cvt = 0;
+    for (int ni = 0; ni < 2; ++ni)
+        for (int l = 0; l < e->nh[ni] && a->n_cvt < kMaxCvt; ++l) {
+            CvtRange& c = a->cvt[a->n_cvt++];
+            c.w_off = (int)s.w_off[ni][l]; c.b_off = (int)s.b_off[ni][l];
+            c.in = s.in[ni][l]; c.out = s.out[ni][l]; c.out_p = s.out_p[ni][l];
+            c.wt = e->wt[ni][l]; c.ld_wt = l == 0 ? e->kp[ni] : e->pw[ni][l - 1];
+            c.wn = l > 0 ? e->wn[ni][l] : nullptr; c.ld_wn = e->pw[ni][l];
+            c.bias_pad = e->bias_pad[ni][l];
+        }
+}
+
 cudaError_t umma_refresh_weights(UmmaEngine* e) {
     dim3 grid(std::max(1, std::min(64, (e->cvt_max + 255) / 256)), e->n_cvt);
     LaunchScope scope_("convert_weights", e->s.stream);

@@ -25,8 +25,11 @@ UmmaEngine* umma_create(const UmmaSetup& s, std::string* err);
 void umma_destroy(UmmaEngine* e);
 // Number of 128-row x <=256-column output tiles of all weight gradients (for choosing splits).
 int umma_wgrad_tiles(const UmmaSetup& s);
-// Re-derive the low-precision operand copies of the weights from the FP32 masters.
+// Re-derive the low-precision operand copies of the weights from the FP32 masters (after
+// rslrl_set_params; the optimiser step refreshes them itself, see umma_fill_cvt).
 cudaError_t umma_refresh_weights(UmmaEngine* e);
+// Tell the Adam kernel where the operand copies of every hidden layer live.
+void umma_fill_cvt(UmmaEngine* e, AdamArgs* a);
 // Hidden layers on N rollout rows.  d_obs_* are dense [N][dim] FP32 rows; when store_* is not
 // null the padded FP32 copy of the observations is also written there (row strides sa / sc).
 // Returns the last hidden activations of both nets (actor's only when do_actor).

@@ -12,9 +12,9 @@ namespace {
 constexpr float kHalfLog2Pi = 0.91893853320467274178f;
 
 // =======================================================================================
-// Gather.  A block takes 32 minibatch rows: one warp resolves their source transitions through
-// the Feistel shuffle (one row per lane), then all warps stream the rows into the minibatch
-// buffers.
+// Gather.  The epoch's shuffle is resolved once by perm_rows_kernel (one thread per index);
+// here one warp per minibatch row reads its source index and streams the row (float4 per
+// lane) into the minibatch buffers.
 // =======================================================================================
 template <bool BF16>
 __device__ __forceinline__ void copy_obs_row(const float* __restrict__ src, int dim, int ld_src,
@@ -45,65 +45,45 @@ __device__ __forceinline__ void copy_obs_row(const float* __restrict__ src, int 
     }
 }
 
-constexpr int kGatherRows = 32;      // minibatch rows per block
-
 template <bool BF16>
 __global__ void __launch_bounds__(256) gather_kernel(const GatherArgs a) {
-    __shared__ uint32_t s_src[kGatherRows];
-    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
-    PermKey pk{a.seed_lo, a.seed_hi, a.iteration, a.epoch, a.batch, feistel_half_bits(a.batch)};
-    for (int j0 = blockIdx.x * kGatherRows; j0 < a.Bmb; j0 += gridDim.x * kGatherRows) {
-        // Phase 1: warp 0 resolves the source transition of the block's rows, one row per lane
-        // (the shuffle costs a few hundred integer instructions: once per row, not per lane),
-        // and moves the per-row scalars.
-        if (warp == 0) {
-            const int jm = j0 + lane;
-            if (jm < a.Bmb) {
-                const uint32_t src = feistel_permute(pk, a.first + (uint32_t)jm);
-                s_src[lane] = src;
-                if (a.rows_out) a.rows_out[jm] = (int)src;
-                a.logp_old[jm] = a.logp[src];
-                a.v_old[jm] = a.values[src];
-                a.ret[jm] = a.returns[src];
-                a.adv_mb[jm] = a.adv[src];
-            }
-        }
-        __syncthreads();
-        // Phase 2: each warp streams its share of the rows (float4 per lane).
-        const int nrows = min(kGatherRows, a.Bmb - j0);
-        for (int rr = warp; rr < nrows; rr += 8) {
-            const int j = j0 + rr;
-            const uint32_t src = s_src[rr];
-            const int t = (int)(src / (uint32_t)a.N);
-            const float* oa = a.obs_a + (size_t)src * a.sa;
-            const int ldxa = BF16 ? a.ldxa16 : a.ldxa;
-            copy_obs_row<BF16>(oa, a.Da, a.sa, a.x_a ? a.x_a + (size_t)j * ldxa : nullptr,
-                               a.x_a16 ? a.x_a16 + (size_t)j * ldxa : nullptr, ldxa, nullptr, nullptr, lane);
+    const int lane = threadIdx.x & 31;
+    const int warps = (gridDim.x * blockDim.x) >> 5;
+    for (int j = (blockIdx.x * blockDim.x + threadIdx.x) >> 5; j < a.Bmb; j += warps) {
+        const uint32_t src = (uint32_t)a.rows[j];
+        const int t = (int)(src / (uint32_t)a.N);
+        // the four per-row scalars move on four lanes
+        if (lane == 0) a.logp_old[j] = a.logp[src];
+        else if (lane == 1) a.v_old[j] = a.values[src];
+        else if (lane == 2) a.ret[j] = a.returns[src];
+        else if (lane == 3) a.adv_mb[j] = a.adv[src];
+        const float* oa = a.obs_a + (size_t)src * a.sa;
+        const int ldxa = BF16 ? a.ldxa16 : a.ldxa;
+        copy_obs_row<BF16>(oa, a.Da, a.sa, a.x_a ? a.x_a + (size_t)j * ldxa : nullptr,
+                           a.x_a16 ? a.x_a16 + (size_t)j * ldxa : nullptr, ldxa, nullptr, nullptr, lane);
+        if (a.sym)
+            copy_obs_row<BF16>(oa, a.Da, a.sa, a.x_a ? a.x_a + (size_t)(j + a.Bmb) * ldxa : nullptr,
+                               a.x_a16 ? a.x_a16 + (size_t)(j + a.Bmb) * ldxa : nullptr, ldxa,
+                               a.st.obs_perm, a.st.obs_sign, lane);
+        if (!a.shared_obs) {
+            const float* oc = a.obs_c + (size_t)src * a.sc;
+            const int ldxc = BF16 ? a.ldxc16 : a.ldxc;
+            copy_obs_row<BF16>(oc, a.Dc, a.sc, a.x_c ? a.x_c + (size_t)j * ldxc : nullptr,
+                               a.x_c16 ? a.x_c16 + (size_t)j * ldxc : nullptr, ldxc, nullptr, nullptr, lane);
             if (a.sym)
-                copy_obs_row<BF16>(oa, a.Da, a.sa, a.x_a ? a.x_a + (size_t)(j + a.Bmb) * ldxa : nullptr,
-                                   a.x_a16 ? a.x_a16 + (size_t)(j + a.Bmb) * ldxa : nullptr, ldxa,
-                                   a.st.obs_perm, a.st.obs_sign, lane);
-            if (!a.shared_obs) {
-                const float* oc = a.obs_c + (size_t)src * a.sc;
-                const int ldxc = BF16 ? a.ldxc16 : a.ldxc;
-                copy_obs_row<BF16>(oc, a.Dc, a.sc, a.x_c ? a.x_c + (size_t)j * ldxc : nullptr,
-                                   a.x_c16 ? a.x_c16 + (size_t)j * ldxc : nullptr, ldxc, nullptr, nullptr, lane);
-                if (a.sym)
-                    copy_obs_row<BF16>(oc, a.Dc, a.sc, a.x_c ? a.x_c + (size_t)(j + a.Bmb) * ldxc : nullptr,
-                                       a.x_c16 ? a.x_c16 + (size_t)(j + a.Bmb) * ldxc : nullptr, ldxc,
-                                       a.st.cobs_perm, a.st.cobs_sign, lane);
-            }
-            const float* act = a.actions + (size_t)src * a.as;
-            for (int c = lane; c < a.as; c += 32) {
-                a.act_mb[(size_t)j * a.as + c] = act[c];
-                a.mu_old[(size_t)j * a.as + c] = a.mu[(size_t)src * a.as + c];
-                a.sigma_old[(size_t)j * a.as + c] = a.sigma[(size_t)t * a.as + c];
-                if (a.sym)
-                    a.act_mb[(size_t)(j + a.Bmb) * a.as + c] =
-                        c < a.A ? a.st.act_sign[c] * act[a.st.act_perm[c]] : 0.f;
-            }
+                copy_obs_row<BF16>(oc, a.Dc, a.sc, a.x_c ? a.x_c + (size_t)(j + a.Bmb) * ldxc : nullptr,
+                                   a.x_c16 ? a.x_c16 + (size_t)(j + a.Bmb) * ldxc : nullptr, ldxc,
+                                   a.st.cobs_perm, a.st.cobs_sign, lane);
         }
-        __syncthreads();
+        const float* act = a.actions + (size_t)src * a.as;
+        for (int c = lane; c < a.as; c += 32) {
+            a.act_mb[(size_t)j * a.as + c] = act[c];
+            a.mu_old[(size_t)j * a.as + c] = a.mu[(size_t)src * a.as + c];
+            a.sigma_old[(size_t)j * a.as + c] = a.sigma[(size_t)t * a.as + c];
+            if (a.sym)
+                a.act_mb[(size_t)(j + a.Bmb) * a.as + c] =
+                    c < a.A ? a.st.act_sign[c] * act[a.st.act_perm[c]] : 0.f;
+        }
     }
 }
 
@@ -436,60 +416,68 @@ __global__ void __launch_bounds__(kHLThreads) head_loss_kernel(const HeadLossArg
 }
 
 // =======================================================================================
-// Head partial finalisation: sums the head_loss block partials in block order and drops the
-// head-bias / log_std gradients into split 0 of the weight-gradient partials, the loss sums
-// into loss_sums.  One block.
-// =======================================================================================
-__global__ void __launch_bounds__(256) head_finalize_kernel(const float* __restrict__ block_partials,
-                                                            int nblocks, float* __restrict__ partials0,
-                                                            int off_ba, int off_logstd, int off_bc,
-                                                            int A, float entropy_coef,
-                                                            const float* __restrict__ log_std,
-                                                            float* __restrict__ loss_sums) {
-    if (threadIdx.x == 0) {   // policy entropy of the parameters this step's forward used
-        float ent = 0.f;
-        for (int i = 0; i < A; ++i) ent += 0.5f + kHalfLog2Pi + log_std[i];
-        loss_sums[LS_COUNT] = ent;
-    }
-    // one warp per entry: lane l adds blocks l, l+32, ... in order, then a fixed shuffle tree
-    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5, nwarps = blockDim.x >> 5;
-    for (int e = warp; e < kPartialStride; e += nwarps) {
-        if (e >= 5 && e < 8) continue;
-        if (e >= 8 && e < 8 + kMaxActions && e - 8 >= A) continue;
-        if (e >= 8 + kMaxActions && e - 8 - kMaxActions >= A) continue;
-        float s = 0.f;
-        for (int b = lane; b < nblocks; b += 32) s += block_partials[(size_t)b * kPartialStride + e];
-#pragma unroll
-        for (int o = 16; o > 0; o >>= 1) s += __shfl_down_sync(0xffffffffu, s, o);
-        if (lane != 0) continue;
-        if (e < LS_COUNT) loss_sums[e] = s;
-        else if (e == 4) partials0[off_bc] = s;
-        else if (e < 8 + kMaxActions) partials0[off_ba + e - 8] = s;
-        else partials0[off_logstd + e - 8 - kMaxActions] = s - entropy_coef;
-    }
-}
-
-// =======================================================================================
 // Gradient reduction: grad[p] = sum over splits (fixed order), plus a per-block sum of squares.
+// The head-bias and log_std entries come from the head_loss block partials instead (summed in
+// block order), and block 0 also finishes the loss sums and the policy entropy.
 // =======================================================================================
 constexpr int kRedThreads = 256;
 constexpr int kRedPerThread = 4;
 
+__device__ __forceinline__ bool head_entry(const ReduceArgs& a, int p) {
+    return (p >= a.off_ba && p < a.off_ba + a.A) || (p >= a.off_logstd && p < a.off_logstd + a.A) || p == a.off_bc;
+}
+
+// grid = reduce_blocks(P) blocks over the parameter vector + one extra block for the entries
+// that come from the head/loss kernel and for the loss sums.
 __global__ void __launch_bounds__(kRedThreads) reduce_kernel(const ReduceArgs a) {
-    const int base = (blockIdx.x * kRedThreads + threadIdx.x) * kRedPerThread;   // P is a multiple of 4
+    __shared__ float ws[kRedThreads / 32];
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
     float sq = 0.f;
-    if (base < a.P) {
-        float4 s = make_float4(0.f, 0.f, 0.f, 0.f);
-        for (int sp = 0; sp < a.splits; ++sp) {
-            const float4 v = *reinterpret_cast<const float4*>(a.partials + (size_t)sp * a.split_stride + base);
-            s.x += v.x; s.y += v.y; s.z += v.z; s.w += v.w;
+    if (blockIdx.x + 1 < gridDim.x) {
+        const int base = (blockIdx.x * kRedThreads + threadIdx.x) * kRedPerThread;   // P is a multiple of 4
+        if (base < a.P) {
+            float4 s = make_float4(0.f, 0.f, 0.f, 0.f);
+            for (int sp = 0; sp < a.splits; ++sp) {
+                const float4 v = *reinterpret_cast<const float4*>(a.partials + (size_t)sp * a.split_stride + base);
+                s.x += v.x; s.y += v.y; s.z += v.z; s.w += v.w;
+            }
+            if ((base + 3 >= a.off_ba && base < a.off_logstd + a.A) || (base <= a.off_bc && base + 3 >= a.off_bc)) {
+                // a group that touches head entries: those are written (and squared) by the extra block
+                const float g[4] = {s.x, s.y, s.z, s.w};
+#pragma unroll
+                for (int q = 0; q < 4; ++q)
+                    if (!head_entry(a, base + q)) { a.grad[base + q] = g[q]; sq += g[q] * g[q]; }
+            } else {
+                *reinterpret_cast<float4*>(a.grad + base) = s;
+                sq = (s.x * s.x + s.y * s.y) + (s.z * s.z + s.w * s.w);
+            }
         }
-        *reinterpret_cast<float4*>(a.grad + base) = s;
-        sq = (s.x * s.x + s.y * s.y) + (s.z * s.z + s.w * s.w);
+    } else {
+        // one warp per entry: lane l adds blocks l, l+32, ... in order, then a fixed shuffle tree
+        const int entries = 2 * a.A + 1 + LS_COUNT;
+        for (int e = warp; e < entries; e += kRedThreads / 32) {
+            int slot, p = -1; float shift = 0.f;
+            if (e < a.A) { slot = 8 + e; p = a.off_ba + e; }
+            else if (e < 2 * a.A) { slot = 8 + kMaxActions + e - a.A; p = a.off_logstd + e - a.A; shift = -a.entropy_coef; }
+            else if (e == 2 * a.A) { slot = 4; p = a.off_bc; }
+            else slot = e - 2 * a.A - 1;                                   // loss sums
+            float s = 0.f;
+            for (int b = lane; b < a.nblocks; b += 32) s += a.block_partials[(size_t)b * kPartialStride + slot];
+#pragma unroll
+            for (int o = 16; o > 0; o >>= 1) s += __shfl_down_sync(0xffffffffu, s, o);
+            if (lane == 0) {
+                if (p >= 0) { s += shift; a.grad[p] = s; sq += s * s; }
+                else a.loss_sums[slot] = s;
+            }
+        }
+        if (threadIdx.x == 0) {   // entropy of the policy this step's forward used
+            float ent = 0.f;
+            for (int i = 0; i < a.A; ++i) ent += 0.5f + kHalfLog2Pi + a.log_std[i];
+            a.loss_sums[LS_COUNT] = ent;
+        }
     }
     sq = warp_sum(sq);
-    __shared__ float ws[kRedThreads / 32];
-    if ((threadIdx.x & 31) == 0) ws[threadIdx.x >> 5] = sq;
+    if (lane == 0) ws[warp] = sq;
     __syncthreads();
     if (threadIdx.x == 0) {
         float t = 0.f;
@@ -564,6 +552,31 @@ __global__ void __launch_bounds__(kAdamThreads) adam_kernel(const AdamArgs a) {
         reinterpret_cast<float4*>(a.param)[i] = make_float4(p[0], p[1], p[2], p[3]);
         reinterpret_cast<float4*>(a.m)[i] = make_float4(m[0], m[1], m[2], m[3]);
         reinterpret_cast<float4*>(a.v)[i] = make_float4(v[0], v[1], v[2], v[3]);
+        // BF16 mode: refresh the operand copies of the hidden-layer weights and biases in place.
+        // A group of four parameters lies in one row of one layer (rows are padded to 4).
+        const int idx = 4 * i;
+        for (int e = 0; e < a.n_cvt; ++e) {
+            const CvtRange& c = a.cvt[e];
+            if (idx >= c.w_off && idx < c.w_off + c.in * c.out_p) {
+                const int rel = idx - c.w_off, row = rel / c.out_p, o = rel - row * c.out_p;
+#pragma unroll
+                for (int q = 0; q < 4; ++q) {
+                    if (o + q < c.out) {
+                        const __nv_bfloat16 w = __float2bfloat16_rn(p[q]);
+                        c.wt[(size_t)(o + q) * c.ld_wt + row] = w;
+                        if (c.wn) c.wn[(size_t)row * c.ld_wn + o + q] = w;
+                    }
+                }
+                break;
+            }
+            if (idx >= c.b_off && idx < c.b_off + c.out_p) {
+                const int o = idx - c.b_off;
+#pragma unroll
+                for (int q = 0; q < 4; ++q)
+                    if (o + q < c.out) c.bias_pad[o + q] = p[q];
+                break;
+            }
+        }
     }
 }
 
@@ -618,16 +631,7 @@ cudaError_t launch_head_loss(const HeadLossArgs& a, cudaStream_t s) {
     return a.bf16_act ? launch_head_loss_np<__nv_bfloat16>(a, s) : launch_head_loss_np<float>(a, s);
 }
 
-cudaError_t launch_head_finalize(const float* block_partials, int nblocks, float* partials0, int off_ba,
-                                 int off_logstd, int off_bc, int A, float entropy_coef,
-                                 const float* log_std, float* loss_sums, cudaStream_t s) {
-    LaunchScope scope_("head_finalize", s);
-    head_finalize_kernel<<<1, 256, 0, s>>>(block_partials, nblocks, partials0, off_ba, off_logstd, off_bc, A,
-                                           entropy_coef, log_std, loss_sums);
-    return cudaGetLastError();
-}
-
-int reduce_blocks(int P) { return (P + kRedThreads * kRedPerThread - 1) / (kRedThreads * kRedPerThread); }
+int reduce_blocks(int P) { return (P + kRedThreads * kRedPerThread - 1) / (kRedThreads * kRedPerThread) + 1; }
 
 cudaError_t launch_reduce(const ReduceArgs& a, cudaStream_t s) {
     LaunchScope scope_("grad_reduce", s);
