@@ -16,73 +16,109 @@ constexpr float kHalfLog2Pi = 0.91893853320467274178f;
 // here one warp per minibatch row reads its source index and streams the row (float4 per
 // lane) into the minibatch buffers.
 // =======================================================================================
-template <bool BF16>
+// All loads of a row are issued before its first store: the destination arrays are plain
+// pointers, so a store in between would order the loads behind it.
+constexpr int kObsVec = 2;            // float4 pieces per lane held at once (32 lanes x 2 x 4 floats = 256 floats)
+
+__device__ __forceinline__ void store_obs_piece(float* dst, __nv_bfloat16* dst16, int c, const float4 v) {
+    if (dst16) {
+        __nv_bfloat162 lo = __floats2bfloat162_rn(v.x, v.y), hi = __floats2bfloat162_rn(v.z, v.w);
+        uint2 pk;
+        pk.x = *reinterpret_cast<uint32_t*>(&lo);
+        pk.y = *reinterpret_cast<uint32_t*>(&hi);
+        *reinterpret_cast<uint2*>(dst16 + c) = pk;
+    } else {
+        *reinterpret_cast<float4*>(dst + c) = v;
+    }
+}
+
+// dst row (ld_dst columns, pads zero) <- src row (ld_src columns, storage pad is zero); when perm
+// is given also the mirrored row dst_m[c] = sign[c] * src[perm[c]].
 __device__ __forceinline__ void copy_obs_row(const float* __restrict__ src, int dim, int ld_src,
-                                             float* __restrict__ dst, __nv_bfloat16* __restrict__ dst16,
+                                             float* dst, __nv_bfloat16* dst16, float* dst_m, __nv_bfloat16* dst16_m,
                                              int ld_dst, const int* __restrict__ perm,
                                              const float* __restrict__ sign, int lane) {
-    // ld_dst may exceed ld_src (the bf16 rows are padded further); pad columns are zero.
-    if (perm == nullptr) {
-        for (int c = lane * 4; c < ld_dst; c += 128) {
-            float4 v = make_float4(0.f, 0.f, 0.f, 0.f);
-            if (c < ld_src) v = *reinterpret_cast<const float4*>(src + c);   // storage pad is zero
-            if (BF16) {
-                __nv_bfloat162 lo = __floats2bfloat162_rn(v.x, v.y), hi = __floats2bfloat162_rn(v.z, v.w);
-                uint2 pk;
-                pk.x = *reinterpret_cast<uint32_t*>(&lo);
-                pk.y = *reinterpret_cast<uint32_t*>(&hi);
-                *reinterpret_cast<uint2*>(dst16 + c) = pk;
-            } else {
-                *reinterpret_cast<float4*>(dst + c) = v;
+    for (int c0 = 0; c0 < ld_dst; c0 += 128 * kObsVec) {
+        float4 v[kObsVec];
+        float4 m[kObsVec];
+#pragma unroll
+        for (int i = 0; i < kObsVec; ++i) {
+            const int c = c0 + 128 * i + lane * 4;
+            v[i] = make_float4(0.f, 0.f, 0.f, 0.f);
+            m[i] = v[i];
+            if (c < ld_src) v[i] = *reinterpret_cast<const float4*>(src + c);
+            if (perm && c < ld_dst) {
+                float t[4];
+#pragma unroll
+                for (int q = 0; q < 4; ++q) t[q] = c + q < dim ? sign[c + q] * src[perm[c + q]] : 0.f;
+                m[i] = make_float4(t[0], t[1], t[2], t[3]);
             }
         }
-    } else {
-        for (int c = lane; c < ld_dst; c += 32) {
-            const float v = c < dim ? sign[c] * src[perm[c]] : 0.f;
-            if (BF16) dst16[c] = __float2bfloat16_rn(v);
-            else dst[c] = v;
+#pragma unroll
+        for (int i = 0; i < kObsVec; ++i) {
+            const int c = c0 + 128 * i + lane * 4;
+            if (c < ld_dst) {
+                store_obs_piece(dst, dst16, c, v[i]);
+                if (perm) store_obs_piece(dst_m, dst16_m, c, m[i]);
+            }
         }
     }
 }
 
-template <bool BF16>
-__global__ void __launch_bounds__(256) gather_kernel(const GatherArgs a) {
+__global__ void __launch_bounds__(256, 3) gather_kernel(const GatherArgs a) {
     const int lane = threadIdx.x & 31;
     const int warps = (gridDim.x * blockDim.x) >> 5;
+    const bool bf16 = a.x_a16 != nullptr;
     for (int j = (blockIdx.x * blockDim.x + threadIdx.x) >> 5; j < a.Bmb; j += warps) {
         const uint32_t src = (uint32_t)a.rows[j];
         const int t = (int)(src / (uint32_t)a.N);
-        // the four per-row scalars move on four lanes
-        if (lane == 0) a.logp_old[j] = a.logp[src];
-        else if (lane == 1) a.v_old[j] = a.values[src];
-        else if (lane == 2) a.ret[j] = a.returns[src];
-        else if (lane == 3) a.adv_mb[j] = a.adv[src];
-        const float* oa = a.obs_a + (size_t)src * a.sa;
-        const int ldxa = BF16 ? a.ldxa16 : a.ldxa;
-        copy_obs_row<BF16>(oa, a.Da, a.sa, a.x_a ? a.x_a + (size_t)j * ldxa : nullptr,
-                           a.x_a16 ? a.x_a16 + (size_t)j * ldxa : nullptr, ldxa, nullptr, nullptr, lane);
-        if (a.sym)
-            copy_obs_row<BF16>(oa, a.Da, a.sa, a.x_a ? a.x_a + (size_t)(j + a.Bmb) * ldxa : nullptr,
-                               a.x_a16 ? a.x_a16 + (size_t)(j + a.Bmb) * ldxa : nullptr, ldxa,
-                               a.st.obs_perm, a.st.obs_sign, lane);
-        if (!a.shared_obs) {
-            const float* oc = a.obs_c + (size_t)src * a.sc;
-            const int ldxc = BF16 ? a.ldxc16 : a.ldxc;
-            copy_obs_row<BF16>(oc, a.Dc, a.sc, a.x_c ? a.x_c + (size_t)j * ldxc : nullptr,
-                               a.x_c16 ? a.x_c16 + (size_t)j * ldxc : nullptr, ldxc, nullptr, nullptr, lane);
-            if (a.sym)
-                copy_obs_row<BF16>(oc, a.Dc, a.sc, a.x_c ? a.x_c + (size_t)(j + a.Bmb) * ldxc : nullptr,
-                                   a.x_c16 ? a.x_c16 + (size_t)(j + a.Bmb) * ldxc : nullptr, ldxc,
-                                   a.st.cobs_perm, a.st.cobs_sign, lane);
+        // ---- loads of the small per-row items (lanes 0..3: scalars; lanes < as: action-sized rows)
+        float sc = 0.f;
+        if (lane == 0) sc = a.logp[src];
+        else if (lane == 1) sc = a.values[src];
+        else if (lane == 2) sc = a.returns[src];
+        else if (lane == 3) sc = a.adv[src];
+        float av[2], mv[2], sv[2], am[2];
+#pragma unroll
+        for (int h = 0; h < 2; ++h) {
+            const int c = lane + 32 * h;
+            av[h] = mv[h] = sv[h] = am[h] = 0.f;
+            if (c < a.as) {
+                av[h] = a.actions[(size_t)src * a.as + c];
+                mv[h] = a.mu[(size_t)src * a.as + c];
+                sv[h] = a.sigma[(size_t)t * a.as + c];
+                if (a.sym && c < a.A) am[h] = a.st.act_sign[c] * a.actions[(size_t)src * a.as + a.st.act_perm[c]];
+            }
         }
-        const float* act = a.actions + (size_t)src * a.as;
-        for (int c = lane; c < a.as; c += 32) {
-            a.act_mb[(size_t)j * a.as + c] = act[c];
-            a.mu_old[(size_t)j * a.as + c] = a.mu[(size_t)src * a.as + c];
-            a.sigma_old[(size_t)j * a.as + c] = a.sigma[(size_t)t * a.as + c];
-            if (a.sym)
-                a.act_mb[(size_t)(j + a.Bmb) * a.as + c] =
-                    c < a.A ? a.st.act_sign[c] * act[a.st.act_perm[c]] : 0.f;
+        // ---- observation rows (loads, then stores, inside copy_obs_row)
+        const int ldxa = bf16 ? a.ldxa16 : a.ldxa;
+        copy_obs_row(a.obs_a + (size_t)src * a.sa, a.Da, a.sa,
+                     bf16 ? nullptr : a.x_a + (size_t)j * ldxa, bf16 ? a.x_a16 + (size_t)j * ldxa : nullptr,
+                     (bf16 || !a.sym) ? nullptr : a.x_a + (size_t)(j + a.Bmb) * ldxa,
+                     (bf16 && a.sym) ? a.x_a16 + (size_t)(j + a.Bmb) * ldxa : nullptr,
+                     ldxa, a.sym ? a.st.obs_perm : nullptr, a.st.obs_sign, lane);
+        if (!a.shared_obs) {
+            const int ldxc = bf16 ? a.ldxc16 : a.ldxc;
+            copy_obs_row(a.obs_c + (size_t)src * a.sc, a.Dc, a.sc,
+                         bf16 ? nullptr : a.x_c + (size_t)j * ldxc, bf16 ? a.x_c16 + (size_t)j * ldxc : nullptr,
+                         (bf16 || !a.sym) ? nullptr : a.x_c + (size_t)(j + a.Bmb) * ldxc,
+                         (bf16 && a.sym) ? a.x_c16 + (size_t)(j + a.Bmb) * ldxc : nullptr,
+                         ldxc, a.sym ? a.st.cobs_perm : nullptr, a.st.cobs_sign, lane);
+        }
+        // ---- stores of the small items
+        if (lane == 0) a.logp_old[j] = sc;
+        else if (lane == 1) a.v_old[j] = sc;
+        else if (lane == 2) a.ret[j] = sc;
+        else if (lane == 3) a.adv_mb[j] = sc;
+#pragma unroll
+        for (int h = 0; h < 2; ++h) {
+            const int c = lane + 32 * h;
+            if (c < a.as) {
+                a.act_mb[(size_t)j * a.as + c] = av[h];
+                a.mu_old[(size_t)j * a.as + c] = mv[h];
+                a.sigma_old[(size_t)j * a.as + c] = sv[h];
+                if (a.sym) a.act_mb[(size_t)(j + a.Bmb) * a.as + c] = am[h];
+            }
         }
     }
 }
@@ -586,8 +622,7 @@ cudaError_t launch_gather(const GatherArgs& a, cudaStream_t s) {
     if (a.Bmb <= 0) return cudaSuccess;
     const int blocks = std::min((a.Bmb + 7) / 8, 148 * 8);
     LaunchScope scope_("gather", s);
-    if (a.x_a16) gather_kernel<true><<<blocks, 256, 0, s>>>(a);
-    else gather_kernel<false><<<blocks, 256, 0, s>>>(a);
+    gather_kernel<<<blocks, 256, 0, s>>>(a);
     return cudaGetLastError();
 }
 
