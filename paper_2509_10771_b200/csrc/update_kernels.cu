@@ -129,32 +129,18 @@ __global__ void perm_rows_kernel(PermKey pk, uint32_t first, int count, int* __r
 }
 
 // =======================================================================================
-// Head + loss.  One thread per minibatch row (and its mirrored twin): the thread walks the row
-// of last-hidden activations in 16-byte pieces against head weights broadcast from shared
-// memory, finishes the PPO loss terms of the row, and walks the row again to emit dL/dz of the
-// last hidden layers.  No cross-lane traffic until the block-level sums at the end.
-// NP = number of 16-action passes (actions are padded to 16 * NP in registers).
+// Head + loss.  Four threads per minibatch row (and its mirrored twin).  Thread q of the quad
+// owns the actions 4q .. 4q+3 (+16 per further pass): all four walk the whole row of
+// last-hidden activations in 16-byte pieces against head weights read from shared memory
+// (the quad reads one contiguous 64-byte span, lanes of equal q broadcast), so the heads need
+// no cross-lane traffic; the row's loss terms are finished with two shuffles; the backward walk
+// ends in a transposing reduction that leaves every thread with one finished 16-byte piece
+// of dL/dz to store.  NP = number of 16-action passes.
 // =======================================================================================
 constexpr int kHLThreads = 128;
+constexpr int kHLRows = kHLThreads / 4;               // minibatch rows per block
 constexpr int kPartialStride = 8 + 2 * kMaxActions;   // [0..3] loss sums, [4] db_critic, [8..) db_actor, dlog_std
 
-__device__ __forceinline__ void load8(const float* p, float (&h)[8]) {
-    const float4 a = *reinterpret_cast<const float4*>(p), b = *reinterpret_cast<const float4*>(p + 4);
-    h[0] = a.x; h[1] = a.y; h[2] = a.z; h[3] = a.w; h[4] = b.x; h[5] = b.y; h[6] = b.z; h[7] = b.w;
-}
-__device__ __forceinline__ void load8(const __nv_bfloat16* p, float (&h)[8]) {
-    const uint4 v = *reinterpret_cast<const uint4*>(p);
-    const uint32_t w[4] = {v.x, v.y, v.z, v.w};
-#pragma unroll
-    for (int e = 0; e < 4; ++e) {
-        const __nv_bfloat162 h2 = *reinterpret_cast<const __nv_bfloat162*>(&w[e]);
-        h[2 * e] = __low2float(h2); h[2 * e + 1] = __high2float(h2);
-    }
-}
-__device__ __forceinline__ void store8(float* p, const float (&v)[8]) {
-    *reinterpret_cast<float4*>(p) = make_float4(v[0], v[1], v[2], v[3]);
-    *reinterpret_cast<float4*>(p + 4) = make_float4(v[4], v[5], v[6], v[7]);
-}
 __device__ __forceinline__ void store8(__nv_bfloat16* p, const float (&v)[8]) {
     uint32_t w[4];
 #pragma unroll
@@ -164,27 +150,28 @@ __device__ __forceinline__ void store8(__nv_bfloat16* p, const float (&v)[8]) {
     }
     *reinterpret_cast<uint4*>(p) = make_uint4(w[0], w[1], w[2], w[3]);
 }
+__device__ __forceinline__ void store_piece(float* p, const float (&o)[4]) {
+    *reinterpret_cast<float4*>(p) = make_float4(o[0], o[1], o[2], o[3]);
+}
+__device__ __forceinline__ void store_piece(__nv_bfloat16* p, const float (&o)[8]) { store8(p, o); }
 
-// A block of kRowPieces consecutive 16-byte pieces of an activation row, fetched with all loads
-// in flight at once (the row walk is latency bound otherwise; longer blocks bloat the unrolled
-// code past the instruction cache).
-constexpr int kRowPieces = 4;
+// Four consecutive 16-byte pieces of an activation row, fetched with all loads in flight.
 template <typename T>
 struct RowBlock {
     static constexpr int EPV = 16 / (int)sizeof(T);     // elements per piece
-    static constexpr int N = kRowPieces * EPV;          // elements per block
-    uint4 v[kRowPieces];
+    static constexpr int N = 4 * EPV;                   // elements per block
+    uint4 v[4];
     __device__ __forceinline__ void load(const T* row, int k0, int ld) {
 #pragma unroll
-        for (int i = 0; i < kRowPieces; ++i)
-            if (k0 + i * EPV < ld) v[i] = *reinterpret_cast<const uint4*>(row + k0 + i * EPV);
+        for (int i = 0; i < 4; ++i)
+            v[i] = k0 + i * EPV < ld ? *reinterpret_cast<const uint4*>(row + k0 + i * EPV) : make_uint4(0u, 0u, 0u, 0u);
     }
-    __device__ __forceinline__ void unpack(int i, float (&h)[EPV]) const {
+    __device__ __forceinline__ static void unpack(const uint4 x, float (&h)[EPV]) {
         if (sizeof(T) == 4) {
-            h[0] = __uint_as_float(v[i].x); h[1] = __uint_as_float(v[i].y);
-            h[2] = __uint_as_float(v[i].z); h[3] = __uint_as_float(v[i].w);
+            h[0] = __uint_as_float(x.x); h[1] = __uint_as_float(x.y);
+            h[2] = __uint_as_float(x.z); h[3] = __uint_as_float(x.w);
         } else {
-            const uint32_t w[4] = {v[i].x, v[i].y, v[i].z, v[i].w};
+            const uint32_t w[4] = {x.x, x.y, x.z, x.w};
 #pragma unroll
             for (int e = 0; e < 4; ++e) {
                 const __nv_bfloat162 h2 = *reinterpret_cast<const __nv_bfloat162*>(&w[e]);
@@ -192,13 +179,10 @@ struct RowBlock {
             }
         }
     }
+    __device__ __forceinline__ uint4 pick(int q) const { return q == 0 ? v[0] : q == 1 ? v[1] : q == 2 ? v[2] : v[3]; }
 };
-__device__ __forceinline__ void store_piece(float* p, const float (&o)[4]) {
-    *reinterpret_cast<float4*>(p) = make_float4(o[0], o[1], o[2], o[3]);
-}
-__device__ __forceinline__ void store_piece(__nv_bfloat16* p, const float (&o)[8]) { store8(p, o); }
 
-// Block-wide sum in a fixed order: shuffle tree inside each warp, then warp 0 adds the warps.
+// Block-wide sum in a fixed order: shuffle tree inside each warp, then the warps in order.
 __device__ __forceinline__ float block_sum(float v, float* scratch /* [warps] */) {
 #pragma unroll
     for (int o = 16; o > 0; o >>= 1) v += __shfl_down_sync(0xffffffffu, v, o);
@@ -213,14 +197,16 @@ __device__ __forceinline__ float block_sum(float v, float* scratch /* [warps] */
 
 template <typename T, int NP>
 __global__ void __launch_bounds__(kHLThreads) head_loss_kernel(const HeadLossArgs a) {
-    constexpr int AP = 16 * NP;
+    constexpr int AP = 16 * NP;                          // padded number of actions
+    constexpr int AQ = 4 * NP;                           // actions per thread
+    constexpr int EPV = RowBlock<T>::EPV;
     extern __shared__ float smem[];
     const HeadParams& hp = a.hp;
     const int A = hp.A;
-    float* Wa_s = smem;                                 // [n_a][AP], zero padded
-    float* Wc_s = Wa_s + hp.n_a * AP;                   // [n_c]
-    float* mu_s = Wc_s + ((hp.n_c + 3) & ~3);           // [threads][AP + 1]  policy mean of the original row
-    float* red = mu_s + kHLThreads * (AP + 1);          // [warps]
+    float* Wa_s = smem;                                  // [n_a][AP], zero padded
+    float* Wc_s = Wa_s + hp.n_a * AP;                    // [n_c]
+    float* mu_s = Wc_s + ((hp.n_c + 3) & ~3);            // [rows][AP + 1]  policy mean of the original row
+    float* red = mu_s + kHLRows * (AP + 1);              // [warps]
     for (int e = threadIdx.x; e < hp.n_a * AP; e += kHLThreads) {
         const int k = e / AP, i = e % AP;
         Wa_s[e] = i < A ? hp.Wa[(size_t)k * hp.ldwa + i] : 0.f;
@@ -228,98 +214,104 @@ __global__ void __launch_bounds__(kHLThreads) head_loss_kernel(const HeadLossArg
     for (int k = threadIdx.x; k < hp.n_c; k += kHLThreads) Wc_s[k] = hp.Wc[(size_t)k * hp.ldwc];
     __syncthreads();
 
-    const int j = blockIdx.x * kHLThreads + threadIdx.x;
+    const int qt = threadIdx.x & 3;                      // position in the quad
+    const int row_local = threadIdx.x >> 2;
+    const int j = blockIdx.x * kHLRows + row_local;
     const bool live = j < a.Bmb;
+    const bool lead = qt == 0;                           // accounts the per-row scalars, writes dL/dV
+    const unsigned qmask = 0xFu << (threadIdx.x & 28);   // the four lanes of this quad
     const int R = a.sym ? 2 * a.Bmb : a.Bmb;
     const float inv_R = 1.0f / (float)R;
     const float inv_sym = 1.0f / ((float)a.Bmb * (float)A);
-    float s_surr = 0.f, s_val = 0.f, s_kl = 0.f, s_sym = 0.f, s_dbc = 0.f;
-    float s_dba[AP], s_dls[AP];
+    // slot s of this thread is action 16 (s / 4) + 4 qt + s % 4
+    float ls[AQ], ivar[AQ];
 #pragma unroll
-    for (int i = 0; i < AP; ++i) { s_dba[i] = 0.f; s_dls[i] = 0.f; }
+    for (int s = 0; s < AQ; ++s) {
+        const int i = 16 * (s >> 2) + 4 * qt + (s & 3);
+        ls[s] = i < A ? hp.log_std[i] : 0.f;
+        ivar[s] = __expf(-2.0f * ls[s]);                 // 1 / sigma^2
+    }
+    float s_surr = 0.f, s_val = 0.f, s_kl = 0.f, s_sym = 0.f, s_dbc = 0.f;
+    float s_dba[AQ], s_dls[AQ];
+#pragma unroll
+    for (int s = 0; s < AQ; ++s) { s_dba[s] = 0.f; s_dls[s] = 0.f; }
 
     if (live) {
         const float logp_old = a.logp_old[j], v_old = a.v_old[j], ret = a.ret[j], adv = a.adv[j];
-        float* mu_mine = mu_s + threadIdx.x * (AP + 1);
+        float* mu_row = mu_s + row_local * (AP + 1);
         for (int copy = 0; copy < (a.sym ? 2 : 1); ++copy) {
             const int r = j + copy * a.Bmb;
             const T* ha = reinterpret_cast<const T*>(a.Ha) + (size_t)r * a.ldha;
             const T* hc = reinterpret_cast<const T*>(a.Hc) + (size_t)r * a.ldhc;
-            // ---- heads ------------------------------------------------------------------
-            float mu[AP];
-#pragma unroll
-            for (int i = 0; i < AP; ++i) mu[i] = i < A ? hp.ba[i] : 0.f;
-            constexpr int EPV = RowBlock<T>::EPV;
             RowBlock<T> blk;
-            for (int k0 = 0; k0 < hp.n_a; k0 += RowBlock<T>::N) {   // row strides are multiples of 8
+            // ---- actor head: own actions over the whole row -------------------------------
+            float mu[AQ];
+#pragma unroll
+            for (int s = 0; s < AQ; ++s) {
+                const int i = 16 * (s >> 2) + 4 * qt + (s & 3);
+                mu[s] = i < A ? hp.ba[i] : 0.f;
+            }
+            for (int k0 = 0; k0 < hp.n_a; k0 += RowBlock<T>::N) {     // row strides are multiples of 8
                 blk.load(ha, k0, a.ldha);
 #pragma unroll
-                for (int pi = 0; pi < kRowPieces; ++pi) {
-                    if (k0 + pi * EPV >= hp.n_a) break;
+                for (int pi = 0; pi < 4; ++pi) {
                     float h[EPV];
-                    blk.unpack(pi, h);
+                    RowBlock<T>::unpack(blk.v[pi], h);
 #pragma unroll
                     for (int kk = 0; kk < EPV; ++kk) {
                         const int k = k0 + pi * EPV + kk;
                         if (k < hp.n_a) {
-                            const float4* w4 = reinterpret_cast<const float4*>(Wa_s + k * AP);
 #pragma unroll
-                            for (int i4 = 0; i4 < AP / 4; ++i4) {
-                                const float4 w = w4[i4];
-                                mu[4 * i4] = fmaf(h[kk], w.x, mu[4 * i4]); mu[4 * i4 + 1] = fmaf(h[kk], w.y, mu[4 * i4 + 1]);
-                                mu[4 * i4 + 2] = fmaf(h[kk], w.z, mu[4 * i4 + 2]); mu[4 * i4 + 3] = fmaf(h[kk], w.w, mu[4 * i4 + 3]);
+                            for (int p = 0; p < NP; ++p) {
+                                const float4 w = *reinterpret_cast<const float4*>(Wa_s + k * AP + 16 * p + 4 * qt);
+                                mu[4 * p] = fmaf(h[kk], w.x, mu[4 * p]); mu[4 * p + 1] = fmaf(h[kk], w.y, mu[4 * p + 1]);
+                                mu[4 * p + 2] = fmaf(h[kk], w.z, mu[4 * p + 2]); mu[4 * p + 3] = fmaf(h[kk], w.w, mu[4 * p + 3]);
                             }
                         }
                     }
                 }
             }
-            float v = hp.bc[0];
-            {
-                float v1 = 0.f, v2 = 0.f, v3 = 0.f;
-                for (int k0 = 0; k0 < hp.n_c; k0 += RowBlock<T>::N) {
-                    blk.load(hc, k0, a.ldhc);
+            // ---- critic head: the quad splits the row, piece pi goes to thread pi -------------
+            float v = 0.f;
+            for (int k0 = 0; k0 < hp.n_c; k0 += RowBlock<T>::N) {
+                const int kp = k0 + qt * EPV;
+                if (kp < hp.n_c) {
+                    float h[EPV];
+                    RowBlock<T>::unpack(*reinterpret_cast<const uint4*>(hc + kp), h);
 #pragma unroll
-                    for (int pi = 0; pi < kRowPieces; ++pi) {
-                        if (k0 + pi * EPV >= hp.n_c) break;
-                        float h[EPV];
-                        blk.unpack(pi, h);
-#pragma unroll
-                        for (int kk = 0; kk < EPV; kk += 4) {
-                            const int k = k0 + pi * EPV + kk;
-                            if (k < hp.n_c) v = fmaf(h[kk], Wc_s[k], v);
-                            if (k + 1 < hp.n_c) v1 = fmaf(h[kk + 1], Wc_s[k + 1], v1);
-                            if (k + 2 < hp.n_c) v2 = fmaf(h[kk + 2], Wc_s[k + 2], v2);
-                            if (k + 3 < hp.n_c) v3 = fmaf(h[kk + 3], Wc_s[k + 3], v3);
-                        }
-                    }
+                    for (int kk = 0; kk < EPV; ++kk)
+                        if (kp + kk < hp.n_c) v = fmaf(h[kk], Wc_s[kp + kk], v);
                 }
-                v += (v1 + v2) + v3;
             }
-            // ---- log-density, KL ---------------------------------------------------------
-            float dmu[AP];
+            v += __shfl_xor_sync(qmask, v, 1);
+            v += __shfl_xor_sync(qmask, v, 2);
+            v += hp.bc[0];
+            // ---- log-density, KL (own actions, then two shuffles) --------------------------------
+            float dmu[AQ];
             float lp = 0.f, kl = 0.f;
 #pragma unroll
-            for (int i = 0; i < AP; ++i) {
-                dmu[i] = 0.f;
+            for (int s = 0; s < AQ; ++s) {
+                const int i = 16 * (s >> 2) + 4 * qt + (s & 3);
+                dmu[s] = 0.f;
                 if (i < A) {
-                    const float ls = hp.log_std[i];
-                    const float iv = __expf(-2.0f * ls);              // 1 / sigma^2
-                    const float d = a.act_mb[(size_t)r * a.as + i] - mu[i];
-                    lp += -(d * d) * 0.5f * iv - ls - kHalfLog2Pi;
-                    dmu[i] = d * iv;                                    // d logp / d mu_i
+                    const float d = a.act_mb[(size_t)r * a.as + i] - mu[s];
+                    lp += -(d * d) * 0.5f * ivar[s] - ls[s] - kHalfLog2Pi;
+                    dmu[s] = d * ivar[s];                               // d logp / d mu_i
                     if (copy == 0) {
                         const float so = a.sigma_old[(size_t)j * a.as + i];
-                        const float dm = a.mu_old[(size_t)j * a.as + i] - mu[i];
-                        kl += (ls - logf(so)) + (so * so + dm * dm) * 0.5f * iv - 0.5f;
+                        const float dm = a.mu_old[(size_t)j * a.as + i] - mu[s];
+                        kl += (ls[s] - logf(so)) + (so * so + dm * dm) * 0.5f * ivar[s] - 0.5f;
                     }
                 }
             }
-            if (copy == 0) s_kl += kl;
+            lp += __shfl_xor_sync(qmask, lp, 1); lp += __shfl_xor_sync(qmask, lp, 2);
+            kl += __shfl_xor_sync(qmask, kl, 1); kl += __shfl_xor_sync(qmask, kl, 2);
+            if (copy == 0 && lead) s_kl += kl;
             // ---- surrogate ---------------------------------------------------------------
             const float ratio = expf(lp - logp_old);
             const float s1 = -adv * ratio;
             const float s2 = -adv * fminf(fmaxf(ratio, 1.0f - a.h.clip), 1.0f + a.h.clip);
-            s_surr += fmaxf(s1, s2);
+            if (lead) s_surr += fmaxf(s1, s2);
             const bool inside = ratio >= 1.0f - a.h.clip && ratio <= 1.0f + a.h.clip;
             const float dlogp = (inside || s1 > s2) ? s1 * inv_R : 0.f;
             // ---- value -------------------------------------------------------------------
@@ -328,108 +320,124 @@ __global__ void __launch_bounds__(kHLThreads) head_loss_kernel(const HeadLossArg
             if (a.h.use_clipped_value_loss) {
                 const float vc = v_old + fminf(fmaxf(v - v_old, -a.h.value_clip), a.h.value_clip);
                 const float e2 = (vc - ret) * (vc - ret);
-                s_val += fmaxf(e1, e2);
+                if (lead) s_val += fmaxf(e1, e2);
                 const bool vin = fabsf(v - v_old) <= a.h.value_clip;
                 dv = (vin || e1 > e2) ? 2.0f * (v - ret) : 0.f;
             } else {
-                s_val += e1;
+                if (lead) s_val += e1;
                 dv = 2.0f * (v - ret);
             }
             dv *= a.h.value_coef * inv_R;
-            s_dbc += dv;
+            if (lead) s_dbc += dv;
             // ---- dL/dmu, dL/dlog_std, symmetry -------------------------------------------
+            if (copy == 1) __syncwarp(qmask);                           // mu of the original row is in mu_row
 #pragma unroll
-            for (int i = 0; i < AP; ++i) {
+            for (int s = 0; s < AQ; ++s) {
+                const int i = 16 * (s >> 2) + 4 * qt + (s & 3);
                 if (i < A) {
-                    const float ls = hp.log_std[i];
-                    const float var = __expf(2.0f * ls);
-                    const float dlp_dmu = dmu[i];                       // (a - mu) / sigma^2
-                    s_dls[i] += dlogp * (dlp_dmu * dlp_dmu * var - 1.0f);
+                    const float dlp_dmu = dmu[s];                       // (a - mu) / sigma^2
+                    s_dls[s] += dlogp * (dlp_dmu * dlp_dmu * __expf(2.0f * ls[s]) - 1.0f);
                     float g = dlogp * dlp_dmu;
                     if (copy == 1) {
-                        const float diff = mu[i] - a.act_sign[i] * mu_mine[a.act_perm[i]];
+                        const float diff = mu[s] - a.act_sign[i] * mu_row[a.act_perm[i]];
                         s_sym += diff * diff;
                         g += a.h.sym_coef * 2.0f * diff * inv_sym;
                     }
-                    dmu[i] = g;
-                    s_dba[i] += g;
+                    dmu[s] = g;
+                    s_dba[s] += g;
                 }
             }
             if (copy == 0 && a.sym) {
 #pragma unroll
-                for (int i = 0; i < AP; ++i) mu_mine[i] = mu[i];
+                for (int s = 0; s < AQ; ++s) mu_row[16 * (s >> 2) + 4 * qt + (s & 3)] = mu[s];
             }
-            // ---- outputs -------------------------------------------------------------------
-            for (int i = 0; i < a.lddmu; i += 4) {
-                float4 o;
-                o.x = dmu[0]; o.y = 0.f; o.z = 0.f; o.w = 0.f;
+            // ---- row outputs -----------------------------------------------------------------
 #pragma unroll
-                for (int q = 0; q < AP; q += 4)
-                    if (q == i) o = make_float4(dmu[q], dmu[q + 1], dmu[q + 2], dmu[q + 3]);
-                *reinterpret_cast<float4*>(a.dmu + (size_t)r * a.lddmu + i) = o;
-            }
-            *reinterpret_cast<float4*>(a.dv + (size_t)r * 4) = make_float4(dv, 0.f, 0.f, 0.f);
-            if (a.dmu16) {
-#pragma unroll
-                for (int q = 0; q < AP; q += 8) {
-                    if (q < a.lddmu16) {
-                        const float o8[8] = {dmu[q], dmu[q + 1], dmu[q + 2], dmu[q + 3], dmu[q + 4], dmu[q + 5], dmu[q + 6], dmu[q + 7]};
-                        store8(a.dmu16 + (size_t)r * a.lddmu16 + q, o8);
-                    }
+            for (int p = 0; p < NP; ++p) {
+                const int c = 16 * p + 4 * qt;
+                if (c < a.lddmu)
+                    *reinterpret_cast<float4*>(a.dmu + (size_t)r * a.lddmu + c) =
+                        make_float4(dmu[4 * p], dmu[4 * p + 1], dmu[4 * p + 2], dmu[4 * p + 3]);
+                if (a.dmu16 && c < a.lddmu16) {
+                    __nv_bfloat162 lo = __floats2bfloat162_rn(dmu[4 * p], dmu[4 * p + 1]);
+                    __nv_bfloat162 hi = __floats2bfloat162_rn(dmu[4 * p + 2], dmu[4 * p + 3]);
+                    uint2 pk;
+                    pk.x = *reinterpret_cast<uint32_t*>(&lo); pk.y = *reinterpret_cast<uint32_t*>(&hi);
+                    *reinterpret_cast<uint2*>(a.dmu16 + (size_t)r * a.lddmu16 + c) = pk;
                 }
-                const float d8[8] = {dv, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f};
-                store8(a.dv16 + (size_t)r * a.lddv16, d8);
+                if (a.mu_out && c < a.as)
+                    *reinterpret_cast<float4*>(a.mu_out + (size_t)r * a.as + c) =
+                        make_float4(mu[4 * p], mu[4 * p + 1], mu[4 * p + 2], mu[4 * p + 3]);
             }
-            if (a.mu_out) for (int i = 0; i < A; ++i) {
-                float m = 0.f;
-#pragma unroll
-                for (int q = 0; q < AP; ++q) if (q == i) m = mu[q];
-                a.mu_out[(size_t)r * a.as + i] = m;
+            if (lead) {
+                *reinterpret_cast<float4*>(a.dv + (size_t)r * 4) = make_float4(dv, 0.f, 0.f, 0.f);
+                if (a.dv16) {
+                    const float d8[8] = {dv, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f};
+                    store8(a.dv16 + (size_t)r * a.lddv16, d8);
+                }
+                if (a.v_out) a.v_out[r] = v;
             }
-            if (a.v_out) a.v_out[r] = v;
-            // ---- dL/dz of the last hidden layers --------------------------------------------
+            // ---- dL/dz of the actor's last hidden layer --------------------------------------------
+            // every thread forms its actions' share of four pieces, then a transposing reduction
+            // (exchange two pieces with lane^2, one with lane^1) leaves thread q with piece q
             T* dza = reinterpret_cast<T*>(a.dZa) + (size_t)r * a.lddza;
             for (int k0 = 0; k0 < a.lddza; k0 += RowBlock<T>::N) {
                 blk.load(ha, k0, min(a.ldha, a.lddza));
+                float part[4][EPV];
 #pragma unroll
-                for (int pi = 0; pi < kRowPieces; ++pi) {
-                    if (k0 + pi * EPV >= a.lddza) break;
-                    float h[EPV], o[EPV];
-                    blk.unpack(pi, h);
+                for (int pi = 0; pi < 4; ++pi) {
 #pragma unroll
                     for (int kk = 0; kk < EPV; ++kk) {
                         const int k = k0 + pi * EPV + kk;
                         float acc = 0.f;
                         if (k < hp.n_a) {
-                            const float4* w4 = reinterpret_cast<const float4*>(Wa_s + k * AP);
-                            float acc1 = 0.f;
 #pragma unroll
-                            for (int i4 = 0; i4 < AP / 4; ++i4) {
-                                const float4 w = w4[i4];
-                                acc = fmaf(dmu[4 * i4], w.x, acc); acc1 = fmaf(dmu[4 * i4 + 1], w.y, acc1);
-                                acc = fmaf(dmu[4 * i4 + 2], w.z, acc); acc1 = fmaf(dmu[4 * i4 + 3], w.w, acc1);
+                            for (int p = 0; p < NP; ++p) {
+                                const float4 w = *reinterpret_cast<const float4*>(Wa_s + k * AP + 16 * p + 4 * qt);
+                                acc = fmaf(dmu[4 * p], w.x, acc); acc = fmaf(dmu[4 * p + 1], w.y, acc);
+                                acc = fmaf(dmu[4 * p + 2], w.z, acc); acc = fmaf(dmu[4 * p + 3], w.w, acc);
                             }
-                            acc = (acc + acc1) * elu_grad_from_h(h[kk], a.h.alpha);
                         }
-                        o[kk] = acc;
+                        part[pi][kk] = acc;
                     }
-                    store_piece(dza + k0 + pi * EPV, o);
                 }
-            }
-            T* dzc = reinterpret_cast<T*>(a.dZc) + (size_t)r * a.lddzc;
-            for (int k0 = 0; k0 < a.lddzc; k0 += RowBlock<T>::N) {
-                blk.load(hc, k0, min(a.ldhc, a.lddzc));
+                float half[2][EPV], tot[EPV];
 #pragma unroll
-                for (int pi = 0; pi < kRowPieces; ++pi) {
-                    if (k0 + pi * EPV >= a.lddzc) break;
-                    float h[EPV], o[EPV];
-                    blk.unpack(pi, h);
+                for (int pp = 0; pp < 2; ++pp) {
 #pragma unroll
                     for (int kk = 0; kk < EPV; ++kk) {
-                        const int k = k0 + pi * EPV + kk;
-                        o[kk] = k < hp.n_c ? dv * Wc_s[k] * elu_grad_from_h(h[kk], a.h.alpha) : 0.f;
+                        const float send = (qt & 2) ? part[pp][kk] : part[pp + 2][kk];
+                        const float keep = (qt & 2) ? part[pp + 2][kk] : part[pp][kk];
+                        half[pp][kk] = keep + __shfl_xor_sync(qmask, send, 2);
                     }
-                    store_piece(dzc + k0 + pi * EPV, o);
+                }
+#pragma unroll
+                for (int kk = 0; kk < EPV; ++kk) {
+                    const float send = (qt & 1) ? half[0][kk] : half[1][kk];
+                    const float keep = (qt & 1) ? half[1][kk] : half[0][kk];
+                    tot[kk] = keep + __shfl_xor_sync(qmask, send, 1);
+                }
+                const int kp = k0 + qt * EPV;                            // thread q finishes piece q
+                if (kp < a.lddza) {
+                    float h[EPV], o[EPV];
+                    RowBlock<T>::unpack(blk.pick(qt), h);
+#pragma unroll
+                    for (int kk = 0; kk < EPV; ++kk)
+                        o[kk] = kp + kk < hp.n_a ? tot[kk] * elu_grad_from_h(h[kk], a.h.alpha) : 0.f;
+                    store_piece(dza + kp, o);
+                }
+            }
+            // ---- critic: thread q handles piece q of every block -------------------------------------
+            T* dzc = reinterpret_cast<T*>(a.dZc) + (size_t)r * a.lddzc;
+            for (int k0 = 0; k0 < a.lddzc; k0 += RowBlock<T>::N) {
+                const int kp = k0 + qt * EPV;
+                if (kp < a.lddzc) {
+                    float h[EPV], o[EPV];
+                    RowBlock<T>::unpack(kp < a.ldhc ? *reinterpret_cast<const uint4*>(hc + kp) : make_uint4(0u, 0u, 0u, 0u), h);
+#pragma unroll
+                    for (int kk = 0; kk < EPV; ++kk)
+                        o[kk] = kp + kk < hp.n_c ? dv * Wc_s[kp + kk] * elu_grad_from_h(h[kk], a.h.alpha) : 0.f;
+                    store_piece(dzc + kp, o);
                 }
             }
         }
@@ -445,8 +453,11 @@ __global__ void __launch_bounds__(kHLThreads) head_loss_kernel(const HeadLossArg
 #pragma unroll
     for (int i = 0; i < AP; ++i) {
         if (i < A) {                                    // uniform across the block
-            t = block_sum(s_dba[i], red); if (threadIdx.x == 0) out[8 + i] = t;
-            t = block_sum(s_dls[i], red); if (threadIdx.x == 0) out[8 + kMaxActions + i] = t;
+            const bool mine = qt == ((i & 15) >> 2);    // the quad member that owns action i
+            constexpr int unused = 0; (void)unused;
+            const int s = 4 * (i >> 4) + (i & 3);
+            t = block_sum(mine ? s_dba[s] : 0.f, red); if (threadIdx.x == 0) out[8 + i] = t;
+            t = block_sum(mine ? s_dls[s] : 0.f, red); if (threadIdx.x == 0) out[8 + kMaxActions + i] = t;
         }
     }
 }
@@ -635,14 +646,14 @@ cudaError_t launch_perm_rows(uint64_t seed, uint32_t iteration, uint32_t epoch, 
     return cudaGetLastError();
 }
 
-int head_loss_blocks(int Bmb) { return std::max(1, (Bmb + kHLThreads - 1) / kHLThreads); }
+int head_loss_blocks(int Bmb) { return std::max(1, (Bmb + kHLRows - 1) / kHLRows); }
 int head_partial_stride() { return kPartialStride; }
 
 namespace {
 template <typename T, int NP>
 cudaError_t launch_head_loss_t(const HeadLossArgs& a, cudaStream_t s) {
     const int AP = 16 * NP;
-    const size_t smem = sizeof(float) * ((size_t)a.hp.n_a * AP + ((a.hp.n_c + 3) & ~3) + (size_t)kHLThreads * (AP + 1) +
+    const size_t smem = sizeof(float) * ((size_t)a.hp.n_a * AP + ((a.hp.n_c + 3) & ~3) + (size_t)kHLRows * (AP + 1) +
                                          kHLThreads / 32);
     cudaError_t e = cudaFuncSetAttribute(head_loss_kernel<T, NP>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
     if (e != cudaSuccess) return e;
