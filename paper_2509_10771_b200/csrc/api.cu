@@ -650,7 +650,7 @@ rslrl_status rslrl_ppo_update_steps(rslrl_ctx* c, int32_t max_steps, rslrl_updat
             ReduceArgs r{};
             r.partials = c->partials; r.splits = c->splits; r.split_stride = c->P_dev;
             r.grad = c->grad; r.P = c->P_dev; r.sumsq_partials = c->sumsq_partials;
-            r.block_partials = c->block_partials; r.nblocks = head_loss_blocks(c->Bmb);
+            r.block_partials = c->block_partials; r.nblocks = hl.nblocks_used;
             r.off_ba = (int)ha.b_off; r.off_logstd = (int)c->logstd_off; r.off_bc = (int)hc.b_off; r.A = A;
             r.entropy_coef = pc.entropy_coef; r.log_std = c->param + c->logstd_off; r.loss_sums = c->loss_sums;
             CU(c, launch_reduce(r, c->stream));

@@ -139,10 +139,14 @@ struct HeadLossArgs {
     void* dZa; void* dZc; int lddza, lddzc;           // dL/dz of the last hidden layers
     float* block_partials;          // [blocks][head_partial_stride()]  (losses, db_head, dlog_std)
     float* mu_out; float* v_out;    // optional copies of mu [R][as] and V [R] (may be null)
+    int nblocks_used;               // set by the launcher: rows of block_partials that were written
 };
-int head_loss_blocks(int Bmb);
+int head_loss_blocks(int Bmb);      // upper bound of nblocks_used (for sizing block_partials)
 int head_partial_stride();
-cudaError_t launch_head_loss(const HeadLossArgs& a, cudaStream_t stream);
+cudaError_t launch_head_loss(HeadLossArgs& a, cudaStream_t stream);
+// BF16 activations: the heads and dL/dz on warp-level tensor-core instructions.
+bool head_loss_mma_applicable(const HeadLossArgs& a);
+cudaError_t launch_head_loss_mma(HeadLossArgs& a, cudaStream_t stream);
 
 struct ReduceArgs {
     const float* partials; int splits; long long split_stride;   // gradient partials [splits][P]

@@ -651,18 +651,19 @@ int head_partial_stride() { return kPartialStride; }
 
 namespace {
 template <typename T, int NP>
-cudaError_t launch_head_loss_t(const HeadLossArgs& a, cudaStream_t s) {
+cudaError_t launch_head_loss_t(HeadLossArgs& a, cudaStream_t s) {
     const int AP = 16 * NP;
     const size_t smem = sizeof(float) * ((size_t)a.hp.n_a * AP + ((a.hp.n_c + 3) & ~3) + (size_t)kHLRows * (AP + 1) +
                                          kHLThreads / 32);
     cudaError_t e = cudaFuncSetAttribute(head_loss_kernel<T, NP>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
     if (e != cudaSuccess) return e;
+    a.nblocks_used = head_loss_blocks(a.Bmb);
     LaunchScope scope_("head_loss", s);
     head_loss_kernel<T, NP><<<head_loss_blocks(a.Bmb), kHLThreads, smem, s>>>(a);
     return cudaGetLastError();
 }
 template <typename T>
-cudaError_t launch_head_loss_np(const HeadLossArgs& a, cudaStream_t s) {
+cudaError_t launch_head_loss_np(HeadLossArgs& a, cudaStream_t s) {
     const int np = (a.hp.A + 15) / 16;
     if (np == 1) return launch_head_loss_t<T, 1>(a, s);
     if (np == 2) return launch_head_loss_t<T, 2>(a, s);
@@ -671,7 +672,8 @@ cudaError_t launch_head_loss_np(const HeadLossArgs& a, cudaStream_t s) {
 }
 }  // namespace
 
-cudaError_t launch_head_loss(const HeadLossArgs& a, cudaStream_t s) {
+cudaError_t launch_head_loss(HeadLossArgs& a, cudaStream_t s) {
+    if (head_loss_mma_applicable(a)) return launch_head_loss_mma(a, s);
     // row strides of the hidden activations must allow 16-byte pieces
     if ((a.ldha % 8) || (a.ldhc % 8) || (a.lddza % 8) || (a.lddzc % 8)) return cudaErrorInvalidValue;
     return a.bf16_act ? launch_head_loss_np<__nv_bfloat16>(a, s) : launch_head_loss_np<float>(a, s);
