@@ -645,7 +645,7 @@ rslrl_status rslrl_ppo_update_steps(rslrl_ctx* c, int32_t max_steps, rslrl_updat
             CU(c, launch_head_loss(hl, c->stream));
             // ---- backward ---------------------------------------------------------------
             if (c->prec == RSLRL_FP32) TRY(backward_fp32(c));
-            else CU(c, umma_update_backward(c->umma));
+            else CU(c, umma_update_backward(c->umma, hl.colsum_written != 0));
             // ---- reduce, clip, adaptive lr, Adam ------------------------------------------
             ReduceArgs r{};
             r.partials = c->partials; r.splits = c->splits; r.split_stride = c->P_dev;
@@ -653,6 +653,7 @@ rslrl_status rslrl_ppo_update_steps(rslrl_ctx* c, int32_t max_steps, rslrl_updat
             r.block_partials = c->block_partials; r.nblocks = hl.nblocks_used;
             r.off_ba = (int)ha.b_off; r.off_logstd = (int)c->logstd_off; r.off_bc = (int)hc.b_off; r.A = A;
             r.entropy_coef = pc.entropy_coef; r.log_std = c->param + c->logstd_off; r.loss_sums = c->loss_sums;
+            if (c->umma) umma_fill_bias_sources(c->umma, &r, hl);
             CU(c, launch_reduce(r, c->stream));
             AdamArgs ad{};
             ad.param = c->param; ad.m = c->adam_m; ad.v = c->adam_v; ad.grad = c->grad; ad.P = c->P_dev;

@@ -45,7 +45,8 @@ __device__ __forceinline__ float quad_sum(float v) {
 }
 
 // NT = number of 8-wide action tiles (actions padded to 8 * NT, NT even).
-template <int NT>
+// CS: also emit the block's column sums of dZa / dZc (partial bias gradients of the last hidden layers).
+template <int NT, bool CS>
 __global__ void __launch_bounds__(kThreads) head_loss_mma_kernel(const HeadLossArgs a) {
     constexpr int AP = 8 * NT;
     extern __shared__ __align__(16) uint8_t smem_raw[];
@@ -59,6 +60,11 @@ __global__ void __launch_bounds__(kThreads) head_loss_mma_kernel(const HeadLossA
     float* Wc_s = reinterpret_cast<float*>(Wn_s + 16 * ksa * lda);       // [16 ksc]
     float* mu_s = Wc_s + 16 * ksc;                                       // [warps][16][AP + 1]
     float* red = mu_s + kWarps * 16 * (AP + 1);                          // [warps][kPartialStride]
+    // [warps][8][cs_ld]: lane (g, t) keeps the running sums of its own columns of dZa | dZc
+    const int cs_ld = (16 * (ksa + ksc) + 31) / 32 * 32 + 8;              // = 8 (mod 32): conflict-free float2 accesses
+    float* cs_s = red + kWarps * kPartialStride;
+    if (CS)
+        for (int e = threadIdx.x; e < kWarps * 8 * cs_ld; e += kThreads) cs_s[e] = 0.f;
     for (int e = threadIdx.x; e < AP * 16 * ksa; e += kThreads) {
         const int i = e / (16 * ksa), k = e % (16 * ksa);
         const float w = (i < A && k < hp.n_a) ? hp.Wa[(size_t)k * hp.ldwa + i] : 0.f;
@@ -73,11 +79,13 @@ __global__ void __launch_bounds__(kThreads) head_loss_mma_kernel(const HeadLossA
     const int R = a.sym ? 2 * a.Bmb : a.Bmb;
     const float inv_R = 1.0f / (float)R;
     const float inv_sym = 1.0f / ((float)a.Bmb * (float)A);
-    const __nv_bfloat16* Ha = reinterpret_cast<const __nv_bfloat16*>(a.Ha);
-    const __nv_bfloat16* Hc = reinterpret_cast<const __nv_bfloat16*>(a.Hc);
-    __nv_bfloat16* dZa = reinterpret_cast<__nv_bfloat16*>(a.dZa);
-    __nv_bfloat16* dZc = reinterpret_cast<__nv_bfloat16*>(a.dZc);
+    // the activation rows that are read and the gradient rows that are written never overlap
+    const __nv_bfloat16* __restrict__ Ha = reinterpret_cast<const __nv_bfloat16*>(a.Ha);
+    const __nv_bfloat16* __restrict__ Hc = reinterpret_cast<const __nv_bfloat16*>(a.Hc);
+    __nv_bfloat16* __restrict__ dZa = reinterpret_cast<__nv_bfloat16*>(a.dZa);
+    __nv_bfloat16* __restrict__ dZc = reinterpret_cast<__nv_bfloat16*>(a.dZc);
     float* mu_w = mu_s + warp * 16 * (AP + 1);
+    float* cs_mine = cs_s + (warp * 8 + g) * cs_ld;
 
     // per-thread constants of its action columns: tile j -> actions 8j + 2t, 8j + 2t + 1
     float ls[NT][2], ivar[NT][2], var[NT][2], bias_a[NT][2];
@@ -109,12 +117,13 @@ __global__ void __launch_bounds__(kThreads) head_loss_mma_kernel(const HeadLossA
         const float adv[2] = {a.adv[jc0], a.adv[jc1]};
         for (int copy = 0; copy < (a.sym ? 2 : 1); ++copy) {
             const size_t r0 = (size_t)jc0 + (size_t)copy * a.Bmb, r1 = (size_t)jc1 + (size_t)copy * a.Bmb;
-            const __nv_bfloat16* ha0 = Ha + r0 * a.ldha; const __nv_bfloat16* ha1 = Ha + r1 * a.ldha;
-            const __nv_bfloat16* hc0 = Hc + r0 * a.ldhc; const __nv_bfloat16* hc1 = Hc + r1 * a.ldhc;
+            const __nv_bfloat16* __restrict__ ha0 = Ha + r0 * a.ldha; const __nv_bfloat16* __restrict__ ha1 = Ha + r1 * a.ldha;
+            const __nv_bfloat16* __restrict__ hc0 = Hc + r0 * a.ldhc; const __nv_bfloat16* __restrict__ hc1 = Hc + r1 * a.ldhc;
             // ---- heads ------------------------------------------------------------------------
             float mu[NT][4];
 #pragma unroll
             for (int j = 0; j < NT; ++j) { mu[j][0] = mu[j][2] = bias_a[j][0]; mu[j][1] = mu[j][3] = bias_a[j][1]; }
+#pragma unroll 4
             for (int ks = 0; ks < ksa; ++ks) {
                 uint32_t af[4];
                 af[0] = *reinterpret_cast<const uint32_t*>(ha0 + 16 * ks + 2 * t);
@@ -249,7 +258,8 @@ __global__ void __launch_bounds__(kThreads) head_loss_mma_kernel(const HeadLossA
                 df[ka][2] = pack_bf16(dmu[2 * ka + 1][0], dmu[2 * ka + 1][1]);
                 df[ka][3] = pack_bf16(dmu[2 * ka + 1][2], dmu[2 * ka + 1][3]);
             }
-            __nv_bfloat16* dza0 = dZa + r0 * a.lddza; __nv_bfloat16* dza1 = dZa + r1 * a.lddza;
+            __nv_bfloat16* __restrict__ dza0 = dZa + r0 * a.lddza; __nv_bfloat16* __restrict__ dza1 = dZa + r1 * a.lddza;
+#pragma unroll 4
             for (int jn = 0; jn < 2 * ksa; ++jn) {                        // 8 hidden units per step
                 float acc[4] = {0.f, 0.f, 0.f, 0.f};
 #pragma unroll
@@ -260,22 +270,33 @@ __global__ void __launch_bounds__(kThreads) head_loss_mma_kernel(const HeadLossA
                 const int col = 8 * jn + 2 * t;
                 const float2 h0 = unpack_bf16(*reinterpret_cast<const uint32_t*>(ha0 + col));
                 const float2 h1 = unpack_bf16(*reinterpret_cast<const uint32_t*>(ha1 + col));
-                if (live0) *reinterpret_cast<uint32_t*>(dza0 + col) =
-                    pack_bf16(acc[0] * elu_grad_from_h(h0.x, a.h.alpha), acc[1] * elu_grad_from_h(h0.y, a.h.alpha));
-                if (live1) *reinterpret_cast<uint32_t*>(dza1 + col) =
-                    pack_bf16(acc[2] * elu_grad_from_h(h1.x, a.h.alpha), acc[3] * elu_grad_from_h(h1.y, a.h.alpha));
+                const float z00 = acc[0] * elu_grad_from_h(h0.x, a.h.alpha), z01 = acc[1] * elu_grad_from_h(h0.y, a.h.alpha);
+                const float z10 = acc[2] * elu_grad_from_h(h1.x, a.h.alpha), z11 = acc[3] * elu_grad_from_h(h1.y, a.h.alpha);
+                if (live0) *reinterpret_cast<uint32_t*>(dza0 + col) = pack_bf16(z00, z01);
+                if (live1) *reinterpret_cast<uint32_t*>(dza1 + col) = pack_bf16(z10, z11);
+                if (CS) {                                                 // rows that are not live carry dL/dmu = 0
+                    float2* cs = reinterpret_cast<float2*>(cs_mine + col);
+                    const float2 o = *cs;
+                    *cs = make_float2(o.x + (z00 + z10), o.y + (z01 + z11));
+                }
             }
             // ---- critic: dz = dV * Wc * ELU'(h), element-wise on the same column pairs ------------------
-            __nv_bfloat16* dzc0 = dZc + r0 * a.lddzc; __nv_bfloat16* dzc1 = dZc + r1 * a.lddzc;
+            __nv_bfloat16* __restrict__ dzc0 = dZc + r0 * a.lddzc; __nv_bfloat16* __restrict__ dzc1 = dZc + r1 * a.lddzc;
+#pragma unroll 4
             for (int jn = 0; jn < 2 * ksc; ++jn) {
                 const int col = 8 * jn + 2 * t;
                 const float2 w = *reinterpret_cast<const float2*>(Wc_s + col);
                 const float2 h0 = unpack_bf16(*reinterpret_cast<const uint32_t*>(hc0 + col));
                 const float2 h1 = unpack_bf16(*reinterpret_cast<const uint32_t*>(hc1 + col));
-                if (live0) *reinterpret_cast<uint32_t*>(dzc0 + col) =
-                    pack_bf16(dv[0] * w.x * elu_grad_from_h(h0.x, a.h.alpha), dv[0] * w.y * elu_grad_from_h(h0.y, a.h.alpha));
-                if (live1) *reinterpret_cast<uint32_t*>(dzc1 + col) =
-                    pack_bf16(dv[1] * w.x * elu_grad_from_h(h1.x, a.h.alpha), dv[1] * w.y * elu_grad_from_h(h1.y, a.h.alpha));
+                const float z00 = dv[0] * w.x * elu_grad_from_h(h0.x, a.h.alpha), z01 = dv[0] * w.y * elu_grad_from_h(h0.y, a.h.alpha);
+                const float z10 = dv[1] * w.x * elu_grad_from_h(h1.x, a.h.alpha), z11 = dv[1] * w.y * elu_grad_from_h(h1.y, a.h.alpha);
+                if (live0) *reinterpret_cast<uint32_t*>(dzc0 + col) = pack_bf16(z00, z01);
+                if (live1) *reinterpret_cast<uint32_t*>(dzc1 + col) = pack_bf16(z10, z11);
+                if (CS) {                                                 // rows that are not live carry dV = 0
+                    float2* cs = reinterpret_cast<float2*>(cs_mine + 16 * ksa + col);
+                    const float2 o = *cs;
+                    *cs = make_float2(o.x + (z00 + z10), o.y + (z01 + z11));
+                }
             }
             if (a.sym) __syncwarp();                                      // mu_w is rewritten by the next original rows
         }
@@ -306,21 +327,37 @@ __global__ void __launch_bounds__(kThreads) head_loss_mma_kernel(const HeadLossA
         for (int w = 0; w < kWarps; ++w) s += red[w * kPartialStride + e];
         a.block_partials[(size_t)blockIdx.x * kPartialStride + e] = s;
     }
+    if (CS) {
+        // column sums of the block: the 8 row slots of each warp in order, then the warps in order
+        for (int c = threadIdx.x; c < 16 * (ksa + ksc); c += kThreads) {
+            float s = 0.f;
+            for (int w = 0; w < kWarps * 8; ++w) s += cs_s[w * cs_ld + c];
+            if (c < 16 * ksa) a.colsum_a[(size_t)blockIdx.x * a.lddza + c] = s;
+            else a.colsum_c[(size_t)blockIdx.x * a.lddzc + (c - 16 * ksa)] = s;
+        }
+    }
 }
+
+constexpr size_t kMaxColsumSmem = 96 * 1024;   // above this the column sums are left to their own kernel
 
 template <int NT>
 cudaError_t launch_nt(HeadLossArgs& a, cudaStream_t s) {
     const int AP = 8 * NT;
     const int ksa = (a.hp.n_a + 15) / 16, ksc = (a.hp.n_c + 15) / 16;
-    const size_t smem = 2 * ((size_t)AP * (16 * ksa + 8) + (size_t)16 * ksa * (AP + 8)) +
-                        4 * ((size_t)16 * ksc + (size_t)kWarps * 16 * (AP + 1) + (size_t)kWarps * kPartialStride);
-    cudaError_t e = cudaFuncSetAttribute(head_loss_mma_kernel<NT>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+    size_t smem = 2 * ((size_t)AP * (16 * ksa + 8) + (size_t)16 * ksa * (AP + 8)) +
+                  4 * ((size_t)16 * ksc + (size_t)kWarps * 16 * (AP + 1) + (size_t)kWarps * kPartialStride);
+    const size_t cs_bytes = 4 * (size_t)kWarps * 8 * ((16 * (ksa + ksc) + 31) / 32 * 32 + 8);
+    const bool cs = a.colsum_a && a.colsum_c && cs_bytes <= kMaxColsumSmem;
+    if (cs) smem += cs_bytes;
+    a.colsum_written = cs ? 1 : 0;
+    auto kernel = cs ? head_loss_mma_kernel<NT, true> : head_loss_mma_kernel<NT, false>;
+    cudaError_t e = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
     if (e != cudaSuccess) return e;
     const int tiles = (a.Bmb + 15) / 16;
     const int blocks = std::max(1, std::min((tiles + kWarps - 1) / kWarps, 148 * 4));
     a.nblocks_used = blocks;
     LaunchScope scope_("head_loss", s);
-    head_loss_mma_kernel<NT><<<blocks, kThreads, smem, s>>>(a);
+    kernel<<<blocks, kThreads, smem, s>>>(a);
     return cudaGetLastError();
 }
 

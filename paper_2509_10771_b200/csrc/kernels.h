@@ -140,6 +140,10 @@ struct HeadLossArgs {
     float* block_partials;          // [blocks][head_partial_stride()]  (losses, db_head, dlog_std)
     float* mu_out; float* v_out;    // optional copies of mu [R][as] and V [R] (may be null)
     int nblocks_used;               // set by the launcher: rows of block_partials that were written
+    // optional (tensor-core head kernel only): per-block column sums of dZa / dZc, i.e. partial bias
+    // gradients of the last hidden layers, [blocks][lddza] and [blocks][lddzc]
+    float* colsum_a; float* colsum_c;
+    int colsum_written;             // set by the launcher: 1 when those rows were produced
 };
 int head_loss_blocks(int Bmb);      // upper bound of nblocks_used (for sizing block_partials)
 int head_partial_stride();
@@ -147,6 +151,11 @@ cudaError_t launch_head_loss(HeadLossArgs& a, cudaStream_t stream);
 // BF16 activations: the heads and dL/dz on warp-level tensor-core instructions.
 bool head_loss_mma_applicable(const HeadLossArgs& a);
 cudaError_t launch_head_loss_mma(HeadLossArgs& a, cudaStream_t stream);
+
+// A run of parameters (hidden-layer biases) whose gradient is the sum of `nslots` partial rows
+// produced by the kernels that emit dZ, instead of the split partials.
+struct BiasSource { int p_off, n; const float* slots; int nslots, ld; };
+constexpr int kMaxBiasSources = 16;
 
 struct ReduceArgs {
     const float* partials; int splits; long long split_stride;   // gradient partials [splits][P]
@@ -157,6 +166,7 @@ struct ReduceArgs {
     const float* block_partials; int nblocks;
     int off_ba, off_logstd, off_bc, A;
     float entropy_coef; const float* log_std; float* loss_sums;
+    int n_bias; BiasSource bias[kMaxBiasSources];
 };
 int reduce_blocks(int P);
 cudaError_t launch_reduce(const ReduceArgs& a, cudaStream_t stream);

@@ -52,6 +52,7 @@ struct TcProblem {
     __nv_bfloat16* out16; int ld_out;
     const __nv_bfloat16* aux16; int ld_aux;
     float* out32; int ld_out32; long long split_stride;
+    float* colsum; int ld_colsum;  // data gradient: column sums of each 32-row slice, [4 m_tiles][ld_colsum] (may be null)
 };
 
 struct TcParams {
@@ -431,6 +432,20 @@ __global__ void __launch_bounds__(kThreads, 1) tc_gemm_kernel(const __grid_const
                 // rows at or beyond the tensor's extent are clipped by the store itself
                 if (lane == 0 && it.m0 + 32 * q < p.m_extent)
                     tma_store_2d(&P.tmOut[it.prob], tile, col0, it.m0 + 32 * q);
+                if (MODE == TC_DGRAD && p.colsum) {
+                    // partial bias gradient: lane l adds columns 2l, 2l+1 of the tile's 32 rows (rows past
+                    // the extent hold zeros); the 32 words of a row sit in 32 different banks
+                    float s0 = 0.f, s1 = 0.f;
+                    const uint8_t* mine = tile + ((lane & 3) << 2);
+#pragma unroll
+                    for (int r = 0; r < 32; ++r) {
+                        const uint32_t w = *reinterpret_cast<const uint32_t*>(mine + r * 128 + ((((lane >> 2) ^ (r & 7))) << 4));
+                        const __nv_bfloat162 v2 = *reinterpret_cast<const __nv_bfloat162*>(&w);
+                        s0 += __low2float(v2); s1 += __high2float(v2);
+                    }
+                    *reinterpret_cast<float2*>(p.colsum + (size_t)(it.m0 / BLOCK_M * 4 + q) * p.ld_colsum + col0 + 2 * lane) =
+                        make_float2(s0, s1);
+                }
             }
         }
         if (MODE != TC_WGRAD && lane == 0) {
@@ -516,11 +531,14 @@ struct UmmaEngine {
     __nv_bfloat16 *dmu16 = nullptr, *dv16 = nullptr;
     __nv_bfloat16 *wt[2][kMaxLayers] = {}, *wn[2][kMaxLayers] = {};
     float* bias_pad[2][kMaxLayers] = {};         // [pw] zero-padded copies of the hidden biases
+    float* bias_slots[2][kMaxLayers] = {};       // [4 m_tiles][pw] bias-gradient partials written by the data-gradient epilogue
+    int n_slots = 0, n_sources = 0;
+    float* head_slots[2] = {};                   // [head/loss blocks][pw of the last hidden layer]: its bias-gradient partials
     CvtEntry* cvt_dev = nullptr; int n_cvt = 0; int cvt_max = 0;
     int* error_dev = nullptr;
     int num_sms = 148;
     std::vector<TcParams> act_fwd, act_fwd_critic, upd_fwd, upd_dgrad, upd_wgrad;
-    ColsumBatch colsum{};
+    ColsumBatch colsum{}, colsum_rest{};         // all layers the epilogue does not cover / those minus the last ones
 };
 
 namespace {
@@ -681,6 +699,12 @@ UmmaEngine* umma_create(const UmmaSetup& s, std::string* err) {
             TcProblem& p = P.p[P.count - 1];
             p.out16 = e->dz[ni][l - 1]; p.ld_out = e->pw[ni][l - 1];
             p.aux16 = e->h[ni][l - 1]; p.ld_aux = e->pw[ni][l - 1];
+            if (e->n_sources < kMaxBiasSources) {     // beyond that the column-sum kernel takes the layer
+                e->n_sources++;
+                e->n_slots = 4 * p.m_tiles;
+                if (!ealloc(e, &e->bias_slots[ni][l - 1], (size_t)e->n_slots * e->pw[ni][l - 1])) return bail("allocation failed");
+                p.colsum = e->bias_slots[ni][l - 1]; p.ld_colsum = e->pw[ni][l - 1];
+            }
             if (!make_tmap(&P.tmOut[P.count - 1], p.out16, R, e->pw[ni][l - 1], e->pw[ni][l - 1], 64, 32) ||
                 !make_tmap(&P.tmAux[P.count - 1], p.aux16, R, e->pw[ni][l - 1], e->pw[ni][l - 1], 64, 32))
                 return bail("tensor map encoding failed");
@@ -716,14 +740,22 @@ UmmaEngine* umma_create(const UmmaSetup& s, std::string* err) {
             }
         flush();
     }
+    // ---- bias-gradient partials of the last hidden layers, written by the head/loss kernel ----
+    if (e->n_sources + 2 <= kMaxBiasSources)
+        for (int ni = 0; ni < 2; ++ni)
+            if (!ealloc(e, &e->head_slots[ni], (size_t)head_loss_blocks(s.Bmb) * e->pw[ni][e->nh[ni] - 1])) return bail("allocation failed");
     // ---- bias gradients of the hidden layers: column sums of dZ -------------------------------
     e->colsum.count = 0; e->colsum.splits = s.splits; e->colsum.split_stride = s.P_dev; e->colsum.is_bf16 = 1;
+    // (only of the last one of each net: the others come from the data-gradient epilogue)
     for (int ni = 0; ni < 2; ++ni)
         for (int l = 0; l < e->nh[ni]; ++l) {
+            if (e->bias_slots[ni][l]) continue;
             if (e->colsum.count == kMaxColsum) return bail("too many layers for the bias-gradient launch");
             ColsumProblem& q = e->colsum.p[e->colsum.count++];
             q.X = e->dz[ni][l]; q.out = s.partials + s.b_off[ni][l]; q.rows = R; q.n = s.out[ni][l]; q.ld = e->pw[ni][l];
+            if (l < e->nh[ni] - 1) e->colsum_rest.p[e->colsum_rest.count++] = q;
         }
+    e->colsum_rest.splits = e->colsum.splits; e->colsum_rest.split_stride = e->colsum.split_stride; e->colsum_rest.is_bf16 = 1;
     if (cudaStreamSynchronize(s.stream) != cudaSuccess) return bail("stream synchronisation failed");
     return e;
 }
@@ -745,6 +777,25 @@ void umma_fill_cvt(UmmaEngine* e, AdamArgs* a) {
             c.wt = e->wt[ni][l]; c.ld_wt = l == 0 ? e->kp[ni] : e->pw[ni][l - 1];
             c.wn = l > 0 ? e->wn[ni][l] : nullptr; c.ld_wn = e->pw[ni][l];
             c.bias_pad = e->bias_pad[ni][l];
+        }
+}
+
+void umma_fill_bias_sources(UmmaEngine* e, ReduceArgs* r, const HeadLossArgs& hl) {
+    const UmmaSetup& s = e->s;
+    r->n_bias = 0;
+    if (hl.colsum_written)
+        for (int ni = 0; ni < 2; ++ni) {
+            const int l = e->nh[ni] - 1;
+            BiasSource& b = r->bias[r->n_bias++];
+            b.p_off = (int)s.b_off[ni][l]; b.n = s.out[ni][l];
+            b.slots = e->head_slots[ni]; b.nslots = hl.nblocks_used; b.ld = e->pw[ni][l];
+        }
+    for (int ni = 0; ni < 2; ++ni)
+        for (int l = 0; l < e->nh[ni]; ++l) {
+            if (!e->bias_slots[ni][l]) continue;
+            BiasSource& b = r->bias[r->n_bias++];
+            b.p_off = (int)s.b_off[ni][l]; b.n = s.out[ni][l];
+            b.slots = e->bias_slots[ni][l]; b.nslots = e->n_slots; b.ld = e->pw[ni][l];
         }
 }
 
@@ -802,9 +853,10 @@ void umma_head_loss_targets(UmmaEngine* e, HeadLossArgs* a) {
     a->dZa = e->dz[0][e->nh[0] - 1]; a->lddza = a->ldha;
     a->dZc = e->dz[1][e->nh[1] - 1]; a->lddzc = a->ldhc;
     a->dmu16 = e->dmu16; a->lddmu16 = 64; a->dv16 = e->dv16; a->lddv16 = 64;
+    a->colsum_a = e->head_slots[0]; a->colsum_c = e->head_slots[1];
 }
 
-cudaError_t umma_update_backward(UmmaEngine* e) {
+cudaError_t umma_update_backward(UmmaEngine* e, bool last_bias_done) {
     cudaError_t err;
     for (const TcParams& P : e->upd_dgrad) {
         err = launch_tc<TC_DGRAD>(P, e->num_sms, e->s.stream);
@@ -814,7 +866,7 @@ cudaError_t umma_update_backward(UmmaEngine* e) {
         err = launch_tc<TC_WGRAD>(P, e->num_sms, e->s.stream);
         if (err != cudaSuccess) return err;
     }
-    return launch_colsum(e->colsum, e->s.stream);
+    return launch_colsum(last_bias_done ? e->colsum_rest : e->colsum, e->s.stream);
 }
 
 cudaError_t umma_read_error(UmmaEngine* e, int* host_code) {

@@ -30,6 +30,9 @@ int umma_wgrad_tiles(const UmmaSetup& s);
 cudaError_t umma_refresh_weights(UmmaEngine* e);
 // Tell the Adam kernel where the operand copies of every hidden layer live.
 void umma_fill_cvt(UmmaEngine* e, AdamArgs* a);
+// Tell the gradient reduction which hidden-layer bias gradients arrive as partial rows written by
+// the data-gradient epilogue and, when hl.colsum_written, by the head/loss kernel.
+void umma_fill_bias_sources(UmmaEngine* e, ReduceArgs* r, const HeadLossArgs& hl);
 // Hidden layers on N rollout rows.  d_obs_* are dense [N][dim] FP32 rows; when store_* is not
 // null the padded FP32 copy of the observations is also written there (row strides sa / sc).
 // Returns the last hidden activations of both nets (actor's only when do_actor).
@@ -42,8 +45,9 @@ cudaError_t umma_update_forward(UmmaEngine* e);
 // Point the head/loss kernel at the engine's last hidden activations and dZ buffers.
 void umma_head_loss_targets(UmmaEngine* e, HeadLossArgs* a);
 // Data gradients, weight-gradient partials and bias-gradient partials of all hidden layers
-// and heads, from the dZ / d_head buffers the head/loss kernel filled.
-cudaError_t umma_update_backward(UmmaEngine* e);
+// and heads, from the dZ / d_head buffers the head/loss kernel filled.  last_bias_done: the
+// head/loss kernel already produced the bias-gradient partials of the last hidden layers.
+cudaError_t umma_update_backward(UmmaEngine* e, bool last_bias_done);
 // Synchronises the stream and returns the device error code (0 = none; otherwise the role
 // whose bounded wait expired).
 cudaError_t umma_read_error(UmmaEngine* e, int* host_code);

@@ -473,6 +473,12 @@ constexpr int kRedPerThread = 4;
 __device__ __forceinline__ bool head_entry(const ReduceArgs& a, int p) {
     return (p >= a.off_ba && p < a.off_ba + a.A) || (p >= a.off_logstd && p < a.off_logstd + a.A) || p == a.off_bc;
 }
+__device__ __forceinline__ bool bias_entry(const ReduceArgs& a, int p) {
+    for (int b = 0; b < a.n_bias; ++b)
+        if (p >= a.bias[b].p_off && p < a.bias[b].p_off + a.bias[b].n) return true;
+    return false;
+}
+constexpr int kRedExtraBlocks = 24;     // blocks that finish the entries coming from partial rows
 
 // grid = reduce_blocks(P) blocks over the parameter vector + one extra block for the entries
 // that come from the head/loss kernel and for the loss sums.
@@ -480,7 +486,7 @@ __global__ void __launch_bounds__(kRedThreads) reduce_kernel(const ReduceArgs a)
     __shared__ float ws[kRedThreads / 32];
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
     float sq = 0.f;
-    if (blockIdx.x + 1 < gridDim.x) {
+    if (blockIdx.x + kRedExtraBlocks < gridDim.x) {
         const int base = (blockIdx.x * kRedThreads + threadIdx.x) * kRedPerThread;   // P is a multiple of 4
         if (base < a.P) {
             float4 s = make_float4(0.f, 0.f, 0.f, 0.f);
@@ -488,21 +494,62 @@ __global__ void __launch_bounds__(kRedThreads) reduce_kernel(const ReduceArgs a)
                 const float4 v = *reinterpret_cast<const float4*>(a.partials + (size_t)sp * a.split_stride + base);
                 s.x += v.x; s.y += v.y; s.z += v.z; s.w += v.w;
             }
-            if ((base + 3 >= a.off_ba && base < a.off_logstd + a.A) || (base <= a.off_bc && base + 3 >= a.off_bc)) {
-                // a group that touches head entries: those are written (and squared) by the extra block
+            bool special = (base + 3 >= a.off_ba && base < a.off_logstd + a.A) || (base <= a.off_bc && base + 3 >= a.off_bc);
+            for (int b = 0; b < a.n_bias; ++b)
+                special = special || (base + 3 >= a.bias[b].p_off && base < a.bias[b].p_off + a.bias[b].n);
+            if (special) {
+                // a group that touches entries finished by the extra blocks: those are written (and squared) there
                 const float g[4] = {s.x, s.y, s.z, s.w};
 #pragma unroll
                 for (int q = 0; q < 4; ++q)
-                    if (!head_entry(a, base + q)) { a.grad[base + q] = g[q]; sq += g[q] * g[q]; }
+                    if (!head_entry(a, base + q) && !bias_entry(a, base + q)) { a.grad[base + q] = g[q]; sq += g[q] * g[q]; }
             } else {
                 *reinterpret_cast<float4*>(a.grad + base) = s;
                 sq = (s.x * s.x + s.y * s.y) + (s.z * s.z + s.w * s.w);
             }
         }
     } else {
-        // one warp per entry: lane l adds blocks l, l+32, ... in order, then a fixed shuffle tree
+        // one warp per entry: lane l adds partial rows l, l+32, ... in order, then a fixed shuffle tree
+        const int xwarp = (blockIdx.x - (gridDim.x - kRedExtraBlocks)) * (kRedThreads / 32) + warp;
+        const int xwarps = kRedExtraBlocks * (kRedThreads / 32);
+        // bias sources: a warp takes 8 consecutive columns (two lanes x float4) and spreads the partial
+        // rows over its 16 lane pairs; every lane walks its rows in order, then a fixed butterfly
+        int total_units = 0;
+        for (int b = 0; b < a.n_bias; ++b) total_units += (a.bias[b].n + 7) / 8;
+        for (int u = xwarp; u < total_units; u += xwarps) {
+            int b = 0, ul = u;
+            while (ul >= (a.bias[b].n + 7) / 8) { ul -= (a.bias[b].n + 7) / 8; ++b; }
+            const BiasSource& src = a.bias[b];
+            const int c = 8 * ul + 4 * (lane & 1);                     // < ld: the rows are padded to 64 columns
+            const float* __restrict__ base = src.slots + c;
+            const size_t ld = (size_t)src.ld;
+            float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
+            int r = lane >> 1;
+            for (; r + 16 * 7 < src.nslots; r += 16 * 8) {
+                float4 v[8];
+#pragma unroll
+                for (int i = 0; i < 8; ++i) v[i] = __ldg(reinterpret_cast<const float4*>(base + (size_t)(r + 16 * i) * ld));
+#pragma unroll
+                for (int i = 0; i < 8; ++i) { acc.x += v[i].x; acc.y += v[i].y; acc.z += v[i].z; acc.w += v[i].w; }
+            }
+            for (; r < src.nslots; r += 16) {
+                const float4 v = __ldg(reinterpret_cast<const float4*>(base + (size_t)r * ld));
+                acc.x += v.x; acc.y += v.y; acc.z += v.z; acc.w += v.w;
+            }
+#pragma unroll
+            for (int o = 2; o < 32; o <<= 1) {
+                acc.x += __shfl_xor_sync(0xffffffffu, acc.x, o); acc.y += __shfl_xor_sync(0xffffffffu, acc.y, o);
+                acc.z += __shfl_xor_sync(0xffffffffu, acc.z, o); acc.w += __shfl_xor_sync(0xffffffffu, acc.w, o);
+            }
+            if (lane < 2) {
+                const float g[4] = {acc.x, acc.y, acc.z, acc.w};
+#pragma unroll
+                for (int q = 0; q < 4; ++q)
+                    if (c + q < src.n) { a.grad[src.p_off + c + q] = g[q]; sq += g[q] * g[q]; }
+            }
+        }
         const int entries = 2 * a.A + 1 + LS_COUNT;
-        for (int e = warp; e < entries; e += kRedThreads / 32) {
+        for (int e = xwarp; e < entries; e += xwarps) {
             int slot, p = -1; float shift = 0.f;
             if (e < a.A) { slot = 8 + e; p = a.off_ba + e; }
             else if (e < 2 * a.A) { slot = 8 + kMaxActions + e - a.A; p = a.off_logstd + e - a.A; shift = -a.entropy_coef; }
@@ -517,7 +564,7 @@ __global__ void __launch_bounds__(kRedThreads) reduce_kernel(const ReduceArgs a)
                 else a.loss_sums[slot] = s;
             }
         }
-        if (threadIdx.x == 0) {   // entropy of the policy this step's forward used
+        if (threadIdx.x == 0 && blockIdx.x + 1 == gridDim.x) {   // entropy of the policy this step's forward used
             float ent = 0.f;
             for (int i = 0; i < a.A; ++i) ent += 0.5f + kHalfLog2Pi + a.log_std[i];
             a.loss_sums[LS_COUNT] = ent;
@@ -673,13 +720,14 @@ cudaError_t launch_head_loss_np(HeadLossArgs& a, cudaStream_t s) {
 }  // namespace
 
 cudaError_t launch_head_loss(HeadLossArgs& a, cudaStream_t s) {
+    a.colsum_written = 0;
     if (head_loss_mma_applicable(a)) return launch_head_loss_mma(a, s);
     // row strides of the hidden activations must allow 16-byte pieces
     if ((a.ldha % 8) || (a.ldhc % 8) || (a.lddza % 8) || (a.lddzc % 8)) return cudaErrorInvalidValue;
     return a.bf16_act ? launch_head_loss_np<__nv_bfloat16>(a, s) : launch_head_loss_np<float>(a, s);
 }
 
-int reduce_blocks(int P) { return (P + kRedThreads * kRedPerThread - 1) / (kRedThreads * kRedPerThread) + 1; }
+int reduce_blocks(int P) { return (P + kRedThreads * kRedPerThread - 1) / (kRedThreads * kRedPerThread) + kRedExtraBlocks; }
 
 cudaError_t launch_reduce(const ReduceArgs& a, cudaStream_t s) {
     LaunchScope scope_("grad_reduce", s);
