@@ -105,6 +105,15 @@ __device__ __forceinline__ float elu_grad_from_h(float h, float alpha) {
     return h > 0.0f ? 1.0f : h + alpha;
 }
 
+// Programmatic dependent launch: a kernel launched with launch_chained() may be scheduled while its
+// predecessor in the stream still runs.  chain_begin() waits until every earlier grid has completed
+// and its memory is visible, then lets the successor be scheduled (which in turn waits for this grid
+// to complete): at most one waiting grid is resident at a time.  It comes before the first access to
+// global memory, by every thread, and is a no-op for a plainly launched kernel.
+__device__ __forceinline__ void chain_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+__device__ __forceinline__ void chain_release() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
+__device__ __forceinline__ void chain_begin() { chain_wait(); chain_release(); }
+
 __device__ __forceinline__ float warp_sum(float v) {
 #pragma unroll
     for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);

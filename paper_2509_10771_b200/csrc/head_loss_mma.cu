@@ -50,6 +50,7 @@ template <int NT, bool CS>
 __global__ void __launch_bounds__(kThreads) head_loss_mma_kernel(const HeadLossArgs a) {
     constexpr int AP = 8 * NT;
     extern __shared__ __align__(16) uint8_t smem_raw[];
+    chain_begin();
     const HeadParams& hp = a.hp;
     const int A = hp.A;
     const int ksa = (hp.n_a + 15) / 16, ksc = (hp.n_c + 15) / 16;        // 16-wide steps over the hidden units
@@ -357,8 +358,7 @@ cudaError_t launch_nt(HeadLossArgs& a, cudaStream_t s) {
     const int blocks = std::max(1, std::min((tiles + kWarps - 1) / kWarps, 148 * 4));
     a.nblocks_used = blocks;
     LaunchScope scope_("head_loss", s);
-    kernel<<<blocks, kThreads, smem, s>>>(a);
-    return cudaGetLastError();
+    return launch_chained(kernel, blocks, kThreads, smem, s, a);
 }
 
 }  // namespace

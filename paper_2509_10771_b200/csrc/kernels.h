@@ -2,6 +2,7 @@
 // include/rslrl_b200.h).  Every launcher enqueues on `stream` and returns the CUDA status of
 // the launch.
 #pragma once
+#include <utility>
 #include <cuda_runtime.h>
 #include <cuda_bf16.h>
 #include <stdint.h>
@@ -15,6 +16,21 @@ struct LaunchScope {
     ~LaunchScope();
     const char* name; cudaStream_t stream; int slot;
 };
+
+// Launch of a kernel that begins with chain_begin(): it may be scheduled before the preceding kernel
+// of the stream has drained (programmatic stream serialisation), which hides launch latency and
+// prologue.  Falls back to a plain launch when chained launches are switched off.
+bool chained_launches_enabled();
+template <typename... KArgs, typename... Args>
+cudaError_t launch_chained(void (*kernel)(KArgs...), dim3 grid, dim3 block, size_t smem, cudaStream_t s, Args&&... args) {
+    cudaLaunchConfig_t cfg{};
+    cfg.gridDim = grid; cfg.blockDim = block; cfg.dynamicSmemBytes = smem; cfg.stream = s;
+    cudaLaunchAttribute at[1];
+    at[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    at[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = at; cfg.numAttrs = chained_launches_enabled() ? 1 : 0;
+    return cudaLaunchKernelEx(&cfg, kernel, std::forward<Args>(args)...);
+}
 
 // ------------------------------------------------------------------------- SIMT FP32 GEMM
 // C[M x N] = op(A)[M x K] * op(B)[K x N] followed by an epilogue.  Leading dimensions are

@@ -6,6 +6,7 @@
 
 #include <atomic>
 #include <cstdio>
+#include <cstdlib>
 #include <cstring>
 #include <map>
 #include <mutex>
@@ -29,6 +30,12 @@ cudaEvent_t take_event() {
     return e;
 }
 }  // namespace
+
+// RSLRL_SERIAL_LAUNCHES=1 in the environment switches programmatic dependent launch off.
+bool chained_launches_enabled() {
+    static const bool on = [] { const char* v = std::getenv("RSLRL_SERIAL_LAUNCHES"); return !(v && v[0] == '1'); }();
+    return on;
+}
 
 LaunchScope::LaunchScope(const char* n, cudaStream_t s) : name(n), stream(s), slot(-1) {
     g_launches.fetch_add(1, std::memory_order_relaxed);

@@ -15,6 +15,7 @@ namespace {
 __global__ void pad_rows_kernel(const float* __restrict__ src, int dim, float* __restrict__ dst,
                                 int dst_ld, __nv_bfloat16* __restrict__ dst16, int dst16_ld,
                                 int rows) {
+    chain_begin();
     const int ld = max(dst ? dst_ld : 0, dst16 ? dst16_ld : 0);
     const long long total = (long long)rows * ld;
     for (long long i = blockIdx.x * (long long)blockDim.x + threadIdx.x; i < total;
@@ -66,6 +67,7 @@ __global__ void __launch_bounds__(256) act_head_kernel(const T* __restrict__ Ha,
                                                        const HeadParams hp, const ActOut out, int N,
                                                        uint32_t seed_lo, uint32_t seed_hi,
                                                        uint32_t global_step) {
+    chain_begin();
     const int warp = (blockIdx.x * blockDim.x + threadIdx.x) >> 5;
     const int lane = threadIdx.x & 31;
     if (warp == 0) {
@@ -110,6 +112,7 @@ template <typename T>
 __global__ void __launch_bounds__(256) value_head_kernel(const T* __restrict__ Hc, int ldhc,
                                                          const HeadParams hp, float* __restrict__ values,
                                                          int N) {
+    chain_begin();
     const int warp = (blockIdx.x * blockDim.x + threadIdx.x) >> 5;
     if (warp >= N) return;
     float v, unused;
@@ -121,6 +124,7 @@ __global__ void record_step_kernel(const float* __restrict__ rew, const uint8_t*
                                    const uint8_t* __restrict__ timeouts, float* __restrict__ s_rew,
                                    uint8_t* __restrict__ s_dones, uint8_t* __restrict__ s_timeouts,
                                    int N) {
+    chain_begin();
     const int i = blockIdx.x * blockDim.x + threadIdx.x;
     if (i < N) {
         s_rew[i] = rew[i];
@@ -266,8 +270,7 @@ cudaError_t launch_pad_rows(const float* src, int dim, float* dst, int dst_ld, _
     const long long total = (long long)rows * ld;
     const int blocks = (int)std::min((total + 255) / 256, (long long)(148 * 16));
     LaunchScope scope_("pad_rows", s);
-    pad_rows_kernel<<<blocks, 256, 0, s>>>(src, dim, dst, dst_ld, dst16, dst16_ld, rows);
-    return cudaGetLastError();
+    return launch_chained(pad_rows_kernel, blocks, 256, 0, s, src, dim, dst, dst_ld, dst16, dst16_ld, rows);
 }
 
 cudaError_t launch_act_head(const void* Ha, int ldha, const void* Hc, int ldhc, bool bf16_act,
@@ -277,12 +280,10 @@ cudaError_t launch_act_head(const void* Ha, int ldha, const void* Hc, int ldhc, 
     const uint32_t lo = (uint32_t)seed, hi = (uint32_t)(seed >> 32);
     LaunchScope scope_("act_head", s);
     if (bf16_act)
-        act_head_kernel<__nv_bfloat16><<<blocks, 256, 0, s>>>(
-            (const __nv_bfloat16*)Ha, ldha, (const __nv_bfloat16*)Hc, ldhc, hp, out, N, lo, hi, global_step);
-    else
-        act_head_kernel<float><<<blocks, 256, 0, s>>>((const float*)Ha, ldha, (const float*)Hc, ldhc,
-                                                      hp, out, N, lo, hi, global_step);
-    return cudaGetLastError();
+        return launch_chained(act_head_kernel<__nv_bfloat16>, blocks, 256, 0, s, (const __nv_bfloat16*)Ha, ldha,
+                              (const __nv_bfloat16*)Hc, ldhc, hp, out, N, lo, hi, global_step);
+    return launch_chained(act_head_kernel<float>, blocks, 256, 0, s, (const float*)Ha, ldha, (const float*)Hc, ldhc,
+                          hp, out, N, lo, hi, global_step);
 }
 
 cudaError_t launch_value_head(const void* Hc, int ldhc, bool bf16_act, const HeadParams& hp,
@@ -290,18 +291,15 @@ cudaError_t launch_value_head(const void* Hc, int ldhc, bool bf16_act, const Hea
     const int blocks = (N * 32 + 255) / 256;
     LaunchScope scope_("value_head", s);
     if (bf16_act)
-        value_head_kernel<__nv_bfloat16><<<blocks, 256, 0, s>>>((const __nv_bfloat16*)Hc, ldhc, hp, values, N);
-    else
-        value_head_kernel<float><<<blocks, 256, 0, s>>>((const float*)Hc, ldhc, hp, values, N);
-    return cudaGetLastError();
+        return launch_chained(value_head_kernel<__nv_bfloat16>, blocks, 256, 0, s, (const __nv_bfloat16*)Hc, ldhc, hp, values, N);
+    return launch_chained(value_head_kernel<float>, blocks, 256, 0, s, (const float*)Hc, ldhc, hp, values, N);
 }
 
 cudaError_t launch_record_step(const float* rew, const uint8_t* dones, const uint8_t* timeouts,
                                float* s_rew, uint8_t* s_dones, uint8_t* s_timeouts, int N,
                                cudaStream_t s) {
     LaunchScope scope_("record_step", s);
-    record_step_kernel<<<(N + 255) / 256, 256, 0, s>>>(rew, dones, timeouts, s_rew, s_dones, s_timeouts, N);
-    return cudaGetLastError();
+    return launch_chained(record_step_kernel, (N + 255) / 256, 256, 0, s, rew, dones, timeouts, s_rew, s_dones, s_timeouts, N);
 }
 
 int gae_scan_blocks(int N) { return (N + kGaeThreads - 1) / kGaeThreads; }

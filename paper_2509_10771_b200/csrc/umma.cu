@@ -227,6 +227,8 @@ __global__ void __launch_bounds__(kThreads, 1) tc_gemm_kernel(const __grid_const
     volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    // the set-up below touches only shared memory, tensor memory and the kernel parameters: it may
+    // overlap the tail of the preceding kernel; global memory is first touched after the wait
     if (threadIdx.x == 0) {
         for (int s = 0; s < kStages; ++s) { mbar_init(&full[s], 1); mbar_init(&empty[s], 1); }
         for (int b = 0; b < 2; ++b) { mbar_init(&tfull[b], 1); mbar_init(&tempty[b], kEpiWarps); }
@@ -237,15 +239,21 @@ __global__ void __launch_bounds__(kThreads, 1) tc_gemm_kernel(const __grid_const
         asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
     }
     if (warp == 1) tmem_alloc(tmem_slot, kTmemCols);
+    if (warp == 0 && lane == 0)
+        for (int i = 0; i < P.count; ++i) {
+            tma_prefetch_desc(&P.tmA[i]); tma_prefetch_desc(&P.tmB[i]);
+            if (MODE != TC_WGRAD) tma_prefetch_desc(&P.tmOut[i]);
+            if (MODE == TC_DGRAD) tma_prefetch_desc(&P.tmAux[i]);
+        }
     tc_fence_before();
     __syncthreads();
     tc_fence_after();
     const uint32_t tmem_base = *tmem_slot;
+    chain_wait();
 
     if (warp == 0) {
         // ================================ TMA producer =================================
         if (lane == 0) {
-            for (int i = 0; i < P.count; ++i) { tma_prefetch_desc(&P.tmA[i]); tma_prefetch_desc(&P.tmB[i]); }
             int stage = 0; uint32_t phase = 0;
             uint32_t issued_mask = 0, issued_parity = 0;
             bool ok = true;
@@ -320,6 +328,9 @@ __global__ void __launch_bounds__(kThreads, 1) tc_gemm_kernel(const __grid_const
                 }
                 if (ok) umma_commit(&tfull[buf]);     // accumulator complete
             }
+            // all products of this CTA are issued: the next kernel of the stream may be scheduled and set
+            // itself up while the last accumulators drain (it waits for this grid before it reads)
+            chain_release();
             if (!ok) {
                 umma_commit(drain);
                 const unsigned long long t0 = global_ns();
@@ -586,8 +597,7 @@ cudaError_t launch_tc(const TcParams& P, int num_sms, cudaStream_t s) {
     if (P.total_items == 0) return cudaSuccess;
     const int grid = std::min(P.total_items, num_sms);
     LaunchScope scope_(MODE == TC_FWD ? "tc_gemm_fwd" : MODE == TC_DGRAD ? "tc_gemm_dgrad" : "tc_gemm_wgrad", s);
-    tc_gemm_kernel<MODE><<<grid, kThreads, smem_bytes_of(MODE), s>>>(P);
-    return cudaGetLastError();
+    return launch_chained(tc_gemm_kernel<MODE>, grid, kThreads, smem_bytes_of(MODE), s, P);
 }
 
 }  // namespace

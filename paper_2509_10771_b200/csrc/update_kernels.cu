@@ -66,6 +66,7 @@ __device__ __forceinline__ void copy_obs_row(const float* __restrict__ src, int 
 }
 
 __global__ void __launch_bounds__(256, 3) gather_kernel(const GatherArgs a) {
+    chain_begin();
     const int lane = threadIdx.x & 31;
     const int warps = (gridDim.x * blockDim.x) >> 5;
     const bool bf16 = a.x_a16 != nullptr;
@@ -124,6 +125,7 @@ __global__ void __launch_bounds__(256, 3) gather_kernel(const GatherArgs a) {
 }
 
 __global__ void perm_rows_kernel(PermKey pk, uint32_t first, int count, int* __restrict__ rows_out) {
+    chain_begin();
     const int j = blockIdx.x * blockDim.x + threadIdx.x;
     if (j < count) rows_out[j] = (int)feistel_permute(pk, first + (uint32_t)j);
 }
@@ -483,6 +485,7 @@ constexpr int kRedExtraBlocks = 24;     // blocks that finish the entries coming
 // grid = reduce_blocks(P) blocks over the parameter vector + one extra block for the entries
 // that come from the head/loss kernel and for the loss sums.
 __global__ void __launch_bounds__(kRedThreads) reduce_kernel(const ReduceArgs a) {
+    chain_begin();
     __shared__ float ws[kRedThreads / 32];
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
     float sq = 0.f;
@@ -588,6 +591,7 @@ __global__ void __launch_bounds__(kRedThreads) reduce_kernel(const ReduceArgs a)
 constexpr int kAdamThreads = 256;
 
 __global__ void __launch_bounds__(kAdamThreads) adam_kernel(const AdamArgs a) {
+    chain_begin();
     __shared__ float s_scal[4];   // clip coefficient, lr, bias corrections
     __shared__ int s_skip;
     if (threadIdx.x < 32) {
@@ -680,8 +684,7 @@ cudaError_t launch_gather(const GatherArgs& a, cudaStream_t s) {
     if (a.Bmb <= 0) return cudaSuccess;
     const int blocks = std::min((a.Bmb + 7) / 8, 148 * 8);
     LaunchScope scope_("gather", s);
-    gather_kernel<<<blocks, 256, 0, s>>>(a);
-    return cudaGetLastError();
+    return launch_chained(gather_kernel, blocks, 256, 0, s, a);
 }
 
 cudaError_t launch_perm_rows(uint64_t seed, uint32_t iteration, uint32_t epoch, uint32_t batch,
@@ -689,8 +692,7 @@ cudaError_t launch_perm_rows(uint64_t seed, uint32_t iteration, uint32_t epoch, 
     if (count <= 0) return cudaSuccess;
     PermKey pk{(uint32_t)seed, (uint32_t)(seed >> 32), iteration, epoch, batch, feistel_half_bits(batch)};
     LaunchScope scope_("perm_rows", s);
-    perm_rows_kernel<<<(count + 255) / 256, 256, 0, s>>>(pk, first, count, rows_out);
-    return cudaGetLastError();
+    return launch_chained(perm_rows_kernel, (count + 255) / 256, 256, 0, s, pk, first, count, rows_out);
 }
 
 int head_loss_blocks(int Bmb) { return std::max(1, (Bmb + kHLRows - 1) / kHLRows); }
@@ -731,15 +733,13 @@ int reduce_blocks(int P) { return (P + kRedThreads * kRedPerThread - 1) / (kRedT
 
 cudaError_t launch_reduce(const ReduceArgs& a, cudaStream_t s) {
     LaunchScope scope_("grad_reduce", s);
-    reduce_kernel<<<reduce_blocks(a.P), kRedThreads, 0, s>>>(a);
-    return cudaGetLastError();
+    return launch_chained(reduce_kernel, reduce_blocks(a.P), kRedThreads, 0, s, a);
 }
 
 cudaError_t launch_adam(const AdamArgs& a, cudaStream_t s) {
     const int blocks = std::max(1, std::min((a.P / 4 + kAdamThreads - 1) / kAdamThreads, 148 * 4));
     LaunchScope scope_("adam", s);
-    adam_kernel<<<blocks, kAdamThreads, 0, s>>>(a);
-    return cudaGetLastError();
+    return launch_chained(adam_kernel, blocks, kAdamThreads, 0, s, a);
 }
 
 }  // namespace rslrl
