@@ -389,10 +389,9 @@ rslrl_status rslrl_create(const rslrl_model_cfg* m, const rslrl_ppo_cfg* p, void
     if (c->prec == RSLRL_FP32) {
         c->splits = std::max(1, std::min(32, c->R / 512));
     } else {
-        // one wave of weight-gradient work items over the SMs, at least 64 rows per split
+        // one wave of weight-gradient work items over the SMs; every problem has its own number of splits
         UmmaSetup probe{}; fill_setup(c, probe);
-        const int tiles = std::max(1, umma_wgrad_tiles(probe));
-        c->splits = std::max(1, std::min({32, (148 + tiles - 1) / tiles, (c->R + 63) / 64}));
+        c->splits = umma_wgrad_plan(probe).max_splits;
     }
     c->kchunk = round_up((c->R + c->splits - 1) / c->splits, 8);
     c->lddmu = as;

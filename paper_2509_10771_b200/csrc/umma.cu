@@ -106,7 +106,6 @@ __device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity, volati
         }
     }
 }
-
 __device__ __forceinline__ void tma_load_2d(void* smem_dst, const CUtensorMap* tm, int x, int y, uint64_t* bar) {
     asm volatile(
         "cp.async.bulk.tensor.2d.shared::cluster.global.tile.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];"
@@ -203,10 +202,14 @@ __device__ __forceinline__ Item decode_item(const TcParams& P, int item) {
     return it;
 }
 
-// Branch-free ELU; the exponential is the fast hardware one, which is ample for a BF16 result.
+// Branch-free ELU in six instructions: the epilogues are bound by instruction issue, not by the
+// exponential unit.  ex2.approx.ftz needs no range handling; for z > 0 the exponential may
+// overflow to infinity, which the select discards.
 __device__ __forceinline__ float elu_fast(float z, float alpha) {
-    const float e = alpha * (__expf(fminf(z, 0.f)) - 1.0f);
-    return z > 0.f ? z : e;
+    float e;
+    asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(e) : "f"(z * 1.4426950408889634f));
+    const float neg = fmaf(alpha, e, -alpha);
+    return z > 0.f ? z : neg;
 }
 
 template <int MODE>
@@ -475,6 +478,265 @@ __global__ void __launch_bounds__(kThreads, 1) tc_gemm_kernel(const __grid_const
     }
 }
 
+// ------------------------------------------------------------------ fused forward chain
+// All hidden layers of a net on one 128-row tile inside one CTA: the BF16 activations of a layer
+// stay in shared memory, in the K-major swizzled layout the next layer's MMA reads as its A
+// operand (and the TMA store reads to write them to global memory for the backward pass); only
+// the weights (and the observations of the first layer) stream through the ring.  A tile runs a
+// short program the host compiled from the layer widths: MMA jobs, each a run of k-blocks into
+// one accumulator of up to 256 tensor-memory columns, and epilogues, each turning one
+// accumulator into activations.  Jobs and epilogues name what they wait for, so an epilogue
+// overlaps the jobs that do not need its result.  A first layer wider than 256 is produced in
+// two halves, and the second layer accumulates over each half as soon as it exists.
+constexpr int kChainLayers = 4;                  // hidden layers per net
+constexpr int kChainJobs = 8;
+constexpr int kChainEpis = 6;
+// The operand ring is cut into 16 KiB slots: a k-block takes one slot for its A tile (first layer only)
+// and one or two for its B tile, contiguous, and both ends of the ring skip the tail when a k-block
+// would wrap.  Jobs with small tiles therefore keep more k-blocks in flight.
+constexpr int kSlots = 9;
+constexpr uint32_t kSlotBytes = 16384;
+constexpr uint32_t kActBytes = BLOCK_M * kMaxBN * 2;     // 64 KiB = four [128 rows][64] blocks
+constexpr int kChainBiasFloats = 2 * (512 + (kChainLayers - 1) * 256);
+constexpr size_t kChainSmem = 1024 + (size_t)kSlots * kSlotBytes + kActBytes + kChainBiasFloats * 4 + 512;
+__host__ __device__ constexpr int slots_of(int a_ring, int bn) { return a_ring + (bn * BLOCK_K * 2 + (int)kSlotBytes - 1) / (int)kSlotBytes; }
+constexpr int kPrevItem = 16;                    // added to an epilogue index: that epilogue of the CTA's previous item
+
+struct ChainJob {
+    int layer;           // whose weights
+    int n0, bn;          // output columns [n0, n0 + bn) = rows of the weight operand
+    int kb0, nkb;        // k-blocks [kb0, kb0 + nkb) of that layer's contraction
+    int a_ring;          // 1: A k-blocks (observations) come through the ring; 0: block i of the activation buffer
+    int tmem_col;        // accumulator columns [tmem_col, tmem_col + bn)
+    int accumulate;      // 1: adds to what the accumulator holds
+    int wait_epi;        // epilogue that must have finished before the first MMA (-1: none; + kPrevItem: of the previous item):
+                         // it wrote the activations this job reads, or drained the accumulator this job overwrites
+};
+struct ChainEpi {
+    int layer, n0, ncols, tmem_col;   // columns [n0, n0 + ncols) of `layer` from these accumulator columns
+    int wait_job;        // the job that completes the accumulator
+    int write_job;       // a later job that still reads the activation buffer (-1: none): done before the buffer is rewritten
+};
+struct ChainNet {
+    int nlayers, njobs, nepis;
+    int flip;            // 1: odd items of a CTA use the other half of tensor memory for every accumulator
+    ChainJob job[kChainJobs];
+    ChainEpi epi[kChainEpis];
+    const float* bias[kChainLayers];  // zero-padded to the padded width
+    int bias_n[kChainLayers];         // that width
+    int bias_off[kChainLayers];       // where the kernel keeps the layer's bias in shared memory (floats)
+};
+struct ChainParams {
+    CUtensorMap tmX[2];                       // first-layer input, boxes of 64 x 128 rows
+    CUtensorMap tmW[2][kChainLayers];         // [out][in] weights, boxes of 64 x (columns per job)
+    CUtensorMap tmOut[2][kChainLayers];       // activations, boxes of 64 columns x 32 rows
+    ChainNet net[2];                          // same numbers of jobs and epilogues, same waits
+    int nnets, rows, total_items;             // items = (row tile, net), nets interleaved
+    float alpha;
+    int* error;
+};
+
+__global__ void __launch_bounds__(kThreads, 1) chain_fwd_kernel(const __grid_constant__ ChainParams P) {
+    extern __shared__ uint8_t smem_raw[];
+    uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
+    uint8_t* sRing = smem;
+    uint8_t* sAct = sRing + kSlots * kSlotBytes;
+    float* sBias = reinterpret_cast<float*>(sAct + kActBytes);
+    uint64_t* full = reinterpret_cast<uint64_t*>(sBias + kChainBiasFloats);
+    uint64_t* empty = full + kSlots;
+    uint64_t* job_done = empty + kSlots;       // one completion per item each
+    uint64_t* epi_done = job_done + kChainJobs;
+    uint64_t* drain = epi_done + kChainEpis;
+    uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(drain + 1);
+    volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
+
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    if (threadIdx.x == 0) {
+        for (int s = 0; s < kSlots; ++s) { mbar_init(&full[s], 1); mbar_init(&empty[s], 1); }
+        for (int j = 0; j < kChainJobs; ++j) mbar_init(&job_done[j], 1);
+        for (int e = 0; e < kChainEpis; ++e) mbar_init(&epi_done[e], kEpiWarps);
+        mbar_init(drain, 1);
+        *abort_flag = 0;
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+        asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+    }
+    if (warp == 1) tmem_alloc(tmem_slot, kTmemCols);
+    if (warp == 0 && lane == 0)
+        for (int n = 0; n < P.nnets; ++n) {
+            tma_prefetch_desc(&P.tmX[n]);
+            for (int l = 0; l < P.net[n].nlayers; ++l) { tma_prefetch_desc(&P.tmW[n][l]); tma_prefetch_desc(&P.tmOut[n][l]); }
+        }
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    const uint32_t tmem_base = *tmem_slot;
+    chain_wait();
+    // the epilogues read the biases between two MMA jobs: keep them close
+    for (int n = 0; n < P.nnets; ++n)
+        for (int l = 0; l < P.net[n].nlayers; ++l)
+            for (int i = threadIdx.x; i < P.net[n].bias_n[l]; i += kThreads) sBias[P.net[n].bias_off[l] + i] = P.net[n].bias[l][i];
+    __syncthreads();
+
+    if (warp == 0) {
+        // ================================ TMA producer =================================
+        if (lane == 0) {
+            int pos = 0;
+            uint32_t full_bits = 0, empty_bits = 0;     // parity of the next use of each slot's barriers
+            uint32_t issued_mask = 0, issued_parity = 0;
+            bool ok = true;
+            for (int item = blockIdx.x; ok && item < P.total_items; item += gridDim.x) {
+                const int ni = item % P.nnets, m0 = (item / P.nnets) * BLOCK_M;
+                const ChainNet& N = P.net[ni];
+                for (int j = 0; ok && j < N.njobs; ++j) {
+                    const ChainJob& J = N.job[j];
+                    const int need = slots_of(J.a_ring, J.bn);
+                    const uint32_t bytes = (uint32_t)J.bn * BLOCK_K * 2 + (J.a_ring ? kSlotBytes : 0u);
+                    for (int kb = J.kb0; ok && kb < J.kb0 + J.nkb; ++kb) {
+                        if (pos + need > kSlots) pos = 0;
+                        for (int s = pos; s < pos + need; ++s)
+                            if (!mbar_wait(&empty[s], ((empty_bits >> s) & 1u) ^ 1u, abort_flag, P.error, 11)) { ok = false; break; }
+                        if (!ok) break;
+                        mbar_expect_tx(&full[pos], bytes);
+                        uint8_t* dst = sRing + pos * kSlotBytes;
+                        if (J.a_ring) { tma_load_2d(dst, &P.tmX[ni], kb * BLOCK_K, m0, &full[pos]); dst += kSlotBytes; }
+                        tma_load_2d(dst, &P.tmW[ni][J.layer], kb * BLOCK_K, J.n0, &full[pos]);
+                        issued_mask |= 1u << pos;
+                        issued_parity = (issued_parity & ~(1u << pos)) | (((full_bits >> pos) & 1u) << pos);
+                        full_bits ^= 1u << pos;
+                        empty_bits ^= ((1u << need) - 1u) << pos;
+                        pos += need;
+                    }
+                }
+            }
+            if (!ok) {
+                // let the copies already issued land before the CTA's shared memory goes away
+                for (int s = 0; s < kSlots; ++s) {
+                    if (!(issued_mask & (1u << s))) continue;
+                    const unsigned long long t0 = global_ns();
+                    while (!mbar_try_wait(&full[s], (issued_parity >> s) & 1u) && global_ns() - t0 < kWaitLimitNs) {}
+                }
+            }
+        }
+    } else if (warp == 1) {
+        // ================================ MMA issuer ===================================
+        if (lane == 0) {
+            int pos = 0;
+            uint32_t full_bits = 0;
+            bool ok = true;
+            uint32_t t = 0;                          // items this CTA has started
+            for (int item = blockIdx.x; ok && item < P.total_items; item += gridDim.x, ++t) {
+                const ChainNet& N = P.net[item % P.nnets];
+                const uint32_t flip = (N.flip && (t & 1u)) ? 256u : 0u;
+                for (int j = 0; ok && j < N.njobs; ++j) {
+                    const ChainJob& J = N.job[j];
+                    if (J.wait_epi >= kPrevItem) {
+                        if (t > 0 && !mbar_wait(&epi_done[J.wait_epi - kPrevItem], (t - 1) & 1u, abort_flag, P.error, 12)) { ok = false; break; }
+                    } else if (J.wait_epi >= 0) {
+                        if (!mbar_wait(&epi_done[J.wait_epi], t & 1u, abort_flag, P.error, 12)) { ok = false; break; }
+                    }
+                    tc_fence_after();
+                    const uint32_t d_tmem = tmem_base + ((uint32_t)J.tmem_col ^ flip);
+                    const uint32_t idesc = instr_desc(J.bn, 0, 0);
+                    const int need = slots_of(J.a_ring, J.bn);
+                    for (int i = 0; i < J.nkb; ++i) {
+                        if (pos + need > kSlots) pos = 0;
+                        if (!mbar_wait(&full[pos], (full_bits >> pos) & 1u, abort_flag, P.error, 13)) { ok = false; break; }
+                        full_bits ^= 1u << pos;
+                        tc_fence_after();
+                        const uint32_t ring_addr = smem_u32(sRing + pos * kSlotBytes);
+                        const uint32_t a_addr = J.a_ring ? ring_addr : smem_u32(sAct + i * kStageA);
+                        const uint32_t b_addr = ring_addr + (J.a_ring ? kSlotBytes : 0u);
+#pragma unroll
+                        for (int k = 0; k < BLOCK_K / UMMA_K; ++k)
+                            umma_bf16(d_tmem, smem_desc(a_addr + k * (UMMA_K * 2), 16, 1024),
+                                      smem_desc(b_addr + k * (UMMA_K * 2), 16, 1024), idesc,
+                                      (J.accumulate || i > 0 || k > 0) ? 1u : 0u);
+                        for (int s2 = pos; s2 < pos + need; ++s2) umma_commit(&empty[s2]);   // frees the slots once these MMAs have read them
+                        pos += need;
+                    }
+                    if (ok) umma_commit(&job_done[j]);
+                }
+            }
+            // all products of this CTA are issued: the next kernel of the stream may be scheduled
+            chain_release();
+            if (!ok) {
+                umma_commit(drain);
+                const unsigned long long t0 = global_ns();
+                while (!mbar_try_wait(drain, 0) && global_ns() - t0 < kWaitLimitNs) {}
+            }
+        }
+    } else {
+        // ================================ epilogue =====================================
+        const int q = warp & 3;                    // accumulator lanes (= tile rows) 32q .. 32q+31
+        const int g = (warp - 2) >> 2;             // columns [64 g, 64 g + 64) of the epilogue's output
+        // block g of the activation buffer, rows 32q..: lane r owns row r (128 bytes = eight 16-byte
+        // pieces), piece j is kept at j ^ (r & 7), the 128-byte swizzle both the MMA and the store expect
+        uint8_t* tile = sAct + g * kStageA + q * (32 * 128);
+        uint8_t* tile_row = tile + lane * 128;
+        const int sw = lane & 7;
+        bool ok = true;
+        uint32_t t = 0;
+        for (int item = blockIdx.x; ok && item < P.total_items; item += gridDim.x, ++t) {
+            const int ni = item % P.nnets, m0 = (item / P.nnets) * BLOCK_M;
+            const ChainNet& N = P.net[ni];
+            const uint32_t flip = (N.flip && (t & 1u)) ? 256u : 0u;
+            for (int e = 0; e < N.nepis; ++e) {
+                const ChainEpi& E = N.epi[e];
+                if (!mbar_wait(&job_done[E.wait_job], t & 1u, abort_flag, P.error, 14)) { ok = false; break; }
+                tc_fence_after();
+                const bool active = 64 * g < E.ncols;          // uniform across the warp
+                uint4 outv[8];
+                if (active) {
+                    const float* bias = sBias + N.bias_off[E.layer] + E.n0 + 64 * g;
+#pragma unroll
+                    for (int ci = 0; ci < 2; ++ci) {
+                        uint32_t acc[32];
+                        tmem_ld32(tmem_base + ((uint32_t)(32 * q) << 16) + (((uint32_t)E.tmem_col ^ flip) + (uint32_t)(64 * g + 32 * ci)), acc);
+                        const float4* b4 = reinterpret_cast<const float4*>(bias + 32 * ci);
+#pragma unroll
+                        for (int gg = 0; gg < 4; ++gg) {
+                            const float4 ba = b4[2 * gg], bb = b4[2 * gg + 1];
+                            const float bv[8] = {ba.x, ba.y, ba.z, ba.w, bb.x, bb.y, bb.z, bb.w};
+                            uint32_t o[4];
+#pragma unroll
+                            for (int k = 0; k < 4; ++k) {
+                                const float v0 = elu_fast(__uint_as_float(acc[8 * gg + 2 * k]) + bv[2 * k], P.alpha);
+                                const float v1 = elu_fast(__uint_as_float(acc[8 * gg + 2 * k + 1]) + bv[2 * k + 1], P.alpha);
+                                __nv_bfloat162 h2 = __floats2bfloat162_rn(v0, v1);
+                                o[k] = *reinterpret_cast<uint32_t*>(&h2);
+                            }
+                            outv[4 * ci + gg] = make_uint4(o[0], o[1], o[2], o[3]);
+                        }
+                    }
+                }
+                // the accumulator is in registers; the buffer may still feed a job that runs meanwhile
+                if (E.write_job >= 0 && !mbar_wait(&job_done[E.write_job], t & 1u, abort_flag, P.error, 15)) { ok = false; break; }
+                if (active) {
+                    if (lane == 0) tma_store_wait_read();       // this warp's last store has read the rows
+                    __syncwarp();
+#pragma unroll
+                    for (int p8 = 0; p8 < 8; ++p8) *reinterpret_cast<uint4*>(tile_row + ((p8 ^ sw) << 4)) = outv[p8];
+                    fence_async_smem();                         // rows -> visible to the MMA and the copy engine
+                }
+                tc_fence_before();
+                __syncwarp();
+                if (lane == 0) {
+                    // rows at or beyond the tensor's extent are clipped by the store itself
+                    if (active && m0 + 32 * q < P.rows) tma_store_2d(&P.tmOut[ni][E.layer], tile, E.n0 + 64 * g, m0 + 32 * q);
+                    mbar_arrive(&epi_done[e]);
+                }
+            }
+        }
+        if (lane == 0) tma_store_wait_all();        // stores done before the CTA retires
+    }
+    tc_fence_before();
+    __syncthreads();
+    if (warp == 1) {
+        tc_fence_after();
+        tmem_dealloc(tmem_base, kTmemCols);
+    }
+}
+
 // ------------------------------------------------------------------------- small kernels
 struct CvtEntry {
     const float* bsrc; float* bdst;             // bias -> zero-padded FP32 copy
@@ -549,6 +811,8 @@ struct UmmaEngine {
     int* error_dev = nullptr;
     int num_sms = 148;
     std::vector<TcParams> act_fwd, act_fwd_critic, upd_fwd, upd_dgrad, upd_wgrad;
+    // fused forward (one launch for all hidden layers) where the widths allow it, else empty
+    std::vector<ChainParams> chain_act, chain_act_critic, chain_upd;
     ColsumBatch colsum{}, colsum_rest{};         // all layers the epilogue does not cover / those minus the last ones
 };
 
@@ -600,19 +864,125 @@ cudaError_t launch_tc(const TcParams& P, int num_sms, cudaStream_t s) {
     return launch_chained(tc_gemm_kernel<MODE>, grid, kThreads, smem_bytes_of(MODE), s, P);
 }
 
+// The program of one net for the fused forward; false when the widths do not fit the kernel
+// (first hidden layer <= 512 and a multiple of 128 beyond 256, the others <= 256).
+bool compile_chain(ChainNet& N, int nh, const int* pw, int kp, int* bn_of_layer) {
+    memset(&N, 0, sizeof N);
+    if (nh < 1 || nh > kChainLayers || pw[0] > 512 || (pw[0] > 256 && pw[0] % 128 != 0)) return false;
+    for (int l = 1; l < nh; ++l)
+        if (pw[l] > 256) return false;
+    int nj = 0, ne = 0;
+    auto job = [&](int layer, int n0, int bn, int kb0, int nkb, int a_ring, int tmem_col, int accumulate, int wait_epi) {
+        N.job[nj] = ChainJob{layer, n0, bn, kb0, nkb, a_ring, tmem_col, accumulate, wait_epi};
+        return nj++;
+    };
+    auto epi = [&](int layer, int n0, int ncols, int tmem_col, int wait_job, int write_job) {
+        N.epi[ne] = ChainEpi{layer, n0, ncols, tmem_col, wait_job, write_job};
+        return ne++;
+    };
+    const int kb_in = kp / BLOCK_K;
+    for (int l = 0; l < nh; ++l) bn_of_layer[l] = pw[l];
+    if (pw[0] <= 256 || nh < 2) {
+        if (pw[0] > 256) {
+            // a single wide layer: two independent halves, each waiting for its own accumulator to be drained
+            const int half = pw[0] / 2;
+            bn_of_layer[0] = half;
+            const int j0 = job(0, 0, half, 0, kb_in, 1, 0, 0, kPrevItem + 0);
+            const int j1 = job(0, half, half, 0, kb_in, 1, 256, 0, kPrevItem + 1);
+            epi(0, 0, half, 0, j0, -1);
+            epi(0, half, half, 256, j1, -1);
+        } else if (nh == 1) {
+            const int j0 = job(0, 0, pw[0], 0, kb_in, 1, 0, 0, kPrevItem + 0);
+            epi(0, 0, pw[0], 0, j0, -1);
+        } else {
+            // plain chain: the accumulators alternate between the halves of tensor memory, and a job waits
+            // for the epilogue of the layer before.  The half the first job of an item overwrites was
+            // drained by an epilogue that a later job of the item before already waited for; with an odd
+            // number of layers that holds because the halves swap from item to item.
+            int prev_e = -1;
+            for (int l = 0; l < nh; ++l) {
+                const int col = (l & 1) ? 256 : 0;
+                const int j = l == 0 ? job(0, 0, pw[0], 0, kb_in, 1, col, 0, -1)
+                                     : job(l, 0, pw[l], 0, pw[l - 1] / BLOCK_K, 0, col, 0, prev_e);
+                prev_e = epi(l, 0, pw[l], col, j, -1);
+            }
+            N.flip = (nh & 1) ? 1 : 0;
+        }
+    } else {
+        // wide first layer: both halves up front, the second layer accumulates over them
+        const int half = pw[0] / 2, hk = half / BLOCK_K;
+        bn_of_layer[0] = half;
+        const int last_e = nh;                                    // index of the item's last epilogue (nh + 1 epilogues)
+        const bool last_in_256 = ((nh - 2) & 1) != 0;             // layers 2.. alternate 256, 0, 256, ...
+        const int j0 = job(0, 0, half, 0, kb_in, 1, 0, 0, last_in_256 ? -1 : kPrevItem + last_e);
+        const int j1 = job(0, half, half, 0, kb_in, 1, 256, 0, last_in_256 ? kPrevItem + last_e : -1);
+        const int e0 = epi(0, 0, half, 0, j0, -1);
+        const int j2 = job(1, 0, pw[1], 0, hk, 0, 0, 0, e0);
+        const int e1 = epi(0, half, half, 256, j1, j2);
+        const int j3 = job(1, 0, pw[1], hk, hk, 0, 0, 1, e1);
+        int prev_e = epi(1, 0, pw[1], 0, j3, -1);
+        for (int l = 2; l < nh; ++l) {
+            const int col = (l & 1) ? 0 : 256;
+            const int j = job(l, 0, pw[l], 0, pw[l - 1] / BLOCK_K, 0, col, 0, prev_e);
+            prev_e = epi(l, 0, pw[l], col, j, -1);
+        }
+    }
+    N.nlayers = nh; N.njobs = nj; N.nepis = ne;
+    return nj <= kChainJobs && ne <= kChainEpis;
+}
+
+cudaError_t launch_chain(const ChainParams& P, int num_sms, cudaStream_t s) {
+    if (P.total_items == 0) return cudaSuccess;
+    const int grid = std::min(P.total_items, num_sms);
+    LaunchScope scope_("tc_mlp_fwd", s);
+    return launch_chained(chain_fwd_kernel, grid, kThreads, kChainSmem, s, P);
+}
+
 }  // namespace
 
-int umma_wgrad_tiles(const UmmaSetup& s) {
-    int tiles = 0;
+// Splits of the contraction (the minibatch rows) for every weight-gradient problem, chosen so that
+// the work items (tile x split) fill the SMs once with items of about equal cost: starting from one
+// split each, the problem with the most expensive item gets another split while the items still fit.
+// The cost of an item is the bytes it streams, (128 + columns) per contraction row.
+WgradPlan umma_wgrad_plan(const UmmaSetup& s) {
+    WgradPlan plan{};
+    int sms = 148, dev = 0;
+    if (cudaGetDevice(&dev) == cudaSuccess) cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
+    const int kblocks = (s.R + BLOCK_K - 1) / BLOCK_K;
+    struct Prob { int ni, l, tiles, unit, splits; };
+    std::vector<Prob> probs;
+    int items = 0;
     for (int ni = 0; ni < 2; ++ni) {
         const int nh = s.nl[ni] - 1;
         for (int l = 0; l <= nh; ++l) {
             const int wa = round_up(l == 0 ? s.in_dim[ni] : s.out[ni][l - 1], 64);
             const int wb = l == nh ? 64 : round_up(s.out[ni][l], 64);
-            tiles += ((wa + BLOCK_M - 1) / BLOCK_M) * ((wb + pick_bn(wb) - 1) / pick_bn(wb));
+            const int bn = pick_bn(wb);
+            Prob q{ni, l, ((wa + BLOCK_M - 1) / BLOCK_M) * ((wb + bn - 1) / bn), BLOCK_M + bn, 1};
+            probs.push_back(q);
+            items += q.tiles;
         }
     }
-    return tiles;
+    const int max_splits = std::max(1, std::min(32, kblocks));
+    auto item_cost = [&](const Prob& q) { return (long long)q.unit * ((kblocks + q.splits - 1) / q.splits); };
+    while (true) {
+        int best = -1;
+        for (int i = 0; i < (int)probs.size(); ++i) {
+            const Prob& q = probs[i];
+            if (q.splits >= max_splits || items + q.tiles > sms) continue;
+            if (best < 0 || item_cost(q) > item_cost(probs[best])) best = i;
+        }
+        if (best < 0) break;
+        // stop when the most expensive item overall can no longer be split: more splits elsewhere gain nothing
+        bool is_max = true;
+        for (const Prob& q : probs) if (item_cost(q) > item_cost(probs[best])) is_max = false;
+        if (!is_max) break;
+        probs[best].splits++;
+        items += probs[best].tiles;
+    }
+    plan.max_splits = 1;
+    for (const Prob& q : probs) { plan.splits[q.ni][q.l] = q.splits; plan.max_splits = std::max(plan.max_splits, q.splits); }
+    return plan;
 }
 
 UmmaEngine* umma_create(const UmmaSetup& s, std::string* err) {
@@ -626,6 +996,8 @@ UmmaEngine* umma_create(const UmmaSetup& s, std::string* err) {
         cudaFuncSetAttribute(tc_gemm_kernel<TC_DGRAD>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem_bytes_of(TC_DGRAD)) != cudaSuccess ||
         cudaFuncSetAttribute(tc_gemm_kernel<TC_WGRAD>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem_bytes_of(TC_WGRAD)) != cudaSuccess)
         return failmsg("could not reserve shared memory for the tensor-core kernels");
+    if (cudaFuncSetAttribute(chain_fwd_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kChainSmem) != cudaSuccess)
+        return failmsg("could not reserve shared memory for the fused forward kernel");
     UmmaEngine* e = new UmmaEngine();
     e->s = s;
     e->num_sms = prop.multiProcessorCount;
@@ -698,6 +1070,48 @@ UmmaEngine* umma_create(const UmmaSetup& s, std::string* err) {
     if (!build_fwd(e->act_fwd, N, true, true, true) || !build_fwd(e->act_fwd_critic, N, false, true, true) ||
         !build_fwd(e->upd_fwd, R, true, true, false))
         return bail("tensor map encoding failed");
+    // ---- fused forward: every hidden layer of both nets in one launch ------------------------
+    auto build_chain = [&](std::vector<ChainParams>& out, int rows, bool actor, bool critic, bool act_buffers) -> bool {
+        ChainParams P; memset(&P, 0, sizeof P);
+        int bias_floats = 0;
+        for (int ni = 0; ni < 2; ++ni) {
+            if ((ni == 0 && !actor) || (ni == 1 && !critic)) continue;
+            const int n = P.nnets;
+            int bn[kChainLayers] = {};
+            if (e->nh[ni] > kChainLayers || !compile_chain(P.net[n], e->nh[ni], e->pw[ni], e->kp[ni], bn)) return true;   // not applicable
+            if (!make_tmap(&P.tmX[n], act_buffers ? e->obs16_act[ni] : e->x16[ni], rows, e->kp[ni], e->kp[ni], BLOCK_K, BLOCK_M)) return false;
+            for (int l = 0; l < e->nh[ni]; ++l) {
+                const int kin = l == 0 ? e->kp[ni] : e->pw[ni][l - 1];
+                __nv_bfloat16* o = act_buffers ? e->h_act[ni][l] : e->h[ni][l];
+                if (!make_tmap(&P.tmW[n][l], e->wt[ni][l], e->pw[ni][l], kin, kin, BLOCK_K, bn[l]) ||
+                    !make_tmap(&P.tmOut[n][l], o, rows, e->pw[ni][l], e->pw[ni][l], 64, 32))
+                    return false;
+                P.net[n].bias[l] = e->bias_pad[ni][l];
+                P.net[n].bias_n[l] = e->pw[ni][l];
+                P.net[n].bias_off[l] = bias_floats;
+                bias_floats += e->pw[ni][l];
+            }
+            P.nnets++;
+        }
+        if (P.nnets == 2) {
+            // items of both nets alternate in a CTA and wait for each other's epilogues by index
+            const ChainNet &a = P.net[0], &b = P.net[1];
+            bool same = a.njobs == b.njobs && a.nepis == b.nepis && a.flip == b.flip;
+            for (int j = 0; same && j < a.njobs; ++j) same = a.job[j].wait_epi == b.job[j].wait_epi && a.job[j].tmem_col == b.job[j].tmem_col;
+            for (int k = 0; same && k < a.nepis; ++k)
+                same = a.epi[k].wait_job == b.epi[k].wait_job && a.epi[k].write_job == b.epi[k].write_job && a.epi[k].tmem_col == b.epi[k].tmem_col;
+            if (!same) return true;   // not applicable
+        }
+        P.rows = rows;
+        P.total_items = P.nnets * ((rows + BLOCK_M - 1) / BLOCK_M);
+        P.alpha = alpha; P.error = e->error_dev;
+        out.push_back(P);
+        return true;
+    };
+    // (the rollout's few row tiles gain from the single launch; on the many tiles of a minibatch the
+    // per-layer launches, whose epilogues overlap the next tile's MMAs, measured slightly faster)
+    if (!build_chain(e->chain_act, N, true, true, true) || !build_chain(e->chain_act_critic, N, false, true, true))
+        return bail("tensor map encoding failed");
     // ---- data-gradient launches: step b produces dZ of hidden layer nh-2-b -------------------
     for (int b = 0; b + 1 < maxh; ++b) {
         TcParams P; memset(&P, 0, sizeof P);
@@ -725,8 +1139,7 @@ UmmaEngine* umma_create(const UmmaSetup& s, std::string* err) {
     // ---- weight-gradient problems (all layers of both nets, heads included) ------------------
     {
         const int kblocks = (R + BLOCK_K - 1) / BLOCK_K;
-        const int kb_per_split = (kblocks + s.splits - 1) / s.splits;
-        const int splits_eff = (kblocks + kb_per_split - 1) / kb_per_split;
+        const WgradPlan plan = umma_wgrad_plan(s);
         TcParams P; memset(&P, 0, sizeof P);
         auto flush = [&]() { if (P.count) { finish_params(P, alpha, e->error_dev); e->upd_wgrad.push_back(P); memset(&P, 0, sizeof P); } };
         for (int ni = 0; ni < 2; ++ni)
@@ -742,7 +1155,9 @@ UmmaEngine* umma_create(const UmmaSetup& s, std::string* err) {
                 p.bn = pick_bn(wb);
                 p.m_extent = s.in[ni][l]; p.n_extent = s.out_p[ni][l];
                 p.m_tiles = (wa + BLOCK_M - 1) / BLOCK_M; p.n_tiles = (wb + p.bn - 1) / p.bn;
-                p.kblocks = kblocks; p.splits = splits_eff; p.kb_per_split = kb_per_split;
+                const int want = std::min(plan.splits[ni][l], s.splits);      // s.splits rows of partials exist
+                p.kb_per_split = (kblocks + want - 1) / want;
+                p.kblocks = kblocks; p.splits = (kblocks + p.kb_per_split - 1) / p.kb_per_split;
                 p.out32 = s.partials + s.w_off[ni][l]; p.ld_out32 = s.out_p[ni][l]; p.split_stride = s.P_dev;
                 if (!make_tmap(&P.tmA[i], A, R, wa, wa, 64, BLOCK_K) || !make_tmap(&P.tmB[i], B, R, wb, wb, 64, BLOCK_K))
                     return bail("tensor map encoding failed");
@@ -832,10 +1247,16 @@ cudaError_t umma_act_forward(UmmaEngine* e, const float* d_obs_a, const float* d
         err = launch_pad_rows(d_obs_c, s.in_dim[1], nullptr, 0, e->obs16_act[1], e->kp[1], s.N, s.stream);
         if (err != cudaSuccess) return err;
     }
-    const std::vector<TcParams>& seq = do_actor ? e->act_fwd : e->act_fwd_critic;
-    for (const TcParams& P : seq) {
-        err = launch_tc<TC_FWD>(P, e->num_sms, s.stream);
+    const std::vector<ChainParams>& fused = do_actor ? e->chain_act : e->chain_act_critic;
+    if (!fused.empty()) {
+        err = launch_chain(fused[0], e->num_sms, s.stream);
         if (err != cudaSuccess) return err;
+    } else {
+        const std::vector<TcParams>& seq = do_actor ? e->act_fwd : e->act_fwd_critic;
+        for (const TcParams& P : seq) {
+            err = launch_tc<TC_FWD>(P, e->num_sms, s.stream);
+            if (err != cudaSuccess) return err;
+        }
     }
     *ha = e->h_act[0][e->nh[0] - 1]; *ldha = e->pw[0][e->nh[0] - 1];
     *hc = e->h_act[1][e->nh[1] - 1]; *ldhc = e->pw[1][e->nh[1] - 1];
@@ -849,6 +1270,7 @@ void umma_gather_targets(UmmaEngine* e, GatherArgs* g) {
 }
 
 cudaError_t umma_update_forward(UmmaEngine* e) {
+    if (!e->chain_upd.empty()) return launch_chain(e->chain_upd[0], e->num_sms, e->s.stream);
     for (const TcParams& P : e->upd_fwd) {
         cudaError_t err = launch_tc<TC_FWD>(P, e->num_sms, e->s.stream);
         if (err != cudaSuccess) return err;

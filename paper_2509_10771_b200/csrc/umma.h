@@ -23,8 +23,10 @@ struct UmmaEngine;
 
 UmmaEngine* umma_create(const UmmaSetup& s, std::string* err);
 void umma_destroy(UmmaEngine* e);
-// Number of 128-row x <=256-column output tiles of all weight gradients (for choosing splits).
-int umma_wgrad_tiles(const UmmaSetup& s);
+// Splits of the contraction per weight-gradient problem [net][layer] (head = last layer) and their
+// maximum, which is the number of partial rows the gradient buffer needs.
+struct WgradPlan { int splits[2][kMaxLayers]; int max_splits; };
+WgradPlan umma_wgrad_plan(const UmmaSetup& s);
 // Re-derive the low-precision operand copies of the weights from the FP32 masters (after
 // rslrl_set_params; the optimiser step refreshes them itself, see umma_fill_cvt).
 cudaError_t umma_refresh_weights(UmmaEngine* e);
