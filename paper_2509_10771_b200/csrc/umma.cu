@@ -11,6 +11,7 @@
 // Every wait on an mbarrier is bounded in time; on expiry the CTA raises an error flag that
 // the host reads, drains its own asynchronous work, frees its tensor memory and returns.
 #include "umma.h"
+#include "tc_ptx.cuh"
 
 #include <cuda.h>
 #include <algorithm>
@@ -19,26 +20,19 @@
 
 namespace rslrl {
 
+using namespace tc;
+
 namespace {
 
 // Forward and data gradient: 3 pipeline stages + a 4 KiB result tile per epilogue warp;
 // weight gradient (long contraction, FP32 results stored from registers): 4 stages.
 __host__ __device__ constexpr int stages_of(int mode) { return mode == 2 ? 4 : 3; }
-constexpr int BLOCK_M = 128;
-constexpr int BLOCK_K = 64;                      // bf16 elements = one 128-byte swizzle row
-constexpr int UMMA_K = 16;
-constexpr int kMaxBN = 256;
-constexpr int kEpiWarps = 16;
-constexpr int kThreads = 32 * (2 + kEpiWarps);
-constexpr uint32_t kStageA = BLOCK_M * BLOCK_K * 2;      // 16 KiB
 constexpr uint32_t kStageB = kMaxBN * BLOCK_K * 2;       // 32 KiB
-constexpr uint32_t kTmemCols = 512;                      // two accumulator buffers of 256 columns
 constexpr int kMaxProblems = 8;
 constexpr uint32_t kStageOut = 32 * 64 * 2;              // 4 KiB result tile per epilogue warp (32 rows x 64 bf16)
 __host__ __device__ constexpr size_t smem_bytes_of(int mode) {
     return 1024 + (size_t)stages_of(mode) * (kStageA + kStageB) + (mode == 2 ? 0 : kEpiWarps * kStageOut) + 512;
 }
-constexpr unsigned long long kWaitLimitNs = 2000000000ull;   // 2 s
 
 enum TcMode { TC_FWD = 0, TC_DGRAD = 1, TC_WGRAD = 2 };
 
@@ -53,6 +47,7 @@ struct TcProblem {
     const __nv_bfloat16* aux16; int ld_aux;
     float* out32; int ld_out32; long long split_stride;
     float* colsum; int ld_colsum;  // data gradient: column sums of each 32-row slice, [4 m_tiles][ld_colsum] (may be null)
+    const __nv_bfloat16* a_ptr; const __nv_bfloat16* b_ptr; int k_elems;   // host side: operands [rows][k], [columns][k]
 };
 
 struct TcParams {
@@ -65,121 +60,6 @@ struct TcParams {
     float alpha;
     int* error;
 };
-
-// ------------------------------------------------------------------------------ PTX wrappers
-__device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
-
-__device__ __forceinline__ void mbar_init(uint64_t* bar, uint32_t count) {
-    asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(smem_u32(bar)), "r"(count));
-}
-__device__ __forceinline__ void mbar_expect_tx(uint64_t* bar, uint32_t bytes) {
-    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(smem_u32(bar)), "r"(bytes) : "memory");
-}
-__device__ __forceinline__ void mbar_arrive(uint64_t* bar) {
-    asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(smem_u32(bar)) : "memory");
-}
-__device__ __forceinline__ bool mbar_try_wait(uint64_t* bar, uint32_t parity) {
-    uint32_t ok;
-    asm volatile(
-        "{\n\t.reg .pred p;\n\t"
-        "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
-        "selp.b32 %0, 1, 0, p;\n\t}"
-        : "=r"(ok) : "r"(smem_u32(bar)), "r"(parity) : "memory");
-    return ok != 0;
-}
-__device__ __forceinline__ unsigned long long global_ns() {
-    unsigned long long t;
-    asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
-    return t;
-}
-// Bounded wait.  Returns false when the wait ran out of time or another role gave up.
-__device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity, volatile int* abort_flag, int* error, int code) {
-    if (mbar_try_wait(bar, parity)) return true;
-    const unsigned long long t0 = global_ns();
-    while (true) {
-        if (mbar_try_wait(bar, parity)) return true;
-        if (*abort_flag) return false;
-        if (global_ns() - t0 > kWaitLimitNs) {
-            *abort_flag = 1;
-            atomicExch(error, code);
-            return false;
-        }
-    }
-}
-__device__ __forceinline__ void tma_load_2d(void* smem_dst, const CUtensorMap* tm, int x, int y, uint64_t* bar) {
-    asm volatile(
-        "cp.async.bulk.tensor.2d.shared::cluster.global.tile.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];"
-        ::"r"(smem_u32(smem_dst)), "l"(tm), "r"(x), "r"(y), "r"(smem_u32(bar)) : "memory");
-}
-// Shared -> global tile store, tracked by the issuing thread's bulk async-group.
-__device__ __forceinline__ void tma_store_2d(const CUtensorMap* tm, const void* smem_src, int x, int y) {
-    asm volatile("cp.async.bulk.tensor.2d.global.shared::cta.bulk_group [%0, {%2, %3}], [%1];"
-                 ::"l"(tm), "r"(smem_u32(smem_src)), "r"(x), "r"(y) : "memory");
-    asm volatile("cp.async.bulk.commit_group;" ::: "memory");
-}
-__device__ __forceinline__ void tma_store_wait_read() { asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory"); }
-__device__ __forceinline__ void tma_store_wait_all() { asm volatile("cp.async.bulk.wait_group 0;" ::: "memory"); }
-__device__ __forceinline__ void fence_async_smem() { asm volatile("fence.proxy.async.shared::cta;" ::: "memory"); }
-
-__device__ __forceinline__ void tma_prefetch_desc(const CUtensorMap* tm) {
-    asm volatile("prefetch.tensormap [%0];" ::"l"(tm) : "memory");
-}
-
-__device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
-__device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
-
-__device__ __forceinline__ void tmem_alloc(uint32_t* slot, uint32_t cols) {
-    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(slot)), "r"(cols) : "memory");
-    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
-}
-__device__ __forceinline__ void tmem_dealloc(uint32_t addr, uint32_t cols) {
-    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(addr), "r"(cols) : "memory");
-}
-// D[tmem] (+)= A[smem] * B[smem]
-__device__ __forceinline__ void umma_bf16(uint32_t d_tmem, uint64_t a_desc, uint64_t b_desc, uint32_t idesc, uint32_t accumulate) {
-    asm volatile(
-        "{\n\t.reg .pred p;\n\t"
-        "setp.ne.b32 p, %4, 0;\n\t"
-        "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}"
-        ::"r"(d_tmem), "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(accumulate) : "memory");
-}
-// The mbarrier gets one arrival when all tcgen05 operations issued so far by this thread are done.
-__device__ __forceinline__ void umma_commit(uint64_t* bar) {
-    asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(smem_u32(bar)) : "memory");
-}
-__device__ __forceinline__ void tmem_ld32(uint32_t taddr, uint32_t (&r)[32]) {
-    asm volatile(
-        "tcgen05.ld.sync.aligned.32x32b.x32.b32 "
-        "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, "
-        "%16, %17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31}, [%32];"
-        : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]),
-          "=r"(r[8]), "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15]),
-          "=r"(r[16]), "=r"(r[17]), "=r"(r[18]), "=r"(r[19]), "=r"(r[20]), "=r"(r[21]), "=r"(r[22]), "=r"(r[23]),
-          "=r"(r[24]), "=r"(r[25]), "=r"(r[26]), "=r"(r[27]), "=r"(r[28]), "=r"(r[29]), "=r"(r[30]), "=r"(r[31])
-        : "r"(taddr) : "memory");
-    asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
-}
-
-// Shared-memory matrix descriptor, 128-byte swizzle.  Byte offsets are encoded in 16-byte units.
-//   K-major tile (rows of 128 bytes along the contraction): groups of 8 rows are 1024 bytes
-//     apart (stride offset); the leading offset is not used by swizzled K-major layouts.
-//   MN-major tile (rows of 128 bytes along M/N, one row per contraction index): consecutive
-//     blocks of 64 M/N elements are `lead_bytes` apart, groups of 8 contraction rows 1024 bytes.
-__device__ __forceinline__ uint64_t smem_desc(uint32_t addr, uint32_t lead_bytes, uint32_t stride_bytes) {
-    uint64_t d = 0;
-    d |= (uint64_t)((addr >> 4) & 0x3FFFu);
-    d |= (uint64_t)((lead_bytes >> 4) & 0x3FFFu) << 16;
-    d |= (uint64_t)((stride_bytes >> 4) & 0x3FFFu) << 32;
-    d |= 1ull << 46;                 // descriptor version of this architecture
-    d |= 2ull << 61;                 // 128-byte swizzle
-    return d;
-}
-
-// Instruction descriptor: BF16 x BF16 -> FP32, M = 128, N = bn; major bits: 0 = K-major, 1 = MN-major.
-__device__ __forceinline__ uint32_t instr_desc(int bn, int a_mn_major, int b_mn_major) {
-    return (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)a_mn_major << 15) | ((uint32_t)b_mn_major << 16) |
-           ((uint32_t)(bn >> 3) << 17) | ((uint32_t)(BLOCK_M >> 4) << 24);
-}
 
 struct Item { int prob, m0, n0, kb0, kb1, split; };
 
@@ -200,16 +80,6 @@ __device__ __forceinline__ Item decode_item(const TcParams& P, int item) {
     it.kb0 = it.split * p.kb_per_split;
     it.kb1 = min(p.kblocks, it.kb0 + p.kb_per_split);
     return it;
-}
-
-// Branch-free ELU in six instructions: the epilogues are bound by instruction issue, not by the
-// exponential unit.  ex2.approx.ftz needs no range handling; for z > 0 the exponential may
-// overflow to infinity, which the select discards.
-__device__ __forceinline__ float elu_fast(float z, float alpha) {
-    float e;
-    asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(e) : "f"(z * 1.4426950408889634f));
-    const float neg = fmaf(alpha, e, -alpha);
-    return z > 0.f ? z : neg;
 }
 
 template <int MODE>
@@ -467,6 +337,293 @@ __global__ void __launch_bounds__(kThreads, 1) tc_gemm_kernel(const __grid_const
                 const unsigned long long t0 = global_ns();
                 while (!mbar_try_wait(my_aux, aux_phase) && global_ns() - t0 < kWaitLimitNs) {}
             }
+            tma_store_wait_all();   // stores done before the CTA retires
+        }
+    }
+    tc_fence_before();
+    __syncthreads();
+    if (warp == 1) {
+        tc_fence_after();
+        tmem_dealloc(tmem_base, kTmemCols);
+    }
+}
+
+// ------------------------------------------------------------- weight-stationary products
+// Forward and data-gradient products of a minibatch have few output columns and many rows, and
+// with both operands streamed every 128-row tile re-reads its weight tile from the L2 cache:
+// the cache-to-SM traffic, not the tensor pipe, sets the pace.  Here a CTA belongs to one group
+// = (problem, column tile), loads that group's slice of the weights (all k-blocks, at most
+// 128 KiB) into shared memory once, and then streams only the row tiles of the other operand.
+// Results leave through 32 x 32 tiles (2 KiB, 64-byte swizzle), one or two per epilogue warp.
+constexpr int kWsGroups = 32;
+constexpr int kWsStagesA = 4;
+constexpr uint32_t kWsMaxSlice = 131072;                 // bytes of weights a CTA keeps
+constexpr uint32_t kWsTile = 32 * 32 * 2;                // 2 KiB result tile: 32 rows x 32 bf16
+__host__ __device__ constexpr size_t ws_smem_bytes(uint32_t slice_bytes, int tiles_per_warp) {
+    return 1024 + (size_t)slice_bytes + (size_t)kWsStagesA * kStageA + (size_t)kEpiWarps * tiles_per_warp * kWsTile + 512;
+}
+
+struct WsGroup { int prob, n0, cta_begin, cta_count; };
+struct WsParams {
+    CUtensorMap tmA[kMaxProblems];     // streamed operand, boxes of 64 x 128 rows, 128-byte swizzle
+    CUtensorMap tmB[kMaxProblems];     // weights [columns][contraction], boxes of 64 x bn rows
+    CUtensorMap tmOut[kMaxProblems];   // BF16 output, boxes of 32 columns x 32 rows, 64-byte swizzle
+    CUtensorMap tmAux[kMaxProblems];   // data gradient: stored post-activations, same boxes
+    TcProblem p[kMaxProblems];
+    WsGroup g[kWsGroups];
+    int count, ngroups, grid;
+    int tiles_per_warp;                // result tiles per epilogue warp (1 or 2)
+    uint32_t slice_bytes;              // shared memory reserved for the weight slice (multiple of 1 KiB)
+    float alpha;
+    int* error;
+};
+
+template <int N>
+__device__ __forceinline__ void tma_store_wait_read_n() { asm volatile("cp.async.bulk.wait_group.read %0;" ::"n"(N) : "memory"); }
+
+template <int MODE>
+__global__ void __launch_bounds__(kThreads, 1) ws_gemm_kernel(const __grid_constant__ WsParams P) {
+    extern __shared__ uint8_t smem_raw[];
+    uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
+    uint8_t* sB = smem;
+    uint8_t* sA = sB + P.slice_bytes;
+    uint8_t* sOut = sA + kWsStagesA * kStageA;
+    uint64_t* full = reinterpret_cast<uint64_t*>(sOut + kEpiWarps * P.tiles_per_warp * kWsTile);
+    uint64_t* empty = full + kWsStagesA;
+    uint64_t* tfull = empty + kWsStagesA;
+    uint64_t* tempty = tfull + 2;
+    uint64_t* bfull = tempty + 2;
+    uint64_t* drain = bfull + 1;
+    uint64_t* auxbar = drain + 1;                           // two per epilogue warp
+    uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(auxbar + 2 * kEpiWarps);
+    volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
+
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    if (threadIdx.x == 0) {
+        for (int s = 0; s < kWsStagesA; ++s) { mbar_init(&full[s], 1); mbar_init(&empty[s], 1); }
+        for (int b = 0; b < 2; ++b) { mbar_init(&tfull[b], 1); mbar_init(&tempty[b], kEpiWarps); }
+        mbar_init(bfull, 1);
+        mbar_init(drain, 1);
+        for (int w = 0; w < 2 * kEpiWarps; ++w) mbar_init(&auxbar[w], 1);
+        *abort_flag = 0;
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+        asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+    }
+    // the group of this CTA and its share of the row tiles
+    int gi = 0;
+#pragma unroll 1
+    for (int i = 1; i < P.ngroups; ++i)
+        if ((int)blockIdx.x >= P.g[i].cta_begin) gi = i;
+    const WsGroup G = P.g[gi];
+    const TcProblem& p = P.p[G.prob];
+    const int rank = (int)blockIdx.x - G.cta_begin;
+    const int my_tiles = rank < p.m_tiles ? (p.m_tiles - rank + G.cta_count - 1) / G.cta_count : 0;
+    const uint32_t kb_bytes = (uint32_t)p.bn * BLOCK_K * 2;        // one k-block of the slice
+
+    if (warp == 1) tmem_alloc(tmem_slot, kTmemCols);
+    if (warp == 0 && lane == 0) {
+        tma_prefetch_desc(&P.tmA[G.prob]); tma_prefetch_desc(&P.tmB[G.prob]); tma_prefetch_desc(&P.tmOut[G.prob]);
+        if (MODE == TC_DGRAD) tma_prefetch_desc(&P.tmAux[G.prob]);
+    }
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    const uint32_t tmem_base = *tmem_slot;
+    chain_wait();
+
+    if (warp == 0) {
+        // ================================ TMA producer =================================
+        if (lane == 0 && my_tiles > 0) {
+            mbar_expect_tx(bfull, kb_bytes * (uint32_t)p.kblocks);
+            for (int kb = 0; kb < p.kblocks; ++kb)
+                tma_load_2d(sB + (size_t)kb * kb_bytes, &P.tmB[G.prob], kb * BLOCK_K, G.n0, bfull);
+            int stage = 0; uint32_t phase = 0;
+            uint32_t issued_mask = 0, issued_parity = 0;
+            bool ok = true;
+            for (int local = 0; ok && local < my_tiles; ++local) {
+                const int m0 = (rank + local * G.cta_count) * BLOCK_M;
+                for (int kb = 0; kb < p.kblocks; ++kb) {
+                    if (!mbar_wait(&empty[stage], phase ^ 1u, abort_flag, P.error, 1)) { ok = false; break; }
+                    mbar_expect_tx(&full[stage], kStageA);
+                    tma_load_2d(sA + stage * kStageA, &P.tmA[G.prob], kb * BLOCK_K, m0, &full[stage]);
+                    issued_mask |= 1u << stage;
+                    issued_parity = (issued_parity & ~(1u << stage)) | (phase << stage);
+                    if (++stage == kWsStagesA) { stage = 0; phase ^= 1u; }
+                }
+            }
+            if (!ok) {
+                // let the copies already issued land before the CTA's shared memory goes away
+                const unsigned long long t0 = global_ns();
+                while (!mbar_try_wait(bfull, 0) && global_ns() - t0 < kWaitLimitNs) {}
+                for (int s = 0; s < kWsStagesA; ++s) {
+                    if (!(issued_mask & (1u << s))) continue;
+                    const unsigned long long t1 = global_ns();
+                    while (!mbar_try_wait(&full[s], (issued_parity >> s) & 1u) && global_ns() - t1 < kWaitLimitNs) {}
+                }
+            }
+        }
+    } else if (warp == 1) {
+        // ================================ MMA issuer ===================================
+        if (lane == 0) {
+            int stage = 0; uint32_t phase = 0;
+            bool ok = my_tiles == 0 || mbar_wait(bfull, 0, abort_flag, P.error, 6);
+            const uint32_t idesc = instr_desc(p.bn, 0, 0);
+            const uint32_t b_base = smem_u32(sB);
+            for (int local = 0; ok && local < my_tiles; ++local) {
+                const int buf = local & 1;
+                const uint32_t use = (uint32_t)(local >> 1);
+                if (!mbar_wait(&tempty[buf], (use & 1u) ^ 1u, abort_flag, P.error, 2)) { ok = false; break; }
+                tc_fence_after();
+                const uint32_t d_tmem = tmem_base + (uint32_t)buf * kMaxBN;
+                for (int kb = 0; kb < p.kblocks; ++kb) {
+                    if (!mbar_wait(&full[stage], phase, abort_flag, P.error, 3)) { ok = false; break; }
+                    tc_fence_after();
+                    const uint32_t a_addr = smem_u32(sA + stage * kStageA);
+                    const uint32_t b_addr = b_base + (uint32_t)kb * kb_bytes;
+#pragma unroll
+                    for (int k = 0; k < BLOCK_K / UMMA_K; ++k)
+                        umma_bf16(d_tmem, smem_desc(a_addr + k * (UMMA_K * 2), 16, 1024),
+                                  smem_desc(b_addr + k * (UMMA_K * 2), 16, 1024), idesc, (kb > 0 || k > 0) ? 1u : 0u);
+                    umma_commit(&empty[stage]);       // frees the stage once these MMAs have read it
+                    if (++stage == kWsStagesA) { stage = 0; phase ^= 1u; }
+                }
+                if (ok) umma_commit(&tfull[buf]);     // accumulator complete
+            }
+            chain_release();
+            if (!ok) {
+                umma_commit(drain);
+                const unsigned long long t0 = global_ns();
+                while (!mbar_try_wait(drain, 0) && global_ns() - t0 < kWaitLimitNs) {}
+            }
+        }
+    } else {
+        // ================================ epilogue =====================================
+        const int q = warp & 3;                    // accumulator lanes 32q .. 32q+31
+        const int grp = (warp - 2) >> 2;           // takes the 32-column chunks grp and grp + 4 of the tile
+        // lane r owns row r of a result tile (64 bytes = four 16-byte pieces); piece j is kept at
+        // j ^ ((r >> 1) & 3), the 64-byte swizzle of the tensor map (conflict-free for the warp)
+        uint8_t* tiles = sOut + (size_t)(warp - 2) * P.tiles_per_warp * kWsTile;
+        const int sw = (lane >> 1) & 3;
+        uint64_t* my_aux = &auxbar[2 * (warp - 2)];
+        uint32_t aux_phase = 0;                    // bit i: parity of the next completion of my_aux[i]
+        uint32_t aux_pending = 0;
+        const int nchunks = p.bn / 32;
+        int n_my = 0;                              // chunks of this warp that exist (uniform across the warp)
+        for (int i = 0; i < 2; ++i)
+            if (grp + 4 * i < nchunks && G.n0 + 32 * (grp + 4 * i) < p.n_extent) n_my = i + 1;
+        const bool two_tiles = P.tiles_per_warp == 2;
+        bool ok = true;
+        for (int local = 0; ok && local < my_tiles; ++local) {
+            const int m0 = (rank + local * G.cta_count) * BLOCK_M;
+            const int buf = local & 1;
+            const uint32_t use = (uint32_t)(local >> 1);
+            const int row0 = m0 + 32 * q;
+            if (MODE == TC_DGRAD && n_my > 0) {
+                // stored post-activations of this warp's chunks, fetched while the products run
+                // (every lane has finished reading the tiles of the item before)
+                fence_async_smem();
+                __syncwarp();
+                if (lane == 0) {
+                    tma_store_wait_read_n<0>();
+                    for (int i = 0; i < n_my; ++i) {
+                        mbar_expect_tx(&my_aux[i], kWsTile);
+                        tma_load_2d(tiles + i * kWsTile, &P.tmAux[G.prob], G.n0 + 32 * (grp + 4 * i), row0, &my_aux[i]);
+                    }
+                }
+                aux_pending = (1u << n_my) - 1u;
+                __syncwarp();
+            }
+            if (!mbar_wait(&tfull[buf], use & 1u, abort_flag, P.error, 4)) { ok = false; break; }
+            tc_fence_after();
+            for (int i = 0; i < n_my; ++i) {
+                const int c = grp + 4 * i;
+                const int col = G.n0 + 32 * c;
+                uint8_t* tile = tiles + ((two_tiles && i == 1) ? kWsTile : 0u);
+                uint8_t* tile_row = tile + lane * 64;
+                if (MODE == TC_FWD) {
+                    // the store that last used this tile must have read it
+                    if (lane == 0) {
+                        if (two_tiles && n_my == 2) tma_store_wait_read_n<1>(); else tma_store_wait_read_n<0>();
+                    }
+                    __syncwarp();
+                } else {
+                    if (!mbar_wait(&my_aux[i], (aux_phase >> i) & 1u, abort_flag, P.error, 5)) { ok = false; break; }
+                    aux_phase ^= 1u << i;
+                    aux_pending &= ~(1u << i);
+                }
+                uint32_t acc[32];
+                tmem_ld32(tmem_base + ((uint32_t)(32 * q) << 16) + (uint32_t)(buf * kMaxBN + 32 * c), acc);
+                if (i == n_my - 1) {
+                    // the accumulator has been read: hand the tensor-memory buffer back
+                    tc_fence_before();
+                    __syncwarp();
+                    if (lane == 0) mbar_arrive(&tempty[buf]);
+                }
+                if (MODE == TC_FWD) {
+                    const float4* b4 = reinterpret_cast<const float4*>(p.bias + col);   // zero-padded to the padded width
+#pragma unroll
+                    for (int g = 0; g < 4; ++g) {
+                        const float4 ba = __ldg(b4 + 2 * g), bb = __ldg(b4 + 2 * g + 1);
+                        const float bv[8] = {ba.x, ba.y, ba.z, ba.w, bb.x, bb.y, bb.z, bb.w};
+                        uint32_t o[4];
+#pragma unroll
+                        for (int e = 0; e < 4; ++e) {
+                            const float v0 = elu_fast(__uint_as_float(acc[8 * g + 2 * e]) + bv[2 * e], P.alpha);
+                            const float v1 = elu_fast(__uint_as_float(acc[8 * g + 2 * e + 1]) + bv[2 * e + 1], P.alpha);
+                            __nv_bfloat162 h2 = __floats2bfloat162_rn(v0, v1);
+                            o[e] = *reinterpret_cast<uint32_t*>(&h2);
+                        }
+                        *reinterpret_cast<uint4*>(tile_row + ((g ^ sw) << 4)) = make_uint4(o[0], o[1], o[2], o[3]);
+                    }
+                } else {
+#pragma unroll
+                    for (int g = 0; g < 4; ++g) {
+                        uint4* piece = reinterpret_cast<uint4*>(tile_row + ((g ^ sw) << 4));
+                        const uint4 hv = *piece;
+                        const uint32_t hw[4] = {hv.x, hv.y, hv.z, hv.w};
+                        uint32_t o[4];
+#pragma unroll
+                        for (int e = 0; e < 4; ++e) {
+                            const __nv_bfloat162 h2 = *reinterpret_cast<const __nv_bfloat162*>(&hw[e]);
+                            const float h0 = __low2float(h2), h1 = __high2float(h2);
+                            const float v0 = __uint_as_float(acc[8 * g + 2 * e]) * (h0 > 0.f ? 1.0f : h0 + P.alpha);
+                            const float v1 = __uint_as_float(acc[8 * g + 2 * e + 1]) * (h1 > 0.f ? 1.0f : h1 + P.alpha);
+                            __nv_bfloat162 r2 = __floats2bfloat162_rn(v0, v1);
+                            o[e] = *reinterpret_cast<uint32_t*>(&r2);
+                        }
+                        *piece = make_uint4(o[0], o[1], o[2], o[3]);
+                    }
+                }
+                fence_async_smem();                           // tile writes -> visible to the copy engine
+                __syncwarp();
+                // rows at or beyond the tensor's extent are clipped by the store itself
+                if (lane == 0 && row0 < p.m_extent) tma_store_2d(&P.tmOut[G.prob], tile, col, row0);
+                if (MODE == TC_DGRAD && p.colsum) {
+                    // partial bias gradient: lane l adds column l of the tile's 32 rows (rows past the
+                    // extent hold zeros); two lanes share a word, the 16 words of a row sit in 16 banks
+                    float s = 0.f;
+                    const uint8_t* mine = tile + ((lane & 7) << 1);
+#pragma unroll
+                    for (int r = 0; r < 32; ++r) {
+                        const __nv_bfloat16 v = *reinterpret_cast<const __nv_bfloat16*>(mine + r * 64 + (((lane >> 3) ^ ((r >> 1) & 3)) << 4));
+                        s += __bfloat162float(v);
+                    }
+                    p.colsum[(size_t)(m0 / BLOCK_M * 4 + q) * p.ld_colsum + col + lane] = s;
+                }
+            }
+            if (ok && n_my == 0) {
+                // nothing to read from this accumulator (columns beyond the extent)
+                tc_fence_before();
+                __syncwarp();
+                if (lane == 0) mbar_arrive(&tempty[buf]);
+            }
+        }
+        if (lane == 0) {
+            for (int i = 0; i < 2; ++i)
+                if (aux_pending & (1u << i)) {      // gave up with a load in flight: let it land first
+                    const unsigned long long t0 = global_ns();
+                    while (!mbar_try_wait(&my_aux[i], (aux_phase >> i) & 1u) && global_ns() - t0 < kWaitLimitNs) {}
+                }
             tma_store_wait_all();   // stores done before the CTA retires
         }
     }
@@ -758,36 +915,6 @@ __global__ void convert_weights_kernel(const CvtEntry* __restrict__ table) {
 }
 
 // ------------------------------------------------------------------------------- host side
-typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
-                                  const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
-                                  CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
-
-EncodeTiledFn get_encode_fn() {
-    static EncodeTiledFn fn = nullptr;
-    if (fn) return fn;
-    void* p = nullptr;
-    cudaDriverEntryPointQueryResult qres;
-    if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &p, cudaEnableDefault, &qres) != cudaSuccess ||
-        qres != cudaDriverEntryPointSuccess)
-        return nullptr;
-    fn = reinterpret_cast<EncodeTiledFn>(p);
-    return fn;
-}
-
-// 2-D BF16 tensor [rows][cols] with row stride ld (elements); box = box_cols x box_rows.
-bool make_tmap(CUtensorMap* tm, const void* base, int rows, int cols, int ld, int box_cols, int box_rows,
-               CUtensorMapSwizzle swizzle = CU_TENSOR_MAP_SWIZZLE_128B) {
-    EncodeTiledFn fn = get_encode_fn();
-    if (!fn) return false;
-    const cuuint64_t dims[2] = {(cuuint64_t)cols, (cuuint64_t)rows};
-    const cuuint64_t strides[1] = {(cuuint64_t)ld * 2};
-    const cuuint32_t box[2] = {(cuuint32_t)box_cols, (cuuint32_t)box_rows};
-    const cuuint32_t estr[2] = {1, 1};
-    return fn(tm, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(base), dims, strides, box, estr,
-              CU_TENSOR_MAP_INTERLEAVE_NONE, swizzle, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
-              CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
-}
-
 inline int round_up(int x, int m) { return (x + m - 1) / m * m; }
 inline int pick_bn(int width) { return std::min(kMaxBN, width); }   // widths are multiples of 64
 
@@ -811,6 +938,8 @@ struct UmmaEngine {
     int* error_dev = nullptr;
     int num_sms = 148;
     std::vector<TcParams> act_fwd, act_fwd_critic, upd_fwd, upd_dgrad, upd_wgrad;
+    // weight-stationary forms of upd_fwd / upd_dgrad, entry by entry (grid == 0: not applicable, use the streamed form)
+    std::vector<WsParams> upd_fwd_ws, upd_dgrad_ws;
     // fused forward (one launch for all hidden layers) where the widths allow it, else empty
     std::vector<ChainParams> chain_act, chain_act_critic, chain_upd;
     ColsumBatch colsum{}, colsum_rest{};         // all layers the epilogue does not cover / those minus the last ones
@@ -850,6 +979,7 @@ bool add_rowmajor_problem(TcParams& P, const __nv_bfloat16* A, int rows, int k, 
     p.m_tiles = (rows + BLOCK_M - 1) / BLOCK_M;
     p.n_tiles = (width_out + p.bn - 1) / p.bn;
     p.kblocks = k / BLOCK_K; p.splits = 1; p.kb_per_split = p.kblocks;
+    p.a_ptr = A; p.b_ptr = B; p.k_elems = k;
     if (!make_tmap(&P.tmA[i], A, rows, k, k, BLOCK_K, BLOCK_M)) return false;
     if (!make_tmap(&P.tmB[i], B, width_out, k, k, BLOCK_K, p.bn)) return false;
     P.count++;
@@ -862,6 +992,75 @@ cudaError_t launch_tc(const TcParams& P, int num_sms, cudaStream_t s) {
     const int grid = std::min(P.total_items, num_sms);
     LaunchScope scope_(MODE == TC_FWD ? "tc_gemm_fwd" : MODE == TC_DGRAD ? "tc_gemm_dgrad" : "tc_gemm_wgrad", s);
     return launch_chained(tc_gemm_kernel<MODE>, grid, kThreads, smem_bytes_of(MODE), s, P);
+}
+
+
+// Column tile of a weight-stationary problem: the widest of 256, 192, 128, 64 columns (not beyond
+// the output width) whose slice of the weights, all k-blocks, fits `limit` bytes; 0 if none does.
+int ws_pick_bn(int width_out, int k, uint32_t limit) {
+    for (int bn : {256, 192, 128, 64})
+        if (bn <= std::max(64, std::min(kMaxBN, width_out)) && (size_t)bn * k * 2 <= limit) return bn;
+    return 0;
+}
+
+// The weight-stationary form of a forward / data-gradient launch: same problems, column tiles
+// chosen so that a slice fits shared memory, the SMs shared out among the (problem, column tile)
+// groups in proportion to their work.  W.grid stays 0 when the form does not apply.
+bool make_ws(WsParams& W, const TcParams& T, int mode, int num_sms) {
+    memset(&W, 0, sizeof W);
+    // the data-gradient epilogue prefetches the stored activations of all its chunks: two tiles per warp
+    const uint32_t limit = mode == TC_DGRAD ? kWsMaxSlice / 2 : kWsMaxSlice;
+    uint32_t slice = 0;
+    int ng = 0;
+    struct Cost { long long per_tile; int tiles; };
+    Cost cost[kWsGroups];
+    for (int i = 0; i < T.count; ++i) {
+        const TcProblem& t = T.p[i];
+        const int bn = ws_pick_bn(t.n_extent, t.k_elems, limit);
+        if (bn == 0) return true;
+        TcProblem& p = W.p[i];
+        p = t;
+        p.bn = bn;
+        p.n_tiles = (t.n_extent + bn - 1) / bn;
+        W.tmA[i] = T.tmA[i];
+        if (!make_tmap(&W.tmB[i], t.b_ptr, t.n_extent, t.k_elems, t.k_elems, BLOCK_K, bn)) return false;
+        if (!make_tmap(&W.tmOut[i], t.out16, t.m_extent, t.n_extent, t.ld_out, 32, 32, CU_TENSOR_MAP_SWIZZLE_64B)) return false;
+        if (mode == TC_DGRAD &&
+            !make_tmap(&W.tmAux[i], t.aux16, t.m_extent, t.n_extent, t.ld_aux, 32, 32, CU_TENSOR_MAP_SWIZZLE_64B))
+            return false;
+        slice = std::max(slice, (uint32_t)bn * (uint32_t)t.k_elems * 2u);
+        for (int j = 0; j < p.n_tiles; ++j) {
+            if (ng == kWsGroups) return true;
+            W.g[ng] = WsGroup{i, j * bn, 0, 1};
+            cost[ng] = Cost{(long long)p.kblocks * bn, p.m_tiles};
+            ++ng;
+        }
+    }
+    if (ng == 0 || ng > num_sms) return true;
+    // one CTA per group, then the group whose CTAs have the longest queue gets the next one
+    int left = num_sms - ng;
+    auto queue = [&](int g) { return cost[g].per_tile * ((cost[g].tiles + W.g[g].cta_count - 1) / W.g[g].cta_count); };
+    while (left > 0) {
+        int best = -1;
+        for (int g = 0; g < ng; ++g)
+            if (W.g[g].cta_count < cost[g].tiles && (best < 0 || queue(g) > queue(best))) best = g;
+        if (best < 0) break;
+        W.g[best].cta_count++;
+        --left;
+    }
+    int begin = 0;
+    for (int g = 0; g < ng; ++g) { W.g[g].cta_begin = begin; begin += W.g[g].cta_count; }
+    W.count = T.count; W.ngroups = ng; W.grid = begin;
+    W.slice_bytes = (slice + 1023u) & ~1023u;
+    W.tiles_per_warp = (mode == TC_DGRAD || W.slice_bytes <= kWsMaxSlice / 2) ? 2 : 1;
+    W.alpha = T.alpha; W.error = T.error;
+    return true;
+}
+
+template <int MODE>
+cudaError_t launch_ws(const WsParams& W, cudaStream_t s) {
+    LaunchScope scope_(MODE == TC_FWD ? "tc_gemm_fwd" : "tc_gemm_dgrad", s);
+    return launch_chained(ws_gemm_kernel<MODE>, W.grid, kThreads, ws_smem_bytes(W.slice_bytes, W.tiles_per_warp), s, W);
 }
 
 // The program of one net for the fused forward; false when the widths do not fit the kernel
@@ -998,6 +1197,9 @@ UmmaEngine* umma_create(const UmmaSetup& s, std::string* err) {
         return failmsg("could not reserve shared memory for the tensor-core kernels");
     if (cudaFuncSetAttribute(chain_fwd_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kChainSmem) != cudaSuccess)
         return failmsg("could not reserve shared memory for the fused forward kernel");
+    if (cudaFuncSetAttribute(ws_gemm_kernel<TC_FWD>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)ws_smem_bytes(kWsMaxSlice, 1)) != cudaSuccess ||
+        cudaFuncSetAttribute(ws_gemm_kernel<TC_DGRAD>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)ws_smem_bytes(kWsMaxSlice / 2, 2)) != cudaSuccess)
+        return failmsg("could not reserve shared memory for the weight-stationary kernels");
     UmmaEngine* e = new UmmaEngine();
     e->s = s;
     e->num_sms = prop.multiProcessorCount;
@@ -1136,6 +1338,17 @@ UmmaEngine* umma_create(const UmmaSetup& s, std::string* err) {
         finish_params(P, alpha, e->error_dev);
         e->upd_dgrad.push_back(P);
     }
+    // ---- weight-stationary forms of the minibatch forward and data-gradient launches ------------
+    for (const TcParams& T : e->upd_fwd) {
+        WsParams W;
+        if (!make_ws(W, T, TC_FWD, e->num_sms)) return bail("tensor map encoding failed");
+        e->upd_fwd_ws.push_back(W);
+    }
+    for (const TcParams& T : e->upd_dgrad) {
+        WsParams W;
+        if (!make_ws(W, T, TC_DGRAD, e->num_sms)) return bail("tensor map encoding failed");
+        e->upd_dgrad_ws.push_back(W);
+    }
     // ---- weight-gradient problems (all layers of both nets, heads included) ------------------
     {
         const int kblocks = (R + BLOCK_K - 1) / BLOCK_K;
@@ -1271,8 +1484,9 @@ void umma_gather_targets(UmmaEngine* e, GatherArgs* g) {
 
 cudaError_t umma_update_forward(UmmaEngine* e) {
     if (!e->chain_upd.empty()) return launch_chain(e->chain_upd[0], e->num_sms, e->s.stream);
-    for (const TcParams& P : e->upd_fwd) {
-        cudaError_t err = launch_tc<TC_FWD>(P, e->num_sms, e->s.stream);
+    for (size_t i = 0; i < e->upd_fwd.size(); ++i) {
+        cudaError_t err = e->upd_fwd_ws[i].grid > 0 ? launch_ws<TC_FWD>(e->upd_fwd_ws[i], e->s.stream)
+                                                    : launch_tc<TC_FWD>(e->upd_fwd[i], e->num_sms, e->s.stream);
         if (err != cudaSuccess) return err;
     }
     return cudaSuccess;
@@ -1290,8 +1504,9 @@ void umma_head_loss_targets(UmmaEngine* e, HeadLossArgs* a) {
 
 cudaError_t umma_update_backward(UmmaEngine* e, bool last_bias_done) {
     cudaError_t err;
-    for (const TcParams& P : e->upd_dgrad) {
-        err = launch_tc<TC_DGRAD>(P, e->num_sms, e->s.stream);
+    for (size_t i = 0; i < e->upd_dgrad.size(); ++i) {
+        err = e->upd_dgrad_ws[i].grid > 0 ? launch_ws<TC_DGRAD>(e->upd_dgrad_ws[i], e->s.stream)
+                                          : launch_tc<TC_DGRAD>(e->upd_dgrad[i], e->num_sms, e->s.stream);
         if (err != cudaSuccess) return err;
     }
     for (const TcParams& P : e->upd_wgrad) {
