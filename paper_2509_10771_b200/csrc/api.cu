@@ -66,12 +66,15 @@ struct rslrl_ctx {
     // update workspace
     int Bmb = 0, R = 0, splits = 1, kchunk = 0;
     float *x_a = nullptr, *x_c = nullptr;
-    float *act_mb = nullptr, *mu_old = nullptr, *sigma_old = nullptr;
-    float *logp_old = nullptr, *v_old = nullptr, *ret_mb = nullptr, *adv_mb = nullptr;
+    // gathered minibatch items, two sets: while one minibatch is worked on, the next is gathered
+    float *act_mb[2] = {}, *mu_old[2] = {}, *sigma_old[2] = {};
+    float *logp_old[2] = {}, *v_old[2] = {}, *ret_mb[2] = {}, *adv_mb[2] = {};
+    cudaStream_t side = nullptr;          // the gather of the next minibatch runs here
+    cudaEvent_t ev_ready = nullptr, ev_gathered[2] = {}, ev_consumed[2] = {};
     void* up_h[2][kMaxLayers] = {};
     void* up_dz[2][kMaxLayers] = {};
     float *dmu = nullptr, *dv = nullptr; int lddmu = 0;
-    int* perm = nullptr;                  // [T*N] shuffle of the current epoch
+    int* perm = nullptr;                  // [epochs][T*N] shuffles of the current iteration
     float *partials = nullptr, *block_partials = nullptr, *sumsq_partials = nullptr, *loss_sums = nullptr;
     float* stats_dev = nullptr; float* stats_host = nullptr; int max_stat_rows = 0;
     SymTables sym{};
@@ -190,6 +193,7 @@ HeadParams head_params(const rslrl_ctx* c) {
 void fill_setup(const rslrl_ctx* c, UmmaSetup& us) {
     us.model = c->mc; us.N = c->st.N; us.Bmb = c->Bmb; us.R = c->R; us.stream = c->stream;
     us.param = c->param; us.P_dev = c->P_dev; us.partials = c->partials; us.splits = c->splits;
+    us.logstd_off = c->logstd_off;
     const Net* nets[2] = {&c->actor, &c->critic};
     for (int ni = 0; ni < 2; ++ni) {
         us.nl[ni] = nets[ni]->nl; us.in_dim[ni] = nets[ni]->in_dim;
@@ -322,6 +326,12 @@ const char* rslrl_last_error(const rslrl_ctx* c) { return c ? c->err.c_str() : g
 rslrl_status rslrl_destroy(rslrl_ctx* c) {
     if (!c) return RSLRL_ERR_INVALID_ARG;
     cudaStreamSynchronize(c->stream);
+    if (c->side) { cudaStreamSynchronize(c->side); cudaStreamDestroy(c->side); }
+    if (c->ev_ready) cudaEventDestroy(c->ev_ready);
+    for (int b = 0; b < 2; ++b) {
+        if (c->ev_gathered[b]) cudaEventDestroy(c->ev_gathered[b]);
+        if (c->ev_consumed[b]) cudaEventDestroy(c->ev_consumed[b]);
+    }
     if (c->umma) umma_destroy(c->umma);
     for (void* p : c->allocs) cudaFree(p);
     if (c->stats_host) cudaFreeHost(c->stats_host);
@@ -395,12 +405,14 @@ rslrl_status rslrl_create(const rslrl_model_cfg* m, const rslrl_ppo_cfg* p, void
     }
     c->kchunk = round_up((c->R + c->splits - 1) / c->splits, 8);
     c->lddmu = as;
-    A_(c->act_mb, (size_t)c->R * as); A_(c->mu_old, (size_t)c->Bmb * as); A_(c->sigma_old, (size_t)c->Bmb * as);
-    A_(c->logp_old, c->Bmb); A_(c->v_old, c->Bmb); A_(c->ret_mb, c->Bmb); A_(c->adv_mb, c->Bmb);
+    for (int b = 0; b < 2; ++b) {
+        A_(c->act_mb[b], (size_t)c->R * as); A_(c->mu_old[b], (size_t)c->Bmb * as); A_(c->sigma_old[b], (size_t)c->Bmb * as);
+        A_(c->logp_old[b], c->Bmb); A_(c->v_old[b], c->Bmb); A_(c->ret_mb[b], c->Bmb); A_(c->adv_mb[b], c->Bmb);
+    }
     A_(c->dmu, (size_t)c->R * as); A_(c->dv, (size_t)c->R * 4);
-    A_(c->perm, (size_t)B);
+    A_(c->perm, (size_t)B * p->epochs);
     A_(c->partials, (size_t)c->splits * c->P_dev);
-    A_(c->block_partials, (size_t)head_loss_blocks(c->Bmb) * head_partial_stride());
+    A_(c->block_partials, (size_t)std::max(head_loss_blocks(c->Bmb), 256) * head_partial_stride());
     A_(c->sumsq_partials, reduce_blocks(c->P_dev)); A_(c->loss_sums, 8);
     c->max_stat_rows = p->epochs * p->minibatches;
     A_(c->stats_dev, (size_t)c->max_stat_rows * 8);
@@ -423,6 +435,14 @@ rslrl_status rslrl_create(const rslrl_model_cfg* m, const rslrl_ppo_cfg* p, void
         std::string uerr;
         c->umma = umma_create(us, &uerr);
         if (!c->umma) { c->err = "tensor-core engine: " + uerr; return bail(RSLRL_ERR_UNSUPPORTED); }
+        if (umma_two_input_buffers(c->umma)) {
+            bool okv = cudaStreamCreateWithFlags(&c->side, cudaStreamNonBlocking) == cudaSuccess &&
+                       cudaEventCreateWithFlags(&c->ev_ready, cudaEventDisableTiming) == cudaSuccess;
+            for (int b = 0; b < 2 && okv; ++b)
+                okv = cudaEventCreateWithFlags(&c->ev_gathered[b], cudaEventDisableTiming) == cudaSuccess &&
+                      cudaEventCreateWithFlags(&c->ev_consumed[b], cudaEventDisableTiming) == cudaSuccess;
+            if (!okv) { c->err = "could not create the gather stream"; return bail(RSLRL_ERR_CUDA); }
+        }
     }
     // staging for the host-buffer variants
     A_(c->stage_obs_a, (size_t)N * m->actor_obs_dim);
@@ -600,26 +620,65 @@ rslrl_status rslrl_ppo_update_steps(rslrl_ctx* c, int32_t max_steps, rslrl_updat
     const HeadParams hp_base = head_params(c);
     const Layer& ha = c->actor.L[c->actor.nl - 1];
     const Layer& hc = c->critic.L[c->critic.nl - 1];
+    // Minibatch `step` gathered into input set `buf` on stream `st`.
+    auto enqueue_gather = [&](int step, int buf, cudaStream_t st) -> rslrl_status {
+        const int e = step / pc.minibatches, k = step % pc.minibatches;
+        GatherArgs g{};
+        g.obs_a = c->st.obs_actor; g.obs_c = c->st.obs_critic; g.actions = c->st.actions; g.mu = c->st.mu;
+        g.sigma = c->st.sigma; g.logp = c->st.logp; g.values = c->st.values; g.returns = c->st.returns;
+        g.adv = c->st.advantages;
+        g.N = N; g.sa = c->st.obs_a_stride; g.sc = c->st.obs_c_stride; g.as = c->st.act_stride;
+        g.Da = c->mc.actor_obs_dim; g.Dc = c->mc.critic_obs_dim; g.A = A; g.shared_obs = c->mc.shared_obs;
+        g.x_a = c->x_a; g.x_c = c->x_c; g.ldxa = c->actor.in_ld; g.ldxc = c->critic.in_ld;
+        if (c->umma) umma_gather_targets(c->umma, &g, buf);
+        g.act_mb = c->act_mb[buf]; g.mu_old = c->mu_old[buf]; g.sigma_old = c->sigma_old[buf];
+        g.logp_old = c->logp_old[buf]; g.v_old = c->v_old[buf]; g.ret = c->ret_mb[buf]; g.adv_mb = c->adv_mb[buf];
+        g.rows = c->perm + (size_t)e * T * N + (size_t)k * c->Bmb; g.Bmb = c->Bmb; g.sym = pc.sym_enable; g.st = c->sym;
+        CU(c, launch_gather(g, st));
+        return RSLRL_OK;
+    };
+    // With a gather stream, minibatch s+1 is gathered into the other input set while minibatch s is
+    // worked on: the gather waits for the kernels that read that set two steps ago, the step for its gather.
+    const bool overlap = c->side != nullptr;
+    if (overlap) {
+        CU(c, cudaEventRecord(c->ev_ready, c->stream));           // advantages and returns are in storage
+        CU(c, cudaStreamWaitEvent(c->side, c->ev_ready, 0));
+    }
+    // the shuffles of all epochs of this iteration, resolved in one launch
+    CU(c, launch_perm_epochs(pc.seed, c->iteration, pc.epochs, (uint32_t)(T * N), c->perm, overlap ? c->side : c->stream));
+    if (overlap) {
+        TRY(enqueue_gather(0, 0, c->side));
+        CU(c, cudaEventRecord(c->ev_gathered[0], c->side));
+    }
     int done_steps = 0;
     for (int e = 0; e < pc.epochs && done_steps < nsteps; ++e) {
         for (int k = 0; k < pc.minibatches && done_steps < nsteps; ++k, ++done_steps) {
             // ---- gather -----------------------------------------------------------------
-            GatherArgs g{};
-            g.obs_a = c->st.obs_actor; g.obs_c = c->st.obs_critic; g.actions = c->st.actions; g.mu = c->st.mu;
-            g.sigma = c->st.sigma; g.logp = c->st.logp; g.values = c->st.values; g.returns = c->st.returns;
-            g.adv = c->st.advantages;
-            g.N = N; g.sa = c->st.obs_a_stride; g.sc = c->st.obs_c_stride; g.as = c->st.act_stride;
-            g.Da = c->mc.actor_obs_dim; g.Dc = c->mc.critic_obs_dim; g.A = A; g.shared_obs = c->mc.shared_obs;
-            g.x_a = c->x_a; g.x_c = c->x_c; g.ldxa = c->actor.in_ld; g.ldxc = c->critic.in_ld;
-            if (c->umma) umma_gather_targets(c->umma, &g);
-            g.act_mb = c->act_mb; g.mu_old = c->mu_old; g.sigma_old = c->sigma_old;
-            g.logp_old = c->logp_old; g.v_old = c->v_old; g.ret = c->ret_mb; g.adv_mb = c->adv_mb;
-            g.rows = c->perm + (size_t)k * c->Bmb; g.Bmb = c->Bmb; g.sym = pc.sym_enable; g.st = c->sym;
-            if (k == 0)   // the epoch's shuffle, resolved once for all of its minibatches
-                CU(c, launch_perm_rows(pc.seed, c->iteration, (uint32_t)e, (uint32_t)(T * N), 0u, T * N, c->perm, c->stream));
-            CU(c, launch_gather(g, c->stream));
-            // ---- forward ----------------------------------------------------------------
+            const int buf = overlap ? (done_steps & 1) : 0;
+            if (overlap) {
+                if (done_steps + 1 < nsteps) {
+                    if (done_steps >= 1) CU(c, cudaStreamWaitEvent(c->side, c->ev_consumed[buf ^ 1], 0));
+                    TRY(enqueue_gather(done_steps + 1, buf ^ 1, c->side));
+                    CU(c, cudaEventRecord(c->ev_gathered[buf ^ 1], c->side));
+                }
+                CU(c, cudaStreamWaitEvent(c->stream, c->ev_gathered[buf], 0));
+            } else {
+                TRY(enqueue_gather(done_steps, 0, c->stream));
+            }
+            // ---- forward, heads, loss, backward ----------------------------------------------
+            const bool fused = c->umma && umma_has_step_chain(c->umma);
             HeadLossArgs hl{};
+            if (fused) {
+                // row-local work in one kernel, then the weight-gradient partials
+                StepChainLoss sl{};
+                sl.act_mb = c->act_mb[buf]; sl.mu_old = c->mu_old[buf]; sl.sigma_old = c->sigma_old[buf]; sl.as = c->st.act_stride;
+                sl.logp_old = c->logp_old[buf]; sl.v_old = c->v_old[buf]; sl.ret = c->ret_mb[buf]; sl.adv = c->adv_mb[buf];
+                sl.clip = pc.clip; sl.value_clip = pc.value_clip; sl.value_coef = pc.value_coef;
+                sl.use_clipped_value_loss = pc.use_clipped_value_loss;
+                sl.block_partials = c->block_partials;
+                CU(c, umma_step_chain(c->umma, sl, &hl.nblocks_used));
+                CU(c, umma_update_wgrad(c->umma));
+            } else {
             if (c->prec == RSLRL_FP32) {
                 TRY(forward_hidden_fp32(c, true, true, c->x_a, c->mc.shared_obs ? c->x_a : c->x_c, c->R, c->up_h));
                 hl.Ha = c->up_h[0][c->actor.nl - 2]; hl.ldha = c->actor.hid_ld[c->actor.nl - 2];
@@ -628,12 +687,12 @@ rslrl_status rslrl_ppo_update_steps(rslrl_ctx* c, int32_t max_steps, rslrl_updat
                 hl.dZa = c->up_dz[0][c->actor.nl - 2]; hl.lddza = hl.ldha;
                 hl.dZc = c->up_dz[1][c->critic.nl - 2]; hl.lddzc = hl.ldhc;
             } else {
-                CU(c, umma_update_forward(c->umma));
+                CU(c, umma_update_forward(c->umma, buf));
                 umma_head_loss_targets(c->umma, &hl);
             }
             hl.hp = hp_base;
-            hl.act_mb = c->act_mb; hl.mu_old = c->mu_old; hl.sigma_old = c->sigma_old; hl.as = c->st.act_stride;
-            hl.logp_old = c->logp_old; hl.v_old = c->v_old; hl.ret = c->ret_mb; hl.adv = c->adv_mb;
+            hl.act_mb = c->act_mb[buf]; hl.mu_old = c->mu_old[buf]; hl.sigma_old = c->sigma_old[buf]; hl.as = c->st.act_stride;
+            hl.logp_old = c->logp_old[buf]; hl.v_old = c->v_old[buf]; hl.ret = c->ret_mb[buf]; hl.adv = c->adv_mb[buf];
             hl.act_sign = c->sym.act_sign; hl.act_perm = c->sym.act_perm;
             hl.Bmb = c->Bmb; hl.sym = pc.sym_enable;
             hl.h.clip = pc.clip; hl.h.value_clip = pc.value_clip; hl.h.value_coef = pc.value_coef;
@@ -644,7 +703,9 @@ rslrl_status rslrl_ppo_update_steps(rslrl_ctx* c, int32_t max_steps, rslrl_updat
             CU(c, launch_head_loss(hl, c->stream));
             // ---- backward ---------------------------------------------------------------
             if (c->prec == RSLRL_FP32) TRY(backward_fp32(c));
-            else CU(c, umma_update_backward(c->umma, hl.colsum_written != 0));
+            else CU(c, umma_update_backward(c->umma, hl.colsum_written != 0, buf));
+            }
+            if (overlap) CU(c, cudaEventRecord(c->ev_consumed[buf], c->stream));   // this input set may be refilled
             // ---- reduce, clip, adaptive lr, Adam ------------------------------------------
             ReduceArgs r{};
             r.partials = c->partials; r.splits = c->splits; r.split_stride = c->P_dev;
@@ -652,7 +713,8 @@ rslrl_status rslrl_ppo_update_steps(rslrl_ctx* c, int32_t max_steps, rslrl_updat
             r.block_partials = c->block_partials; r.nblocks = hl.nblocks_used;
             r.off_ba = (int)ha.b_off; r.off_logstd = (int)c->logstd_off; r.off_bc = (int)hc.b_off; r.A = A;
             r.entropy_coef = pc.entropy_coef; r.log_std = c->param + c->logstd_off; r.loss_sums = c->loss_sums;
-            if (c->umma) umma_fill_bias_sources(c->umma, &r, hl);
+            if (fused) umma_fill_step_bias_sources(c->umma, &r);
+            else if (c->umma) umma_fill_bias_sources(c->umma, &r, hl);
             CU(c, launch_reduce(r, c->stream));
             AdamArgs ad{};
             ad.param = c->param; ad.m = c->adam_m; ad.v = c->adam_v; ad.grad = c->grad; ad.P = c->P_dev;

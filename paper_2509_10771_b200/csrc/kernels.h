@@ -131,6 +131,9 @@ struct GatherArgs {
 cudaError_t launch_gather(const GatherArgs& a, cudaStream_t stream);
 cudaError_t launch_perm_rows(uint64_t seed, uint32_t iteration, uint32_t epoch, uint32_t batch,
                              uint32_t first, int count, int* rows_out, cudaStream_t stream);
+// The shuffles of epochs 0 .. epochs-1 of one iteration in one launch: rows_out[epoch][batch].
+cudaError_t launch_perm_epochs(uint64_t seed, uint32_t iteration, int epochs, uint32_t batch, int* rows_out,
+                               cudaStream_t stream);
 
 struct LossHyper {
     float clip, value_clip, value_coef, entropy_coef, sym_coef, alpha;

@@ -12,9 +12,11 @@
 // the host reads, drains its own asynchronous work, frees its tensor memory and returns.
 #include "umma.h"
 #include "tc_ptx.cuh"
+#include "step_chain.h"
 
 #include <cuda.h>
 #include <algorithm>
+#include <cstdlib>
 #include <cstring>
 #include <vector>
 
@@ -47,7 +49,7 @@ struct TcProblem {
     const __nv_bfloat16* aux16; int ld_aux;
     float* out32; int ld_out32; long long split_stride;
     float* colsum; int ld_colsum;  // data gradient: column sums of each 32-row slice, [4 m_tiles][ld_colsum] (may be null)
-    const __nv_bfloat16* a_ptr; const __nv_bfloat16* b_ptr; int k_elems;   // host side: operands [rows][k], [columns][k]
+    int net_id, layer_id;          // host side: which net and layer the problem belongs to
 };
 
 struct TcParams {
@@ -337,293 +339,6 @@ __global__ void __launch_bounds__(kThreads, 1) tc_gemm_kernel(const __grid_const
                 const unsigned long long t0 = global_ns();
                 while (!mbar_try_wait(my_aux, aux_phase) && global_ns() - t0 < kWaitLimitNs) {}
             }
-            tma_store_wait_all();   // stores done before the CTA retires
-        }
-    }
-    tc_fence_before();
-    __syncthreads();
-    if (warp == 1) {
-        tc_fence_after();
-        tmem_dealloc(tmem_base, kTmemCols);
-    }
-}
-
-// ------------------------------------------------------------- weight-stationary products
-// Forward and data-gradient products of a minibatch have few output columns and many rows, and
-// with both operands streamed every 128-row tile re-reads its weight tile from the L2 cache:
-// the cache-to-SM traffic, not the tensor pipe, sets the pace.  Here a CTA belongs to one group
-// = (problem, column tile), loads that group's slice of the weights (all k-blocks, at most
-// 128 KiB) into shared memory once, and then streams only the row tiles of the other operand.
-// Results leave through 32 x 32 tiles (2 KiB, 64-byte swizzle), one or two per epilogue warp.
-constexpr int kWsGroups = 32;
-constexpr int kWsStagesA = 4;
-constexpr uint32_t kWsMaxSlice = 131072;                 // bytes of weights a CTA keeps
-constexpr uint32_t kWsTile = 32 * 32 * 2;                // 2 KiB result tile: 32 rows x 32 bf16
-__host__ __device__ constexpr size_t ws_smem_bytes(uint32_t slice_bytes, int tiles_per_warp) {
-    return 1024 + (size_t)slice_bytes + (size_t)kWsStagesA * kStageA + (size_t)kEpiWarps * tiles_per_warp * kWsTile + 512;
-}
-
-struct WsGroup { int prob, n0, cta_begin, cta_count; };
-struct WsParams {
-    CUtensorMap tmA[kMaxProblems];     // streamed operand, boxes of 64 x 128 rows, 128-byte swizzle
-    CUtensorMap tmB[kMaxProblems];     // weights [columns][contraction], boxes of 64 x bn rows
-    CUtensorMap tmOut[kMaxProblems];   // BF16 output, boxes of 32 columns x 32 rows, 64-byte swizzle
-    CUtensorMap tmAux[kMaxProblems];   // data gradient: stored post-activations, same boxes
-    TcProblem p[kMaxProblems];
-    WsGroup g[kWsGroups];
-    int count, ngroups, grid;
-    int tiles_per_warp;                // result tiles per epilogue warp (1 or 2)
-    uint32_t slice_bytes;              // shared memory reserved for the weight slice (multiple of 1 KiB)
-    float alpha;
-    int* error;
-};
-
-template <int N>
-__device__ __forceinline__ void tma_store_wait_read_n() { asm volatile("cp.async.bulk.wait_group.read %0;" ::"n"(N) : "memory"); }
-
-template <int MODE>
-__global__ void __launch_bounds__(kThreads, 1) ws_gemm_kernel(const __grid_constant__ WsParams P) {
-    extern __shared__ uint8_t smem_raw[];
-    uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
-    uint8_t* sB = smem;
-    uint8_t* sA = sB + P.slice_bytes;
-    uint8_t* sOut = sA + kWsStagesA * kStageA;
-    uint64_t* full = reinterpret_cast<uint64_t*>(sOut + kEpiWarps * P.tiles_per_warp * kWsTile);
-    uint64_t* empty = full + kWsStagesA;
-    uint64_t* tfull = empty + kWsStagesA;
-    uint64_t* tempty = tfull + 2;
-    uint64_t* bfull = tempty + 2;
-    uint64_t* drain = bfull + 1;
-    uint64_t* auxbar = drain + 1;                           // two per epilogue warp
-    uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(auxbar + 2 * kEpiWarps);
-    volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
-
-    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-    if (threadIdx.x == 0) {
-        for (int s = 0; s < kWsStagesA; ++s) { mbar_init(&full[s], 1); mbar_init(&empty[s], 1); }
-        for (int b = 0; b < 2; ++b) { mbar_init(&tfull[b], 1); mbar_init(&tempty[b], kEpiWarps); }
-        mbar_init(bfull, 1);
-        mbar_init(drain, 1);
-        for (int w = 0; w < 2 * kEpiWarps; ++w) mbar_init(&auxbar[w], 1);
-        *abort_flag = 0;
-        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
-        asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
-    }
-    // the group of this CTA and its share of the row tiles
-    int gi = 0;
-#pragma unroll 1
-    for (int i = 1; i < P.ngroups; ++i)
-        if ((int)blockIdx.x >= P.g[i].cta_begin) gi = i;
-    const WsGroup G = P.g[gi];
-    const TcProblem& p = P.p[G.prob];
-    const int rank = (int)blockIdx.x - G.cta_begin;
-    const int my_tiles = rank < p.m_tiles ? (p.m_tiles - rank + G.cta_count - 1) / G.cta_count : 0;
-    const uint32_t kb_bytes = (uint32_t)p.bn * BLOCK_K * 2;        // one k-block of the slice
-
-    if (warp == 1) tmem_alloc(tmem_slot, kTmemCols);
-    if (warp == 0 && lane == 0) {
-        tma_prefetch_desc(&P.tmA[G.prob]); tma_prefetch_desc(&P.tmB[G.prob]); tma_prefetch_desc(&P.tmOut[G.prob]);
-        if (MODE == TC_DGRAD) tma_prefetch_desc(&P.tmAux[G.prob]);
-    }
-    tc_fence_before();
-    __syncthreads();
-    tc_fence_after();
-    const uint32_t tmem_base = *tmem_slot;
-    chain_wait();
-
-    if (warp == 0) {
-        // ================================ TMA producer =================================
-        if (lane == 0 && my_tiles > 0) {
-            mbar_expect_tx(bfull, kb_bytes * (uint32_t)p.kblocks);
-            for (int kb = 0; kb < p.kblocks; ++kb)
-                tma_load_2d(sB + (size_t)kb * kb_bytes, &P.tmB[G.prob], kb * BLOCK_K, G.n0, bfull);
-            int stage = 0; uint32_t phase = 0;
-            uint32_t issued_mask = 0, issued_parity = 0;
-            bool ok = true;
-            for (int local = 0; ok && local < my_tiles; ++local) {
-                const int m0 = (rank + local * G.cta_count) * BLOCK_M;
-                for (int kb = 0; kb < p.kblocks; ++kb) {
-                    if (!mbar_wait(&empty[stage], phase ^ 1u, abort_flag, P.error, 1)) { ok = false; break; }
-                    mbar_expect_tx(&full[stage], kStageA);
-                    tma_load_2d(sA + stage * kStageA, &P.tmA[G.prob], kb * BLOCK_K, m0, &full[stage]);
-                    issued_mask |= 1u << stage;
-                    issued_parity = (issued_parity & ~(1u << stage)) | (phase << stage);
-                    if (++stage == kWsStagesA) { stage = 0; phase ^= 1u; }
-                }
-            }
-            if (!ok) {
-                // let the copies already issued land before the CTA's shared memory goes away
-                const unsigned long long t0 = global_ns();
-                while (!mbar_try_wait(bfull, 0) && global_ns() - t0 < kWaitLimitNs) {}
-                for (int s = 0; s < kWsStagesA; ++s) {
-                    if (!(issued_mask & (1u << s))) continue;
-                    const unsigned long long t1 = global_ns();
-                    while (!mbar_try_wait(&full[s], (issued_parity >> s) & 1u) && global_ns() - t1 < kWaitLimitNs) {}
-                }
-            }
-        }
-    } else if (warp == 1) {
-        // ================================ MMA issuer ===================================
-        if (lane == 0) {
-            int stage = 0; uint32_t phase = 0;
-            bool ok = my_tiles == 0 || mbar_wait(bfull, 0, abort_flag, P.error, 6);
-            const uint32_t idesc = instr_desc(p.bn, 0, 0);
-            const uint32_t b_base = smem_u32(sB);
-            for (int local = 0; ok && local < my_tiles; ++local) {
-                const int buf = local & 1;
-                const uint32_t use = (uint32_t)(local >> 1);
-                if (!mbar_wait(&tempty[buf], (use & 1u) ^ 1u, abort_flag, P.error, 2)) { ok = false; break; }
-                tc_fence_after();
-                const uint32_t d_tmem = tmem_base + (uint32_t)buf * kMaxBN;
-                for (int kb = 0; kb < p.kblocks; ++kb) {
-                    if (!mbar_wait(&full[stage], phase, abort_flag, P.error, 3)) { ok = false; break; }
-                    tc_fence_after();
-                    const uint32_t a_addr = smem_u32(sA + stage * kStageA);
-                    const uint32_t b_addr = b_base + (uint32_t)kb * kb_bytes;
-#pragma unroll
-                    for (int k = 0; k < BLOCK_K / UMMA_K; ++k)
-                        umma_bf16(d_tmem, smem_desc(a_addr + k * (UMMA_K * 2), 16, 1024),
-                                  smem_desc(b_addr + k * (UMMA_K * 2), 16, 1024), idesc, (kb > 0 || k > 0) ? 1u : 0u);
-                    umma_commit(&empty[stage]);       // frees the stage once these MMAs have read it
-                    if (++stage == kWsStagesA) { stage = 0; phase ^= 1u; }
-                }
-                if (ok) umma_commit(&tfull[buf]);     // accumulator complete
-            }
-            chain_release();
-            if (!ok) {
-                umma_commit(drain);
-                const unsigned long long t0 = global_ns();
-                while (!mbar_try_wait(drain, 0) && global_ns() - t0 < kWaitLimitNs) {}
-            }
-        }
-    } else {
-        // ================================ epilogue =====================================
-        const int q = warp & 3;                    // accumulator lanes 32q .. 32q+31
-        const int grp = (warp - 2) >> 2;           // takes the 32-column chunks grp and grp + 4 of the tile
-        // lane r owns row r of a result tile (64 bytes = four 16-byte pieces); piece j is kept at
-        // j ^ ((r >> 1) & 3), the 64-byte swizzle of the tensor map (conflict-free for the warp)
-        uint8_t* tiles = sOut + (size_t)(warp - 2) * P.tiles_per_warp * kWsTile;
-        const int sw = (lane >> 1) & 3;
-        uint64_t* my_aux = &auxbar[2 * (warp - 2)];
-        uint32_t aux_phase = 0;                    // bit i: parity of the next completion of my_aux[i]
-        uint32_t aux_pending = 0;
-        const int nchunks = p.bn / 32;
-        int n_my = 0;                              // chunks of this warp that exist (uniform across the warp)
-        for (int i = 0; i < 2; ++i)
-            if (grp + 4 * i < nchunks && G.n0 + 32 * (grp + 4 * i) < p.n_extent) n_my = i + 1;
-        const bool two_tiles = P.tiles_per_warp == 2;
-        bool ok = true;
-        for (int local = 0; ok && local < my_tiles; ++local) {
-            const int m0 = (rank + local * G.cta_count) * BLOCK_M;
-            const int buf = local & 1;
-            const uint32_t use = (uint32_t)(local >> 1);
-            const int row0 = m0 + 32 * q;
-            if (MODE == TC_DGRAD && n_my > 0) {
-                // stored post-activations of this warp's chunks, fetched while the products run
-                // (every lane has finished reading the tiles of the item before)
-                fence_async_smem();
-                __syncwarp();
-                if (lane == 0) {
-                    tma_store_wait_read_n<0>();
-                    for (int i = 0; i < n_my; ++i) {
-                        mbar_expect_tx(&my_aux[i], kWsTile);
-                        tma_load_2d(tiles + i * kWsTile, &P.tmAux[G.prob], G.n0 + 32 * (grp + 4 * i), row0, &my_aux[i]);
-                    }
-                }
-                aux_pending = (1u << n_my) - 1u;
-                __syncwarp();
-            }
-            if (!mbar_wait(&tfull[buf], use & 1u, abort_flag, P.error, 4)) { ok = false; break; }
-            tc_fence_after();
-            for (int i = 0; i < n_my; ++i) {
-                const int c = grp + 4 * i;
-                const int col = G.n0 + 32 * c;
-                uint8_t* tile = tiles + ((two_tiles && i == 1) ? kWsTile : 0u);
-                uint8_t* tile_row = tile + lane * 64;
-                if (MODE == TC_FWD) {
-                    // the store that last used this tile must have read it
-                    if (lane == 0) {
-                        if (two_tiles && n_my == 2) tma_store_wait_read_n<1>(); else tma_store_wait_read_n<0>();
-                    }
-                    __syncwarp();
-                } else {
-                    if (!mbar_wait(&my_aux[i], (aux_phase >> i) & 1u, abort_flag, P.error, 5)) { ok = false; break; }
-                    aux_phase ^= 1u << i;
-                    aux_pending &= ~(1u << i);
-                }
-                uint32_t acc[32];
-                tmem_ld32(tmem_base + ((uint32_t)(32 * q) << 16) + (uint32_t)(buf * kMaxBN + 32 * c), acc);
-                if (i == n_my - 1) {
-                    // the accumulator has been read: hand the tensor-memory buffer back
-                    tc_fence_before();
-                    __syncwarp();
-                    if (lane == 0) mbar_arrive(&tempty[buf]);
-                }
-                if (MODE == TC_FWD) {
-                    const float4* b4 = reinterpret_cast<const float4*>(p.bias + col);   // zero-padded to the padded width
-#pragma unroll
-                    for (int g = 0; g < 4; ++g) {
-                        const float4 ba = __ldg(b4 + 2 * g), bb = __ldg(b4 + 2 * g + 1);
-                        const float bv[8] = {ba.x, ba.y, ba.z, ba.w, bb.x, bb.y, bb.z, bb.w};
-                        uint32_t o[4];
-#pragma unroll
-                        for (int e = 0; e < 4; ++e) {
-                            const float v0 = elu_fast(__uint_as_float(acc[8 * g + 2 * e]) + bv[2 * e], P.alpha);
-                            const float v1 = elu_fast(__uint_as_float(acc[8 * g + 2 * e + 1]) + bv[2 * e + 1], P.alpha);
-                            __nv_bfloat162 h2 = __floats2bfloat162_rn(v0, v1);
-                            o[e] = *reinterpret_cast<uint32_t*>(&h2);
-                        }
-                        *reinterpret_cast<uint4*>(tile_row + ((g ^ sw) << 4)) = make_uint4(o[0], o[1], o[2], o[3]);
-                    }
-                } else {
-#pragma unroll
-                    for (int g = 0; g < 4; ++g) {
-                        uint4* piece = reinterpret_cast<uint4*>(tile_row + ((g ^ sw) << 4));
-                        const uint4 hv = *piece;
-                        const uint32_t hw[4] = {hv.x, hv.y, hv.z, hv.w};
-                        uint32_t o[4];
-#pragma unroll
-                        for (int e = 0; e < 4; ++e) {
-                            const __nv_bfloat162 h2 = *reinterpret_cast<const __nv_bfloat162*>(&hw[e]);
-                            const float h0 = __low2float(h2), h1 = __high2float(h2);
-                            const float v0 = __uint_as_float(acc[8 * g + 2 * e]) * (h0 > 0.f ? 1.0f : h0 + P.alpha);
-                            const float v1 = __uint_as_float(acc[8 * g + 2 * e + 1]) * (h1 > 0.f ? 1.0f : h1 + P.alpha);
-                            __nv_bfloat162 r2 = __floats2bfloat162_rn(v0, v1);
-                            o[e] = *reinterpret_cast<uint32_t*>(&r2);
-                        }
-                        *piece = make_uint4(o[0], o[1], o[2], o[3]);
-                    }
-                }
-                fence_async_smem();                           // tile writes -> visible to the copy engine
-                __syncwarp();
-                // rows at or beyond the tensor's extent are clipped by the store itself
-                if (lane == 0 && row0 < p.m_extent) tma_store_2d(&P.tmOut[G.prob], tile, col, row0);
-                if (MODE == TC_DGRAD && p.colsum) {
-                    // partial bias gradient: lane l adds column l of the tile's 32 rows (rows past the
-                    // extent hold zeros); two lanes share a word, the 16 words of a row sit in 16 banks
-                    float s = 0.f;
-                    const uint8_t* mine = tile + ((lane & 7) << 1);
-#pragma unroll
-                    for (int r = 0; r < 32; ++r) {
-                        const __nv_bfloat16 v = *reinterpret_cast<const __nv_bfloat16*>(mine + r * 64 + (((lane >> 3) ^ ((r >> 1) & 3)) << 4));
-                        s += __bfloat162float(v);
-                    }
-                    p.colsum[(size_t)(m0 / BLOCK_M * 4 + q) * p.ld_colsum + col + lane] = s;
-                }
-            }
-            if (ok && n_my == 0) {
-                // nothing to read from this accumulator (columns beyond the extent)
-                tc_fence_before();
-                __syncwarp();
-                if (lane == 0) mbar_arrive(&tempty[buf]);
-            }
-        }
-        if (lane == 0) {
-            for (int i = 0; i < 2; ++i)
-                if (aux_pending & (1u << i)) {      // gave up with a load in flight: let it land first
-                    const unsigned long long t0 = global_ns();
-                    while (!mbar_try_wait(&my_aux[i], (aux_phase >> i) & 1u) && global_ns() - t0 < kWaitLimitNs) {}
-                }
             tma_store_wait_all();   // stores done before the CTA retires
         }
     }
@@ -928,6 +643,7 @@ struct UmmaEngine {
     std::vector<void*> allocs;
     __nv_bfloat16 *obs16_act[2] = {}, *h_act[2][kMaxLayers] = {};
     __nv_bfloat16 *x16[2] = {}, *h[2][kMaxLayers] = {}, *dz[2][kMaxLayers] = {};
+    __nv_bfloat16* x16_alt[2] = {};               // second minibatch input buffer (the gather of the next step fills it)
     __nv_bfloat16 *dmu16 = nullptr, *dv16 = nullptr;
     __nv_bfloat16 *wt[2][kMaxLayers] = {}, *wn[2][kMaxLayers] = {};
     float* bias_pad[2][kMaxLayers] = {};         // [pw] zero-padded copies of the hidden biases
@@ -938,11 +654,17 @@ struct UmmaEngine {
     int* error_dev = nullptr;
     int num_sms = 148;
     std::vector<TcParams> act_fwd, act_fwd_critic, upd_fwd, upd_dgrad, upd_wgrad;
-    // weight-stationary forms of upd_fwd / upd_dgrad, entry by entry (grid == 0: not applicable, use the streamed form)
-    std::vector<WsParams> upd_fwd_ws, upd_dgrad_ws;
+    // the launches that read the minibatch observations, once more for the second input buffer
+    std::vector<TcParams> upd_fwd_alt, upd_wgrad_alt;
     // fused forward (one launch for all hidden layers) where the widths allow it, else empty
-    std::vector<ChainParams> chain_act, chain_act_critic, chain_upd;
+    std::vector<ChainParams> chain_act, chain_act_critic;
     ColsumBatch colsum{}, colsum_rest{};         // all layers the epilogue does not cover / those minus the last ones
+    // fused row-local step kernel (no mirrored rows): head operand copies, bias-gradient partials of every hidden layer
+    StepChain* step = nullptr;
+    __nv_bfloat16 *wht[2] = {}, *whn[2] = {};
+    float* head_bias_pad[2] = {};
+    float* step_slots[2][kMaxLayers] = {};
+    int step_slot_rows = 0;
 };
 
 namespace {
@@ -979,7 +701,6 @@ bool add_rowmajor_problem(TcParams& P, const __nv_bfloat16* A, int rows, int k, 
     p.m_tiles = (rows + BLOCK_M - 1) / BLOCK_M;
     p.n_tiles = (width_out + p.bn - 1) / p.bn;
     p.kblocks = k / BLOCK_K; p.splits = 1; p.kb_per_split = p.kblocks;
-    p.a_ptr = A; p.b_ptr = B; p.k_elems = k;
     if (!make_tmap(&P.tmA[i], A, rows, k, k, BLOCK_K, BLOCK_M)) return false;
     if (!make_tmap(&P.tmB[i], B, width_out, k, k, BLOCK_K, p.bn)) return false;
     P.count++;
@@ -995,73 +716,6 @@ cudaError_t launch_tc(const TcParams& P, int num_sms, cudaStream_t s) {
 }
 
 
-// Column tile of a weight-stationary problem: the widest of 256, 192, 128, 64 columns (not beyond
-// the output width) whose slice of the weights, all k-blocks, fits `limit` bytes; 0 if none does.
-int ws_pick_bn(int width_out, int k, uint32_t limit) {
-    for (int bn : {256, 192, 128, 64})
-        if (bn <= std::max(64, std::min(kMaxBN, width_out)) && (size_t)bn * k * 2 <= limit) return bn;
-    return 0;
-}
-
-// The weight-stationary form of a forward / data-gradient launch: same problems, column tiles
-// chosen so that a slice fits shared memory, the SMs shared out among the (problem, column tile)
-// groups in proportion to their work.  W.grid stays 0 when the form does not apply.
-bool make_ws(WsParams& W, const TcParams& T, int mode, int num_sms) {
-    memset(&W, 0, sizeof W);
-    // the data-gradient epilogue prefetches the stored activations of all its chunks: two tiles per warp
-    const uint32_t limit = mode == TC_DGRAD ? kWsMaxSlice / 2 : kWsMaxSlice;
-    uint32_t slice = 0;
-    int ng = 0;
-    struct Cost { long long per_tile; int tiles; };
-    Cost cost[kWsGroups];
-    for (int i = 0; i < T.count; ++i) {
-        const TcProblem& t = T.p[i];
-        const int bn = ws_pick_bn(t.n_extent, t.k_elems, limit);
-        if (bn == 0) return true;
-        TcProblem& p = W.p[i];
-        p = t;
-        p.bn = bn;
-        p.n_tiles = (t.n_extent + bn - 1) / bn;
-        W.tmA[i] = T.tmA[i];
-        if (!make_tmap(&W.tmB[i], t.b_ptr, t.n_extent, t.k_elems, t.k_elems, BLOCK_K, bn)) return false;
-        if (!make_tmap(&W.tmOut[i], t.out16, t.m_extent, t.n_extent, t.ld_out, 32, 32, CU_TENSOR_MAP_SWIZZLE_64B)) return false;
-        if (mode == TC_DGRAD &&
-            !make_tmap(&W.tmAux[i], t.aux16, t.m_extent, t.n_extent, t.ld_aux, 32, 32, CU_TENSOR_MAP_SWIZZLE_64B))
-            return false;
-        slice = std::max(slice, (uint32_t)bn * (uint32_t)t.k_elems * 2u);
-        for (int j = 0; j < p.n_tiles; ++j) {
-            if (ng == kWsGroups) return true;
-            W.g[ng] = WsGroup{i, j * bn, 0, 1};
-            cost[ng] = Cost{(long long)p.kblocks * bn, p.m_tiles};
-            ++ng;
-        }
-    }
-    if (ng == 0 || ng > num_sms) return true;
-    // one CTA per group, then the group whose CTAs have the longest queue gets the next one
-    int left = num_sms - ng;
-    auto queue = [&](int g) { return cost[g].per_tile * ((cost[g].tiles + W.g[g].cta_count - 1) / W.g[g].cta_count); };
-    while (left > 0) {
-        int best = -1;
-        for (int g = 0; g < ng; ++g)
-            if (W.g[g].cta_count < cost[g].tiles && (best < 0 || queue(g) > queue(best))) best = g;
-        if (best < 0) break;
-        W.g[best].cta_count++;
-        --left;
-    }
-    int begin = 0;
-    for (int g = 0; g < ng; ++g) { W.g[g].cta_begin = begin; begin += W.g[g].cta_count; }
-    W.count = T.count; W.ngroups = ng; W.grid = begin;
-    W.slice_bytes = (slice + 1023u) & ~1023u;
-    W.tiles_per_warp = (mode == TC_DGRAD || W.slice_bytes <= kWsMaxSlice / 2) ? 2 : 1;
-    W.alpha = T.alpha; W.error = T.error;
-    return true;
-}
-
-template <int MODE>
-cudaError_t launch_ws(const WsParams& W, cudaStream_t s) {
-    LaunchScope scope_(MODE == TC_FWD ? "tc_gemm_fwd" : "tc_gemm_dgrad", s);
-    return launch_chained(ws_gemm_kernel<MODE>, W.grid, kThreads, ws_smem_bytes(W.slice_bytes, W.tiles_per_warp), s, W);
-}
 
 // The program of one net for the fused forward; false when the widths do not fit the kernel
 // (first hidden layer <= 512 and a multiple of 128 beyond 256, the others <= 256).
@@ -1197,9 +851,6 @@ UmmaEngine* umma_create(const UmmaSetup& s, std::string* err) {
         return failmsg("could not reserve shared memory for the tensor-core kernels");
     if (cudaFuncSetAttribute(chain_fwd_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kChainSmem) != cudaSuccess)
         return failmsg("could not reserve shared memory for the fused forward kernel");
-    if (cudaFuncSetAttribute(ws_gemm_kernel<TC_FWD>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)ws_smem_bytes(kWsMaxSlice, 1)) != cudaSuccess ||
-        cudaFuncSetAttribute(ws_gemm_kernel<TC_DGRAD>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)ws_smem_bytes(kWsMaxSlice / 2, 2)) != cudaSuccess)
-        return failmsg("could not reserve shared memory for the weight-stationary kernels");
     UmmaEngine* e = new UmmaEngine();
     e->s = s;
     e->num_sms = prop.multiProcessorCount;
@@ -1213,10 +864,11 @@ UmmaEngine* umma_create(const UmmaSetup& s, std::string* err) {
     }
     const bool shared = s.model.shared_obs != 0;
     for (int ni = 0; ni < 2; ++ni) {
-        if (ni == 1 && shared) { e->obs16_act[1] = e->obs16_act[0]; e->x16[1] = e->x16[0]; }
+        if (ni == 1 && shared) { e->obs16_act[1] = e->obs16_act[0]; e->x16[1] = e->x16[0]; e->x16_alt[1] = e->x16_alt[0]; }
         else {
             if (!ealloc(e, &e->obs16_act[ni], (size_t)N * e->kp[ni])) return bail("allocation failed");
-            if (!ealloc(e, &e->x16[ni], (size_t)R * e->kp[ni])) return bail("allocation failed");
+            if (!ealloc(e, &e->x16[ni], (size_t)R * e->kp[ni]) || !ealloc(e, &e->x16_alt[ni], (size_t)R * e->kp[ni]))
+                return bail("allocation failed");
         }
         for (int l = 0; l < e->nh[ni]; ++l) {
             const int kin = l == 0 ? e->kp[ni] : e->pw[ni][l - 1];
@@ -1228,6 +880,13 @@ UmmaEngine* umma_create(const UmmaSetup& s, std::string* err) {
         }
     }
     if (!ealloc(e, &e->dmu16, (size_t)R * 64) || !ealloc(e, &e->dv16, (size_t)R * 64)) return bail("allocation failed");
+    // head weights as tensor-core operands (output-major and input-major, padded to 64 outputs)
+    for (int ni = 0; ni < 2; ++ni) {
+        const int pl = e->pw[ni][e->nh[ni] - 1];
+        if (!ealloc(e, &e->wht[ni], (size_t)64 * pl) || !ealloc(e, &e->whn[ni], (size_t)pl * 64) ||
+            !ealloc(e, &e->head_bias_pad[ni], (size_t)64))
+            return bail("allocation failed");
+    }
 
     // weight conversion table
     std::vector<CvtEntry> table;
@@ -1241,6 +900,17 @@ UmmaEngine* umma_create(const UmmaSetup& s, std::string* err) {
             table.push_back(c);
             e->cvt_max = std::max(e->cvt_max, c.in * c.out);
         }
+    for (int ni = 0; ni < 2; ++ni) {
+        const int l = e->nh[ni];                       // the head
+        if (s.out[ni][l] > 64) continue;
+        CvtEntry c{};
+        c.bsrc = s.param + s.b_off[ni][l]; c.bdst = e->head_bias_pad[ni];
+        c.src = s.param + s.w_off[ni][l]; c.in = s.in[ni][l]; c.out = s.out[ni][l]; c.ld_src = s.out_p[ni][l];
+        c.wt = e->wht[ni]; c.ld_wt = e->pw[ni][l - 1];
+        c.wn = e->whn[ni]; c.ld_wn = 64;
+        table.push_back(c);
+        e->cvt_max = std::max(e->cvt_max, c.in * c.out);
+    }
     e->n_cvt = (int)table.size();
     if (!ealloc(e, &e->cvt_dev, table.size())) return bail("allocation failed");
     if (cudaMemcpyAsync(e->cvt_dev, table.data(), table.size() * sizeof(CvtEntry), cudaMemcpyHostToDevice, s.stream) != cudaSuccess ||
@@ -1261,6 +931,7 @@ UmmaEngine* umma_create(const UmmaSetup& s, std::string* err) {
                 if (!add_rowmajor_problem(P, in, rows, k, e->wt[ni][l], e->pw[ni][l])) return false;
                 TcProblem& p = P.p[P.count - 1];
                 p.bias = e->bias_pad[ni][l]; p.bias_n = e->pw[ni][l];
+                p.net_id = ni; p.layer_id = l;
                 p.out16 = act_buffers ? e->h_act[ni][l] : e->h[ni][l]; p.ld_out = e->pw[ni][l];
                 if (!make_tmap(&P.tmOut[P.count - 1], p.out16, rows, e->pw[ni][l], e->pw[ni][l], 64, 32)) return false;
             }
@@ -1338,17 +1009,6 @@ UmmaEngine* umma_create(const UmmaSetup& s, std::string* err) {
         finish_params(P, alpha, e->error_dev);
         e->upd_dgrad.push_back(P);
     }
-    // ---- weight-stationary forms of the minibatch forward and data-gradient launches ------------
-    for (const TcParams& T : e->upd_fwd) {
-        WsParams W;
-        if (!make_ws(W, T, TC_FWD, e->num_sms)) return bail("tensor map encoding failed");
-        e->upd_fwd_ws.push_back(W);
-    }
-    for (const TcParams& T : e->upd_dgrad) {
-        WsParams W;
-        if (!make_ws(W, T, TC_DGRAD, e->num_sms)) return bail("tensor map encoding failed");
-        e->upd_dgrad_ws.push_back(W);
-    }
     // ---- weight-gradient problems (all layers of both nets, heads included) ------------------
     {
         const int kblocks = (R + BLOCK_K - 1) / BLOCK_K;
@@ -1372,12 +1032,29 @@ UmmaEngine* umma_create(const UmmaSetup& s, std::string* err) {
                 p.kb_per_split = (kblocks + want - 1) / want;
                 p.kblocks = kblocks; p.splits = (kblocks + p.kb_per_split - 1) / p.kb_per_split;
                 p.out32 = s.partials + s.w_off[ni][l]; p.ld_out32 = s.out_p[ni][l]; p.split_stride = s.P_dev;
+                p.net_id = ni; p.layer_id = l;
                 if (!make_tmap(&P.tmA[i], A, R, wa, wa, 64, BLOCK_K) || !make_tmap(&P.tmB[i], B, R, wb, wb, 64, BLOCK_K))
                     return bail("tensor map encoding failed");
                 P.count++;
             }
         flush();
     }
+    // ---- the same launches reading the second minibatch input buffer ----------------------------
+    e->upd_fwd_alt = e->upd_fwd; e->upd_wgrad_alt = e->upd_wgrad;
+    for (size_t li = 0; li < e->upd_fwd_alt.size(); ++li) {
+        TcParams& P = e->upd_fwd_alt[li];
+        for (int i = 0; i < P.count; ++i) {
+            if (P.p[i].layer_id != 0) continue;
+            const int ni = P.p[i].net_id;
+            if (!make_tmap(&P.tmA[i], e->x16_alt[ni], R, e->kp[ni], e->kp[ni], BLOCK_K, BLOCK_M)) return bail("tensor map encoding failed");
+        }
+    }
+    for (TcParams& P : e->upd_wgrad_alt)
+        for (int i = 0; i < P.count; ++i) {
+            if (P.p[i].layer_id != 0) continue;
+            const int ni = P.p[i].net_id;
+            if (!make_tmap(&P.tmA[i], e->x16_alt[ni], R, e->kp[ni], e->kp[ni], 64, BLOCK_K)) return bail("tensor map encoding failed");
+        }
     // ---- bias-gradient partials of the last hidden layers, written by the head/loss kernel ----
     if (e->n_sources + 2 <= kMaxBiasSources)
         for (int ni = 0; ni < 2; ++ni)
@@ -1394,12 +1071,41 @@ UmmaEngine* umma_create(const UmmaSetup& s, std::string* err) {
             if (l < e->nh[ni] - 1) e->colsum_rest.p[e->colsum_rest.count++] = q;
         }
     e->colsum_rest.splits = e->colsum.splits; e->colsum_rest.split_stride = e->colsum.split_stride; e->colsum_rest.is_bf16 = 1;
+    // ---- fused row-local step kernel -------------------------------------------------------------
+    // (off unless RSLRL_FUSED_STEP=1: on the workloads measured so far its items, which run their layers
+    // one after the other, take longer than the per-layer launches whose tiles overlap)
+    const char* fused_env = std::getenv("RSLRL_FUSED_STEP");
+    if (fused_env && fused_env[0] == '1' && R == s.Bmb && e->nh[0] <= kStepChainLayers && e->nh[1] <= kStepChainLayers && s.out[0][e->nh[0]] <= 64 &&
+        e->n_cvt + 0 <= kMaxCvt) {
+        StepChainSetup cs{};
+        cs.rows = R; cs.alpha = alpha; cs.error = e->error_dev; cs.num_sms = e->num_sms;
+        cs.log_std = s.param + s.logstd_off;
+        e->step_slot_rows = step_chain_colsum_rows(R);
+        bool okc = true;
+        for (int ni = 0; ni < 2 && okc; ++ni) {
+            StepChainNet& n = cs.net[ni];
+            n.nh = e->nh[ni]; n.kp = e->kp[ni]; n.is_actor = ni == 0; n.A = s.out[ni][e->nh[ni]];
+            n.x16 = e->x16[ni]; n.wht = e->wht[ni]; n.whn = e->whn[ni]; n.head_bias = e->head_bias_pad[ni];
+            n.dhead16 = ni == 0 ? e->dmu16 : e->dv16;
+            for (int l = 0; l < e->nh[ni]; ++l) {
+                n.pw[l] = e->pw[ni][l]; n.wt[l] = e->wt[ni][l]; n.wn[l] = e->wn[ni][l];
+                n.bias_pad[l] = e->bias_pad[ni][l]; n.h[l] = e->h[ni][l]; n.dz[l] = e->dz[ni][l];
+                okc = okc && ealloc(e, &e->step_slots[ni][l], (size_t)e->step_slot_rows * e->pw[ni][l]);
+                n.colsum[l] = e->step_slots[ni][l];
+            }
+        }
+        if (!okc) return bail("allocation failed");
+        std::string serr;
+        e->step = step_chain_create(cs, &serr);
+        if (!e->step && !serr.empty()) return bail("fused step kernel: tensor map encoding failed");
+    }
     if (cudaStreamSynchronize(s.stream) != cudaSuccess) return bail("stream synchronisation failed");
     return e;
 }
 
 void umma_destroy(UmmaEngine* e) {
     if (!e) return;
+    if (e->step) step_chain_destroy(e->step);
     for (void* p : e->allocs) cudaFree(p);
     delete e;
 }
@@ -1416,6 +1122,16 @@ void umma_fill_cvt(UmmaEngine* e, AdamArgs* a) {
             c.wn = l > 0 ? e->wn[ni][l] : nullptr; c.ld_wn = e->pw[ni][l];
             c.bias_pad = e->bias_pad[ni][l];
         }
+    for (int ni = 0; ni < 2 && e->step; ++ni) {
+        if (a->n_cvt == kMaxCvt) break;
+        const int l = e->nh[ni];
+        CvtRange& c = a->cvt[a->n_cvt++];
+        c.w_off = (int)s.w_off[ni][l]; c.b_off = (int)s.b_off[ni][l];
+        c.in = s.in[ni][l]; c.out = s.out[ni][l]; c.out_p = s.out_p[ni][l];
+        c.wt = e->wht[ni]; c.ld_wt = e->pw[ni][l - 1];
+        c.wn = e->whn[ni]; c.ld_wn = 64;
+        c.bias_pad = e->head_bias_pad[ni];
+    }
 }
 
 void umma_fill_bias_sources(UmmaEngine* e, ReduceArgs* r, const HeadLossArgs& hl) {
@@ -1476,17 +1192,17 @@ cudaError_t umma_act_forward(UmmaEngine* e, const float* d_obs_a, const float* d
     return cudaSuccess;
 }
 
-void umma_gather_targets(UmmaEngine* e, GatherArgs* g) {
+void umma_gather_targets(UmmaEngine* e, GatherArgs* g, int buf) {
     g->x_a = nullptr; g->x_c = nullptr;
-    g->x_a16 = e->x16[0]; g->ldxa16 = e->kp[0];
-    g->x_c16 = e->x16[1]; g->ldxc16 = e->kp[1];
+    g->x_a16 = buf ? e->x16_alt[0] : e->x16[0]; g->ldxa16 = e->kp[0];
+    g->x_c16 = buf ? e->x16_alt[1] : e->x16[1]; g->ldxc16 = e->kp[1];
 }
 
-cudaError_t umma_update_forward(UmmaEngine* e) {
-    if (!e->chain_upd.empty()) return launch_chain(e->chain_upd[0], e->num_sms, e->s.stream);
-    for (size_t i = 0; i < e->upd_fwd.size(); ++i) {
-        cudaError_t err = e->upd_fwd_ws[i].grid > 0 ? launch_ws<TC_FWD>(e->upd_fwd_ws[i], e->s.stream)
-                                                    : launch_tc<TC_FWD>(e->upd_fwd[i], e->num_sms, e->s.stream);
+bool umma_two_input_buffers(const UmmaEngine* e) { return e->step == nullptr; }
+
+cudaError_t umma_update_forward(UmmaEngine* e, int buf) {
+    for (const TcParams& P : buf ? e->upd_fwd_alt : e->upd_fwd) {
+        cudaError_t err = launch_tc<TC_FWD>(P, e->num_sms, e->s.stream);
         if (err != cudaSuccess) return err;
     }
     return cudaSuccess;
@@ -1502,18 +1218,43 @@ void umma_head_loss_targets(UmmaEngine* e, HeadLossArgs* a) {
     a->colsum_a = e->head_slots[0]; a->colsum_c = e->head_slots[1];
 }
 
-cudaError_t umma_update_backward(UmmaEngine* e, bool last_bias_done) {
+cudaError_t umma_update_backward(UmmaEngine* e, bool last_bias_done, int buf) {
     cudaError_t err;
-    for (size_t i = 0; i < e->upd_dgrad.size(); ++i) {
-        err = e->upd_dgrad_ws[i].grid > 0 ? launch_ws<TC_DGRAD>(e->upd_dgrad_ws[i], e->s.stream)
-                                          : launch_tc<TC_DGRAD>(e->upd_dgrad[i], e->num_sms, e->s.stream);
+    for (const TcParams& P : e->upd_dgrad) {
+        err = launch_tc<TC_DGRAD>(P, e->num_sms, e->s.stream);
         if (err != cudaSuccess) return err;
     }
-    for (const TcParams& P : e->upd_wgrad) {
+    for (const TcParams& P : buf ? e->upd_wgrad_alt : e->upd_wgrad) {
         err = launch_tc<TC_WGRAD>(P, e->num_sms, e->s.stream);
         if (err != cudaSuccess) return err;
     }
     return launch_colsum(last_bias_done ? e->colsum_rest : e->colsum, e->s.stream);
+}
+
+bool umma_has_step_chain(const UmmaEngine* e) { return e->step != nullptr; }
+
+cudaError_t umma_step_chain(UmmaEngine* e, const StepChainLoss& loss, int* nblocks) {
+    *nblocks = step_chain_blocks(e->step);
+    return step_chain_launch(e->step, loss, e->s.stream);
+}
+
+cudaError_t umma_update_wgrad(UmmaEngine* e) {
+    for (const TcParams& P : e->upd_wgrad) {
+        cudaError_t err = launch_tc<TC_WGRAD>(P, e->num_sms, e->s.stream);
+        if (err != cudaSuccess) return err;
+    }
+    return cudaSuccess;
+}
+
+void umma_fill_step_bias_sources(UmmaEngine* e, ReduceArgs* r) {
+    const UmmaSetup& s = e->s;
+    r->n_bias = 0;
+    for (int ni = 0; ni < 2; ++ni)
+        for (int l = 0; l < e->nh[ni]; ++l) {
+            BiasSource& b = r->bias[r->n_bias++];
+            b.p_off = (int)s.b_off[ni][l]; b.n = s.out[ni][l];
+            b.slots = e->step_slots[ni][l]; b.nslots = e->step_slot_rows; b.ld = e->pw[ni][l];
+        }
 }
 
 cudaError_t umma_read_error(UmmaEngine* e, int* host_code) {

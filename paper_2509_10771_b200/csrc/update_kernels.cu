@@ -124,10 +124,16 @@ __global__ void __launch_bounds__(256, 3) gather_kernel(const GatherArgs a) {
     }
 }
 
-__global__ void perm_rows_kernel(PermKey pk, uint32_t first, int count, int* __restrict__ rows_out) {
+// rows_out[e * count + j] = shuffle of epoch (pk.epoch + e) at position first + j, e < epochs
+__global__ void perm_rows_kernel(PermKey pk, uint32_t first, int count, int epochs, int* __restrict__ rows_out) {
     chain_begin();
     const int j = blockIdx.x * blockDim.x + threadIdx.x;
-    if (j < count) rows_out[j] = (int)feistel_permute(pk, first + (uint32_t)j);
+    if (j >= count) return;
+    for (int e = blockIdx.y; e < epochs; e += gridDim.y) {
+        PermKey k = pk;
+        k.epoch = pk.epoch + (uint32_t)e;
+        rows_out[(size_t)e * count + j] = (int)feistel_permute(k, first + (uint32_t)j);
+    }
 }
 
 // =======================================================================================
@@ -692,7 +698,14 @@ cudaError_t launch_perm_rows(uint64_t seed, uint32_t iteration, uint32_t epoch, 
     if (count <= 0) return cudaSuccess;
     PermKey pk{(uint32_t)seed, (uint32_t)(seed >> 32), iteration, epoch, batch, feistel_half_bits(batch)};
     LaunchScope scope_("perm_rows", s);
-    return launch_chained(perm_rows_kernel, (count + 255) / 256, 256, 0, s, pk, first, count, rows_out);
+    return launch_chained(perm_rows_kernel, (count + 255) / 256, 256, 0, s, pk, first, count, 1, rows_out);
+}
+
+cudaError_t launch_perm_epochs(uint64_t seed, uint32_t iteration, int epochs, uint32_t batch, int* rows_out, cudaStream_t s) {
+    if (batch == 0 || epochs <= 0) return cudaSuccess;
+    PermKey pk{(uint32_t)seed, (uint32_t)(seed >> 32), iteration, 0u, batch, feistel_half_bits(batch)};
+    LaunchScope scope_("perm_rows", s);
+    return launch_chained(perm_rows_kernel, dim3((batch + 255) / 256, std::min(epochs, 65535)), 256, 0, s, pk, 0u, (int)batch, epochs, rows_out);
 }
 
 int head_loss_blocks(int Bmb) { return std::max(1, (Bmb + kHLRows - 1) / kHLRows); }
