@@ -566,9 +566,11 @@ rslrl_status rslrl_act(rslrl_ctx* c, const float* d_actor_obs, const float* d_cr
                               c->pc.seed, c->global_step, c->stream));
     } else {
         const void *ha, *hc; int ldha, ldhc;
+        bool heads_done = false;
         CU(c, umma_act_forward(c->umma, d_actor_obs, c->mc.shared_obs ? nullptr : d_critic_obs, oa,
-                               c->mc.shared_obs ? nullptr : oc, sa, sc, true, &ha, &ldha, &hc, &ldhc));
-        CU(c, launch_act_head(ha, ldha, hc, ldhc, true, hp, out, N, c->pc.seed, c->global_step, c->stream));
+                               c->mc.shared_obs ? nullptr : oc, sa, sc, true, out, hp.log_std, c->pc.seed, c->global_step,
+                               &heads_done, &ha, &ldha, &hc, &ldhc));
+        if (!heads_done) CU(c, launch_act_head(ha, ldha, hc, ldhc, true, hp, out, N, c->pc.seed, c->global_step, c->stream));
     }
     c->global_step++;
     c->act_pending = true;
@@ -599,8 +601,12 @@ rslrl_status rslrl_gae(rslrl_ctx* c, const float* d_last_critic_obs) {
         CU(c, launch_value_head(c->act_h[1][c->critic.nl - 2], c->critic.hid_ld[c->critic.nl - 2], false, hp, c->last_values, N, c->stream));
     } else {
         const void *ha, *hc; int ldha, ldhc;
-        CU(c, umma_act_forward(c->umma, nullptr, d_last_critic_obs, nullptr, nullptr, 0, 0, false, &ha, &ldha, &hc, &ldhc));
-        CU(c, launch_value_head(hc, ldhc, true, hp, c->last_values, N, c->stream));
+        bool heads_done = false;
+        ActOut vout{};
+        vout.values = c->last_values; vout.act_stride = c->st.act_stride;
+        CU(c, umma_act_forward(c->umma, nullptr, d_last_critic_obs, nullptr, nullptr, 0, 0, false, vout, hp.log_std, c->pc.seed,
+                               c->global_step, &heads_done, &ha, &ldha, &hc, &ldhc));
+        if (!heads_done) CU(c, launch_value_head(hc, ldhc, true, hp, c->last_values, N, c->stream));
     }
     CU(c, launch_gae(c->st.rewards, c->st.values, c->st.dones, c->st.timeouts, c->last_values, c->st.returns,
                      c->st.advantages, T, N, c->pc.gamma, c->pc.lam, c->pc.normalize_adv, c->pc.adv_std_unbiased,

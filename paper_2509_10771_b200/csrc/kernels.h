@@ -195,6 +195,7 @@ struct CvtRange {
     int w_off, b_off, in, out, out_p;          // location in the padded FP32 parameter vector
     __nv_bfloat16* wt; int ld_wt;               // [out][ld_wt]
     __nv_bfloat16* wn; int ld_wn;               // [in][ld_wn], may be null
+    __nv_bfloat16* wt_lo;                       // [out][ld_wt] what BF16 rounding left of the weight, may be null
     float* bias_pad;                            // [>= out] zero-padded FP32 bias copy
 };
 constexpr int kMaxCvt = 16;

@@ -370,7 +370,8 @@ constexpr int kSlots = 9;
 constexpr uint32_t kSlotBytes = 16384;
 constexpr uint32_t kActBytes = BLOCK_M * kMaxBN * 2;     // 64 KiB = four [128 rows][64] blocks
 constexpr int kChainBiasFloats = 2 * (512 + (kChainLayers - 1) * 256);
-constexpr size_t kChainSmem = 1024 + (size_t)kSlots * kSlotBytes + kActBytes + kChainBiasFloats * 4 + 512;
+constexpr int kChainHeadFloats = 256;
+constexpr size_t kChainSmem = 1024 + (size_t)kSlots * kSlotBytes + kActBytes + kChainBiasFloats * 4 + kChainHeadFloats * 4 + 512;
 __host__ __device__ constexpr int slots_of(int a_ring, int bn) { return a_ring + (bn * BLOCK_K * 2 + (int)kSlotBytes - 1) / (int)kSlotBytes; }
 constexpr int kPrevItem = 16;                    // added to an epilogue index: that epilogue of the CTA's previous item
 
@@ -385,6 +386,7 @@ struct ChainJob {
                          // it wrote the activations this job reads, or drained the accumulator this job overwrites
 };
 struct ChainEpi {
+    int head;            // 1: the head epilogue (rollout outputs) instead of bias + ELU
     int layer, n0, ncols, tmem_col;   // columns [n0, n0 + ncols) of `layer` from these accumulator columns
     int wait_job;        // the job that completes the accumulator
     int write_job;       // a later job that still reads the activation buffer (-1: none): done before the buffer is rewritten
@@ -397,10 +399,21 @@ struct ChainNet {
     const float* bias[kChainLayers];  // zero-padded to the padded width
     int bias_n[kChainLayers];         // that width
     int bias_off[kChainLayers];       // where the kernel keeps the layer's bias in shared memory (floats)
+    int is_actor, A, head_n;          // head epilogue: policy head with A outputs, or the value head; its accumulator holds
+                                      // h Wt_hi in columns [0, head_n) and h Wt_lo in [head_n, 2 head_n)
+    const float* head_bias;           // [64] zero-padded
+};
+// What the head epilogue of the rollout writes (storage row of the current step).
+struct ChainHeadOut {
+    float* actions; float* mu; float* sigma; float* logp; float* values; float* actions_out;   // actions_out may be null
+    int act_stride;
+    const float* log_std;
+    uint32_t seed_lo, seed_hi, global_step;
 };
 struct ChainParams {
     CUtensorMap tmX[2];                       // first-layer input, boxes of 64 x 128 rows
-    CUtensorMap tmW[2][kChainLayers];         // [out][in] weights, boxes of 64 x (columns per job)
+    CUtensorMap tmW[2][kChainLayers + 1];     // [out][in] weights, boxes of 64 x (columns per job); last: the head
+    ChainHeadOut ho;
     CUtensorMap tmOut[2][kChainLayers];       // activations, boxes of 64 columns x 32 rows
     ChainNet net[2];                          // same numbers of jobs and epilogues, same waits
     int nnets, rows, total_items;             // items = (row tile, net), nets interleaved
@@ -414,7 +427,8 @@ __global__ void __launch_bounds__(kThreads, 1) chain_fwd_kernel(const __grid_con
     uint8_t* sRing = smem;
     uint8_t* sAct = sRing + kSlots * kSlotBytes;
     float* sBias = reinterpret_cast<float*>(sAct + kActBytes);
-    uint64_t* full = reinterpret_cast<uint64_t*>(sBias + kChainBiasFloats);
+    float* sHead = sBias + kChainBiasFloats;   // policy head bias [64], log_std [64], sigma [64], value head bias
+    uint64_t* full = reinterpret_cast<uint64_t*>(sHead + kChainHeadFloats);
     uint64_t* empty = full + kSlots;
     uint64_t* job_done = empty + kSlots;       // one completion per item each
     uint64_t* epi_done = job_done + kChainJobs;
@@ -447,6 +461,23 @@ __global__ void __launch_bounds__(kThreads, 1) chain_fwd_kernel(const __grid_con
     for (int n = 0; n < P.nnets; ++n)
         for (int l = 0; l < P.net[n].nlayers; ++l)
             for (int i = threadIdx.x; i < P.net[n].bias_n[l]; i += kThreads) sBias[P.net[n].bias_off[l] + i] = P.net[n].bias[l][i];
+    for (int n = 0; n < P.nnets; ++n) {
+        const ChainNet& N = P.net[n];
+        if (N.A <= 0) continue;                  // no head epilogue
+        if (N.is_actor) {
+            for (int i = threadIdx.x; i < 64; i += kThreads) {
+                const float ls = i < N.A ? P.ho.log_std[i] : 0.f;
+                sHead[i] = N.head_bias[i];
+                sHead[64 + i] = ls;
+                sHead[128 + i] = expf(ls);
+            }
+            // sigma does not depend on the state: one vector per rollout step
+            if (blockIdx.x == 0)
+                for (int i = threadIdx.x; i < P.ho.act_stride; i += kThreads) P.ho.sigma[i] = i < N.A ? expf(P.ho.log_std[i]) : 0.f;
+        } else if (threadIdx.x == 0) {
+            sHead[192] = N.head_bias[0];
+        }
+    }
     __syncthreads();
 
     if (warp == 0) {
@@ -556,6 +587,60 @@ __global__ void __launch_bounds__(kThreads, 1) chain_fwd_kernel(const __grid_con
                 const ChainEpi& E = N.epi[e];
                 if (!mbar_wait(&job_done[E.wait_job], t & 1u, abort_flag, P.error, 14)) { ok = false; break; }
                 tc_fence_after();
+                if (E.head) {
+                    // rollout outputs of the tile's rows, one thread per row (the first column group's warps)
+                    // (the accumulator loads are warp-wide; only the stores depend on the row being there)
+                    const int n = m0 + 32 * q + lane;
+                    const bool live = n < P.rows;
+                    if (g == 0) {
+                        const uint32_t taddr = tmem_base + ((uint32_t)(32 * q) << 16) + ((uint32_t)E.tmem_col ^ flip);
+                        const ChainHeadOut& H = P.ho;
+                        if (N.is_actor) {
+                            float* arow = H.actions + (size_t)n * H.act_stride;
+                            float* mrow = H.mu + (size_t)n * H.act_stride;
+                            float* orow = H.actions_out ? H.actions_out + (size_t)n * H.act_stride : nullptr;
+                            float logp = 0.f;
+                            for (int c = 0; c < H.act_stride; c += 4) {
+                                // four actions share one Philox block
+                                float av[4] = {0.f, 0.f, 0.f, 0.f}, mv[4] = {0.f, 0.f, 0.f, 0.f};
+                                if (c < N.A) {
+                                    uint32_t a4[4], l4[4];
+                                    tmem_ld4(taddr + (uint32_t)c, a4);
+                                    tmem_ld4(taddr + (uint32_t)(N.head_n + c), l4);
+                                    float eps[4];
+                                    gaussian_quad(H.seed_lo, H.seed_hi, (uint32_t)n, H.global_step, (uint32_t)(c >> 2), eps);
+#pragma unroll
+                                    for (int k = 0; k < 4; ++k) {
+                                        const int i = c + k;
+                                        if (i < N.A) {
+                                            const float m = (__uint_as_float(a4[k]) + __uint_as_float(l4[k])) + sHead[i];
+                                            const float ls = sHead[64 + i], sg = sHead[128 + i];
+                                            const float a = fmaf(sg, eps[k], m);
+                                            const float d = a - m;
+                                            logp += -(d * d) / (2.0f * sg * sg) - ls - 0.91893853320467274178f;
+                                            av[k] = a; mv[k] = m;
+                                        }
+                                    }
+                                }
+                                if (live) {
+                                    *reinterpret_cast<float4*>(arow + c) = make_float4(av[0], av[1], av[2], av[3]);
+                                    *reinterpret_cast<float4*>(mrow + c) = make_float4(mv[0], mv[1], mv[2], mv[3]);
+                                    if (orow) { orow[c] = av[0]; orow[c + 1] = av[1]; orow[c + 2] = av[2]; orow[c + 3] = av[3]; }   // caller's buffer: 4-byte aligned only
+                                }
+                            }
+                            if (live) H.logp[n] = logp;
+                        } else {
+                            uint32_t a4[4], l4[4];
+                            tmem_ld4(taddr, a4);
+                            tmem_ld4(taddr + (uint32_t)N.head_n, l4);
+                            if (live) H.values[n] = (__uint_as_float(a4[0]) + __uint_as_float(l4[0])) + sHead[192];
+                        }
+                    }
+                    tc_fence_before();
+                    __syncwarp();
+                    if (lane == 0) mbar_arrive(&epi_done[e]);
+                    continue;
+                }
                 const bool active = 64 * g < E.ncols;          // uniform across the warp
                 uint4 outv[8];
                 if (active) {
@@ -615,6 +700,7 @@ struct CvtEntry {
     const float* src; int in, out, ld_src;      // FP32 master W[in][ld_src]
     __nv_bfloat16* wt; int ld_wt;               // [out][ld_wt]  (contraction = in)   forward operand
     __nv_bfloat16* wn; int ld_wn;               // [in][ld_wn]   (contraction = out)  data-gradient operand, may be null
+    __nv_bfloat16* wt_lo;                       // [out][ld_wt]  what BF16 rounding left of the weight (heads only, else null)
 };
 
 __global__ void convert_weights_kernel(const CvtEntry* __restrict__ table) {
@@ -626,6 +712,7 @@ __global__ void convert_weights_kernel(const CvtEntry* __restrict__ table) {
         const __nv_bfloat16 v = __float2bfloat16_rn(e.src[(size_t)i * e.ld_src + o]);
         e.wt[(size_t)o * e.ld_wt + i] = v;
         if (e.wn) e.wn[(size_t)i * e.ld_wn + o] = v;
+        if (e.wt_lo) e.wt_lo[(size_t)o * e.ld_wt + i] = __float2bfloat16_rn(e.src[(size_t)i * e.ld_src + o] - __bfloat162float(v));
     }
 }
 
@@ -663,6 +750,9 @@ struct UmmaEngine {
     StepChain* step = nullptr;
     __nv_bfloat16 *wht[2] = {}, *whn[2] = {};
     float* head_bias_pad[2] = {};
+    bool head_copies = false;                    // the optimiser step keeps wht / whn / head_bias_pad current
+    int head_n[2] = {};                          // head outputs rounded up to 16; wht rows [head_n, 2 head_n) hold the
+                                                 // low-order parts of the weights (what BF16 rounding left)
     float* step_slots[2][kMaxLayers] = {};
     int step_slot_rows = 0;
 };
@@ -719,8 +809,10 @@ cudaError_t launch_tc(const TcParams& P, int num_sms, cudaStream_t s) {
 
 // The program of one net for the fused forward; false when the widths do not fit the kernel
 // (first hidden layer <= 512 and a multiple of 128 beyond 256, the others <= 256).
-bool compile_chain(ChainNet& N, int nh, const int* pw, int kp, int* bn_of_layer) {
+// head_n > 0: a head job of that many output columns (a multiple of 16, at most 64) follows the last layer.
+bool compile_chain(ChainNet& N, int nh, const int* pw, int kp, int* bn_of_layer, int head_n) {
     memset(&N, 0, sizeof N);
+    if (head_n > 0 && nh == 1 && pw[0] > 256) return false;
     if (nh < 1 || nh > kChainLayers || pw[0] > 512 || (pw[0] > 256 && pw[0] % 128 != 0)) return false;
     for (int l = 1; l < nh; ++l)
         if (pw[l] > 256) return false;
@@ -729,8 +821,10 @@ bool compile_chain(ChainNet& N, int nh, const int* pw, int kp, int* bn_of_layer)
         N.job[nj] = ChainJob{layer, n0, bn, kb0, nkb, a_ring, tmem_col, accumulate, wait_epi};
         return nj++;
     };
+    int last_col = 0;                  // accumulator half of the most recent epilogue
     auto epi = [&](int layer, int n0, int ncols, int tmem_col, int wait_job, int write_job) {
-        N.epi[ne] = ChainEpi{layer, n0, ncols, tmem_col, wait_job, write_job};
+        N.epi[ne] = ChainEpi{0, layer, n0, ncols, tmem_col, wait_job, write_job};
+        last_col = tmem_col;
         return ne++;
     };
     const int kb_in = kp / BLOCK_K;
@@ -779,6 +873,19 @@ bool compile_chain(ChainNet& N, int nh, const int* pw, int kp, int* bn_of_layer)
             const int j = job(l, 0, pw[l], 0, pw[l - 1] / BLOCK_K, 0, col, 0, prev_e);
             prev_e = epi(l, 0, pw[l], col, j, -1);
         }
+    }
+    if (head_n > 0) {
+        if (nj == kChainJobs || ne == kChainEpis) return false;
+        // the head reads the last activations from the buffer and accumulates in the half the last layer left free
+        const int last_e = ne - 1;
+        const int jh = job(nh, 0, 2 * head_n, 0, pw[nh - 1] / BLOCK_K, 0, last_col ^ 256, 0, last_e);
+        N.epi[ne] = ChainEpi{1, nh - 1, 0, 2 * head_n, last_col ^ 256, jh, -1};
+        N.head_n = head_n;
+        const int eh = ne++;
+        // an item starts once the head epilogue of the item before is done: every accumulator is drained by then
+        N.flip = 0;
+        for (int j = 0; j < nj; ++j)
+            if (N.job[j].wait_epi < 0 || N.job[j].wait_epi >= kPrevItem) N.job[j].wait_epi = j == 0 ? kPrevItem + eh : -1;
     }
     N.nlayers = nh; N.njobs = nj; N.nepis = ne;
     return nj <= kChainJobs && ne <= kChainEpis;
@@ -883,7 +990,8 @@ UmmaEngine* umma_create(const UmmaSetup& s, std::string* err) {
     // head weights as tensor-core operands (output-major and input-major, padded to 64 outputs)
     for (int ni = 0; ni < 2; ++ni) {
         const int pl = e->pw[ni][e->nh[ni] - 1];
-        if (!ealloc(e, &e->wht[ni], (size_t)64 * pl) || !ealloc(e, &e->whn[ni], (size_t)pl * 64) ||
+        e->head_n[ni] = ((ni == 0 ? s.out[0][e->nh[0]] : 1) + 15) / 16 * 16;
+        if (!ealloc(e, &e->wht[ni], (size_t)128 * pl) || !ealloc(e, &e->whn[ni], (size_t)pl * 64) ||
             !ealloc(e, &e->head_bias_pad[ni], (size_t)64))
             return bail("allocation failed");
     }
@@ -908,10 +1016,12 @@ UmmaEngine* umma_create(const UmmaSetup& s, std::string* err) {
         c.src = s.param + s.w_off[ni][l]; c.in = s.in[ni][l]; c.out = s.out[ni][l]; c.ld_src = s.out_p[ni][l];
         c.wt = e->wht[ni]; c.ld_wt = e->pw[ni][l - 1];
         c.wn = e->whn[ni]; c.ld_wn = 64;
+        c.wt_lo = e->wht[ni] + (size_t)e->head_n[ni] * c.ld_wt;
         table.push_back(c);
         e->cvt_max = std::max(e->cvt_max, c.in * c.out);
     }
     e->n_cvt = (int)table.size();
+    e->head_copies = e->n_cvt <= kMaxCvt && s.out[0][e->nh[0]] <= 64;
     if (!ealloc(e, &e->cvt_dev, table.size())) return bail("allocation failed");
     if (cudaMemcpyAsync(e->cvt_dev, table.data(), table.size() * sizeof(CvtEntry), cudaMemcpyHostToDevice, s.stream) != cudaSuccess ||
         cudaStreamSynchronize(s.stream) != cudaSuccess)
@@ -951,7 +1061,14 @@ UmmaEngine* umma_create(const UmmaSetup& s, std::string* err) {
             if ((ni == 0 && !actor) || (ni == 1 && !critic)) continue;
             const int n = P.nnets;
             int bn[kChainLayers] = {};
-            if (e->nh[ni] > kChainLayers || !compile_chain(P.net[n], e->nh[ni], e->pw[ni], e->kp[ni], bn)) return true;   // not applicable
+            const int n_out = ni == 0 ? s.out[0][e->nh[0]] : 1;
+            const int head_n = e->head_copies ? e->head_n[ni] : 0;
+            if (e->nh[ni] > kChainLayers || !compile_chain(P.net[n], e->nh[ni], e->pw[ni], e->kp[ni], bn, head_n)) return true;   // not applicable
+            if (head_n > 0) {
+                const int pl = e->pw[ni][e->nh[ni] - 1];
+                if (!make_tmap(&P.tmW[n][e->nh[ni]], e->wht[ni], 128, pl, pl, BLOCK_K, 2 * head_n)) return false;
+                P.net[n].is_actor = ni == 0; P.net[n].A = n_out; P.net[n].head_bias = e->head_bias_pad[ni];
+            }
             if (!make_tmap(&P.tmX[n], act_buffers ? e->obs16_act[ni] : e->x16[ni], rows, e->kp[ni], e->kp[ni], BLOCK_K, BLOCK_M)) return false;
             for (int l = 0; l < e->nh[ni]; ++l) {
                 const int kin = l == 0 ? e->kp[ni] : e->pw[ni][l - 1];
@@ -1075,8 +1192,7 @@ UmmaEngine* umma_create(const UmmaSetup& s, std::string* err) {
     // (off unless RSLRL_FUSED_STEP=1: on the workloads measured so far its items, which run their layers
     // one after the other, take longer than the per-layer launches whose tiles overlap)
     const char* fused_env = std::getenv("RSLRL_FUSED_STEP");
-    if (fused_env && fused_env[0] == '1' && R == s.Bmb && e->nh[0] <= kStepChainLayers && e->nh[1] <= kStepChainLayers && s.out[0][e->nh[0]] <= 64 &&
-        e->n_cvt + 0 <= kMaxCvt) {
+    if (fused_env && fused_env[0] == '1' && R == s.Bmb && e->nh[0] <= kStepChainLayers && e->nh[1] <= kStepChainLayers && e->head_copies) {
         StepChainSetup cs{};
         cs.rows = R; cs.alpha = alpha; cs.error = e->error_dev; cs.num_sms = e->num_sms;
         cs.log_std = s.param + s.logstd_off;
@@ -1120,9 +1236,10 @@ void umma_fill_cvt(UmmaEngine* e, AdamArgs* a) {
             c.in = s.in[ni][l]; c.out = s.out[ni][l]; c.out_p = s.out_p[ni][l];
             c.wt = e->wt[ni][l]; c.ld_wt = l == 0 ? e->kp[ni] : e->pw[ni][l - 1];
             c.wn = l > 0 ? e->wn[ni][l] : nullptr; c.ld_wn = e->pw[ni][l];
+            c.wt_lo = nullptr;
             c.bias_pad = e->bias_pad[ni][l];
         }
-    for (int ni = 0; ni < 2 && e->step; ++ni) {
+    for (int ni = 0; ni < 2 && e->head_copies; ++ni) {
         if (a->n_cvt == kMaxCvt) break;
         const int l = e->nh[ni];
         CvtRange& c = a->cvt[a->n_cvt++];
@@ -1130,6 +1247,7 @@ void umma_fill_cvt(UmmaEngine* e, AdamArgs* a) {
         c.in = s.in[ni][l]; c.out = s.out[ni][l]; c.out_p = s.out_p[ni][l];
         c.wt = e->wht[ni]; c.ld_wt = e->pw[ni][l - 1];
         c.wn = e->whn[ni]; c.ld_wn = 64;
+        c.wt_lo = e->wht[ni] + (size_t)e->head_n[ni] * c.ld_wt;
         c.bias_pad = e->head_bias_pad[ni];
     }
 }
@@ -1161,10 +1279,12 @@ cudaError_t umma_refresh_weights(UmmaEngine* e) {
 }
 
 cudaError_t umma_act_forward(UmmaEngine* e, const float* d_obs_a, const float* d_obs_c, float* store_a, float* store_c,
-                             int sa, int sc, bool do_actor, const void** ha, int* ldha, const void** hc, int* ldhc) {
+                             int sa, int sc, bool do_actor, const ActOut& out, const float* log_std, uint64_t seed,
+                             uint32_t global_step, bool* heads_done, const void** ha, int* ldha, const void** hc, int* ldhc) {
     const UmmaSetup& s = e->s;
     cudaError_t err;
     const bool shared = s.model.shared_obs != 0;
+    *heads_done = false;
     if (do_actor) {
         err = launch_pad_rows(d_obs_a, s.in_dim[0], store_a, sa, e->obs16_act[0], e->kp[0], s.N, s.stream);
         if (err != cudaSuccess) return err;
@@ -1176,9 +1296,18 @@ cudaError_t umma_act_forward(UmmaEngine* e, const float* d_obs_a, const float* d
         err = launch_pad_rows(d_obs_c, s.in_dim[1], nullptr, 0, e->obs16_act[1], e->kp[1], s.N, s.stream);
         if (err != cudaSuccess) return err;
     }
-    const std::vector<ChainParams>& fused = do_actor ? e->chain_act : e->chain_act_critic;
+    std::vector<ChainParams>& fused = do_actor ? e->chain_act : e->chain_act_critic;
     if (!fused.empty()) {
-        err = launch_chain(fused[0], e->num_sms, s.stream);
+        ChainParams& P = fused[0];
+        if (P.net[0].A > 0) {
+            // the heads run in the same launch and write the rollout outputs of this step
+            P.ho.actions = out.actions; P.ho.mu = out.mu; P.ho.sigma = out.sigma; P.ho.logp = out.logp;
+            P.ho.values = out.values; P.ho.actions_out = out.actions_out; P.ho.act_stride = out.act_stride;
+            P.ho.log_std = log_std;
+            P.ho.seed_lo = (uint32_t)seed; P.ho.seed_hi = (uint32_t)(seed >> 32); P.ho.global_step = global_step;
+            *heads_done = true;
+        }
+        err = launch_chain(P, e->num_sms, s.stream);
         if (err != cudaSuccess) return err;
     } else {
         const std::vector<TcParams>& seq = do_actor ? e->act_fwd : e->act_fwd_critic;

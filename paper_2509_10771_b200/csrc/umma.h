@@ -39,10 +39,13 @@ void umma_fill_cvt(UmmaEngine* e, AdamArgs* a);
 void umma_fill_bias_sources(UmmaEngine* e, ReduceArgs* r, const HeadLossArgs& hl);
 // Hidden layers on N rollout rows.  d_obs_* are dense [N][dim] FP32 rows; when store_* is not
 // null the padded FP32 copy of the observations is also written there (row strides sa / sc).
-// Returns the last hidden activations of both nets (actor's only when do_actor).
+// Returns the last hidden activations of both nets (actor's only when do_actor).  Where the
+// fused kernel applies the heads run in the same launch: it samples the actions (do_actor) and
+// writes the rollout outputs named by `out` (values only when !do_actor) and sets *heads_done.
 cudaError_t umma_act_forward(UmmaEngine* e, const float* d_obs_a, const float* d_obs_c, float* store_a,
-                             float* store_c, int sa, int sc, bool do_actor, const void** ha, int* ldha,
-                             const void** hc, int* ldhc);
+                             float* store_c, int sa, int sc, bool do_actor, const ActOut& out,
+                             const float* log_std, uint64_t seed, uint32_t global_step, bool* heads_done,
+                             const void** ha, int* ldha, const void** hc, int* ldhc);
 // Point the gather at one of the engine's two minibatch input buffers (buf = 0 or 1); the forward
 // and backward launches take the same index.  With two buffers the gather of the next minibatch
 // can run while the current one is worked on (not with the fused step kernel, which has one).

@@ -669,6 +669,7 @@ __global__ void __launch_bounds__(kAdamThreads) adam_kernel(const AdamArgs a) {
                         const __nv_bfloat16 w = __float2bfloat16_rn(p[q]);
                         c.wt[(size_t)(o + q) * c.ld_wt + row] = w;
                         if (c.wn) c.wn[(size_t)row * c.ld_wn + o + q] = w;
+                        if (c.wt_lo) c.wt_lo[(size_t)(o + q) * c.ld_wt + row] = __float2bfloat16_rn(p[q] - __bfloat162float(w));
                     }
                 }
                 break;
