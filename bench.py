@@ -58,15 +58,38 @@ def hidden_flops_per_row(w, net):
 
 
 def family_flops(w):
-    """FLOPs of one learn iteration attributed to the three tensor-core kernel families."""
+    """FLOPs of one learn iteration attributed to the tensor-core kernel families."""
     T, N = w.num_steps, w.num_envs
     steps = w.epochs * w.minibatches
     R = w.minibatch_rows * (2 if w.sym_enable else 1)
     fa, fc = hidden_flops_per_row(w, "actor"), hidden_flops_per_row(w, "critic")
-    fwd = T * N * (fa + fc) + N * fc + steps * R * (fa + fc)
+    ha, hc = (2 * i * o for i, o in (w.layer_dims("actor")[-1], w.layer_dims("critic")[-1]))
+    rollout = T * N * (fa + fc + ha + hc) + N * (fc + hc)        # fused forward + heads of act and of the last value
+    fwd = steps * R * (fa + fc)
     dgrad = steps * R * sum(2 * i * o for net in ("actor", "critic") for i, o in w.layer_dims(net)[1:-1])
     wgrad = steps * R * sum(2 * i * o for net in ("actor", "critic") for i, o in w.layer_dims(net))
-    return {"tc_gemm_fwd": fwd, "tc_gemm_dgrad": dgrad, "tc_gemm_wgrad": wgrad}
+    return {"tc_mlp_fwd": rollout, "tc_gemm_fwd": fwd, "tc_gemm_dgrad": dgrad, "tc_gemm_wgrad": wgrad}
+
+
+# DRAM bytes per launch (dram__bytes_read.sum + dram__bytes_write.sum, mean over the family's launches of one
+# minibatch step) from the ncu capture summarised under profiles/, valid while the kernel source is the one
+# that capture ran (recognised by its SHA-256); otherwise the traffic is reported as null.
+NCU_TRAFFIC = {
+    "source": "paper_2509_10771_b200/csrc/umma.cu",
+    "sha256": "@UMMA_SHA@",
+    "bytes_per_launch": {"tc_gemm_fwd": 30.86e6, "tc_gemm_dgrad": 64.89e6, "tc_gemm_wgrad": 203.48e6},
+}
+
+
+def ncu_traffic(family):
+    import hashlib
+    try:
+        digest = hashlib.sha256(open(os.path.join(ROOT, NCU_TRAFFIC["source"]), "rb").read()).hexdigest()
+    except OSError:
+        return None
+    if digest != NCU_TRAFFIC["sha256"]:
+        return None
+    return NCU_TRAFFIC["bytes_per_launch"].get(family)
 
 
 def iteration_flops(w):
@@ -109,11 +132,17 @@ def blas_threads():
 def run_reference(args, rank):
     if rank != 0:
         return
-    w = WORKLOAD.scaled(ORACLE_SAMPLE_ENVS)
-    times = oracle_iteration_seconds(w, repeats=args.warmup + args.steps)[args.warmup:]
+    # every step is one whole learn iteration on a sample of the environments; the sample shrinks with the
+    # number of steps asked for so that the run stays within about two minutes (about 8 ms per environment)
+    n_iter = args.warmup + args.steps
+    envs = ORACLE_SAMPLE_ENVS
+    while envs > 64 and n_iter * envs * 0.008 > 120.0:
+        envs //= 2
+    w = WORKLOAD.scaled(envs)
+    times = oracle_iteration_seconds(w, repeats=n_iter)[args.warmup:]
     total = sum(times)
     value = w.batch * len(times) / total
-    sample = (f"{ORACLE_SAMPLE_ENVS} of the {WORKLOAD.num_envs} environments of {WORKLOAD.name}, whole learn "
+    sample = (f"{envs} of the {WORKLOAD.num_envs} environments of {WORKLOAD.name}, whole learn "
               f"iterations (T={w.num_steps}, E={w.epochs}, M={w.minibatches}), numpy float64")
     line = {
         "impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus,
@@ -297,7 +326,8 @@ def run_ours(args, rank, world, local_rank):
     achieved = fam_flops[top] * args.steps / (tc[top]["ms"] * 1e-3) / 1e12
     peak = peaks["bf16_tflops_sustained"]
     roofline = {"bound": "tensor", "kernel": top, "achieved": achieved, "peak": peak, "unit": "TFLOP/s",
-                "frac": achieved / peak, "traffic": None, "peak_source": f"bf16 sustained, {peaks['source']}",
+                "frac": achieved / peak, "traffic": ncu_traffic(top), "traffic_unit": "bytes per launch (ncu, dram read + write)",
+                "peak_source": f"bf16 sustained, {peaks['source']}",
                 "avg_launch_us": 1e3 * tc[top]["ms"] / tc[top]["launches"],
                 "families": {k: {"tflops": fam_flops[k] * args.steps / (tc[k]["ms"] * 1e-3) / 1e12,
                                  "frac": fam_flops[k] * args.steps / (tc[k]["ms"] * 1e-3) / 1e12 / peak} for k in tc},
@@ -335,7 +365,7 @@ def run_ours(args, rank, world, local_rank):
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=10)
+    ap.add_argument("--steps", type=int, default=50)
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     args = ap.parse_args()

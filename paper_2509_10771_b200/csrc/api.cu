@@ -74,7 +74,8 @@ struct rslrl_ctx {
     void* up_h[2][kMaxLayers] = {};
     void* up_dz[2][kMaxLayers] = {};
     float *dmu = nullptr, *dv = nullptr; int lddmu = 0;
-    int* perm = nullptr;                  // [epochs][T*N] shuffles of the current iteration
+    int* perm = nullptr;                  // [epochs][T*N] shuffles of one iteration
+    uint32_t perm_iteration = 0xFFFFFFFFu; // which iteration's shuffles perm holds (or is being filled with)
     float *partials = nullptr, *block_partials = nullptr, *sumsq_partials = nullptr, *loss_sums = nullptr;
     float* stats_dev = nullptr; float* stats_host = nullptr; int max_stat_rows = 0;
     SymTables sym{};
@@ -650,8 +651,12 @@ rslrl_status rslrl_ppo_update_steps(rslrl_ctx* c, int32_t max_steps, rslrl_updat
         CU(c, cudaEventRecord(c->ev_ready, c->stream));           // advantages and returns are in storage
         CU(c, cudaStreamWaitEvent(c->side, c->ev_ready, 0));
     }
-    // the shuffles of all epochs of this iteration, resolved in one launch
-    CU(c, launch_perm_epochs(pc.seed, c->iteration, pc.epochs, (uint32_t)(T * N), c->perm, overlap ? c->side : c->stream));
+    // the shuffles of all epochs of this iteration, resolved in one launch (with a gather stream the end of
+    // the update before has already started them, so that they run beside the rollout)
+    if (c->perm_iteration != c->iteration) {
+        CU(c, launch_perm_epochs(pc.seed, c->iteration, pc.epochs, (uint32_t)(T * N), c->perm, overlap ? c->side : c->stream));
+        c->perm_iteration = c->iteration;
+    }
     if (overlap) {
         TRY(enqueue_gather(0, 0, c->side));
         CU(c, cudaEventRecord(c->ev_gathered[0], c->side));
@@ -739,6 +744,11 @@ rslrl_status rslrl_ppo_update_steps(rslrl_ctx* c, int32_t max_steps, rslrl_updat
     }
     c->iteration++;
     c->step = 0; c->gae_done = false; c->act_pending = false;
+    if (overlap) {
+        // the next iteration's shuffles depend on the seed and the iteration number only
+        CU(c, launch_perm_epochs(pc.seed, c->iteration, pc.epochs, (uint32_t)(T * N), c->perm, c->side));
+        c->perm_iteration = c->iteration;
+    }
     if (h_stats) {
         CU(c, cudaMemcpyAsync(c->stats_host, c->stats_dev, (size_t)nsteps * 8 * sizeof(float), cudaMemcpyDeviceToHost, c->stream));
         CU(c, cudaStreamSynchronize(c->stream));

@@ -12,18 +12,32 @@ namespace {
 // ---------------------------------------------------------------------------------------
 // dst[r][0..dst_ld) = src[r][0..dim) followed by zeros; optional bf16 twin.
 // ---------------------------------------------------------------------------------------
+// One warp per row, lanes on consecutive columns: coalesced loads and stores, no index division.
 __global__ void pad_rows_kernel(const float* __restrict__ src, int dim, float* __restrict__ dst,
                                 int dst_ld, __nv_bfloat16* __restrict__ dst16, int dst16_ld,
                                 int rows) {
     chain_begin();
+    const int lane = threadIdx.x & 31;
+    const int warps = (gridDim.x * blockDim.x) >> 5;
     const int ld = max(dst ? dst_ld : 0, dst16 ? dst16_ld : 0);
-    const long long total = (long long)rows * ld;
-    for (long long i = blockIdx.x * (long long)blockDim.x + threadIdx.x; i < total;
-         i += (long long)gridDim.x * blockDim.x) {
-        const int r = (int)(i / ld), c = (int)(i % ld);
-        const float v = c < dim ? src[(size_t)r * dim + c] : 0.f;
-        if (dst && c < dst_ld) dst[(size_t)r * dst_ld + c] = v;
-        if (dst16 && c < dst16_ld) dst16[(size_t)r * dst16_ld + c] = __float2bfloat16_rn(v);
+    for (int r = (blockIdx.x * blockDim.x + threadIdx.x) >> 5; r < rows; r += warps) {
+        const float* __restrict__ s = src + (size_t)r * dim;
+        float* __restrict__ d = dst ? dst + (size_t)r * dst_ld : nullptr;
+        __nv_bfloat16* __restrict__ d16 = dst16 ? dst16 + (size_t)r * dst16_ld : nullptr;
+        for (int c0 = 0; c0 < ld; c0 += 128) {
+            float v[4];
+#pragma unroll
+            for (int q = 0; q < 4; ++q) {
+                const int c = c0 + 32 * q + lane;
+                v[q] = c < dim ? s[c] : 0.f;
+            }
+#pragma unroll
+            for (int q = 0; q < 4; ++q) {
+                const int c = c0 + 32 * q + lane;
+                if (d && c < dst_ld) d[c] = v[q];
+                if (d16 && c < dst16_ld) d16[c] = __float2bfloat16_rn(v[q]);
+            }
+        }
     }
 }
 
@@ -266,9 +280,7 @@ __global__ void __launch_bounds__(256) gae_normalize_kernel(float* __restrict__ 
 cudaError_t launch_pad_rows(const float* src, int dim, float* dst, int dst_ld, __nv_bfloat16* dst16,
                             int dst16_ld, int rows, cudaStream_t s) {
     if (rows <= 0) return cudaSuccess;
-    const int ld = std::max(dst ? dst_ld : 0, dst16 ? dst16_ld : 0);
-    const long long total = (long long)rows * ld;
-    const int blocks = (int)std::min((total + 255) / 256, (long long)(148 * 16));
+    const int blocks = std::min((rows + 7) / 8, 148 * 8);      // a warp per row
     LaunchScope scope_("pad_rows", s);
     return launch_chained(pad_rows_kernel, blocks, 256, 0, s, src, dim, dst, dst_ld, dst16, dst16_ld, rows);
 }
