@@ -76,8 +76,8 @@ def family_flops(w):
 # that capture ran (recognised by its SHA-256); otherwise the traffic is reported as null.
 NCU_TRAFFIC = {
     "source": "paper_2509_10771_b200/csrc/umma.cu",
-    "sha256": "@UMMA_SHA@",
-    "bytes_per_launch": {"tc_gemm_fwd": 30.86e6, "tc_gemm_dgrad": 64.89e6, "tc_gemm_wgrad": 203.48e6},
+    "sha256": "d72e1db0d3da93455f7806659c9690d88f45eb1efe9def50ebd9c62c555592df",
+    "bytes_per_launch": {"tc_gemm_fwd": 30.7e6, "tc_gemm_dgrad": 65.05e6, "tc_gemm_wgrad": 203.3e6},
 }
 
 
