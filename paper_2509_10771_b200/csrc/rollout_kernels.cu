@@ -244,18 +244,24 @@ __global__ void __launch_bounds__(256) gae_normalize_kernel(float* __restrict__ 
                                                             const float* __restrict__ block_moments,
                                                             int nblocks, int unbiased, float eps) {
     __shared__ float s_mean, s_inv;
-    if (threadIdx.x < 32) {
+    __shared__ Moments s_wm[8];
+    {
+        // thread i merges triples i, i+256, ... in order; then a fixed shuffle tree per warp and the
+        // eight warps in order
         Moments mom{0.f, 0.f, 0.f};
-        // lane l merges triples l, l+32, ... in order; then a fixed shuffle tree
-        for (int b = threadIdx.x; b < nblocks; b += 32) {
+        for (int b = threadIdx.x; b < nblocks; b += 256) {
             Moments o{block_moments[3 * b], block_moments[3 * b + 1], block_moments[3 * b + 2]};
             mom = merge(mom, o);
         }
         mom = warp_merge(mom);
+        if ((threadIdx.x & 31) == 0) s_wm[threadIdx.x >> 5] = mom;
+        __syncthreads();
         if (threadIdx.x == 0) {
-            const float denom = unbiased ? (mom.n - 1.f) : mom.n;
-            const float var = denom > 0.f ? mom.m2 / denom : 0.f;
-            s_mean = mom.mean;
+            Moments tot = s_wm[0];
+            for (int w = 1; w < 8; ++w) tot = merge(tot, s_wm[w]);
+            const float denom = unbiased ? (tot.n - 1.f) : tot.n;
+            const float var = denom > 0.f ? tot.m2 / denom : 0.f;
+            s_mean = tot.mean;
             s_inv = 1.0f / (sqrtf(var) + eps);
         }
     }
