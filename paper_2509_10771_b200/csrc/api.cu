@@ -82,6 +82,10 @@ struct rslrl_ctx {
     // host-variant staging
     float *stage_obs_a = nullptr, *stage_obs_c = nullptr, *stage_act = nullptr, *stage_rew = nullptr;
     uint8_t *stage_done = nullptr, *stage_to = nullptr;
+    // rewards | dones | time-outs of one step, packed: pinned host copy and its device twin, so that
+    // rslrl_record_step_host needs one transfer; the event marks the last transfer out of the host copy
+    uint8_t *pack_host = nullptr, *pack_dev = nullptr;
+    cudaEvent_t pack_sent = nullptr; bool pack_in_flight = false;
     // tensor-core engine (BF16 mode)
     UmmaEngine* umma = nullptr;
     // host state
@@ -336,6 +340,8 @@ rslrl_status rslrl_destroy(rslrl_ctx* c) {
     if (c->umma) umma_destroy(c->umma);
     for (void* p : c->allocs) cudaFree(p);
     if (c->stats_host) cudaFreeHost(c->stats_host);
+    if (c->pack_host) cudaFreeHost(c->pack_host);
+    if (c->pack_sent) cudaEventDestroy(c->pack_sent);
     delete c;
     return RSLRL_OK;
 }
@@ -449,6 +455,11 @@ rslrl_status rslrl_create(const rslrl_model_cfg* m, const rslrl_ppo_cfg* p, void
     A_(c->stage_obs_a, (size_t)N * m->actor_obs_dim);
     A_(c->stage_obs_c, (size_t)N * m->critic_obs_dim);
     A_(c->stage_act, (size_t)N * as); A_(c->stage_rew, N); A_(c->stage_done, N); A_(c->stage_to, N);
+    A_(c->pack_dev, (size_t)N * 6);
+    if (cudaMallocHost((void**)&c->pack_host, (size_t)N * 6) != cudaSuccess ||
+        cudaEventCreateWithFlags(&c->pack_sent, cudaEventDisableTiming) != cudaSuccess) {
+        c->err = "could not allocate the pinned staging buffer"; return bail(RSLRL_ERR_CUDA);
+    }
     if (p->sym_enable) {
         auto up_i = [&](const int32_t* h, int n, const int** d) -> rslrl_status {
             int* q; TRY(dev_alloc(c, &q, n));
@@ -785,8 +796,11 @@ rslrl_status rslrl_act_host(rslrl_ctx* c, const float* h_actor_obs, const float*
         CU(c, cudaMemcpyAsync(c->stage_obs_c, h_critic_obs, (size_t)N * c->mc.critic_obs_dim * sizeof(float), cudaMemcpyHostToDevice, c->stream));
     TRY(rslrl_act(c, c->stage_obs_a, c->mc.shared_obs ? nullptr : c->stage_obs_c, h_actions_out ? c->stage_act : nullptr));
     if (h_actions_out) {
-        CU(c, cudaMemcpy2DAsync(h_actions_out, (size_t)A * sizeof(float), c->stage_act, (size_t)as * sizeof(float),
-                                (size_t)A * sizeof(float), N, cudaMemcpyDeviceToHost, c->stream));
+        if (A == as)
+            CU(c, cudaMemcpyAsync(h_actions_out, c->stage_act, (size_t)N * A * sizeof(float), cudaMemcpyDeviceToHost, c->stream));
+        else
+            CU(c, cudaMemcpy2DAsync(h_actions_out, (size_t)A * sizeof(float), c->stage_act, (size_t)as * sizeof(float),
+                                    (size_t)A * sizeof(float), N, cudaMemcpyDeviceToHost, c->stream));
         CU(c, cudaStreamSynchronize(c->stream));
     }
     return RSLRL_OK;
@@ -795,10 +809,16 @@ rslrl_status rslrl_act_host(rslrl_ctx* c, const float* h_actor_obs, const float*
 rslrl_status rslrl_record_step_host(rslrl_ctx* c, const float* h_rewards, const uint8_t* h_dones, const uint8_t* h_timeouts) {
     if (!c || !h_rewards || !h_dones || !h_timeouts) return RSLRL_ERR_INVALID_ARG;
     const int N = c->st.N;
-    CU(c, cudaMemcpyAsync(c->stage_rew, h_rewards, (size_t)N * sizeof(float), cudaMemcpyHostToDevice, c->stream));
-    CU(c, cudaMemcpyAsync(c->stage_done, h_dones, (size_t)N, cudaMemcpyHostToDevice, c->stream));
-    CU(c, cudaMemcpyAsync(c->stage_to, h_timeouts, (size_t)N, cudaMemcpyHostToDevice, c->stream));
-    return rslrl_record_step(c, c->stage_rew, c->stage_done, c->stage_to);
+    // one transfer instead of three: the three arrays are packed into the pinned buffer first (it is free
+    // again once the transfer of the step before has left it)
+    if (c->pack_in_flight) CU(c, cudaEventSynchronize(c->pack_sent));
+    memcpy(c->pack_host, h_rewards, (size_t)N * sizeof(float));
+    memcpy(c->pack_host + (size_t)N * 4, h_dones, (size_t)N);
+    memcpy(c->pack_host + (size_t)N * 5, h_timeouts, (size_t)N);
+    CU(c, cudaMemcpyAsync(c->pack_dev, c->pack_host, (size_t)N * 6, cudaMemcpyHostToDevice, c->stream));
+    CU(c, cudaEventRecord(c->pack_sent, c->stream));
+    c->pack_in_flight = true;
+    return rslrl_record_step(c, reinterpret_cast<const float*>(c->pack_dev), c->pack_dev + (size_t)N * 4, c->pack_dev + (size_t)N * 5);
 }
 
 rslrl_status rslrl_gae_host(rslrl_ctx* c, const float* h_last_critic_obs) {
