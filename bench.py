@@ -203,6 +203,24 @@ class ClockSampler:
 
 
 # ------------------------------------------------------------------------------------------
+# replicas: every rank times its own copy of the workload; the job's time is the slowest rank's
+# ------------------------------------------------------------------------------------------
+def max_over_ranks(values, world, device):
+    """Element-wise maximum of `values` over the ranks of the default process group (identity for one rank)."""
+    if world <= 1:
+        return [float(v) for v in values]
+    import torch
+    import torch.distributed as dist
+    t = torch.tensor(list(values), dtype=torch.float64, device=device)
+    dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return t.tolist()
+
+
+def whole_job_value(transitions_per_rank, world, ms):
+    """Transitions per second of the whole job: every rank processed transitions_per_rank in ms (the slowest's)."""
+    return transitions_per_rank * world / (ms * 1e-3)
+
+
 def run_ours(args, rank, world, local_rank):
     import torch
     import torch.distributed as dist
@@ -303,19 +321,15 @@ def run_ours(args, rank, world, local_rank):
     prof = binding.profile_report()
     binding.profile_enable(False)
 
-    if world > 1:
-        t = torch.tensor([ms_total, ms_e2e], dtype=torch.float64, device=dev)
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        ms_total, ms_e2e = t.tolist()
+    ms_total, ms_e2e = max_over_ranks([ms_total, ms_e2e], world, dev)
     if rank != 0:
         if world > 1:
             dist.destroy_process_group()
         return
 
     peaks = read_peaks()
-    transitions = T * N * args.steps * world
-    value = transitions / (ms_total * 1e-3)
-    e2e_value = transitions / (ms_e2e * 1e-3)
+    value = whole_job_value(T * N * args.steps, world, ms_total)
+    e2e_value = whole_job_value(T * N * args.steps, world, ms_e2e)
 
     total_prof_ms = sum(v["ms"] for v in prof.values()) or 1.0
     shares = {k: {"launches": v["launches"], "ms": round(v["ms"], 3), "share": round(v["ms"] / total_prof_ms, 4)}
