@@ -27,6 +27,8 @@ CASES = {
     "rough": WL.ROUGH.scaled(300, minibatches=4),
     "humanoid": WL.HUMANOID.scaled(200, minibatches=8),
     "rough_sym": WL.ROUGH_SYM.scaled(150, minibatches=16, precision=FP32),
+    # the configuration bench.py times, at its full size (4096 envs x 24 steps, 24,576-row minibatches)
+    "rough_full": WL.ROUGH,
 }
 
 
@@ -80,6 +82,23 @@ def test_rollout_and_gae_match_oracle_bf16(case):
         assert_close(got[k], want[k], 2e-2, f"{case}.{k}")
     assert np.array_equal(got["obs_actor"], inputs["obs_actor"][:w.num_steps])
     ctx.destroy()
+
+
+def test_bench_configuration_full_size_bf16():
+    """rough_terrain at full size, BF16: every stored rollout output and the first minibatch step
+    against the oracle (which needs a few seconds at this size)."""
+    w = CASES["rough_full"]
+    theta, inputs = WL.make_params(w), WL.make_rollout_inputs(w)
+    ctx = make_ctx(w, BF16)
+    ctx.set_params(theta)
+    gpu_rollout(ctx, w, inputs)
+    got = read_storage(ctx, w)
+    want = oracle_rollout(w, theta, inputs)
+    for k in ("actions", "mu", "values", "returns", "advantages"):
+        assert_close(got[k], want[k], 2e-2, f"rough_full.{k}")
+    assert_close(got["logp"], want["logp"], 1e-5, "rough_full.logp")
+    ctx.destroy()
+    _first_step("rough_full", BF16, from_oracle_storage=True)
 
 
 def test_noise_is_the_shared_philox_stream():
