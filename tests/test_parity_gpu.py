@@ -27,8 +27,10 @@ CASES = {
     "rough": WL.ROUGH.scaled(300, minibatches=4),
     "humanoid": WL.HUMANOID.scaled(200, minibatches=8),
     "rough_sym": WL.ROUGH_SYM.scaled(150, minibatches=16, precision=FP32),
-    # the configuration bench.py times, at its full size (4096 envs x 24 steps, 24,576-row minibatches)
+    # full sizes: rough_terrain is the configuration bench.py times (4096 envs x 24 steps, 24,576-row minibatches)
+    "flat_full": WL.FLAT,
     "rough_full": WL.ROUGH,
+    "humanoid_full": WL.HUMANOID,
 }
 
 
@@ -84,10 +86,11 @@ def test_rollout_and_gae_match_oracle_bf16(case):
     ctx.destroy()
 
 
-def test_bench_configuration_full_size_bf16():
-    """rough_terrain at full size, BF16: every stored rollout output and the first minibatch step
-    against the oracle (which needs a few seconds at this size)."""
-    w = CASES["rough_full"]
+@pytest.mark.parametrize("case", ["flat_full", "rough_full", "humanoid_full"])
+def test_full_size_workloads_bf16(case):
+    """The flat, rough (the benchmarked one) and humanoid workloads at full size, BF16: every stored rollout
+    output and the first minibatch step against the oracle (which needs some seconds at these sizes)."""
+    w = CASES[case]
     theta, inputs = WL.make_params(w), WL.make_rollout_inputs(w)
     ctx = make_ctx(w, BF16)
     ctx.set_params(theta)
@@ -95,10 +98,10 @@ def test_bench_configuration_full_size_bf16():
     got = read_storage(ctx, w)
     want = oracle_rollout(w, theta, inputs)
     for k in ("actions", "mu", "values", "returns", "advantages"):
-        assert_close(got[k], want[k], 2e-2, f"rough_full.{k}")
-    assert_close(got["logp"], want["logp"], 1e-5, "rough_full.logp")
+        assert_close(got[k], want[k], 2e-2, f"{case}.{k}")
+    assert_close(got["logp"], want["logp"], 1e-5, f"{case}.logp")
     ctx.destroy()
-    _first_step("rough_full", BF16, from_oracle_storage=True)
+    _first_step(case, BF16, from_oracle_storage=True)
 
 
 def test_noise_is_the_shared_philox_stream():
@@ -135,7 +138,13 @@ def _first_step(case, precision, from_oracle_storage):
     state = O.OptimState(theta, w.lr)
     ref = O.ppo_update(state, dims_of(w), want_st, w, seed=w.seed, iteration=0, sym=mir, max_steps=1)[0]
     tol = 1e-4 if precision == FP32 else 1e-2
-    assert_close(stats["first_surrogate"], ref["surrogate"], tol, "surrogate")
+    if case.endswith("_full"):
+        # the surrogate is a mean of -A r over the minibatch with A normalised (mean 0, |A| ~ 1) and r ~ 1:
+        # over 24,576 rows it cancels to ~1e-4, so the bound is relative to the size of the terms, mean |A|
+        scale = float(np.abs(want_st["advantages"]).mean())
+        assert abs(stats["first_surrogate"] - ref["surrogate"]) <= tol * (abs(ref["surrogate"]) + scale), "surrogate"
+    else:
+        assert_close(stats["first_surrogate"], ref["surrogate"], tol, "surrogate")
     assert_close(stats["first_value_loss"], ref["value_loss"], tol, "value_loss")
     assert_close(stats["entropy"], ref["entropy"], tol, "entropy")
     assert abs(stats["first_kl"] - ref["kl"]) < (1e-6 if precision == FP32 else 1e-4)
