@@ -23,6 +23,11 @@ denote, written out in numpy float64 with no blocking, fusion or reordering:
                              KL-adaptive learning-rate rule, Adam (Kingma & Ba) with bias
                              correction
 * ``ppo_update``          -- the epoch x minibatch loop over a keyed permutation
+* ``distill_loss_and_grads`` / ``distill_update`` -- the behaviour-cloning step of "Algorithms": the
+                             student (the actor net) is rolled out, its transitions are relabelled
+                             with the expert's actions, and the student's mean is regressed on them
+                             (mean squared error, the paper names no loss) over the same keyed
+                             minibatches, with global-norm clipping and Adam, no learning-rate rule
 * ``philox4x32_10``, ``gaussian_noise``, ``feistel_permutation`` -- the counter-based random
                              streams the method draws from (Salmon et al., SC'11), so that a
                              second implementation can reproduce noise and shuffles bit for bit.
@@ -503,6 +508,62 @@ def ppo_update(state: OptimState, dims, storage: Dict[str, np.ndarray], hp, seed
                 for key in ("mu", "values", "logp", "ratio", "dmu", "dV"):
                     st.pop(key, None)
             st["rows"] = rows if not out else None
+            out.append(st)
+    return out
+
+
+# ======================================================================================
+# Distillation ("Algorithms": a behaviour-cloning algorithm similar to DAgger: roll out the
+# student, relabel the data with expert actions, train the student on it).  The paper names no
+# loss; the reading taken is the mean squared error between the student's action mean and the
+# expert's action, L = mean over rows and actions of (mu_student - a_expert)^2.  Only the actor
+# net receives a gradient (log_std and the critic get zero), the learning rate stays fixed.
+# ======================================================================================
+def distill_loss_and_grads(params, obs_actor: np.ndarray, expert_actions: np.ndarray, hp):
+    """L = sum_{r,i} (mu_i(o_r) - a*_{r,i})^2 / (B A) and its exact gradient (same layout as params)."""
+    oa = np.asarray(obs_actor, dtype=F64)
+    target = np.asarray(expert_actions, dtype=F64)
+    B, nA = target.shape
+    mu, hs = mlp_forward(oa, params["actor"], hp.elu_alpha)
+    diff = mu - target
+    L = (diff ** 2).sum() / (B * nA)
+    dmu = 2.0 * diff / (B * nA)
+    g_actor = mlp_backward(dmu, hs, params["actor"], hp.elu_alpha)
+    g_critic = [(np.zeros_like(np.asarray(W, dtype=F64)), np.zeros_like(np.asarray(b, dtype=F64)))
+                for W, b in params["critic"]]
+    grads = {"actor": g_actor, "critic": g_critic, "log_std": np.zeros(nA)}
+    return {"loss": float(L), "mu": mu, "dmu": dmu}, grads
+
+
+def distill_update(state: OptimState, dims, obs_actor: np.ndarray, expert_actions: np.ndarray, hp, seed: int,
+                   iteration: int, max_steps: Optional[int] = None) -> List[Dict]:
+    """Epoch x minibatch loop of the distillation step over obs_actor[T][N][Da] / expert_actions[T][N][A]:
+    the same keyed permutation and contiguous chunks as ``ppo_update``; per minibatch the loss above,
+    global-norm clipping and Adam with the fixed learning rate ``state.lr``."""
+    T, N = expert_actions.shape[:2]
+    B = T * N
+    if B % hp.minibatches:
+        raise ValueError("batch not divisible by the number of minibatches")
+    rows_per = B // hp.minibatches
+    actor_dims, critic_dims, nA = dims
+    obs = np.asarray(obs_actor)[:T].reshape(B, -1)
+    tgt = np.asarray(expert_actions).reshape(B, -1)
+    out = []
+    for e in range(hp.epochs):
+        perm = feistel_permutation(seed, iteration, e, B)
+        for k in range(hp.minibatches):
+            if max_steps is not None and len(out) >= max_steps:
+                return out
+            rows = perm[k * rows_per:(k + 1) * rows_per]
+            params = unpack_params(state.theta, actor_dims, critic_dims, nA)
+            stats, grads = distill_loss_and_grads(params, obs[rows], tgt[rows], hp)
+            g = pack_grads(grads)
+            g_norm = math.sqrt(float((g * g).sum()))
+            coef = clip_coefficient(g_norm, hp.max_grad_norm)
+            state.step += 1
+            state.theta, state.m, state.v = adam_step(state.theta, g * coef, state.m, state.v, state.step,
+                                                      state.lr, hp.adam_b1, hp.adam_b2, hp.adam_eps)
+            st = {"loss": stats["loss"], "grad": g, "grad_norm": g_norm, "lr": state.lr}
             out.append(st)
     return out
 

@@ -468,3 +468,102 @@ def test_rollout_storage_shapes_and_normalised_advantages():
     a = st["advantages"]
     assert abs(a.mean()) < 1e-12 and a.std(ddof=1) == pytest.approx(1.0, rel=1e-6)
     assert np.allclose(st["returns"], st["advantages_raw"] + st["values"])
+
+
+# --------------------------------------------------------------------------------------
+# distillation (paper, "Algorithms": behaviour cloning similar to DAgger)
+# --------------------------------------------------------------------------------------
+def _distill_problem(seed=3, B=30):
+    theta, dims, batch = small_problem(seed, B=B)
+    rng = np.random.default_rng(seed + 100)
+    target = rng.normal(size=batch["actions"].shape)
+    return theta, dims, batch["obs_actor"], target
+
+
+def test_distill_loss_matches_torch_mse_and_autograd():
+    theta, dims, obs, target = _distill_problem()
+    adims, cdims, A = dims
+    h = hp()
+    stats, grads = O.distill_loss_and_grads(O.unpack_params(theta, adims, cdims, A), obs, target, h)
+    p = torch.tensor(theta, dtype=torch.float64, requires_grad=True)
+    off, x = 0, torch.as_tensor(obs, dtype=torch.float64)
+    for li, (fi, fo) in enumerate(adims):
+        W = p[off:off + fi * fo].reshape(fi, fo); off += fi * fo
+        b = p[off:off + fo]; off += fo
+        x = x @ W + b
+        if li < len(adims) - 1:
+            x = torch.nn.functional.elu(x, alpha=h.elu_alpha)
+    L = torch.nn.functional.mse_loss(x, torch.as_tensor(target, dtype=torch.float64))
+    L.backward()
+    assert stats["loss"] == pytest.approx(L.item(), rel=1e-12)
+    g = O.pack_grads(grads)
+    assert np.allclose(g, p.grad.numpy(), rtol=1e-9, atol=1e-13)
+    # log_std and the critic take no part
+    n_actor = sum(i * o + o for i, o in adims)
+    assert np.all(g[n_actor:] == 0.0)
+
+
+def test_distill_gradient_matches_central_finite_differences():
+    theta, dims, obs, target = _distill_problem(5, B=16)
+    adims, cdims, A = dims
+    h = hp()
+    loss = lambda th: O.distill_loss_and_grads(O.unpack_params(th, adims, cdims, A), obs, target, h)[0]["loss"]
+    g = O.pack_grads(O.distill_loss_and_grads(O.unpack_params(theta, adims, cdims, A), obs, target, h)[1])
+    n_actor = sum(i * o + o for i, o in adims)
+    rng = np.random.default_rng(2)
+    for i in rng.integers(0, n_actor, 40):
+        e = np.zeros_like(theta); e[i] = 1e-6
+        fd = (loss(theta + e) - loss(theta - e)) / 2e-6
+        assert g[i] == pytest.approx(fd, rel=2e-5, abs=1e-9), i
+
+
+def test_distill_zero_when_the_student_already_matches_and_quadratic_in_the_error():
+    theta, dims, obs, _ = _distill_problem(9)
+    adims, cdims, A = dims
+    h = hp()
+    params = O.unpack_params(theta, adims, cdims, A)
+    mu, _ = O.mlp_forward(obs, params["actor"], h.elu_alpha)
+    stats, grads = O.distill_loss_and_grads(params, obs, mu, h)
+    assert stats["loss"] == 0.0 and np.all(O.pack_grads(grads) == 0.0)
+    d = np.random.default_rng(0).normal(size=mu.shape)
+    l1 = O.distill_loss_and_grads(params, obs, mu + d, h)[0]["loss"]
+    l2 = O.distill_loss_and_grads(params, obs, mu + 2 * d, h)[0]["loss"]
+    assert l1 == pytest.approx((d ** 2).mean(), rel=1e-12) and l2 == pytest.approx(4 * l1, rel=1e-12)
+
+
+def test_distill_update_loop_matches_torch_reference_loop():
+    """Same shuffle and chunks as the PPO update, clip, Adam with a fixed learning rate."""
+    w = WL.TINY.scaled(16, epochs=2, minibatches=2)
+    dims = (w.layer_dims("actor"), w.layer_dims("critic"), w.num_actions)
+    theta0 = WL.make_params(w).astype(np.float64)
+    inp = WL.make_rollout_inputs(w)
+    T, N, A = w.num_steps, w.num_envs, w.num_actions
+    expert = np.random.default_rng(4).normal(size=(T, N, A))
+    state = O.OptimState(theta0, w.lr)
+    steps = O.distill_update(state, dims, inp["obs_actor"], expert, w, seed=w.seed, iteration=3)
+    assert len(steps) == 4 and state.step == 4 and state.lr == w.lr
+
+    adims = dims[0]
+    p = torch.tensor(theta0, dtype=torch.float64, requires_grad=True)
+    opt = torch.optim.Adam([p], lr=w.lr)
+    B = T * N
+    obs = torch.as_tensor(inp["obs_actor"][:T].reshape(B, -1), dtype=torch.float64)
+    tgt = torch.as_tensor(expert.reshape(B, A))
+    for e in range(2):
+        perm = O.feistel_permutation(w.seed, 3, e, B)
+        for k in range(2):
+            rows = torch.as_tensor(perm[k * (B // 2):(k + 1) * (B // 2)].astype(np.int64))
+            opt.zero_grad()
+            off, x = 0, obs[rows]
+            for li, (fi, fo) in enumerate(adims):
+                W = p[off:off + fi * fo].reshape(fi, fo); off += fi * fo
+                b = p[off:off + fo]; off += fo
+                x = x @ W + b
+                if li < len(adims) - 1:
+                    x = torch.nn.functional.elu(x, alpha=w.elu_alpha)
+            L = torch.nn.functional.mse_loss(x, tgt[rows])
+            L.backward()
+            torch.nn.utils.clip_grad_norm_([p], w.max_grad_norm)
+            opt.step()
+            assert steps[e * 2 + k]["loss"] == pytest.approx(L.item(), rel=1e-9)
+    assert np.allclose(state.theta, p.detach().numpy(), rtol=1e-9, atol=1e-12)
