@@ -376,18 +376,99 @@ def run_ours(args, rank, world, local_rank):
         dist.destroy_process_group()
 
 
+def run_distill(args):
+    """--task distill: the distillation iteration (T x (act + record_step) with the student, then
+    rslrl_distill_update on stand-in expert actions) on the same workload, one GPU.  Prints its own JSON line:
+    device-timed transitions/s, per-kernel shares, and the oracle's distillation update timed on a sample."""
+    import torch
+    from paper_2509_10771_b200 import binding, build
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device: the path has no CPU fallback")
+    torch.cuda.set_device(0)
+    build.build()
+    w = WORKLOAD
+    T, N = w.num_steps, w.num_envs
+    dev = torch.device("cuda", 0)
+    stream = torch.cuda.current_stream()
+    inputs = WL.make_rollout_inputs(w)
+    ctx = binding.Context(w, precision=PRECISION, stream=stream.cuda_stream)
+    ctx.set_params(WL.make_params(w))
+    d_obs = torch.from_numpy(inputs["obs_actor"]).to(dev)
+    d_rew = torch.from_numpy(inputs["rewards"]).to(dev)
+    d_done = torch.from_numpy(inputs["dones"]).to(dev)
+    d_to = torch.from_numpy(inputs["timeouts"]).to(dev)
+    stride = ctx.storage_view().act_stride
+    expert = np.zeros((T, N, stride), dtype=np.float32)
+    expert[..., :w.num_actions] = WL.make_expert_actions(w)
+    d_expert = torch.from_numpy(expert).to(dev)
+    flush_buf = torch.empty(256 << 20, dtype=torch.uint8, device=dev)
+
+    def iteration():
+        for t in range(T):
+            ctx.act(d_obs[t])
+            ctx.record_step(d_rew[t], d_done[t], d_to[t])
+        ctx.distill_update(d_expert, want_stats=False)
+
+    for _ in range(max(args.warmup, 3)):
+        iteration()
+    torch.cuda.synchronize()
+    evs = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(args.steps)]
+    for a, b in evs:
+        flush_buf.zero_()
+        a.record(stream)
+        iteration()
+        b.record(stream)
+    torch.cuda.synchronize()
+    ms = sum(a.elapsed_time(b) for a, b in evs)
+    binding.profile_enable(True)
+    binding.profile_report()
+    for _ in range(args.steps):
+        iteration()
+    torch.cuda.synchronize()
+    prof = binding.profile_report()
+    binding.profile_enable(False)
+    total = sum(v["ms"] for v in prof.values()) or 1.0
+    shares = {k: {"launches": v["launches"], "ms": round(v["ms"], 3), "share": round(v["ms"] / total, 4)}
+              for k, v in sorted(prof.items(), key=lambda kv: -kv[1]["ms"])}
+    # the oracle's distillation update on a sample of the environments
+    from oracle import ppo_oracle as O
+    ws = WORKLOAD.scaled(ORACLE_SAMPLE_ENVS)
+    dims = (ws.layer_dims("actor"), ws.layer_dims("critic"), ws.num_actions)
+    state = O.OptimState(WL.make_params(ws).astype(np.float64), ws.lr)
+    t0 = time.perf_counter()
+    O.distill_update(state, dims, WL.make_rollout_inputs(ws)["obs_actor"], WL.make_expert_actions(ws), ws, seed=ws.seed, iteration=0)
+    cpu_s = time.perf_counter() - t0
+    line = {
+        "metric": "distillation iteration transitions/s", "value": T * N * args.steps / (ms * 1e-3), "unit": UNIT, "n_gpus": 1,
+        "steps": args.steps, "warmup": max(args.warmup, 3), "ms_per_step": ms / args.steps, "higher_is_better": True,
+        "dtype": "bf16", "data": "synthetic",
+        "config": {"workload": w.name, "task": "distill", "num_envs": N, "num_steps": T, "epochs": w.epochs,
+                   "minibatches": w.minibatches, "l2": "256 MiB buffer written between timed steps"},
+        "kernel_shares": shares,
+        "cpu_baseline": {"value": ws.batch / cpu_s, "unit": UNIT, "cores": blas_threads(), "kind": "oracle",
+                         "sample": f"the oracle's distillation update on {ORACLE_SAMPLE_ENVS} of the {N} environments (rollout not included)"},
+    }
+    print(json.dumps(line), flush=True)
+    ctx.destroy()
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
     ap.add_argument("--steps", type=int, default=50)
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--task", default="ppo", choices=["ppo", "distill"],
+                    help="ppo: the learn iteration the metric is quoted on (default); distill: the distillation iteration")
     args = ap.parse_args()
     rank = int(os.environ.get("RANK", "0"))
     world = int(os.environ.get("WORLD_SIZE", "1"))
     local_rank = int(os.environ.get("LOCAL_RANK", "0"))
     if args.impl == "reference":
         run_reference(args, rank)
+    elif args.task == "distill":
+        if rank == 0:
+            run_distill(args)
     else:
         run_ours(args, rank, world, local_rank)
 

@@ -212,6 +212,22 @@ rslrl_status rslrl_ppo_update(rslrl_ctx *ctx, rslrl_update_stats *h_stats);
  * state after exactly one optimiser step).  max_steps <= 0 means all E*M steps. */
 rslrl_status rslrl_ppo_update_steps(rslrl_ctx *ctx, int32_t max_steps, rslrl_update_stats *h_stats);
 
+/* Distillation step (paper: "Algorithms", the behaviour-cloning algorithm similar to DAgger: roll out the
+ * student, relabel its data with expert actions, train the student on it).  The student is this
+ * context's actor net; the rollout is the T steps collected with rslrl_act / rslrl_record_step
+ * (rslrl_gae is not needed).  For E epochs over the same keyed minibatches as rslrl_ppo_update:
+ * gather, actor forward, L = mean over rows and actions of (mu - a_expert)^2 (the paper names no
+ * loss), backward, global grad-norm clip, Adam with the current learning rate (no KL rule).  The
+ * critic and log_std receive a zero gradient.  Starts a new rollout (step = 0).
+ *   d_expert_actions [T][N][act_stride] float32 (device), act_stride as in rslrl_storage; columns
+ *   at and beyond num_actions are ignored.
+ * Stats: surrogate / first_surrogate carry L; value_loss, kl, sym_loss are 0.
+ * RSLRL_ERR_STATE unless exactly T steps were recorded; RSLRL_ERR_UNSUPPORTED with sym_enable. */
+rslrl_status rslrl_distill_update(rslrl_ctx *ctx, const float *d_expert_actions, rslrl_update_stats *h_stats);
+/* The same, stopping after `max_steps` minibatch steps (max_steps <= 0: all). */
+rslrl_status rslrl_distill_update_steps(rslrl_ctx *ctx, const float *d_expert_actions, int32_t max_steps,
+                                        rslrl_update_stats *h_stats);
+
 /* Host-buffer variants of the per-step calls: the same work with the host<->device copies
  * inside the call (pinned host memory makes them asynchronous).  h_actions_out[N][A] dense;
  * when it is not NULL the call waits for the actions. */

@@ -79,7 +79,7 @@ EXPORTS = [
     "rslrl_num_params", "rslrl_create", "rslrl_destroy", "rslrl_last_error", "rslrl_storage_view",
     "rslrl_set_params", "rslrl_get_params", "rslrl_get_grads", "rslrl_get_adam", "rslrl_set_adam",
     "rslrl_get_counters", "rslrl_set_counters", "rslrl_act", "rslrl_record_step", "rslrl_gae",
-    "rslrl_ppo_update", "rslrl_ppo_update_steps", "rslrl_act_host", "rslrl_record_step_host",
+    "rslrl_ppo_update", "rslrl_ppo_update_steps", "rslrl_distill_update", "rslrl_distill_update_steps", "rslrl_act_host", "rslrl_record_step_host",
     "rslrl_gae_host", "rslrl_gae_scratch_bytes", "rslrl_gae_scan", "rslrl_minibatch_indices",
     "rslrl_kernel_launch_count", "rslrl_profile_enable", "rslrl_profile_report", "rslrl_gae_scan_static",
 ]
@@ -115,6 +115,8 @@ def load_library() -> C.CDLL:
         "rslrl_gae": (i32, [vp, vp]),
         "rslrl_ppo_update": (i32, [vp, C.POINTER(UpdateStats)]),
         "rslrl_ppo_update_steps": (i32, [vp, i32, C.POINTER(UpdateStats)]),
+        "rslrl_distill_update": (i32, [vp, vp, C.POINTER(UpdateStats)]),
+        "rslrl_distill_update_steps": (i32, [vp, vp, i32, C.POINTER(UpdateStats)]),
         "rslrl_act_host": (i32, [vp, vp, vp, vp]),
         "rslrl_record_step_host": (i32, [vp, vp, vp, vp]),
         "rslrl_gae_host": (i32, [vp, vp]),
@@ -273,6 +275,13 @@ class Context:
             self._check(self.lib.rslrl_ppo_update_steps(self.handle, max_steps, ref))
         else:
             self._check(self.lib.rslrl_ppo_update(self.handle, ref))
+        return st.as_dict() if want_stats else None
+
+    def distill_update(self, d_expert_actions, want_stats: bool = True, max_steps: int = 0) -> Optional[Dict[str, float]]:
+        """rslrl_distill_update: the student's mean regressed on d_expert_actions [T][N][act_stride]."""
+        st = UpdateStats()
+        ref = C.byref(st) if want_stats else None
+        self._check(self.lib.rslrl_distill_update_steps(self.handle, _ptr(d_expert_actions), max_steps, ref))
         return st.as_dict() if want_stats else None
 
     def act_host(self, h_actor_obs: np.ndarray, h_critic_obs=None, h_actions_out=None):

@@ -628,9 +628,11 @@ rslrl_status rslrl_gae(rslrl_ctx* c, const float* d_last_critic_obs) {
 }
 
 // -------------------------------------------------------------------------------- update
-rslrl_status rslrl_ppo_update_steps(rslrl_ctx* c, int32_t max_steps, rslrl_update_stats* h_stats) {
-    if (!c) return RSLRL_ERR_INVALID_ARG;
-    if (!c->gae_done) return fail(c, RSLRL_ERR_STATE, "rslrl_gae must precede rslrl_ppo_update");
+// The epoch x minibatch loop.  d_expert == nullptr: the PPO update.  Otherwise the distillation step: the
+// gathered "actions" are the expert's, the head/loss kernel regresses the policy mean on them, the critic
+// and log_std get no gradient and the learning rate is not adapted.
+static rslrl_status update_impl(rslrl_ctx* c, int32_t max_steps, rslrl_update_stats* h_stats, const float* d_expert) {
+    const bool distill = d_expert != nullptr;
     const rslrl_ppo_cfg& pc = c->pc;
     const int N = c->st.N, T = c->st.T, A = c->mc.num_actions;
     const int total_steps = pc.epochs * pc.minibatches;
@@ -642,7 +644,7 @@ rslrl_status rslrl_ppo_update_steps(rslrl_ctx* c, int32_t max_steps, rslrl_updat
     auto enqueue_gather = [&](int step, int buf, cudaStream_t st) -> rslrl_status {
         const int e = step / pc.minibatches, k = step % pc.minibatches;
         GatherArgs g{};
-        g.obs_a = c->st.obs_actor; g.obs_c = c->st.obs_critic; g.actions = c->st.actions; g.mu = c->st.mu;
+        g.obs_a = c->st.obs_actor; g.obs_c = c->st.obs_critic; g.actions = distill ? d_expert : c->st.actions; g.mu = c->st.mu;
         g.sigma = c->st.sigma; g.logp = c->st.logp; g.values = c->st.values; g.returns = c->st.returns;
         g.adv = c->st.advantages;
         g.N = N; g.sa = c->st.obs_a_stride; g.sc = c->st.obs_c_stride; g.as = c->st.act_stride;
@@ -688,7 +690,7 @@ rslrl_status rslrl_ppo_update_steps(rslrl_ctx* c, int32_t max_steps, rslrl_updat
                 TRY(enqueue_gather(done_steps, 0, c->stream));
             }
             // ---- forward, heads, loss, backward ----------------------------------------------
-            const bool fused = c->umma && umma_has_step_chain(c->umma);
+            const bool fused = c->umma && umma_has_step_chain(c->umma) && !distill;
             HeadLossArgs hl{};
             if (fused) {
                 // row-local work in one kernel, then the weight-gradient partials
@@ -716,7 +718,7 @@ rslrl_status rslrl_ppo_update_steps(rslrl_ctx* c, int32_t max_steps, rslrl_updat
             hl.act_mb = c->act_mb[buf]; hl.mu_old = c->mu_old[buf]; hl.sigma_old = c->sigma_old[buf]; hl.as = c->st.act_stride;
             hl.logp_old = c->logp_old[buf]; hl.v_old = c->v_old[buf]; hl.ret = c->ret_mb[buf]; hl.adv = c->adv_mb[buf];
             hl.act_sign = c->sym.act_sign; hl.act_perm = c->sym.act_perm;
-            hl.Bmb = c->Bmb; hl.sym = pc.sym_enable;
+            hl.Bmb = c->Bmb; hl.sym = pc.sym_enable; hl.distill = distill ? 1 : 0;
             hl.h.clip = pc.clip; hl.h.value_clip = pc.value_clip; hl.h.value_coef = pc.value_coef;
             hl.h.entropy_coef = pc.entropy_coef; hl.h.sym_coef = pc.sym_coef; hl.h.alpha = c->mc.elu_alpha;
             hl.h.use_clipped_value_loss = pc.use_clipped_value_loss;
@@ -734,7 +736,7 @@ rslrl_status rslrl_ppo_update_steps(rslrl_ctx* c, int32_t max_steps, rslrl_updat
             r.grad = c->grad; r.P = c->P_dev; r.sumsq_partials = c->sumsq_partials;
             r.block_partials = c->block_partials; r.nblocks = hl.nblocks_used;
             r.off_ba = (int)ha.b_off; r.off_logstd = (int)c->logstd_off; r.off_bc = (int)hc.b_off; r.A = A;
-            r.entropy_coef = pc.entropy_coef; r.log_std = c->param + c->logstd_off; r.loss_sums = c->loss_sums;
+            r.entropy_coef = distill ? 0.f : pc.entropy_coef; r.log_std = c->param + c->logstd_off; r.loss_sums = c->loss_sums;
             if (fused) umma_fill_step_bias_sources(c->umma, &r);
             else if (c->umma) umma_fill_bias_sources(c->umma, &r, hl);
             CU(c, launch_reduce(r, c->stream));
@@ -745,7 +747,7 @@ rslrl_status rslrl_ppo_update_steps(rslrl_ctx* c, int32_t max_steps, rslrl_updat
             ad.inv_sym = 1.0f / ((float)c->Bmb * (float)A);
             ad.lr_io = c->lr_io; ad.step_io = c->step_io; ad.parity = c->parity;
             ad.lr_min = pc.lr_min; ad.lr_max = pc.lr_max; ad.lr_factor = pc.lr_factor; ad.desired_kl = pc.desired_kl;
-            ad.adaptive = pc.adaptive_lr; ad.max_norm = pc.max_grad_norm;
+            ad.adaptive = distill ? 0 : pc.adaptive_lr; ad.max_norm = pc.max_grad_norm;
             ad.b1 = pc.adam_b1; ad.b2 = pc.adam_b2; ad.eps = pc.adam_eps;
             ad.stats_row = c->stats_dev + (size_t)done_steps * 8;
             if (c->umma) umma_fill_cvt(c->umma, &ad);
@@ -784,7 +786,26 @@ rslrl_status rslrl_ppo_update_steps(rslrl_ctx* c, int32_t max_steps, rslrl_updat
     return RSLRL_OK;
 }
 
+rslrl_status rslrl_ppo_update_steps(rslrl_ctx* c, int32_t max_steps, rslrl_update_stats* h_stats) {
+    if (!c) return RSLRL_ERR_INVALID_ARG;
+    if (!c->gae_done) return fail(c, RSLRL_ERR_STATE, "rslrl_gae must precede rslrl_ppo_update");
+    return update_impl(c, max_steps, h_stats, nullptr);
+}
+
 rslrl_status rslrl_ppo_update(rslrl_ctx* c, rslrl_update_stats* h_stats) { return rslrl_ppo_update_steps(c, 0, h_stats); }
+
+rslrl_status rslrl_distill_update_steps(rslrl_ctx* c, const float* d_expert_actions, int32_t max_steps, rslrl_update_stats* h_stats) {
+    if (!c || !d_expert_actions) return RSLRL_ERR_INVALID_ARG;
+    if (!aligned4(d_expert_actions)) return fail(c, RSLRL_ERR_ALIGNMENT, "float buffers must be 4-byte aligned");
+    if (c->pc.sym_enable) return fail(c, RSLRL_ERR_UNSUPPORTED, "distillation with symmetry augmentation is not available");
+    if (c->step != c->st.T || c->act_pending)
+        return fail(c, RSLRL_ERR_STATE, "rslrl_distill_update needs exactly T = %d recorded steps (have %d)", c->st.T, c->step);
+    return update_impl(c, max_steps, h_stats, d_expert_actions);
+}
+
+rslrl_status rslrl_distill_update(rslrl_ctx* c, const float* d_expert_actions, rslrl_update_stats* h_stats) {
+    return rslrl_distill_update_steps(c, d_expert_actions, 0, h_stats);
+}
 
 // ------------------------------------------------------------------------ host variants
 rslrl_status rslrl_act_host(rslrl_ctx* c, const float* h_actor_obs, const float* h_critic_obs, float* h_actions_out) {

@@ -152,7 +152,7 @@ __global__ void __launch_bounds__(kThreads) head_loss_mma_kernel(const HeadLossA
             v[1] = quad_sum(v[1]) + bias_c;
             // ---- per-row loss terms (h = 0: row g, h = 1: row g + 8) ----------------------------
             float dmu[NT][4];
-            float lp[2] = {0.f, 0.f}, kl[2] = {0.f, 0.f};
+            float lp[2] = {0.f, 0.f}, kl[2] = {0.f, 0.f}, sq[2] = {0.f, 0.f};
 #pragma unroll
             for (int j = 0; j < NT; ++j)
 #pragma unroll
@@ -164,6 +164,7 @@ __global__ void __launch_bounds__(kThreads) head_loss_mma_kernel(const HeadLossA
                         const size_t r = h ? r1 : r0;
                         const int jj = h ? jc1 : jc0;
                         const float d = a.act_mb[r * a.as + i] - mu[j][e];
+                        if (a.distill) { sq[h] += d * d; dmu[j][e] = d; continue; }      // (a* - mu_i)^2
                         lp[h] += -(d * d) * 0.5f * ivar[j][c] - ls[j][c] - kHalfLog2Pi;
                         dmu[j][e] = d * ivar[j][c];                       // d logp / d mu_i
                         if (copy == 0) {
@@ -181,10 +182,12 @@ __global__ void __launch_bounds__(kThreads) head_loss_mma_kernel(const HeadLossA
                 lp[h] = quad_sum(lp[h]);
                 kl[h] = quad_sum(kl[h]);
                 if (copy == 0 && lead) s_kl += kl[h];
+                sq[h] = quad_sum(sq[h]);
+                if (a.distill && lead) s_surr += sq[h] / (float)A;      // the row's mean squared error
                 const float ratio = expf(lp[h] - logp_old[h]);
                 const float s1 = -adv[h] * ratio;
                 const float s2 = -adv[h] * fminf(fmaxf(ratio, 1.0f - a.h.clip), 1.0f + a.h.clip);
-                if (lead) s_surr += fmaxf(s1, s2);
+                if (lead && !a.distill) s_surr += fmaxf(s1, s2);
                 const bool inside = ratio >= 1.0f - a.h.clip && ratio <= 1.0f + a.h.clip;
                 dlogp[h] = (live && (inside || s1 > s2)) ? s1 * inv_R : 0.f;
                 const float e1 = (v[h] - ret[h]) * (v[h] - ret[h]);
@@ -192,14 +195,14 @@ __global__ void __launch_bounds__(kThreads) head_loss_mma_kernel(const HeadLossA
                 if (a.h.use_clipped_value_loss) {
                     const float vc = v_old[h] + fminf(fmaxf(v[h] - v_old[h], -a.h.value_clip), a.h.value_clip);
                     const float e2 = (vc - ret[h]) * (vc - ret[h]);
-                    if (lead) s_val += fmaxf(e1, e2);
+                    if (lead && !a.distill) s_val += fmaxf(e1, e2);
                     const bool vin = fabsf(v[h] - v_old[h]) <= a.h.value_clip;
                     d = (vin || e1 > e2) ? 2.0f * (v[h] - ret[h]) : 0.f;
                 } else {
-                    if (lead) s_val += e1;
+                    if (lead && !a.distill) s_val += e1;
                     d = 2.0f * (v[h] - ret[h]);
                 }
-                dv[h] = live ? d * a.h.value_coef * inv_R : 0.f;
+                dv[h] = (live && !a.distill) ? d * a.h.value_coef * inv_R : 0.f;      // no critic term when distilling
                 if (lead) s_dbc += dv[h];
             }
             // ---- dL/dmu, dL/dlog_std, symmetry ------------------------------------------------
@@ -214,8 +217,8 @@ __global__ void __launch_bounds__(kThreads) head_loss_mma_kernel(const HeadLossA
                     float gmu = 0.f;
                     if (i < A && live) {
                         const float dlp = dmu[j][e];
-                        s_dls[j][c] += dlogp[h] * (dlp * dlp * var[j][c] - 1.0f);
-                        gmu = dlogp[h] * dlp;
+                        if (!a.distill) s_dls[j][c] += dlogp[h] * (dlp * dlp * var[j][c] - 1.0f);
+                        gmu = a.distill ? -2.0f * dlp * inv_R / (float)A : dlogp[h] * dlp;
                         if (copy == 1) {
                             const float diff = mu[j][e] - a.act_sign[i] * mu_w[(g + 8 * h) * (AP + 1) + a.act_perm[i]];
                             s_sym += diff * diff;

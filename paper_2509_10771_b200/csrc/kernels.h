@@ -150,6 +150,8 @@ struct HeadLossArgs {
     const float* logp_old; const float* v_old; const float* ret; const float* adv;
     const float* act_sign; const int* act_perm;       // mirror of actions (null when sym off)
     int Bmb; int sym;
+    int distill;                    // 1: act_mb holds expert actions and the loss is the mean squared error between the
+                                    // policy mean and them (no critic, log_std, KL terms); its row sum lands in LS_SURR
     LossHyper h;
     // outputs
     float* dmu; int lddmu;          // [R][round4(A)]   fp32

@@ -296,13 +296,18 @@ __global__ void __launch_bounds__(kHLThreads) head_loss_kernel(const HeadLossArg
             v += hp.bc[0];
             // ---- log-density, KL (own actions, then two shuffles) --------------------------------
             float dmu[AQ];
-            float lp = 0.f, kl = 0.f;
+            float lp = 0.f, kl = 0.f, sq = 0.f;
 #pragma unroll
             for (int s = 0; s < AQ; ++s) {
                 const int i = 16 * (s >> 2) + 4 * qt + (s & 3);
                 dmu[s] = 0.f;
                 if (i < A) {
                     const float d = a.act_mb[(size_t)r * a.as + i] - mu[s];
+                    if (a.distill) {
+                        sq += d * d;                                    // (a* - mu_i)^2
+                        dmu[s] = d;
+                        continue;
+                    }
                     lp += -(d * d) * 0.5f * ivar[s] - ls[s] - kHalfLog2Pi;
                     dmu[s] = d * ivar[s];                               // d logp / d mu_i
                     if (copy == 0) {
@@ -315,11 +320,15 @@ __global__ void __launch_bounds__(kHLThreads) head_loss_kernel(const HeadLossArg
             lp += __shfl_xor_sync(qmask, lp, 1); lp += __shfl_xor_sync(qmask, lp, 2);
             kl += __shfl_xor_sync(qmask, kl, 1); kl += __shfl_xor_sync(qmask, kl, 2);
             if (copy == 0 && lead) s_kl += kl;
+            if (a.distill) {
+                sq += __shfl_xor_sync(qmask, sq, 1); sq += __shfl_xor_sync(qmask, sq, 2);
+                if (lead) s_surr += sq / (float)A;                      // the row's mean squared error
+            }
             // ---- surrogate ---------------------------------------------------------------
             const float ratio = expf(lp - logp_old);
             const float s1 = -adv * ratio;
             const float s2 = -adv * fminf(fmaxf(ratio, 1.0f - a.h.clip), 1.0f + a.h.clip);
-            if (lead) s_surr += fmaxf(s1, s2);
+            if (lead && !a.distill) s_surr += fmaxf(s1, s2);
             const bool inside = ratio >= 1.0f - a.h.clip && ratio <= 1.0f + a.h.clip;
             const float dlogp = (inside || s1 > s2) ? s1 * inv_R : 0.f;
             // ---- value -------------------------------------------------------------------
@@ -328,14 +337,15 @@ __global__ void __launch_bounds__(kHLThreads) head_loss_kernel(const HeadLossArg
             if (a.h.use_clipped_value_loss) {
                 const float vc = v_old + fminf(fmaxf(v - v_old, -a.h.value_clip), a.h.value_clip);
                 const float e2 = (vc - ret) * (vc - ret);
-                if (lead) s_val += fmaxf(e1, e2);
+                if (lead && !a.distill) s_val += fmaxf(e1, e2);
                 const bool vin = fabsf(v - v_old) <= a.h.value_clip;
                 dv = (vin || e1 > e2) ? 2.0f * (v - ret) : 0.f;
             } else {
-                if (lead) s_val += e1;
+                if (lead && !a.distill) s_val += e1;
                 dv = 2.0f * (v - ret);
             }
             dv *= a.h.value_coef * inv_R;
+            if (a.distill) dv = 0.f;                                    // the critic takes no part
             if (lead) s_dbc += dv;
             // ---- dL/dmu, dL/dlog_std, symmetry -------------------------------------------
             if (copy == 1) __syncwarp(qmask);                           // mu of the original row is in mu_row
@@ -344,8 +354,8 @@ __global__ void __launch_bounds__(kHLThreads) head_loss_kernel(const HeadLossArg
                 const int i = 16 * (s >> 2) + 4 * qt + (s & 3);
                 if (i < A) {
                     const float dlp_dmu = dmu[s];                       // (a - mu) / sigma^2
-                    s_dls[s] += dlogp * (dlp_dmu * dlp_dmu * __expf(2.0f * ls[s]) - 1.0f);
-                    float g = dlogp * dlp_dmu;
+                    if (!a.distill) s_dls[s] += dlogp * (dlp_dmu * dlp_dmu * __expf(2.0f * ls[s]) - 1.0f);
+                    float g = a.distill ? -2.0f * dmu[s] * inv_R / (float)A : dlogp * dlp_dmu;
                     if (copy == 1) {
                         const float diff = mu[s] - a.act_sign[i] * mu_row[a.act_perm[i]];
                         s_sym += diff * diff;

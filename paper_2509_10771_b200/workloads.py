@@ -190,6 +190,13 @@ def make_rollout_inputs(w: Workload, seed: Optional[int] = None) -> Dict[str, np
     }
 
 
+def make_expert_actions(w: Workload, seed: Optional[int] = None) -> np.ndarray:
+    """Stand-in for an expert policy's relabelling of a student rollout: ``[T][N][A]`` float32 ~ N(0,1)
+    (stream 9 of the workload's seed)."""
+    seed = w.seed if seed is None else seed
+    return _rng(seed, 9).standard_normal((w.num_steps, w.num_envs, w.num_actions), dtype=np.float32)
+
+
 def param_layout(w: Workload) -> List[Tuple[str, int, Tuple[int, ...]]]:
     """Flat parameter order: (name, offset, shape).
 
