@@ -659,6 +659,7 @@ static rslrl_status update_impl(rslrl_ctx* c, int32_t max_steps, rslrl_update_st
     };
     // With a gather stream, minibatch s+1 is gathered into the other input set while minibatch s is
     // worked on: the gather waits for the kernels that read that set two steps ago, the step for its gather.
+    if (distill && c->umma) CU(c, umma_zero_critic_gradients(c->umma));
     const bool overlap = c->side != nullptr;
     if (overlap) {
         CU(c, cudaEventRecord(c->ev_ready, c->stream));           // advantages and returns are in storage
@@ -711,7 +712,7 @@ static rslrl_status update_impl(rslrl_ctx* c, int32_t max_steps, rslrl_update_st
                 hl.dZa = c->up_dz[0][c->actor.nl - 2]; hl.lddza = hl.ldha;
                 hl.dZc = c->up_dz[1][c->critic.nl - 2]; hl.lddzc = hl.ldhc;
             } else {
-                CU(c, umma_update_forward(c->umma, buf));
+                CU(c, umma_update_forward(c->umma, buf, distill));
                 umma_head_loss_targets(c->umma, &hl);
             }
             hl.hp = hp_base;
@@ -727,7 +728,7 @@ static rslrl_status update_impl(rslrl_ctx* c, int32_t max_steps, rslrl_update_st
             CU(c, launch_head_loss(hl, c->stream));
             // ---- backward ---------------------------------------------------------------
             if (c->prec == RSLRL_FP32) TRY(backward_fp32(c));
-            else CU(c, umma_update_backward(c->umma, hl.colsum_written != 0, buf));
+            else CU(c, umma_update_backward(c->umma, hl.colsum_written != 0, buf, distill));
             }
             if (overlap) CU(c, cudaEventRecord(c->ev_consumed[buf], c->stream));   // this input set may be refilled
             // ---- reduce, clip, adaptive lr, Adam ------------------------------------------

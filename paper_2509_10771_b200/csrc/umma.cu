@@ -743,6 +743,8 @@ struct UmmaEngine {
     std::vector<TcParams> act_fwd, act_fwd_critic, upd_fwd, upd_dgrad, upd_wgrad;
     // the launches that read the minibatch observations, once more for the second input buffer
     std::vector<TcParams> upd_fwd_alt, upd_wgrad_alt;
+    // forward and data-gradient launches of the actor alone (the distillation step trains no critic)
+    std::vector<TcParams> fwd_actor[2], dgrad_actor;
     // fused forward (one launch for all hidden layers) where the widths allow it, else empty
     std::vector<ChainParams> chain_act, chain_act_critic;
     ColsumBatch colsum{}, colsum_rest{};         // all layers the epilogue does not cover / those minus the last ones
@@ -779,6 +781,20 @@ void finish_params(TcParams& P, float alpha, int* error) {
     P.total_items = items;
     P.alpha = alpha;
     P.error = error;
+}
+
+// The problems of one net out of a launch's parameters, as a launch of their own (no items if there are none).
+TcParams only_net(const TcParams& P, int ni) {
+    TcParams Q;
+    memset(&Q, 0, sizeof Q);
+    for (int i = 0; i < P.count; ++i) {
+        if (P.p[i].net_id != ni) continue;
+        const int j = Q.count++;
+        Q.tmA[j] = P.tmA[i]; Q.tmB[j] = P.tmB[i]; Q.tmOut[j] = P.tmOut[i]; Q.tmAux[j] = P.tmAux[i];
+        Q.p[j] = P.p[i];
+    }
+    finish_params(Q, P.alpha, P.error);
+    return Q;
 }
 
 // D[rows x width_out] = A[rows x k] * B[width_out x k]^T, both operands contraction-major.
@@ -1113,6 +1129,7 @@ UmmaEngine* umma_create(const UmmaSetup& s, std::string* err) {
             TcProblem& p = P.p[P.count - 1];
             p.out16 = e->dz[ni][l - 1]; p.ld_out = e->pw[ni][l - 1];
             p.aux16 = e->h[ni][l - 1]; p.ld_aux = e->pw[ni][l - 1];
+            p.net_id = ni; p.layer_id = l - 1;
             if (e->n_sources < kMaxBiasSources) {     // beyond that the column-sum kernel takes the layer
                 e->n_sources++;
                 e->n_slots = 4 * p.m_tiles;
@@ -1172,6 +1189,9 @@ UmmaEngine* umma_create(const UmmaSetup& s, std::string* err) {
             const int ni = P.p[i].net_id;
             if (!make_tmap(&P.tmA[i], e->x16_alt[ni], R, e->kp[ni], e->kp[ni], 64, BLOCK_K)) return bail("tensor map encoding failed");
         }
+    for (const TcParams& P : e->upd_fwd) e->fwd_actor[0].push_back(only_net(P, 0));
+    for (const TcParams& P : e->upd_fwd_alt) e->fwd_actor[1].push_back(only_net(P, 0));
+    for (const TcParams& P : e->upd_dgrad) e->dgrad_actor.push_back(only_net(P, 0));
     // ---- bias-gradient partials of the last hidden layers, written by the head/loss kernel ----
     if (e->n_sources + 2 <= kMaxBiasSources)
         for (int ni = 0; ni < 2; ++ni)
@@ -1329,8 +1349,8 @@ void umma_gather_targets(UmmaEngine* e, GatherArgs* g, int buf) {
 
 bool umma_two_input_buffers(const UmmaEngine* e) { return e->step == nullptr; }
 
-cudaError_t umma_update_forward(UmmaEngine* e, int buf) {
-    for (const TcParams& P : buf ? e->upd_fwd_alt : e->upd_fwd) {
+cudaError_t umma_update_forward(UmmaEngine* e, int buf, bool actor_only) {
+    for (const TcParams& P : actor_only ? e->fwd_actor[buf] : buf ? e->upd_fwd_alt : e->upd_fwd) {
         cudaError_t err = launch_tc<TC_FWD>(P, e->num_sms, e->s.stream);
         if (err != cudaSuccess) return err;
     }
@@ -1347,9 +1367,24 @@ void umma_head_loss_targets(UmmaEngine* e, HeadLossArgs* a) {
     a->colsum_a = e->head_slots[0]; a->colsum_c = e->head_slots[1];
 }
 
-cudaError_t umma_update_backward(UmmaEngine* e, bool last_bias_done, int buf) {
+cudaError_t umma_zero_critic_gradients(UmmaEngine* e) {
+    // what the critic's data-gradient launches would write: dL/dz of its hidden layers below the last one
+    // (the head/loss kernel writes the last) and the bias-gradient partials of their epilogues
+    const int R = e->s.R;
+    for (int l = 0; l + 1 < e->nh[1]; ++l) {
+        cudaError_t err = cudaMemsetAsync(e->dz[1][l], 0, (size_t)R * e->pw[1][l] * sizeof(__nv_bfloat16), e->s.stream);
+        if (err != cudaSuccess) return err;
+        if (e->bias_slots[1][l]) {
+            err = cudaMemsetAsync(e->bias_slots[1][l], 0, (size_t)e->n_slots * e->pw[1][l] * sizeof(float), e->s.stream);
+            if (err != cudaSuccess) return err;
+        }
+    }
+    return cudaSuccess;
+}
+
+cudaError_t umma_update_backward(UmmaEngine* e, bool last_bias_done, int buf, bool actor_only) {
     cudaError_t err;
-    for (const TcParams& P : e->upd_dgrad) {
+    for (const TcParams& P : actor_only ? e->dgrad_actor : e->upd_dgrad) {
         err = launch_tc<TC_DGRAD>(P, e->num_sms, e->s.stream);
         if (err != cudaSuccess) return err;
     }

@@ -51,13 +51,17 @@ cudaError_t umma_act_forward(UmmaEngine* e, const float* d_obs_a, const float* d
 // can run while the current one is worked on (not with the fused step kernel, which has one).
 void umma_gather_targets(UmmaEngine* e, GatherArgs* g, int buf);
 bool umma_two_input_buffers(const UmmaEngine* e);
-cudaError_t umma_update_forward(UmmaEngine* e, int buf);
+// actor_only (distillation): the critic's launches are left out; umma_zero_critic_gradients, once before the
+// first such step, zeroes what its data-gradient launches would have written, so that the weight-gradient
+// launch (which still covers both nets) yields a zero critic gradient.
+cudaError_t umma_update_forward(UmmaEngine* e, int buf, bool actor_only);
+cudaError_t umma_zero_critic_gradients(UmmaEngine* e);
 // Point the head/loss kernel at the engine's last hidden activations and dZ buffers.
 void umma_head_loss_targets(UmmaEngine* e, HeadLossArgs* a);
 // Data gradients, weight-gradient partials and bias-gradient partials of all hidden layers
 // and heads, from the dZ / d_head buffers the head/loss kernel filled.  last_bias_done: the
 // head/loss kernel already produced the bias-gradient partials of the last hidden layers.
-cudaError_t umma_update_backward(UmmaEngine* e, bool last_bias_done, int buf);
+cudaError_t umma_update_backward(UmmaEngine* e, bool last_bias_done, int buf, bool actor_only);
 // The fused row-local step kernel (forward, heads, loss, data gradients in one launch) exists when
 // the minibatch has no mirrored rows and the widths fit.  umma_step_chain runs it (nblocks: rows of
 // loss.block_partials it writes), umma_update_wgrad the weight-gradient partials after it, and

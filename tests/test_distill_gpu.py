@@ -117,3 +117,38 @@ def test_distillation_call_order_and_arguments():
     assert ctx.storage_view().step == 0
     ctx.destroy()
     torch.cuda.synchronize()
+
+
+@pytest.mark.parametrize("precision", [FP32, BF16])
+def test_distillation_after_a_ppo_update_leaves_the_critic_alone(precision):
+    """A PPO iteration first (it leaves critic gradients in the work buffers), then a distillation step
+    from the optimiser state the PPO update ended with: the critic's gradient must be exactly zero and the
+    step must match the oracle started from the same state."""
+    import torch
+    from paper_2509_10771_b200 import binding
+    from parity_utils import gpu_rollout
+    w = CASES["rough"]
+    theta, inputs = WL.make_params(w), WL.make_rollout_inputs(w)
+    ctx = binding.Context(w, precision=precision)
+    ctx.set_params(theta)
+    gpu_rollout(ctx, w, inputs)
+    ctx.ppo_update()
+    theta1 = ctx.get_params().astype(np.float64)
+    m1, v1 = ctx.get_adam()
+    c1 = ctx.get_counters()
+    inputs2 = WL.make_rollout_inputs(w, seed=w.seed + 1)
+    expert = WL.make_expert_actions(w, seed=w.seed + 1)
+    _student_rollout(ctx, w, inputs2)
+    stats = ctx.distill_update(_expert_on_device(ctx, w, expert), max_steps=1)
+    state = O.OptimState(theta1, float(c1.lr))
+    state.m, state.v, state.step = m1.astype(np.float64), v1.astype(np.float64), int(c1.adam_step)
+    ref = O.distill_update(state, dims_of(w), inputs2["obs_actor"], expert, w, seed=w.seed, iteration=int(c1.iteration),
+                           max_steps=1)
+    tol = 1e-4 if precision == FP32 else 1e-2
+    assert_close(stats["first_surrogate"], ref[0]["loss"], tol, "loss")
+    g = ctx.get_grads()
+    n_actor = sum(i * o + o for i, o in w.layer_dims("actor"))
+    assert np.all(g[n_actor:] == 0.0)
+    assert rel_l2(g, ref[0]["grad"]) < (1e-4 if precision == FP32 else 1e-2)
+    ctx.destroy()
+    torch.cuda.synchronize()
