@@ -28,6 +28,10 @@ denote, written out in numpy float64 with no blocking, fusion or reordering:
                              with the expert's actions, and the student's mean is regressed on them
                              (mean squared error, the paper names no loss) over the same keyed
                              minibatches, with global-norm clipping and Adam, no learning-rate rule
+* ``rnd_reward`` / ``rnd_loss_and_grads`` / ``rnd_update`` -- the curiosity bonus of "Auxiliary
+                             Techniques": random network distillation (Burda et al. 2019) on a subset of
+                             the state: r_int = mean_j (f_j(s) - g_j(s))^2 with a fixed random target g and
+                             a trained predictor f, and the predictor's regression step
 * ``philox4x32_10``, ``gaussian_noise``, ``feistel_permutation`` -- the counter-based random
                              streams the method draws from (Salmon et al., SC'11), so that a
                              second implementation can reproduce noise and shuffles bit for bit.
@@ -565,6 +569,68 @@ def distill_update(state: OptimState, dims, obs_actor: np.ndarray, expert_action
                                                       state.lr, hp.adam_b1, hp.adam_b2, hp.adam_eps)
             st = {"loss": stats["loss"], "grad": g, "grad_norm": g_norm, "lr": state.lr}
             out.append(st)
+    return out
+
+
+# ======================================================================================
+# Random network distillation on a subset of the state ("Auxiliary Techniques": a curiosity-driven
+# intrinsic reward based on RND, computed "using only a subset of the full state").  Following Burda
+# et al. 2019: a fixed, randomly initialised target MLP g and a predictor MLP f of the same shape read
+# s = o[idx]; the bonus is the predictor's squared error, the predictor is trained to reduce it.
+# Readings where the paper is silent: the error is averaged over the E outputs; the bonus enters the
+# stored reward as r + w * r_int; the predictor has its own Adam (no clipping, fixed learning rate)
+# and sees the same keyed minibatches as the policy update.
+# ======================================================================================
+def unpack_mlp(flat: np.ndarray, dims: Sequence[Tuple[int, int]]):
+    """[(W[in][out], b), ...] from the flat order W1, b1, W2, b2, ..."""
+    flat = np.asarray(flat, dtype=F64)
+    off, layers = 0, []
+    for fi, fo in dims:
+        W = flat[off:off + fi * fo].reshape(fi, fo); off += fi * fo
+        b = flat[off:off + fo]; off += fo
+        layers.append((W, b))
+    assert off == flat.size, (off, flat.size)
+    return layers
+
+
+def rnd_reward(theta_f: np.ndarray, theta_g: np.ndarray, dims, obs: np.ndarray, idx: np.ndarray, alpha: float):
+    """r_int[row] = mean_j (f_j(s) - g_j(s))^2 with s = obs[row][idx]; also returns f(s), g(s) and f's activations."""
+    s = np.asarray(obs, dtype=F64)[:, np.asarray(idx)]
+    f, hs = mlp_forward(s, unpack_mlp(theta_f, dims), alpha)
+    g, _ = mlp_forward(s, unpack_mlp(theta_g, dims), alpha)
+    return ((f - g) ** 2).mean(axis=1), f, g, hs
+
+
+def rnd_loss_and_grads(theta_f: np.ndarray, theta_g: np.ndarray, dims, obs: np.ndarray, idx: np.ndarray, alpha: float):
+    """L = mean over rows of r_int, and dL/dtheta_f (flat, same order as theta_f)."""
+    r, f, g, hs = rnd_reward(theta_f, theta_g, dims, obs, idx, alpha)
+    B, E = f.shape
+    d_out = 2.0 * (f - g) / (B * E)
+    grads = mlp_backward(d_out, hs, unpack_mlp(theta_f, dims), alpha)
+    flat = np.concatenate([x.ravel() for W, b in grads for x in (W, b)])
+    return float(r.mean()), flat
+
+
+def rnd_update(state: OptimState, theta_g: np.ndarray, dims, obs: np.ndarray, idx: np.ndarray, hp, seed: int,
+               iteration: int, max_steps: Optional[int] = None) -> List[Dict]:
+    """Predictor training over obs[B][D]: hp.epochs x hp.minibatches steps over ``feistel_permutation`` chunks,
+    Adam on ``state`` (the predictor's parameters and moments) with the fixed learning rate state.lr."""
+    B = obs.shape[0]
+    if B % hp.minibatches:
+        raise ValueError("batch not divisible by the number of minibatches")
+    rows_per = B // hp.minibatches
+    out = []
+    for e in range(hp.epochs):
+        perm = feistel_permutation(seed, iteration, e, B)
+        for k in range(hp.minibatches):
+            if max_steps is not None and len(out) >= max_steps:
+                return out
+            rows = perm[k * rows_per:(k + 1) * rows_per]
+            L, g = rnd_loss_and_grads(state.theta, theta_g, dims, obs[rows], idx, hp.elu_alpha)
+            state.step += 1
+            state.theta, state.m, state.v = adam_step(state.theta, g, state.m, state.v, state.step, state.lr,
+                                                      hp.adam_b1, hp.adam_b2, hp.adam_eps)
+            out.append({"loss": L, "grad": g})
     return out
 
 

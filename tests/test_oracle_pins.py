@@ -567,3 +567,82 @@ def test_distill_update_loop_matches_torch_reference_loop():
             opt.step()
             assert steps[e * 2 + k]["loss"] == pytest.approx(L.item(), rel=1e-9)
     assert np.allclose(state.theta, p.detach().numpy(), rtol=1e-9, atol=1e-12)
+
+
+# --------------------------------------------------------------------------------------
+# random network distillation on a state subset (paper, "Auxiliary Techniques")
+# --------------------------------------------------------------------------------------
+def _rnd_problem(seed=11, B=28, D=9, idx=(7, 1, 4, 2), hidden=(6, 5), E=3):
+    rng = np.random.default_rng(seed)
+    dims = list(zip([len(idx), *hidden], [*hidden, E]))
+    P = sum(i * o + o for i, o in dims)
+    return rng.normal(0, 0.6, P), rng.normal(0, 0.6, P), dims, rng.normal(size=(B, D)), np.array(idx)
+
+
+def _torch_mlp(p, dims, x, alpha):
+    off = 0
+    for li, (fi, fo) in enumerate(dims):
+        W = p[off:off + fi * fo].reshape(fi, fo); off += fi * fo
+        b = p[off:off + fo]; off += fo
+        x = x @ W + b
+        if li < len(dims) - 1:
+            x = torch.nn.functional.elu(x, alpha=alpha)
+    return x
+
+
+def test_rnd_reward_and_gradient_match_torch():
+    tf, tg, dims, obs, idx = _rnd_problem()
+    r, f, g, _ = O.rnd_reward(tf, tg, dims, obs, idx, 1.0)
+    p = torch.tensor(tf, dtype=torch.float64, requires_grad=True)
+    s = torch.as_tensor(obs[:, idx])
+    ft = _torch_mlp(p, dims, s, 1.0)
+    gt = _torch_mlp(torch.as_tensor(tg), dims, s, 1.0)
+    rt = ((ft - gt) ** 2).mean(dim=1)
+    assert np.allclose(r, rt.detach().numpy(), rtol=1e-12, atol=1e-15)
+    L, grad = O.rnd_loss_and_grads(tf, tg, dims, obs, idx, 1.0)
+    rt.mean().backward()
+    assert L == pytest.approx(rt.mean().item(), rel=1e-12)
+    assert np.allclose(grad, p.grad.numpy(), rtol=1e-9, atol=1e-13)
+
+
+def test_rnd_reads_only_the_subset_and_vanishes_for_equal_nets():
+    tf, tg, dims, obs, idx = _rnd_problem(13)
+    r0 = O.rnd_reward(tf, tg, dims, obs, idx, 1.0)[0]
+    other = [c for c in range(obs.shape[1]) if c not in idx]
+    obs2 = obs.copy(); obs2[:, other] += 5.0               # columns outside the subset do not matter
+    assert np.array_equal(O.rnd_reward(tf, tg, dims, obs2, idx, 1.0)[0], r0)
+    obs3 = obs.copy(); obs3[:, idx[0]] += 0.5              # one inside does
+    assert not np.allclose(O.rnd_reward(tf, tg, dims, obs3, idx, 1.0)[0], r0)
+    assert np.all(r0 >= 0.0)
+    L, grad = O.rnd_loss_and_grads(tf, tf, dims, obs, idx, 1.0)     # predictor == target
+    assert L == 0.0 and np.all(grad == 0.0)
+
+
+def test_rnd_gradient_matches_central_finite_differences():
+    tf, tg, dims, obs, idx = _rnd_problem(17, B=12)
+    _, grad = O.rnd_loss_and_grads(tf, tg, dims, obs, idx, 1.0)
+    for i in np.random.default_rng(1).integers(0, tf.size, 30):
+        e = np.zeros_like(tf); e[i] = 1e-6
+        fd = (O.rnd_loss_and_grads(tf + e, tg, dims, obs, idx, 1.0)[0] - O.rnd_loss_and_grads(tf - e, tg, dims, obs, idx, 1.0)[0]) / 2e-6
+        assert grad[i] == pytest.approx(fd, rel=2e-5, abs=1e-9), i
+
+
+def test_rnd_update_loop_matches_torch_reference_loop():
+    tf, tg, dims, obs, idx = _rnd_problem(19, B=32)
+    h = hp(epochs=2, minibatches=4, lr=3e-3)
+    state = O.OptimState(tf.copy(), h.lr)
+    steps = O.rnd_update(state, tg, dims, obs, idx, h, seed=5, iteration=2)
+    assert len(steps) == 8 and state.step == 8
+    p = torch.tensor(tf, dtype=torch.float64, requires_grad=True)
+    opt = torch.optim.Adam([p], lr=h.lr)
+    s_all = torch.as_tensor(obs[:, idx]); tgt = torch.as_tensor(tg)
+    k = 0
+    for e in range(2):
+        perm = O.feistel_permutation(5, 2, e, 32)
+        for c in range(4):
+            rows = torch.as_tensor(perm[c * 8:(c + 1) * 8].astype(np.int64))
+            opt.zero_grad()
+            L = ((_torch_mlp(p, dims, s_all[rows], 1.0) - _torch_mlp(tgt, dims, s_all[rows], 1.0)) ** 2).mean()
+            L.backward(); opt.step()
+            assert steps[k]["loss"] == pytest.approx(L.item(), rel=1e-9); k += 1
+    assert np.allclose(state.theta, p.detach().numpy(), rtol=1e-9, atol=1e-12)
