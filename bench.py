@@ -446,14 +446,94 @@ def run_distill(args):
     ctx.destroy()
 
 
+def run_rnd(args):
+    """--task rnd: random network distillation on a state subset over one rollout's transitions, one GPU: the
+    intrinsic reward of all T x N rows (rslrl_rnd_reward) followed by the predictor's training loop
+    (rslrl_rnd_update, the workload's epochs x minibatches).  Prints its own JSON line."""
+    import torch
+    from paper_2509_10771_b200 import binding, build
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device: the path has no CPU fallback")
+    torch.cuda.set_device(0)
+    build.build()
+    w = WORKLOAD
+    T, N = w.num_steps, w.num_envs
+    B = T * N
+    dev = torch.device("cuda", 0)
+    stream = torch.cuda.current_stream()
+    setup = WL.make_rnd_setup(w, num_idx=48, hidden=(256, 128, 64), embed_dim=32)
+    obs = WL.make_rollout_inputs(w)["obs_actor"][:T].reshape(B, w.actor_obs_dim)
+    d_obs = torch.from_numpy(obs).to(dev)
+    d_rew = torch.zeros(B, device=dev)
+    rnd = binding.Rnd(w.actor_obs_dim, setup["idx"], setup["hidden"], setup["embed_dim"], max_rows=B, lr=1e-3,
+                      stream=stream.cuda_stream)
+    rnd.set_params(setup["predictor"], setup["target"])
+    flush_buf = torch.empty(256 << 20, dtype=torch.uint8, device=dev)
+    it = [0]
+
+    def iteration():
+        rnd.reward(d_obs, B, w.actor_obs_dim, weight=0.1, d_rewards_inout=d_rew)
+        rnd.update(d_obs, B, w.actor_obs_dim, w.epochs, w.minibatches, seed=w.seed, iteration=it[0], want_loss=False)
+        it[0] += 1
+
+    for _ in range(max(args.warmup, 3)):
+        iteration()
+    torch.cuda.synchronize()
+    evs = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(args.steps)]
+    for a, b in evs:
+        flush_buf.zero_()
+        a.record(stream)
+        iteration()
+        b.record(stream)
+    torch.cuda.synchronize()
+    ms = sum(a.elapsed_time(b) for a, b in evs)
+    binding.profile_enable(True)
+    binding.profile_report()
+    for _ in range(min(args.steps, 10)):
+        iteration()
+    torch.cuda.synchronize()
+    prof = binding.profile_report()
+    binding.profile_enable(False)
+    total = sum(v["ms"] for v in prof.values()) or 1.0
+    shares = {k: {"launches": v["launches"], "ms": round(v["ms"], 3), "share": round(v["ms"] / total, 4)}
+              for k, v in sorted(prof.items(), key=lambda kv: -kv[1]["ms"])}
+    # FP32 multiply-adds of one iteration: 2 nets forward on B rows, then per training row 2 forwards + 2 backward products
+    mac = sum(fi * fo for fi, fo in setup["dims"])
+    flops = 2.0 * mac * (2 * B + w.epochs * B * (2 + 2))
+    from types import SimpleNamespace
+    from oracle import ppo_oracle as O
+    rows_s = ORACLE_SAMPLE_ENVS * T
+    hp = SimpleNamespace(epochs=w.epochs, minibatches=w.minibatches, elu_alpha=1.0, adam_b1=0.9, adam_b2=0.999, adam_eps=1e-8)
+    state = O.OptimState(setup["predictor"].astype(np.float64), 1e-3)
+    t0 = time.perf_counter()
+    O.rnd_reward(state.theta, setup["target"], setup["dims"], obs[:rows_s], setup["idx"], 1.0)
+    O.rnd_update(state, setup["target"], setup["dims"], obs[:rows_s], setup["idx"], hp, seed=w.seed, iteration=0)
+    cpu_s = time.perf_counter() - t0
+    line = {
+        "metric": "random network distillation transitions/s", "value": B * args.steps / (ms * 1e-3), "unit": UNIT, "n_gpus": 1,
+        "steps": args.steps, "warmup": max(args.warmup, 3), "ms_per_step": ms / args.steps, "higher_is_better": True,
+        "dtype": "f32", "data": "synthetic",
+        "config": {"workload": w.name, "task": "rnd", "num_envs": N, "num_steps": T, "epochs": w.epochs,
+                   "minibatches": w.minibatches, "num_idx": 48, "hidden": [256, 128, 64], "embed_dim": 32,
+                   "l2": "256 MiB buffer written between timed steps"},
+        "fp32_tflops": flops / (ms / args.steps * 1e-3) / 1e12,
+        "kernel_shares": shares,
+        "cpu_baseline": {"value": rows_s / cpu_s, "unit": UNIT, "cores": blas_threads(), "kind": "oracle",
+                         "sample": f"the oracle's reward and predictor training on {ORACLE_SAMPLE_ENVS} of the {N} environments"},
+    }
+    print(json.dumps(line), flush=True)
+    rnd.destroy()
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
     ap.add_argument("--steps", type=int, default=50)
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
-    ap.add_argument("--task", default="ppo", choices=["ppo", "distill"],
-                    help="ppo: the learn iteration the metric is quoted on (default); distill: the distillation iteration")
+    ap.add_argument("--task", default="ppo", choices=["ppo", "distill", "rnd"],
+                    help="ppo: the learn iteration the metric is quoted on (default); distill: the distillation iteration; "
+                         "rnd: random network distillation over one rollout")
     args = ap.parse_args()
     rank = int(os.environ.get("RANK", "0"))
     world = int(os.environ.get("WORLD_SIZE", "1"))
@@ -463,6 +543,9 @@ def main():
     elif args.task == "distill":
         if rank == 0:
             run_distill(args)
+    elif args.task == "rnd":
+        if rank == 0:
+            run_rnd(args)
     else:
         run_ours(args, rank, world, local_rank)
 

@@ -279,6 +279,63 @@ rslrl_status rslrl_gae_scan_static(const float *d_rewards, const float *d_values
                                    float gamma, float lam, int32_t normalize, int32_t unbiased,
                                    float adv_eps, void *cuda_stream);
 
+/* ---------------------------------------------------------------------------------------------
+ * Random network distillation on a subset of the state (paper: "Auxiliary Techniques", the
+ * curiosity-driven intrinsic reward computed on selected states only).
+ *
+ * Two MLPs of the same shape read s = o[idx] (num_idx selected entries of an observation row):
+ * a target g with fixed random weights and a predictor f.  Intrinsic reward of a row:
+ *   r_int = (1/E) sum_j (f_j(s) - g_j(s))^2          (E = embed_dim)
+ * rslrl_rnd_reward adds weight * r_int to a reward vector; rslrl_rnd_update regresses f on g
+ * (loss = mean over the minibatch rows of r_int) with Adam at a fixed learning rate, over the
+ * same kind of keyed minibatches as rslrl_ppo_update.  All arithmetic is FP32.  (Observation
+ * normalisation and reward-weight schedules, which the paper's library offers around this, are
+ * left to the caller.)
+ *
+ * An rslrl_rnd owns its parameters, Adam moments and work buffers (device memory); calls on one
+ * object are not thread-safe; all work is enqueued on the stream given at creation.
+ * Parameter vectors (host, float32) are in the order W1[in][out], b1, W2, b2, ... for the
+ * layers num_idx -> hidden[0] -> ... -> embed_dim; hidden layers use ELU(alpha). */
+typedef struct rslrl_rnd rslrl_rnd;
+
+typedef struct {
+    int32_t obs_dim;                    /* entries of an observation row; idx values are < obs_dim   */
+    int32_t num_idx;                    /* 1..obs_dim                                                */
+    const int32_t *h_idx;               /* [num_idx] host; copied                                    */
+    int32_t num_hidden;                 /* 1..RSLRL_MAX_HIDDEN                                       */
+    int32_t hidden[RSLRL_MAX_HIDDEN];
+    int32_t embed_dim;                  /* E >= 1                                                    */
+    float   elu_alpha;
+    int32_t max_rows;                   /* largest `rows` of rslrl_rnd_reward and largest minibatch  */
+    float   lr, adam_b1, adam_b2, adam_eps;
+} rslrl_rnd_cfg;
+
+size_t       rslrl_rnd_num_params(const rslrl_rnd_cfg *cfg);      /* of one net; 0 if cfg is invalid */
+rslrl_status rslrl_rnd_create(const rslrl_rnd_cfg *cfg, void *cuda_stream, rslrl_rnd **out);
+rslrl_status rslrl_rnd_destroy(rslrl_rnd *rnd);
+const char  *rslrl_rnd_last_error(const rslrl_rnd *rnd);          /* NULL: last create error         */
+/* Host vectors of rslrl_rnd_num_params floats; set also zeroes the Adam moments and step count.
+ * These calls synchronise the stream. */
+rslrl_status rslrl_rnd_set_params(rslrl_rnd *rnd, const float *h_predictor, const float *h_target, size_t n);
+rslrl_status rslrl_rnd_get_params(rslrl_rnd *rnd, float *h_predictor, size_t n);
+rslrl_status rslrl_rnd_get_grads(rslrl_rnd *rnd, float *h_grad, size_t n);   /* of the last step     */
+
+/* d_obs [rows][obs_stride] float32 (device), rows <= max_rows, obs_stride >= obs_dim.
+ * d_rewards_inout [rows] (device, may be NULL): += weight * r_int.  d_r_int_out [rows] (device,
+ * may be NULL): = r_int.  Only enqueues. */
+rslrl_status rslrl_rnd_reward(rslrl_rnd *rnd, const float *d_obs, int32_t rows, int32_t obs_stride,
+                              float weight, float *d_rewards_inout, float *d_r_int_out);
+
+/* Predictor training on d_obs [batch][obs_stride]: for `epochs` epochs, shuffle the rows with
+ * the keyed bijection of (seed, iteration, epoch), cut into `minibatches` chunks (batch must be
+ * divisible; batch / minibatches <= max_rows), one Adam step per chunk; stops after max_steps
+ * steps if max_steps > 0.  h_mean_loss (host, may be NULL): mean of the step losses, which makes
+ * the call synchronise; h_first_loss likewise for the first step.
+ * RSLRL_ERR_SHAPE for an indivisible batch, RSLRL_ERR_UNSUPPORTED beyond max_rows. */
+rslrl_status rslrl_rnd_update(rslrl_rnd *rnd, const float *d_obs, int32_t batch, int32_t obs_stride,
+                              int32_t epochs, int32_t minibatches, uint64_t seed, uint32_t iteration,
+                              int32_t max_steps, float *h_mean_loss, float *h_first_loss);
+
 /* Number of kernels this library has launched in the current process (all contexts). */
 uint64_t     rslrl_kernel_launch_count(void);
 

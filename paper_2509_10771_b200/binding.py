@@ -70,6 +70,12 @@ class UpdateStats(C.Structure):
         return {n: getattr(self, n) for n, _ in self._fields_}
 
 
+class RndCfg(C.Structure):
+    _fields_ = [("obs_dim", C.c_int32), ("num_idx", C.c_int32), ("h_idx", C.c_void_p), ("num_hidden", C.c_int32),
+                ("hidden", C.c_int32 * 8), ("embed_dim", C.c_int32), ("elu_alpha", C.c_float), ("max_rows", C.c_int32),
+                ("lr", C.c_float), ("adam_b1", C.c_float), ("adam_b2", C.c_float), ("adam_eps", C.c_float)]
+
+
 class Counters(C.Structure):
     _fields_ = [("lr", C.c_float), ("adam_step", C.c_int32), ("global_step", C.c_uint32),
                 ("iteration", C.c_uint32)]
@@ -82,6 +88,8 @@ EXPORTS = [
     "rslrl_ppo_update", "rslrl_ppo_update_steps", "rslrl_distill_update", "rslrl_distill_update_steps", "rslrl_act_host", "rslrl_record_step_host",
     "rslrl_gae_host", "rslrl_gae_scratch_bytes", "rslrl_gae_scan", "rslrl_minibatch_indices",
     "rslrl_kernel_launch_count", "rslrl_profile_enable", "rslrl_profile_report", "rslrl_gae_scan_static",
+    "rslrl_rnd_num_params", "rslrl_rnd_create", "rslrl_rnd_destroy", "rslrl_rnd_last_error", "rslrl_rnd_set_params",
+    "rslrl_rnd_get_params", "rslrl_rnd_get_grads", "rslrl_rnd_reward", "rslrl_rnd_update",
 ]
 
 _lib = None
@@ -127,6 +135,15 @@ def load_library() -> C.CDLL:
         "rslrl_kernel_launch_count": (u64, []),
         "rslrl_profile_enable": (i32, [i32]),
         "rslrl_profile_report": (i32, [C.c_char_p, sz]),
+        "rslrl_rnd_num_params": (sz, [C.POINTER(RndCfg)]),
+        "rslrl_rnd_create": (i32, [C.POINTER(RndCfg), vp, C.POINTER(vp)]),
+        "rslrl_rnd_destroy": (i32, [vp]),
+        "rslrl_rnd_last_error": (C.c_char_p, [vp]),
+        "rslrl_rnd_set_params": (i32, [vp, vp, vp, sz]),
+        "rslrl_rnd_get_params": (i32, [vp, vp, sz]),
+        "rslrl_rnd_get_grads": (i32, [vp, vp, sz]),
+        "rslrl_rnd_reward": (i32, [vp, vp, i32, i32, f32, vp, vp]),
+        "rslrl_rnd_update": (i32, [vp, vp, i32, i32, i32, i32, u64, u32, i32, C.POINTER(f32), C.POINTER(f32)]),
     }
     for name, (res, args) in sig.items():
         fn = getattr(lib, name)
@@ -292,6 +309,71 @@ class Context:
 
     def gae_host(self, h_last_critic_obs):
         self._check(self.lib.rslrl_gae_host(self.handle, _ptr(h_last_critic_obs)))
+
+
+class Rnd:
+    """One rslrl_rnd: target and predictor MLPs on the entries ``idx`` of an observation row."""
+
+    def __init__(self, obs_dim: int, idx, hidden, embed_dim: int, max_rows: int, lr: float = 1e-3, elu_alpha: float = 1.0,
+                 adam_b1: float = 0.9, adam_b2: float = 0.999, adam_eps: float = 1e-8, stream: int = 0):
+        self.lib = load_library()
+        self.handle = None
+        self._idx = np.ascontiguousarray(idx, dtype=np.int32)
+        cfg = RndCfg()
+        cfg.obs_dim, cfg.num_idx, cfg.h_idx = obs_dim, self._idx.size, self._idx.ctypes.data
+        cfg.num_hidden = len(hidden)
+        for i, h in enumerate(hidden):
+            cfg.hidden[i] = h
+        cfg.embed_dim, cfg.elu_alpha, cfg.max_rows = embed_dim, elu_alpha, max_rows
+        cfg.lr, cfg.adam_b1, cfg.adam_b2, cfg.adam_eps = lr, adam_b1, adam_b2, adam_eps
+        self.num_params = int(self.lib.rslrl_rnd_num_params(C.byref(cfg)))
+        h = C.c_void_p()
+        st = self.lib.rslrl_rnd_create(C.byref(cfg), stream, C.byref(h))
+        if st != 0:
+            raise RslrlError(st, (self.lib.rslrl_rnd_last_error(None) or b"").decode())
+        self.handle = h
+
+    def _check(self, st: int):
+        if st != 0:
+            raise RslrlError(st, (self.lib.rslrl_rnd_last_error(self.handle) or b"").decode())
+
+    def destroy(self):
+        if self.handle is not None:
+            self.lib.rslrl_rnd_destroy(self.handle)
+            self.handle = None
+
+    def __del__(self):
+        try:
+            self.destroy()
+        except Exception:
+            pass
+
+    def set_params(self, predictor: np.ndarray, target: np.ndarray):
+        f = np.ascontiguousarray(predictor, dtype=np.float32)
+        g = np.ascontiguousarray(target, dtype=np.float32)
+        self._check(self.lib.rslrl_rnd_set_params(self.handle, f.ctypes.data, g.ctypes.data, f.size))
+
+    def get_params(self) -> np.ndarray:
+        out = np.empty(self.num_params, dtype=np.float32)
+        self._check(self.lib.rslrl_rnd_get_params(self.handle, out.ctypes.data, out.size))
+        return out
+
+    def get_grads(self) -> np.ndarray:
+        out = np.empty(self.num_params, dtype=np.float32)
+        self._check(self.lib.rslrl_rnd_get_grads(self.handle, out.ctypes.data, out.size))
+        return out
+
+    def reward(self, d_obs, rows: int, obs_stride: int, weight: float = 0.0, d_rewards_inout=None, d_r_int_out=None):
+        self._check(self.lib.rslrl_rnd_reward(self.handle, _ptr(d_obs), rows, obs_stride, weight, _ptr(d_rewards_inout),
+                                              _ptr(d_r_int_out)))
+
+    def update(self, d_obs, batch: int, obs_stride: int, epochs: int, minibatches: int, seed: int, iteration: int,
+               max_steps: int = 0, want_loss: bool = True):
+        mean, first = C.c_float(0), C.c_float(0)
+        self._check(self.lib.rslrl_rnd_update(self.handle, _ptr(d_obs), batch, obs_stride, epochs, minibatches, seed,
+                                              iteration, max_steps, C.byref(mean) if want_loss else None,
+                                              C.byref(first) if want_loss else None))
+        return {"mean_loss": mean.value, "first_loss": first.value} if want_loss else None
 
 
 def gae_scan(d_rewards, d_values, d_dones, d_timeouts, d_last_values, d_returns, d_advantages, T: int, N: int,

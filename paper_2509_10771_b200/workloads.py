@@ -15,7 +15,7 @@ are the ones this library is measured on.
 from __future__ import annotations
 
 from dataclasses import dataclass, field, replace
-from typing import Dict, List, Optional, Tuple
+from typing import Dict, List, Optional, Sequence, Tuple
 
 import numpy as np
 
@@ -195,6 +195,34 @@ def make_expert_actions(w: Workload, seed: Optional[int] = None) -> np.ndarray:
     (stream 9 of the workload's seed)."""
     seed = w.seed if seed is None else seed
     return _rng(seed, 9).standard_normal((w.num_steps, w.num_envs, w.num_actions), dtype=np.float32)
+
+
+def rnd_layer_dims(num_idx: int, hidden: Sequence[int], embed_dim: int) -> List[Tuple[int, int]]:
+    """(fan_in, fan_out) of the layers num_idx -> hidden... -> embed_dim of a distillation net."""
+    widths = [num_idx, *hidden, embed_dim]
+    return [(widths[i], widths[i + 1]) for i in range(len(widths) - 1)]
+
+
+def make_rnd_setup(w: Workload, num_idx: int = 12, hidden: Sequence[int] = (128, 64), embed_dim: int = 32,
+                   seed: Optional[int] = None) -> Dict[str, object]:
+    """A state subset and the two nets of random network distillation for workload ``w`` (stream 10):
+    ``idx`` = num_idx distinct entries of the actor observation (sorted), ``predictor`` / ``target`` = flat
+    float32 vectors W1[in][out], b1, ... drawn like ``make_params``; the target is drawn four times wider
+    so that the two nets differ at the start."""
+    seed = w.seed if seed is None else seed
+    rng = _rng(seed, 10)
+    idx = np.sort(rng.choice(w.actor_obs_dim, size=num_idx, replace=False)).astype(np.int32)
+    dims = rnd_layer_dims(num_idx, hidden, embed_dim)
+
+    def draw(scale):
+        parts = []
+        for fi, fo in dims:
+            bound = scale / np.sqrt(fi)
+            parts.append(((rng.random(fi * fo + fo, dtype=np.float32) * 2.0 - 1.0) * bound).astype(np.float32))
+        return np.concatenate(parts)
+
+    return {"idx": idx, "dims": dims, "hidden": tuple(hidden), "embed_dim": embed_dim, "predictor": draw(1.0),
+            "target": draw(4.0)}
 
 
 def param_layout(w: Workload) -> List[Tuple[str, int, Tuple[int, ...]]]:

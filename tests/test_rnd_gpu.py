@@ -1,0 +1,132 @@
+"""GPU parity of random network distillation on a state subset (rslrl_rnd_*) against the FP64 oracle:
+intrinsic reward per row, reward mixing, the first predictor step (loss, gradient, parameters) and the whole
+epoch x minibatch training loop on the same keyed minibatches.
+
+The CUDA path computes in FP32; tolerance 1e-4 (relative to the element plus the array's rms), as for
+the FP32 mode of the PPO update.  The intrinsic reward is a mean of squared differences of two nets that start
+far apart (the target is drawn four times wider), so it carries no cancellation at these inputs."""
+from types import SimpleNamespace
+
+import numpy as np
+import pytest
+
+from oracle import ppo_oracle as O
+from paper_2509_10771_b200 import workloads as WL
+
+from parity_utils import assert_close, rel_l2
+
+pytestmark = pytest.mark.gpu
+
+CASES = {
+    # name: (workload for the observation recipe, rows, RND net keywords, minibatches, epochs)
+    "tiny": (WL.TINY, 8 * 64, dict(num_idx=5, hidden=(16,), embed_dim=3), 2, 1),
+    "flat": (WL.FLAT, 24 * 300, dict(num_idx=12, hidden=(128, 64), embed_dim=32), 4, 2),
+    "rough": (WL.ROUGH, 24 * 257, dict(num_idx=48, hidden=(256, 128, 64), embed_dim=50), 8, 2),   # ragged rows
+}
+
+
+def _setup(case, lr=1e-3):
+    import torch
+    from paper_2509_10771_b200 import binding
+    w, rows, kw, mbs, epochs = CASES[case]
+    envs = rows // w.num_steps
+    ws = w.scaled(envs)
+    obs = WL.make_rollout_inputs(ws)["obs_actor"][:w.num_steps].reshape(rows, w.actor_obs_dim)
+    setup = WL.make_rnd_setup(ws, **kw)
+    rnd = binding.Rnd(w.actor_obs_dim, setup["idx"], setup["hidden"], setup["embed_dim"], max_rows=rows, lr=lr)
+    rnd.set_params(setup["predictor"], setup["target"])
+    d_obs = torch.from_numpy(obs).to("cuda")
+    return w, rows, setup, rnd, obs, d_obs, mbs, epochs
+
+
+@pytest.mark.parametrize("case", ["tiny", "flat", "rough"])
+def test_intrinsic_reward_matches_oracle(case):
+    import torch
+    w, rows, setup, rnd, obs, d_obs, _, _ = _setup(case)
+    ref, _, _, _ = O.rnd_reward(setup["predictor"], setup["target"], setup["dims"], obs, setup["idx"], 1.0)
+    rng = np.random.default_rng(1)
+    r_ext = rng.standard_normal(rows).astype(np.float32)
+    d_rew = torch.from_numpy(r_ext.copy()).to("cuda")
+    d_int = torch.full((rows,), -1.0, device="cuda")
+    rnd.reward(d_obs, rows, w.actor_obs_dim, weight=0.25, d_rewards_inout=d_rew, d_r_int_out=d_int)
+    torch.cuda.synchronize()
+    assert_close(d_int.cpu().numpy(), ref, 1e-4, "r_int")
+    assert_close(d_rew.cpu().numpy(), r_ext.astype(np.float64) + 0.25 * ref, 1e-4, "mixed reward")
+    # a prefix of the rows, and a wider row stride, give the same rewards
+    wide = torch.zeros((rows, w.actor_obs_dim + 5), device="cuda")
+    wide[:, :w.actor_obs_dim] = d_obs
+    d_int2 = torch.full((rows,), -1.0, device="cuda")
+    rnd.reward(wide, rows // 3, w.actor_obs_dim + 5, d_r_int_out=d_int2)
+    torch.cuda.synchronize()
+    assert torch.equal(d_int2[:rows // 3], d_int[:rows // 3])
+    assert bool((d_int2[rows // 3:] == -1.0).all())
+    rnd.destroy()
+
+
+@pytest.mark.parametrize("case", ["tiny", "flat", "rough"])
+def test_first_predictor_step_matches_oracle(case):
+    w, rows, setup, rnd, obs, d_obs, mbs, epochs = _setup(case)
+    hp = SimpleNamespace(epochs=epochs, minibatches=mbs, elu_alpha=1.0, adam_b1=0.9, adam_b2=0.999, adam_eps=1e-8)
+    out = rnd.update(d_obs, rows, w.actor_obs_dim, epochs, mbs, seed=7, iteration=3, max_steps=1)
+    state = O.OptimState(setup["predictor"], 1e-3)
+    ref = O.rnd_update(state, setup["target"], setup["dims"], obs, setup["idx"], hp, seed=7, iteration=3, max_steps=1)
+    assert_close(out["first_loss"], ref[0]["loss"], 1e-4, "loss")
+    assert_close(rnd.get_grads(), ref[0]["grad"], 1e-4, "grad")
+    # Adam's first step moves every entry by lr * sign(g): entries whose gradient is zero to rounding may differ
+    assert_close(rnd.get_params(), state.theta, 1e-4, "params", max_outlier_frac=2e-3, outlier_abs=2.05e-3)
+    rnd.destroy()
+
+
+@pytest.mark.parametrize("case", ["tiny", "flat", "rough"])
+def test_predictor_training_tracks_oracle(case):
+    import torch
+    w, rows, setup, rnd, obs, d_obs, mbs, epochs = _setup(case)
+    hp = SimpleNamespace(epochs=epochs, minibatches=mbs, elu_alpha=1.0, adam_b1=0.9, adam_b2=0.999, adam_eps=1e-8)
+    out = rnd.update(d_obs, rows, w.actor_obs_dim, epochs, mbs, seed=11, iteration=0)
+    state = O.OptimState(setup["predictor"], 1e-3)
+    ref = O.rnd_update(state, setup["target"], setup["dims"], obs, setup["idx"], hp, seed=11, iteration=0)
+    assert len(ref) == epochs * mbs
+    assert_close(out["first_loss"], ref[0]["loss"], 1e-4, "first loss")
+    assert_close(out["mean_loss"], float(np.mean([r["loss"] for r in ref])), 1e-4, "mean loss")
+    assert rel_l2(rnd.get_params(), state.theta) < 1e-4
+    assert rel_l2(rnd.get_grads(), ref[-1]["grad"]) < 1e-3
+    # training lowers the intrinsic reward of the rows it was trained on
+    d_int = torch.empty((rows,), device="cuda")
+    rnd.reward(d_obs, rows, w.actor_obs_dim, d_r_int_out=d_int)
+    before, _, _, _ = O.rnd_reward(setup["predictor"], setup["target"], setup["dims"], obs, setup["idx"], 1.0)
+    after, _, _, _ = O.rnd_reward(state.theta, setup["target"], setup["dims"], obs, setup["idx"], 1.0)
+    assert after.mean() < before.mean()
+    assert_close(d_int.cpu().numpy(), after, 2e-4, "r_int after training")
+    rnd.destroy()
+
+
+def test_rnd_argument_checks():
+    import torch
+    from paper_2509_10771_b200 import binding
+    with pytest.raises(binding.RslrlError) as e:
+        binding.Rnd(8, [0, 9], (4,), 2, max_rows=16)                # index out of range
+    assert e.value.status == 1
+    rnd = binding.Rnd(8, [0, 3, 5], (4,), 2, max_rows=16)
+    n = rnd.num_params
+    assert n == 3 * 4 + 4 + 4 * 2 + 2
+    rnd.set_params(np.zeros(n, np.float32), np.ones(n, np.float32))
+    d_obs = torch.zeros((64, 8), device="cuda")
+    with pytest.raises(binding.RslrlError) as e:
+        rnd.reward(d_obs, 17, 8, d_r_int_out=torch.zeros(17, device="cuda"))
+    assert e.value.status == 5
+    with pytest.raises(binding.RslrlError) as e:
+        rnd.update(d_obs, 30, 8, 1, 4, seed=0, iteration=0)          # 30 rows do not divide into 4
+    assert e.value.status == 2
+    with pytest.raises(binding.RslrlError) as e:
+        rnd.update(d_obs, 64, 8, 1, 2, seed=0, iteration=0)          # 32 rows per minibatch > max_rows
+    assert e.value.status == 5
+    with pytest.raises(binding.RslrlError) as e:
+        rnd.set_params(np.zeros(n + 1, np.float32), np.zeros(n + 1, np.float32))
+    assert e.value.status == 2
+    # zero observations, zero predictor, target of ones: g = bias path only, reward is finite and equal on all rows
+    d_int = torch.empty(16, device="cuda")
+    rnd.reward(d_obs, 16, 8, d_r_int_out=d_int)
+    torch.cuda.synchronize()
+    v = d_int.cpu().numpy()
+    assert np.all(v == v[0]) and np.isfinite(v[0]) and v[0] > 0
+    rnd.destroy()
