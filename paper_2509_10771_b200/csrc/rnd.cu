@@ -90,10 +90,18 @@ __global__ void __launch_bounds__(256) rnd_adam_kernel(const float* __restrict__
         m[p] = mm; v[p] = vv;
         param[p] -= lr * (mm * c1) / (sqrtf(vv * c2) + eps);
     }
-    if (blockIdx.x == 0 && threadIdx.x == 0) {
+    if (blockIdx.x == 0) {
+        // fixed order: thread t adds partials t, t + 256, ...; then a tree over the 256 sums
+        __shared__ float red[256];
         float t = 0.f;
-        for (int i = 0; i < nloss; ++i) t += loss_partials[i];
-        *step_loss = t * inv_rows;
+        for (int i = threadIdx.x; i < nloss; i += 256) t += loss_partials[i];
+        red[threadIdx.x] = t;
+        __syncthreads();
+        for (int w = 128; w > 0; w >>= 1) {
+            if ((int)threadIdx.x < w) red[threadIdx.x] += red[threadIdx.x + w];
+            __syncthreads();
+        }
+        if (threadIdx.x == 0) *step_loss = red[0] * inv_rows;
     }
 }
 
