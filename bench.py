@@ -95,6 +95,15 @@ def ncu_traffic(family):
     return NCU_TRAFFIC["bytes_per_launch"].get(family)
 
 
+def iteration_flops(w):
+    T, N = w.num_steps, w.num_envs
+    steps = w.epochs * w.minibatches
+    R = w.minibatch_rows * (2 if w.sym_enable else 1)
+    full = sum(2 * i * o for net in ("actor", "critic") for i, o in w.layer_dims(net))
+    first = sum(2 * i * o for net in ("actor", "critic") for i, o in w.layer_dims(net)[:1])
+    return T * N * full + steps * R * (3 * full - first)
+
+
 # ------------------------------------------------------------------------------------------
 # the oracle arm (CPU baseline and --impl reference)
 # ------------------------------------------------------------------------------------------

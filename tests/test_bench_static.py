@@ -1,0 +1,33 @@
+"""Static check of the scripts that only run on a GPU machine: every name they load is defined somewhere in the
+file (a function deleted by mistake would otherwise show up only at the end of a GPU run)."""
+import ast
+import builtins
+import os
+
+import pytest
+
+ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+
+
+def undefined_names(path):
+    tree = ast.parse(open(path).read())
+    defined = set(dir(builtins)) | {"__file__", "__name__"}
+    for n in ast.walk(tree):
+        if isinstance(n, (ast.FunctionDef, ast.ClassDef)):
+            defined.add(n.name)
+        elif isinstance(n, ast.arg):
+            defined.add(n.arg)
+        elif isinstance(n, ast.Name) and isinstance(n.ctx, (ast.Store, ast.Del)):
+            defined.add(n.id)
+        elif isinstance(n, (ast.Import, ast.ImportFrom)):
+            defined.update((a.asname or a.name).split(".")[0] for a in n.names)
+        elif isinstance(n, ast.ExceptHandler) and n.name:
+            defined.add(n.name)
+    return sorted({n.id for n in ast.walk(tree)
+                   if isinstance(n, ast.Name) and isinstance(n.ctx, ast.Load) and n.id not in defined})
+
+
+@pytest.mark.parametrize("rel", ["bench.py", "__graft_entry__.py", "paper_2509_10771_b200/bandwidth_report.py",
+                                 "paper_2509_10771_b200/binding.py"])
+def test_every_loaded_name_is_defined(rel):
+    assert undefined_names(os.path.join(ROOT, rel)) == []
