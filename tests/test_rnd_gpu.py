@@ -130,3 +130,44 @@ def test_rnd_argument_checks():
     v = d_int.cpu().numpy()
     assert np.all(v == v[0]) and np.isfinite(v[0]) and v[0] > 0
     rnd.destroy()
+
+
+def test_intrinsic_reward_enters_gae_like_the_oracle():
+    """The place of the reward in the learn iteration: r_t + w * r_int(o_t) is what record_step stores and what
+    the advantage estimator sees.  The oracle's rollout runs on the mixed rewards computed by the oracle."""
+    import torch
+    from paper_2509_10771_b200 import binding
+    from parity_utils import oracle_rollout, read_storage
+    w = WL.ROUGH.scaled(300, minibatches=4)
+    T, N, Da = w.num_steps, w.num_envs, w.actor_obs_dim
+    theta, inputs = WL.make_params(w), WL.make_rollout_inputs(w)
+    setup = WL.make_rnd_setup(w, num_idx=20, hidden=(64, 32), embed_dim=16)
+    weight = 0.05
+    ctx = binding.Context(w, precision=WL.PRECISION_FP32)
+    ctx.set_params(theta)
+    rnd = binding.Rnd(Da, setup["idx"], setup["hidden"], setup["embed_dim"], max_rows=N)
+    rnd.set_params(setup["predictor"], setup["target"])
+    dev = torch.device("cuda")
+    oa = torch.from_numpy(inputs["obs_actor"]).to(dev)
+    rew = torch.from_numpy(inputs["rewards"]).to(dev)
+    dn = torch.from_numpy(inputs["dones"]).to(dev)
+    to = torch.from_numpy(inputs["timeouts"]).to(dev)
+    for t in range(T):
+        ctx.act(oa[t])
+        r = rew[t].clone()
+        rnd.reward(oa[t], N, Da, weight=weight, d_rewards_inout=r)
+        ctx.record_step(r, dn[t], to[t])
+    ctx.gae(oa[T])
+    torch.cuda.synchronize()
+    got = read_storage(ctx, w)
+    r_int, _, _, _ = O.rnd_reward(setup["predictor"], setup["target"], setup["dims"],
+                                  inputs["obs_actor"][:T].reshape(T * N, Da), setup["idx"], 1.0)
+    mixed = dict(inputs)
+    mixed["rewards"] = inputs["rewards"].astype(np.float64) + weight * r_int.reshape(T, N)
+    want = oracle_rollout(w, theta, mixed)
+    assert float(np.abs(weight * r_int).mean()) > 0.1 * float(np.abs(inputs["rewards"]).mean())   # the term matters here
+    assert_close(got["rewards"], mixed["rewards"], 1e-4, "rewards")
+    for k in ("returns", "advantages"):
+        assert_close(got[k], want[k], 1e-4, k)
+    rnd.destroy()
+    ctx.destroy()
