@@ -336,6 +336,47 @@ rslrl_status rslrl_rnd_update(rslrl_rnd *rnd, const float *d_obs, int32_t batch,
                               int32_t epochs, int32_t minibatches, uint64_t seed, uint32_t iteration,
                               int32_t max_steps, float *h_mean_loss, float *h_first_loss);
 
+/* ---------------------------------------------------------------------------------------------
+ * Recurrent memory layer (paper: "Implementation Details": recurrent networks through explicit
+ * management of hidden states across rollouts and back-propagation through time).
+ *
+ * A GRU layer over a time-major rollout.  Per step t (gate order r, z, n):
+ *   h_in(t) = h0 for t = 0, else (1 - done[t-1]) * h(t-1)      (same-step reset: zero state after done)
+ *   r = sigmoid(x_t W_ir + b_ir + h_in W_hr + b_hr),  z likewise,
+ *   n = tanh(x_t W_in + b_in + r * (h_in W_hn + b_hn)),  h(t) = (1 - z) n + z h_in
+ * The paper names neither the cell nor the reset rule; these are this library's choices.
+ * Parameters (host, float32): W_i[D][3H], b_i[3H], W_h[H][3H], b_h[3H], in this order.
+ * All arithmetic is FP32.  The object owns parameters, gradient and work buffers sized for
+ * max_steps x max_envs; calls on one object are not thread-safe and enqueue on its stream. */
+typedef struct rslrl_gru rslrl_gru;
+
+typedef struct {
+    int32_t input_dim;                  /* D >= 1                                                    */
+    int32_t hidden_dim;                 /* H, a multiple of 4                                        */
+    int32_t max_steps;                  /* largest T                                                 */
+    int32_t max_envs;                   /* largest N                                                 */
+} rslrl_gru_cfg;
+
+size_t       rslrl_gru_num_params(const rslrl_gru_cfg *cfg);      /* 0 if cfg is invalid             */
+rslrl_status rslrl_gru_create(const rslrl_gru_cfg *cfg, void *cuda_stream, rslrl_gru **out);
+rslrl_status rslrl_gru_destroy(rslrl_gru *gru);
+const char  *rslrl_gru_last_error(const rslrl_gru *gru);          /* NULL: last create error         */
+rslrl_status rslrl_gru_set_params(rslrl_gru *gru, const float *h_params, size_t n);   /* synchronises */
+rslrl_status rslrl_gru_get_grads(rslrl_gru *gru, float *h_grad, size_t n);            /* synchronises */
+
+/* Forward over T steps of N environments (device pointers, float buffers 16-byte aligned):
+ *   d_x [T][N][x_stride] (x_stride a multiple of 4, >= D rounded up to 4; padding is not read as data),
+ *   d_h0 [N][H] the state entering step 0, d_dones [T][N] uint8, d_h_out [T][N][H] = h(t).
+ * d_x and d_dones must stay unchanged until rslrl_gru_backward has run.  Only enqueues. */
+rslrl_status rslrl_gru_forward(rslrl_gru *gru, const float *d_x, int32_t x_stride, const float *d_h0,
+                               const uint8_t *d_dones, int32_t T, int32_t N, float *d_h_out);
+
+/* Back-propagation through the T steps of the last forward for L = sum_t <d_dh[t], h(t)>:
+ *   d_dh [T][N][H]; d_dx [T][N][dx_stride] (may be NULL) = dL/dx; d_dh0 [N][H] (may be NULL) = dL/dh0;
+ * the parameter gradient is kept in the object (rslrl_gru_get_grads).  No gradient crosses a reset.
+ * One backward per forward: RSLRL_ERR_STATE otherwise.  Only enqueues. */
+rslrl_status rslrl_gru_backward(rslrl_gru *gru, const float *d_dh, float *d_dx, int32_t dx_stride, float *d_dh0);
+
 /* Number of kernels this library has launched in the current process (all contexts). */
 uint64_t     rslrl_kernel_launch_count(void);
 

@@ -76,6 +76,10 @@ class RndCfg(C.Structure):
                 ("lr", C.c_float), ("adam_b1", C.c_float), ("adam_b2", C.c_float), ("adam_eps", C.c_float)]
 
 
+class GruCfg(C.Structure):
+    _fields_ = [("input_dim", C.c_int32), ("hidden_dim", C.c_int32), ("max_steps", C.c_int32), ("max_envs", C.c_int32)]
+
+
 class Counters(C.Structure):
     _fields_ = [("lr", C.c_float), ("adam_step", C.c_int32), ("global_step", C.c_uint32),
                 ("iteration", C.c_uint32)]
@@ -90,6 +94,8 @@ EXPORTS = [
     "rslrl_kernel_launch_count", "rslrl_profile_enable", "rslrl_profile_report", "rslrl_gae_scan_static",
     "rslrl_rnd_num_params", "rslrl_rnd_create", "rslrl_rnd_destroy", "rslrl_rnd_last_error", "rslrl_rnd_set_params",
     "rslrl_rnd_get_params", "rslrl_rnd_get_grads", "rslrl_rnd_reward", "rslrl_rnd_update",
+    "rslrl_gru_num_params", "rslrl_gru_create", "rslrl_gru_destroy", "rslrl_gru_last_error", "rslrl_gru_set_params",
+    "rslrl_gru_get_grads", "rslrl_gru_forward", "rslrl_gru_backward",
 ]
 
 _lib = None
@@ -144,6 +150,14 @@ def load_library() -> C.CDLL:
         "rslrl_rnd_get_grads": (i32, [vp, vp, sz]),
         "rslrl_rnd_reward": (i32, [vp, vp, i32, i32, f32, vp, vp]),
         "rslrl_rnd_update": (i32, [vp, vp, i32, i32, i32, i32, u64, u32, i32, C.POINTER(f32), C.POINTER(f32)]),
+        "rslrl_gru_num_params": (sz, [C.POINTER(GruCfg)]),
+        "rslrl_gru_create": (i32, [C.POINTER(GruCfg), vp, C.POINTER(vp)]),
+        "rslrl_gru_destroy": (i32, [vp]),
+        "rslrl_gru_last_error": (C.c_char_p, [vp]),
+        "rslrl_gru_set_params": (i32, [vp, vp, sz]),
+        "rslrl_gru_get_grads": (i32, [vp, vp, sz]),
+        "rslrl_gru_forward": (i32, [vp, vp, i32, vp, vp, i32, i32, vp]),
+        "rslrl_gru_backward": (i32, [vp, vp, vp, i32, vp]),
     }
     for name, (res, args) in sig.items():
         fn = getattr(lib, name)
@@ -374,6 +388,51 @@ class Rnd:
                                               iteration, max_steps, C.byref(mean) if want_loss else None,
                                               C.byref(first) if want_loss else None))
         return {"mean_loss": mean.value, "first_loss": first.value} if want_loss else None
+
+
+class Gru:
+    """One rslrl_gru: a GRU memory layer over time-major rollouts with state resets and BPTT."""
+
+    def __init__(self, input_dim: int, hidden_dim: int, max_steps: int, max_envs: int, stream: int = 0):
+        self.lib = load_library()
+        self.handle = None
+        cfg = GruCfg(input_dim, hidden_dim, max_steps, max_envs)
+        self.num_params = int(self.lib.rslrl_gru_num_params(C.byref(cfg)))
+        h = C.c_void_p()
+        st = self.lib.rslrl_gru_create(C.byref(cfg), stream, C.byref(h))
+        if st != 0:
+            raise RslrlError(st, (self.lib.rslrl_gru_last_error(None) or b"").decode())
+        self.handle = h
+
+    def _check(self, st: int):
+        if st != 0:
+            raise RslrlError(st, (self.lib.rslrl_gru_last_error(self.handle) or b"").decode())
+
+    def destroy(self):
+        if self.handle is not None:
+            self.lib.rslrl_gru_destroy(self.handle)
+            self.handle = None
+
+    def __del__(self):
+        try:
+            self.destroy()
+        except Exception:
+            pass
+
+    def set_params(self, flat: np.ndarray):
+        f = np.ascontiguousarray(flat, dtype=np.float32)
+        self._check(self.lib.rslrl_gru_set_params(self.handle, f.ctypes.data, f.size))
+
+    def get_grads(self) -> np.ndarray:
+        out = np.empty(self.num_params, dtype=np.float32)
+        self._check(self.lib.rslrl_gru_get_grads(self.handle, out.ctypes.data, out.size))
+        return out
+
+    def forward(self, d_x, x_stride: int, d_h0, d_dones, T: int, N: int, d_h_out):
+        self._check(self.lib.rslrl_gru_forward(self.handle, _ptr(d_x), x_stride, _ptr(d_h0), _ptr(d_dones), T, N, _ptr(d_h_out)))
+
+    def backward(self, d_dh, d_dx=None, dx_stride: int = 0, d_dh0=None):
+        self._check(self.lib.rslrl_gru_backward(self.handle, _ptr(d_dh), _ptr(d_dx), dx_stride, _ptr(d_dh0)))
 
 
 def gae_scan(d_rewards, d_values, d_dones, d_timeouts, d_last_values, d_returns, d_advantages, T: int, N: int,

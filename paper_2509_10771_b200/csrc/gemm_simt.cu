@@ -212,6 +212,7 @@ cudaError_t launch_tiles(const GemmBatch& b, bool ta, bool tb, int epi, cudaStre
     RSLRL_SGEMM_CASE(false, false, EPI_BIAS_ELU, "sgemm_fwd")
     RSLRL_SGEMM_CASE(false, false, EPI_BIAS, "sgemm_fwd_linear")
     RSLRL_SGEMM_CASE(false, true, EPI_DELU, "sgemm_dgrad")
+    RSLRL_SGEMM_CASE(false, true, EPI_PLAIN, "sgemm_dgrad_plain")
     RSLRL_SGEMM_CASE(true, false, EPI_PLAIN, "sgemm_wgrad")
 #undef RSLRL_SGEMM_CASE
     return cudaErrorInvalidValue;

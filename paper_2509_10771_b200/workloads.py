@@ -225,6 +225,22 @@ def make_rnd_setup(w: Workload, num_idx: int = 12, hidden: Sequence[int] = (128,
             "target": draw(4.0)}
 
 
+def make_gru_setup(w: Workload, hidden_dim: int = 256, seed: Optional[int] = None) -> Dict[str, np.ndarray]:
+    """Inputs of a recurrent memory layer over one rollout of workload ``w`` (stream 11): ``params`` flat float32
+    in the order W_i[D][3H], b_i, W_h[H][3H], b_h drawn U(-1/sqrt(H), 1/sqrt(H)), ``h0[N][H]`` ~ 0.5 N(0,1) and
+    ``dh[T][N][H]`` ~ N(0,1) / (T N) standing in for the gradient a downstream network sends back.  Observations
+    and done flags are those of ``make_rollout_inputs``."""
+    seed = w.seed if seed is None else seed
+    rng = _rng(seed, 11)
+    D, H, T, N = w.actor_obs_dim, hidden_dim, w.num_steps, w.num_envs
+    n = D * 3 * H + 3 * H + H * 3 * H + 3 * H
+    bound = 1.0 / np.sqrt(H)
+    params = ((rng.random(n, dtype=np.float32) * 2.0 - 1.0) * bound).astype(np.float32)
+    h0 = (rng.standard_normal((N, H), dtype=np.float32) * np.float32(0.5))
+    dh = (rng.standard_normal((T, N, H), dtype=np.float32) / np.float32(T * N))
+    return {"params": params, "h0": h0, "dh": dh, "hidden_dim": H}
+
+
 def param_layout(w: Workload) -> List[Tuple[str, int, Tuple[int, ...]]]:
     """Flat parameter order: (name, offset, shape).
 
