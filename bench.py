@@ -534,15 +534,93 @@ def run_rnd(args):
     rnd.destroy()
 
 
+def run_gru(args):
+    """--task gru: the recurrent memory layer over one rollout (rslrl_gru_forward + rslrl_gru_backward, T steps
+    of N environments, hidden width 256, resets at the workload's done rate), one GPU.  Prints its own JSON line."""
+    import torch
+    from paper_2509_10771_b200 import binding, build
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device: the path has no CPU fallback")
+    torch.cuda.set_device(0)
+    build.build()
+    w = WORKLOAD
+    T, N, D, H = w.num_steps, w.num_envs, w.actor_obs_dim, 256
+    dev = torch.device("cuda", 0)
+    stream = torch.cuda.current_stream()
+    inputs = WL.make_rollout_inputs(w)
+    setup = WL.make_gru_setup(w, hidden_dim=H)
+    stride = (D + 3) // 4 * 4
+    xp = np.zeros((T, N, stride), dtype=np.float32)
+    xp[..., :D] = inputs["obs_actor"][:T]
+    d_x = torch.from_numpy(xp).to(dev)
+    d_h0 = torch.from_numpy(setup["h0"]).to(dev)
+    d_dn = torch.from_numpy(inputs["dones"]).to(dev)
+    d_dh = torch.from_numpy(setup["dh"]).to(dev)
+    d_h = torch.empty((T, N, H), device=dev)
+    d_dx = torch.empty((T, N, stride), device=dev)
+    d_dh0 = torch.empty((N, H), device=dev)
+    gru = binding.Gru(D, H, T, N, stream=stream.cuda_stream)
+    gru.set_params(setup["params"])
+    flush_buf = torch.empty(256 << 20, dtype=torch.uint8, device=dev)
+
+    def iteration():
+        gru.forward(d_x, stride, d_h0, d_dn, T, N, d_h)
+        gru.backward(d_dh, d_dx, stride, d_dh0)
+
+    for _ in range(max(args.warmup, 3)):
+        iteration()
+    torch.cuda.synchronize()
+    evs = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(args.steps)]
+    for a, b in evs:
+        flush_buf.zero_()
+        a.record(stream)
+        iteration()
+        b.record(stream)
+    torch.cuda.synchronize()
+    ms = sum(a.elapsed_time(b) for a, b in evs)
+    binding.profile_enable(True)
+    binding.profile_report()
+    for _ in range(min(args.steps, 10)):
+        iteration()
+    torch.cuda.synchronize()
+    prof = binding.profile_report()
+    binding.profile_enable(False)
+    total = sum(v["ms"] for v in prof.values()) or 1.0
+    shares = {k: {"launches": v["launches"], "ms": round(v["ms"], 3), "share": round(v["ms"] / total, 4)}
+              for k, v in sorted(prof.items(), key=lambda kv: -kv[1]["ms"])}
+    # multiply-adds per transition: forward (D + H) 3H, backward twice that (data and weight gradients)
+    flops = 2.0 * 3 * (D + H) * 3 * H * T * N
+    from oracle import gru_oracle as G
+    ns = ORACLE_SAMPLE_ENVS
+    p = G.unpack_gru(setup["params"], D, H)
+    t0 = time.perf_counter()
+    c = G.gru_sequence_forward(p, inputs["obs_actor"][:T, :ns], setup["h0"][:ns], inputs["dones"][:, :ns])
+    G.gru_sequence_backward(p, c, setup["dh"][:, :ns])
+    cpu_s = time.perf_counter() - t0
+    line = {
+        "metric": "recurrent layer forward + BPTT transitions/s", "value": T * N * args.steps / (ms * 1e-3), "unit": UNIT,
+        "n_gpus": 1, "steps": args.steps, "warmup": max(args.warmup, 3), "ms_per_step": ms / args.steps,
+        "higher_is_better": True, "dtype": "f32", "data": "synthetic",
+        "config": {"workload": w.name, "task": "gru", "num_envs": N, "num_steps": T, "input_dim": D, "hidden_dim": H,
+                   "l2": "256 MiB buffer written between timed steps"},
+        "fp32_tflops": flops / (ms / args.steps * 1e-3) / 1e12,
+        "kernel_shares": shares,
+        "cpu_baseline": {"value": T * ns / cpu_s, "unit": UNIT, "cores": blas_threads(), "kind": "oracle",
+                         "sample": f"the oracle's forward and backward pass on {ns} of the {N} environments"},
+    }
+    print(json.dumps(line), flush=True)
+    gru.destroy()
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
     ap.add_argument("--steps", type=int, default=50)
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
-    ap.add_argument("--task", default="ppo", choices=["ppo", "distill", "rnd"],
+    ap.add_argument("--task", default="ppo", choices=["ppo", "distill", "rnd", "gru"],
                     help="ppo: the learn iteration the metric is quoted on (default); distill: the distillation iteration; "
-                         "rnd: random network distillation over one rollout")
+                         "rnd: random network distillation over one rollout; gru: the recurrent layer over one rollout")
     args = ap.parse_args()
     rank = int(os.environ.get("RANK", "0"))
     world = int(os.environ.get("WORLD_SIZE", "1"))
@@ -555,6 +633,9 @@ def main():
     elif args.task == "rnd":
         if rank == 0:
             run_rnd(args)
+    elif args.task == "gru":
+        if rank == 0:
+            run_gru(args)
     else:
         run_ours(args, rank, world, local_rank)
 
