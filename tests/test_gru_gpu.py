@@ -136,3 +136,33 @@ def test_gru_argument_checks():
         gru.set_params(np.zeros(3, np.float32))
     assert e.value.status == 2
     gru.destroy()
+
+
+def test_full_size_rollout_matches_oracle():
+    """The size the benchmark's recurrent task runs: 24 steps x 4096 environments of 235 observations, H = 256,
+    the workload's own done rate.  Every state and every gradient entry is compared."""
+    import torch
+    from paper_2509_10771_b200 import binding
+    w = WL.ROUGH
+    T, N, D, H = w.num_steps, w.num_envs, w.actor_obs_dim, 256
+    inputs = WL.make_rollout_inputs(w)
+    setup = WL.make_gru_setup(w, hidden_dim=H)
+    stride = (D + 3) // 4 * 4
+    xp = np.zeros((T, N, stride), dtype=np.float32)
+    xp[..., :D] = inputs["obs_actor"][:T]
+    gru = binding.Gru(D, H, T, N)
+    gru.set_params(setup["params"])
+    d_x, d_h0 = torch.from_numpy(xp).to("cuda"), torch.from_numpy(setup["h0"]).to("cuda")
+    d_dn, d_dh = torch.from_numpy(inputs["dones"]).to("cuda"), torch.from_numpy(setup["dh"]).to("cuda")
+    d_h, d_dx, d_dh0 = torch.empty((T, N, H), device="cuda"), torch.empty((T, N, stride), device="cuda"), torch.empty((N, H), device="cuda")
+    gru.forward(d_x, stride, d_h0, d_dn, T, N, d_h)
+    gru.backward(d_dh, d_dx, stride, d_dh0)
+    torch.cuda.synchronize()
+    p = G.unpack_gru(setup["params"], D, H)
+    c = G.gru_sequence_forward(p, inputs["obs_actor"][:T], setup["h0"], inputs["dones"])
+    g = G.gru_sequence_backward(p, c, setup["dh"])
+    assert_close(d_h.cpu().numpy(), c["h"], 2e-5, "h")
+    assert_close(d_dx.cpu().numpy()[..., :D], g["x"], 1e-4, "dx")
+    assert_close(d_dh0.cpu().numpy(), g["h0"], 1e-4, "dh0")
+    assert_close(gru.get_grads(), G.flat_grads(g), 1e-4, "grad")
+    gru.destroy()

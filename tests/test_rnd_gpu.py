@@ -171,3 +171,30 @@ def test_intrinsic_reward_enters_gae_like_the_oracle():
         assert_close(got[k], want[k], 1e-4, k)
     rnd.destroy()
     ctx.destroy()
+
+
+def test_full_size_reward_and_first_step_match_oracle():
+    """The size the benchmark's distillation-reward task runs: 98,304 rows of rough_terrain observations, 48 selected
+    entries, nets 48-256-128-64-32; the reward of every row and the first predictor step (24,576-row minibatch)."""
+    import torch
+    from paper_2509_10771_b200 import binding
+    w = WL.ROUGH
+    T, N, Da = w.num_steps, w.num_envs, w.actor_obs_dim
+    B = T * N
+    setup = WL.make_rnd_setup(w, num_idx=48, hidden=(256, 128, 64), embed_dim=32)
+    obs = WL.make_rollout_inputs(w)["obs_actor"][:T].reshape(B, Da)
+    d_obs = torch.from_numpy(obs).to("cuda")
+    rnd = binding.Rnd(Da, setup["idx"], setup["hidden"], setup["embed_dim"], max_rows=B)
+    rnd.set_params(setup["predictor"], setup["target"])
+    d_int = torch.empty(B, device="cuda")
+    rnd.reward(d_obs, B, Da, d_r_int_out=d_int)
+    torch.cuda.synchronize()
+    ref, _, _, _ = O.rnd_reward(setup["predictor"], setup["target"], setup["dims"], obs, setup["idx"], 1.0)
+    assert_close(d_int.cpu().numpy(), ref, 1e-4, "r_int")
+    hp = SimpleNamespace(epochs=w.epochs, minibatches=w.minibatches, elu_alpha=1.0, adam_b1=0.9, adam_b2=0.999, adam_eps=1e-8)
+    out = rnd.update(d_obs, B, Da, w.epochs, w.minibatches, seed=w.seed, iteration=0, max_steps=1)
+    state = O.OptimState(setup["predictor"], 1e-3)
+    r = O.rnd_update(state, setup["target"], setup["dims"], obs, setup["idx"], hp, seed=w.seed, iteration=0, max_steps=1)
+    assert_close(out["first_loss"], r[0]["loss"], 1e-4, "loss")
+    assert_close(rnd.get_grads(), r[0]["grad"], 1e-4, "grad")
+    rnd.destroy()
