@@ -506,9 +506,10 @@ def run_rnd(args):
     total = sum(v["ms"] for v in prof.values()) or 1.0
     shares = {k: {"launches": v["launches"], "ms": round(v["ms"], 3), "share": round(v["ms"] / total, 4)}
               for k, v in sorted(prof.items(), key=lambda kv: -kv[1]["ms"])}
-    # FP32 multiply-adds of one iteration: 2 nets forward on B rows, then per training row 2 forwards + 2 backward products
+    # FP32 multiply-adds of one iteration: both nets forward on B rows for the reward, the target once more on B rows
+    # for the update, then per training row the predictor's forward and its two backward products
     mac = sum(fi * fo for fi, fo in setup["dims"])
-    flops = 2.0 * mac * (2 * B + w.epochs * B * (2 + 2))
+    flops = 2.0 * mac * (2 * B + B + w.epochs * B * 3)
     from types import SimpleNamespace
     from oracle import ppo_oracle as O
     rows_s = ORACLE_SAMPLE_ENVS * T

@@ -18,7 +18,7 @@ __global__ void __launch_bounds__(NT) sgemm_kernel(const GemmBatch batch) {
     constexpr int TM = BM / 16, TN = BN / 16;
     // z = problem * max_splits + split
     int max_splits = batch.p[0].splits;
-    if (batch.count > 1 && batch.p[1].splits > max_splits) max_splits = batch.p[1].splits;
+    for (int i = 1; i < batch.count; ++i) max_splits = max(max_splits, batch.p[i].splits);
     const int prob = blockIdx.z / max_splits;
     const int split = blockIdx.z % max_splits;
     const GemmProblem& g = batch.p[prob];

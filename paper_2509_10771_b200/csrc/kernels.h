@@ -53,8 +53,9 @@ struct GemmProblem {
     long long split_stride; // distance in floats between the C of consecutive splits
 };
 
+constexpr int kMaxGemmBatch = 8;
 struct GemmBatch {
-    GemmProblem p[2];
+    GemmProblem p[kMaxGemmBatch];
     int count;
     float alpha;            // ELU alpha
 };

@@ -38,10 +38,12 @@ __global__ void rnd_subset_kernel(const float* __restrict__ obs, int obs_stride,
 }
 
 // One warp per row: e = sum_j (f_j - g_j)^2 / E.
+//   g_rows != null: row r of f is compared with row g_rows[r] of g
 //   rewards != null:  rewards[r] += weight * e;  r_int != null: r_int[r] = e
 //   dout != null (training): dout[r][j] = 2 (f_j - g_j) * scale (scale = 1 / (rows E)), and the block's sum of e
 //   goes to loss_partials[block] (warps added in order)
-__global__ void __launch_bounds__(256) rnd_error_kernel(const float* __restrict__ f, const float* __restrict__ g, int ld,
+__global__ void __launch_bounds__(256) rnd_error_kernel(const float* __restrict__ f, const float* __restrict__ g,
+                                                        const int* __restrict__ g_rows, int ld,
                                                         int E, int n, float weight, float* __restrict__ rewards,
                                                         float* __restrict__ r_int, float* __restrict__ dout, float scale,
                                                         float* __restrict__ loss_partials) {
@@ -51,8 +53,9 @@ __global__ void __launch_bounds__(256) rnd_error_kernel(const float* __restrict_
     const int r = blockIdx.x * 8 + warp;
     float e = 0.f;
     if (r < n) {
+        const float* grow = g + (size_t)(g_rows ? g_rows[r] : r) * ld;       // the target's outputs may be stored per batch row
         for (int j = lane; j < E; j += 32) {
-            const float d = f[(size_t)r * ld + j] - g[(size_t)r * ld + j];
+            const float d = f[(size_t)r * ld + j] - grow[j];
             e += d * d;
             if (dout) dout[(size_t)r * ld + j] = 2.0f * d * scale;
         }
@@ -123,6 +126,7 @@ struct rslrl_rnd {
     float* loss_partials = nullptr; int max_loss_blocks = 0;
     float* step_loss = nullptr; int step_loss_cap = 0;
     int* perm = nullptr; size_t perm_cap = 0;
+    float* gall = nullptr; size_t gall_cap = 0;   // [batch][ldE] the target's outputs for every row of the batch
     long long adam_step = 0;
     std::string err;
 };
@@ -191,20 +195,22 @@ bool dalloc(rslrl_rnd* r, T** p, size_t count) {
 
 int splits_for(int rows) { return std::max(1, std::min(32, rows / 512)); }
 
-// both nets (or the predictor alone) through all layers on `rows` rows of r->s
-rslrl_status forward(rslrl_rnd* r, int rows, bool with_target) {
+// the predictor (do_f) and / or the target (do_g) through all layers on `rows` rows of r->s; g_last, if not
+// null, receives the target's last layer instead of the work buffer
+rslrl_status forward(rslrl_rnd* r, int rows, bool do_f, bool do_g, float* g_last) {
     const int nl = (int)r->L.size();
     for (int l = 0; l < nl; ++l) {
         const RLayer& Ly = r->L[l];
         GemmBatch b{};
         b.alpha = r->cfg.elu_alpha;
-        for (int net = 0; net < (with_target ? 2 : 1); ++net) {
+        for (int net = 0; net < 2; ++net) {
+            if (net == 0 ? !do_f : !do_g) continue;
             const float* par = net == 0 ? r->pf : r->pg;
             std::vector<float*>& h = net == 0 ? r->hf : r->hg;
             GemmProblem& p = b.p[b.count++];
             p.A = l == 0 ? r->s : h[l - 1]; p.lda = l == 0 ? r->lds : r->L[l - 1].ld;
             p.B = par + Ly.w_off; p.ldb = Ly.out_p;
-            p.C = h[l]; p.ldc = Ly.ld;
+            p.C = (net == 1 && l + 1 == nl && g_last) ? g_last : h[l]; p.ldc = Ly.ld;
             p.bias = par + Ly.b_off;
             p.M = rows; p.N = Ly.out; p.K = Ly.in; p.Cn = Ly.out_p;
             p.splits = 1; p.kchunk = round_up(Ly.in, 8); p.split_stride = 0;
@@ -223,37 +229,44 @@ rslrl_status subset(rslrl_rnd* r, const float* d_obs, int obs_stride, const int*
     return RSLRL_OK;
 }
 
-// gradients of the predictor from dz[last] (already filled) into r->partials
+// gradients of the predictor from dz[last] (already filled) into r->partials: first the chain of data
+// gradients, then the weight gradients of all layers in one launch and all bias gradients in another
 rslrl_status backward(rslrl_rnd* r, int rows, int splits, int kchunk) {
     const int nl = (int)r->L.size();
-    for (int l = nl - 1; l >= 0; --l) {
+    for (int l = nl - 1; l > 0; --l) {
         const RLayer& Ly = r->L[l];
+        GemmBatch dg{};
+        dg.alpha = r->cfg.elu_alpha;
+        GemmProblem& d = dg.p[dg.count++];
+        d.A = r->dz[l]; d.lda = Ly.ld;
+        d.B = r->pf + Ly.w_off; d.ldb = Ly.out_p;
+        d.C = r->dz[l - 1]; d.ldc = r->L[l - 1].ld;
+        d.aux = r->hf[l - 1]; d.ldaux = r->L[l - 1].ld;
+        d.M = rows; d.N = Ly.in; d.K = Ly.out; d.Cn = r->L[l - 1].ld;
+        d.splits = 1; d.kchunk = round_up(Ly.out, 8); d.split_stride = 0;
+        RCU(r, launch_sgemm(dg, false, true, EPI_DELU, r->stream));
+    }
+    for (int l0 = 0; l0 < nl; l0 += kMaxGemmBatch) {
         GemmBatch wg{};
-        GemmProblem& p = wg.p[wg.count++];
-        p.A = l == 0 ? r->s : r->hf[l - 1]; p.lda = l == 0 ? r->lds : r->L[l - 1].ld;
-        p.B = r->dz[l]; p.ldb = Ly.ld;
-        p.C = r->partials + Ly.w_off; p.ldc = Ly.out_p;
-        p.M = Ly.in; p.N = Ly.out; p.K = rows; p.Cn = Ly.out_p;
-        p.splits = splits; p.kchunk = kchunk; p.split_stride = r->P_dev;
+        for (int l = l0; l < std::min(nl, l0 + kMaxGemmBatch); ++l) {
+            const RLayer& Ly = r->L[l];
+            GemmProblem& p = wg.p[wg.count++];
+            p.A = l == 0 ? r->s : r->hf[l - 1]; p.lda = l == 0 ? r->lds : r->L[l - 1].ld;
+            p.B = r->dz[l]; p.ldb = Ly.ld;
+            p.C = r->partials + Ly.w_off; p.ldc = Ly.out_p;
+            p.M = Ly.in; p.N = Ly.out; p.K = rows; p.Cn = Ly.out_p;
+            p.splits = splits; p.kchunk = kchunk; p.split_stride = r->P_dev;
+        }
         RCU(r, launch_sgemm(wg, true, false, EPI_PLAIN, r->stream));
-        ColsumBatch cs{};
-        cs.splits = splits; cs.split_stride = r->P_dev; cs.is_bf16 = 0;
+    }
+    ColsumBatch cs{};
+    cs.splits = splits; cs.split_stride = r->P_dev; cs.is_bf16 = 0;
+    for (int l = 0; l < nl; ++l) {
+        const RLayer& Ly = r->L[l];
         ColsumProblem& q = cs.p[cs.count++];
         q.X = r->dz[l]; q.out = r->partials + Ly.b_off; q.rows = rows; q.n = Ly.out; q.ld = Ly.ld;
-        RCU(r, launch_colsum(cs, r->stream));
-        if (l > 0) {
-            GemmBatch dg{};
-            dg.alpha = r->cfg.elu_alpha;
-            GemmProblem& d = dg.p[dg.count++];
-            d.A = r->dz[l]; d.lda = Ly.ld;
-            d.B = r->pf + Ly.w_off; d.ldb = Ly.out_p;
-            d.C = r->dz[l - 1]; d.ldc = r->L[l - 1].ld;
-            d.aux = r->hf[l - 1]; d.ldaux = r->L[l - 1].ld;
-            d.M = rows; d.N = Ly.in; d.K = Ly.out; d.Cn = r->L[l - 1].ld;
-            d.splits = 1; d.kchunk = round_up(Ly.out, 8); d.split_stride = 0;
-            RCU(r, launch_sgemm(dg, false, true, EPI_DELU, r->stream));
-        }
     }
+    RCU(r, launch_colsum(cs, r->stream));
     return RSLRL_OK;
 }
 
@@ -360,11 +373,11 @@ rslrl_status rslrl_rnd_reward(rslrl_rnd* r, const float* d_obs, int32_t rows, in
     if (rows == 0 || (!d_rewards_inout && !d_r_int_out)) return RSLRL_OK;
     rslrl_status s = subset(r, d_obs, obs_stride, nullptr, rows);
     if (s != RSLRL_OK) return s;
-    s = forward(r, rows, true);
+    s = forward(r, rows, true, true, nullptr);
     if (s != RSLRL_OK) return s;
     LaunchScope scope_("rnd_error", r->stream);
     RCU(r, launch_chained(rnd_error_kernel, dim3((rows + 7) / 8), dim3(256), 0, r->stream, (const float*)r->hf.back(),
-                          (const float*)r->hg.back(), r->ldE, r->E, (int)rows, weight, d_rewards_inout, d_r_int_out,
+                          (const float*)r->hg.back(), (const int*)nullptr, r->ldE, r->E, (int)rows, weight, d_rewards_inout, d_r_int_out,
                           (float*)nullptr, 0.f, (float*)nullptr));
     return RSLRL_OK;
 }
@@ -389,7 +402,18 @@ rslrl_status rslrl_rnd_update(rslrl_rnd* r, const float* d_obs, int32_t batch, i
         if (!dalloc(r, &r->step_loss, (size_t)nsteps)) return rfail(r, RSLRL_ERR_CUDA, "could not allocate the loss buffer");
         r->step_loss_cap = (int)nsteps;
     }
+    if ((size_t)batch > r->gall_cap) {
+        if (!dalloc(r, &r->gall, (size_t)batch * r->ldE)) return rfail(r, RSLRL_ERR_CUDA, "could not allocate the target-output buffer");
+        r->gall_cap = (size_t)batch;
+    }
     RCU(r, launch_perm_epochs(seed, iteration, epochs, (uint32_t)batch, r->perm, r->stream));
+    // the target is fixed: its outputs for all rows of the batch are computed once and looked up by the steps
+    for (int r0 = 0; r0 < batch; r0 += r->max_rows) {
+        const int n = std::min(r->max_rows, batch - r0);
+        rslrl_status s = subset(r, d_obs + (size_t)r0 * obs_stride, obs_stride, nullptr, n);
+        if (s != RSLRL_OK) return s;
+        if ((s = forward(r, n, false, true, r->gall + (size_t)r0 * r->ldE)) != RSLRL_OK) return s;
+    }
     const int splits = splits_for(rows);
     const int kchunk = round_up((rows + splits - 1) / splits, 8);
     const int nloss = (rows + 7) / 8;
@@ -401,11 +425,11 @@ rslrl_status rslrl_rnd_update(rslrl_rnd* r, const float* d_obs, int32_t batch, i
             const int* rows_idx = r->perm + (size_t)e * batch + (size_t)k * rows;
             rslrl_status s = subset(r, d_obs, obs_stride, rows_idx, rows);
             if (s != RSLRL_OK) return s;
-            if ((s = forward(r, rows, true)) != RSLRL_OK) return s;
+            if ((s = forward(r, rows, true, false, nullptr)) != RSLRL_OK) return s;
             {
                 LaunchScope scope_("rnd_error", r->stream);
                 RCU(r, launch_chained(rnd_error_kernel, dim3(nloss), dim3(256), 0, r->stream, (const float*)r->hf.back(),
-                                      (const float*)r->hg.back(), r->ldE, r->E, rows, 0.f, (float*)nullptr, (float*)nullptr,
+                                      (const float*)r->gall, rows_idx, r->ldE, r->E, rows, 0.f, (float*)nullptr, (float*)nullptr,
                                       r->dz.back(), scale, r->loss_partials));
             }
             if ((s = backward(r, rows, splits, kchunk)) != RSLRL_OK) return s;
