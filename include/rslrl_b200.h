@@ -341,7 +341,7 @@ rslrl_status rslrl_rnd_update(rslrl_rnd *rnd, const float *d_obs, int32_t batch,
  * management of hidden states across rollouts and back-propagation through time).
  *
  * A GRU layer over a time-major rollout.  Per step t (gate order r, z, n):
- *   h_in(t) = h0 for t = 0, else (1 - done[t-1]) * h(t-1)      (same-step reset: zero state after done)
+ *   h_in(t) = (1 - reset) * h0 for t = 0, else (1 - done[t-1]) * h(t-1)   (same-step reset: zero state after done)
  *   r = sigmoid(x_t W_ir + b_ir + h_in W_hr + b_hr),  z likewise,
  *   n = tanh(x_t W_in + b_in + r * (h_in W_hn + b_hn)),  h(t) = (1 - z) n + z h_in
  * The paper names neither the cell nor the reset rule; these are this library's choices.
@@ -366,13 +366,17 @@ rslrl_status rslrl_gru_get_grads(rslrl_gru *gru, float *h_grad, size_t n);      
 
 /* Forward over T steps of N environments (device pointers, float buffers 16-byte aligned):
  *   d_x [T][N][x_stride] (x_stride a multiple of 4, >= D rounded up to 4; padding is not read as data),
- *   d_h0 [N][H] the state entering step 0, d_dones [T][N] uint8, d_h_out [T][N][H] = h(t).
- * d_x and d_dones must stay unchanged until rslrl_gru_backward has run.  Only enqueues. */
+ *   d_h0 [N][H] the state carried in, d_h0_reset [N] uint8 (may be NULL): environments whose step before
+ *   this call reported done and therefore start from the zero state (with it, T calls of one step each
+ *   give the states of one call of T steps), d_dones [T][N] uint8, d_h_out [T][N][H] = h(t).
+ * d_x, d_dones and d_h0_reset must stay unchanged until rslrl_gru_backward has run.  Only enqueues. */
 rslrl_status rslrl_gru_forward(rslrl_gru *gru, const float *d_x, int32_t x_stride, const float *d_h0,
-                               const uint8_t *d_dones, int32_t T, int32_t N, float *d_h_out);
+                               const uint8_t *d_h0_reset, const uint8_t *d_dones, int32_t T, int32_t N,
+                               float *d_h_out);
 
 /* Back-propagation through the T steps of the last forward for L = sum_t <d_dh[t], h(t)>:
- *   d_dh [T][N][H]; d_dx [T][N][dx_stride] (may be NULL) = dL/dx; d_dh0 [N][H] (may be NULL) = dL/dh0;
+ *   d_dh [T][N][H]; d_dx [T][N][dx_stride] (may be NULL) = dL/dx; d_dh0 [N][H] (may be NULL) = dL/dh0
+ *   (zero in the rows d_h0_reset flagged);
  * the parameter gradient is kept in the object (rslrl_gru_get_grads).  No gradient crosses a reset.
  * One backward per forward: RSLRL_ERR_STATE otherwise.  Only enqueues. */
 rslrl_status rslrl_gru_backward(rslrl_gru *gru, const float *d_dh, float *d_dx, int32_t dx_stride, float *d_dh0);

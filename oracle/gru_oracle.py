@@ -14,7 +14,8 @@ The paper names the feature but neither the cell nor the reset rule, so the read
     with W_i = [W_ir | W_iz | W_in] of shape [D][3H] and W_h = [W_hr | W_hz | W_hn] of shape [H][3H];
   * sequences are time-major, x[T][N][D]; the state entering step 0 is h0[N][H] (carried over from the
     previous rollout by the caller); with same-step resets an environment that reports done at step t
-    starts step t + 1 from the zero state: h_in(t) = (1 - done[t-1]) * h(t-1) for t >= 1;
+    starts step t + 1 from the zero state: h_in(t) = (1 - done[t-1]) * h(t-1) for t >= 1; the same rule at
+    the seam between two calls is an optional flag vector that zeroes carried-in states;
   * back-propagation runs through all T steps of the rollout and stops where the state was reset
     (the factor (1 - done) carries that), and it returns the gradient with respect to h0.
 
@@ -24,7 +25,7 @@ one-step closed form, and independence of everything after a reset from everythi
 """
 from __future__ import annotations
 
-from typing import Dict
+from typing import Dict, Optional
 
 import numpy as np
 
@@ -45,12 +46,17 @@ def unpack_gru(flat: np.ndarray, D: int, H: int) -> Dict[str, np.ndarray]:
             "W_h": flat[o[2]:o[3]].reshape(H, 3 * H), "b_h": flat[o[3]:o[4]]}
 
 
-def gru_sequence_forward(p: Dict[str, np.ndarray], x: np.ndarray, h0: np.ndarray, dones: np.ndarray) -> Dict[str, np.ndarray]:
-    """h[T][N][H] (the state after every step) and what the backward pass needs."""
+def gru_sequence_forward(p: Dict[str, np.ndarray], x: np.ndarray, h0: np.ndarray, dones: np.ndarray,
+                         h0_reset: Optional[np.ndarray] = None) -> Dict[str, np.ndarray]:
+    """h[T][N][H] (the state after every step) and what the backward pass needs.  ``h0_reset[N]`` (optional) marks
+    environments whose step before this sequence reported done: their carried-in state is replaced by zero, which
+    is what makes a rollout taken one step per call equal to the same rollout taken in one call."""
     x = np.asarray(x, dtype=F64); h0 = np.asarray(h0, dtype=F64)
     T, N, _ = x.shape
     H = h0.shape[1]
     keep = 1.0 - np.asarray(dones, dtype=F64)                    # [T][N]
+    keep0 = np.ones(N) if h0_reset is None else 1.0 - np.asarray(h0_reset, dtype=F64)
+    h0 = keep0[:, None] * h0
     out = {k: np.zeros((T, N, H)) for k in ("h", "h_in", "r", "z", "n", "gh_n")}
     h = h0
     for t in range(T):
@@ -65,6 +71,7 @@ def gru_sequence_forward(p: Dict[str, np.ndarray], x: np.ndarray, h0: np.ndarray
             out[k][t] = v
     out["x"] = x
     out["keep"] = keep
+    out["keep0"] = keep0
     return out
 
 
@@ -89,7 +96,7 @@ def gru_sequence_backward(p: Dict[str, np.ndarray], c: Dict[str, np.ndarray], dh
         g["x"][t] = dgi @ p["W_i"].T
         dh_in = dh * z + dgh @ p["W_h"].T
         carry = dh_in if t == 0 else c["keep"][t - 1][:, None] * dh_in
-    g["h0"] = carry
+    g["h0"] = c["keep0"][:, None] * carry
     return g
 
 

@@ -156,7 +156,7 @@ def load_library() -> C.CDLL:
         "rslrl_gru_last_error": (C.c_char_p, [vp]),
         "rslrl_gru_set_params": (i32, [vp, vp, sz]),
         "rslrl_gru_get_grads": (i32, [vp, vp, sz]),
-        "rslrl_gru_forward": (i32, [vp, vp, i32, vp, vp, i32, i32, vp]),
+        "rslrl_gru_forward": (i32, [vp, vp, i32, vp, vp, vp, i32, i32, vp]),
         "rslrl_gru_backward": (i32, [vp, vp, vp, i32, vp]),
     }
     for name, (res, args) in sig.items():
@@ -428,8 +428,9 @@ class Gru:
         self._check(self.lib.rslrl_gru_get_grads(self.handle, out.ctypes.data, out.size))
         return out
 
-    def forward(self, d_x, x_stride: int, d_h0, d_dones, T: int, N: int, d_h_out):
-        self._check(self.lib.rslrl_gru_forward(self.handle, _ptr(d_x), x_stride, _ptr(d_h0), _ptr(d_dones), T, N, _ptr(d_h_out)))
+    def forward(self, d_x, x_stride: int, d_h0, d_dones, T: int, N: int, d_h_out, d_h0_reset=None):
+        self._check(self.lib.rslrl_gru_forward(self.handle, _ptr(d_x), x_stride, _ptr(d_h0), _ptr(d_h0_reset), _ptr(d_dones),
+                                               T, N, _ptr(d_h_out)))
 
     def backward(self, d_dh, d_dx=None, dx_stride: int = 0, d_dh0=None):
         self._check(self.lib.rslrl_gru_backward(self.handle, _ptr(d_dh), _ptr(d_dx), dx_stride, _ptr(d_dh0)))

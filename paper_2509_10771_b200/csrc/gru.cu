@@ -68,10 +68,20 @@ __global__ void __launch_bounds__(256) gru_gate_bwd_kernel(float* __restrict__ r
     dhz[i] = dh * z;
 }
 
-__global__ void gru_add_kernel(const float* __restrict__ a, const float* __restrict__ b, float* __restrict__ out, int n) {
+// out = a + b, zero in the rows flagged by reset (may be null)
+__global__ void gru_add_kernel(const float* __restrict__ a, const float* __restrict__ b, const uint8_t* __restrict__ reset,
+                               float* __restrict__ out, int N, int H) {
     chain_begin();
     const int i = blockIdx.x * blockDim.x + threadIdx.x;
-    if (i < n) out[i] = a[i] + b[i];
+    if (i < N * H) out[i] = (reset && reset[i / H]) ? 0.f : a[i] + b[i];
+}
+
+// h_in(0) = h0, zero in the rows flagged by reset (may be null)
+__global__ void gru_init_state_kernel(const float* __restrict__ h0, const uint8_t* __restrict__ reset, float* __restrict__ h_in,
+                                      int N, int H) {
+    chain_begin();
+    const int i = blockIdx.x * blockDim.x + threadIdx.x;
+    if (i < N * H) h_in[i] = (reset && reset[i / H]) ? 0.f : h0[i];
 }
 
 __global__ void gru_reduce_kernel(const float* __restrict__ partials, int splits, size_t stride, float* __restrict__ grad, int P) {
@@ -94,7 +104,8 @@ struct rslrl_gru {
     float *param = nullptr, *grad = nullptr, *partials = nullptr;
     float *gi = nullptr, *gh = nullptr, *hin = nullptr, *dhz = nullptr, *tmp = nullptr;
     // what the last forward saw (backward reads them again)
-    const float* x = nullptr; int x_stride = 0; const uint8_t* dones = nullptr; int T = 0, N = 0;
+    const float* x = nullptr; int x_stride = 0; const uint8_t* dones = nullptr; const uint8_t* h0_reset = nullptr;
+    int T = 0, N = 0;
     bool forward_done = false;
     std::string err;
 };
@@ -205,8 +216,8 @@ rslrl_status rslrl_gru_get_grads(rslrl_gru* g, float* h, size_t n) {
     return RSLRL_OK;
 }
 
-rslrl_status rslrl_gru_forward(rslrl_gru* g, const float* d_x, int32_t x_stride, const float* d_h0, const uint8_t* d_dones,
-                               int32_t T, int32_t N, float* d_h_out) {
+rslrl_status rslrl_gru_forward(rslrl_gru* g, const float* d_x, int32_t x_stride, const float* d_h0, const uint8_t* d_h0_reset,
+                               const uint8_t* d_dones, int32_t T, int32_t N, float* d_h_out) {
     if (!g || !d_x || !d_h0 || !d_dones || !d_h_out) return RSLRL_ERR_INVALID_ARG;
     if (T < 1 || N < 1) return gfail(g, RSLRL_ERR_INVALID_ARG, "T and N must be positive");
     if (T > g->max_T || N > g->max_N) return gfail(g, RSLRL_ERR_UNSUPPORTED, "T = %d, N = %d exceed max_steps = %d, max_envs = %d", T, N, g->max_T, g->max_N);
@@ -224,8 +235,11 @@ rslrl_status rslrl_gru_forward(rslrl_gru* g, const float* d_x, int32_t x_stride,
         p.splits = 1; p.kchunk = round_up(D, 8); p.split_stride = 0;
         GCU(g, launch_sgemm(b, false, false, EPI_BIAS, g->stream));
     }
-    GCU(g, cudaMemcpyAsync(g->hin, d_h0, sizeof(float) * (size_t)N * H, cudaMemcpyDeviceToDevice, g->stream));
     const int blocks = (N * H + 255) / 256;
+    {
+        LaunchScope scope_("gru_init_state", g->stream);
+        GCU(g, launch_chained(gru_init_state_kernel, dim3(blocks), dim3(256), 0, g->stream, d_h0, d_h0_reset, g->hin, (int)N, H));
+    }
     for (int t = 0; t < T; ++t) {
         float* gi_t = g->gi + (size_t)t * N * G3;
         float* gh_t = g->gh + (size_t)t * N * G3;
@@ -241,7 +255,7 @@ rslrl_status rslrl_gru_forward(rslrl_gru* g, const float* d_x, int32_t x_stride,
                               d_dones + (size_t)t * N, d_h_out + (size_t)t * N * H,
                               t + 1 < T ? g->hin + (size_t)(t + 1) * N * H : (float*)nullptr, (int)N, H));
     }
-    g->x = d_x; g->x_stride = x_stride; g->dones = d_dones; g->T = T; g->N = N;
+    g->x = d_x; g->x_stride = x_stride; g->dones = d_dones; g->h0_reset = d_h0_reset; g->T = T; g->N = N;
     g->forward_done = true;
     return RSLRL_OK;
 }
@@ -273,7 +287,7 @@ rslrl_status rslrl_gru_backward(rslrl_gru* g, const float* d_dh, float* d_dx, in
     }
     if (d_dh0) {
         LaunchScope scope_("gru_add", g->stream);
-        GCU(g, launch_chained(gru_add_kernel, dim3(blocks), dim3(256), 0, g->stream, (const float*)g->dhz, (const float*)g->tmp, d_dh0, N * H));
+        GCU(g, launch_chained(gru_add_kernel, dim3(blocks), dim3(256), 0, g->stream, (const float*)g->dhz, (const float*)g->tmp, g->h0_reset, d_dh0, N, H));
     }
     if (d_dx) {
         GemmBatch b{};

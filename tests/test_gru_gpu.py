@@ -166,3 +166,43 @@ def test_full_size_rollout_matches_oracle():
     assert_close(d_dh0.cpu().numpy(), g["h0"], 1e-4, "dh0")
     assert_close(gru.get_grads(), G.flat_grads(g), 1e-4, "grad")
     gru.destroy()
+
+
+def test_rollout_taken_step_by_step_equals_the_rollout_taken_at_once():
+    """Acting uses the layer one step per call: the state comes back in with the previous step's done flags as the
+    reset vector.  The states equal those of the single T-step call up to FP32 rounding (the input product runs
+    with a different tile shape when all steps are batched), the flagged form matches the oracle, and the gradient with respect to a flagged carried-in state is exactly zero."""
+    import torch
+    from dataclasses import replace
+    from paper_2509_10771_b200 import binding
+    w = replace(WL.FLAT.scaled(130), done_prob=0.1)
+    T, N, D, H = w.num_steps, w.num_envs, w.actor_obs_dim, 64
+    inputs = WL.make_rollout_inputs(w)
+    setup = WL.make_gru_setup(w, hidden_dim=H)
+    x, dones = inputs["obs_actor"][:T], inputs["dones"]
+    gru = binding.Gru(D, H, T, N)
+    gru.set_params(setup["params"])
+    d_x, d_dn = torch.from_numpy(x).to("cuda"), torch.from_numpy(dones).to("cuda")
+    d_h0 = torch.from_numpy(setup["h0"]).to("cuda")
+    whole = torch.empty((T, N, H), device="cuda")
+    gru.forward(d_x, D, d_h0, d_dn, T, N, whole)
+    steps = torch.empty((T, N, H), device="cuda")
+    for t in range(T):
+        gru.forward(d_x[t], D, d_h0 if t == 0 else steps[t - 1], d_dn[t], 1, N, steps[t],
+                    d_h0_reset=None if t == 0 else d_dn[t - 1])
+    torch.cuda.synchronize()
+    assert float((whole - steps).abs().max()) <= 2e-6
+    flags = (np.arange(N) % 3 == 0).astype(np.uint8)
+    d_flags = torch.from_numpy(flags).to("cuda")
+    d_h, d_dh0 = torch.empty((T, N, H), device="cuda"), torch.empty((N, H), device="cuda")
+    gru.forward(d_x, D, d_h0, d_dn, T, N, d_h, d_h0_reset=d_flags)
+    gru.backward(torch.from_numpy(setup["dh"]).to("cuda"), None, 0, d_dh0)
+    torch.cuda.synchronize()
+    p = G.unpack_gru(setup["params"], D, H)
+    c = G.gru_sequence_forward(p, x, setup["h0"], dones, h0_reset=flags)
+    g = G.gru_sequence_backward(p, c, setup["dh"])
+    assert_close(d_h.cpu().numpy(), c["h"], 2e-5, "h")
+    assert_close(d_dh0.cpu().numpy(), g["h0"], 1e-4, "dh0")
+    assert np.all(d_dh0.cpu().numpy()[flags == 1] == 0.0)
+    assert_close(gru.get_grads(), G.flat_grads(g), 1e-4, "grad")
+    gru.destroy()

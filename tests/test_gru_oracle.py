@@ -142,3 +142,24 @@ def test_nothing_crosses_a_reset():
     d_last = dones.copy(); d_last[-1, :] = 1
     c = G.gru_sequence_forward(p, x, h0, d_last)
     assert np.array_equal(c["h"], a["h"])
+
+
+def test_a_rollout_taken_step_by_step_equals_the_rollout_taken_at_once():
+    """T calls of one step each, every call carrying the previous state in and flagging the environments whose
+    previous step was done, give the states of the single T-step call; and the gradient with respect to a
+    flagged carried-in state is zero."""
+    flat, x, h0, dones, dh = problem(seed=7, T=6, N=5, D=4, H=3, done_prob=0.4)
+    D, H = 4, 3
+    p = G.unpack_gru(flat, D, H)
+    whole = G.gru_sequence_forward(p, x, h0, dones)
+    h, prev_done = h0, np.zeros(5, np.uint8)
+    for t in range(6):
+        c = G.gru_sequence_forward(p, x[t:t + 1], h, dones[t:t + 1], h0_reset=prev_done)
+        h, prev_done = c["h"][0], dones[t]
+        np.testing.assert_allclose(h, whole["h"][t], rtol=1e-13, atol=1e-14)
+    flags = np.array([1, 0, 0, 1, 0], np.uint8)
+    c = G.gru_sequence_forward(p, x, h0, dones, h0_reset=flags)
+    g = G.gru_sequence_backward(p, c, dh)
+    assert np.all(g["h0"][flags == 1] == 0.0) and np.all(np.abs(g["h0"][flags == 0]).sum(axis=1) > 0)
+    h0z = h0.copy(); h0z[flags == 1] = 0.0
+    np.testing.assert_array_equal(c["h"], G.gru_sequence_forward(p, x, h0z, dones)["h"])
