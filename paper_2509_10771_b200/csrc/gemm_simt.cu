@@ -220,11 +220,19 @@ cudaError_t launch_tiles(const GemmBatch& b, bool ta, bool tb, int epi, cudaStre
 
 }  // namespace
 
+// Tile shape: the one with the smallest estimated time.  The SM that gets the most tiles decides the time of a
+// launch, so the estimate is ceil(tiles / SMs) x tile area / efficiency; the efficiencies (share of the FMA
+// rate a tile shape can reach: smaller tiles read more shared memory per multiply-add) are measured ratios.
 cudaError_t launch_sgemm(const GemmBatch& b, bool ta, bool tb, int epi, cudaStream_t s) {
-    long long tiles128 = 0;
-    for (int i = 0; i < b.count; ++i)
-        tiles128 += (long long)((b.p[i].M + 127) / 128) * ((b.p[i].Cn + 127) / 128) * b.p[i].splits;
-    if (tiles128 >= 2 * 148) return launch_tiles<128, 128>(b, ta, tb, epi, s);
+    auto cost = [&](int bm, int bn, double eff) {
+        long long tiles = 0;
+        for (int i = 0; i < b.count; ++i)
+            tiles += (long long)((b.p[i].M + bm - 1) / bm) * ((b.p[i].Cn + bn - 1) / bn) * b.p[i].splits;
+        return (double)((tiles + 147) / 148) * bm * bn / eff;
+    };
+    const double c128 = cost(128, 128, 1.0), c12864 = cost(128, 64, 0.85), c64 = cost(64, 64, 0.55);
+    if (c128 <= c12864 && c128 <= c64) return launch_tiles<128, 128>(b, ta, tb, epi, s);
+    if (c12864 <= c64) return launch_tiles<128, 64>(b, ta, tb, epi, s);
     return launch_tiles<64, 64>(b, ta, tb, epi, s);
 }
 
