@@ -22,6 +22,10 @@ namespace {
 
 inline int round_up(int x, int m) { return (x + m - 1) / m * m; }
 
+// d h_in = d gh W_h^T has few output tiles and a K range of 3H: it is computed as kTmpSplits partial products
+// over thirds of that range, which the consumers add in a fixed order
+constexpr int kTmpSplits = 3;
+
 __device__ __forceinline__ float sigmoid_f(float a) { return 1.0f / (1.0f + expf(-a)); }
 
 // Step t, one thread per (row, j).  gi/gh: [N][3H] pre-activations of this step; on return gi holds (r, z, n).
@@ -46,11 +50,11 @@ __global__ void __launch_bounds__(256) gru_gate_kernel(float* __restrict__ gi, c
 }
 
 // Step t of the reverse pass.  rzn: (r, z, n) of the step, replaced by d gi; gh: third block holds gh_n, replaced by d gh.
-// dh = dh_seq + (carry_done ? (carry_done[row] ? 0 : dhz + tmp) : 0); dhz <- dh * z.
+// dh = dh_seq + (carry_done ? (carry_done[row] ? 0 : dhz + sum of the tmp slabs) : 0); dhz <- dh * z.
 __global__ void __launch_bounds__(256) gru_gate_bwd_kernel(float* __restrict__ rzn, float* __restrict__ gh,
                                                            const float* __restrict__ h_in, const float* __restrict__ dh_seq,
                                                            const uint8_t* __restrict__ carry_done, float* __restrict__ dhz,
-                                                           const float* __restrict__ tmp, int N, int H) {
+                                                           const float* __restrict__ tmp, size_t tmp_stride, int N, int H) {
     chain_begin();
     const int i = blockIdx.x * blockDim.x + threadIdx.x;
     if (i >= N * H) return;
@@ -58,7 +62,12 @@ __global__ void __launch_bounds__(256) gru_gate_bwd_kernel(float* __restrict__ r
     float* a = rzn + (size_t)row * 3 * H;
     float* b = gh + (size_t)row * 3 * H;
     float dh = dh_seq[i];
-    if (carry_done && !carry_done[row]) dh += dhz[i] + tmp[i];
+    if (carry_done && !carry_done[row]) {
+        float back = tmp[i];
+#pragma unroll
+        for (int k = 1; k < kTmpSplits; ++k) back += tmp[i + k * tmp_stride];
+        dh += dhz[i] + back;
+    }
     const float r = a[j], z = a[H + j], n = a[2 * H + j], ghn = b[2 * H + j], hp = h_in[i];
     const float da_n = dh * (1.0f - z) * (1.0f - n * n);
     const float da_z = dh * (hp - n) * z * (1.0f - z);
@@ -68,12 +77,16 @@ __global__ void __launch_bounds__(256) gru_gate_bwd_kernel(float* __restrict__ r
     dhz[i] = dh * z;
 }
 
-// out = a + b, zero in the rows flagged by reset (may be null)
-__global__ void gru_add_kernel(const float* __restrict__ a, const float* __restrict__ b, const uint8_t* __restrict__ reset,
-                               float* __restrict__ out, int N, int H) {
+// out = a + (sum of the slabs of b), zero in the rows flagged by reset (may be null)
+__global__ void gru_add_kernel(const float* __restrict__ a, const float* __restrict__ b, size_t b_stride,
+                               const uint8_t* __restrict__ reset, float* __restrict__ out, int N, int H) {
     chain_begin();
     const int i = blockIdx.x * blockDim.x + threadIdx.x;
-    if (i < N * H) out[i] = (reset && reset[i / H]) ? 0.f : a[i] + b[i];
+    if (i >= N * H) return;
+    float back = b[i];
+#pragma unroll
+    for (int k = 1; k < kTmpSplits; ++k) back += b[i + k * b_stride];
+    out[i] = (reset && reset[i / H]) ? 0.f : a[i] + back;
 }
 
 // h_in(0) = h0, zero in the rows flagged by reset (may be null)
@@ -188,7 +201,7 @@ rslrl_status rslrl_gru_create(const rslrl_gru_cfg* cfg, void* cuda_stream, rslrl
     const bool ok = dalloc(g, &g->param, (size_t)g->P) && dalloc(g, &g->grad, (size_t)g->P) &&
                     dalloc(g, &g->partials, (size_t)g->P * g->max_splits) && dalloc(g, &g->gi, rows * 3 * H) &&
                     dalloc(g, &g->gh, rows * 3 * H) && dalloc(g, &g->hin, rows * H) &&
-                    dalloc(g, &g->dhz, (size_t)g->max_N * H) && dalloc(g, &g->tmp, (size_t)g->max_N * H) &&
+                    dalloc(g, &g->dhz, (size_t)g->max_N * H) && dalloc(g, &g->tmp, (size_t)kTmpSplits * g->max_N * H) &&
                     cudaStreamSynchronize(g->stream) == cudaSuccess;
     if (!ok) {
         g_gru_create_error = std::string("device allocation failed: ") + cudaGetErrorString(cudaGetLastError());
@@ -276,18 +289,20 @@ rslrl_status rslrl_gru_backward(rslrl_gru* g, const float* d_dh, float* d_dx, in
             LaunchScope scope_("gru_gate_bwd", g->stream);
             GCU(g, launch_chained(gru_gate_bwd_kernel, dim3(blocks), dim3(256), 0, g->stream, gi_t, gh_t,
                                   (const float*)(g->hin + (size_t)t * N * H), d_dh + (size_t)t * N * H,
-                                  t + 1 < T ? g->dones + (size_t)t * N : (const uint8_t*)nullptr, g->dhz, (const float*)g->tmp, N, H));
+                                  t + 1 < T ? g->dones + (size_t)t * N : (const uint8_t*)nullptr, g->dhz, (const float*)g->tmp,
+                                  (size_t)g->max_N * H, N, H));
         }
         // tmp = d gh W_h^T
         GemmBatch b{};
         GemmProblem& p = b.p[b.count++];
         p.A = gh_t; p.lda = G3; p.B = g->param + g->off_wh; p.ldb = G3; p.C = g->tmp; p.ldc = H;
-        p.M = N; p.N = H; p.K = G3; p.Cn = H; p.splits = 1; p.kchunk = round_up(G3, 8); p.split_stride = 0;
+        p.M = N; p.N = H; p.K = G3; p.Cn = H;
+        p.splits = kTmpSplits; p.kchunk = round_up((G3 + kTmpSplits - 1) / kTmpSplits, 8); p.split_stride = (long long)g->max_N * H;
         GCU(g, launch_sgemm(b, false, true, EPI_PLAIN, g->stream));
     }
     if (d_dh0) {
         LaunchScope scope_("gru_add", g->stream);
-        GCU(g, launch_chained(gru_add_kernel, dim3(blocks), dim3(256), 0, g->stream, (const float*)g->dhz, (const float*)g->tmp, g->h0_reset, d_dh0, N, H));
+        GCU(g, launch_chained(gru_add_kernel, dim3(blocks), dim3(256), 0, g->stream, (const float*)g->dhz, (const float*)g->tmp, (size_t)g->max_N * H, g->h0_reset, d_dh0, N, H));
     }
     if (d_dx) {
         GemmBatch b{};
