@@ -354,7 +354,7 @@ typedef struct {
     int32_t input_dim;                  /* D >= 1                                                    */
     int32_t hidden_dim;                 /* H, a multiple of 4                                        */
     int32_t max_steps;                  /* largest T                                                 */
-    int32_t max_envs;                   /* largest N                                                 */
+    int32_t max_envs;                   /* largest N; T * N < 2^30 and N * 3H < 2^31                 */
 } rslrl_gru_cfg;
 
 size_t       rslrl_gru_num_params(const rslrl_gru_cfg *cfg);      /* 0 if cfg is invalid             */

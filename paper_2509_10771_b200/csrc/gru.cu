@@ -148,6 +148,7 @@ bool valid_cfg(const rslrl_gru_cfg* c, std::string* why) {
     if (c->hidden_dim < 4 || c->hidden_dim > 4096 || c->hidden_dim % 4) return bad("hidden_dim must be a multiple of 4 in [4, 4096]");
     if (c->max_steps < 1 || c->max_envs < 1) return bad("max_steps and max_envs must be positive");
     if ((long long)c->max_steps * c->max_envs >= (1ll << 30)) return bad("max_steps * max_envs must be below 2^30");
+    if ((long long)c->max_envs * 3 * c->hidden_dim >= (1ll << 31)) return bad("max_envs * 3 * hidden_dim must be below 2^31");
     return true;
 }
 

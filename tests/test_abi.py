@@ -56,3 +56,28 @@ def test_num_params_and_config_validation_without_a_device():
     assert lib.rslrl_gae_scan(None, None, None, None, None, None, None, 0, 0, 0.99, 0.95, 1, 1, 1e-8, None, None) == 0
     assert lib.rslrl_gae_scan(None, None, None, None, None, None, None, 4, 4, 0.99, 0.95, 1, 1, 1e-8, None, None) == 1
     assert lib.rslrl_minibatch_indices(0, 0, 0, 10, 3, 0, None, None) == 2
+
+
+def test_rnd_and_gru_configs_without_a_device():
+    """Parameter counts and config validation of the two side objects are host-only code."""
+    import numpy as np
+    from paper_2509_10771_b200 import binding, build
+    build.build()
+    lib = binding.load_library()
+    idx = np.array([0, 3, 5], dtype=np.int32)
+    cfg = binding.RndCfg()
+    cfg.obs_dim, cfg.num_idx, cfg.h_idx, cfg.num_hidden = 8, 3, idx.ctypes.data, 2
+    cfg.hidden[0], cfg.hidden[1] = 16, 8
+    cfg.embed_dim, cfg.elu_alpha, cfg.max_rows = 4, 1.0, 64
+    cfg.lr, cfg.adam_b1, cfg.adam_b2, cfg.adam_eps = 1e-3, 0.9, 0.999, 1e-8
+    assert lib.rslrl_rnd_num_params(ctypes.byref(cfg)) == 3 * 16 + 16 + 16 * 8 + 8 + 8 * 4 + 4
+    cfg.num_idx = 9                                    # more selected entries than the observation has
+    assert lib.rslrl_rnd_num_params(ctypes.byref(cfg)) == 0
+    cfg.num_idx, cfg.lr = 3, 0.0
+    assert lib.rslrl_rnd_num_params(ctypes.byref(cfg)) == 0
+    assert ctypes.sizeof(binding.RndCfg) == 4 + 4 + 8 + 4 + 32 + 4 + 4 + 4 + 16 and binding.RndCfg.h_idx.offset == 8
+    g = binding.GruCfg(235, 256, 24, 4096)
+    assert lib.rslrl_gru_num_params(ctypes.byref(g)) == 235 * 768 + 768 + 256 * 768 + 768
+    assert lib.rslrl_gru_num_params(ctypes.byref(binding.GruCfg(235, 250, 24, 4096))) == 0     # H not a multiple of 4
+    assert lib.rslrl_gru_num_params(ctypes.byref(binding.GruCfg(235, 256, 1 << 15, 1 << 15))) == 0   # T * N too large
+    assert ctypes.sizeof(binding.GruCfg) == 16
