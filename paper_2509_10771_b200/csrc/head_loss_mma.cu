@@ -47,7 +47,7 @@ __device__ __forceinline__ float quad_sum(float v) {
 // NT = number of 8-wide action tiles (actions padded to 8 * NT, NT even).
 // CS: also emit the block's column sums of dZa / dZc (partial bias gradients of the last hidden layers).
 template <int NT, bool CS>
-__global__ void __launch_bounds__(kThreads) head_loss_mma_kernel(const HeadLossArgs a) {
+__global__ void __launch_bounds__(kThreads, NT <= 6 ? 3 : 2) head_loss_mma_kernel(const HeadLossArgs a) {
     constexpr int AP = 8 * NT;
     extern __shared__ __align__(16) uint8_t smem_raw[];
     chain_begin();
