@@ -629,9 +629,6 @@ __global__ void __launch_bounds__(kAdamThreads) adam_kernel(const AdamArgs a) {
             }
             s_scal[0] = fminf(1.0f, a.max_norm / (gnorm + 1e-6f));
             s_scal[1] = lr;
-            // 1 - b^step in double: exact enough for any step count, computed once per block
-            s_scal[2] = (float)(1.0 / (1.0 - pow((double)a.b1, (double)step)));
-            s_scal[3] = (float)(1.0 / (1.0 - pow((double)a.b2, (double)step)));
             s_skip = finite ? 0 : 1;
             if (blockIdx.x == 0) {
                 a.lr_io[a.parity ^ 1] = lr;
@@ -642,6 +639,12 @@ __global__ void __launch_bounds__(kAdamThreads) adam_kernel(const AdamArgs a) {
                 a.stats_row[7] = finite ? 0.f : 1.f;
             }
         }
+    } else if (threadIdx.x == 32 || threadIdx.x == 64) {
+        // 1 - b^step in double: exact enough for any step count; one thread of two other warps each, so that
+        // the two powers run beside the norm instead of after it
+        const int step = a.step_io[a.parity] + 1;
+        const double b = threadIdx.x == 32 ? (double)a.b1 : (double)a.b2;
+        s_scal[threadIdx.x == 32 ? 2 : 3] = (float)(1.0 / (1.0 - pow(b, (double)step)));
     }
     __syncthreads();
     if (s_skip) return;          // non-finite step: parameters and moments stay untouched
