@@ -206,3 +206,34 @@ def test_rollout_taken_step_by_step_equals_the_rollout_taken_at_once():
     assert np.all(d_dh0.cpu().numpy()[flags == 1] == 0.0)
     assert_close(gru.get_grads(), G.flat_grads(g), 1e-4, "grad")
     gru.destroy()
+
+
+@pytest.mark.parametrize("T,N,D,H", [(1, 1, 1, 4), (3, 5, 7, 12), (32, 33, 9, 20)])
+def test_smallest_and_odd_shapes(T, N, D, H):
+    """One step of one environment with one input, and shapes that are multiples of nothing."""
+    import torch
+    from paper_2509_10771_b200 import binding
+    rng = np.random.default_rng(T * 100 + N)
+    n = D * 3 * H + 3 * H + H * 3 * H + 3 * H
+    params = (rng.standard_normal(n) * 0.4).astype(np.float32)
+    stride = (D + 3) // 4 * 4
+    x = rng.standard_normal((T, N, D)).astype(np.float32)
+    xp = np.zeros((T, N, stride), np.float32); xp[..., :D] = x
+    h0 = rng.standard_normal((N, H)).astype(np.float32)
+    dones = (rng.random((T, N)) < 0.3).astype(np.uint8)
+    dh = rng.standard_normal((T, N, H)).astype(np.float32)
+    gru = binding.Gru(D, H, T, N)
+    gru.set_params(params)
+    d_x, d_h0, d_dn, d_dh = (torch.from_numpy(a).to("cuda") for a in (xp, h0, dones, dh))
+    d_h, d_dx, d_dh0 = torch.empty((T, N, H), device="cuda"), torch.zeros((T, N, stride), device="cuda"), torch.empty((N, H), device="cuda")
+    gru.forward(d_x, stride, d_h0, d_dn, T, N, d_h)
+    gru.backward(d_dh, d_dx, stride, d_dh0)
+    torch.cuda.synchronize()
+    p = G.unpack_gru(params, D, H)
+    c = G.gru_sequence_forward(p, x, h0, dones)
+    g = G.gru_sequence_backward(p, c, dh)
+    assert_close(d_h.cpu().numpy(), c["h"], 2e-5, "h")
+    assert_close(d_dx.cpu().numpy()[..., :D], g["x"], 1e-4, "dx")
+    assert_close(d_dh0.cpu().numpy(), g["h0"], 1e-4, "dh0")
+    assert_close(gru.get_grads(), G.flat_grads(g), 1e-4, "grad")
+    gru.destroy()

@@ -198,3 +198,32 @@ def test_full_size_reward_and_first_step_match_oracle():
     assert_close(out["first_loss"], r[0]["loss"], 1e-4, "loss")
     assert_close(rnd.get_grads(), r[0]["grad"], 1e-4, "grad")
     rnd.destroy()
+
+
+def test_degenerate_sizes():
+    """No rows, one row, one minibatch of an odd number of rows, a single selected entry and a one-wide embedding."""
+    import torch
+    from paper_2509_10771_b200 import binding
+    rng = np.random.default_rng(3)
+    obs = rng.standard_normal((37, 6)).astype(np.float32)
+    idx = np.array([4], dtype=np.int32)
+    dims = WL.rnd_layer_dims(1, (5,), 1)
+    n = sum(i * o + o for i, o in dims)
+    f, g = (rng.standard_normal(n) * 0.7).astype(np.float32), (rng.standard_normal(n) * 0.7).astype(np.float32)
+    rnd = binding.Rnd(6, idx, (5,), 1, max_rows=37, lr=1e-2)
+    rnd.set_params(f, g)
+    d_obs = torch.from_numpy(obs).to("cuda")
+    d_int = torch.full((37,), -1.0, device="cuda")
+    rnd.reward(d_obs, 0, 6, d_r_int_out=d_int)                      # nothing to do, nothing written
+    rnd.reward(d_obs, 1, 6, d_r_int_out=d_int)
+    torch.cuda.synchronize()
+    ref, _, _, _ = O.rnd_reward(f, g, dims, obs, idx, 1.0)
+    got = d_int.cpu().numpy()
+    assert_close(got[:1], ref[:1], 1e-4, "one row") ; assert np.all(got[1:] == -1.0)
+    hp = SimpleNamespace(epochs=3, minibatches=1, elu_alpha=1.0, adam_b1=0.9, adam_b2=0.999, adam_eps=1e-8)
+    out = rnd.update(d_obs, 37, 6, 3, 1, seed=5, iteration=2)
+    state = O.OptimState(f, 1e-2)
+    r = O.rnd_update(state, g, dims, obs, idx, hp, seed=5, iteration=2)
+    assert_close(out["mean_loss"], float(np.mean([x["loss"] for x in r])), 1e-4, "mean loss")
+    assert_close(rnd.get_params(), state.theta, 2e-4, "params")
+    rnd.destroy()
