@@ -496,7 +496,7 @@ __device__ __forceinline__ bool bias_entry(const ReduceArgs& a, int p) {
         if (p >= a.bias[b].p_off && p < a.bias[b].p_off + a.bias[b].n) return true;
     return false;
 }
-constexpr int kRedExtraBlocks = 24;     // blocks that finish the entries coming from partial rows
+constexpr int kRedExtraBlocks = 96;     // blocks that finish the entries coming from partial rows: a warp per four columns
 
 // grid = reduce_blocks(P) blocks over the parameter vector + one extra block for the entries
 // that come from the head/loss kernel and for the loss sums.
@@ -531,36 +531,36 @@ __global__ void __launch_bounds__(kRedThreads) reduce_kernel(const ReduceArgs a)
         // one warp per entry: lane l adds partial rows l, l+32, ... in order, then a fixed shuffle tree
         const int xwarp = (blockIdx.x - (gridDim.x - kRedExtraBlocks)) * (kRedThreads / 32) + warp;
         const int xwarps = kRedExtraBlocks * (kRedThreads / 32);
-        // bias sources: a warp takes 8 consecutive columns (two lanes x float4) and spreads the partial
-        // rows over its 16 lane pairs; every lane walks its rows in order, then a fixed butterfly
+        // bias sources: a warp takes 4 consecutive columns (one float4) and spreads the partial rows over
+        // its 32 lanes; every lane walks its rows in order, then a fixed butterfly
         int total_units = 0;
-        for (int b = 0; b < a.n_bias; ++b) total_units += (a.bias[b].n + 7) / 8;
+        for (int b = 0; b < a.n_bias; ++b) total_units += (a.bias[b].n + 3) / 4;
         for (int u = xwarp; u < total_units; u += xwarps) {
             int b = 0, ul = u;
-            while (ul >= (a.bias[b].n + 7) / 8) { ul -= (a.bias[b].n + 7) / 8; ++b; }
+            while (ul >= (a.bias[b].n + 3) / 4) { ul -= (a.bias[b].n + 3) / 4; ++b; }
             const BiasSource& src = a.bias[b];
-            const int c = 8 * ul + 4 * (lane & 1);                     // < ld: the rows are padded to 64 columns
+            const int c = 4 * ul;                                       // < ld: the rows are padded to 64 columns
             const float* __restrict__ base = src.slots + c;
             const size_t ld = (size_t)src.ld;
             float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
-            int r = lane >> 1;
-            for (; r + 16 * 7 < src.nslots; r += 16 * 8) {
+            int r = lane;
+            for (; r + 32 * 7 < src.nslots; r += 32 * 8) {
                 float4 v[8];
 #pragma unroll
-                for (int i = 0; i < 8; ++i) v[i] = __ldg(reinterpret_cast<const float4*>(base + (size_t)(r + 16 * i) * ld));
+                for (int i = 0; i < 8; ++i) v[i] = __ldg(reinterpret_cast<const float4*>(base + (size_t)(r + 32 * i) * ld));
 #pragma unroll
                 for (int i = 0; i < 8; ++i) { acc.x += v[i].x; acc.y += v[i].y; acc.z += v[i].z; acc.w += v[i].w; }
             }
-            for (; r < src.nslots; r += 16) {
+            for (; r < src.nslots; r += 32) {
                 const float4 v = __ldg(reinterpret_cast<const float4*>(base + (size_t)r * ld));
                 acc.x += v.x; acc.y += v.y; acc.z += v.z; acc.w += v.w;
             }
 #pragma unroll
-            for (int o = 2; o < 32; o <<= 1) {
+            for (int o = 1; o < 32; o <<= 1) {
                 acc.x += __shfl_xor_sync(0xffffffffu, acc.x, o); acc.y += __shfl_xor_sync(0xffffffffu, acc.y, o);
                 acc.z += __shfl_xor_sync(0xffffffffu, acc.z, o); acc.w += __shfl_xor_sync(0xffffffffu, acc.w, o);
             }
-            if (lane < 2) {
+            if (lane == 0) {
                 const float g[4] = {acc.x, acc.y, acc.z, acc.w};
 #pragma unroll
                 for (int q = 0; q < 4; ++q)
