@@ -417,6 +417,7 @@ struct ChainParams {
     CUtensorMap tmOut[2][kChainLayers];       // activations, boxes of 64 columns x 32 rows
     ChainNet net[2];                          // same numbers of jobs and epilogues, same waits
     int nnets, rows, total_items;             // items = (row tile, net), nets interleaved
+    int store;                                // 1: the activations are also written to global memory (tmOut)
     float alpha;
     int* error;
 };
@@ -669,8 +670,10 @@ __global__ void __launch_bounds__(kThreads, 1) chain_fwd_kernel(const __grid_con
                 // the accumulator is in registers; the buffer may still feed a job that runs meanwhile
                 if (E.write_job >= 0 && !mbar_wait(&job_done[E.write_job], t & 1u, abort_flag, P.error, 15)) { ok = false; break; }
                 if (active) {
-                    if (lane == 0) tma_store_wait_read();       // this warp's last store has read the rows
-                    __syncwarp();
+                    if (P.store) {
+                        if (lane == 0) tma_store_wait_read();   // this warp's last store has read the rows
+                        __syncwarp();
+                    }
 #pragma unroll
                     for (int p8 = 0; p8 < 8; ++p8) *reinterpret_cast<uint4*>(tile_row + ((p8 ^ sw) << 4)) = outv[p8];
                     fence_async_smem();                         // rows -> visible to the MMA and the copy engine
@@ -679,12 +682,12 @@ __global__ void __launch_bounds__(kThreads, 1) chain_fwd_kernel(const __grid_con
                 __syncwarp();
                 if (lane == 0) {
                     // rows at or beyond the tensor's extent are clipped by the store itself
-                    if (active && m0 + 32 * q < P.rows) tma_store_2d(&P.tmOut[ni][E.layer], tile, E.n0 + 64 * g, m0 + 32 * q);
+                    if (P.store && active && m0 + 32 * q < P.rows) tma_store_2d(&P.tmOut[ni][E.layer], tile, E.n0 + 64 * g, m0 + 32 * q);
                     mbar_arrive(&epi_done[e]);
                 }
             }
         }
-        if (lane == 0) tma_store_wait_all();        // stores done before the CTA retires
+        if (P.store && lane == 0) tma_store_wait_all();   // stores done before the CTA retires
     }
     tc_fence_before();
     __syncthreads();
@@ -1110,6 +1113,9 @@ UmmaEngine* umma_create(const UmmaSetup& s, std::string* err) {
         }
         P.rows = rows;
         P.total_items = P.nnets * ((rows + BLOCK_M - 1) / BLOCK_M);
+        // with the heads inside the kernel nothing reads the hidden activations of a rollout step afterwards
+        P.store = 0;
+        for (int n = 0; n < P.nnets; ++n) if (P.net[n].head_n == 0) P.store = 1;
         P.alpha = alpha; P.error = e->error_dev;
         out.push_back(P);
         return true;
