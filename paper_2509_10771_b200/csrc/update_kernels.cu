@@ -651,6 +651,57 @@ __global__ void __launch_bounds__(kAdamThreads) adam_kernel(const AdamArgs a) {
     const float coef = s_scal[0], lr = s_scal[1], c1 = s_scal[2], c2 = s_scal[3];
     const int n4 = a.P / 4;
     for (int i = blockIdx.x * kAdamThreads + threadIdx.x; i < n4; i += gridDim.x * kAdamThreads) {
+        // BF16 mode, hidden-layer weights: a thread takes four consecutive ROWS of one column instead of four
+        // consecutive columns of one row, so that its entries of the transposed operand copy Wt[out][in] are
+        // one 8-byte store (neighbouring threads: neighbouring columns, every FP32 access still coalesced).
+        // Those groups cover the rows below the last multiple of four, the same elements as before in another
+        // assignment; the remaining rows, biases and everything else take the path below.
+        {
+            const int idx0 = 4 * i;
+            int e = 0;
+            while (e < a.n_cvt && !(idx0 >= a.cvt[e].w_off && idx0 < a.cvt[e].w_off + a.cvt[e].in * a.cvt[e].out_p)) ++e;
+            if (e < a.n_cvt) {
+                const CvtRange& c = a.cvt[e];
+                const int lg = (idx0 - c.w_off) >> 2;
+                if (lg < (c.in >> 2) * c.out_p) {
+                    const int r4 = lg / c.out_p, o = lg - r4 * c.out_p;
+                    const size_t base = (size_t)c.w_off + (size_t)(4 * r4) * c.out_p + o;
+                    float g[4], p[4], m[4], v[4];
+#pragma unroll
+                    for (int q = 0; q < 4; ++q) {
+                        const size_t at = base + (size_t)q * c.out_p;
+                        g[q] = a.grad[at]; p[q] = a.param[at]; m[q] = a.m[at]; v[q] = a.v[at];
+                    }
+#pragma unroll
+                    for (int q = 0; q < 4; ++q) {
+                        const float gc = g[q] * coef;
+                        m[q] = a.b1 * m[q] + (1.0f - a.b1) * gc;
+                        v[q] = a.b2 * v[q] + (1.0f - a.b2) * gc * gc;
+                        p[q] = p[q] - lr * (m[q] * c1) / (sqrtf(v[q] * c2) + a.eps);
+                        const size_t at = base + (size_t)q * c.out_p;
+                        a.param[at] = p[q]; a.m[at] = m[q]; a.v[at] = v[q];
+                    }
+                    if (o < c.out) {
+                        __nv_bfloat16 w[4];
+#pragma unroll
+                        for (int q = 0; q < 4; ++q) {
+                            w[q] = __float2bfloat16_rn(p[q]);
+                            if (c.wn) c.wn[(size_t)(4 * r4 + q) * c.ld_wn + o] = w[q];
+                        }
+                        __nv_bfloat162 lo2 = __halves2bfloat162(w[0], w[1]), hi2 = __halves2bfloat162(w[2], w[3]);
+                        *reinterpret_cast<uint2*>(c.wt + (size_t)o * c.ld_wt + 4 * r4) =
+                            make_uint2(*reinterpret_cast<uint32_t*>(&lo2), *reinterpret_cast<uint32_t*>(&hi2));
+                        if (c.wt_lo) {
+                            __nv_bfloat162 l0 = __floats2bfloat162_rn(p[0] - __bfloat162float(w[0]), p[1] - __bfloat162float(w[1]));
+                            __nv_bfloat162 l1 = __floats2bfloat162_rn(p[2] - __bfloat162float(w[2]), p[3] - __bfloat162float(w[3]));
+                            *reinterpret_cast<uint2*>(c.wt_lo + (size_t)o * c.ld_wt + 4 * r4) =
+                                make_uint2(*reinterpret_cast<uint32_t*>(&l0), *reinterpret_cast<uint32_t*>(&l1));
+                        }
+                    }
+                    continue;
+                }
+            }
+        }
         const float4 g4 = reinterpret_cast<const float4*>(a.grad)[i];
         float4 p4 = reinterpret_cast<float4*>(a.param)[i];
         float4 m4 = reinterpret_cast<float4*>(a.m)[i];
