@@ -1,7 +1,7 @@
 #!/usr/bin/env python
 """Benchmark of the PPO learn-iteration hot path (rollout inference + GAE + PPO update).
 
-    python bench.py [--gpus N] [--steps K] [--warmup W] [--impl ours|reference]
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--impl ours|reference] [--workload NAME]
 
 One "step" is one whole learn iteration over one rollout of synthetic data:
 T x (rslrl_act + rslrl_record_step), rslrl_gae, rslrl_ppo_update (E x M minibatch steps).
@@ -14,8 +14,9 @@ The metric is transitions/s = T * N_envs * K / time.  Rank 0 prints ONE JSON lin
           the same K steps with one CUDA event pair per launch
   cpu_baseline  the FP64 oracle, as it stands, on the host cores, on a bounded sample
 
-With --gpus N > 1 (launched by torch.distributed.run) every rank runs an independent replica
-of the workload on its own GPU: the path has no inter-GPU exchange ("replicas only").
+With --gpus N > 1 every rank runs an independent replica of the workload on its own GPU: the path
+has no inter-GPU exchange ("replicas only").  Started plainly (no WORLD_SIZE in the environment) the
+script launches its N ranks itself through torch.distributed.run on 127.0.0.1.
 """
 from __future__ import annotations
 
@@ -37,6 +38,7 @@ from paper_2509_10771_b200 import workloads as WL  # noqa: E402
 METRIC = "PPO learn-iteration transitions/s"
 UNIT = "transitions/s"
 WORKLOAD = WL.ROUGH                       # rough-terrain locomotion shape: the config the metric is quoted on
+                                          # (--workload selects another of the five)
 PRECISION = WL.PRECISION_BF16
 ORACLE_SAMPLE_ENVS = 512                  # bounded sample for the CPU baseline: 512 of the 4096 environments
 
@@ -69,6 +71,22 @@ def family_flops(w):
     dgrad = steps * R * sum(2 * i * o for net in ("actor", "critic") for i, o in w.layer_dims(net)[1:-1])
     wgrad = steps * R * sum(2 * i * o for net in ("actor", "critic") for i, o in w.layer_dims(net))
     return {"tc_mlp_fwd": rollout, "tc_gemm_fwd": fwd, "tc_gemm_dgrad": dgrad, "tc_gemm_wgrad": wgrad}
+
+
+def hbm_family_bytes(w, storage_strides):
+    """Algorithmic bytes per launch of the bandwidth-shaped kernels (what must be read plus what must be written)."""
+    sa, sc, as_ = storage_strides
+    T, N = w.num_steps, w.num_envs
+    Bmb = w.minibatch_rows
+    R = Bmb * (2 if w.sym_enable else 1)
+    kp_a = -(-w.actor_obs_dim // 64) * 64
+    kp_c = -(-w.critic_obs_dim // 64) * 64
+    obs_read = 4 * w.actor_obs_dim + (0 if w.shared_obs else 4 * w.critic_obs_dim)
+    obs_written = 2 * kp_a + (0 if w.shared_obs else 2 * kp_c)                    # BF16 operand rows
+    gather = Bmb * (4 + obs_read + 4 * 2 * w.num_actions + 4 * 4) \
+        + R * (obs_written + 4 * as_) + Bmb * (2 * 4 * as_ + 4 * 4)
+    P = w.num_params()
+    return {"gather": gather, "adam": 28 * P, "gae_scan": 18 * T * N, "gae_normalize": 8 * T * N}
 
 
 # DRAM bytes per launch (dram__bytes_read.sum + dram__bytes_write.sum, mean over the family's launches of one
@@ -141,7 +159,8 @@ def run_reference(args, rank):
     envs = ORACLE_SAMPLE_ENVS
     while envs > 64 and n_iter * envs * 0.008 > 120.0:
         envs //= 2
-    w = WORKLOAD.scaled(envs)
+    w = WORKLOAD.scaled(min(envs, WORKLOAD.num_envs))
+    envs = w.num_envs
     times = oracle_iteration_seconds(w, repeats=n_iter)[args.warmup:]
     total = sum(times)
     value = w.batch * len(times) / total
@@ -174,7 +193,7 @@ class ClockSampler:
     def start(self):
         try:
             self.proc = subprocess.Popen(["nvidia-smi", f"--query-gpu={self.QUERY}", "--format=csv,noheader,nounits",
-                                          "-lms", "100", "-i", str(self.idx)], stdout=subprocess.PIPE,
+                                          "-lms", "20", "-i", str(self.idx)], stdout=subprocess.PIPE,
                                          stderr=subprocess.DEVNULL, text=True)
         except Exception:
             self.proc = None
@@ -243,12 +262,15 @@ def run_ours(args, rank, world, local_rank):
     T, N, A = w.num_steps, w.num_envs, w.num_actions
     inputs = WL.make_rollout_inputs(w, seed=rank)          # every replica draws its own rollout
     theta = WL.make_params(w, seed=rank)
+    mirror = WL.make_mirror(w, seed=rank) if w.sym_enable else None
     dev = torch.device("cuda", local_rank)
     stream = torch.cuda.current_stream()
-    ctx = binding.Context(w, precision=PRECISION, stream=stream.cuda_stream)
+    ctx = binding.Context(w, precision=PRECISION, stream=stream.cuda_stream, mirror=mirror)
     ctx.set_params(theta)
+    view = ctx.storage_view()
 
     d_obs = torch.from_numpy(inputs["obs_actor"]).to(dev)
+    d_obc = None if w.shared_obs else torch.from_numpy(inputs["obs_critic"]).to(dev)
     d_rew = torch.from_numpy(inputs["rewards"]).to(dev)
     d_done = torch.from_numpy(inputs["dones"]).to(dev)
     d_to = torch.from_numpy(inputs["timeouts"]).to(dev)
@@ -256,26 +278,29 @@ def run_ours(args, rank, world, local_rank):
 
     def iteration_device():
         for t in range(T):
-            ctx.act(d_obs[t])
+            ctx.act(d_obs[t], None if d_obc is None else d_obc[t])
             ctx.record_step(d_rew[t], d_done[t], d_to[t])
-        ctx.gae(d_obs[T])
+        ctx.gae(d_obs[T] if d_obc is None else d_obc[T])
         ctx.ppo_update(want_stats=False)
 
     h_obs = torch.from_numpy(inputs["obs_actor"]).pin_memory()
+    h_obc = None if w.shared_obs else torch.from_numpy(inputs["obs_critic"]).pin_memory()
     h_rew = torch.from_numpy(inputs["rewards"]).pin_memory()
     h_done = torch.from_numpy(inputs["dones"]).pin_memory()
     h_to = torch.from_numpy(inputs["timeouts"]).pin_memory()
     h_act = torch.empty((N, A), dtype=torch.float32).pin_memory()
     np_obs, np_rew, np_done, np_to, np_act = (x.numpy() for x in (h_obs, h_rew, h_done, h_to, h_act))
+    np_obc = None if h_obc is None else h_obc.numpy()
 
     def iteration_host():
         for t in range(T):
-            ctx.act_host(np_obs[t], None, np_act)          # H2D obs, D2H actions (waits for them)
+            ctx.act_host(np_obs[t], None if np_obc is None else np_obc[t], np_act)   # H2D obs, D2H actions (waits for them)
             ctx.record_step_host(np_rew[t], np_done[t], np_to[t])
-        ctx.gae_host(np_obs[T])
+        ctx.gae_host(np_obs[T] if np_obc is None else np_obc[T])
         return ctx.ppo_update(want_stats=True)             # D2H of the update's scalars
 
-    h2d = T * (N * w.actor_obs_dim * 4 + N * 4 + 2 * N) + N * w.critic_obs_dim * 4
+    obs_bytes = N * w.actor_obs_dim * 4 + (0 if w.shared_obs else N * w.critic_obs_dim * 4)
+    h2d = T * (obs_bytes + N * 4 + 2 * N) + N * w.critic_obs_dim * 4
     d2h = T * N * A * 4 + w.epochs * w.minibatches * 8 * 4
 
     def barrier():
@@ -296,6 +321,19 @@ def run_ours(args, rank, world, local_rank):
         barrier()
         return sum(a.elapsed_time(b) for a, b in evs)      # ms
 
+    def timed_one_interval(fn, steps):
+        """The same K steps as ONE event interval (back to back, no flush in between: one iteration's working
+        set, storage plus activations, is itself larger than the L2)."""
+        a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        barrier()
+        flush_buf.zero_()
+        a.record(stream)
+        for _ in range(steps):
+            fn()
+        b.record(stream)
+        barrier()
+        return a.elapsed_time(b)
+
     for _ in range(max(args.warmup, 3)):
         iteration_device()
     torch.cuda.synchronize()
@@ -304,12 +342,12 @@ def run_ours(args, rank, world, local_rank):
         gpu_id = "GPU-" + str(torch.cuda.get_device_properties(local_rank).uuid)
     except Exception:
         gpu_id = str(local_rank)
-    sampler = ClockSampler(gpu_id)
+    sampler = ClockSampler(gpu_id)                          # runs across all timed passes below
     launches0 = binding.kernel_launch_count()
     sampler.start()
     ms_total = timed(iteration_device, args.steps)
-    clocks = sampler.stop()
     launches = binding.kernel_launch_count() - launches0
+    ms_interval = timed_one_interval(iteration_device, args.steps)
 
     iteration_host()
     ms_e2e = timed(iteration_host, args.steps)
@@ -323,8 +361,9 @@ def run_ours(args, rank, world, local_rank):
     torch.cuda.synchronize()
     prof = binding.profile_report()
     binding.profile_enable(False)
+    clocks = sampler.stop()
 
-    ms_total, ms_e2e = max_over_ranks([ms_total, ms_e2e], world, dev)
+    ms_total, ms_e2e, ms_interval = max_over_ranks([ms_total, ms_e2e, ms_interval], world, dev)
     if rank != 0:
         if world > 1:
             dist.destroy_process_group()
@@ -341,19 +380,42 @@ def run_ours(args, rank, world, local_rank):
     tc = {k: v for k, v in prof.items() if k in fam_flops}
     top = max(tc, key=lambda k: tc[k]["ms"])
     achieved = fam_flops[top] * args.steps / (tc[top]["ms"] * 1e-3) / 1e12
-    peak = peaks["bf16_tflops_sustained"]
-    roofline = {"bound": "tensor", "kernel": top, "achieved": achieved, "peak": peak, "unit": "TFLOP/s",
-                "frac": achieved / peak, "traffic": ncu_traffic(top), "traffic_unit": "bytes per launch (ncu, dram read + write)",
-                "peak_source": f"bf16 sustained, {peaks['source']}",
-                "avg_launch_us": 1e3 * tc[top]["ms"] / tc[top]["launches"],
-                "families": {k: {"tflops": fam_flops[k] * args.steps / (tc[k]["ms"] * 1e-3) / 1e12,
-                                 "frac": fam_flops[k] * args.steps / (tc[k]["ms"] * 1e-3) / 1e12 / peak} for k in tc},
-                "timing": "one CUDA event pair per launch, separate pass over the same K steps"}
+    # the launches of the per-kernel pass are timed one by one (tens of microseconds each, clocks at their maximum,
+    # no power cap): the burst peak is their denominator; the sustained one is printed beside it
+    peak, peak_sus = peaks["bf16_tflops"], peaks["bf16_tflops_sustained"]
 
-    ws = WORKLOAD.scaled(ORACLE_SAMPLE_ENVS)
+    def fam(k):
+        tf = fam_flops[k] * args.steps / (tc[k]["ms"] * 1e-3) / 1e12
+        return {"tflops": tf, "frac": tf / peak, "frac_of_sustained": tf / peak_sus,
+                "avg_launch_us": 1e3 * tc[k]["ms"] / tc[k]["launches"]}
+
+    roofline = {"bound": "tensor", "kernel": top, "achieved": achieved, "peak": peak, "unit": "TFLOP/s",
+                "frac": achieved / peak, "frac_of_sustained": achieved / peak_sus, "frac_of_nominal_2250": achieved / 2250.0,
+                "traffic": ncu_traffic(top), "traffic_unit": "bytes per launch (ncu, dram read + write)",
+                "peak_source": f"bf16 burst (launches timed alone), {peaks['source']}; sustained {peak_sus}",
+                "avg_launch_us": 1e3 * tc[top]["ms"] / tc[top]["launches"],
+                "families": {k: fam(k) for k in tc},
+                "timing": "separate pass over the same K steps with one CUDA event pair per launch; the forward and the "
+                          "data-gradient launches of a minibatch step (one per layer, chained by programmatic dependent "
+                          "launch) share one pair per step, divided by their number"}
+    # bandwidth-shaped kernels of the same pass: algorithmic bytes per launch / mean launch time
+    hbm_bytes = hbm_family_bytes(w, (view.obs_a_stride, view.obs_c_stride, view.act_stride))
+    hbm = {}
+    for k, nbytes in hbm_bytes.items():
+        if k in prof and prof[k]["launches"]:
+            us = 1e3 * prof[k]["ms"] / prof[k]["launches"]
+            gbs = nbytes / (us * 1e-6) / 1e9
+            hbm[k] = {"bytes_per_launch": nbytes, "avg_launch_us": us, "gbs": gbs, "frac": gbs / peaks["hbm_gbs"],
+                      "frac_of_nominal_7700": gbs / 7700.0}
+    roofline["hbm_families"] = hbm
+    roofline["hbm_peak_gbs"] = peaks["hbm_gbs"]
+
+    ws = WORKLOAD.scaled(min(ORACLE_SAMPLE_ENVS, WORKLOAD.num_envs))
+    oracle_iteration_seconds(WORKLOAD.scaled(32), repeats=1)            # warms numpy / BLAS threads once (not timed)
     o_times = oracle_iteration_seconds(ws, repeats=1)
-    sample = (f"one whole learn iteration on {ORACLE_SAMPLE_ENVS} of the {w.num_envs} environments of {w.name} "
-              f"(T={w.num_steps}, E={w.epochs}, M={w.minibatches}), numpy float64")
+    sample = (f"one whole learn iteration on {ws.num_envs} of the {w.num_envs} environments of {w.name} "
+              f"(T={w.num_steps}, E={w.epochs}, M={w.minibatches}), numpy float64, after one untimed warm-up "
+              f"iteration on 32 environments")
     cpu = {"value": ws.batch / o_times[0], "unit": UNIT, "cores": blas_threads(), "kind": "oracle", "sample": sample}
 
     line = {
@@ -361,10 +423,13 @@ def run_ours(args, rank, world, local_rank):
         "ms_per_step": ms_total / args.steps, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
         "dtype": "bf16", "data": "synthetic",
         "config": {"workload": w.name, "num_envs": N, "num_steps": T, "obs_dim": w.actor_obs_dim, "actions": A,
-                   "hidden": list(w.actor_hidden), "epochs": w.epochs, "minibatches": w.minibatches,
+                   "epochs": w.epochs, "minibatches": w.minibatches, "symmetry": bool(w.sym_enable),
                    "precision": "bf16 operands, fp32 accumulate", "l2": "256 MiB buffer written between timed steps",
                    "parallelism": "replicas only" if world > 1 else "1 gpu"},
         "clocks": clocks,
+        "one_interval": {"ms_per_step": ms_interval / args.steps,
+                         "value": whole_job_value(T * N * args.steps, world, ms_interval),
+                         "note": "the same K steps as one CUDA event interval, back to back, no L2 flush in between"},
         "e2e": {"value": e2e_value, "unit": UNIT, "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h,
                 "ms_per_step": ms_e2e / args.steps},
         "gpu_launches": int(launches),
@@ -613,16 +678,36 @@ def run_gru(args):
     gru.destroy()
 
 
+def free_port():
+    import socket
+    with socket.socket(socket.AF_INET, socket.SOCK_STREAM) as so:
+        so.bind(("127.0.0.1", 0))
+        return so.getsockname()[1]
+
+
+def spawn_ranks(n):
+    """Started plainly with --gpus N > 1: run this script again as N ranks (one per GPU) under torch.distributed.run."""
+    cmd = [sys.executable, "-m", "torch.distributed.run", "--nnodes=1", f"--nproc-per-node={n}",
+           "--master-addr", "127.0.0.1", "--master-port", str(free_port()), os.path.abspath(__file__), *sys.argv[1:]]
+    return subprocess.call(cmd)
+
+
 def main():
+    global WORKLOAD
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
     ap.add_argument("--steps", type=int, default=50)
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--workload", default=WORKLOAD.name, choices=sorted(WL.WORKLOADS),
+                    help="which of the five synthetic workloads to time (default: the one the metric is quoted on)")
     ap.add_argument("--task", default="ppo", choices=["ppo", "distill", "rnd", "gru"],
                     help="ppo: the learn iteration the metric is quoted on (default); distill: the distillation iteration; "
                          "rnd: random network distillation over one rollout; gru: the recurrent layer over one rollout")
     args = ap.parse_args()
+    WORKLOAD = WL.WORKLOADS[args.workload]
+    if args.gpus > 1 and "WORLD_SIZE" not in os.environ:
+        raise SystemExit(spawn_ranks(args.gpus))
     rank = int(os.environ.get("RANK", "0"))
     world = int(os.environ.get("WORLD_SIZE", "1"))
     local_rank = int(os.environ.get("LOCAL_RANK", "0"))

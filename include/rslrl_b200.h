@@ -19,12 +19,10 @@
  *     executed the call.  Buffers owned by the library are 16-byte aligned.
  *   - All calls enqueue on the CUDA stream given to rslrl_create and return without a host
  *     synchronisation unless stated.  A context is not thread-safe.  In RSLRL_BF16 mode
- *     rslrl_ppo_update also uses a stream of its own for the minibatch gather; it is joined
- *     to the caller's stream by events before the update's last kernel is enqueued.
- *   - Environment: RSLRL_FUSED_STEP=1 at rslrl_create selects, in RSLRL_BF16 mode without
- *     symmetry, a kernel that runs forward, heads, loss and data gradients of a row tile in one
- *     launch instead of one launch per layer (same results; slower on the workloads measured).
- *     RSLRL_SERIAL_LAUNCHES=1 switches programmatic dependent launch off.
+ *     rslrl_ppo_update also uses a stream of its own for the minibatch gather and the
+ *     shuffles; the caller's stream waits for everything enqueued there before the call
+ *     returns, so work enqueued after the call is ordered behind all of the update's kernels.
+ *   - Environment: RSLRL_SERIAL_LAUNCHES=1 switches programmatic dependent launch off.
  *   - Every function returns an rslrl_status; nothing throws, aborts or traps the device.
  *     Argument errors are found on the host before anything is launched.
  *     rslrl_last_error gives a human-readable message for the last failure of a context.

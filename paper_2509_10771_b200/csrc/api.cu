@@ -74,8 +74,11 @@ struct rslrl_ctx {
     void* up_h[2][kMaxLayers] = {};
     void* up_dz[2][kMaxLayers] = {};
     float *dmu = nullptr, *dv = nullptr; int lddmu = 0;
-    int* perm = nullptr;                  // [epochs][T*N] shuffles of one iteration
-    uint32_t perm_iteration = 0xFFFFFFFFu; // which iteration's shuffles perm holds (or is being filled with)
+    int* perm[2] = {};                    // [epochs][T*N] shuffles of one iteration; with a gather stream two sets, so that
+                                          // the next iteration's are resolved while this one's are still being read
+    int perm_cur = 0;                     // the set the current iteration reads
+    uint32_t perm_iteration[2] = {0xFFFFFFFFu, 0xFFFFFFFFu};   // which iteration's shuffles each set holds (or is being filled with)
+    cudaEvent_t ev_side_idle = nullptr;   // everything enqueued on the gather stream so far
     float *partials = nullptr, *block_partials = nullptr, *sumsq_partials = nullptr, *loss_sums = nullptr;
     float* stats_dev = nullptr; float* stats_host = nullptr; int max_stat_rows = 0;
     SymTables sym{};
@@ -333,6 +336,7 @@ rslrl_status rslrl_destroy(rslrl_ctx* c) {
     cudaStreamSynchronize(c->stream);
     if (c->side) { cudaStreamSynchronize(c->side); cudaStreamDestroy(c->side); }
     if (c->ev_ready) cudaEventDestroy(c->ev_ready);
+    if (c->ev_side_idle) cudaEventDestroy(c->ev_side_idle);
     for (int b = 0; b < 2; ++b) {
         if (c->ev_gathered[b]) cudaEventDestroy(c->ev_gathered[b]);
         if (c->ev_consumed[b]) cudaEventDestroy(c->ev_consumed[b]);
@@ -417,7 +421,7 @@ rslrl_status rslrl_create(const rslrl_model_cfg* m, const rslrl_ppo_cfg* p, void
         A_(c->logp_old[b], c->Bmb); A_(c->v_old[b], c->Bmb); A_(c->ret_mb[b], c->Bmb); A_(c->adv_mb[b], c->Bmb);
     }
     A_(c->dmu, (size_t)c->R * as); A_(c->dv, (size_t)c->R * 4);
-    A_(c->perm, (size_t)B * p->epochs);
+    A_(c->perm[0], (size_t)B * p->epochs);
     A_(c->partials, (size_t)c->splits * c->P_dev);
     A_(c->block_partials, (size_t)std::max(head_loss_blocks(c->Bmb), 256) * head_partial_stride());
     A_(c->sumsq_partials, reduce_blocks(c->P_dev)); A_(c->loss_sums, 8);
@@ -442,13 +446,15 @@ rslrl_status rslrl_create(const rslrl_model_cfg* m, const rslrl_ppo_cfg* p, void
         std::string uerr;
         c->umma = umma_create(us, &uerr);
         if (!c->umma) { c->err = "tensor-core engine: " + uerr; return bail(RSLRL_ERR_UNSUPPORTED); }
-        if (umma_two_input_buffers(c->umma)) {
+        {
             bool okv = cudaStreamCreateWithFlags(&c->side, cudaStreamNonBlocking) == cudaSuccess &&
-                       cudaEventCreateWithFlags(&c->ev_ready, cudaEventDisableTiming) == cudaSuccess;
+                       cudaEventCreateWithFlags(&c->ev_ready, cudaEventDisableTiming) == cudaSuccess &&
+                       cudaEventCreateWithFlags(&c->ev_side_idle, cudaEventDisableTiming) == cudaSuccess;
             for (int b = 0; b < 2 && okv; ++b)
                 okv = cudaEventCreateWithFlags(&c->ev_gathered[b], cudaEventDisableTiming) == cudaSuccess &&
                       cudaEventCreateWithFlags(&c->ev_consumed[b], cudaEventDisableTiming) == cudaSuccess;
             if (!okv) { c->err = "could not create the gather stream"; return bail(RSLRL_ERR_CUDA); }
+            A_(c->perm[1], (size_t)B * p->epochs);
         }
     }
     // staging for the host-buffer variants
@@ -653,7 +659,7 @@ static rslrl_status update_impl(rslrl_ctx* c, int32_t max_steps, rslrl_update_st
         if (c->umma) umma_gather_targets(c->umma, &g, buf);
         g.act_mb = c->act_mb[buf]; g.mu_old = c->mu_old[buf]; g.sigma_old = c->sigma_old[buf];
         g.logp_old = c->logp_old[buf]; g.v_old = c->v_old[buf]; g.ret = c->ret_mb[buf]; g.adv_mb = c->adv_mb[buf];
-        g.rows = c->perm + (size_t)e * T * N + (size_t)k * c->Bmb; g.Bmb = c->Bmb; g.sym = pc.sym_enable; g.st = c->sym;
+        g.rows = c->perm[c->perm_cur] + (size_t)e * T * N + (size_t)k * c->Bmb; g.Bmb = c->Bmb; g.sym = pc.sym_enable; g.st = c->sym;
         CU(c, launch_gather(g, st));
         return RSLRL_OK;
     };
@@ -665,15 +671,19 @@ static rslrl_status update_impl(rslrl_ctx* c, int32_t max_steps, rslrl_update_st
         CU(c, cudaEventRecord(c->ev_ready, c->stream));           // advantages and returns are in storage
         CU(c, cudaStreamWaitEvent(c->side, c->ev_ready, 0));
     }
-    // the shuffles of all epochs of this iteration, resolved in one launch (with a gather stream the end of
-    // the update before has already started them, so that they run beside the rollout)
-    if (c->perm_iteration != c->iteration) {
-        CU(c, launch_perm_epochs(pc.seed, c->iteration, pc.epochs, (uint32_t)(T * N), c->perm, overlap ? c->side : c->stream));
-        c->perm_iteration = c->iteration;
+    // the shuffles of all epochs of this iteration, resolved in one launch (with a gather stream the update
+    // before has already resolved them into the other set, beside its own kernels)
+    if (c->perm_iteration[c->perm_cur] != c->iteration) {
+        CU(c, launch_perm_epochs(pc.seed, c->iteration, pc.epochs, (uint32_t)(T * N), c->perm[c->perm_cur], overlap ? c->side : c->stream));
+        c->perm_iteration[c->perm_cur] = c->iteration;
     }
     if (overlap) {
         TRY(enqueue_gather(0, 0, c->side));
         CU(c, cudaEventRecord(c->ev_gathered[0], c->side));
+        // the next iteration's shuffles depend on the seed and the iteration number only: they go into the
+        // other set now, behind the first gather and beside this update's kernels
+        CU(c, launch_perm_epochs(pc.seed, c->iteration + 1, pc.epochs, (uint32_t)(T * N), c->perm[c->perm_cur ^ 1], c->side));
+        c->perm_iteration[c->perm_cur ^ 1] = c->iteration + 1;
     }
     int done_steps = 0;
     for (int e = 0; e < pc.epochs && done_steps < nsteps; ++e) {
@@ -691,19 +701,7 @@ static rslrl_status update_impl(rslrl_ctx* c, int32_t max_steps, rslrl_update_st
                 TRY(enqueue_gather(done_steps, 0, c->stream));
             }
             // ---- forward, heads, loss, backward ----------------------------------------------
-            const bool fused = c->umma && umma_has_step_chain(c->umma) && !distill;
             HeadLossArgs hl{};
-            if (fused) {
-                // row-local work in one kernel, then the weight-gradient partials
-                StepChainLoss sl{};
-                sl.act_mb = c->act_mb[buf]; sl.mu_old = c->mu_old[buf]; sl.sigma_old = c->sigma_old[buf]; sl.as = c->st.act_stride;
-                sl.logp_old = c->logp_old[buf]; sl.v_old = c->v_old[buf]; sl.ret = c->ret_mb[buf]; sl.adv = c->adv_mb[buf];
-                sl.clip = pc.clip; sl.value_clip = pc.value_clip; sl.value_coef = pc.value_coef;
-                sl.use_clipped_value_loss = pc.use_clipped_value_loss;
-                sl.block_partials = c->block_partials;
-                CU(c, umma_step_chain(c->umma, sl, &hl.nblocks_used));
-                CU(c, umma_update_wgrad(c->umma));
-            } else {
             if (c->prec == RSLRL_FP32) {
                 TRY(forward_hidden_fp32(c, true, true, c->x_a, c->mc.shared_obs ? c->x_a : c->x_c, c->R, c->up_h));
                 hl.Ha = c->up_h[0][c->actor.nl - 2]; hl.ldha = c->actor.hid_ld[c->actor.nl - 2];
@@ -729,7 +727,6 @@ static rslrl_status update_impl(rslrl_ctx* c, int32_t max_steps, rslrl_update_st
             // ---- backward ---------------------------------------------------------------
             if (c->prec == RSLRL_FP32) TRY(backward_fp32(c));
             else CU(c, umma_update_backward(c->umma, hl.colsum_written != 0, buf, distill));
-            }
             if (overlap) CU(c, cudaEventRecord(c->ev_consumed[buf], c->stream));   // this input set may be refilled
             // ---- reduce, clip, adaptive lr, Adam ------------------------------------------
             ReduceArgs r{};
@@ -738,8 +735,7 @@ static rslrl_status update_impl(rslrl_ctx* c, int32_t max_steps, rslrl_update_st
             r.block_partials = c->block_partials; r.nblocks = hl.nblocks_used;
             r.off_ba = (int)ha.b_off; r.off_logstd = (int)c->logstd_off; r.off_bc = (int)hc.b_off; r.A = A;
             r.entropy_coef = distill ? 0.f : pc.entropy_coef; r.log_std = c->param + c->logstd_off; r.loss_sums = c->loss_sums;
-            if (fused) umma_fill_step_bias_sources(c->umma, &r);
-            else if (c->umma) umma_fill_bias_sources(c->umma, &r, hl);
+            if (c->umma) umma_fill_bias_sources(c->umma, &r, hl);
             CU(c, launch_reduce(r, c->stream));
             AdamArgs ad{};
             ad.param = c->param; ad.m = c->adam_m; ad.v = c->adam_v; ad.grad = c->grad; ad.P = c->P_dev;
@@ -759,9 +755,11 @@ static rslrl_status update_impl(rslrl_ctx* c, int32_t max_steps, rslrl_update_st
     c->iteration++;
     c->step = 0; c->gae_done = false; c->act_pending = false;
     if (overlap) {
-        // the next iteration's shuffles depend on the seed and the iteration number only
-        CU(c, launch_perm_epochs(pc.seed, c->iteration, pc.epochs, (uint32_t)(T * N), c->perm, c->side));
-        c->perm_iteration = c->iteration;
+        // join: whatever the gather stream still holds (the next iteration's shuffles when the update was cut
+        // short) completes before anything the caller enqueues after this call
+        c->perm_cur ^= 1;
+        CU(c, cudaEventRecord(c->ev_side_idle, c->side));
+        CU(c, cudaStreamWaitEvent(c->stream, c->ev_side_idle, 0));
     }
     if (h_stats) {
         CU(c, cudaMemcpyAsync(c->stats_host, c->stats_dev, (size_t)nsteps * 8 * sizeof(float), cudaMemcpyDeviceToHost, c->stream));

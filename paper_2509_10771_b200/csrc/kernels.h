@@ -17,6 +17,14 @@ struct LaunchScope {
     const char* name; cudaStream_t stream; int slot;
 };
 
+// Brackets a run of consecutive launches of one kernel family with ONE event pair while profiling is on
+// (the launches inside are counted, not bracketed), so that their dependent-launch overlap is kept.
+struct FamilyScope {
+    FamilyScope(const char* name, cudaStream_t stream);
+    ~FamilyScope();
+    cudaStream_t stream; int slot;
+};
+
 // Launch of a kernel that begins with chain_begin(): it may be scheduled before the preceding kernel
 // of the stream has drained (programmatic stream serialisation), which hides launch latency and
 // prologue.  Falls back to a plain launch when chained launches are switched off.

@@ -2,7 +2,8 @@
 // persistent tcgen05 GEMM kernels.  Operands are BF16 tiles staged in shared memory by TMA
 // (128-byte swizzle), accumulators are FP32 in tensor memory (two buffers, so the epilogue of
 // one tile overlaps the main loop of the next), and the epilogues fuse bias+ELU (forward),
-// the ELU derivative (data gradient) or the split-partial store (weight gradient).
+// the ELU derivative (data gradient) or the split-partial store (weight gradient).  Forward and
+// data gradient keep the weight operand of a CTA resident in shared memory and stream the rows.
 //
 // Warp roles in a CTA of 576 threads: warp 0 = TMA producer, warp 1 = MMA issuer and owner of
 // the tensor-memory allocation, warps 2..17 = epilogue (each reads its quarter of the 128
@@ -12,7 +13,6 @@
 // the host reads, drains its own asynchronous work, frees its tensor memory and returns.
 #include "umma.h"
 #include "tc_ptx.cuh"
-#include "step_chain.h"
 
 #include <cuda.h>
 #include <algorithm>
@@ -26,15 +26,11 @@ using namespace tc;
 
 namespace {
 
-// Forward and data gradient: 3 pipeline stages + a 4 KiB result tile per epilogue warp;
-// weight gradient (long contraction, FP32 results stored from registers): 4 stages.
-__host__ __device__ constexpr int stages_of(int mode) { return mode == 2 ? 4 : 3; }
+// Weight gradient (long contraction, FP32 results stored from registers): 4 pipeline stages of A + B.
+constexpr int kWgradStages = 4;
 constexpr uint32_t kStageB = kMaxBN * BLOCK_K * 2;       // 32 KiB
 constexpr int kMaxProblems = 8;
-constexpr uint32_t kStageOut = 32 * 64 * 2;              // 4 KiB result tile per epilogue warp (32 rows x 64 bf16)
-__host__ __device__ constexpr size_t smem_bytes_of(int mode) {
-    return 1024 + (size_t)stages_of(mode) * (kStageA + kStageB) + (mode == 2 ? 0 : kEpiWarps * kStageOut) + 512;
-}
+constexpr size_t kWgradSmem = 1024 + (size_t)kWgradStages * (kStageA + kStageB) + 512;
 
 enum TcMode { TC_FWD = 0, TC_DGRAD = 1, TC_WGRAD = 2 };
 
@@ -52,15 +48,34 @@ struct TcProblem {
     int net_id, layer_id;          // host side: which net and layer the problem belongs to
 };
 
+// Forward and data gradient run "weight-stationary": a CTA is bound to one slab (a problem's column
+// block of up to 256 output columns), keeps that slab of the weight operand in shared memory for the
+// whole launch where it fits, and walks the row tiles rank, rank + ctas, ... of the slab, so that only
+// the activations stream through the pipeline.
+constexpr int kMaxSlabs = 32;
+constexpr int kMaxCtas = 160;
+struct WsSlab {
+    int prob, n0;                  // problem and first output column
+    int cta_begin, cta_count;      // CTAs [cta_begin, cta_begin + cta_count) work on this slab
+    int resident;                  // 1: all k-blocks of the weight slab stay in shared memory
+    int stages;                    // pipeline stages (of A alone when resident, of A + B otherwise)
+};
+struct WsPlan {
+    WsSlab slab[kMaxSlabs];
+    int nslabs, grid, num_sms, mode;
+    unsigned char cta_slab[kMaxCtas];
+};
+
 struct TcParams {
     CUtensorMap tmA[kMaxProblems];
     CUtensorMap tmB[kMaxProblems];
-    CUtensorMap tmOut[kMaxProblems];   // BF16 output, boxes of 64 columns x 32 rows, 128-byte swizzle
+    CUtensorMap tmOut[kMaxProblems];   // BF16 output, boxes of 32 columns x 32 rows, 64-byte swizzle
     CUtensorMap tmAux[kMaxProblems];   // data gradient: stored post-activations, same boxes
     TcProblem p[kMaxProblems];
     int count, total_items;
     float alpha;
     int* error;
+    WsPlan ws;                         // forward / data gradient only
 };
 
 struct Item { int prob, m0, n0, kb0, kb1, split; };
@@ -84,21 +99,21 @@ __device__ __forceinline__ Item decode_item(const TcParams& P, int item) {
     return it;
 }
 
-template <int MODE>
-__global__ void __launch_bounds__(kThreads, 1) tc_gemm_kernel(const __grid_constant__ TcParams P) {
-    constexpr int kStages = stages_of(MODE);
+// Weight gradient: D[features_in x features_out] = A^T B over the minibatch rows, both operands as stored
+// ([row][feature], the contraction index outermost: MN-major tiles).  A work item is a 128 x (<= 256) tile of one
+// problem over one split of the row range; its FP32 result is a partial that the gradient reduction sums.
+__global__ void __launch_bounds__(kThreads, 1) wgrad_gemm_kernel(const __grid_constant__ TcParams P) {
+    constexpr int kStages = kWgradStages;
     extern __shared__ uint8_t smem_raw[];
     uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
     uint8_t* sA = smem;
     uint8_t* sB = smem + kStages * kStageA;
-    uint8_t* sOut = sB + kStages * kStageB;                 // kEpiWarps result tiles, 1 KiB aligned
-    uint64_t* full = reinterpret_cast<uint64_t*>(sOut + (MODE == TC_WGRAD ? 0 : kEpiWarps * kStageOut));
+    uint64_t* full = reinterpret_cast<uint64_t*>(sB + kStages * kStageB);
     uint64_t* empty = full + kStages;
     uint64_t* tfull = empty + kStages;
     uint64_t* tempty = tfull + 2;
     uint64_t* drain = tempty + 2;
-    uint64_t* auxbar = drain + 1;                           // one per epilogue warp
-    uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(auxbar + kEpiWarps);
+    uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(drain + 1);
     volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
@@ -108,18 +123,13 @@ __global__ void __launch_bounds__(kThreads, 1) tc_gemm_kernel(const __grid_const
         for (int s = 0; s < kStages; ++s) { mbar_init(&full[s], 1); mbar_init(&empty[s], 1); }
         for (int b = 0; b < 2; ++b) { mbar_init(&tfull[b], 1); mbar_init(&tempty[b], kEpiWarps); }
         mbar_init(drain, 1);
-        for (int w = 0; w < kEpiWarps; ++w) mbar_init(&auxbar[w], 1);
         *abort_flag = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
         asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
     }
     if (warp == 1) tmem_alloc(tmem_slot, kTmemCols);
     if (warp == 0 && lane == 0)
-        for (int i = 0; i < P.count; ++i) {
-            tma_prefetch_desc(&P.tmA[i]); tma_prefetch_desc(&P.tmB[i]);
-            if (MODE != TC_WGRAD) tma_prefetch_desc(&P.tmOut[i]);
-            if (MODE == TC_DGRAD) tma_prefetch_desc(&P.tmAux[i]);
-        }
+        for (int i = 0; i < P.count; ++i) { tma_prefetch_desc(&P.tmA[i]); tma_prefetch_desc(&P.tmB[i]); }
     tc_fence_before();
     __syncthreads();
     tc_fence_after();
@@ -128,42 +138,40 @@ __global__ void __launch_bounds__(kThreads, 1) tc_gemm_kernel(const __grid_const
 
     if (warp == 0) {
         // ================================ TMA producer =================================
-        if (lane == 0) {
-            int stage = 0; uint32_t phase = 0;
-            uint32_t issued_mask = 0, issued_parity = 0;
-            bool ok = true;
-            for (int item = blockIdx.x; ok && item < P.total_items; item += gridDim.x) {
-                const Item it = decode_item(P, item);
-                const TcProblem& p = P.p[it.prob];
-                const uint32_t bytes = (uint32_t)(BLOCK_M + p.bn) * BLOCK_K * 2;
-                for (int kb = it.kb0; kb < it.kb1; ++kb) {
-                    if (!mbar_wait(&empty[stage], phase ^ 1u, abort_flag, P.error, 1)) { ok = false; break; }
-                    mbar_expect_tx(&full[stage], bytes);
-                    uint8_t* a_dst = sA + stage * kStageA;
-                    uint8_t* b_dst = sB + stage * kStageB;
-                    if (MODE == TC_WGRAD) {
-                        // operands are [row][feature] with the feature contiguous: boxes of
-                        // 64 features x 64 rows, one 8 KiB block per 64 features
-                        for (int i = 0; i < 2; ++i)
-                            tma_load_2d(a_dst + i * 8192, &P.tmA[it.prob], it.m0 + 64 * i, kb * BLOCK_K, &full[stage]);
-                        for (int j = 0; j < p.bn / 64; ++j)
-                            tma_load_2d(b_dst + j * 8192, &P.tmB[it.prob], it.n0 + 64 * j, kb * BLOCK_K, &full[stage]);
-                    } else {
-                        tma_load_2d(a_dst, &P.tmA[it.prob], kb * BLOCK_K, it.m0, &full[stage]);
-                        tma_load_2d(b_dst, &P.tmB[it.prob], kb * BLOCK_K, it.n0, &full[stage]);
-                    }
-                    issued_mask |= 1u << stage;
-                    issued_parity = (issued_parity & ~(1u << stage)) | (phase << stage);
-                    if (++stage == kStages) { stage = 0; phase ^= 1u; }
+        // a k-block is six boxes of 64 features x 64 rows (two of A, up to four of B), one 8 KiB block per 64
+        // features: lane l issues box l, so that the whole k-block goes out in one pass of the loop
+        int stage = 0; uint32_t phase = 0;
+        uint32_t issued_mask = 0, issued_parity = 0;
+        bool ok = true;
+        for (int item = blockIdx.x; ok && item < P.total_items; item += gridDim.x) {
+            const Item it = decode_item(P, item);
+            const TcProblem& p = P.p[it.prob];
+            const uint32_t bytes = (uint32_t)(BLOCK_M + p.bn) * BLOCK_K * 2;
+            const bool mine = lane < 2 + p.bn / 64;
+            const CUtensorMap* tm = lane < 2 ? &P.tmA[it.prob] : &P.tmB[it.prob];
+            const int x = lane < 2 ? it.m0 + 64 * lane : it.n0 + 64 * (lane - 2);
+            uint8_t* base = lane < 2 ? sA + (uint32_t)lane * 8192u : sB + (uint32_t)(lane - 2) * 8192u;
+            const uint32_t per_stage = lane < 2 ? kStageA : kStageB;
+            for (int kb = it.kb0; kb < it.kb1; ++kb) {
+                int good = 1;
+                if (lane == 0) {
+                    good = mbar_wait(&empty[stage], phase ^ 1u, abort_flag, P.error, 1) ? 1 : 0;
+                    if (good) mbar_expect_tx(&full[stage], bytes);
                 }
+                good = __shfl_sync(0xffffffffu, good, 0);
+                if (!good) { ok = false; break; }
+                if (mine) tma_load_2d(base + (uint32_t)stage * per_stage, tm, x, kb * BLOCK_K, &full[stage]);
+                issued_mask |= 1u << stage;
+                issued_parity = (issued_parity & ~(1u << stage)) | (phase << stage);
+                if (++stage == kStages) { stage = 0; phase ^= 1u; }
             }
-            if (!ok) {
-                // let the copies already issued land before the CTA's shared memory goes away
-                for (int s = 0; s < kStages; ++s) {
-                    if (!(issued_mask & (1u << s))) continue;
-                    const unsigned long long t0 = global_ns();
-                    while (!mbar_try_wait(&full[s], (issued_parity >> s) & 1u) && global_ns() - t0 < kWaitLimitNs) {}
-                }
+        }
+        if (!ok && lane == 0) {
+            // let the copies already issued land before the CTA's shared memory goes away
+            for (int s = 0; s < kStages; ++s) {
+                if (!(issued_mask & (1u << s))) continue;
+                const unsigned long long t0 = global_ns();
+                while (!mbar_try_wait(&full[s], (issued_parity >> s) & 1u) && global_ns() - t0 < kWaitLimitNs) {}
             }
         }
     } else if (warp == 1) {
@@ -172,6 +180,10 @@ __global__ void __launch_bounds__(kThreads, 1) tc_gemm_kernel(const __grid_const
             int stage = 0; uint32_t phase = 0;
             bool ok = true;
             int local = 0;
+            // descriptors differ only in their address field (16-byte units): one add per stage and k-step
+            const uint64_t a_desc0 = smem_desc(smem_u32(sA), 8192, 1024);
+            const uint64_t b_desc0 = smem_desc(smem_u32(sB), 8192, 1024);
+            constexpr uint32_t kstep = (UMMA_K * 128) >> 4;
             for (int item = blockIdx.x; ok && item < P.total_items; item += gridDim.x, ++local) {
                 const Item it = decode_item(P, item);
                 const TcProblem& p = P.p[it.prob];
@@ -180,24 +192,16 @@ __global__ void __launch_bounds__(kThreads, 1) tc_gemm_kernel(const __grid_const
                 if (!mbar_wait(&tempty[buf], (use & 1u) ^ 1u, abort_flag, P.error, 2)) { ok = false; break; }
                 tc_fence_after();
                 const uint32_t d_tmem = tmem_base + (uint32_t)buf * kMaxBN;
-                const uint32_t idesc = instr_desc(p.bn, MODE == TC_WGRAD, MODE == TC_WGRAD);
+                const uint32_t idesc = instr_desc(p.bn, 1, 1);
                 for (int kb = it.kb0; kb < it.kb1; ++kb) {
                     if (!mbar_wait(&full[stage], phase, abort_flag, P.error, 3)) { ok = false; break; }
                     tc_fence_after();
-                    const uint32_t a_addr = smem_u32(sA + stage * kStageA);
-                    const uint32_t b_addr = smem_u32(sB + stage * kStageB);
-#pragma unroll
-                    for (int k = 0; k < BLOCK_K / UMMA_K; ++k) {
-                        uint64_t da, db;
-                        if (MODE == TC_WGRAD) {
-                            da = smem_desc(a_addr + k * (UMMA_K * 128), 8192, 1024);
-                            db = smem_desc(b_addr + k * (UMMA_K * 128), 8192, 1024);
-                        } else {
-                            da = smem_desc(a_addr + k * (UMMA_K * 2), 16, 1024);
-                            db = smem_desc(b_addr + k * (UMMA_K * 2), 16, 1024);
-                        }
-                        umma_bf16(d_tmem, da, db, idesc, (kb > it.kb0 || k > 0) ? 1u : 0u);
-                    }
+                    const uint64_t da = a_desc0 + (uint64_t)((uint32_t)stage * (kStageA >> 4));
+                    const uint64_t db = b_desc0 + (uint64_t)((uint32_t)stage * (kStageB >> 4));
+                    umma_bf16(d_tmem, da, db, idesc, kb > it.kb0 ? 1u : 0u);
+                    umma_bf16(d_tmem, da + kstep, db + kstep, idesc, 1u);
+                    umma_bf16(d_tmem, da + 2 * kstep, db + 2 * kstep, idesc, 1u);
+                    umma_bf16(d_tmem, da + 3 * kstep, db + 3 * kstep, idesc, 1u);
                     umma_commit(&empty[stage]);       // frees the stage once these MMAs have read it
                     if (++stage == kStages) { stage = 0; phase ^= 1u; }
                 }
@@ -216,16 +220,6 @@ __global__ void __launch_bounds__(kThreads, 1) tc_gemm_kernel(const __grid_const
         // ================================ epilogue =====================================
         const int q = warp & 3;                    // accumulator lanes 32q .. 32q+31
         const int group = (warp - 2) >> 2;         // handles the 64 columns [64 group, 64 group + 64) of the tile
-        // BF16 results leave through a 32 x 64 tile per warp and one TMA store per work item:
-        // lane r owns row r (128 bytes = eight 16-byte pieces), piece j is kept at j ^ (r & 7)
-        // (the 128-byte swizzle of the tensor map; conflict-free for the warp).  For the data
-        // gradient the same tile first receives the stored post-activations by TMA load.
-        uint8_t* tile = sOut + (warp - 2) * kStageOut;
-        uint8_t* tile_row = tile + lane * 128;
-        const int sw = lane & 7;
-        uint64_t* my_aux = &auxbar[warp - 2];
-        uint32_t aux_phase = 0;
-        bool aux_pending = false;
         bool ok = true;
         int local = 0;
         for (int item = blockIdx.x; ok && item < P.total_items; item += gridDim.x, ++local) {
@@ -235,27 +229,9 @@ __global__ void __launch_bounds__(kThreads, 1) tc_gemm_kernel(const __grid_const
             const uint32_t use = (uint32_t)(local >> 1);
             const int row = it.m0 + 32 * q + lane;
             const int chunks = p.bn / 32;
-            const int col0 = it.n0 + 64 * group;                          // first column of this warp
-            const bool active = 2 * group < chunks && col0 < p.n_extent;  // uniform across the warp
-            if (MODE != TC_WGRAD && active) {
-                // the previous item's store must have read the tile before it is reused
-                if (lane == 0) {
-                    tma_store_wait_read();
-                    if (MODE == TC_DGRAD) {
-                        mbar_expect_tx(my_aux, kStageOut);
-                        tma_load_2d(tile, &P.tmAux[it.prob], col0, it.m0 + 32 * q, my_aux);
-                    }
-                }
-                if (MODE == TC_DGRAD) aux_pending = true;
-                __syncwarp();
-            }
+            const bool active = 2 * group < chunks && it.n0 + 64 * group < p.n_extent;   // uniform across the warp
             if (!mbar_wait(&tfull[buf], use & 1u, abort_flag, P.error, 4)) { ok = false; break; }
             tc_fence_after();
-            if (MODE == TC_DGRAD && active) {
-                if (!mbar_wait(my_aux, aux_phase, abort_flag, P.error, 5)) { ok = false; break; }
-                aux_phase ^= 1u;
-                aux_pending = false;
-            }
 #pragma unroll
             for (int ci = 0; ci < 2; ++ci) {
                 if (!active) break;
@@ -263,42 +239,7 @@ __global__ void __launch_bounds__(kThreads, 1) tc_gemm_kernel(const __grid_const
                 uint32_t acc[32];
                 tmem_ld32(tmem_base + ((uint32_t)(32 * q) << 16) + (uint32_t)(buf * kMaxBN + 32 * c), acc);
                 const int col = it.n0 + 32 * c;
-                if (MODE == TC_FWD) {
-                    // p.bias is zero-padded to the padded width: no bounds checks
-                    const float4* b4 = reinterpret_cast<const float4*>(p.bias + col);
-#pragma unroll
-                    for (int g = 0; g < 4; ++g) {
-                        const float4 ba = __ldg(b4 + 2 * g), bb = __ldg(b4 + 2 * g + 1);
-                        const float bv[8] = {ba.x, ba.y, ba.z, ba.w, bb.x, bb.y, bb.z, bb.w};
-                        uint32_t o[4];
-#pragma unroll
-                        for (int e = 0; e < 4; ++e) {
-                            const float v0 = elu_fast(__uint_as_float(acc[8 * g + 2 * e]) + bv[2 * e], P.alpha);
-                            const float v1 = elu_fast(__uint_as_float(acc[8 * g + 2 * e + 1]) + bv[2 * e + 1], P.alpha);
-                            __nv_bfloat162 h2 = __floats2bfloat162_rn(v0, v1);
-                            o[e] = *reinterpret_cast<uint32_t*>(&h2);
-                        }
-                        *reinterpret_cast<uint4*>(tile_row + (((4 * ci + g) ^ sw) << 4)) = make_uint4(o[0], o[1], o[2], o[3]);
-                    }
-                } else if (MODE == TC_DGRAD) {
-#pragma unroll
-                    for (int g = 0; g < 4; ++g) {
-                        uint4* piece = reinterpret_cast<uint4*>(tile_row + (((4 * ci + g) ^ sw) << 4));
-                        const uint4 hv = *piece;
-                        const uint32_t hw[4] = {hv.x, hv.y, hv.z, hv.w};
-                        uint32_t o[4];
-#pragma unroll
-                        for (int e = 0; e < 4; ++e) {
-                            const __nv_bfloat162 h2 = *reinterpret_cast<const __nv_bfloat162*>(&hw[e]);
-                            const float h0 = __low2float(h2), h1 = __high2float(h2);
-                            const float v0 = __uint_as_float(acc[8 * g + 2 * e]) * (h0 > 0.f ? 1.0f : h0 + P.alpha);
-                            const float v1 = __uint_as_float(acc[8 * g + 2 * e + 1]) * (h1 > 0.f ? 1.0f : h1 + P.alpha);
-                            __nv_bfloat162 r2 = __floats2bfloat162_rn(v0, v1);
-                            o[e] = *reinterpret_cast<uint32_t*>(&r2);
-                        }
-                        *piece = make_uint4(o[0], o[1], o[2], o[3]);
-                    }
-                } else if (row < p.m_extent) {
+                if (row < p.m_extent) {
                     float* dst = p.out32 + (size_t)it.split * p.split_stride + (size_t)row * p.ld_out32 + col;
 #pragma unroll
                     for (int g = 0; g < 8; ++g)
@@ -308,39 +249,316 @@ __global__ void __launch_bounds__(kThreads, 1) tc_gemm_kernel(const __grid_const
                                             __uint_as_float(acc[4 * g + 2]), __uint_as_float(acc[4 * g + 3]));
                 }
             }
-            // the accumulator has been read: hand the tensor-memory buffer back first
+            // the accumulator has been read: hand the tensor-memory buffer back
             tc_fence_before();
             __syncwarp();
             if (lane == 0) mbar_arrive(&tempty[buf]);
-            if (MODE != TC_WGRAD && active) {
-                fence_async_smem();                           // tile writes -> visible to the copy engine
-                __syncwarp();
-                // rows at or beyond the tensor's extent are clipped by the store itself
-                if (lane == 0 && it.m0 + 32 * q < p.m_extent)
-                    tma_store_2d(&P.tmOut[it.prob], tile, col0, it.m0 + 32 * q);
-                if (MODE == TC_DGRAD && p.colsum) {
-                    // partial bias gradient: lane l adds columns 2l, 2l+1 of the tile's 32 rows (rows past
-                    // the extent hold zeros); the 32 words of a row sit in 32 different banks
-                    float s0 = 0.f, s1 = 0.f;
-                    const uint8_t* mine = tile + ((lane & 3) << 2);
-#pragma unroll
-                    for (int r = 0; r < 32; ++r) {
-                        const uint32_t w = *reinterpret_cast<const uint32_t*>(mine + r * 128 + ((((lane >> 2) ^ (r & 7))) << 4));
-                        const __nv_bfloat162 v2 = *reinterpret_cast<const __nv_bfloat162*>(&w);
-                        s0 += __low2float(v2); s1 += __high2float(v2);
-                    }
-                    *reinterpret_cast<float2*>(p.colsum + (size_t)(it.m0 / BLOCK_M * 4 + q) * p.ld_colsum + col0 + 2 * lane) =
-                        make_float2(s0, s1);
+        }
+    }
+    tc_fence_before();
+    __syncthreads();
+    if (warp == 1) {
+        tc_fence_after();
+        tmem_dealloc(tmem_base, kTmemCols);
+    }
+}
+
+// ------------------------------------------------------------------ weight-stationary GEMM
+// Forward (MODE 0) and data gradient (MODE 1).  Shared memory: a 2 KiB result tile per epilogue warp
+// (32 rows x 32 BF16, 64-byte swizzle, one TMA store per 32-column chunk), then the operands: the
+// resident weight slab (k-blocks of bn rows x 128 bytes) followed by the A stages of 16 KiB, or, where
+// the slab does not fit, stages of A + B.  Tensor memory: two accumulators of 256 columns, so that the
+// epilogue of a row tile overlaps the products of the next.
+constexpr int kWsMaxStages = 8;
+constexpr uint32_t kWsStageOut = 32 * 32 * 2;
+constexpr uint32_t kWsBarBytes = 512;
+constexpr uint32_t kWsSmem = 232448;                                // the 227 KiB a CTA may have
+constexpr uint32_t kWsAuxBox = 128 * 32 * 2;                         // 32 columns x 128 rows of stored post-activations
+constexpr uint32_t kWsAuxTile = 4 * kWsAuxBox;                       // a row tile of up to 128 columns
+// result tiles (one per epilogue warp) and, for the data gradient, two tiles of stored post-activations
+__host__ __device__ constexpr uint32_t ws_staging(int mode) { return kEpiWarps * kWsStageOut + (mode == 1 ? 2u * kWsAuxTile : 0u); }
+__host__ __device__ constexpr uint32_t ws_operand_bytes(int mode) { return (kWsSmem - 1024 - ws_staging(mode) - kWsBarBytes) / 1024 * 1024; }
+
+template <int MODE>
+__global__ void __launch_bounds__(kThreads, 1) ws_gemm_kernel(const __grid_constant__ TcParams P) {
+    extern __shared__ uint8_t smem_raw[];
+    uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
+    uint8_t* sOut = smem;                                   // a 2 KiB result tile per epilogue warp
+    uint8_t* sAux = smem + kEpiWarps * kWsStageOut;          // data gradient: two tiles of stored post-activations
+    uint8_t* sOp = smem + ws_staging(MODE);
+    uint64_t* full = reinterpret_cast<uint64_t*>(sOp + ws_operand_bytes(MODE));
+    uint64_t* empty = full + kWsMaxStages;
+    uint64_t* tfull = empty + kWsMaxStages;
+    uint64_t* tempty = tfull + 2;
+    uint64_t* bfull = tempty + 2;
+    uint64_t* drain = bfull + 1;
+    uint64_t* auxfull = drain + 1;                           // data gradient: post-activations of a row tile have landed
+    uint64_t* auxempty = auxfull + 2;                        // ... and have been read by every epilogue warp
+    uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(auxempty + 2);
+    volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
+
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const WsSlab& S = P.ws.slab[P.ws.cta_slab[blockIdx.x]];
+    const TcProblem& p = P.p[S.prob];
+    const int rank = (int)blockIdx.x - S.cta_begin;
+    const int nst = S.stages;
+    const uint32_t b_kb_bytes = (uint32_t)p.bn * 128u;
+    const uint32_t stage_bytes = S.resident ? kStageA : kStageA + b_kb_bytes;
+    uint8_t* sB = sOp;
+    uint8_t* sA = sOp + (S.resident ? (uint32_t)p.kblocks * b_kb_bytes : 0u);
+    // set-up: shared memory, tensor memory and kernel parameters only (may overlap the preceding kernel's tail)
+    if (threadIdx.x == 0) {
+        for (int s = 0; s < kWsMaxStages; ++s) { mbar_init(&full[s], 1); mbar_init(&empty[s], 1); }
+        for (int b = 0; b < 2; ++b) { mbar_init(&tfull[b], 1); mbar_init(&tempty[b], kEpiWarps); }
+        mbar_init(bfull, 1); mbar_init(drain, 1);
+        for (int b = 0; b < 2; ++b) { mbar_init(&auxfull[b], 1); mbar_init(&auxempty[b], kEpiWarps); }
+        *abort_flag = 0;
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+        asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+    }
+    if (warp == 1) tmem_alloc(tmem_slot, kTmemCols);
+    if (warp == 0 && lane == 0) {
+        tma_prefetch_desc(&P.tmA[S.prob]); tma_prefetch_desc(&P.tmB[S.prob]); tma_prefetch_desc(&P.tmOut[S.prob]);
+        if (MODE == TC_DGRAD) tma_prefetch_desc(&P.tmAux[S.prob]);
+    }
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    const uint32_t tmem_base = *tmem_slot;
+    chain_wait();
+
+    if (warp == 0) {
+        // ================================ TMA producer =================================
+        if (lane == 0) {
+            const CUtensorMap* tmA = &P.tmA[S.prob];
+            const CUtensorMap* tmB = &P.tmB[S.prob];
+            if (S.resident) {
+                mbar_expect_tx(bfull, (uint32_t)p.kblocks * b_kb_bytes);
+                for (int kb = 0; kb < p.kblocks; ++kb) tma_load_2d(sB + (uint32_t)kb * b_kb_bytes, tmB, kb * BLOCK_K, S.n0, bfull);
+            }
+            int stage = 0; uint32_t phase = 0;
+            uint32_t issued_mask = 0, issued_parity = 0, aux_issued = 0, aux_parity = 0;
+            bool ok = true;
+            int local = 0;
+            const int nchunks = min(p.bn, p.n_extent - S.n0) / 32;     // 32-column chunks of the slab that exist
+            for (int mt = rank; ok && mt < p.m_tiles; mt += S.cta_count, ++local) {
+                const int m0 = mt * BLOCK_M;
+                for (int kb = 0; kb < p.kblocks; ++kb) {
+                    if (!mbar_wait(&empty[stage], phase ^ 1u, abort_flag, P.error, 1)) { ok = false; break; }
+                    mbar_expect_tx(&full[stage], stage_bytes);
+                    uint8_t* dst = sA + (uint32_t)stage * stage_bytes;
+                    tma_load_2d(dst, tmA, kb * BLOCK_K, m0, &full[stage]);
+                    if (!S.resident) tma_load_2d(dst + kStageA, tmB, kb * BLOCK_K, S.n0, &full[stage]);
+                    issued_mask |= 1u << stage;
+                    issued_parity = (issued_parity & ~(1u << stage)) | (phase << stage);
+                    if (++stage == nst) { stage = 0; phase ^= 1u; }
+                }
+                if (MODE == TC_DGRAD && ok) {
+                    // stored post-activations of the row tile, one box of 32 columns x 128 rows per chunk, fetched
+                    // behind the operands of the tile (the epilogue reads them after the products)
+                    const int ab = local & 1;
+                    if (!mbar_wait(&auxempty[ab], (((uint32_t)local >> 1) & 1u) ^ 1u, abort_flag, P.error, 7)) { ok = false; break; }
+                    mbar_expect_tx(&auxfull[ab], (uint32_t)nchunks * kWsAuxBox);
+                    for (int c = 0; c < nchunks; ++c)
+                        tma_load_2d(sAux + (uint32_t)ab * kWsAuxTile + (uint32_t)c * kWsAuxBox, &P.tmAux[S.prob], S.n0 + 32 * c, m0, &auxfull[ab]);
+                    aux_issued |= 1u << ab;
+                    aux_parity = (aux_parity & ~(1u << ab)) | ((((uint32_t)local >> 1) & 1u) << ab);
+                }
+            }
+            if (!ok) {
+                // let the copies already issued land before the CTA's shared memory goes away
+                for (int s = 0; s < nst; ++s) {
+                    if (!(issued_mask & (1u << s))) continue;
+                    const unsigned long long t0 = global_ns();
+                    while (!mbar_try_wait(&full[s], (issued_parity >> s) & 1u) && global_ns() - t0 < kWaitLimitNs) {}
+                }
+                if (S.resident) {
+                    const unsigned long long t0 = global_ns();
+                    while (!mbar_try_wait(bfull, 0) && global_ns() - t0 < kWaitLimitNs) {}
+                }
+                for (int ab = 0; ab < 2; ++ab) {
+                    if (!(aux_issued & (1u << ab))) continue;
+                    const unsigned long long t0 = global_ns();
+                    while (!mbar_try_wait(&auxfull[ab], (aux_parity >> ab) & 1u) && global_ns() - t0 < kWaitLimitNs) {}
                 }
             }
         }
-        if (MODE != TC_WGRAD && lane == 0) {
-            if (aux_pending) {      // gave up with a load in flight: let it land first
-                const unsigned long long t0 = global_ns();
-                while (!mbar_try_wait(my_aux, aux_phase) && global_ns() - t0 < kWaitLimitNs) {}
+    } else if (warp == 1) {
+        // ================================ MMA issuer ===================================
+        if (lane == 0) {
+            int stage = 0; uint32_t phase = 0;
+            bool ok = true;
+            const uint32_t idesc = instr_desc(p.bn, 0, 0);
+            // operand descriptors differ only in their address field (16-byte units, no carry out of it for
+            // shared-memory addresses): one add per stage / k-block / k-step instead of a rebuild
+            const uint64_t a_desc0 = smem_desc(smem_u32(sA), 16, 1024);
+            const uint64_t b_desc0 = smem_desc(smem_u32(S.resident ? sB : sA + kStageA), 16, 1024);
+            const uint64_t a_step = stage_bytes >> 4;
+            const uint64_t b_step = S.resident ? (b_kb_bytes >> 4) : a_step;
+            const int kblocks = p.kblocks;
+            const bool resident = S.resident != 0;
+            if (resident && !mbar_wait(bfull, 0, abort_flag, P.error, 6)) ok = false;
+            uint64_t a_desc = a_desc0, b_desc_stream = b_desc0;
+            int local = 0;
+            for (int mt = rank; ok && mt < p.m_tiles; mt += S.cta_count, ++local) {
+                const int buf = local & 1;
+                const uint32_t use = (uint32_t)(local >> 1);
+                if (!mbar_wait(&tempty[buf], (use & 1u) ^ 1u, abort_flag, P.error, 2)) { ok = false; break; }
+                tc_fence_after();
+                const uint32_t d_tmem = tmem_base + (uint32_t)buf * kMaxBN;
+                uint64_t b_res = b_desc0;
+                for (int kb = 0; kb < kblocks; ++kb) {
+                    if (!mbar_wait(&full[stage], phase, abort_flag, P.error, 3)) { ok = false; break; }
+                    tc_fence_after();
+                    const uint64_t db = resident ? b_res : b_desc_stream;
+                    umma_bf16(d_tmem, a_desc, db, idesc, kb > 0 ? 1u : 0u);
+                    umma_bf16(d_tmem, a_desc + 2, db + 2, idesc, 1u);
+                    umma_bf16(d_tmem, a_desc + 4, db + 4, idesc, 1u);
+                    umma_bf16(d_tmem, a_desc + 6, db + 6, idesc, 1u);
+                    umma_commit(&empty[stage]);       // frees the stage once these MMAs have read it
+                    b_res += b_step;
+                    a_desc += a_step; b_desc_stream += a_step;
+                    if (++stage == nst) { stage = 0; phase ^= 1u; a_desc = a_desc0; b_desc_stream = b_desc0; }
+                }
+                if (ok) umma_commit(&tfull[buf]);     // accumulator complete
             }
-            tma_store_wait_all();   // stores done before the CTA retires
+            // all products of this CTA are issued: the next kernel of the stream may be scheduled and set
+            // itself up while the last accumulators drain (it waits for this grid before it reads)
+            chain_release();
+            if (!ok) {
+                umma_commit(drain);
+                const unsigned long long t0 = global_ns();
+                while (!mbar_try_wait(drain, 0) && global_ns() - t0 < kWaitLimitNs) {}
+            }
         }
+    } else {
+        // ================================ epilogue =====================================
+        const int q = warp & 3;                    // accumulator lanes 32q .. 32q+31
+        const int group = (warp - 2) >> 2;         // the 32-column chunks group and group + 4 of the tile
+        // lane r owns row r of a 32 x 32 BF16 tile (64 bytes = four 16-byte pieces); piece j is kept at
+        // j ^ ((r >> 1) & 3), the 64-byte swizzle of the tensor maps (conflict-free for the warp).
+        // Data gradient: the stored post-activations of the row tile are read from the tile the producer fetched
+        // (same layout, rows 32q.. of the chunk's box).
+        uint8_t* tile = sOut + (warp - 2) * kWsStageOut;
+        uint8_t* tile_row = tile + lane * 64;
+        const int sw = (lane >> 1) & 3;
+        bool ok = true;
+        const int chunks = p.bn / 32;
+        // this warp's chunks that exist (uniform across the warp): with up to 128 columns every warp has at most one
+        int nact = 0;
+        for (int ci = 0; ci < 2; ++ci)
+            if (group + 4 * ci < chunks && S.n0 + 32 * (group + 4 * ci) < p.n_extent) nact = ci + 1;
+        const CUtensorMap* tmOut = &P.tmOut[S.prob];
+        int local = 0;
+        for (int mt = rank; ok && mt < p.m_tiles; mt += S.cta_count, ++local) {
+            const int m0 = mt * BLOCK_M;
+            const int buf = local & 1;
+            const uint32_t use = (uint32_t)(local >> 1);
+            const int row0 = m0 + 32 * q;
+            if (!mbar_wait(&tfull[buf], use & 1u, abort_flag, P.error, 4)) { ok = false; break; }
+            tc_fence_after();
+            if (MODE == TC_DGRAD && !mbar_wait(&auxfull[buf], use & 1u, abort_flag, P.error, 5)) { ok = false; break; }
+            const uint32_t t_row = tmem_base + ((uint32_t)(32 * q) << 16) + (uint32_t)(buf * kMaxBN);
+            // the accumulator is read in pieces of 16 columns, each fetched while the piece before is worked on
+            uint32_t acc[2][16];
+            if (nact > 0) tmem_ld16_issue(t_row + (uint32_t)(32 * group), acc[0]);
+#pragma unroll
+            for (int ci = 0; ci < 2; ++ci) {
+                if (ci >= nact) break;
+                const int c = group + 4 * ci;
+                const int col = S.n0 + 32 * c;
+                const uint8_t* aux_row = sAux + (uint32_t)buf * kWsAuxTile + (uint32_t)c * kWsAuxBox + (uint32_t)(32 * q + lane) * 64u;
+                // the previous chunk's store must have read the tile before it is rewritten
+                if (lane == 0) tma_store_wait_read();
+                __syncwarp();
+#pragma unroll
+                for (int half = 0; half < 2; ++half) {
+                    uint32_t (&cur)[16] = acc[half];
+                    float bv[16];
+                    if (MODE == TC_FWD) {
+                        // p.bias is zero-padded to the padded width: no bounds checks
+                        const float4* b4 = reinterpret_cast<const float4*>(p.bias + col + 16 * half);
+#pragma unroll
+                        for (int g = 0; g < 4; ++g) {
+                            const float4 t4 = __ldg(b4 + g);
+                            bv[4 * g] = t4.x; bv[4 * g + 1] = t4.y; bv[4 * g + 2] = t4.z; bv[4 * g + 3] = t4.w;
+                        }
+                    }
+                    tmem_ld16_wait(cur);
+                    // next piece: the other half of this chunk, or the first half of the warp's second chunk
+                    if (half == 0) tmem_ld16_issue(t_row + (uint32_t)(32 * c + 16), acc[1]);
+                    else if (ci + 1 < nact) tmem_ld16_issue(t_row + (uint32_t)(32 * (c + 4)), acc[0]);
+                    else {
+                        // (issued loads are complete at this point) the accumulator has been read: hand the buffer back
+                        tc_fence_before();
+                        __syncwarp();
+                        if (lane == 0) mbar_arrive(&tempty[buf]);
+                    }
+#pragma unroll
+                    for (int g = 0; g < 2; ++g) {
+                        uint32_t o[4];
+                        uint4* piece = reinterpret_cast<uint4*>(tile_row + (((2 * half + g) ^ sw) << 4));
+                        if (MODE == TC_FWD) {
+#pragma unroll
+                            for (int e = 0; e < 4; ++e) {
+                                const float v0 = elu_fast(__uint_as_float(cur[8 * g + 2 * e]) + bv[8 * g + 2 * e], P.alpha);
+                                const float v1 = elu_fast(__uint_as_float(cur[8 * g + 2 * e + 1]) + bv[8 * g + 2 * e + 1], P.alpha);
+                                __nv_bfloat162 h2 = __floats2bfloat162_rn(v0, v1);
+                                o[e] = *reinterpret_cast<uint32_t*>(&h2);
+                            }
+                        } else {
+                            const uint4 hv = *reinterpret_cast<const uint4*>(aux_row + (((2 * half + g) ^ sw) << 4));
+                            const uint32_t hw[4] = {hv.x, hv.y, hv.z, hv.w};
+#pragma unroll
+                            for (int e = 0; e < 4; ++e) {
+                                const __nv_bfloat162 h2 = *reinterpret_cast<const __nv_bfloat162*>(&hw[e]);
+                                const float h0 = __low2float(h2), h1 = __high2float(h2);
+                                const float v0 = __uint_as_float(cur[8 * g + 2 * e]) * (h0 > 0.f ? 1.0f : h0 + P.alpha);
+                                const float v1 = __uint_as_float(cur[8 * g + 2 * e + 1]) * (h1 > 0.f ? 1.0f : h1 + P.alpha);
+                                __nv_bfloat162 r2 = __floats2bfloat162_rn(v0, v1);
+                                o[e] = *reinterpret_cast<uint32_t*>(&r2);
+                            }
+                        }
+                        *piece = make_uint4(o[0], o[1], o[2], o[3]);
+                    }
+                }
+                fence_async_smem();                           // tile writes -> visible to the copy engine
+                __syncwarp();
+                // rows at or beyond the tensor's extent are clipped by the store itself
+                if (lane == 0 && row0 < p.m_extent) tma_store_2d(tmOut, tile, col, row0);
+                if (MODE == TC_DGRAD) {
+                    if (p.colsum) {
+                        // partial bias gradient: lanes 0..15 add columns 2l, 2l+1 over rows 0..15 of the tile, lanes
+                        // 16..31 over rows 16..31 (rows past the extent hold zeros)
+                        float s0 = 0.f, s1 = 0.f;
+                        const int cp = lane & 15, rbase = lane & 16;
+                        const uint8_t* mine = tile + ((cp & 3) << 2);
+#pragma unroll
+                        for (int r = 0; r < 16; ++r) {
+                            const int rr = rbase + r;
+                            const uint32_t w = *reinterpret_cast<const uint32_t*>(mine + rr * 64 + (((cp >> 2) ^ ((rr >> 1) & 3)) << 4));
+                            const __nv_bfloat162 v2 = *reinterpret_cast<const __nv_bfloat162*>(&w);
+                            s0 += __low2float(v2); s1 += __high2float(v2);
+                        }
+                        s0 += __shfl_xor_sync(0xffffffffu, s0, 16);
+                        s1 += __shfl_xor_sync(0xffffffffu, s1, 16);
+                        if (lane < 16)
+                            *reinterpret_cast<float2*>(p.colsum + (size_t)(mt * 4 + q) * p.ld_colsum + col + 2 * cp) = make_float2(s0, s1);
+                    }
+                }
+            }
+            if (MODE == TC_DGRAD) {
+                // this warp has read its part of the row tile's post-activations
+                __syncwarp();
+                if (lane == 0) mbar_arrive(&auxempty[buf]);
+            }
+            if (nact == 0) {
+                tc_fence_before();
+                __syncwarp();
+                if (lane == 0) mbar_arrive(&tempty[buf]);
+            }
+        }
+        if (lane == 0) tma_store_wait_all();   // stores done before the CTA retires
     }
     tc_fence_before();
     __syncthreads();
@@ -751,15 +969,12 @@ struct UmmaEngine {
     // fused forward (one launch for all hidden layers) where the widths allow it, else empty
     std::vector<ChainParams> chain_act, chain_act_critic;
     ColsumBatch colsum{}, colsum_rest{};         // all layers the epilogue does not cover / those minus the last ones
-    // fused row-local step kernel (no mirrored rows): head operand copies, bias-gradient partials of every hidden layer
-    StepChain* step = nullptr;
+    // head operand copies (output-major with high and low parts, input-major)
     __nv_bfloat16 *wht[2] = {}, *whn[2] = {};
     float* head_bias_pad[2] = {};
     bool head_copies = false;                    // the optimiser step keeps wht / whn / head_bias_pad current
     int head_n[2] = {};                          // head outputs rounded up to 16; wht rows [head_n, 2 head_n) hold the
                                                  // low-order parts of the weights (what BF16 rounding left)
-    float* step_slots[2][kMaxLayers] = {};
-    int step_slot_rows = 0;
 };
 
 namespace {
@@ -786,6 +1001,8 @@ void finish_params(TcParams& P, float alpha, int* error) {
     P.error = error;
 }
 
+void plan_ws(TcParams& P, int num_sms, int mode);
+
 // The problems of one net out of a launch's parameters, as a launch of their own (no items if there are none).
 TcParams only_net(const TcParams& P, int ni) {
     TcParams Q;
@@ -797,15 +1014,16 @@ TcParams only_net(const TcParams& P, int ni) {
         Q.p[j] = P.p[i];
     }
     finish_params(Q, P.alpha, P.error);
+    plan_ws(Q, P.ws.num_sms, P.ws.mode);
     return Q;
 }
 
 // D[rows x width_out] = A[rows x k] * B[width_out x k]^T, both operands contraction-major.
-bool add_rowmajor_problem(TcParams& P, const __nv_bfloat16* A, int rows, int k, const __nv_bfloat16* B, int width_out) {
+bool add_rowmajor_problem(TcParams& P, const __nv_bfloat16* A, int rows, int k, const __nv_bfloat16* B, int width_out, int max_bn = kMaxBN) {
     const int i = P.count;
     TcProblem& p = P.p[i];
     memset(&p, 0, sizeof p);
-    p.bn = pick_bn(width_out);
+    p.bn = std::min(max_bn, pick_bn(width_out));
     p.m_extent = rows; p.n_extent = width_out;
     p.m_tiles = (rows + BLOCK_M - 1) / BLOCK_M;
     p.n_tiles = (width_out + p.bn - 1) / p.bn;
@@ -816,12 +1034,63 @@ bool add_rowmajor_problem(TcParams& P, const __nv_bfloat16* A, int rows, int k, 
     return true;
 }
 
+// Binds the CTAs of a forward / data-gradient launch to slabs.  Every slab starts with one CTA; the rest go,
+// one at a time, to the slab whose busiest CTA has the most work left (row tiles x cost of a tile), so that
+// the slabs finish together.  The cost of a tile is what bounds it: its products or its epilogue.
+void plan_ws(TcParams& P, int num_sms, int mode) {
+    WsPlan& W = P.ws;
+    memset(&W, 0, sizeof W);
+    W.num_sms = num_sms; W.mode = mode;
+    const uint32_t kWsOperandBytes = ws_operand_bytes(mode);
+    struct Cost { int m_tiles; double tile; };
+    Cost cost[kMaxSlabs];
+    for (int i = 0; i < P.count; ++i) {
+        const TcProblem& p = P.p[i];
+        for (int nt = 0; nt < p.n_tiles && W.nslabs < kMaxSlabs; ++nt) {
+            WsSlab& S = W.slab[W.nslabs];
+            S.prob = i; S.n0 = nt * p.bn;
+            const uint32_t b_bytes = (uint32_t)p.kblocks * (uint32_t)p.bn * 128u;
+            S.resident = b_bytes + 3u * kStageA <= kWsOperandBytes ? 1 : 0;
+            const uint32_t per_stage = S.resident ? kStageA : kStageA + (uint32_t)p.bn * 128u;
+            S.stages = (int)std::min<uint32_t>(kWsMaxStages, (kWsOperandBytes - (S.resident ? b_bytes : 0u)) / per_stage);
+            const double mma = 512.0 * p.kblocks * p.bn / 256.0, epi = 2800.0 * p.bn / 256.0;
+            cost[W.nslabs] = Cost{p.m_tiles, std::max(mma, epi) + 300.0};
+            W.nslabs++;
+        }
+    }
+    if (W.nslabs == 0) { W.grid = 0; return; }
+    int alloc[kMaxSlabs];
+    int used = 0;
+    for (int i = 0; i < W.nslabs; ++i) { alloc[i] = 1; used++; }
+    const int max_ctas = std::min(num_sms, kMaxCtas);
+    auto load = [&](int i) { return ((cost[i].m_tiles + alloc[i] - 1) / alloc[i]) * cost[i].tile; };
+    while (used < max_ctas) {
+        int best = -1;
+        for (int i = 0; i < W.nslabs; ++i)
+            if (alloc[i] < cost[i].m_tiles && (best < 0 || load(i) > load(best))) best = i;
+        if (best < 0) break;
+        alloc[best]++; used++;
+    }
+    int cta = 0;
+    for (int i = 0; i < W.nslabs; ++i) {
+        W.slab[i].cta_begin = cta; W.slab[i].cta_count = alloc[i];
+        for (int k = 0; k < alloc[i]; ++k) W.cta_slab[cta++] = (unsigned char)i;
+    }
+    W.grid = cta;
+}
+
 template <int MODE>
-cudaError_t launch_tc(const TcParams& P, int num_sms, cudaStream_t s) {
+cudaError_t launch_ws(const TcParams& P, cudaStream_t s) {
+    if (P.total_items == 0 || P.ws.grid == 0) return cudaSuccess;
+    LaunchScope scope_(MODE == TC_FWD ? "tc_gemm_fwd" : "tc_gemm_dgrad", s);
+    return launch_chained(ws_gemm_kernel<MODE>, P.ws.grid, kThreads, kWsSmem, s, P);
+}
+
+cudaError_t launch_wgrad(const TcParams& P, int num_sms, cudaStream_t s) {
     if (P.total_items == 0) return cudaSuccess;
     const int grid = std::min(P.total_items, num_sms);
-    LaunchScope scope_(MODE == TC_FWD ? "tc_gemm_fwd" : MODE == TC_DGRAD ? "tc_gemm_dgrad" : "tc_gemm_wgrad", s);
-    return launch_chained(tc_gemm_kernel<MODE>, grid, kThreads, smem_bytes_of(MODE), s, P);
+    LaunchScope scope_("tc_gemm_wgrad", s);
+    return launch_chained(wgrad_gemm_kernel, grid, kThreads, kWgradSmem, s, P);
 }
 
 
@@ -971,9 +1240,10 @@ UmmaEngine* umma_create(const UmmaSetup& s, std::string* err) {
     int dev = 0; cudaDeviceProp prop;
     if (cudaGetDevice(&dev) != cudaSuccess || cudaGetDeviceProperties(&prop, dev) != cudaSuccess) return failmsg("no CUDA device");
     if (prop.major != 10) return failmsg("the tensor-core mode needs an sm_100 device");
-    if (cudaFuncSetAttribute(tc_gemm_kernel<TC_FWD>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem_bytes_of(TC_FWD)) != cudaSuccess ||
-        cudaFuncSetAttribute(tc_gemm_kernel<TC_DGRAD>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem_bytes_of(TC_DGRAD)) != cudaSuccess ||
-        cudaFuncSetAttribute(tc_gemm_kernel<TC_WGRAD>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem_bytes_of(TC_WGRAD)) != cudaSuccess)
+    if (cudaFuncSetAttribute(wgrad_gemm_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kWgradSmem) != cudaSuccess)
+        return failmsg("could not reserve shared memory for the tensor-core kernels");
+    if (cudaFuncSetAttribute(ws_gemm_kernel<TC_FWD>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kWsSmem) != cudaSuccess ||
+        cudaFuncSetAttribute(ws_gemm_kernel<TC_DGRAD>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kWsSmem) != cudaSuccess)
         return failmsg("could not reserve shared memory for the tensor-core kernels");
     if (cudaFuncSetAttribute(chain_fwd_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kChainSmem) != cudaSuccess)
         return failmsg("could not reserve shared memory for the fused forward kernel");
@@ -1062,9 +1332,10 @@ UmmaEngine* umma_create(const UmmaSetup& s, std::string* err) {
                 p.bias = e->bias_pad[ni][l]; p.bias_n = e->pw[ni][l];
                 p.net_id = ni; p.layer_id = l;
                 p.out16 = act_buffers ? e->h_act[ni][l] : e->h[ni][l]; p.ld_out = e->pw[ni][l];
-                if (!make_tmap(&P.tmOut[P.count - 1], p.out16, rows, e->pw[ni][l], e->pw[ni][l], 64, 32)) return false;
+                if (!make_tmap(&P.tmOut[P.count - 1], p.out16, rows, e->pw[ni][l], e->pw[ni][l], 32, 32, CU_TENSOR_MAP_SWIZZLE_64B)) return false;
             }
             finish_params(P, alpha, e->error_dev);
+            plan_ws(P, e->num_sms, TC_FWD);
             out.push_back(P);
         }
         return true;
@@ -1130,7 +1401,9 @@ UmmaEngine* umma_create(const UmmaSetup& s, std::string* err) {
         for (int ni = 0; ni < 2; ++ni) {
             const int l = e->nh[ni] - 1 - b;
             if (l < 1) continue;
-            if (!add_rowmajor_problem(P, e->dz[ni][l], R, e->pw[ni][l], e->wn[ni][l], e->pw[ni][l - 1]))
+            // slabs of 128 columns: every epilogue warp then has one 32-column chunk per row tile, whose stored
+            // post-activations it fetches while the products still run
+            if (!add_rowmajor_problem(P, e->dz[ni][l], R, e->pw[ni][l], e->wn[ni][l], e->pw[ni][l - 1], 128))
                 return bail("tensor map encoding failed");
             TcProblem& p = P.p[P.count - 1];
             p.out16 = e->dz[ni][l - 1]; p.ld_out = e->pw[ni][l - 1];
@@ -1142,11 +1415,12 @@ UmmaEngine* umma_create(const UmmaSetup& s, std::string* err) {
                 if (!ealloc(e, &e->bias_slots[ni][l - 1], (size_t)e->n_slots * e->pw[ni][l - 1])) return bail("allocation failed");
                 p.colsum = e->bias_slots[ni][l - 1]; p.ld_colsum = e->pw[ni][l - 1];
             }
-            if (!make_tmap(&P.tmOut[P.count - 1], p.out16, R, e->pw[ni][l - 1], e->pw[ni][l - 1], 64, 32) ||
-                !make_tmap(&P.tmAux[P.count - 1], p.aux16, R, e->pw[ni][l - 1], e->pw[ni][l - 1], 64, 32))
+            if (!make_tmap(&P.tmOut[P.count - 1], p.out16, R, e->pw[ni][l - 1], e->pw[ni][l - 1], 32, 32, CU_TENSOR_MAP_SWIZZLE_64B) ||
+                !make_tmap(&P.tmAux[P.count - 1], p.aux16, R, e->pw[ni][l - 1], e->pw[ni][l - 1], 32, BLOCK_M, CU_TENSOR_MAP_SWIZZLE_64B))
                 return bail("tensor map encoding failed");
         }
         finish_params(P, alpha, e->error_dev);
+        plan_ws(P, e->num_sms, TC_DGRAD);
         e->upd_dgrad.push_back(P);
     }
     // ---- weight-gradient problems (all layers of both nets, heads included) ------------------
@@ -1214,40 +1488,12 @@ UmmaEngine* umma_create(const UmmaSetup& s, std::string* err) {
             if (l < e->nh[ni] - 1) e->colsum_rest.p[e->colsum_rest.count++] = q;
         }
     e->colsum_rest.splits = e->colsum.splits; e->colsum_rest.split_stride = e->colsum.split_stride; e->colsum_rest.is_bf16 = 1;
-    // ---- fused row-local step kernel -------------------------------------------------------------
-    // (off unless RSLRL_FUSED_STEP=1: on the workloads measured so far its items, which run their layers
-    // one after the other, take longer than the per-layer launches whose tiles overlap)
-    const char* fused_env = std::getenv("RSLRL_FUSED_STEP");
-    if (fused_env && fused_env[0] == '1' && R == s.Bmb && e->nh[0] <= kStepChainLayers && e->nh[1] <= kStepChainLayers && e->head_copies) {
-        StepChainSetup cs{};
-        cs.rows = R; cs.alpha = alpha; cs.error = e->error_dev; cs.num_sms = e->num_sms;
-        cs.log_std = s.param + s.logstd_off;
-        e->step_slot_rows = step_chain_colsum_rows(R);
-        bool okc = true;
-        for (int ni = 0; ni < 2 && okc; ++ni) {
-            StepChainNet& n = cs.net[ni];
-            n.nh = e->nh[ni]; n.kp = e->kp[ni]; n.is_actor = ni == 0; n.A = s.out[ni][e->nh[ni]];
-            n.x16 = e->x16[ni]; n.wht = e->wht[ni]; n.whn = e->whn[ni]; n.head_bias = e->head_bias_pad[ni];
-            n.dhead16 = ni == 0 ? e->dmu16 : e->dv16;
-            for (int l = 0; l < e->nh[ni]; ++l) {
-                n.pw[l] = e->pw[ni][l]; n.wt[l] = e->wt[ni][l]; n.wn[l] = e->wn[ni][l];
-                n.bias_pad[l] = e->bias_pad[ni][l]; n.h[l] = e->h[ni][l]; n.dz[l] = e->dz[ni][l];
-                okc = okc && ealloc(e, &e->step_slots[ni][l], (size_t)e->step_slot_rows * e->pw[ni][l]);
-                n.colsum[l] = e->step_slots[ni][l];
-            }
-        }
-        if (!okc) return bail("allocation failed");
-        std::string serr;
-        e->step = step_chain_create(cs, &serr);
-        if (!e->step && !serr.empty()) return bail("fused step kernel: tensor map encoding failed");
-    }
     if (cudaStreamSynchronize(s.stream) != cudaSuccess) return bail("stream synchronisation failed");
     return e;
 }
 
 void umma_destroy(UmmaEngine* e) {
     if (!e) return;
-    if (e->step) step_chain_destroy(e->step);
     for (void* p : e->allocs) cudaFree(p);
     delete e;
 }
@@ -1338,7 +1584,7 @@ cudaError_t umma_act_forward(UmmaEngine* e, const float* d_obs_a, const float* d
     } else {
         const std::vector<TcParams>& seq = do_actor ? e->act_fwd : e->act_fwd_critic;
         for (const TcParams& P : seq) {
-            err = launch_tc<TC_FWD>(P, e->num_sms, s.stream);
+            err = launch_ws<TC_FWD>(P, s.stream);
             if (err != cudaSuccess) return err;
         }
     }
@@ -1353,11 +1599,10 @@ void umma_gather_targets(UmmaEngine* e, GatherArgs* g, int buf) {
     g->x_c16 = buf ? e->x16_alt[1] : e->x16[1]; g->ldxc16 = e->kp[1];
 }
 
-bool umma_two_input_buffers(const UmmaEngine* e) { return e->step == nullptr; }
-
 cudaError_t umma_update_forward(UmmaEngine* e, int buf, bool actor_only) {
+    FamilyScope family_("tc_gemm_fwd", e->s.stream);
     for (const TcParams& P : actor_only ? e->fwd_actor[buf] : buf ? e->upd_fwd_alt : e->upd_fwd) {
-        cudaError_t err = launch_tc<TC_FWD>(P, e->num_sms, e->s.stream);
+        cudaError_t err = launch_ws<TC_FWD>(P, e->s.stream);
         if (err != cudaSuccess) return err;
     }
     return cudaSuccess;
@@ -1390,41 +1635,18 @@ cudaError_t umma_zero_critic_gradients(UmmaEngine* e) {
 
 cudaError_t umma_update_backward(UmmaEngine* e, bool last_bias_done, int buf, bool actor_only) {
     cudaError_t err;
-    for (const TcParams& P : actor_only ? e->dgrad_actor : e->upd_dgrad) {
-        err = launch_tc<TC_DGRAD>(P, e->num_sms, e->s.stream);
-        if (err != cudaSuccess) return err;
+    {
+        FamilyScope family_("tc_gemm_dgrad", e->s.stream);
+        for (const TcParams& P : actor_only ? e->dgrad_actor : e->upd_dgrad) {
+            err = launch_ws<TC_DGRAD>(P, e->s.stream);
+            if (err != cudaSuccess) return err;
+        }
     }
     for (const TcParams& P : buf ? e->upd_wgrad_alt : e->upd_wgrad) {
-        err = launch_tc<TC_WGRAD>(P, e->num_sms, e->s.stream);
+        err = launch_wgrad(P, e->num_sms, e->s.stream);
         if (err != cudaSuccess) return err;
     }
     return launch_colsum(last_bias_done ? e->colsum_rest : e->colsum, e->s.stream);
-}
-
-bool umma_has_step_chain(const UmmaEngine* e) { return e->step != nullptr; }
-
-cudaError_t umma_step_chain(UmmaEngine* e, const StepChainLoss& loss, int* nblocks) {
-    *nblocks = step_chain_blocks(e->step);
-    return step_chain_launch(e->step, loss, e->s.stream);
-}
-
-cudaError_t umma_update_wgrad(UmmaEngine* e) {
-    for (const TcParams& P : e->upd_wgrad) {
-        cudaError_t err = launch_tc<TC_WGRAD>(P, e->num_sms, e->s.stream);
-        if (err != cudaSuccess) return err;
-    }
-    return cudaSuccess;
-}
-
-void umma_fill_step_bias_sources(UmmaEngine* e, ReduceArgs* r) {
-    const UmmaSetup& s = e->s;
-    r->n_bias = 0;
-    for (int ni = 0; ni < 2; ++ni)
-        for (int l = 0; l < e->nh[ni]; ++l) {
-            BiasSource& b = r->bias[r->n_bias++];
-            b.p_off = (int)s.b_off[ni][l]; b.n = s.out[ni][l];
-            b.slots = e->step_slots[ni][l]; b.nslots = e->step_slot_rows; b.ld = e->pw[ni][l];
-        }
 }
 
 cudaError_t umma_read_error(UmmaEngine* e, int* host_code) {

@@ -4,7 +4,6 @@
 #include "../../include/rslrl_b200.h"
 #include "common.cuh"
 #include "kernels.h"
-#include "step_chain.h"
 #include <string>
 
 namespace rslrl {
@@ -48,9 +47,8 @@ cudaError_t umma_act_forward(UmmaEngine* e, const float* d_obs_a, const float* d
                              const void** ha, int* ldha, const void** hc, int* ldhc);
 // Point the gather at one of the engine's two minibatch input buffers (buf = 0 or 1); the forward
 // and backward launches take the same index.  With two buffers the gather of the next minibatch
-// can run while the current one is worked on (not with the fused step kernel, which has one).
+// can run while the current one is worked on.
 void umma_gather_targets(UmmaEngine* e, GatherArgs* g, int buf);
-bool umma_two_input_buffers(const UmmaEngine* e);
 // actor_only (distillation): the critic's launches are left out; umma_zero_critic_gradients, once before the
 // first such step, zeroes what its data-gradient launches would have written, so that the weight-gradient
 // launch (which still covers both nets) yields a zero critic gradient.
@@ -62,14 +60,6 @@ void umma_head_loss_targets(UmmaEngine* e, HeadLossArgs* a);
 // and heads, from the dZ / d_head buffers the head/loss kernel filled.  last_bias_done: the
 // head/loss kernel already produced the bias-gradient partials of the last hidden layers.
 cudaError_t umma_update_backward(UmmaEngine* e, bool last_bias_done, int buf, bool actor_only);
-// The fused row-local step kernel (forward, heads, loss, data gradients in one launch) exists when
-// the minibatch has no mirrored rows and the widths fit.  umma_step_chain runs it (nblocks: rows of
-// loss.block_partials it writes), umma_update_wgrad the weight-gradient partials after it, and
-// umma_fill_step_bias_sources points the reduction at its bias-gradient partials (all hidden layers).
-bool umma_has_step_chain(const UmmaEngine* e);
-cudaError_t umma_step_chain(UmmaEngine* e, const StepChainLoss& loss, int* nblocks);
-cudaError_t umma_update_wgrad(UmmaEngine* e);
-void umma_fill_step_bias_sources(UmmaEngine* e, ReduceArgs* r);
 // Synchronises the stream and returns the device error code (0 = none; otherwise the role
 // whose bounded wait expired).
 cudaError_t umma_read_error(UmmaEngine* e, int* host_code);

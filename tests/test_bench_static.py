@@ -27,7 +27,6 @@ def undefined_names(path):
                    if isinstance(n, ast.Name) and isinstance(n.ctx, ast.Load) and n.id not in defined})
 
 
-@pytest.mark.parametrize("rel", ["bench.py", "__graft_entry__.py", "paper_2509_10771_b200/bandwidth_report.py",
-                                 "paper_2509_10771_b200/binding.py"])
+@pytest.mark.parametrize("rel", ["bench.py", "__graft_entry__.py", "paper_2509_10771_b200/binding.py"])
 def test_every_loaded_name_is_defined(rel):
     assert undefined_names(os.path.join(ROOT, rel)) == []

@@ -191,23 +191,6 @@ def test_first_update_step_matches_oracle_bf16(case):
     _first_step(case, BF16, from_oracle_storage=True)
 
 
-@pytest.mark.parametrize("case", ["flat", "rough", "humanoid"])
-def test_fused_step_kernel_matches_oracle_bf16(case, monkeypatch):
-    """RSLRL_FUSED_STEP=1 selects the kernel that runs forward, heads, loss and data gradients of a row
-    tile in one launch: same first step as the per-layer kernels, within the same tolerances."""
-    from paper_2509_10771_b200 import binding
-    monkeypatch.setenv("RSLRL_FUSED_STEP", "1")
-    binding.profile_enable(True)
-    binding.profile_report()
-    try:
-        _first_step(case, BF16, from_oracle_storage=True)
-        families = binding.profile_report()
-    finally:
-        binding.profile_enable(False)
-    assert families.get("step_chain", {}).get("launches", 0) == 1, families.keys()
-    assert "head_loss" not in families and "tc_gemm_dgrad" not in families
-
-
 @pytest.mark.parametrize("case,precision", [("tiny", FP32), ("flat", FP32), ("rough_sym", FP32), ("rough", BF16)])
 def test_full_update_tracks_oracle(case, precision):
     """All E*M steps: the trajectories stay together (looser: Adam amplifies rounding)."""
