@@ -48,14 +48,17 @@ typedef enum {
     RSLRL_ERR_UNSUPPORTED = 5,   /* a size beyond a documented limit                          */
     RSLRL_ERR_CUDA = 6,          /* a CUDA runtime call failed; see rslrl_last_error          */
     RSLRL_ERR_NONFINITE = 7,     /* a loss or gradient norm was not finite                    */
-    RSLRL_ERR_TIMEOUT = 8        /* a bounded wait inside a kernel ran out; results invalid   */
+    RSLRL_ERR_TIMEOUT = 8        /* a bounded wait inside a kernel ran out; results since the
+                                    last synchronising call are invalid; reported once         */
 } rslrl_status;
 
 /* Arithmetic of the hidden-layer matrix products.  Accumulation, bias, ELU, losses, master
  * weights, gradients and Adam are FP32 in every mode. */
 typedef enum {
     RSLRL_FP32 = 0,              /* FP32 operands on the FP32 pipes                           */
-    RSLRL_TF32 = 1,              /* TF32 operands on the tensor cores                         */
+    RSLRL_TF32 = 1,              /* FP32 storage; forward and data-gradient products on the
+                                    tensor cores with TF32 operands, weight gradients on the
+                                    FP32 pipes                                                 */
     RSLRL_BF16 = 2               /* BF16 operands on the tensor cores                         */
 } rslrl_precision;
 
@@ -266,7 +269,12 @@ rslrl_status rslrl_minibatch_indices(uint64_t seed, uint32_t iteration, uint32_t
  *   - N may not exceed RSLRL_GAE_STATIC_MAX_ENVS: a larger N returns RSLRL_ERR_UNSUPPORTED and
  *     rslrl_last_error(NULL) says so; nothing is launched.
  *   - The first call on a device looks up the array's device address (once per device, with
- *     that device current); make that first call before starting any stream capture.
+ *     that device current); the CUDA runtime may load the part of the library that holds the
+ *     array at that moment, which is the one point where this entry point can touch device
+ *     memory management.  Make that first call during start-up, before any stream capture and
+ *     before memory gets tight: a call with T = 0 or N = 0 does the lookup and nothing else.
+ *     While the library's per-kernel profiling is switched on (rslrl_profile_enable) a call also
+ *     creates CUDA events; leave profiling off where that matters.
  *   - Every call on a device uses the same array, which keeps what the previous call left in
  *     it.  The call needs nothing in it to start at zero, but two calls that overlap on the GPU
  *     (different streams, no ordering between them) race on it: order them. */

@@ -4,6 +4,7 @@
 #include "common.cuh"
 #include "kernels.h"
 #include "umma.h"
+#include "tf32.h"
 
 #include <algorithm>
 #include <atomic>
@@ -89,8 +90,9 @@ struct rslrl_ctx {
     // rslrl_record_step_host needs one transfer; the event marks the last transfer out of the host copy
     uint8_t *pack_host = nullptr, *pack_dev = nullptr;
     cudaEvent_t pack_sent = nullptr; bool pack_in_flight = false;
-    // tensor-core engine (BF16 mode)
+    // tensor-core engines (BF16 mode; TF32 mode: hidden-layer products on the FP32 mode's buffers)
     UmmaEngine* umma = nullptr;
+    Tf32Engine* tf32 = nullptr;
     // host state
     int step = 0; bool act_pending = false; bool gae_done = false;
     uint32_t global_step = 0, iteration = 0;
@@ -295,7 +297,10 @@ rslrl_status backward_fp32(rslrl_ctx* c) {
         }
         if (wg.count) CU(c, launch_sgemm(wg, true, false, EPI_PLAIN, c->stream));
         if (cs.count) CU(c, launch_colsum(cs, c->stream));
-        if (dg.count) CU(c, launch_sgemm(dg, false, true, EPI_DELU, c->stream));
+        if (dg.count) {
+            if (c->tf32) CU(c, tf32_update_dgrad(c->tf32, back));
+            else CU(c, launch_sgemm(dg, false, true, EPI_DELU, c->stream));
+        }
     }
     return RSLRL_OK;
 }
@@ -305,9 +310,10 @@ bool aligned4(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 3u) == 0
 
 // After a host synchronisation: did a bounded wait inside a tensor-core kernel expire?
 rslrl_status check_engine(rslrl_ctx* c) {
-    if (!c->umma) return RSLRL_OK;
+    if (!c->umma && !c->tf32) return RSLRL_OK;
     int code = 0;
-    CU(c, umma_read_error(c->umma, &code));
+    if (c->umma) CU(c, umma_read_error(c->umma, &code));
+    else CU(c, tf32_read_error(c->tf32, &code));
     if (code != 0) return fail(c, RSLRL_ERR_TIMEOUT, "a bounded wait in a tensor-core kernel expired (role %d)", code);
     return RSLRL_OK;
 }
@@ -342,6 +348,7 @@ rslrl_status rslrl_destroy(rslrl_ctx* c) {
         if (c->ev_consumed[b]) cudaEventDestroy(c->ev_consumed[b]);
     }
     if (c->umma) umma_destroy(c->umma);
+    if (c->tf32) tf32_destroy(c->tf32);
     for (void* p : c->allocs) cudaFree(p);
     if (c->stats_host) cudaFreeHost(c->stats_host);
     if (c->pack_host) cudaFreeHost(c->pack_host);
@@ -360,7 +367,6 @@ rslrl_status rslrl_create(const rslrl_model_cfg* m, const rslrl_ppo_cfg* p, void
     const long long B = (long long)m->num_envs * m->num_steps;
     if (B >= (1ll << 30)) return fail(nullptr, RSLRL_ERR_UNSUPPORTED, "T*N must be below 2^30");
     if (B % p->minibatches) return fail(nullptr, RSLRL_ERR_SHAPE, "T*N = %lld is not divisible by %d minibatches", B, p->minibatches);
-    if (m->precision == RSLRL_TF32) return fail(nullptr, RSLRL_ERR_UNSUPPORTED, "the TF32 mode is not available in this build; use RSLRL_BF16 or RSLRL_FP32");
     if (p->sym_enable && (!p->h_sym_obs_perm || !p->h_sym_obs_sign || !p->h_sym_act_perm || !p->h_sym_act_sign ||
                           (!m->shared_obs && (!p->h_sym_cobs_perm || !p->h_sym_cobs_sign))))
         return fail(nullptr, RSLRL_ERR_INVALID_ARG, "symmetry enabled but a mirror table is null");
@@ -407,7 +413,7 @@ rslrl_status rslrl_create(const rslrl_model_cfg* m, const rslrl_ppo_cfg* p, void
     // update workspace
     c->Bmb = (int)(B / p->minibatches);
     c->R = p->sym_enable ? 2 * c->Bmb : c->Bmb;
-    if (c->prec == RSLRL_FP32) {
+    if (c->prec != RSLRL_BF16) {
         c->splits = std::max(1, std::min(32, c->R / 512));
     } else {
         // one wave of weight-gradient work items over the SMs; every problem has its own number of splits
@@ -430,7 +436,7 @@ rslrl_status rslrl_create(const rslrl_model_cfg* m, const rslrl_ppo_cfg* p, void
     if (cudaMallocHost((void**)&c->stats_host, (size_t)c->max_stat_rows * 8 * sizeof(float)) != cudaSuccess) {
         c->err = "cudaMallocHost failed"; return bail(RSLRL_ERR_CUDA);
     }
-    if (c->prec == RSLRL_FP32) {
+    if (c->prec != RSLRL_BF16) {
         const Net* nets[2] = {&c->actor, &c->critic};
         A_(c->x_a, (size_t)c->R * sa);
         if (!m->shared_obs) A_(c->x_c, (size_t)c->R * sc);
@@ -441,6 +447,26 @@ rslrl_status rslrl_create(const rslrl_model_cfg* m, const rslrl_ppo_cfg* p, void
                 A_(q, (size_t)c->R * nets[ni]->hid_ld[l]); c->up_h[ni][l] = q;
                 A_(q, (size_t)c->R * nets[ni]->hid_ld[l]); c->up_dz[ni][l] = q;
             }
+        if (c->prec == RSLRL_TF32) {
+            Tf32Setup ts{};
+            ts.N = N; ts.R = c->R; ts.T = T; ts.stream = c->stream; ts.elu_alpha = m->elu_alpha; ts.param = c->param;
+            for (int ni = 0; ni < 2; ++ni) {
+                ts.nl[ni] = nets[ni]->nl; ts.in_dim[ni] = nets[ni]->in_dim; ts.in_ld[ni] = nets[ni]->in_ld;
+                for (int l = 0; l < nets[ni]->nl; ++l) {
+                    ts.in[ni][l] = nets[ni]->L[l].in; ts.out[ni][l] = nets[ni]->L[l].out; ts.out_p[ni][l] = nets[ni]->L[l].out_p;
+                    ts.hid_ld[ni][l] = nets[ni]->hid_ld[l];
+                    ts.w_off[ni][l] = nets[ni]->L[l].w_off; ts.b_off[ni][l] = nets[ni]->L[l].b_off;
+                    ts.act_h[ni][l] = (float*)c->act_h[ni][l]; ts.up_h[ni][l] = (float*)c->up_h[ni][l]; ts.up_dz[ni][l] = (float*)c->up_dz[ni][l];
+                }
+            }
+            ts.obs_storage[0] = c->st.obs_actor; ts.obs_stride[0] = sa;
+            ts.obs_storage[1] = c->st.obs_critic; ts.obs_stride[1] = sc;
+            ts.last_obs_c = c->last_obs_c;
+            ts.x[0] = c->x_a; ts.x[1] = m->shared_obs ? c->x_a : c->x_c;
+            std::string terr;
+            c->tf32 = tf32_create(ts, &terr);
+            if (!c->tf32) { c->err = "tensor-core engine: " + terr; return bail(RSLRL_ERR_UNSUPPORTED); }
+        }
     } else {
         UmmaSetup us{}; fill_setup(c, us);
         std::string uerr;
@@ -508,6 +534,7 @@ rslrl_status rslrl_set_params(rslrl_ctx* c, const float* h, size_t n) {
     CU(c, cudaMemcpyAsync(c->param, dev.data(), dev.size() * sizeof(float), cudaMemcpyHostToDevice, c->stream));
     CU(c, cudaStreamSynchronize(c->stream));
     if (c->umma) CU(c, umma_refresh_weights(c->umma));
+    if (c->tf32) CU(c, tf32_refresh_weights(c->tf32));
     return RSLRL_OK;
 }
 
@@ -575,10 +602,11 @@ rslrl_status rslrl_act(rslrl_ctx* c, const float* d_actor_obs, const float* d_cr
     out.sigma = c->st.sigma + (size_t)t * as; out.logp = c->st.logp + (size_t)t * N;
     out.values = c->st.values + (size_t)t * N; out.actions_out = d_actions_out; out.act_stride = as;
     const HeadParams hp = head_params(c);
-    if (c->prec == RSLRL_FP32) {
+    if (c->prec != RSLRL_BF16) {
         CU(c, launch_pad_rows(d_actor_obs, c->mc.actor_obs_dim, oa, sa, nullptr, 0, N, c->stream));
         if (!c->mc.shared_obs) CU(c, launch_pad_rows(d_critic_obs, c->mc.critic_obs_dim, oc, sc, nullptr, 0, N, c->stream));
-        TRY(forward_hidden_fp32(c, true, true, oa, oc, N, c->act_h));
+        if (c->tf32) CU(c, tf32_act_forward(c->tf32, t, true));
+        else TRY(forward_hidden_fp32(c, true, true, oa, oc, N, c->act_h));
         CU(c, launch_act_head(c->act_h[0][c->actor.nl - 2], c->actor.hid_ld[c->actor.nl - 2],
                               c->act_h[1][c->critic.nl - 2], c->critic.hid_ld[c->critic.nl - 2], false, hp, out, N,
                               c->pc.seed, c->global_step, c->stream));
@@ -613,9 +641,10 @@ rslrl_status rslrl_gae(rslrl_ctx* c, const float* d_last_critic_obs) {
     if (c->step != c->st.T || c->act_pending) return fail(c, RSLRL_ERR_STATE, "rslrl_gae needs exactly T = %d recorded steps (have %d)", c->st.T, c->step);
     const int N = c->st.N, T = c->st.T;
     const HeadParams hp = head_params(c);
-    if (c->prec == RSLRL_FP32) {
+    if (c->prec != RSLRL_BF16) {
         CU(c, launch_pad_rows(d_last_critic_obs, c->mc.critic_obs_dim, c->last_obs_c, c->st.obs_c_stride, nullptr, 0, N, c->stream));
-        TRY(forward_hidden_fp32(c, false, true, nullptr, c->last_obs_c, N, c->act_h));
+        if (c->tf32) CU(c, tf32_act_forward(c->tf32, 0, false));
+        else TRY(forward_hidden_fp32(c, false, true, nullptr, c->last_obs_c, N, c->act_h));
         CU(c, launch_value_head(c->act_h[1][c->critic.nl - 2], c->critic.hid_ld[c->critic.nl - 2], false, hp, c->last_values, N, c->stream));
     } else {
         const void *ha, *hc; int ldha, ldhc;
@@ -702,8 +731,9 @@ static rslrl_status update_impl(rslrl_ctx* c, int32_t max_steps, rslrl_update_st
             }
             // ---- forward, heads, loss, backward ----------------------------------------------
             HeadLossArgs hl{};
-            if (c->prec == RSLRL_FP32) {
-                TRY(forward_hidden_fp32(c, true, true, c->x_a, c->mc.shared_obs ? c->x_a : c->x_c, c->R, c->up_h));
+            if (c->prec != RSLRL_BF16) {
+                if (c->tf32) CU(c, tf32_update_forward(c->tf32));
+                else TRY(forward_hidden_fp32(c, true, true, c->x_a, c->mc.shared_obs ? c->x_a : c->x_c, c->R, c->up_h));
                 hl.Ha = c->up_h[0][c->actor.nl - 2]; hl.ldha = c->actor.hid_ld[c->actor.nl - 2];
                 hl.Hc = c->up_h[1][c->critic.nl - 2]; hl.ldhc = c->critic.hid_ld[c->critic.nl - 2];
                 hl.bf16_act = 0;
@@ -725,7 +755,7 @@ static rslrl_status update_impl(rslrl_ctx* c, int32_t max_steps, rslrl_update_st
             hl.block_partials = c->block_partials; hl.mu_out = nullptr; hl.v_out = nullptr;
             CU(c, launch_head_loss(hl, c->stream));
             // ---- backward ---------------------------------------------------------------
-            if (c->prec == RSLRL_FP32) TRY(backward_fp32(c));
+            if (c->prec != RSLRL_BF16) TRY(backward_fp32(c));
             else CU(c, umma_update_backward(c->umma, hl.colsum_written != 0, buf, distill));
             if (overlap) CU(c, cudaEventRecord(c->ev_consumed[buf], c->stream));   // this input set may be refilled
             // ---- reduce, clip, adaptive lr, Adam ------------------------------------------
@@ -749,6 +779,7 @@ static rslrl_status update_impl(rslrl_ctx* c, int32_t max_steps, rslrl_update_st
             ad.stats_row = c->stats_dev + (size_t)done_steps * 8;
             if (c->umma) umma_fill_cvt(c->umma, &ad);
             CU(c, launch_adam(ad, c->stream));
+            if (c->tf32) CU(c, tf32_refresh_weights(c->tf32));
             c->parity ^= 1;
         }
     }

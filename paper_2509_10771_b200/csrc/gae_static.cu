@@ -58,16 +58,19 @@ extern "C" rslrl_status rslrl_gae_scan_static(const float* d_rewards, const floa
                                 "use rslrl_gae_scan with caller-provided scratch");
         return RSLRL_ERR_UNSUPPORTED;
     }
-    if (T == 0 || N == 0) return RSLRL_OK;
-    if (!d_rewards || !d_values || !d_dones || !d_timeouts || !d_last_values || !d_returns || !d_advantages)
-        return RSLRL_ERR_INVALID_ARG;
-    if ((long long)T * N >= (1ll << 31)) return RSLRL_ERR_UNSUPPORTED;
-    if (reinterpret_cast<uintptr_t>(d_advantages) & 15u) return RSLRL_ERR_ALIGNMENT;
+    // The address lookup comes before the empty-size return on purpose: an empty call (T = 0 or N = 0) at
+    // start-up is the way to get the one-time work of a device out of the way (the lookup, and with lazy module
+    // loading the loading of the module that holds the array), so that no later call has any left to do.
     float* scratch = nullptr;
     if (scratch_for_current_device(&scratch) != cudaSuccess) {
         rslrl::set_global_error("rslrl_gae_scan_static: cudaGetSymbolAddress failed");
         return RSLRL_ERR_CUDA;
     }
+    if (T == 0 || N == 0) return RSLRL_OK;
+    if (!d_rewards || !d_values || !d_dones || !d_timeouts || !d_last_values || !d_returns || !d_advantages)
+        return RSLRL_ERR_INVALID_ARG;
+    if ((long long)T * N >= (1ll << 31)) return RSLRL_ERR_UNSUPPORTED;
+    if (reinterpret_cast<uintptr_t>(d_advantages) & 15u) return RSLRL_ERR_ALIGNMENT;
     // Nothing in the array has to start at zero: the scan writes the triple of every block
     // before the normalisation of the same call reads it, and no other slot is read.
     const cudaError_t e = rslrl::launch_gae(d_rewards, d_values, d_dones, d_timeouts, d_last_values, d_returns,

@@ -1,0 +1,45 @@
+// Tensor-core engine of the RSLRL_TF32 mode: the hidden-layer products of act, forward and data
+// gradient as tcgen05 kind::tf32 GEMMs on the FP32 buffers of the FP32 mode (operands are read as
+// FP32 and used with TF32 precision by the tensor cores; accumulation, bias, ELU and everything
+// else stay FP32).  Weight gradients, heads, loss and optimiser are the FP32 mode's kernels.
+#pragma once
+#include "../../include/rslrl_b200.h"
+#include "common.cuh"
+#include "kernels.h"
+#include <string>
+
+namespace rslrl {
+
+struct Tf32Setup {
+    int N, R, T;                            // rollout rows per act call, minibatch rows incl. mirrored, rollout steps
+    cudaStream_t stream;
+    float elu_alpha;
+    const float* param;                     // FP32 master parameters (padded device layout)
+    int nl[2], in_dim[2], in_ld[2];         // layers per net (head included), observation widths and row strides
+    int in[2][kMaxLayers], out[2][kMaxLayers], out_p[2][kMaxLayers], hid_ld[2][kMaxLayers];
+    size_t w_off[2][kMaxLayers], b_off[2][kMaxLayers];
+    const float* obs_storage[2]; int obs_stride[2];   // rollout observations [T * N][stride] (act reads step t in place)
+    const float* last_obs_c;                          // [N][obs_stride[1]]: the observation after the last step
+    const float* x[2];                                // minibatch inputs [R][in_ld]
+    float* act_h[2][kMaxLayers];                      // post-activations of act [N][hid_ld]
+    float* up_h[2][kMaxLayers];                       // post-activations of the update [R][hid_ld]
+    float* up_dz[2][kMaxLayers];                      // dL/dz of the update [R][hid_ld]
+};
+
+struct Tf32Engine;
+
+Tf32Engine* tf32_create(const Tf32Setup& s, std::string* err);
+void tf32_destroy(Tf32Engine* e);
+// Transposed copies of the hidden-layer weights ([out][in], the contraction contiguous): the forward operand.
+// After rslrl_set_params and after every optimiser step.
+cudaError_t tf32_refresh_weights(Tf32Engine* e);
+// Hidden layers of both nets on the rows of rollout step t (do_actor), or of the critic alone on last_obs_c.
+cudaError_t tf32_act_forward(Tf32Engine* e, int t, bool do_actor);
+// Hidden layers of both nets on the minibatch rows.
+cudaError_t tf32_update_forward(Tf32Engine* e);
+// dL/dz of hidden layer (top - back - 1) of every net that has one, from dL/dz of the layer above.
+cudaError_t tf32_update_dgrad(Tf32Engine* e, int back);
+// Synchronises the stream and returns the device error code (0 = none); a non-zero code is cleared once read.
+cudaError_t tf32_read_error(Tf32Engine* e, int* host_code);
+
+}  // namespace rslrl

@@ -1652,7 +1652,10 @@ cudaError_t umma_update_backward(UmmaEngine* e, bool last_bias_done, int buf, bo
 cudaError_t umma_read_error(UmmaEngine* e, int* host_code) {
     cudaError_t err = cudaMemcpyAsync(host_code, e->error_dev, sizeof(int), cudaMemcpyDeviceToHost, e->s.stream);
     if (err != cudaSuccess) return err;
-    return cudaStreamSynchronize(e->s.stream);
+    err = cudaStreamSynchronize(e->s.stream);
+    if (err != cudaSuccess || *host_code == 0) return err;
+    // reported once: the word is cleared so that later calls are judged on their own
+    return cudaMemsetAsync(e->error_dev, 0, sizeof(int), e->s.stream);
 }
 
 }  // namespace rslrl

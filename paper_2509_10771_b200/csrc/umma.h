@@ -61,7 +61,7 @@ void umma_head_loss_targets(UmmaEngine* e, HeadLossArgs* a);
 // head/loss kernel already produced the bias-gradient partials of the last hidden layers.
 cudaError_t umma_update_backward(UmmaEngine* e, bool last_bias_done, int buf, bool actor_only);
 // Synchronises the stream and returns the device error code (0 = none; otherwise the role
-// whose bounded wait expired).
+// whose bounded wait expired); a non-zero code is cleared once it has been read.
 cudaError_t umma_read_error(UmmaEngine* e, int* host_code);
 
 }  // namespace rslrl

@@ -10,12 +10,15 @@ from oracle import ppo_oracle as O
 from paper_2509_10771_b200 import workloads as WL
 
 
-def assert_close(got, want, tol: float, name: str = "", max_outlier_frac: float = 0.0, outlier_abs: float = 0.0):
+def assert_close(got, want, tol: float, name: str = "", max_outlier_frac: float = 0.0, outlier_abs: float = 0.0,
+                 outlier_factor: float = 0.0):
     """|got - want| <= tol * |want| + tol * rms(want), element by element.
 
     ``max_outlier_frac`` > 0 allows that fraction of elements to miss the bound as long as they
     stay within ``outlier_abs`` (used only where an element is a discontinuous function of the
-    inputs, e.g. Adam's first step at a gradient entry that is zero to rounding)."""
+    inputs, e.g. Adam's first step at a gradient entry that is zero to rounding).  With ``outlier_factor``
+    the allowed outliers must instead stay within that multiple of their own bound (used at sizes of tens of
+    millions of elements, where the tail of the BF16 rounding error crosses any fixed multiple of its spread)."""
     got = np.asarray(got, dtype=np.float64)
     want = np.asarray(want, dtype=np.float64)
     assert got.shape == want.shape, (name, got.shape, want.shape)
@@ -31,7 +34,10 @@ def assert_close(got, want, tol: float, name: str = "", max_outlier_frac: float 
         worst = int(np.argmax(err - bound))
         msg = (f"{name}: {bad.sum()} / {bad.size} elements outside tol={tol:g} (rms {rms:.3g}); worst flat index "
                f"{worst}: got {got.ravel()[worst]!r} want {want.ravel()[worst]!r}")
-        assert frac <= max_outlier_frac and err[bad].max() <= outlier_abs, msg
+        if outlier_factor > 0.0:
+            assert frac <= max_outlier_frac and np.all(err[bad] <= outlier_factor * bound[bad]), msg
+        else:
+            assert frac <= max_outlier_frac and err[bad].max() <= outlier_abs, msg
 
 
 def rel_l2(got, want) -> float:
@@ -83,12 +89,13 @@ def gpu_rollout(ctx, w: WL.Workload, inputs: Dict[str, np.ndarray]):
     torch.cuda.synchronize()
 
 
-def read_storage(ctx, w: WL.Workload) -> Dict[str, np.ndarray]:
+def read_storage(ctx, w: WL.Workload, with_obs: bool = True) -> Dict[str, np.ndarray]:
     s = ctx.storage_view()
     T, N, A = w.num_steps, w.num_envs, w.num_actions
     out = {}
-    out["obs_actor"] = dev_to_numpy(s.obs_actor, (T, N, s.obs_a_stride))[..., :w.actor_obs_dim]
-    out["obs_critic"] = dev_to_numpy(s.obs_critic, (T, N, s.obs_c_stride))[..., :w.critic_obs_dim]
+    if with_obs:
+        out["obs_actor"] = dev_to_numpy(s.obs_actor, (T, N, s.obs_a_stride))[..., :w.actor_obs_dim]
+        out["obs_critic"] = dev_to_numpy(s.obs_critic, (T, N, s.obs_c_stride))[..., :w.critic_obs_dim]
     out["actions"] = dev_to_numpy(s.actions, (T, N, s.act_stride))[..., :A]
     out["mu"] = dev_to_numpy(s.mu, (T, N, s.act_stride))[..., :A]
     out["sigma"] = dev_to_numpy(s.sigma, (T, s.act_stride))[..., :A]

@@ -4,6 +4,7 @@ seeded synthetic inputs.
 Tolerances (|x - y| <= tol |y| + tol rms(y), element by element):
   FP32 mode  actions / mu / log-probs / values 1e-5; returns / advantages 1e-5;
              losses, gradient and parameters after one optimiser step 1e-4.
+  TF32 mode  5e-3 for the act outputs and for losses / parameters after one step.
   BF16 mode  2e-2 for the act outputs, 1e-2 for losses / parameters after one step.
 Integer work (shuffle indices, stored flags) is compared bit for bit.
 """
@@ -31,6 +32,8 @@ CASES = {
     "flat_full": WL.FLAT,
     "rough_full": WL.ROUGH,
     "humanoid_full": WL.HUMANOID,
+    # 65,536 envs x 32 steps, minibatches of 131,072 rows doubled by the mirror to 262,144, BF16 operands
+    "rough_sym_full": WL.ROUGH_SYM,
 }
 
 
@@ -86,22 +89,43 @@ def test_rollout_and_gae_match_oracle_bf16(case):
     ctx.destroy()
 
 
-@pytest.mark.parametrize("case", ["flat_full", "rough_full", "humanoid_full"])
-def test_full_size_workloads_bf16(case):
-    """The flat, rough (the benchmarked one) and humanoid workloads at full size, BF16: every stored rollout
-    output and the first minibatch step against the oracle (which needs some seconds at these sizes)."""
+@pytest.mark.parametrize("case", ["tiny", "flat", "rough", "humanoid"])
+def test_rollout_and_gae_match_oracle_tf32(case):
+    """TF32 operands in the hidden-layer products (FP32 storage, accumulation and heads): 5e-3."""
     w = CASES[case]
     theta, inputs = WL.make_params(w), WL.make_rollout_inputs(w)
-    ctx = make_ctx(w, BF16)
+    ctx = make_ctx(w, TF32)
     ctx.set_params(theta)
     gpu_rollout(ctx, w, inputs)
     got = read_storage(ctx, w)
     want = oracle_rollout(w, theta, inputs)
     for k in ("actions", "mu", "values", "returns", "advantages"):
-        assert_close(got[k], want[k], 2e-2, f"{case}.{k}")
+        assert_close(got[k], want[k], 5e-3, f"{case}.{k}")
     assert_close(got["logp"], want["logp"], 1e-5, f"{case}.logp")
+    assert_close(got["sigma"], want["sigma"], 1e-6, f"{case}.sigma")
+    assert np.array_equal(got["obs_actor"], inputs["obs_actor"][:w.num_steps])
+    # the tensor cores did see TF32 operands: the result is not the FP32 mode's
+    ctx32 = make_ctx(w, FP32)
+    ctx32.set_params(theta)
+    gpu_rollout(ctx32, w, inputs)
+    assert np.abs(read_storage(ctx32, w)["mu"] - got["mu"]).max() > 0.0
+    ctx32.destroy()
     ctx.destroy()
-    _first_step(case, BF16, from_oracle_storage=True)
+
+
+@pytest.mark.parametrize("case", ["flat_full", "rough_full", "humanoid_full"])
+def test_full_size_workloads_bf16(case):
+    """The flat, rough (the benchmarked one) and humanoid workloads at full size, BF16: every stored rollout
+    output and the first minibatch step against the oracle (which needs some seconds at these sizes)."""
+    _first_step(case, BF16, from_oracle_storage=True, check_rollout=True)
+
+
+def test_symmetry_workload_at_full_size_bf16():
+    """The massive-parallel symmetry workload as stated: 65,536 environments x 32 steps, 16 minibatches of
+    131,072 rows doubled by the mirror, BF16 operands.  Every stored rollout output (2,097,152 transitions), the
+    advantages and returns, and the first minibatch step (losses, symmetry loss, gradient block by block and
+    element by element, parameters) against the oracle, which needs a few minutes of host time at this size."""
+    _first_step("rough_sym_full", BF16, from_oracle_storage=True, check_rollout=True)
 
 
 def test_noise_is_the_shared_philox_stream():
@@ -125,19 +149,30 @@ def test_noise_is_the_shared_philox_stream():
 # --------------------------------------------------------------------------------------
 # (3) update
 # --------------------------------------------------------------------------------------
-def _first_step(case, precision, from_oracle_storage):
+def _first_step(case, precision, from_oracle_storage, check_rollout=False):
     w = CASES[case]
     theta, inputs, mir = WL.make_params(w), WL.make_rollout_inputs(w), mirror_of(w)
     ctx = make_ctx(w, precision, mir)
     ctx.set_params(theta)
     want_st = oracle_rollout(w, theta, inputs)
     gpu_rollout(ctx, w, inputs)
+    if check_rollout:
+        got = read_storage(ctx, w, with_obs=False)
+        # beyond ten million elements the tail of the BF16 rounding error (a sum of many independent roundings,
+        # about a quarter of the bound in spread) crosses the bound for a few elements per ten million: one per
+        # million may, by at most half the bound
+        many = got["mu"].size > 10_000_000
+        for k in ("actions", "mu", "values", "returns", "advantages"):
+            assert_close(got[k], want_st[k], 2e-2, f"{case}.{k}", max_outlier_frac=1e-6 if many else 0.0,
+                         outlier_factor=1.5 if many else 0.0)
+        assert_close(got["logp"], want_st["logp"], 1e-5, f"{case}.logp")
+        del got
     if from_oracle_storage:
         write_storage(ctx, w, want_st)
     stats = ctx.ppo_update(max_steps=1)
     state = O.OptimState(theta, w.lr)
     ref = O.ppo_update(state, dims_of(w), want_st, w, seed=w.seed, iteration=0, sym=mir, max_steps=1)[0]
-    tol = 1e-4 if precision == FP32 else 1e-2
+    tol = {FP32: 1e-4, TF32: 5e-3, BF16: 1e-2}[precision]
     if case.endswith("_full"):
         # the surrogate is a mean of -A r over the minibatch with A normalised (mean 0, |A| ~ 1) and r ~ 1:
         # over 24,576 rows it cancels to ~1e-4, so the bound is relative to the size of the terms, mean |A|
@@ -147,30 +182,49 @@ def _first_step(case, precision, from_oracle_storage):
         assert_close(stats["first_surrogate"], ref["surrogate"], tol, "surrogate")
     assert_close(stats["first_value_loss"], ref["value_loss"], tol, "value_loss")
     assert_close(stats["entropy"], ref["entropy"], tol, "entropy")
-    assert abs(stats["first_kl"] - ref["kl"]) < (1e-6 if precision == FP32 else 1e-4)
+    assert abs(stats["first_kl"] - ref["kl"]) < (1e-6 if precision == FP32 else 1e-4)   # the exact value is 0
     assert_close(stats["first_grad_norm"], ref["grad_norm"], tol, "grad_norm")
     assert_close(stats["lr"], ref["lr"], 1e-6, "lr")
     if w.sym_enable:
         assert_close(stats["first_sym_loss"], ref["sym_loss"], tol, "sym_loss")
     g = ctx.get_grads()
+    blocks = [(name, off, int(np.prod(shape))) for name, off, shape in WL.param_layout(w)]
     if precision == FP32:
         assert_close(g, ref["grad"], tol, "grad")
+    elif precision == TF32:
+        # forward and data gradient saw TF32 operands (11 significant bits), the weight gradients FP32 ones
+        for name, off, n in blocks:
+            assert_close(g[off:off + n], ref["grad"][off:off + n], 1e-2, f"grad {name}")
+        assert rel_l2(g, ref["grad"]) < 2e-3
     else:
-        # every parameter block on its own, so a wrong layer cannot hide behind a large one
-        for name, off, shape in WL.param_layout(w):
-            n = int(np.prod(shape))
+        # every parameter block on its own, so a wrong layer cannot hide behind a large one: element by element
+        # (a BF16-rounded operand perturbs every product of a three-layer chain: 5e-2 of |y| + rms of the block;
+        # the largest ratio seen on these workloads is 3.2e-2), and in relative L2
+        for name, off, n in blocks:
+            assert_close(g[off:off + n], ref["grad"][off:off + n], 5e-2, f"grad {name}")
             assert rel_l2(g[off:off + n], ref["grad"][off:off + n]) < 3e-2, name
         assert rel_l2(g, ref["grad"]) < 1e-2
-    # Adam's first step is lr * g / (|g| + eps): discontinuous where a gradient entry is zero to
-    # rounding.  Those entries (a small fraction) may differ by up to 2 lr.
-    frac = 2e-3 if precision == FP32 else 5e-2
-    assert_close(ctx.get_params(), state.theta, tol, "params", max_outlier_frac=frac, outlier_abs=2.05 * ref["lr"])
+    # Adam's first step is lr * g / (|g| + eps), i.e. lr * sign(g): discontinuous where a gradient entry is zero to
+    # rounding.  The parameters are therefore compared at the plain tolerance on the entries whose gradient is
+    # clearly non-zero, |g| >= thr * rms(g of the block) (about 95 % of them); the others can differ by up to
+    # 2 lr whatever the implementation, which is only asserted as a sanity bound.
+    thr = 1e-2 if precision == FP32 else 5e-2
+    sure = np.zeros(ref["grad"].shape, dtype=bool)
+    for name, off, n in blocks:
+        b = ref["grad"][off:off + n]
+        sure[off:off + n] = np.abs(b) >= thr * np.sqrt(np.mean(b * b))
+    assert sure.mean() > 0.8
+    got_p = ctx.get_params().astype(np.float64)
+    rms_p = float(np.sqrt(np.mean(state.theta ** 2)))
+    err_p = np.abs(got_p - state.theta)
+    assert np.all(err_p[sure] <= tol * (np.abs(state.theta[sure]) + rms_p)), "params"
+    assert err_p.max() <= 2.05 * ref["lr"]
     m, v = ctx.get_adam()
     if precision == FP32:
         assert_close(m, state.m, tol, "adam_m")
         assert_close(v, state.v, 2 * tol, "adam_v")
     else:
-        assert rel_l2(m, state.m) < 1e-2
+        assert rel_l2(m, state.m) < (2e-3 if precision == TF32 else 1e-2)
     c = ctx.get_counters()
     assert c.adam_step == 1 and c.iteration == 1
     ctx.destroy()
@@ -191,7 +245,12 @@ def test_first_update_step_matches_oracle_bf16(case):
     _first_step(case, BF16, from_oracle_storage=True)
 
 
-@pytest.mark.parametrize("case,precision", [("tiny", FP32), ("flat", FP32), ("rough_sym", FP32), ("rough", BF16)])
+@pytest.mark.parametrize("case", ["tiny", "flat", "rough", "humanoid", "rough_sym"])
+def test_first_update_step_matches_oracle_tf32(case):
+    _first_step(case, TF32, from_oracle_storage=True)
+
+
+@pytest.mark.parametrize("case,precision", [("tiny", FP32), ("flat", FP32), ("rough_sym", FP32), ("rough", BF16), ("rough", TF32)])
 def test_full_update_tracks_oracle(case, precision):
     """All E*M steps: the trajectories stay together (looser: Adam amplifies rounding)."""
     w = CASES[case]
@@ -203,13 +262,13 @@ def test_full_update_tracks_oracle(case, precision):
     state = O.OptimState(theta, w.lr)
     ref = O.ppo_update(state, dims_of(w), oracle_rollout(w, theta, inputs), w, seed=w.seed, iteration=0, sym=mir)
     assert stats["steps"] == len(ref) == w.epochs * w.minibatches
-    loose = 2e-3 if precision == FP32 else 5e-2
+    loose = {FP32: 2e-3, TF32: 2e-2, BF16: 5e-2}[precision]
     assert_close(stats["surrogate"], np.mean([r["surrogate"] for r in ref]), loose, "mean surrogate")
     assert_close(stats["value_loss"], np.mean([r["value_loss"] for r in ref]), loose, "mean value loss")
     assert_close(stats["kl"], np.mean([r["kl"] for r in ref]), 10 * loose, "mean kl")
     if precision == FP32:
         assert_close(stats["lr"], ref[-1]["lr"], 1e-6, "final lr")
-    assert rel_l2(ctx.get_params(), state.theta) < (2e-3 if precision == FP32 else 5e-2)
+    assert rel_l2(ctx.get_params(), state.theta) < loose
     ctx.destroy()
 
 
@@ -369,9 +428,6 @@ def test_call_order_and_argument_errors():
     with pytest.raises(binding.RslrlError) as e:
         make_ctx(WL.TINY.scaled(64, minibatches=7))
     assert e.value.status == 2
-    with pytest.raises(binding.RslrlError) as e:
-        make_ctx(WL.TINY, TF32)
-    assert e.value.status == 5
 
 
 def test_host_buffer_variants_match_device_calls():
@@ -403,3 +459,32 @@ def test_kernels_were_launched_by_this_library():
     ctx.ppo_update()
     ctx.destroy()
     assert binding.kernel_launch_count() - before > 3 * w.num_steps
+
+
+@pytest.mark.parametrize("precision", [FP32, BF16])
+def test_non_finite_step_is_skipped_and_reported(precision):
+    """A NaN among the parameters (set from the host; nothing faults on the device) makes every loss of the
+    update non-finite: each optimiser step is skipped, rslrl_ppo_update returns RSLRL_ERR_NONFINITE with
+    nonfinite = 1 in the statistics, and parameters, Adam moments and the step count are what they were."""
+    import ctypes as C
+    from paper_2509_10771_b200 import binding
+    w = CASES["flat"]
+    theta, inputs = WL.make_params(w), WL.make_rollout_inputs(w)
+    theta[3] = np.nan                                  # an entry of the actor's first weight matrix
+    ctx = make_ctx(w, precision)
+    ctx.set_params(theta)
+    gpu_rollout(ctx, w, inputs)
+    st = binding.UpdateStats()
+    rc = ctx.lib.rslrl_ppo_update(ctx.handle, C.byref(st))
+    assert rc == 7 and st.nonfinite == 1               # RSLRL_ERR_NONFINITE
+    assert "not finite" in ctx.lib.rslrl_last_error(ctx.handle).decode()
+    with pytest.raises(binding.RslrlError) as e:       # the binding turns the status into an exception
+        gpu_rollout(ctx, w, inputs)
+        ctx.ppo_update()
+    assert e.value.status == 7
+    got = ctx.get_params()
+    assert np.isnan(got[3]) and np.array_equal(np.delete(got, 3), np.delete(theta, 3))
+    m, v = ctx.get_adam()
+    assert not m.any() and not v.any()
+    assert ctx.get_counters().adam_step == 0
+    ctx.destroy()
