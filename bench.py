@@ -86,7 +86,7 @@ def hbm_family_bytes(w, storage_strides):
     gather = Bmb * (4 + obs_read + 4 * 2 * w.num_actions + 4 * 4) \
         + R * (obs_written + 4 * as_) + Bmb * (2 * 4 * as_ + 4 * 4)
     P = w.num_params()
-    return {"gather": gather, "adam": 28 * P, "gae_scan": 18 * T * N, "gae_normalize": 8 * T * N}
+    return {"gather": gather, "gather_alone": gather, "adam": 28 * P, "gae_scan": 18 * T * N, "gae_normalize": 8 * T * N}
 
 
 # DRAM bytes per launch (dram__bytes_read.sum + dram__bytes_write.sum, mean over the family's launches of one
@@ -678,6 +678,55 @@ def run_gru(args):
     gru.destroy()
 
 
+def run_streams(args):
+    """--task streams: the scan kernels at a bandwidth-shaped size through the stand-alone entry point (rslrl_gae_scan,
+    T = 32 steps x 1,048,576 environments, 872 MB of algorithmic traffic per call), one GPU.  The learn iteration's own
+    scan moves 2.6 MB and is bound by launch latency; this line is where the scan meets its memory roofline.  Its own
+    JSON line; the gather's and Adam's figures at their own sizes are in the ppo line (roofline.hbm_families)."""
+    import torch
+    from paper_2509_10771_b200 import binding, build
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device: the path has no CPU fallback")
+    torch.cuda.set_device(0)
+    build.build()
+    T, N = 32, 1 << 20
+    dev = torch.device("cuda", 0)
+    stream = torch.cuda.current_stream()
+    g = torch.Generator(device=dev); g.manual_seed(0)
+    r = torch.randn((T, N), device=dev, generator=g) * 0.5
+    v = torch.randn((T, N), device=dev, generator=g)
+    lv = torch.randn((N,), device=dev, generator=g)
+    d = (torch.rand((T, N), device=dev, generator=g) < 0.005).to(torch.uint8)
+    to = d & (torch.rand((T, N), device=dev, generator=g) < 0.5).to(torch.uint8)
+    ret = torch.empty((T, N), device=dev); adv = torch.empty((T, N), device=dev)
+    scratch = torch.empty(binding.gae_scratch_bytes(T, N), dtype=torch.uint8, device=dev)
+    peaks = read_peaks()
+    out = {}
+    for name, normalize, nbytes in (("gae_scan+gae_normalize", True, 26 * T * N), ("gae_scan", False, 18 * T * N)):
+        for _ in range(max(args.warmup, 3)):
+            binding.gae_scan(r, v, d, to, lv, ret, adv, T, N, 0.99, 0.95, normalize, True, 1e-8, scratch, stream=stream.cuda_stream)
+        evs = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(args.steps)]
+        torch.cuda.synchronize()
+        for a, b in evs:                    # 872 MB per call: far beyond the L2, no flush needed
+            a.record(stream)
+            binding.gae_scan(r, v, d, to, lv, ret, adv, T, N, 0.99, 0.95, normalize, True, 1e-8, scratch, stream=stream.cuda_stream)
+            b.record(stream)
+        torch.cuda.synchronize()
+        us = 1e3 * sum(a.elapsed_time(b) for a, b in evs) / args.steps
+        gbs = nbytes / (us * 1e-6) / 1e9
+        out[name] = {"bytes_per_call": nbytes, "us": us, "gbs": gbs, "frac": gbs / peaks["hbm_gbs"], "frac_of_nominal_7700": gbs / 7700.0}
+    both = out["gae_scan+gae_normalize"]
+    line = {
+        "metric": "GAE scan + advantage normalisation transitions/s", "value": T * N / (both["us"] * 1e-6), "unit": UNIT, "n_gpus": 1,
+        "steps": args.steps, "warmup": max(args.warmup, 3), "ms_per_step": both["us"] * 1e-3, "higher_is_better": True,
+        "dtype": "f32", "data": "synthetic",
+        "config": {"workload": "gae_scan_T32_N1048576", "task": "streams", "l2": "inputs (872 MB per call) larger than the L2"},
+        "roofline": {"bound": "hbm", "achieved": both["gbs"], "peak": peaks["hbm_gbs"], "unit": "GB/s", "frac": both["frac"],
+                     "traffic": None, "peak_source": f"copy bandwidth, {peaks['source']}", "kernels": out},
+    }
+    print(json.dumps(line), flush=True)
+
+
 def free_port():
     import socket
     with socket.socket(socket.AF_INET, socket.SOCK_STREAM) as so:
@@ -701,9 +750,10 @@ def main():
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--workload", default=WORKLOAD.name, choices=sorted(WL.WORKLOADS),
                     help="which of the five synthetic workloads to time (default: the one the metric is quoted on)")
-    ap.add_argument("--task", default="ppo", choices=["ppo", "distill", "rnd", "gru"],
+    ap.add_argument("--task", default="ppo", choices=["ppo", "distill", "rnd", "gru", "streams"],
                     help="ppo: the learn iteration the metric is quoted on (default); distill: the distillation iteration; "
-                         "rnd: random network distillation over one rollout; gru: the recurrent layer over one rollout")
+                         "rnd: random network distillation over one rollout; gru: the recurrent layer over one rollout; "
+                         "streams: the GAE scan at a bandwidth-shaped size")
     args = ap.parse_args()
     WORKLOAD = WL.WORKLOADS[args.workload]
     if args.gpus > 1 and "WORLD_SIZE" not in os.environ:
@@ -722,6 +772,9 @@ def main():
     elif args.task == "gru":
         if rank == 0:
             run_gru(args)
+    elif args.task == "streams":
+        if rank == 0:
+            run_streams(args)
     else:
         run_ours(args, rank, world, local_rank)
 

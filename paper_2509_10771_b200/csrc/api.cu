@@ -689,7 +689,7 @@ static rslrl_status update_impl(rslrl_ctx* c, int32_t max_steps, rslrl_update_st
         g.act_mb = c->act_mb[buf]; g.mu_old = c->mu_old[buf]; g.sigma_old = c->sigma_old[buf];
         g.logp_old = c->logp_old[buf]; g.v_old = c->v_old[buf]; g.ret = c->ret_mb[buf]; g.adv_mb = c->adv_mb[buf];
         g.rows = c->perm[c->perm_cur] + (size_t)e * T * N + (size_t)k * c->Bmb; g.Bmb = c->Bmb; g.sym = pc.sym_enable; g.st = c->sym;
-        CU(c, launch_gather(g, st));
+        CU(c, launch_gather(g, st, step == 0 && st == c->side));
         return RSLRL_OK;
     };
     // With a gather stream, minibatch s+1 is gathered into the other input set while minibatch s is

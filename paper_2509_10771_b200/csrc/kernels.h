@@ -137,7 +137,7 @@ struct GatherArgs {
     int Bmb; int sym;
     SymTables st;
 };
-cudaError_t launch_gather(const GatherArgs& a, cudaStream_t stream);
+cudaError_t launch_gather(const GatherArgs& a, cudaStream_t stream, bool alone = false);
 cudaError_t launch_perm_rows(uint64_t seed, uint32_t iteration, uint32_t epoch, uint32_t batch,
                              uint32_t first, int count, int* rows_out, cudaStream_t stream);
 // The shuffles of epochs 0 .. epochs-1 of one iteration in one launch: rows_out[epoch][batch].

@@ -52,7 +52,7 @@ struct TcProblem {
 // block of up to 256 output columns), keeps that slab of the weight operand in shared memory for the
 // whole launch where it fits, and walks the row tiles rank, rank + ctas, ... of the slab, so that only
 // the activations stream through the pipeline.
-constexpr int kMaxSlabs = 32;
+constexpr int kMaxSlabs = 64;
 constexpr int kMaxCtas = 160;
 struct WsSlab {
     int prob, n0;                  // problem and first output column
@@ -63,6 +63,8 @@ struct WsSlab {
 struct WsPlan {
     WsSlab slab[kMaxSlabs];
     int nslabs, grid, num_sms, mode;
+    int b_early;                   // 1: the weight operand was not written by the kernel launched just before this one, so a
+                                   // resident slab may be fetched before the wait for that kernel (during its tail)
     unsigned char cta_slab[kMaxCtas];
 };
 
@@ -325,6 +327,12 @@ __global__ void __launch_bounds__(kThreads, 1) ws_gemm_kernel(const __grid_const
     __syncthreads();
     tc_fence_after();
     const uint32_t tmem_base = *tmem_slot;
+    auto fetch_slab = [&]() {
+        mbar_expect_tx(bfull, (uint32_t)p.kblocks * b_kb_bytes);
+        for (int kb = 0; kb < p.kblocks; ++kb) tma_load_2d(sB + (uint32_t)kb * b_kb_bytes, &P.tmB[S.prob], kb * BLOCK_K, S.n0, bfull);
+    };
+    const bool slab_early = S.resident && P.ws.b_early && rank < p.m_tiles;
+    if (slab_early && warp == 0 && lane == 0) fetch_slab();      // the weights are older than the kernel waited for below
     chain_wait();
 
     if (warp == 0) {
@@ -332,10 +340,7 @@ __global__ void __launch_bounds__(kThreads, 1) ws_gemm_kernel(const __grid_const
         if (lane == 0) {
             const CUtensorMap* tmA = &P.tmA[S.prob];
             const CUtensorMap* tmB = &P.tmB[S.prob];
-            if (S.resident) {
-                mbar_expect_tx(bfull, (uint32_t)p.kblocks * b_kb_bytes);
-                for (int kb = 0; kb < p.kblocks; ++kb) tma_load_2d(sB + (uint32_t)kb * b_kb_bytes, tmB, kb * BLOCK_K, S.n0, bfull);
-            }
+            if (S.resident && !slab_early) fetch_slab();
             int stage = 0; uint32_t phase = 0;
             uint32_t issued_mask = 0, issued_parity = 0, aux_issued = 0, aux_parity = 0;
             bool ok = true;
@@ -1015,6 +1020,7 @@ TcParams only_net(const TcParams& P, int ni) {
     }
     finish_params(Q, P.alpha, P.error);
     plan_ws(Q, P.ws.num_sms, P.ws.mode);
+    Q.ws.b_early = P.ws.b_early;
     return Q;
 }
 
@@ -1257,6 +1263,9 @@ UmmaEngine* umma_create(const UmmaSetup& s, std::string* err) {
         e->nh[ni] = s.nl[ni] - 1;
         e->kp[ni] = round_up(s.in_dim[ni], 64);
         for (int l = 0; l < e->nh[ni]; ++l) e->pw[ni][l] = round_up(s.out[ni][l], 64);
+        // a launch holds both nets' column blocks of one layer (128 columns each in the data gradient)
+        for (int l = 0; l < e->nh[ni]; ++l)
+            if (2 * ((e->pw[ni][l] + 127) / 128) > kMaxSlabs) return bail("hidden layers wider than 4096 are not supported in the BF16 mode");
     }
     const bool shared = s.model.shared_obs != 0;
     for (int ni = 0; ni < 2; ++ni) {
@@ -1336,6 +1345,9 @@ UmmaEngine* umma_create(const UmmaSetup& s, std::string* err) {
             }
             finish_params(P, alpha, e->error_dev);
             plan_ws(P, e->num_sms, TC_FWD);
+            // the launch before the first layer's may be the optimiser step that rewrites the weights; the other
+            // layers follow a forward launch
+            P.ws.b_early = l > 0 ? 1 : 0;
             out.push_back(P);
         }
         return true;
@@ -1421,6 +1433,7 @@ UmmaEngine* umma_create(const UmmaSetup& s, std::string* err) {
         }
         finish_params(P, alpha, e->error_dev);
         plan_ws(P, e->num_sms, TC_DGRAD);
+        P.ws.b_early = 1;                  // data-gradient launches follow the head/loss kernel or each other
         e->upd_dgrad.push_back(P);
     }
     // ---- weight-gradient problems (all layers of both nets, heads included) ------------------

@@ -32,93 +32,132 @@ __device__ __forceinline__ void store_obs_piece(float* dst, __nv_bfloat16* dst16
     }
 }
 
-// dst row (ld_dst columns, pads zero) <- src row (ld_src columns, storage pad is zero); when perm
-// is given also the mirrored row dst_m[c] = sign[c] * src[perm[c]].
-__device__ __forceinline__ void copy_obs_row(const float* __restrict__ src, int dim, int ld_src,
-                                             float* dst, __nv_bfloat16* dst16, float* dst_m, __nv_bfloat16* dst16_m,
-                                             int ld_dst, const int* __restrict__ perm,
-                                             const float* __restrict__ sign, int lane) {
-    for (int c0 = 0; c0 < ld_dst; c0 += 128 * kObsVec) {
-        float4 v[kObsVec];
-        float4 m[kObsVec];
+// One block of up to 128 * kObsVec columns of an observation row: the pieces of the row itself and, when perm
+// is given, of its mirror m[c] = sign[c] * src[perm[c]] (storage pads are zero; columns past ld_dst are not used).
+struct ObsBlock { float4 v[kObsVec]; float4 m[kObsVec]; };
+
+__device__ __forceinline__ void load_obs_block(ObsBlock& b, const float* __restrict__ src, int dim, int ld_src, int ld_dst, int c0,
+                                               const int* __restrict__ perm, const float* __restrict__ sign, int lane) {
 #pragma unroll
-        for (int i = 0; i < kObsVec; ++i) {
-            const int c = c0 + 128 * i + lane * 4;
-            v[i] = make_float4(0.f, 0.f, 0.f, 0.f);
-            m[i] = v[i];
-            if (c < ld_src) v[i] = *reinterpret_cast<const float4*>(src + c);
-            if (perm && c < ld_dst) {
-                float t[4];
+    for (int i = 0; i < kObsVec; ++i) {
+        const int c = c0 + 128 * i + lane * 4;
+        b.v[i] = make_float4(0.f, 0.f, 0.f, 0.f);
+        b.m[i] = b.v[i];
+        if (c < ld_src) b.v[i] = *reinterpret_cast<const float4*>(src + c);
+        if (perm && c < ld_dst) {
+            float t[4];
 #pragma unroll
-                for (int q = 0; q < 4; ++q) t[q] = c + q < dim ? sign[c + q] * src[perm[c + q]] : 0.f;
-                m[i] = make_float4(t[0], t[1], t[2], t[3]);
-            }
-        }
-#pragma unroll
-        for (int i = 0; i < kObsVec; ++i) {
-            const int c = c0 + 128 * i + lane * 4;
-            if (c < ld_dst) {
-                store_obs_piece(dst, dst16, c, v[i]);
-                if (perm) store_obs_piece(dst_m, dst16_m, c, m[i]);
-            }
+            for (int q = 0; q < 4; ++q) t[q] = c + q < dim ? sign[c + q] * src[perm[c + q]] : 0.f;
+            b.m[i] = make_float4(t[0], t[1], t[2], t[3]);
         }
     }
 }
+
+__device__ __forceinline__ void store_obs_block(const ObsBlock& b, float* dst, __nv_bfloat16* dst16, float* dst_m, __nv_bfloat16* dst16_m,
+                                                int ld_dst, int c0, bool mirrored, int lane) {
+#pragma unroll
+    for (int i = 0; i < kObsVec; ++i) {
+        const int c = c0 + 128 * i + lane * 4;
+        if (c < ld_dst) {
+            store_obs_piece(dst, dst16, c, b.v[i]);
+            if (mirrored) store_obs_piece(dst_m, dst16_m, c, b.m[i]);
+        }
+    }
+}
+
+// A warp takes kGatherRows minibatch rows per pass and issues the loads of all of them before the first store
+// (the destination arrays are plain pointers, so a store in between would order the later loads behind it): the
+// bytes a warp keeps in flight, and with them the bandwidth of this latency-bound kernel, grow with that number.
+constexpr int kGatherRows = 2;
 
 __global__ void __launch_bounds__(256, 3) gather_kernel(const GatherArgs a) {
     chain_begin();
     const int lane = threadIdx.x & 31;
     const int warps = (gridDim.x * blockDim.x) >> 5;
     const bool bf16 = a.x_a16 != nullptr;
-    for (int j = (blockIdx.x * blockDim.x + threadIdx.x) >> 5; j < a.Bmb; j += warps) {
-        const uint32_t src = (uint32_t)a.rows[j];
-        const int t = (int)(src / (uint32_t)a.N);
-        // ---- loads of the small per-row items (lanes 0..3: scalars; lanes < as: action-sized rows)
-        float sc = 0.f;
-        if (lane == 0) sc = a.logp[src];
-        else if (lane == 1) sc = a.values[src];
-        else if (lane == 2) sc = a.returns[src];
-        else if (lane == 3) sc = a.adv[src];
-        float av[2], mv[2], sv[2], am[2];
+    const int ldxa = bf16 ? a.ldxa16 : a.ldxa;
+    const int ldxc = bf16 ? a.ldxc16 : a.ldxc;
+    const int* obs_perm = a.sym ? a.st.obs_perm : nullptr;
+    const int* cobs_perm = a.sym ? a.st.cobs_perm : nullptr;
+    for (int j0 = ((blockIdx.x * blockDim.x + threadIdx.x) >> 5) * kGatherRows; j0 < a.Bmb; j0 += warps * kGatherRows) {
+        uint32_t src[kGatherRows];
+        bool live[kGatherRows];
 #pragma unroll
-        for (int h = 0; h < 2; ++h) {
-            const int c = lane + 32 * h;
-            av[h] = mv[h] = sv[h] = am[h] = 0.f;
-            if (c < a.as) {
-                av[h] = a.actions[(size_t)src * a.as + c];
-                mv[h] = a.mu[(size_t)src * a.as + c];
-                sv[h] = a.sigma[(size_t)t * a.as + c];
-                if (a.sym && c < a.A) am[h] = a.st.act_sign[c] * a.actions[(size_t)src * a.as + a.st.act_perm[c]];
+        for (int r = 0; r < kGatherRows; ++r) {
+            live[r] = j0 + r < a.Bmb;
+            src[r] = live[r] ? (uint32_t)a.rows[j0 + r] : 0u;
+        }
+        // ---- loads of the small per-row items (lanes 0..3: scalars; lanes < as: action-sized rows)
+        float sc[kGatherRows], av[kGatherRows][2], mv[kGatherRows][2], sv[kGatherRows][2], am[kGatherRows][2];
+#pragma unroll
+        for (int r = 0; r < kGatherRows; ++r) {
+            const int t = (int)(src[r] / (uint32_t)a.N);
+            sc[r] = 0.f;
+            if (lane == 0) sc[r] = a.logp[src[r]];
+            else if (lane == 1) sc[r] = a.values[src[r]];
+            else if (lane == 2) sc[r] = a.returns[src[r]];
+            else if (lane == 3) sc[r] = a.adv[src[r]];
+#pragma unroll
+            for (int h = 0; h < 2; ++h) {
+                const int c = lane + 32 * h;
+                av[r][h] = mv[r][h] = sv[r][h] = am[r][h] = 0.f;
+                if (c < a.as) {
+                    av[r][h] = a.actions[(size_t)src[r] * a.as + c];
+                    mv[r][h] = a.mu[(size_t)src[r] * a.as + c];
+                    sv[r][h] = a.sigma[(size_t)t * a.as + c];
+                    if (a.sym && c < a.A) am[r][h] = a.st.act_sign[c] * a.actions[(size_t)src[r] * a.as + a.st.act_perm[c]];
+                }
             }
         }
-        // ---- observation rows (loads, then stores, inside copy_obs_row)
-        const int ldxa = bf16 ? a.ldxa16 : a.ldxa;
-        copy_obs_row(a.obs_a + (size_t)src * a.sa, a.Da, a.sa,
-                     bf16 ? nullptr : a.x_a + (size_t)j * ldxa, bf16 ? a.x_a16 + (size_t)j * ldxa : nullptr,
-                     (bf16 || !a.sym) ? nullptr : a.x_a + (size_t)(j + a.Bmb) * ldxa,
-                     (bf16 && a.sym) ? a.x_a16 + (size_t)(j + a.Bmb) * ldxa : nullptr,
-                     ldxa, a.sym ? a.st.obs_perm : nullptr, a.st.obs_sign, lane);
+        // ---- observation rows, a block of columns at a time: loads of every row, then their stores
+        for (int c0 = 0; c0 < ldxa; c0 += 128 * kObsVec) {
+            ObsBlock blk[kGatherRows];
+#pragma unroll
+            for (int r = 0; r < kGatherRows; ++r)
+                load_obs_block(blk[r], a.obs_a + (size_t)src[r] * a.sa, a.Da, a.sa, ldxa, c0, obs_perm, a.st.obs_sign, lane);
+#pragma unroll
+            for (int r = 0; r < kGatherRows; ++r) {
+                if (!live[r]) continue;
+                const size_t j = (size_t)(j0 + r), jm = j + (size_t)a.Bmb;
+                store_obs_block(blk[r], bf16 ? nullptr : a.x_a + j * ldxa, bf16 ? a.x_a16 + j * ldxa : nullptr,
+                                (bf16 || !a.sym) ? nullptr : a.x_a + jm * ldxa, (bf16 && a.sym) ? a.x_a16 + jm * ldxa : nullptr,
+                                ldxa, c0, a.sym != 0, lane);
+            }
+        }
         if (!a.shared_obs) {
-            const int ldxc = bf16 ? a.ldxc16 : a.ldxc;
-            copy_obs_row(a.obs_c + (size_t)src * a.sc, a.Dc, a.sc,
-                         bf16 ? nullptr : a.x_c + (size_t)j * ldxc, bf16 ? a.x_c16 + (size_t)j * ldxc : nullptr,
-                         (bf16 || !a.sym) ? nullptr : a.x_c + (size_t)(j + a.Bmb) * ldxc,
-                         (bf16 && a.sym) ? a.x_c16 + (size_t)(j + a.Bmb) * ldxc : nullptr,
-                         ldxc, a.sym ? a.st.cobs_perm : nullptr, a.st.cobs_sign, lane);
+            for (int c0 = 0; c0 < ldxc; c0 += 128 * kObsVec) {
+                ObsBlock blk[kGatherRows];
+#pragma unroll
+                for (int r = 0; r < kGatherRows; ++r)
+                    load_obs_block(blk[r], a.obs_c + (size_t)src[r] * a.sc, a.Dc, a.sc, ldxc, c0, cobs_perm, a.st.cobs_sign, lane);
+#pragma unroll
+                for (int r = 0; r < kGatherRows; ++r) {
+                    if (!live[r]) continue;
+                    const size_t j = (size_t)(j0 + r), jm = j + (size_t)a.Bmb;
+                    store_obs_block(blk[r], bf16 ? nullptr : a.x_c + j * ldxc, bf16 ? a.x_c16 + j * ldxc : nullptr,
+                                    (bf16 || !a.sym) ? nullptr : a.x_c + jm * ldxc, (bf16 && a.sym) ? a.x_c16 + jm * ldxc : nullptr,
+                                    ldxc, c0, a.sym != 0, lane);
+                }
+            }
         }
         // ---- stores of the small items
-        if (lane == 0) a.logp_old[j] = sc;
-        else if (lane == 1) a.v_old[j] = sc;
-        else if (lane == 2) a.ret[j] = sc;
-        else if (lane == 3) a.adv_mb[j] = sc;
 #pragma unroll
-        for (int h = 0; h < 2; ++h) {
-            const int c = lane + 32 * h;
-            if (c < a.as) {
-                a.act_mb[(size_t)j * a.as + c] = av[h];
-                a.mu_old[(size_t)j * a.as + c] = mv[h];
-                a.sigma_old[(size_t)j * a.as + c] = sv[h];
-                if (a.sym) a.act_mb[(size_t)(j + a.Bmb) * a.as + c] = am[h];
+        for (int r = 0; r < kGatherRows; ++r) {
+            if (!live[r]) continue;
+            const size_t j = (size_t)(j0 + r);
+            if (lane == 0) a.logp_old[j] = sc[r];
+            else if (lane == 1) a.v_old[j] = sc[r];
+            else if (lane == 2) a.ret[j] = sc[r];
+            else if (lane == 3) a.adv_mb[j] = sc[r];
+#pragma unroll
+            for (int h = 0; h < 2; ++h) {
+                const int c = lane + 32 * h;
+                if (c < a.as) {
+                    a.act_mb[j * a.as + c] = av[r][h];
+                    a.mu_old[j * a.as + c] = mv[r][h];
+                    a.sigma_old[j * a.as + c] = sv[r][h];
+                    if (a.sym) a.act_mb[(j + (size_t)a.Bmb) * a.as + c] = am[r][h];
+                }
             }
         }
     }
@@ -751,10 +790,12 @@ __global__ void __launch_bounds__(kAdamThreads) adam_kernel(const AdamArgs a) {
 
 }  // namespace
 
-cudaError_t launch_gather(const GatherArgs& a, cudaStream_t s) {
+cudaError_t launch_gather(const GatherArgs& a, cudaStream_t s, bool alone) {
     if (a.Bmb <= 0) return cudaSuccess;
-    const int blocks = std::min((a.Bmb + 7) / 8, 148 * 8);
-    LaunchScope scope_("gather", s);
+    // (accounting only) the first gather of an update runs while the caller's stream waits for it, the others beside
+    // the kernels of the minibatch step before
+    LaunchScope scope_(alone ? "gather_alone" : "gather", s);
+    const int blocks = std::min((a.Bmb + 8 * kGatherRows - 1) / (8 * kGatherRows), 148 * 8);
     return launch_chained(gather_kernel, blocks, 256, 0, s, a);
 }
 
