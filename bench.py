@@ -82,7 +82,10 @@ def hbm_family_bytes(w, storage_strides):
     kp_a = -(-w.actor_obs_dim // 64) * 64
     kp_c = -(-w.critic_obs_dim // 64) * 64
     obs_read = 4 * w.actor_obs_dim + (0 if w.shared_obs else 4 * w.critic_obs_dim)
-    obs_written = 2 * kp_a + (0 if w.shared_obs else 2 * kp_c)                    # BF16 operand rows
+    if PRECISION == WL.PRECISION_BF16:
+        obs_written = 2 * kp_a + (0 if w.shared_obs else 2 * kp_c)                # BF16 operand rows
+    else:
+        obs_written = 4 * sa + (0 if w.shared_obs else 4 * sc)                    # FP32 rows
     gather = Bmb * (4 + obs_read + 4 * 2 * w.num_actions + 4 * 4) \
         + R * (obs_written + 4 * as_) + Bmb * (2 * 4 * as_ + 4 * 4)
     P = w.num_params()
@@ -90,14 +93,14 @@ def hbm_family_bytes(w, storage_strides):
 
 
 # DRAM bytes per launch (dram__bytes_read.sum + dram__bytes_write.sum, mean over the family's launches of one
-# minibatch step) from the ncu capture summarised under profiles/, valid while the source of the kernel is the
-# text that capture ran (recognised by the SHA-256 of tc_gemm_kernel's definition); otherwise null.
+# minibatch step) from the ncu capture summarised under profiles/, valid while the source of the kernels is the
+# text that capture ran (recognised by the SHA-256 of the definitions of the three GEMM kernels); otherwise null.
 NCU_TRAFFIC = {
     "source": "paper_2509_10771_b200/csrc/umma.cu",
-    "begin": "template <int MODE>\n__global__ void __launch_bounds__(kThreads, 1) tc_gemm_kernel",
+    "begin": "// Weight gradient: D[features_in x features_out] = A^T B over the minibatch rows",
     "end": "// ------------------------------------------------------------------ fused forward chain",
-    "sha256": "708643086e4c3f63f731700fc2417b2ee9d67b7bd5edb0f95b2af530efdbe5cb",
-    "bytes_per_launch": {"tc_gemm_fwd": 30.7e6, "tc_gemm_dgrad": 65.05e6, "tc_gemm_wgrad": 203.3e6},
+    "sha256": "3883d147aad4b94313c0aba63243bd4c37ca1666fdb6ae252240f64cd62b9c70",
+    "bytes_per_launch": {"tc_gemm_fwd": 31.2e6, "tc_gemm_dgrad": 67.2e6, "tc_gemm_wgrad": 203.3e6},
 }
 
 
@@ -383,6 +386,14 @@ def run_ours(args, rank, world, local_rank):
     # the launches of the per-kernel pass are timed one by one (tens of microseconds each, clocks at their maximum,
     # no power cap): the burst peak is their denominator; the sustained one is printed beside it
     peak, peak_sus = peaks["bf16_tflops"], peaks["bf16_tflops_sustained"]
+    tf32 = PRECISION == WL.PRECISION_TF32
+    if tf32:
+        # no TF32 peak has been measured on this machine: the BF16 figures times the nominal ratio of the two dense
+        # peaks (1.1 / 2.25 PFLOP/s); the weight gradients of this mode run on the FP32 pipes and are no tensor family
+        peak, peak_sus = peak * 1.1 / 2.25, peak_sus * 1.1 / 2.25
+        tc = {k: v for k, v in tc.items() if k in ("tc_gemm_fwd", "tc_gemm_dgrad")}
+        top = max(tc, key=lambda k: tc[k]["ms"])
+        achieved = fam_flops[top] * args.steps / (tc[top]["ms"] * 1e-3) / 1e12
 
     def fam(k):
         tf = fam_flops[k] * args.steps / (tc[k]["ms"] * 1e-3) / 1e12
@@ -390,9 +401,11 @@ def run_ours(args, rank, world, local_rank):
                 "avg_launch_us": 1e3 * tc[k]["ms"] / tc[k]["launches"]}
 
     roofline = {"bound": "tensor", "kernel": top, "achieved": achieved, "peak": peak, "unit": "TFLOP/s",
-                "frac": achieved / peak, "frac_of_sustained": achieved / peak_sus, "frac_of_nominal_2250": achieved / 2250.0,
-                "traffic": ncu_traffic(top), "traffic_unit": "bytes per launch (ncu, dram read + write)",
-                "peak_source": f"bf16 burst (launches timed alone), {peaks['source']}; sustained {peak_sus}",
+                "frac": achieved / peak, "frac_of_sustained": achieved / peak_sus,
+                "frac_of_nominal": achieved / (1100.0 if tf32 else 2250.0),
+                "traffic": None if tf32 else ncu_traffic(top), "traffic_unit": "bytes per launch (ncu, dram read + write)",
+                "peak_source": (f"bf16 burst (launches timed alone), {peaks['source']}; sustained {peak_sus}" if not tf32 else
+                                f"bf16 burst, {peaks['source']}, x 1.1 / 2.25 (nominal tf32 / bf16 ratio); no tf32 peak measured"),
                 "avg_launch_us": 1e3 * tc[top]["ms"] / tc[top]["launches"],
                 "families": {k: fam(k) for k in tc},
                 "timing": "separate pass over the same K steps with one CUDA event pair per launch; the forward and the "
@@ -421,10 +434,10 @@ def run_ours(args, rank, world, local_rank):
     line = {
         "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": max(args.warmup, 3),
         "ms_per_step": ms_total / args.steps, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
-        "dtype": "bf16", "data": "synthetic",
+        "dtype": "tf32" if tf32 else "bf16", "data": "synthetic",
         "config": {"workload": w.name, "num_envs": N, "num_steps": T, "obs_dim": w.actor_obs_dim, "actions": A,
                    "epochs": w.epochs, "minibatches": w.minibatches, "symmetry": bool(w.sym_enable),
-                   "precision": "bf16 operands, fp32 accumulate", "l2": "256 MiB buffer written between timed steps",
+                   "precision": ("tf32" if tf32 else "bf16") + " operands, fp32 accumulate", "l2": "256 MiB buffer written between timed steps",
                    "parallelism": "replicas only" if world > 1 else "1 gpu"},
         "clocks": clocks,
         "one_interval": {"ms_per_step": ms_interval / args.steps,
@@ -742,7 +755,7 @@ def spawn_ranks(n):
 
 
 def main():
-    global WORKLOAD
+    global WORKLOAD, PRECISION
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
     ap.add_argument("--steps", type=int, default=50)
@@ -750,12 +763,15 @@ def main():
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--workload", default=WORKLOAD.name, choices=sorted(WL.WORKLOADS),
                     help="which of the five synthetic workloads to time (default: the one the metric is quoted on)")
+    ap.add_argument("--precision", default="bf16", choices=["bf16", "tf32"],
+                    help="operand precision of the hidden-layer products on the tensor cores (ppo task; default bf16)")
     ap.add_argument("--task", default="ppo", choices=["ppo", "distill", "rnd", "gru", "streams"],
                     help="ppo: the learn iteration the metric is quoted on (default); distill: the distillation iteration; "
                          "rnd: random network distillation over one rollout; gru: the recurrent layer over one rollout; "
                          "streams: the GAE scan at a bandwidth-shaped size")
     args = ap.parse_args()
     WORKLOAD = WL.WORKLOADS[args.workload]
+    PRECISION = WL.PRECISION_TF32 if args.precision == "tf32" else WL.PRECISION_BF16
     if args.gpus > 1 and "WORLD_SIZE" not in os.environ:
         raise SystemExit(spawn_ranks(args.gpus))
     rank = int(os.environ.get("RANK", "0"))
