@@ -553,7 +553,7 @@ def run_rnd(args):
     d_obs = torch.from_numpy(obs).to(dev)
     d_rew = torch.zeros(B, device=dev)
     rnd = binding.Rnd(w.actor_obs_dim, setup["idx"], setup["hidden"], setup["embed_dim"], max_rows=B, lr=1e-3,
-                      stream=stream.cuda_stream)
+                      stream=stream.cuda_stream, max_batch=B, max_epochs=w.epochs, max_minibatches=w.minibatches)
     rnd.set_params(setup["predictor"], setup["target"])
     flush_buf = torch.empty(256 << 20, dtype=torch.uint8, device=dev)
     it = [0]

@@ -286,6 +286,24 @@ rslrl_status rslrl_gae_scan_static(const float *d_rewards, const float *d_values
                                    float adv_eps, void *cuda_stream);
 
 /* ---------------------------------------------------------------------------------------------
+ * Checking build.  Compiled with -DRSLRL_DEBUG the library (a) places every device allocation
+ * between two 256-byte guard regions of a fixed pattern and (b) checks, in the kernels that index
+ * through data they read (the shuffled row numbers of the minibatch gather, the row numbers and
+ * the selected entries of the RND subset), that the index is in range; an index that is not is
+ * replaced by 0 and recorded in a device flag.  Nothing traps and no access leaves its buffer
+ * through these indices.  rslrl_debug_report, to be called between steps, synchronises the device
+ * and writes (each pointer is host memory and may be NULL):
+ *   h_debug_build     1 in the checking build, 0 otherwise (the other two are then always 0)
+ *   h_damaged_guards  number of guard regions whose pattern was overwritten (an out-of-bounds write
+ *                     next to an allocation): over all live allocations of the process, plus those
+ *                     found damaged when their allocation was freed (these stay counted)
+ *   h_index_fault     0, or the code of the worst index recorded since the last report (1 = a
+ *                     minibatch row number, 2 = an RND row number, 3 = an RND entry index);
+ *                     reading clears it.
+ * Returns RSLRL_ERR_CUDA if the device reports an error. */
+rslrl_status rslrl_debug_report(int32_t *h_debug_build, int32_t *h_damaged_guards, int32_t *h_index_fault);
+
+/* ---------------------------------------------------------------------------------------------
  * Random network distillation on a subset of the state (paper: "Auxiliary Techniques", the
  * curiosity-driven intrinsic reward computed on selected states only).
  *
@@ -298,7 +316,8 @@ rslrl_status rslrl_gae_scan_static(const float *d_rewards, const float *d_values
  * normalisation and reward-weight schedules, which the paper's library offers around this, are
  * left to the caller.)
  *
- * An rslrl_rnd owns its parameters, Adam moments and work buffers (device memory); calls on one
+ * An rslrl_rnd owns its parameters, Adam moments and work buffers (device memory, all of it
+ * allocated by rslrl_rnd_create from the limits in the config: no later call allocates); calls on one
  * object are not thread-safe; all work is enqueued on the stream given at creation.
  * Parameter vectors (host, float32) are in the order W1[in][out], b1, W2, b2, ... for the
  * layers num_idx -> hidden[0] -> ... -> embed_dim; hidden layers use ELU(alpha). */
@@ -314,6 +333,9 @@ typedef struct {
     float   elu_alpha;
     int32_t max_rows;                   /* largest `rows` of rslrl_rnd_reward and largest minibatch  */
     float   lr, adam_b1, adam_b2, adam_eps;
+    int32_t max_batch;                  /* largest `batch` of rslrl_rnd_update (>= 1)                */
+    int32_t max_epochs;                 /* largest `epochs` of rslrl_rnd_update (>= 1)               */
+    int32_t max_minibatches;            /* largest `minibatches` of rslrl_rnd_update (>= 1)          */
 } rslrl_rnd_cfg;
 
 size_t       rslrl_rnd_num_params(const rslrl_rnd_cfg *cfg);      /* of one net; 0 if cfg is invalid */
@@ -337,7 +359,8 @@ rslrl_status rslrl_rnd_reward(rslrl_rnd *rnd, const float *d_obs, int32_t rows, 
  * divisible; batch / minibatches <= max_rows), one Adam step per chunk; stops after max_steps
  * steps if max_steps > 0.  h_mean_loss (host, may be NULL): mean of the step losses, which makes
  * the call synchronise; h_first_loss likewise for the first step.
- * RSLRL_ERR_SHAPE for an indivisible batch, RSLRL_ERR_UNSUPPORTED beyond max_rows. */
+ * RSLRL_ERR_SHAPE for an indivisible batch, RSLRL_ERR_UNSUPPORTED beyond max_rows, max_batch,
+ * max_epochs or max_minibatches. */
 rslrl_status rslrl_rnd_update(rslrl_rnd *rnd, const float *d_obs, int32_t batch, int32_t obs_stride,
                               int32_t epochs, int32_t minibatches, uint64_t seed, uint32_t iteration,
                               int32_t max_steps, float *h_mean_loss, float *h_first_loss);

@@ -13,6 +13,7 @@ from . import workloads as WL
 
 HERE = os.path.dirname(os.path.abspath(__file__))
 LIB_PATH = os.path.join(HERE, "librslrl_b200.so")
+LIB_PATH_DEBUG = os.path.join(HERE, "librslrl_b200_debug.so")
 
 RSLRL_MAX_HIDDEN = 8
 
@@ -73,7 +74,8 @@ class UpdateStats(C.Structure):
 class RndCfg(C.Structure):
     _fields_ = [("obs_dim", C.c_int32), ("num_idx", C.c_int32), ("h_idx", C.c_void_p), ("num_hidden", C.c_int32),
                 ("hidden", C.c_int32 * 8), ("embed_dim", C.c_int32), ("elu_alpha", C.c_float), ("max_rows", C.c_int32),
-                ("lr", C.c_float), ("adam_b1", C.c_float), ("adam_b2", C.c_float), ("adam_eps", C.c_float)]
+                ("lr", C.c_float), ("adam_b1", C.c_float), ("adam_b2", C.c_float), ("adam_eps", C.c_float),
+                ("max_batch", C.c_int32), ("max_epochs", C.c_int32), ("max_minibatches", C.c_int32)]
 
 
 class GruCfg(C.Structure):
@@ -92,6 +94,7 @@ EXPORTS = [
     "rslrl_ppo_update", "rslrl_ppo_update_steps", "rslrl_distill_update", "rslrl_distill_update_steps", "rslrl_act_host", "rslrl_record_step_host",
     "rslrl_gae_host", "rslrl_gae_scratch_bytes", "rslrl_gae_scan", "rslrl_minibatch_indices",
     "rslrl_kernel_launch_count", "rslrl_profile_enable", "rslrl_profile_report", "rslrl_gae_scan_static",
+    "rslrl_debug_report",
     "rslrl_rnd_num_params", "rslrl_rnd_create", "rslrl_rnd_destroy", "rslrl_rnd_last_error", "rslrl_rnd_set_params",
     "rslrl_rnd_get_params", "rslrl_rnd_get_grads", "rslrl_rnd_reward", "rslrl_rnd_update",
     "rslrl_gru_num_params", "rslrl_gru_create", "rslrl_gru_destroy", "rslrl_gru_last_error", "rslrl_gru_set_params",
@@ -106,13 +109,16 @@ def load_library() -> C.CDLL:
     global _lib
     if _lib is not None:
         return _lib
-    if not os.path.exists(LIB_PATH):
-        raise RuntimeError(f"{LIB_PATH} is missing: run `python -m paper_2509_10771_b200.build` "
+    # RSLRL_B200_DEBUG_LIBRARY=1 selects the checking build (python -m paper_2509_10771_b200.build --debug)
+    path = LIB_PATH_DEBUG if os.environ.get("RSLRL_B200_DEBUG_LIBRARY") == "1" else LIB_PATH
+    if not os.path.exists(path):
+        raise RuntimeError(f"{path} is missing: run `python -m paper_2509_10771_b200.build` "
                            "(there is no CPU fallback)")
-    lib = C.CDLL(LIB_PATH)
+    lib = C.CDLL(path)
     vp, i32, u32, u64, f32, sz = C.c_void_p, C.c_int32, C.c_uint32, C.c_uint64, C.c_float, C.c_size_t
     sig = {
         "rslrl_num_params": (sz, [C.POINTER(ModelCfg)]),
+        "rslrl_debug_report": (i32, [C.POINTER(i32), C.POINTER(i32), C.POINTER(i32)]),
         "rslrl_create": (i32, [C.POINTER(ModelCfg), C.POINTER(PpoCfg), vp, C.POINTER(vp)]),
         "rslrl_destroy": (i32, [vp]),
         "rslrl_last_error": (C.c_char_p, [vp]),
@@ -329,7 +335,9 @@ class Rnd:
     """One rslrl_rnd: target and predictor MLPs on the entries ``idx`` of an observation row."""
 
     def __init__(self, obs_dim: int, idx, hidden, embed_dim: int, max_rows: int, lr: float = 1e-3, elu_alpha: float = 1.0,
-                 adam_b1: float = 0.9, adam_b2: float = 0.999, adam_eps: float = 1e-8, stream: int = 0):
+                 adam_b1: float = 0.9, adam_b2: float = 0.999, adam_eps: float = 1e-8, stream: int = 0,
+                 max_batch: int = 0, max_epochs: int = 8, max_minibatches: int = 16):
+        # max_batch = 0: room for max_minibatches minibatches of max_rows rows
         self.lib = load_library()
         self.handle = None
         self._idx = np.ascontiguousarray(idx, dtype=np.int32)
@@ -340,6 +348,8 @@ class Rnd:
             cfg.hidden[i] = h
         cfg.embed_dim, cfg.elu_alpha, cfg.max_rows = embed_dim, elu_alpha, max_rows
         cfg.lr, cfg.adam_b1, cfg.adam_b2, cfg.adam_eps = lr, adam_b1, adam_b2, adam_eps
+        cfg.max_batch = max_batch if max_batch > 0 else max_rows * max_minibatches
+        cfg.max_epochs, cfg.max_minibatches = max_epochs, max_minibatches
         self.num_params = int(self.lib.rslrl_rnd_num_params(C.byref(cfg)))
         h = C.c_void_p()
         st = self.lib.rslrl_rnd_create(C.byref(cfg), stream, C.byref(h))
@@ -444,6 +454,16 @@ def gae_scan(d_rewards, d_values, d_dones, d_timeouts, d_last_values, d_returns,
                             adv_eps, _ptr(d_scratch), C.c_void_p(stream))
     if st != 0:
         raise RslrlError(st, "rslrl_gae_scan")
+
+
+def debug_report():
+    """(is the checking build loaded, damaged guard regions, worst index-fault code); synchronises the device."""
+    lib = load_library()
+    a, b, c = C.c_int32(0), C.c_int32(0), C.c_int32(0)
+    st = lib.rslrl_debug_report(C.byref(a), C.byref(b), C.byref(c))
+    if st != 0:
+        raise RslrlError(st, "rslrl_debug_report")
+    return bool(a.value), int(b.value), int(c.value)
 
 
 GAE_STATIC_MAX_ENVS = 1048576

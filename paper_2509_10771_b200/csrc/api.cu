@@ -1,5 +1,6 @@
 // The C ABI of rslrl_b200: context, rollout storage, and the host-side sequencing of the
 // kernels that make up act / gae / ppo_update.  No arithmetic of the method lives here.
+#include "guard.h"
 #include "../../include/rslrl_b200.h"
 #include "common.cuh"
 #include "kernels.h"
@@ -156,7 +157,7 @@ template <typename T>
 rslrl_status dev_alloc(rslrl_ctx* c, T** p, size_t count) {
     void* q = nullptr;
     const size_t bytes = std::max<size_t>(count, 1) * sizeof(T);
-    CU(c, cudaMalloc(&q, bytes));
+    CU(c, guarded_malloc(&q, bytes));
     c->allocs.push_back(q);
     CU(c, cudaMemsetAsync(q, 0, bytes, c->stream));
     *p = reinterpret_cast<T*>(q);
@@ -349,7 +350,7 @@ rslrl_status rslrl_destroy(rslrl_ctx* c) {
     }
     if (c->umma) umma_destroy(c->umma);
     if (c->tf32) tf32_destroy(c->tf32);
-    for (void* p : c->allocs) cudaFree(p);
+    for (void* p : c->allocs) guarded_free(p);
     if (c->stats_host) cudaFreeHost(c->stats_host);
     if (c->pack_host) cudaFreeHost(c->pack_host);
     if (c->pack_sent) cudaEventDestroy(c->pack_sent);
@@ -682,7 +683,7 @@ static rslrl_status update_impl(rslrl_ctx* c, int32_t max_steps, rslrl_update_st
         g.obs_a = c->st.obs_actor; g.obs_c = c->st.obs_critic; g.actions = distill ? d_expert : c->st.actions; g.mu = c->st.mu;
         g.sigma = c->st.sigma; g.logp = c->st.logp; g.values = c->st.values; g.returns = c->st.returns;
         g.adv = c->st.advantages;
-        g.N = N; g.sa = c->st.obs_a_stride; g.sc = c->st.obs_c_stride; g.as = c->st.act_stride;
+        g.N = N; g.B = T * N; g.sa = c->st.obs_a_stride; g.sc = c->st.obs_c_stride; g.as = c->st.act_stride;
         g.Da = c->mc.actor_obs_dim; g.Dc = c->mc.critic_obs_dim; g.A = A; g.shared_obs = c->mc.shared_obs;
         g.x_a = c->x_a; g.x_c = c->x_c; g.ldxa = c->actor.in_ld; g.ldxc = c->critic.in_ld;
         if (c->umma) umma_gather_targets(c->umma, &g, buf);

@@ -6,6 +6,7 @@
 //
 //   r = sigmoid(gi_r + gh_r), z = sigmoid(gi_z + gh_z), n = tanh(gi_n + r * gh_n),
 //   h' = (1 - z) n + z h_in,   gi = x W_i + b_i,  gh = h_in W_h + b_h,  h_in(t) = (1 - done[t-1]) h(t-1)
+#include "guard.h"
 #include "../../include/rslrl_b200.h"
 #include "common.cuh"
 #include "kernels.h"
@@ -156,7 +157,7 @@ template <typename T>
 bool dalloc(rslrl_gru* g, T** p, size_t count) {
     void* q = nullptr;
     const size_t bytes = std::max<size_t>(count * sizeof(T), 256);
-    if (cudaMalloc(&q, bytes) != cudaSuccess) return false;
+    if (guarded_malloc(&q, bytes) != cudaSuccess) return false;
     g->allocs.push_back(q);
     if (cudaMemsetAsync(q, 0, bytes, g->stream) != cudaSuccess) return false;
     *p = (T*)q;
@@ -180,7 +181,7 @@ const char* rslrl_gru_last_error(const rslrl_gru* g) { return g ? g->err.c_str()
 rslrl_status rslrl_gru_destroy(rslrl_gru* g) {
     if (!g) return RSLRL_ERR_INVALID_ARG;
     cudaStreamSynchronize(g->stream);
-    for (void* p : g->allocs) cudaFree(p);
+    for (void* p : g->allocs) guarded_free(p);
     delete g;
     return RSLRL_OK;
 }

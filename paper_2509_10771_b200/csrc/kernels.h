@@ -126,7 +126,7 @@ struct GatherArgs {
     const float* obs_a; const float* obs_c; const float* actions; const float* mu;
     const float* sigma; const float* logp; const float* values; const float* returns;
     const float* adv;
-    int N, sa, sc, as, Da, Dc, A;
+    int N, B, sa, sc, as, Da, Dc, A;                        // B = T * N transitions in storage
     int shared_obs;
     // minibatch destination (rows [0,Bmb) originals, [Bmb,2Bmb) mirrored when sym)
     float* x_a; float* x_c; int ldxa, ldxc;                 // fp32 (null in bf16 mode)

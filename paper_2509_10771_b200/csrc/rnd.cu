@@ -4,6 +4,8 @@
 // difference of two nearly equal quantities once the predictor has learnt): the products run on
 // the SIMT GEMM kernels, the rest are the small kernels below.  A context of its own, independent
 // of rslrl_ctx: it works on observation rows the caller passes in.
+#define RSLRL_INDEX_CHECKS
+#include "guard.h"
 #include "../../include/rslrl_b200.h"
 #include "common.cuh"
 #include "kernels.h"
@@ -26,14 +28,14 @@ inline int round_up(int x, int m) { return (x + m - 1) / m * m; }
 struct RLayer { int in, out, out_p; size_t w_off, b_off, w_flat, b_flat; int ld; };
 
 // s[r][j] = obs[row(r)][idx[j]], row(r) = rows ? rows[r] : r; columns [ns, ld) are written as 0
-__global__ void rnd_subset_kernel(const float* __restrict__ obs, int obs_stride, const int* __restrict__ rows,
-                                  const int* __restrict__ idx, int ns, float* __restrict__ s, int ld, int n) {
+__global__ void rnd_subset_kernel(const float* __restrict__ obs, int obs_stride, int obs_dim, const int* __restrict__ rows,
+                                  int rows_limit, const int* __restrict__ idx, int ns, float* __restrict__ s, int ld, int n) {
     chain_begin();
     const long long total = (long long)n * ld;
     for (long long i = blockIdx.x * (long long)blockDim.x + threadIdx.x; i < total; i += (long long)gridDim.x * blockDim.x) {
         const int r = (int)(i / ld), j = (int)(i - (long long)r * ld);
-        const size_t src = rows ? (size_t)rows[r] : (size_t)r;
-        s[i] = j < ns ? obs[src * obs_stride + idx[j]] : 0.f;
+        const size_t src = rows ? (size_t)checked_index((uint32_t)rows[r], (uint32_t)rows_limit, 2) : (size_t)r;
+        s[i] = j < ns ? obs[src * obs_stride + checked_index((uint32_t)idx[j], (uint32_t)obs_dim, 3)] : 0.f;
     }
 }
 
@@ -124,9 +126,9 @@ struct rslrl_rnd {
     float* s = nullptr;                       // [max_rows][lds] the selected state entries
     std::vector<float*> hf, hg, dz;           // per layer: activations of f and g, gradients at f's outputs
     float* loss_partials = nullptr; int max_loss_blocks = 0;
-    float* step_loss = nullptr; int step_loss_cap = 0;
-    int* perm = nullptr; size_t perm_cap = 0;
-    float* gall = nullptr; size_t gall_cap = 0;   // [batch][ldE] the target's outputs for every row of the batch
+    float* step_loss = nullptr;                   // [max_epochs * max_minibatches]
+    int* perm = nullptr;                          // [max_epochs][max_batch]
+    float* gall = nullptr;                        // [max_batch][ldE] the target's outputs for every row of the batch
     long long adam_step = 0;
     std::string err;
 };
@@ -161,6 +163,8 @@ bool valid_cfg(const rslrl_rnd_cfg* c, std::string* why) {
         if (c->hidden[l] < 1 || c->hidden[l] > 8192) return bad("a hidden width is out of range");
     if (c->embed_dim < 1 || c->embed_dim > 8192) return bad("embed_dim out of range");
     if (c->max_rows < 1) return bad("max_rows must be positive");
+    if (c->max_batch < 1 || c->max_epochs < 1 || c->max_minibatches < 1) return bad("max_batch, max_epochs and max_minibatches must be positive");
+    if ((long long)c->max_epochs * c->max_minibatches > (1 << 20)) return bad("max_epochs * max_minibatches exceeds 2^20 steps");
     if (!(c->lr > 0.f) || !(c->adam_eps > 0.f) || c->adam_b1 < 0.f || c->adam_b1 >= 1.f || c->adam_b2 < 0.f || c->adam_b2 >= 1.f)
         return bad("Adam settings out of range");
     return true;
@@ -186,7 +190,7 @@ template <typename T>
 bool dalloc(rslrl_rnd* r, T** p, size_t count) {
     void* q = nullptr;
     const size_t bytes = std::max<size_t>(count * sizeof(T), 256);
-    if (cudaMalloc(&q, bytes) != cudaSuccess) return false;
+    if (guarded_malloc(&q, bytes) != cudaSuccess) return false;
     r->allocs.push_back(q);
     if (cudaMemsetAsync(q, 0, bytes, r->stream) != cudaSuccess) return false;
     *p = (T*)q;
@@ -220,12 +224,12 @@ rslrl_status forward(rslrl_rnd* r, int rows, bool do_f, bool do_g, float* g_last
     return RSLRL_OK;
 }
 
-rslrl_status subset(rslrl_rnd* r, const float* d_obs, int obs_stride, const int* rows_idx, int rows) {
+rslrl_status subset(rslrl_rnd* r, const float* d_obs, int obs_stride, const int* rows_idx, int rows, int rows_limit = 0) {
     const long long total = (long long)rows * r->lds;
     const int blocks = (int)std::min<long long>((total + 255) / 256, 148 * 16);
     LaunchScope scope_("rnd_subset", r->stream);
-    RCU(r, launch_chained(rnd_subset_kernel, dim3(blocks), dim3(256), 0, r->stream, d_obs, obs_stride, rows_idx,
-                          (const int*)r->idx, r->ns, r->s, r->lds, rows));
+    RCU(r, launch_chained(rnd_subset_kernel, dim3(blocks), dim3(256), 0, r->stream, d_obs, obs_stride, (int)r->cfg.obs_dim, rows_idx,
+                          rows_limit, (const int*)r->idx, r->ns, r->s, r->lds, rows));
     return RSLRL_OK;
 }
 
@@ -286,7 +290,7 @@ const char* rslrl_rnd_last_error(const rslrl_rnd* r) { return r ? r->err.c_str()
 rslrl_status rslrl_rnd_destroy(rslrl_rnd* r) {
     if (!r) return RSLRL_ERR_INVALID_ARG;
     cudaStreamSynchronize(r->stream);
-    for (void* p : r->allocs) cudaFree(p);
+    for (void* p : r->allocs) guarded_free(p);
     delete r;
     return RSLRL_OK;
 }
@@ -308,7 +312,10 @@ rslrl_status rslrl_rnd_create(const rslrl_rnd_cfg* cfg, void* cuda_stream, rslrl
     bool ok = dalloc(r, &r->idx, (size_t)r->ns) && dalloc(r, &r->pf, (size_t)r->P_dev) && dalloc(r, &r->pg, (size_t)r->P_dev) &&
               dalloc(r, &r->grad, (size_t)r->P_dev) && dalloc(r, &r->m, (size_t)r->P_dev) && dalloc(r, &r->v, (size_t)r->P_dev) &&
               dalloc(r, &r->partials, (size_t)r->P_dev * r->max_splits) && dalloc(r, &r->s, rows * r->lds) &&
-              dalloc(r, &r->loss_partials, (size_t)r->max_loss_blocks);
+              dalloc(r, &r->loss_partials, (size_t)r->max_loss_blocks) &&
+              dalloc(r, &r->perm, (size_t)cfg->max_epochs * cfg->max_batch) &&
+              dalloc(r, &r->step_loss, (size_t)cfg->max_epochs * cfg->max_minibatches) &&
+              dalloc(r, &r->gall, (size_t)cfg->max_batch * r->ldE);
     for (size_t l = 0; ok && l < r->L.size(); ++l) {
         float *a = nullptr, *b = nullptr, *c = nullptr;
         ok = dalloc(r, &a, rows * r->L[l].ld) && dalloc(r, &b, rows * r->L[l].ld) && dalloc(r, &c, rows * r->L[l].ld);
@@ -393,19 +400,9 @@ rslrl_status rslrl_rnd_update(rslrl_rnd* r, const float* d_obs, int32_t batch, i
     if (rows > r->max_rows) return rfail(r, RSLRL_ERR_UNSUPPORTED, "minibatch of %d rows exceeds max_rows = %d", rows, r->max_rows);
     long long nsteps = (long long)epochs * minibatches;
     if (max_steps > 0) nsteps = std::min<long long>(nsteps, max_steps);
-    if (nsteps > (1 << 20)) return rfail(r, RSLRL_ERR_UNSUPPORTED, "more than 2^20 steps in one call");
-    if ((size_t)epochs * batch > r->perm_cap) {
-        if (!dalloc(r, &r->perm, (size_t)epochs * batch)) return rfail(r, RSLRL_ERR_CUDA, "could not allocate the shuffle buffer");
-        r->perm_cap = (size_t)epochs * batch;
-    }
-    if ((int)nsteps > r->step_loss_cap) {
-        if (!dalloc(r, &r->step_loss, (size_t)nsteps)) return rfail(r, RSLRL_ERR_CUDA, "could not allocate the loss buffer");
-        r->step_loss_cap = (int)nsteps;
-    }
-    if ((size_t)batch > r->gall_cap) {
-        if (!dalloc(r, &r->gall, (size_t)batch * r->ldE)) return rfail(r, RSLRL_ERR_CUDA, "could not allocate the target-output buffer");
-        r->gall_cap = (size_t)batch;
-    }
+    if (batch > r->cfg.max_batch || epochs > r->cfg.max_epochs || minibatches > r->cfg.max_minibatches)
+        return rfail(r, RSLRL_ERR_UNSUPPORTED, "batch %d / epochs %d / minibatches %d exceed the limits given at creation (%d / %d / %d)",
+                     batch, epochs, minibatches, r->cfg.max_batch, r->cfg.max_epochs, r->cfg.max_minibatches);
     RCU(r, launch_perm_epochs(seed, iteration, epochs, (uint32_t)batch, r->perm, r->stream));
     // the target is fixed: its outputs for all rows of the batch are computed once and looked up by the steps
     for (int r0 = 0; r0 < batch; r0 += r->max_rows) {
@@ -423,7 +420,7 @@ rslrl_status rslrl_rnd_update(rslrl_rnd* r, const float* d_obs, int32_t batch, i
     for (int e = 0; e < epochs && done < nsteps; ++e) {
         for (int k = 0; k < minibatches && done < nsteps; ++k, ++done) {
             const int* rows_idx = r->perm + (size_t)e * batch + (size_t)k * rows;
-            rslrl_status s = subset(r, d_obs, obs_stride, rows_idx, rows);
+            rslrl_status s = subset(r, d_obs, obs_stride, rows_idx, rows, batch);
             if (s != RSLRL_OK) return s;
             if ((s = forward(r, rows, true, false, nullptr)) != RSLRL_OK) return s;
             {

@@ -9,6 +9,7 @@
 // memory, warps 2..17 = epilogue (lane quarter warp & 3, 32-column chunk (warp - 2) / 4 of a tile of up to
 // 128 columns).  Every wait is bounded in time; on expiry the CTA raises an error flag, drains its own
 // asynchronous work, frees its tensor memory and returns.
+#include "guard.h"
 #include "tf32.h"
 #include "tc_ptx.cuh"
 
@@ -328,7 +329,7 @@ template <typename T>
 bool talloc(Tf32Engine* e, T** p, size_t count) {
     void* q = nullptr;
     const size_t bytes = std::max<size_t>(count, 1) * sizeof(T);
-    if (cudaMalloc(&q, bytes) != cudaSuccess) return false;
+    if (guarded_malloc(&q, bytes) != cudaSuccess) return false;
     e->allocs.push_back(q);
     if (cudaMemsetAsync(q, 0, bytes, e->s.stream) != cudaSuccess) return false;
     *p = reinterpret_cast<T*>(q);
@@ -445,7 +446,7 @@ Tf32Engine* tf32_create(const Tf32Setup& s, std::string* err) {
 
 void tf32_destroy(Tf32Engine* e) {
     if (!e) return;
-    for (void* p : e->allocs) cudaFree(p);
+    for (void* p : e->allocs) guarded_free(p);
     delete e;
 }
 

@@ -11,6 +11,7 @@
 //
 // Every wait on an mbarrier is bounded in time; on expiry the CTA raises an error flag that
 // the host reads, drains its own asynchronous work, frees its tensor memory and returns.
+#include "guard.h"
 #include "umma.h"
 #include "tc_ptx.cuh"
 
@@ -988,7 +989,7 @@ template <typename T>
 bool ealloc(UmmaEngine* e, T** p, size_t count) {
     void* q = nullptr;
     const size_t bytes = std::max<size_t>(count, 1) * sizeof(T);
-    if (cudaMalloc(&q, bytes) != cudaSuccess) return false;
+    if (guarded_malloc(&q, bytes) != cudaSuccess) return false;
     e->allocs.push_back(q);
     if (cudaMemsetAsync(q, 0, bytes, e->s.stream) != cudaSuccess) return false;
     *p = reinterpret_cast<T*>(q);
@@ -1507,7 +1508,7 @@ UmmaEngine* umma_create(const UmmaSetup& s, std::string* err) {
 
 void umma_destroy(UmmaEngine* e) {
     if (!e) return;
-    for (void* p : e->allocs) cudaFree(p);
+    for (void* p : e->allocs) guarded_free(p);
     delete e;
 }
 

@@ -1,6 +1,8 @@
 // Update-side kernels: keyed-permutation minibatch gather (with mirrored copies), the fused
 // head + PPO loss + loss-gradient kernel, the deterministic gradient reduction, and the
 // single-pass grad-norm / KL-adaptive learning rate / Adam kernel.
+#define RSLRL_INDEX_CHECKS
+#include "guard.h"
 #include "common.cuh"
 #include "kernels.h"
 #include <algorithm>
@@ -85,7 +87,7 @@ __global__ void __launch_bounds__(256, 3) gather_kernel(const GatherArgs a) {
 #pragma unroll
         for (int r = 0; r < kGatherRows; ++r) {
             live[r] = j0 + r < a.Bmb;
-            src[r] = live[r] ? (uint32_t)a.rows[j0 + r] : 0u;
+            src[r] = live[r] ? checked_index((uint32_t)a.rows[j0 + r], (uint32_t)a.B, 1) : 0u;
         }
         // ---- loads of the small per-row items (lanes 0..3: scalars; lanes < as: action-sized rows)
         float sc[kGatherRows], av[kGatherRows][2], mv[kGatherRows][2], sv[kGatherRows][2], am[kGatherRows][2];

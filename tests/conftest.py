@@ -24,3 +24,15 @@ def pytest_collection_modifyitems(config, items):
     for item in items:
         if "gpu" in item.keywords:
             item.add_marker(skip)
+
+
+@pytest.fixture(autouse=True)
+def _checking_build_report(request):
+    """Under the checking build (RSLRL_B200_DEBUG_LIBRARY=1) every GPU test ends with its report: no guard
+    region next to an allocation overwritten, no out-of-range index recorded."""
+    yield
+    if os.environ.get("RSLRL_B200_DEBUG_LIBRARY") == "1" and "gpu" in request.node.keywords:
+        from paper_2509_10771_b200 import binding
+        is_debug, damaged, index_fault = binding.debug_report()
+        assert is_debug, "the checking build was asked for but the plain library is loaded"
+        assert damaged == 0 and index_fault == 0, (damaged, index_fault)

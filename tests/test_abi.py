@@ -70,12 +70,17 @@ def test_rnd_and_gru_configs_without_a_device():
     cfg.hidden[0], cfg.hidden[1] = 16, 8
     cfg.embed_dim, cfg.elu_alpha, cfg.max_rows = 4, 1.0, 64
     cfg.lr, cfg.adam_b1, cfg.adam_b2, cfg.adam_eps = 1e-3, 0.9, 0.999, 1e-8
+    assert lib.rslrl_rnd_num_params(ctypes.byref(cfg)) == 0       # the update's limits are not set yet
+    cfg.max_batch, cfg.max_epochs, cfg.max_minibatches = 256, 5, 4
     assert lib.rslrl_rnd_num_params(ctypes.byref(cfg)) == 3 * 16 + 16 + 16 * 8 + 8 + 8 * 4 + 4
     cfg.num_idx = 9                                    # more selected entries than the observation has
     assert lib.rslrl_rnd_num_params(ctypes.byref(cfg)) == 0
     cfg.num_idx, cfg.lr = 3, 0.0
     assert lib.rslrl_rnd_num_params(ctypes.byref(cfg)) == 0
-    assert ctypes.sizeof(binding.RndCfg) == 4 + 4 + 8 + 4 + 32 + 4 + 4 + 4 + 16 and binding.RndCfg.h_idx.offset == 8
+    cfg.max_epochs, cfg.max_minibatches = 1 << 11, 1 << 10          # more steps than one call may take
+    assert lib.rslrl_rnd_num_params(ctypes.byref(cfg)) == 0
+    assert ctypes.sizeof(binding.RndCfg) == 4 + 4 + 8 + 4 + 32 + 4 + 4 + 4 + 16 + 12 + 4 and binding.RndCfg.h_idx.offset == 8
+    assert binding.RndCfg.max_batch.offset == 80
     g = binding.GruCfg(235, 256, 24, 4096)
     assert lib.rslrl_gru_num_params(ctypes.byref(g)) == 235 * 768 + 768 + 256 * 768 + 768
     assert lib.rslrl_gru_num_params(ctypes.byref(binding.GruCfg(235, 250, 24, 4096))) == 0     # H not a multiple of 4

@@ -33,7 +33,7 @@ def _setup(case, lr=1e-3):
     ws = w.scaled(envs)
     obs = WL.make_rollout_inputs(ws)["obs_actor"][:w.num_steps].reshape(rows, w.actor_obs_dim)
     setup = WL.make_rnd_setup(ws, **kw)
-    rnd = binding.Rnd(w.actor_obs_dim, setup["idx"], setup["hidden"], setup["embed_dim"], max_rows=rows, lr=lr)
+    rnd = binding.Rnd(w.actor_obs_dim, setup["idx"], setup["hidden"], setup["embed_dim"], max_rows=rows, lr=lr, max_batch=rows)
     rnd.set_params(setup["predictor"], setup["target"])
     d_obs = torch.from_numpy(obs).to("cuda")
     return w, rows, setup, rnd, obs, d_obs, mbs, epochs
@@ -120,6 +120,20 @@ def test_rnd_argument_checks():
     with pytest.raises(binding.RslrlError) as e:
         rnd.update(d_obs, 64, 8, 1, 2, seed=0, iteration=0)          # 32 rows per minibatch > max_rows
     assert e.value.status == 5
+    small = binding.Rnd(8, [0, 3, 5], (4,), 2, max_rows=16, max_batch=32, max_epochs=2, max_minibatches=4)
+    small.set_params(np.zeros(n, np.float32), np.ones(n, np.float32))
+    for batch, epochs, mbs in ((64, 1, 4), (32, 3, 4), (32, 1, 8)):  # beyond max_batch, max_epochs, max_minibatches
+        with pytest.raises(binding.RslrlError) as e:
+            small.update(d_obs, batch, 8, epochs, mbs, seed=0, iteration=0)
+        assert e.value.status == 5
+    free0 = torch.cuda.mem_get_info()[0]
+    small.update(d_obs, 32, 8, 2, 4, seed=0, iteration=0)            # at the limits: runs, and allocates nothing
+    torch.cuda.synchronize()
+    assert torch.cuda.mem_get_info()[0] == free0
+    small.destroy()
+    with pytest.raises(binding.RslrlError) as e:
+        binding.Rnd(8, [0, 3, 5], (4,), 2, max_rows=16, max_epochs=0)
+    assert e.value.status == 1
     with pytest.raises(binding.RslrlError) as e:
         rnd.set_params(np.zeros(n + 1, np.float32), np.zeros(n + 1, np.float32))
     assert e.value.status == 2
@@ -145,7 +159,7 @@ def test_intrinsic_reward_enters_gae_like_the_oracle():
     weight = 0.05
     ctx = binding.Context(w, precision=WL.PRECISION_FP32)
     ctx.set_params(theta)
-    rnd = binding.Rnd(Da, setup["idx"], setup["hidden"], setup["embed_dim"], max_rows=N)
+    rnd = binding.Rnd(Da, setup["idx"], setup["hidden"], setup["embed_dim"], max_rows=N, max_batch=N)
     rnd.set_params(setup["predictor"], setup["target"])
     dev = torch.device("cuda")
     oa = torch.from_numpy(inputs["obs_actor"]).to(dev)
@@ -184,7 +198,7 @@ def test_full_size_reward_and_first_step_match_oracle():
     setup = WL.make_rnd_setup(w, num_idx=48, hidden=(256, 128, 64), embed_dim=32)
     obs = WL.make_rollout_inputs(w)["obs_actor"][:T].reshape(B, Da)
     d_obs = torch.from_numpy(obs).to("cuda")
-    rnd = binding.Rnd(Da, setup["idx"], setup["hidden"], setup["embed_dim"], max_rows=B)
+    rnd = binding.Rnd(Da, setup["idx"], setup["hidden"], setup["embed_dim"], max_rows=B, max_batch=B)
     rnd.set_params(setup["predictor"], setup["target"])
     d_int = torch.empty(B, device="cuda")
     rnd.reward(d_obs, B, Da, d_r_int_out=d_int)
