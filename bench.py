@@ -769,8 +769,13 @@ def main():
                     help="ppo: the learn iteration the metric is quoted on (default); distill: the distillation iteration; "
                          "rnd: random network distillation over one rollout; gru: the recurrent layer over one rollout; "
                          "streams: the GAE scan at a bandwidth-shaped size")
+    ap.add_argument("--envs", type=int, default=0,
+                    help="run the workload on this many environments instead of its own number (a size a profiler "
+                         "capture can hold; the workload's name in the JSON line then ends in @<envs>)")
     args = ap.parse_args()
     WORKLOAD = WL.WORKLOADS[args.workload]
+    if args.envs > 0:
+        WORKLOAD = WORKLOAD.scaled(args.envs)
     PRECISION = WL.PRECISION_TF32 if args.precision == "tf32" else WL.PRECISION_BF16
     if args.gpus > 1 and "WORLD_SIZE" not in os.environ:
         raise SystemExit(spawn_ranks(args.gpus))

@@ -34,133 +34,131 @@ __device__ __forceinline__ void store_obs_piece(float* dst, __nv_bfloat16* dst16
     }
 }
 
-// One block of up to 128 * kObsVec columns of an observation row: the pieces of the row itself and, when perm
-// is given, of its mirror m[c] = sign[c] * src[perm[c]] (storage pads are zero; columns past ld_dst are not used).
-struct ObsBlock { float4 v[kObsVec]; float4 m[kObsVec]; };
+// Observation rows: a warp takes kGatherRows minibatch rows per pass and issues the loads of all of them before the
+// first store; the row numbers of a pass are loaded during the pass before, and the rows of the next pass are
+// prefetched into L2 meanwhile (one bulk prefetch per row and matrix, issued by one lane, no registers held).  The
+// bandwidth of this kernel is the bytes it keeps in flight, so this loop carries nothing but the rows; the small
+// per-row items are gathered by a second loop with one thread per row.  Storage is read through the read-only path
+// (it does not change while an update runs).
+constexpr int kGatherRows = 8;
 
-__device__ __forceinline__ void load_obs_block(ObsBlock& b, const float* __restrict__ src, int dim, int ld_src, int ld_dst, int c0,
-                                               const int* __restrict__ perm, const float* __restrict__ sign, int lane) {
+struct MirrorTables { int pc[kObsVec][4]; float sg[kObsVec][4]; };   // of one column block, the same for every row
+
+__device__ __forceinline__ void load_mirror_tables(MirrorTables& t, const int* __restrict__ perm, const float* __restrict__ sign,
+                                                   int dim, int c0, int lane) {
+#pragma unroll
+    for (int i = 0; i < kObsVec; ++i)
+#pragma unroll
+        for (int q = 0; q < 4; ++q) {
+            const int c = c0 + 128 * i + lane * 4 + q;
+            t.pc[i][q] = c < dim ? __ldg(perm + c) : 0;
+            t.sg[i][q] = c < dim ? __ldg(sign + c) : 0.f;
+        }
+}
+
+// float4 pieces of the column block at c0 of one storage row (pads of the storage row are zero)
+__device__ __forceinline__ void load_obs_pieces(float4 (&v)[kObsVec], const float* __restrict__ row, int stride, int c0, int lane) {
 #pragma unroll
     for (int i = 0; i < kObsVec; ++i) {
         const int c = c0 + 128 * i + lane * 4;
-        b.v[i] = make_float4(0.f, 0.f, 0.f, 0.f);
-        b.m[i] = b.v[i];
-        if (c < ld_src) b.v[i] = *reinterpret_cast<const float4*>(src + c);
-        if (perm && c < ld_dst) {
-            float t[4];
+        v[i] = c < stride ? __ldg(reinterpret_cast<const float4*>(row + c)) : make_float4(0.f, 0.f, 0.f, 0.f);
+    }
+}
+
+// Stores the pieces into minibatch row j and, when t is given, the mirror m[c] = sign[c] * row[perm[c]] into row
+// j + Bmb (the row is read back through L1, where it has just landed); destination columns [dim, ld_dst) get zero.
+__device__ __forceinline__ void store_obs_pieces(const float4 (&v)[kObsVec], const float* __restrict__ row, const MirrorTables* t,
+                                                 float* x, __nv_bfloat16* x16, int ld_dst, size_t j, size_t Bmb, int c0, int lane) {
 #pragma unroll
-            for (int q = 0; q < 4; ++q) t[q] = c + q < dim ? sign[c + q] * src[perm[c + q]] : 0.f;
-            b.m[i] = make_float4(t[0], t[1], t[2], t[3]);
+    for (int i = 0; i < kObsVec; ++i) {
+        const int c = c0 + 128 * i + lane * 4;
+        if (c >= ld_dst) continue;
+        store_obs_piece(x16 ? nullptr : x + j * ld_dst, x16 ? x16 + j * ld_dst : nullptr, c, v[i]);
+        if (t) {
+            const float4 m = make_float4(t->sg[i][0] * __ldg(row + t->pc[i][0]), t->sg[i][1] * __ldg(row + t->pc[i][1]),
+                                         t->sg[i][2] * __ldg(row + t->pc[i][2]), t->sg[i][3] * __ldg(row + t->pc[i][3]));
+            store_obs_piece(x16 ? nullptr : x + (j + Bmb) * ld_dst, x16 ? x16 + (j + Bmb) * ld_dst : nullptr, c, m);
         }
     }
 }
 
-__device__ __forceinline__ void store_obs_block(const ObsBlock& b, float* dst, __nv_bfloat16* dst16, float* dst_m, __nv_bfloat16* dst16_m,
-                                                int ld_dst, int c0, bool mirrored, int lane) {
-#pragma unroll
-    for (int i = 0; i < kObsVec; ++i) {
-        const int c = c0 + 128 * i + lane * 4;
-        if (c < ld_dst) {
-            store_obs_piece(dst, dst16, c, b.v[i]);
-            if (mirrored) store_obs_piece(dst_m, dst16_m, c, b.m[i]);
-        }
-    }
+__device__ __forceinline__ void prefetch_row_l2(const float* row, uint32_t bytes) {
+    asm volatile("cp.async.bulk.prefetch.L2.global [%0], %1;" ::"l"(row), "r"(bytes) : "memory");
 }
 
-// A warp takes kGatherRows minibatch rows per pass and issues the loads of all of them before the first store
-// (the destination arrays are plain pointers, so a store in between would order the later loads behind it): the
-// bytes a warp keeps in flight, and with them the bandwidth of this latency-bound kernel, grow with that number.
-constexpr int kGatherRows = 2;
-
-__global__ void __launch_bounds__(256, 3) gather_kernel(const GatherArgs a) {
+__global__ void __launch_bounds__(256, 2) gather_kernel(const GatherArgs a) {
     chain_begin();
     const int lane = threadIdx.x & 31;
     const int warps = (gridDim.x * blockDim.x) >> 5;
     const bool bf16 = a.x_a16 != nullptr;
     const int ldxa = bf16 ? a.ldxa16 : a.ldxa;
+    const int first = ((blockIdx.x * blockDim.x + threadIdx.x) >> 5) * kGatherRows;
+    // ---- observation rows: one sweep over the minibatch per matrix and block of 128 * kObsVec columns
+    const int blocks_a = (ldxa + 128 * kObsVec - 1) / (128 * kObsVec);
     const int ldxc = bf16 ? a.ldxc16 : a.ldxc;
-    const int* obs_perm = a.sym ? a.st.obs_perm : nullptr;
-    const int* cobs_perm = a.sym ? a.st.cobs_perm : nullptr;
-    for (int j0 = ((blockIdx.x * blockDim.x + threadIdx.x) >> 5) * kGatherRows; j0 < a.Bmb; j0 += warps * kGatherRows) {
+    const int sweeps = blocks_a + (a.shared_obs ? 0 : (ldxc + 128 * kObsVec - 1) / (128 * kObsVec));
+    for (int sweep = 0; sweep < sweeps; ++sweep) {
+        const bool critic = sweep >= blocks_a;
+        const float* __restrict__ obs = critic ? a.obs_c : a.obs_a;
+        const int stride = critic ? a.sc : a.sa, dim = critic ? a.Dc : a.Da, ld_dst = critic ? ldxc : ldxa;
+        const int c0 = (critic ? sweep - blocks_a : sweep) * 128 * kObsVec;
+        const int* perm = !a.sym ? nullptr : critic ? a.st.cobs_perm : a.st.obs_perm;
+        float* x = critic ? a.x_c : a.x_a;
+        __nv_bfloat16* x16 = critic ? a.x_c16 : a.x_a16;
+        MirrorTables mt;
+        if (perm) load_mirror_tables(mt, perm, critic ? a.st.cobs_sign : a.st.obs_sign, dim, c0, lane);
         uint32_t src[kGatherRows];
-        bool live[kGatherRows];
 #pragma unroll
-        for (int r = 0; r < kGatherRows; ++r) {
-            live[r] = j0 + r < a.Bmb;
-            src[r] = live[r] ? checked_index((uint32_t)a.rows[j0 + r], (uint32_t)a.B, 1) : 0u;
-        }
-        // ---- loads of the small per-row items (lanes 0..3: scalars; lanes < as: action-sized rows)
-        float sc[kGatherRows], av[kGatherRows][2], mv[kGatherRows][2], sv[kGatherRows][2], am[kGatherRows][2];
-#pragma unroll
-        for (int r = 0; r < kGatherRows; ++r) {
-            const int t = (int)(src[r] / (uint32_t)a.N);
-            sc[r] = 0.f;
-            if (lane == 0) sc[r] = a.logp[src[r]];
-            else if (lane == 1) sc[r] = a.values[src[r]];
-            else if (lane == 2) sc[r] = a.returns[src[r]];
-            else if (lane == 3) sc[r] = a.adv[src[r]];
-#pragma unroll
-            for (int h = 0; h < 2; ++h) {
-                const int c = lane + 32 * h;
-                av[r][h] = mv[r][h] = sv[r][h] = am[r][h] = 0.f;
-                if (c < a.as) {
-                    av[r][h] = a.actions[(size_t)src[r] * a.as + c];
-                    mv[r][h] = a.mu[(size_t)src[r] * a.as + c];
-                    sv[r][h] = a.sigma[(size_t)t * a.as + c];
-                    if (a.sym && c < a.A) am[r][h] = a.st.act_sign[c] * a.actions[(size_t)src[r] * a.as + a.st.act_perm[c]];
-                }
-            }
-        }
-        // ---- observation rows, a block of columns at a time: loads of every row, then their stores
-        for (int c0 = 0; c0 < ldxa; c0 += 128 * kObsVec) {
-            ObsBlock blk[kGatherRows];
-#pragma unroll
-            for (int r = 0; r < kGatherRows; ++r)
-                load_obs_block(blk[r], a.obs_a + (size_t)src[r] * a.sa, a.Da, a.sa, ldxa, c0, obs_perm, a.st.obs_sign, lane);
+        for (int r = 0; r < kGatherRows; ++r)
+            src[r] = first + r < a.Bmb ? checked_index((uint32_t)__ldg(a.rows + first + r), (uint32_t)a.B, 1) : 0u;
+        for (int j0 = first; j0 < a.Bmb; j0 += warps * kGatherRows) {
+            uint32_t nxt[kGatherRows];
 #pragma unroll
             for (int r = 0; r < kGatherRows; ++r) {
-                if (!live[r]) continue;
-                const size_t j = (size_t)(j0 + r), jm = j + (size_t)a.Bmb;
-                store_obs_block(blk[r], bf16 ? nullptr : a.x_a + j * ldxa, bf16 ? a.x_a16 + j * ldxa : nullptr,
-                                (bf16 || !a.sym) ? nullptr : a.x_a + jm * ldxa, (bf16 && a.sym) ? a.x_a16 + jm * ldxa : nullptr,
-                                ldxa, c0, a.sym != 0, lane);
+                const int jn = j0 + warps * kGatherRows + r;
+                nxt[r] = jn < a.Bmb ? (uint32_t)__ldg(a.rows + jn) : 0u;
             }
+            float4 v[kGatherRows][kObsVec];
+#pragma unroll
+            for (int r = 0; r < kGatherRows; ++r) load_obs_pieces(v[r], obs + (size_t)src[r] * stride, stride, c0, lane);
+            // the next pass's rows towards L2 (rows are 16-byte multiples at 16-byte aligned addresses)
+            if (c0 == 0 && lane < kGatherRows && j0 + warps * kGatherRows + lane < a.Bmb) {
+                uint32_t sn = nxt[0];
+#pragma unroll
+                for (int r = 1; r < kGatherRows; ++r) if (lane == r) sn = nxt[r];
+                prefetch_row_l2(obs + (size_t)checked_index(sn, (uint32_t)a.B, 1) * stride, (uint32_t)stride * 4u);
+            }
+#pragma unroll
+            for (int r = 0; r < kGatherRows; ++r)
+                if (j0 + r < a.Bmb)
+                    store_obs_pieces(v[r], obs + (size_t)src[r] * stride, perm ? &mt : nullptr, x, x16, ld_dst, (size_t)(j0 + r),
+                                     (size_t)a.Bmb, c0, lane);
+#pragma unroll
+            for (int r = 0; r < kGatherRows; ++r) src[r] = checked_index(nxt[r], (uint32_t)a.B, 1);
         }
-        if (!a.shared_obs) {
-            for (int c0 = 0; c0 < ldxc; c0 += 128 * kObsVec) {
-                ObsBlock blk[kGatherRows];
-#pragma unroll
-                for (int r = 0; r < kGatherRows; ++r)
-                    load_obs_block(blk[r], a.obs_c + (size_t)src[r] * a.sc, a.Dc, a.sc, ldxc, c0, cobs_perm, a.st.cobs_sign, lane);
-#pragma unroll
-                for (int r = 0; r < kGatherRows; ++r) {
-                    if (!live[r]) continue;
-                    const size_t j = (size_t)(j0 + r), jm = j + (size_t)a.Bmb;
-                    store_obs_block(blk[r], bf16 ? nullptr : a.x_c + j * ldxc, bf16 ? a.x_c16 + j * ldxc : nullptr,
-                                    (bf16 || !a.sym) ? nullptr : a.x_c + jm * ldxc, (bf16 && a.sym) ? a.x_c16 + jm * ldxc : nullptr,
-                                    ldxc, c0, a.sym != 0, lane);
-                }
-            }
+    }
+    // ---- the small per-row items, one thread per minibatch row (action-sized rows are multiples of four floats)
+    const int as4 = a.as >> 2;
+    for (int j = blockIdx.x * blockDim.x + threadIdx.x; j < a.Bmb; j += gridDim.x * blockDim.x) {
+        const uint32_t s = checked_index((uint32_t)__ldg(a.rows + j), (uint32_t)a.B, 1);
+        const int t = (int)(s / (uint32_t)a.N);
+        const float lp = __ldg(a.logp + s), vl = __ldg(a.values + s), rt = __ldg(a.returns + s), ad = __ldg(a.adv + s);
+        const float4* ac = reinterpret_cast<const float4*>(a.actions + (size_t)s * a.as);
+        const float4* mu = reinterpret_cast<const float4*>(a.mu + (size_t)s * a.as);
+        const float4* sg = reinterpret_cast<const float4*>(a.sigma + (size_t)t * a.as);
+        float4* ac_o = reinterpret_cast<float4*>(a.act_mb + (size_t)j * a.as);
+        float4* mu_o = reinterpret_cast<float4*>(a.mu_old + (size_t)j * a.as);
+        float4* sg_o = reinterpret_cast<float4*>(a.sigma_old + (size_t)j * a.as);
+        a.logp_old[j] = lp; a.v_old[j] = vl; a.ret[j] = rt; a.adv_mb[j] = ad;
+        for (int q = 0; q < as4; ++q) {
+            const float4 x = __ldg(ac + q), y = __ldg(mu + q), z = __ldg(sg + q);
+            ac_o[q] = x; mu_o[q] = y; sg_o[q] = z;
         }
-        // ---- stores of the small items
-#pragma unroll
-        for (int r = 0; r < kGatherRows; ++r) {
-            if (!live[r]) continue;
-            const size_t j = (size_t)(j0 + r);
-            if (lane == 0) a.logp_old[j] = sc[r];
-            else if (lane == 1) a.v_old[j] = sc[r];
-            else if (lane == 2) a.ret[j] = sc[r];
-            else if (lane == 3) a.adv_mb[j] = sc[r];
-#pragma unroll
-            for (int h = 0; h < 2; ++h) {
-                const int c = lane + 32 * h;
-                if (c < a.as) {
-                    a.act_mb[j * a.as + c] = av[r][h];
-                    a.mu_old[j * a.as + c] = mv[r][h];
-                    a.sigma_old[j * a.as + c] = sv[r][h];
-                    if (a.sym) a.act_mb[(j + (size_t)a.Bmb) * a.as + c] = am[r][h];
-                }
-            }
+        if (a.sym) {
+            float* am = a.act_mb + ((size_t)j + (size_t)a.Bmb) * a.as;
+            const float* arow = a.actions + (size_t)s * a.as;
+            for (int c = 0; c < a.as; ++c)
+                am[c] = c < a.A ? __ldg(a.st.act_sign + c) * __ldg(arow + __ldg(a.st.act_perm + c)) : 0.f;
         }
     }
 }
@@ -797,7 +795,7 @@ cudaError_t launch_gather(const GatherArgs& a, cudaStream_t s, bool alone) {
     // (accounting only) the first gather of an update runs while the caller's stream waits for it, the others beside
     // the kernels of the minibatch step before
     LaunchScope scope_(alone ? "gather_alone" : "gather", s);
-    const int blocks = std::min((a.Bmb + 8 * kGatherRows - 1) / (8 * kGatherRows), 148 * 8);
+    const int blocks = std::min((a.Bmb + 8 * kGatherRows - 1) / (8 * kGatherRows), 148 * 2);     // one resident wave
     return launch_chained(gather_kernel, blocks, 256, 0, s, a);
 }
 
