@@ -120,11 +120,28 @@ __global__ void __launch_bounds__(kThreads, NT <= 6 ? 3 : 2) head_loss_mma_kerne
             const size_t r0 = (size_t)jc0 + (size_t)copy * a.Bmb, r1 = (size_t)jc1 + (size_t)copy * a.Bmb;
             const __nv_bfloat16* __restrict__ ha0 = Ha + r0 * a.ldha; const __nv_bfloat16* __restrict__ ha1 = Ha + r1 * a.ldha;
             const __nv_bfloat16* __restrict__ hc0 = Hc + r0 * a.ldhc; const __nv_bfloat16* __restrict__ hc1 = Hc + r1 * a.ldhc;
+            // the per-action inputs of the loss terms, requested before the products so that they arrive meanwhile
+            float act_in[NT][4], so_in[NT][4], mo_in[NT][4];
+#pragma unroll
+            for (int j = 0; j < NT; ++j)
+#pragma unroll
+                for (int e = 0; e < 4; ++e) {
+                    const int i = 8 * j + 2 * t + (e & 1);
+                    act_in[j][e] = so_in[j][e] = mo_in[j][e] = 0.f;
+                    if (i < A) {
+                        act_in[j][e] = a.act_mb[((e >> 1) ? r1 : r0) * a.as + i];
+                        if (copy == 0 && !a.distill) {
+                            const int jj = (e >> 1) ? jc1 : jc0;
+                            so_in[j][e] = a.sigma_old[(size_t)jj * a.as + i];
+                            mo_in[j][e] = a.mu_old[(size_t)jj * a.as + i];
+                        }
+                    }
+                }
             // ---- heads ------------------------------------------------------------------------
             float mu[NT][4];
 #pragma unroll
             for (int j = 0; j < NT; ++j) { mu[j][0] = mu[j][2] = bias_a[j][0]; mu[j][1] = mu[j][3] = bias_a[j][1]; }
-#pragma unroll 4
+#pragma unroll 8
             for (int ks = 0; ks < ksa; ++ks) {
                 uint32_t af[4];
                 af[0] = *reinterpret_cast<const uint32_t*>(ha0 + 16 * ks + 2 * t);
@@ -138,6 +155,7 @@ __global__ void __launch_bounds__(kThreads, NT <= 6 ? 3 : 2) head_loss_mma_kerne
                 }
             }
             float v[2] = {0.f, 0.f};
+#pragma unroll 8
             for (int ks = 0; ks < ksc; ++ks) {
                 const float2 w01 = *reinterpret_cast<const float2*>(Wc_s + 16 * ks + 2 * t);
                 const float2 w89 = *reinterpret_cast<const float2*>(Wc_s + 16 * ks + 8 + 2 * t);
@@ -161,15 +179,13 @@ __global__ void __launch_bounds__(kThreads, NT <= 6 ? 3 : 2) head_loss_mma_kerne
                     const int i = 8 * j + 2 * t + c;
                     dmu[j][e] = 0.f;
                     if (i < A) {
-                        const size_t r = h ? r1 : r0;
-                        const int jj = h ? jc1 : jc0;
-                        const float d = a.act_mb[r * a.as + i] - mu[j][e];
+                        const float d = act_in[j][e] - mu[j][e];
                         if (a.distill) { sq[h] += d * d; dmu[j][e] = d; continue; }      // (a* - mu_i)^2
                         lp[h] += -(d * d) * 0.5f * ivar[j][c] - ls[j][c] - kHalfLog2Pi;
                         dmu[j][e] = d * ivar[j][c];                       // d logp / d mu_i
                         if (copy == 0) {
-                            const float so = a.sigma_old[(size_t)jj * a.as + i];
-                            const float dm = a.mu_old[(size_t)jj * a.as + i] - mu[j][e];
+                            const float so = so_in[j][e];
+                            const float dm = mo_in[j][e] - mu[j][e];
                             kl[h] += (ls[j][c] - logf(so)) + (so * so + dm * dm) * 0.5f * ivar[j][c] - 0.5f;
                         }
                     }
@@ -263,7 +279,7 @@ __global__ void __launch_bounds__(kThreads, NT <= 6 ? 3 : 2) head_loss_mma_kerne
                 df[ka][3] = pack_bf16(dmu[2 * ka + 1][2], dmu[2 * ka + 1][3]);
             }
             __nv_bfloat16* __restrict__ dza0 = dZa + r0 * a.lddza; __nv_bfloat16* __restrict__ dza1 = dZa + r1 * a.lddza;
-#pragma unroll 4
+#pragma unroll 8
             for (int jn = 0; jn < 2 * ksa; ++jn) {                        // 8 hidden units per step
                 float acc[4] = {0.f, 0.f, 0.f, 0.f};
 #pragma unroll
@@ -286,7 +302,7 @@ __global__ void __launch_bounds__(kThreads, NT <= 6 ? 3 : 2) head_loss_mma_kerne
             }
             // ---- critic: dz = dV * Wc * ELU'(h), element-wise on the same column pairs ------------------
             __nv_bfloat16* __restrict__ dzc0 = dZc + r0 * a.lddzc; __nv_bfloat16* __restrict__ dzc1 = dZc + r1 * a.lddzc;
-#pragma unroll 4
+#pragma unroll 8
             for (int jn = 0; jn < 2 * ksc; ++jn) {
                 const int col = 8 * jn + 2 * t;
                 const float2 w = *reinterpret_cast<const float2*>(Wc_s + col);

@@ -647,6 +647,47 @@ constexpr int kAdamThreads = 256;
 
 __global__ void __launch_bounds__(kAdamThreads) adam_kernel(const AdamArgs a) {
     chain_begin();
+    // The first group of every thread is loaded before the block derives its scalars: those loads need none of them,
+    // and the sums below are a chain of dependent loads of their own.
+    // BF16 mode, hidden-layer weights: a thread takes four consecutive ROWS of one column instead of four
+    // consecutive columns of one row, so that its entries of the transposed operand copy Wt[out][in] are
+    // one 8-byte store (neighbouring threads: neighbouring columns, every FP32 access still coalesced).
+    // Those groups cover the rows below the last multiple of four, the same elements as before in another
+    // assignment; the remaining rows, biases and everything else take the plain path.
+    struct Group { float g[4], p[4], m[4], v[4]; size_t base; int e, r4, o; bool rows; };
+    auto fetch = [&](int i, Group& G) {
+        const int idx0 = 4 * i;
+        int e = 0;
+        while (e < a.n_cvt && !(idx0 >= a.cvt[e].w_off && idx0 < a.cvt[e].w_off + a.cvt[e].in * a.cvt[e].out_p)) ++e;
+        G.rows = false;
+        if (e < a.n_cvt) {
+            const CvtRange& c = a.cvt[e];
+            const int lg = (idx0 - c.w_off) >> 2;
+            if (lg < (c.in >> 2) * c.out_p) {
+                G.rows = true; G.e = e;
+                G.r4 = lg / c.out_p; G.o = lg - G.r4 * c.out_p;
+                G.base = (size_t)c.w_off + (size_t)(4 * G.r4) * c.out_p + G.o;
+#pragma unroll
+                for (int q = 0; q < 4; ++q) {
+                    const size_t at = G.base + (size_t)q * c.out_p;
+                    G.g[q] = a.grad[at]; G.p[q] = a.param[at]; G.m[q] = a.m[at]; G.v[q] = a.v[at];
+                }
+                return;
+            }
+        }
+        const float4 g4 = reinterpret_cast<const float4*>(a.grad)[i];
+        const float4 p4 = reinterpret_cast<const float4*>(a.param)[i];
+        const float4 m4 = reinterpret_cast<const float4*>(a.m)[i];
+        const float4 v4 = reinterpret_cast<const float4*>(a.v)[i];
+        G.g[0] = g4.x; G.g[1] = g4.y; G.g[2] = g4.z; G.g[3] = g4.w;
+        G.p[0] = p4.x; G.p[1] = p4.y; G.p[2] = p4.z; G.p[3] = p4.w;
+        G.m[0] = m4.x; G.m[1] = m4.y; G.m[2] = m4.z; G.m[3] = m4.w;
+        G.v[0] = v4.x; G.v[1] = v4.y; G.v[2] = v4.z; G.v[3] = v4.w;
+    };
+    const int n4 = a.P / 4;
+    int i = blockIdx.x * kAdamThreads + threadIdx.x;
+    Group G;
+    if (i < n4) fetch(i, G);
     __shared__ float s_scal[4];   // clip coefficient, lr, bias corrections
     __shared__ int s_skip;
     if (threadIdx.x < 32) {
@@ -688,67 +729,8 @@ __global__ void __launch_bounds__(kAdamThreads) adam_kernel(const AdamArgs a) {
     __syncthreads();
     if (s_skip) return;          // non-finite step: parameters and moments stay untouched
     const float coef = s_scal[0], lr = s_scal[1], c1 = s_scal[2], c2 = s_scal[3];
-    const int n4 = a.P / 4;
-    for (int i = blockIdx.x * kAdamThreads + threadIdx.x; i < n4; i += gridDim.x * kAdamThreads) {
-        // BF16 mode, hidden-layer weights: a thread takes four consecutive ROWS of one column instead of four
-        // consecutive columns of one row, so that its entries of the transposed operand copy Wt[out][in] are
-        // one 8-byte store (neighbouring threads: neighbouring columns, every FP32 access still coalesced).
-        // Those groups cover the rows below the last multiple of four, the same elements as before in another
-        // assignment; the remaining rows, biases and everything else take the path below.
-        {
-            const int idx0 = 4 * i;
-            int e = 0;
-            while (e < a.n_cvt && !(idx0 >= a.cvt[e].w_off && idx0 < a.cvt[e].w_off + a.cvt[e].in * a.cvt[e].out_p)) ++e;
-            if (e < a.n_cvt) {
-                const CvtRange& c = a.cvt[e];
-                const int lg = (idx0 - c.w_off) >> 2;
-                if (lg < (c.in >> 2) * c.out_p) {
-                    const int r4 = lg / c.out_p, o = lg - r4 * c.out_p;
-                    const size_t base = (size_t)c.w_off + (size_t)(4 * r4) * c.out_p + o;
-                    float g[4], p[4], m[4], v[4];
-#pragma unroll
-                    for (int q = 0; q < 4; ++q) {
-                        const size_t at = base + (size_t)q * c.out_p;
-                        g[q] = a.grad[at]; p[q] = a.param[at]; m[q] = a.m[at]; v[q] = a.v[at];
-                    }
-#pragma unroll
-                    for (int q = 0; q < 4; ++q) {
-                        const float gc = g[q] * coef;
-                        m[q] = a.b1 * m[q] + (1.0f - a.b1) * gc;
-                        v[q] = a.b2 * v[q] + (1.0f - a.b2) * gc * gc;
-                        p[q] = p[q] - lr * (m[q] * c1) / (sqrtf(v[q] * c2) + a.eps);
-                        const size_t at = base + (size_t)q * c.out_p;
-                        a.param[at] = p[q]; a.m[at] = m[q]; a.v[at] = v[q];
-                    }
-                    if (o < c.out) {
-                        __nv_bfloat16 w[4];
-#pragma unroll
-                        for (int q = 0; q < 4; ++q) {
-                            w[q] = __float2bfloat16_rn(p[q]);
-                            if (c.wn) c.wn[(size_t)(4 * r4 + q) * c.ld_wn + o] = w[q];
-                        }
-                        __nv_bfloat162 lo2 = __halves2bfloat162(w[0], w[1]), hi2 = __halves2bfloat162(w[2], w[3]);
-                        *reinterpret_cast<uint2*>(c.wt + (size_t)o * c.ld_wt + 4 * r4) =
-                            make_uint2(*reinterpret_cast<uint32_t*>(&lo2), *reinterpret_cast<uint32_t*>(&hi2));
-                        if (c.wt_lo) {
-                            __nv_bfloat162 l0 = __floats2bfloat162_rn(p[0] - __bfloat162float(w[0]), p[1] - __bfloat162float(w[1]));
-                            __nv_bfloat162 l1 = __floats2bfloat162_rn(p[2] - __bfloat162float(w[2]), p[3] - __bfloat162float(w[3]));
-                            *reinterpret_cast<uint2*>(c.wt_lo + (size_t)o * c.ld_wt + 4 * r4) =
-                                make_uint2(*reinterpret_cast<uint32_t*>(&l0), *reinterpret_cast<uint32_t*>(&l1));
-                        }
-                    }
-                    continue;
-                }
-            }
-        }
-        const float4 g4 = reinterpret_cast<const float4*>(a.grad)[i];
-        float4 p4 = reinterpret_cast<float4*>(a.param)[i];
-        float4 m4 = reinterpret_cast<float4*>(a.m)[i];
-        float4 v4 = reinterpret_cast<float4*>(a.v)[i];
-        float g[4] = {g4.x, g4.y, g4.z, g4.w};
-        float p[4] = {p4.x, p4.y, p4.z, p4.w};
-        float m[4] = {m4.x, m4.y, m4.z, m4.w};
-        float v[4] = {v4.x, v4.y, v4.z, v4.w};
+    while (i < n4) {
+        float* g = G.g; float* p = G.p; float* m = G.m; float* v = G.v;
 #pragma unroll
         for (int q = 0; q < 4; ++q) {
             const float gc = g[q] * coef;
@@ -756,35 +738,64 @@ __global__ void __launch_bounds__(kAdamThreads) adam_kernel(const AdamArgs a) {
             v[q] = a.b2 * v[q] + (1.0f - a.b2) * gc * gc;
             p[q] = p[q] - lr * (m[q] * c1) / (sqrtf(v[q] * c2) + a.eps);
         }
-        reinterpret_cast<float4*>(a.param)[i] = make_float4(p[0], p[1], p[2], p[3]);
-        reinterpret_cast<float4*>(a.m)[i] = make_float4(m[0], m[1], m[2], m[3]);
-        reinterpret_cast<float4*>(a.v)[i] = make_float4(v[0], v[1], v[2], v[3]);
-        // BF16 mode: refresh the operand copies of the hidden-layer weights and biases in place.
-        // A group of four parameters lies in one row of one layer (rows are padded to 4).
-        const int idx = 4 * i;
-        for (int e = 0; e < a.n_cvt; ++e) {
-            const CvtRange& c = a.cvt[e];
-            if (idx >= c.w_off && idx < c.w_off + c.in * c.out_p) {
-                const int rel = idx - c.w_off, row = rel / c.out_p, o = rel - row * c.out_p;
+        if (G.rows) {
+            const CvtRange& c = a.cvt[G.e];
+            const int r4 = G.r4, o = G.o;
+#pragma unroll
+            for (int q = 0; q < 4; ++q) {
+                const size_t at = G.base + (size_t)q * c.out_p;
+                a.param[at] = p[q]; a.m[at] = m[q]; a.v[at] = v[q];
+            }
+            if (o < c.out) {
+                __nv_bfloat16 w[4];
 #pragma unroll
                 for (int q = 0; q < 4; ++q) {
-                    if (o + q < c.out) {
-                        const __nv_bfloat16 w = __float2bfloat16_rn(p[q]);
-                        c.wt[(size_t)(o + q) * c.ld_wt + row] = w;
-                        if (c.wn) c.wn[(size_t)row * c.ld_wn + o + q] = w;
-                        if (c.wt_lo) c.wt_lo[(size_t)(o + q) * c.ld_wt + row] = __float2bfloat16_rn(p[q] - __bfloat162float(w));
-                    }
+                    w[q] = __float2bfloat16_rn(p[q]);
+                    if (c.wn) c.wn[(size_t)(4 * r4 + q) * c.ld_wn + o] = w[q];
                 }
-                break;
+                __nv_bfloat162 lo2 = __halves2bfloat162(w[0], w[1]), hi2 = __halves2bfloat162(w[2], w[3]);
+                *reinterpret_cast<uint2*>(c.wt + (size_t)o * c.ld_wt + 4 * r4) =
+                    make_uint2(*reinterpret_cast<uint32_t*>(&lo2), *reinterpret_cast<uint32_t*>(&hi2));
+                if (c.wt_lo) {
+                    __nv_bfloat162 l0 = __floats2bfloat162_rn(p[0] - __bfloat162float(w[0]), p[1] - __bfloat162float(w[1]));
+                    __nv_bfloat162 l1 = __floats2bfloat162_rn(p[2] - __bfloat162float(w[2]), p[3] - __bfloat162float(w[3]));
+                    *reinterpret_cast<uint2*>(c.wt_lo + (size_t)o * c.ld_wt + 4 * r4) =
+                        make_uint2(*reinterpret_cast<uint32_t*>(&l0), *reinterpret_cast<uint32_t*>(&l1));
+                }
             }
-            if (idx >= c.b_off && idx < c.b_off + c.out_p) {
-                const int o = idx - c.b_off;
+        } else {
+            reinterpret_cast<float4*>(a.param)[i] = make_float4(p[0], p[1], p[2], p[3]);
+            reinterpret_cast<float4*>(a.m)[i] = make_float4(m[0], m[1], m[2], m[3]);
+            reinterpret_cast<float4*>(a.v)[i] = make_float4(v[0], v[1], v[2], v[3]);
+            // BF16 mode: refresh the operand copies of the hidden-layer weights and biases in place.
+            // A group of four parameters lies in one row of one layer (rows are padded to 4).
+            const int idx = 4 * i;
+            for (int e = 0; e < a.n_cvt; ++e) {
+                const CvtRange& c = a.cvt[e];
+                if (idx >= c.w_off && idx < c.w_off + c.in * c.out_p) {
+                    const int rel = idx - c.w_off, row = rel / c.out_p, o = rel - row * c.out_p;
 #pragma unroll
-                for (int q = 0; q < 4; ++q)
-                    if (o + q < c.out) c.bias_pad[o + q] = p[q];
-                break;
+                    for (int q = 0; q < 4; ++q) {
+                        if (o + q < c.out) {
+                            const __nv_bfloat16 w = __float2bfloat16_rn(p[q]);
+                            c.wt[(size_t)(o + q) * c.ld_wt + row] = w;
+                            if (c.wn) c.wn[(size_t)row * c.ld_wn + o + q] = w;
+                            if (c.wt_lo) c.wt_lo[(size_t)(o + q) * c.ld_wt + row] = __float2bfloat16_rn(p[q] - __bfloat162float(w));
+                        }
+                    }
+                    break;
+                }
+                if (idx >= c.b_off && idx < c.b_off + c.out_p) {
+                    const int o = idx - c.b_off;
+#pragma unroll
+                    for (int q = 0; q < 4; ++q)
+                        if (o + q < c.out) c.bias_pad[o + q] = p[q];
+                    break;
+                }
             }
         }
+        i += gridDim.x * kAdamThreads;
+        if (i < n4) fetch(i, G);
     }
 }
 
