@@ -250,8 +250,8 @@ rslrl_status backward_fp32(rslrl_ctx* c) {
     const float* dhead[2] = {c->dmu, c->dv};
     const int ldhead[2] = {c->lddmu, 4};
     const int R = c->R;
-    // head weight gradients: dW = H_last^T d_head
-    {
+    // head weight gradients: dW = H_last^T d_head (TF32 mode: with the other layers in the tensor-core launch below)
+    if (!c->tf32) {
         GemmBatch b{};
         for (int ni = 0; ni < 2; ++ni) {
             const Net& n = *nets[ni];
@@ -279,11 +279,13 @@ rslrl_status backward_fp32(rslrl_ctx* c) {
             const float* dz = (const float*)c->up_dz[ni][l];
             const float* hin = l == 0 ? x[ni] : (const float*)c->up_h[ni][l - 1];
             const int ldin = l == 0 ? n.in_ld : n.hid_ld[l - 1];
-            GemmProblem& p = wg.p[wg.count++];
-            p.A = hin; p.lda = ldin; p.B = dz; p.ldb = n.hid_ld[l];
-            p.C = c->partials + L.w_off; p.ldc = L.out_p;
-            p.M = L.in; p.N = L.out; p.K = R; p.Cn = L.out_p;
-            p.splits = c->splits; p.kchunk = c->kchunk; p.split_stride = c->P_dev;
+            if (!c->tf32) {                         // TF32 mode: one tensor-core launch for all layers, below
+                GemmProblem& p = wg.p[wg.count++];
+                p.A = hin; p.lda = ldin; p.B = dz; p.ldb = n.hid_ld[l];
+                p.C = c->partials + L.w_off; p.ldc = L.out_p;
+                p.M = L.in; p.N = L.out; p.K = R; p.Cn = L.out_p;
+                p.splits = c->splits; p.kchunk = c->kchunk; p.split_stride = c->P_dev;
+            }
             ColsumProblem& q = cs.p[cs.count++];
             q.X = dz; q.out = c->partials + L.b_off; q.rows = R; q.n = L.out; q.ld = n.hid_ld[l];
             if (l > 0) {
@@ -303,6 +305,7 @@ rslrl_status backward_fp32(rslrl_ctx* c) {
             else CU(c, launch_sgemm(dg, false, true, EPI_DELU, c->stream));
         }
     }
+    if (c->tf32) CU(c, tf32_update_wgrad(c->tf32));
     return RSLRL_OK;
 }
 
@@ -421,7 +424,8 @@ rslrl_status rslrl_create(const rslrl_model_cfg* m, const rslrl_ppo_cfg* p, void
         UmmaSetup probe{}; fill_setup(c, probe);
         c->splits = umma_wgrad_plan(probe).max_splits;
     }
-    c->kchunk = round_up((c->R + c->splits - 1) / c->splits, 8);
+    // rows per split: a multiple of the k-step of whichever kernel forms the weight gradients
+    c->kchunk = round_up((c->R + c->splits - 1) / c->splits, c->prec == RSLRL_TF32 ? 32 : 8);
     c->lddmu = as;
     for (int b = 0; b < 2; ++b) {
         A_(c->act_mb[b], (size_t)c->R * as); A_(c->mu_old[b], (size_t)c->Bmb * as); A_(c->sigma_old[b], (size_t)c->Bmb * as);
@@ -464,6 +468,8 @@ rslrl_status rslrl_create(const rslrl_model_cfg* m, const rslrl_ppo_cfg* p, void
             ts.obs_storage[1] = c->st.obs_critic; ts.obs_stride[1] = sc;
             ts.last_obs_c = c->last_obs_c;
             ts.x[0] = c->x_a; ts.x[1] = m->shared_obs ? c->x_a : c->x_c;
+            ts.dhead[0] = c->dmu; ts.ld_dhead[0] = c->lddmu; ts.dhead[1] = c->dv; ts.ld_dhead[1] = 4;
+            ts.partials = c->partials; ts.split_stride = c->P_dev; ts.splits = c->splits; ts.kchunk = c->kchunk;
             std::string terr;
             c->tf32 = tf32_create(ts, &terr);
             if (!c->tf32) { c->err = "tensor-core engine: " + terr; return bail(RSLRL_ERR_UNSUPPORTED); }

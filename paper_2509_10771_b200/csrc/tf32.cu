@@ -275,6 +275,229 @@ __global__ void __launch_bounds__(kThreads, 1) tf32_gemm_kernel(const __grid_con
     }
 }
 
+// ------------------------------------------------------------------ weight gradient
+// dW[features_in x features_out] = X^T dZ over the minibatch rows, both operands as stored ([row][feature], the
+// contraction index outermost: MN-major tiles of 32 features x 32 rows, one 128-byte row per minibatch row, swizzled
+// in units of 32 bytes, the form the tensor cores take for MN-major operands of 32-bit elements).
+// A work item is a 128 x (<= 128) tile of one layer over one split of the row range; its FP32 result is a partial
+// that the gradient reduction sums.  A split without rows (the row range does not always fill the last one) writes
+// zeros.
+constexpr int kTfWgProblems = 2 * kMaxLayers;     // every layer of both nets
+constexpr int kTfWgStages = 4;
+constexpr uint32_t kTfWgBox = 32 * 32 * 4;        // 4 KiB: 32 features x 32 rows
+constexpr uint32_t kTfWgStageA = 4 * kTfWgBox;    // 128 features
+constexpr uint32_t kTfWgStageB = 4 * kTfWgBox;    // up to 128 features
+constexpr size_t kTfWgSmem = 1024 + (size_t)kTfWgStages * (kTfWgStageA + kTfWgStageB) + 512;
+
+struct TfWgProblem {
+    int m_extent, n_store;         // input features; output columns that are written (the padded width of the layer)
+    int m_tiles, n_tiles, bn;
+    int kblocks, kb_per_split, splits;
+    int item_begin;
+    float* out; int ld_out;        // partial of split 0: [m_extent][ld_out]
+    long long split_stride;
+};
+struct TfWgParams {
+    CUtensorMap tmA[kTfWgProblems], tmB[kTfWgProblems];   // [rows][features], boxes of 32 features x 32 rows
+    TfWgProblem p[kTfWgProblems];
+    int count, total_items;
+    int* error;
+};
+struct TfWgItem { int prob, m0, n0, kb0, kb1, split; };
+__device__ __forceinline__ TfWgItem tf_wg_decode(const TfWgParams& P, int item) {
+    int pi = 0;
+#pragma unroll 1
+    for (int i = 1; i < P.count; ++i)
+        if (item >= P.p[i].item_begin) pi = i;
+    const TfWgProblem& p = P.p[pi];
+    const int local = item - p.item_begin;
+    const int per_split = p.m_tiles * p.n_tiles;
+    TfWgItem it;
+    it.prob = pi;
+    it.split = local / per_split;
+    const int rem = local - it.split * per_split;
+    it.m0 = (rem / p.n_tiles) * BLOCK_M;
+    it.n0 = (rem % p.n_tiles) * p.bn;
+    it.kb0 = min(p.kblocks, it.split * p.kb_per_split);
+    it.kb1 = min(p.kblocks, it.kb0 + p.kb_per_split);
+    return it;
+}
+
+// Shared-memory descriptor of an MN-major operand of 32-bit elements: 128-byte swizzle in units of 32 bytes (the
+// tensor maps' CU_TENSOR_MAP_SWIZZLE_128B_ATOM_32B), whose pattern repeats every four rows of 128 bytes.
+__device__ __forceinline__ uint64_t smem_desc_mn32(uint32_t addr, uint32_t lead_bytes, uint32_t stride_bytes) {
+    uint64_t d = 0;
+    d |= (uint64_t)((addr >> 4) & 0x3FFFu);
+    d |= (uint64_t)((lead_bytes >> 4) & 0x3FFFu) << 16;
+    d |= (uint64_t)((stride_bytes >> 4) & 0x3FFFu) << 32;
+    d |= 1ull << 46;                 // descriptor version of this architecture
+    d |= 1ull << 61;                 // 128-byte swizzle with 32-byte units
+    return d;
+}
+
+// Instruction descriptor: TF32 x TF32 -> FP32, both operands MN-major, M = 128, N = bn.
+__device__ __forceinline__ uint32_t instr_desc_tf32_mn(int bn) {
+    return (1u << 4) | (2u << 7) | (2u << 10) | (1u << 15) | (1u << 16) | ((uint32_t)(bn >> 3) << 17) |
+           ((uint32_t)(BLOCK_M >> 4) << 24);
+}
+
+__global__ void __launch_bounds__(kThreads, 1) tf32_wgrad_kernel(const __grid_constant__ TfWgParams P) {
+    extern __shared__ uint8_t smem_raw[];
+    uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
+    uint8_t* sA = smem;
+    uint8_t* sB = smem + kTfWgStages * kTfWgStageA;
+    uint64_t* full = reinterpret_cast<uint64_t*>(sB + kTfWgStages * kTfWgStageB);
+    uint64_t* empty = full + kTfWgStages;
+    uint64_t* tfull = empty + kTfWgStages;
+    uint64_t* tempty = tfull + 2;
+    uint64_t* drain = tempty + 2;
+    uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(drain + 1);
+    volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
+
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    if (threadIdx.x == 0) {
+        for (int s = 0; s < kTfWgStages; ++s) { mbar_init(&full[s], 1); mbar_init(&empty[s], 1); }
+        for (int b = 0; b < 2; ++b) { mbar_init(&tfull[b], 1); mbar_init(&tempty[b], kEpiWarps); }
+        mbar_init(drain, 1);
+        *abort_flag = 0;
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+        asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+    }
+    if (warp == 1) tmem_alloc(tmem_slot, kTmemCols);
+    if (warp == 0 && lane == 0)
+        for (int i = 0; i < P.count; ++i) { tma_prefetch_desc(&P.tmA[i]); tma_prefetch_desc(&P.tmB[i]); }
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    const uint32_t tmem_base = *tmem_slot;
+    chain_wait();
+
+    if (warp == 0) {
+        // ================================ TMA producer =================================
+        // a k-block is up to eight boxes of 32 features x 32 rows (four of A, up to four of B): lane l issues box l
+        int stage = 0; uint32_t phase = 0;
+        uint32_t issued_mask = 0, issued_parity = 0;
+        bool ok = true;
+        for (int item = blockIdx.x; ok && item < P.total_items; item += gridDim.x) {
+            const TfWgItem it = tf_wg_decode(P, item);
+            const TfWgProblem& p = P.p[it.prob];
+            const uint32_t bytes = kTfWgStageA + (uint32_t)(p.bn / 32) * kTfWgBox;
+            const bool mine = lane < 4 + p.bn / 32;
+            const CUtensorMap* tm = lane < 4 ? &P.tmA[it.prob] : &P.tmB[it.prob];
+            const int x = lane < 4 ? it.m0 + 32 * lane : it.n0 + 32 * (lane - 4);
+            uint8_t* base = lane < 4 ? sA + (uint32_t)lane * kTfWgBox : sB + (uint32_t)(lane - 4) * kTfWgBox;
+            const uint32_t per_stage = lane < 4 ? kTfWgStageA : kTfWgStageB;
+            for (int kb = it.kb0; kb < it.kb1; ++kb) {
+                int good = 1;
+                if (lane == 0) {
+                    good = mbar_wait(&empty[stage], phase ^ 1u, abort_flag, P.error, 21) ? 1 : 0;
+                    if (good) mbar_expect_tx(&full[stage], bytes);
+                }
+                good = __shfl_sync(0xffffffffu, good, 0);
+                if (!good) { ok = false; break; }
+                if (mine) tma_load_2d(base + (uint32_t)stage * per_stage, tm, x, kb * kTfBlockK, &full[stage]);
+                issued_mask |= 1u << stage;
+                issued_parity = (issued_parity & ~(1u << stage)) | (phase << stage);
+                if (++stage == kTfWgStages) { stage = 0; phase ^= 1u; }
+            }
+        }
+        if (!ok && lane == 0) {
+            // let the copies already issued land before the CTA's shared memory goes away
+            for (int s = 0; s < kTfWgStages; ++s) {
+                if (!(issued_mask & (1u << s))) continue;
+                const unsigned long long t0 = global_ns();
+                while (!mbar_try_wait(&full[s], (issued_parity >> s) & 1u) && global_ns() - t0 < kWaitLimitNs) {}
+            }
+        }
+    } else if (warp == 1) {
+        // ================================ MMA issuer ===================================
+        if (lane == 0) {
+            int stage = 0; uint32_t phase = 0;
+            bool ok = true;
+            int local = 0;
+            // MN-major operands: 4096 bytes between blocks of 32 features, 512 between groups of four rows (one
+            // period of the swizzle); a k-step is eight rows (1024 bytes); descriptors differ only in their address
+            // field (16-byte units)
+            const uint64_t a_desc0 = smem_desc_mn32(smem_u32(sA), kTfWgBox, 512);
+            const uint64_t b_desc0 = smem_desc_mn32(smem_u32(sB), kTfWgBox, 512);
+            constexpr uint32_t kstep = 1024 >> 4;
+            for (int item = blockIdx.x; ok && item < P.total_items; item += gridDim.x, ++local) {
+                const TfWgItem it = tf_wg_decode(P, item);
+                const TfWgProblem& p = P.p[it.prob];
+                const int buf = local & 1;
+                const uint32_t use = (uint32_t)(local >> 1);
+                if (!mbar_wait(&tempty[buf], (use & 1u) ^ 1u, abort_flag, P.error, 22)) { ok = false; break; }
+                tc_fence_after();
+                const uint32_t d_tmem = tmem_base + (uint32_t)buf * kMaxBN;
+                const uint32_t idesc = instr_desc_tf32_mn(p.bn);
+                for (int kb = it.kb0; kb < it.kb1; ++kb) {
+                    if (!mbar_wait(&full[stage], phase, abort_flag, P.error, 23)) { ok = false; break; }
+                    tc_fence_after();
+                    const uint64_t da = a_desc0 + (uint64_t)((uint32_t)stage * (kTfWgStageA >> 4));
+                    const uint64_t db = b_desc0 + (uint64_t)((uint32_t)stage * (kTfWgStageB >> 4));
+                    umma_tf32(d_tmem, da, db, idesc, kb > it.kb0 ? 1u : 0u);
+                    umma_tf32(d_tmem, da + kstep, db + kstep, idesc, 1u);
+                    umma_tf32(d_tmem, da + 2 * kstep, db + 2 * kstep, idesc, 1u);
+                    umma_tf32(d_tmem, da + 3 * kstep, db + 3 * kstep, idesc, 1u);
+                    umma_commit(&empty[stage]);       // frees the stage once these MMAs have read it
+                    if (++stage == kTfWgStages) { stage = 0; phase ^= 1u; }
+                }
+                if (ok) umma_commit(&tfull[buf]);     // accumulator complete (at once for a split without rows)
+            }
+            chain_release();
+            if (!ok) {
+                umma_commit(drain);
+                const unsigned long long t0 = global_ns();
+                while (!mbar_try_wait(drain, 0) && global_ns() - t0 < kWaitLimitNs) {}
+            }
+        }
+    } else {
+        // ================================ epilogue =====================================
+        const int q = warp & 3;                    // accumulator lanes 32q .. 32q+31
+        const int group = (warp - 2) >> 2;         // columns [32 group, 32 group + 32) of the tile
+        bool ok = true;
+        int local = 0;
+        for (int item = blockIdx.x; ok && item < P.total_items; item += gridDim.x, ++local) {
+            const TfWgItem it = tf_wg_decode(P, item);
+            const TfWgProblem& p = P.p[it.prob];
+            const int buf = local & 1;
+            const uint32_t use = (uint32_t)(local >> 1);
+            const int row = it.m0 + 32 * q + lane;
+            const int col = it.n0 + 32 * group;
+            const bool active = 32 * group < p.bn && col < p.n_store;   // uniform across the warp
+            if (!mbar_wait(&tfull[buf], use & 1u, abort_flag, P.error, 24)) { ok = false; break; }
+            tc_fence_after();
+            if (active) {
+                uint32_t acc[32];
+                tmem_ld32(tmem_base + ((uint32_t)(32 * q) << 16) + (uint32_t)(buf * kMaxBN + 32 * group), acc);
+                if (it.kb0 >= it.kb1) {
+#pragma unroll
+                    for (int i = 0; i < 32; ++i) acc[i] = 0u;             // nothing was accumulated
+                }
+                if (row < p.m_extent) {
+                    float* dst = p.out + (size_t)it.split * p.split_stride + (size_t)row * p.ld_out + col;
+#pragma unroll
+                    for (int g = 0; g < 8; ++g)
+                        if (col + 4 * g < p.n_store)
+                            *reinterpret_cast<float4*>(dst + 4 * g) =
+                                make_float4(__uint_as_float(acc[4 * g]), __uint_as_float(acc[4 * g + 1]),
+                                            __uint_as_float(acc[4 * g + 2]), __uint_as_float(acc[4 * g + 3]));
+                }
+            }
+            // the accumulator has been read: hand the tensor-memory buffer back
+            tc_fence_before();
+            __syncwarp();
+            if (lane == 0) mbar_arrive(&tempty[buf]);
+        }
+    }
+    tc_fence_before();
+    __syncthreads();
+    if (warp == 1) {
+        tc_fence_after();
+        tmem_dealloc(tmem_base, kTmemCols);
+    }
+}
+
 // Transposed copies of the hidden-layer weights: W[in][ld_src] -> Wt[out][ld_dst].
 struct TransposeEntry { const float* src; float* dst; int in, out, ld_src, ld_dst; };
 
@@ -297,7 +520,8 @@ __global__ void tf32_transpose_kernel(const TransposeEntry* __restrict__ table) 
 inline int round_up(int x, int m) { return (x + m - 1) / m * m; }
 
 // 2-D FP32 tensor [rows][cols] with row stride ld (floats); box = box_cols x box_rows, 128-byte swizzle.
-bool make_tmap_f32(CUtensorMap* tm, const void* base, long long rows, int cols, int ld, int box_cols, int box_rows) {
+bool make_tmap_f32(CUtensorMap* tm, const void* base, long long rows, int cols, int ld, int box_cols, int box_rows,
+                   CUtensorMapSwizzle swizzle = CU_TENSOR_MAP_SWIZZLE_128B) {
     EncodeTiledFn fn = get_encode_fn();
     if (!fn) return false;
     const cuuint64_t dims[2] = {(cuuint64_t)cols, (cuuint64_t)rows};
@@ -305,7 +529,7 @@ bool make_tmap_f32(CUtensorMap* tm, const void* base, long long rows, int cols, 
     const cuuint32_t box[2] = {(cuuint32_t)box_cols, (cuuint32_t)box_rows};
     const cuuint32_t estr[2] = {1, 1};
     return fn(tm, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 2, const_cast<void*>(base), dims, strides, box, estr,
-              CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+              CU_TENSOR_MAP_INTERLEAVE_NONE, swizzle, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
               CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
@@ -321,6 +545,7 @@ struct Tf32Engine {
     int* error_dev = nullptr;
     int num_sms = 148;
     std::vector<TfParams> act_fwd, last_fwd, upd_fwd, upd_dgrad;   // one launch per hidden layer index / backward step
+    TfWgParams upd_wgrad;                                          // one launch for every layer of both nets
 };
 
 namespace {
@@ -379,7 +604,8 @@ Tf32Engine* tf32_create(const Tf32Setup& s, std::string* err) {
     if (cudaGetDevice(&dev) != cudaSuccess || cudaGetDeviceProperties(&prop, dev) != cudaSuccess) return failmsg("no CUDA device");
     if (prop.major != 10) return failmsg("the tensor-core mode needs an sm_100 device");
     if (cudaFuncSetAttribute(tf32_gemm_kernel<TF_FWD>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kTfSmem) != cudaSuccess ||
-        cudaFuncSetAttribute(tf32_gemm_kernel<TF_DGRAD>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kTfSmem) != cudaSuccess)
+        cudaFuncSetAttribute(tf32_gemm_kernel<TF_DGRAD>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kTfSmem) != cudaSuccess ||
+        cudaFuncSetAttribute(tf32_wgrad_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kTfWgSmem) != cudaSuccess)
         return failmsg("could not reserve shared memory for the tensor-core kernels");
     Tf32Engine* e = new Tf32Engine();
     e->s = s;
@@ -440,6 +666,38 @@ Tf32Engine* tf32_create(const Tf32Setup& s, std::string* err) {
         finish(P, s.elu_alpha, e->error_dev);
         e->upd_dgrad.push_back(P);
     }
+    // weight gradients: dW[l] = hin[l]^T dZ[l] over the rows of each split (the heads' dZ is dL/d(head output))
+    {
+        TfWgParams& W = e->upd_wgrad;
+        memset(&W, 0, sizeof W);
+        if (s.kchunk % kTfBlockK != 0 || s.splits < 1) return bail("rows per weight-gradient split must be a multiple of 32");
+        int items = 0;
+        for (int ni = 0; ni < 2; ++ni)
+            for (int l = 0; l < s.nl[ni]; ++l) {
+                if (W.count == kTfWgProblems) return bail("too many layers for the weight-gradient launch");
+                const int i = W.count;
+                TfWgProblem& p = W.p[i];
+                const bool head = l == e->nh[ni];
+                const float* hin = l == 0 ? s.x[ni] : s.up_h[ni][l - 1];
+                const int ldin = l == 0 ? s.in_ld[ni] : s.hid_ld[ni][l - 1];
+                const float* dz = head ? s.dhead[ni] : s.up_dz[ni][l];
+                const int lddz = head ? s.ld_dhead[ni] : s.hid_ld[ni][l];
+                p.m_extent = s.in[ni][l]; p.n_store = s.out_p[ni][l];
+                p.bn = std::min(kTfMaxBN, round_up(s.out[ni][l], 32));
+                p.m_tiles = (p.m_extent + BLOCK_M - 1) / BLOCK_M;
+                p.n_tiles = (p.n_store + p.bn - 1) / p.bn;
+                p.kblocks = (s.R + kTfBlockK - 1) / kTfBlockK;
+                p.kb_per_split = s.kchunk / kTfBlockK;
+                p.splits = s.splits;
+                p.item_begin = items; items += p.m_tiles * p.n_tiles * p.splits;
+                p.out = s.partials + s.w_off[ni][l]; p.ld_out = s.out_p[ni][l]; p.split_stride = s.split_stride;
+                if (!make_tmap_f32(&W.tmA[i], hin, s.R, s.in[ni][l], ldin, 32, 32, CU_TENSOR_MAP_SWIZZLE_128B_ATOM_32B) ||
+                    !make_tmap_f32(&W.tmB[i], dz, s.R, s.out[ni][l], lddz, 32, 32, CU_TENSOR_MAP_SWIZZLE_128B_ATOM_32B))
+                    return bail("tensor map encoding failed");
+                W.count++;
+            }
+        W.total_items = items; W.error = e->error_dev;
+    }
     if (cudaStreamSynchronize(s.stream) != cudaSuccess) return bail("stream synchronisation failed");
     return e;
 }
@@ -482,6 +740,13 @@ cudaError_t tf32_update_forward(Tf32Engine* e) {
 cudaError_t tf32_update_dgrad(Tf32Engine* e, int back) {
     if (back < 0 || back >= (int)e->upd_dgrad.size()) return cudaSuccess;
     return launch_tf<TF_DGRAD>(e->upd_dgrad[back], e->num_sms, e->s.stream);
+}
+
+cudaError_t tf32_update_wgrad(Tf32Engine* e) {
+    const TfWgParams& W = e->upd_wgrad;
+    if (W.total_items == 0) return cudaSuccess;
+    LaunchScope scope_("tc_gemm_wgrad", e->s.stream);
+    return launch_chained(tf32_wgrad_kernel, std::min(W.total_items, e->num_sms), kThreads, kTfWgSmem, e->s.stream, W);
 }
 
 cudaError_t tf32_read_error(Tf32Engine* e, int* host_code) {

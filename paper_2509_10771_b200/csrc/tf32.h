@@ -1,7 +1,8 @@
 // Tensor-core engine of the RSLRL_TF32 mode: the hidden-layer products of act, forward and data
 // gradient as tcgen05 kind::tf32 GEMMs on the FP32 buffers of the FP32 mode (operands are read as
 // FP32 and used with TF32 precision by the tensor cores; accumulation, bias, ELU and everything
-// else stay FP32).  Weight gradients, heads, loss and optimiser are the FP32 mode's kernels.
+// else stay FP32), and the weight gradients of all layers likewise.  Head products, bias gradients, loss and
+// optimiser are the FP32 mode's kernels.
 #pragma once
 #include "../../include/rslrl_b200.h"
 #include "common.cuh"
@@ -24,6 +25,9 @@ struct Tf32Setup {
     float* act_h[2][kMaxLayers];                      // post-activations of act [N][hid_ld]
     float* up_h[2][kMaxLayers];                       // post-activations of the update [R][hid_ld]
     float* up_dz[2][kMaxLayers];                      // dL/dz of the update [R][hid_ld]
+    const float* dhead[2]; int ld_dhead[2];           // dL/d(head output) of the update [R][ld]: policy mean, value
+    float* partials; long long split_stride;          // weight-gradient partials [splits][split_stride], layer l at w_off
+    int splits, kchunk;                               // minibatch rows per split: a multiple of 32
 };
 
 struct Tf32Engine;
@@ -39,6 +43,8 @@ cudaError_t tf32_act_forward(Tf32Engine* e, int t, bool do_actor);
 cudaError_t tf32_update_forward(Tf32Engine* e);
 // dL/dz of hidden layer (top - back - 1) of every net that has one, from dL/dz of the layer above.
 cudaError_t tf32_update_dgrad(Tf32Engine* e, int back);
+// Weight-gradient partials of every layer of both nets, heads included (after the data gradients of the step).
+cudaError_t tf32_update_wgrad(Tf32Engine* e);
 // Synchronises the stream and returns the device error code (0 = none); a non-zero code is cleared once read.
 cudaError_t tf32_read_error(Tf32Engine* e, int* host_code);
 

@@ -192,10 +192,13 @@ def _first_step(case, precision, from_oracle_storage, check_rollout=False):
     if precision == FP32:
         assert_close(g, ref["grad"], tol, "grad")
     elif precision == TF32:
-        # forward and data gradient saw TF32 operands (11 significant bits), the weight gradients FP32 ones
+        # every product of the step saw TF32 operands (11 significant bits): each term of a weight-gradient sum
+        # carries two operand roundings of 2^-11, and the sum over the minibatch rows cancels (the advantages have
+        # mean zero), so the error relative to the result is a few times that of a term: element by element at
+        # twice the mode's tolerance per block, the whole gradient in relative L2 at the mode's tolerance itself
         for name, off, n in blocks:
             assert_close(g[off:off + n], ref["grad"][off:off + n], 1e-2, f"grad {name}")
-        assert rel_l2(g, ref["grad"]) < 2e-3
+        assert rel_l2(g, ref["grad"]) < tol
     else:
         # every parameter block on its own, so a wrong layer cannot hide behind a large one: element by element
         # (a BF16-rounded operand perturbs every product of a three-layer chain: 5e-2 of |y| + rms of the block;
@@ -224,7 +227,7 @@ def _first_step(case, precision, from_oracle_storage, check_rollout=False):
         assert_close(m, state.m, tol, "adam_m")
         assert_close(v, state.v, 2 * tol, "adam_v")
     else:
-        assert rel_l2(m, state.m) < (2e-3 if precision == TF32 else 1e-2)
+        assert rel_l2(m, state.m) < (tol if precision == TF32 else 1e-2)
     c = ctx.get_counters()
     assert c.adam_step == 1 and c.iteration == 1
     ctx.destroy()
