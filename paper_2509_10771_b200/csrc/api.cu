@@ -266,11 +266,11 @@ rslrl_status backward_fp32(rslrl_ctx* c) {
         CU(c, launch_sgemm(b, true, false, EPI_PLAIN, c->stream));
     }
     const int maxh = std::max(c->actor.nl - 1, c->critic.nl - 1);
+    ColsumBatch cs{};                              // bias gradients of every hidden layer: one launch after the loop
+    cs.splits = c->splits; cs.split_stride = c->P_dev; cs.is_bf16 = 0;
     for (int back = 0; back < maxh; ++back) {
         GemmBatch wg{}, dg{};
-        ColsumBatch cs{};
         dg.alpha = c->mc.elu_alpha;
-        cs.splits = c->splits; cs.split_stride = c->P_dev; cs.is_bf16 = 0;
         for (int ni = 0; ni < 2; ++ni) {
             const Net& n = *nets[ni];
             const int l = n.nl - 2 - back;         // hidden layer index, from the top
@@ -299,12 +299,12 @@ rslrl_status backward_fp32(rslrl_ctx* c) {
             }
         }
         if (wg.count) CU(c, launch_sgemm(wg, true, false, EPI_PLAIN, c->stream));
-        if (cs.count) CU(c, launch_colsum(cs, c->stream));
         if (dg.count) {
             if (c->tf32) CU(c, tf32_update_dgrad(c->tf32, back));
             else CU(c, launch_sgemm(dg, false, true, EPI_DELU, c->stream));
         }
     }
+    if (cs.count) CU(c, launch_colsum(cs, c->stream));
     if (c->tf32) CU(c, tf32_update_wgrad(c->tf32));
     return RSLRL_OK;
 }
