@@ -732,7 +732,10 @@ static rslrl_status update_impl(rslrl_ctx* c, int32_t max_steps, rslrl_update_st
                     TRY(enqueue_gather(done_steps + 1, buf ^ 1, c->side));
                     CU(c, cudaEventRecord(c->ev_gathered[buf ^ 1], c->side));
                 }
-                CU(c, cudaStreamWaitEvent(c->stream, c->ev_gathered[buf], 0));
+                // the step's own input set: waited for here only at the first step; later steps wait right behind
+                // the backward pass of the step before (below), so that a step's launches follow one another
+                // without a stream operation in between
+                if (done_steps == 0) CU(c, cudaStreamWaitEvent(c->stream, c->ev_gathered[buf], 0));
             } else {
                 TRY(enqueue_gather(done_steps, 0, c->stream));
             }
@@ -764,7 +767,10 @@ static rslrl_status update_impl(rslrl_ctx* c, int32_t max_steps, rslrl_update_st
             // ---- backward ---------------------------------------------------------------
             if (c->prec != RSLRL_BF16) TRY(backward_fp32(c));
             else CU(c, umma_update_backward(c->umma, hl.colsum_written != 0, buf, distill));
-            if (overlap) CU(c, cudaEventRecord(c->ev_consumed[buf], c->stream));   // this input set may be refilled
+            if (overlap) {
+                CU(c, cudaEventRecord(c->ev_consumed[buf], c->stream));   // this input set may be refilled
+                if (done_steps + 1 < nsteps) CU(c, cudaStreamWaitEvent(c->stream, c->ev_gathered[buf ^ 1], 0));   // the next step's inputs
+            }
             // ---- reduce, clip, adaptive lr, Adam ------------------------------------------
             ReduceArgs r{};
             r.partials = c->partials; r.splits = c->splits; r.split_stride = c->P_dev;

@@ -275,7 +275,8 @@ __global__ void __launch_bounds__(kThreads, 1) wgrad_gemm_kernel(const __grid_co
 constexpr int kWsMaxStages = 8;
 constexpr uint32_t kWsStageOut = 32 * 32 * 2;
 constexpr uint32_t kWsBarBytes = 512;
-constexpr uint32_t kWsSmem = 232448;                                // the 227 KiB a CTA may have
+constexpr uint32_t kWsSmem = 231424;                                // 226 KiB: with the 1 KiB the system keeps per block, 1 KiB of
+                                                                    // the SM is left for a block without shared memory (the gather)
 constexpr uint32_t kWsAuxBox = 128 * 32 * 2;                         // 32 columns x 128 rows of stored post-activations
 constexpr uint32_t kWsAuxTile = 4 * kWsAuxBox;                       // a row tile of up to 128 columns
 // result tiles (one per epilogue warp) and, for the data gradient, two tiles of stored post-activations

@@ -40,7 +40,13 @@ __device__ __forceinline__ void store_obs_piece(float* dst, __nv_bfloat16* dst16
 // bandwidth of this kernel is the bytes it keeps in flight, so this loop carries nothing but the rows; the small
 // per-row items are gathered by a second loop with one thread per row.  Storage is read through the read-only path
 // (it does not change while an update runs).
-constexpr int kGatherRows = 8;
+// Two shapes of the kernel are launched.  The first gather of an update runs alone and is built for bandwidth:
+// eight rows per pass, 256 threads, two blocks per SM.  The others run on a second stream beside the tensor-core
+// kernels of the minibatch step before, whose CTAs hold an SM's shared memory and 55,296 of its 65,536
+// registers: two rows per pass, 128 threads and at most 80 registers make a block that fits beside such a CTA
+// (10,240 registers, no shared memory), so these gathers really run meanwhile instead of taking SMs in turn.
+constexpr int kGatherRowsAlone = 8;
+constexpr int kGatherRowsBeside = 2;
 
 struct MirrorTables { int pc[kObsVec][4]; float sg[kObsVec][4]; };   // of one column block, the same for every row
 
@@ -86,7 +92,8 @@ __device__ __forceinline__ void prefetch_row_l2(const float* row, uint32_t bytes
     asm volatile("cp.async.bulk.prefetch.L2.global [%0], %1;" ::"l"(row), "r"(bytes) : "memory");
 }
 
-__global__ void __launch_bounds__(256, 2) gather_kernel(const GatherArgs a) {
+template <int kGatherRows, int kBlockThreads, int kMinBlocks>
+__global__ void __launch_bounds__(kBlockThreads, kMinBlocks) gather_kernel(const GatherArgs a) {
     chain_begin();
     const int lane = threadIdx.x & 31;
     const int warps = (gridDim.x * blockDim.x) >> 5;
@@ -806,8 +813,12 @@ cudaError_t launch_gather(const GatherArgs& a, cudaStream_t s, bool alone) {
     // (accounting only) the first gather of an update runs while the caller's stream waits for it, the others beside
     // the kernels of the minibatch step before
     LaunchScope scope_(alone ? "gather_alone" : "gather", s);
-    const int blocks = std::min((a.Bmb + 8 * kGatherRows - 1) / (8 * kGatherRows), 148 * 2);     // one resident wave
-    return launch_chained(gather_kernel, blocks, 256, 0, s, a);
+    if (alone) {
+        const int blocks = std::min((a.Bmb + 8 * kGatherRowsAlone - 1) / (8 * kGatherRowsAlone), 148 * 2);   // one resident wave
+        return launch_chained(gather_kernel<kGatherRowsAlone, 256, 2>, blocks, 256, 0, s, a);
+    }
+    const int blocks = std::min((a.Bmb + 4 * kGatherRowsBeside - 1) / (4 * kGatherRowsBeside), 148 * 4);
+    return launch_chained(gather_kernel<kGatherRowsBeside, 128, 6>, blocks, 128, 0, s, a);
 }
 
 cudaError_t launch_perm_rows(uint64_t seed, uint32_t iteration, uint32_t epoch, uint32_t batch,
