@@ -99,8 +99,8 @@ NCU_TRAFFIC = {
     "source": "paper_2509_10771_b200/csrc/umma.cu",
     "begin": "// Weight gradient: D[features_in x features_out] = A^T B over the minibatch rows",
     "end": "// ------------------------------------------------------------------ fused forward chain",
-    "sha256": "3883d147aad4b94313c0aba63243bd4c37ca1666fdb6ae252240f64cd62b9c70",
-    "bytes_per_launch": {"tc_gemm_fwd": 31.2e6, "tc_gemm_dgrad": 67.2e6, "tc_gemm_wgrad": 203.3e6},
+    "sha256": "a7723f3fdc1eccda4f952e97d414ee14fdccc3c233978e074cd2a300bc7fdaeb",
+    "bytes_per_launch": {"tc_gemm_fwd": 31.6e6, "tc_gemm_dgrad": 67.8e6, "tc_gemm_wgrad": 203.4e6},
 }
 
 
