@@ -638,7 +638,8 @@ def run_gru(args):
     d_h = torch.empty((T, N, H), device=dev)
     d_dx = torch.empty((T, N, stride), device=dev)
     d_dh0 = torch.empty((N, H), device=dev)
-    gru = binding.Gru(D, H, T, N, stream=stream.cuda_stream)
+    tf32 = PRECISION == WL.PRECISION_TF32
+    gru = binding.Gru(D, H, T, N, stream=stream.cuda_stream, precision=WL.PRECISION_TF32 if tf32 else WL.PRECISION_FP32)
     gru.set_params(setup["params"])
     flush_buf = torch.empty(256 << 20, dtype=torch.uint8, device=dev)
 
@@ -679,10 +680,10 @@ def run_gru(args):
     line = {
         "metric": "recurrent layer forward + BPTT transitions/s", "value": T * N * args.steps / (ms * 1e-3), "unit": UNIT,
         "n_gpus": 1, "steps": args.steps, "warmup": max(args.warmup, 3), "ms_per_step": ms / args.steps,
-        "higher_is_better": True, "dtype": "f32", "data": "synthetic",
+        "higher_is_better": True, "dtype": "tf32" if tf32 else "f32", "data": "synthetic",
         "config": {"workload": w.name, "task": "gru", "num_envs": N, "num_steps": T, "input_dim": D, "hidden_dim": H,
                    "l2": "256 MiB buffer written between timed steps"},
-        "fp32_tflops": flops / (ms / args.steps * 1e-3) / 1e12,
+        ("tf32_tflops" if tf32 else "fp32_tflops"): flops / (ms / args.steps * 1e-3) / 1e12,
         "kernel_shares": shares,
         "cpu_baseline": {"value": T * ns / cpu_s, "unit": UNIT, "cores": blas_threads(), "kind": "oracle",
                          "sample": f"the oracle's forward and backward pass on {ns} of the {N} environments"},
@@ -764,7 +765,7 @@ def main():
     ap.add_argument("--workload", default=WORKLOAD.name, choices=sorted(WL.WORKLOADS),
                     help="which of the five synthetic workloads to time (default: the one the metric is quoted on)")
     ap.add_argument("--precision", default="bf16", choices=["bf16", "tf32"],
-                    help="operand precision of the hidden-layer products on the tensor cores (ppo task; default bf16)")
+                    help="operand precision of the products on the tensor cores (ppo task, default bf16; gru task: tf32 selects the tensor-core mode, anything else FP32)")
     ap.add_argument("--task", default="ppo", choices=["ppo", "distill", "rnd", "gru", "streams"],
                     help="ppo: the learn iteration the metric is quoted on (default); distill: the distillation iteration; "
                          "rnd: random network distillation over one rollout; gru: the recurrent layer over one rollout; "

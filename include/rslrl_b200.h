@@ -375,7 +375,10 @@ rslrl_status rslrl_rnd_update(rslrl_rnd *rnd, const float *d_obs, int32_t batch,
  *   n = tanh(x_t W_in + b_in + r * (h_in W_hn + b_hn)),  h(t) = (1 - z) n + z h_in
  * The paper names neither the cell nor the reset rule; these are this library's choices.
  * Parameters (host, float32): W_i[D][3H], b_i[3H], W_h[H][3H], b_h[3H], in this order.
- * All arithmetic is FP32.  The object owns parameters, gradient and work buffers sized for
+ * With precision RSLRL_FP32 all arithmetic is FP32.  With RSLRL_TF32 the matrix products (input and state
+ * products, their data gradients, the weight gradients) run on the tensor cores with TF32 operands read from
+ * the same FP32 buffers and FP32 accumulation; gates, biases' gradients and everything else stay FP32
+ * (tolerance class 5e-3 instead of 1e-4).  The object owns parameters, gradient and work buffers sized for
  * max_steps x max_envs; calls on one object are not thread-safe and enqueue on its stream. */
 typedef struct rslrl_gru rslrl_gru;
 
@@ -384,6 +387,7 @@ typedef struct {
     int32_t hidden_dim;                 /* H, a multiple of 4                                        */
     int32_t max_steps;                  /* largest T                                                 */
     int32_t max_envs;                   /* largest N; T * N < 2^30 and N * 3H < 2^31                 */
+    int32_t precision;                  /* RSLRL_FP32 or RSLRL_TF32 (RSLRL_BF16: RSLRL_ERR_UNSUPPORTED) */
 } rslrl_gru_cfg;
 
 size_t       rslrl_gru_num_params(const rslrl_gru_cfg *cfg);      /* 0 if cfg is invalid             */

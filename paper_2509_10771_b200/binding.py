@@ -79,7 +79,8 @@ class RndCfg(C.Structure):
 
 
 class GruCfg(C.Structure):
-    _fields_ = [("input_dim", C.c_int32), ("hidden_dim", C.c_int32), ("max_steps", C.c_int32), ("max_envs", C.c_int32)]
+    _fields_ = [("input_dim", C.c_int32), ("hidden_dim", C.c_int32), ("max_steps", C.c_int32), ("max_envs", C.c_int32),
+                ("precision", C.c_int32)]
 
 
 class Counters(C.Structure):
@@ -403,10 +404,11 @@ class Rnd:
 class Gru:
     """One rslrl_gru: a GRU memory layer over time-major rollouts with state resets and BPTT."""
 
-    def __init__(self, input_dim: int, hidden_dim: int, max_steps: int, max_envs: int, stream: int = 0):
+    def __init__(self, input_dim: int, hidden_dim: int, max_steps: int, max_envs: int, stream: int = 0,
+                 precision: int = 0):
         self.lib = load_library()
         self.handle = None
-        cfg = GruCfg(input_dim, hidden_dim, max_steps, max_envs)
+        cfg = GruCfg(input_dim, hidden_dim, max_steps, max_envs, precision)
         self.num_params = int(self.lib.rslrl_gru_num_params(C.byref(cfg)))
         h = C.c_void_p()
         st = self.lib.rslrl_gru_create(C.byref(cfg), stream, C.byref(h))

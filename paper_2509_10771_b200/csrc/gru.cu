@@ -10,6 +10,7 @@
 #include "../../include/rslrl_b200.h"
 #include "common.cuh"
 #include "kernels.h"
+#include "tf32.h"
 
 #include <algorithm>
 #include <cstdarg>
@@ -122,11 +123,72 @@ struct rslrl_gru {
     int T = 0, N = 0;
     bool forward_done = false;
     std::string err;
+    // RSLRL_TF32: transposed weight copies (the forward operands, contraction contiguous), biases padded to 32
+    // entries, the device error word of the tensor-core kernels, and the prepared launches of the shapes seen last
+    bool tf32 = false;
+    float *wi_t = nullptr, *wh_t = nullptr, *bi_pad = nullptr, *bh_pad = nullptr;
+    int ld_wi_t = 0, ld_wh_t = 0;
+    int* tc_error = nullptr;
+    struct Ops {
+        const float* x = nullptr; int x_stride = 0; float* dx = nullptr; int dx_stride = 0; int T = 0, N = 0;
+        rslrl::Tf32Op* gi = nullptr; rslrl::Tf32Op* dx_op = nullptr; rslrl::Tf32Op* wgrad = nullptr;
+        std::vector<rslrl::Tf32Op*> gh, dh;       // one per step
+    } ops;
 };
 
 namespace {
 
 std::string g_gru_create_error;
+
+rslrl_status gfail(rslrl_gru* g, rslrl_status s, const char* fmt, ...);
+
+// RSLRL_TF32: the prepared tensor-core launches depend on the caller's x pointer and on T and N; they are built when
+// those change (host work only: tensor maps) and kept for the calls that follow.
+constexpr int kGruWgradRowsPerSplit = 32;
+void gru_wgrad_split(size_t rows, int* splits, int* kchunk) {
+    *splits = (int)std::max<size_t>(1, std::min<size_t>(32, rows / 512));
+    const int per = (int)((rows + *splits - 1) / *splits);
+    *kchunk = (per + kGruWgradRowsPerSplit - 1) / kGruWgradRowsPerSplit * kGruWgradRowsPerSplit;
+}
+
+void drop_ops(rslrl_gru* g);
+rslrl_status prepare_ops(rslrl_gru* g, const float* d_x, int x_stride, int T, int N) {
+    rslrl_gru::Ops& o = g->ops;
+    if (o.gi && o.x == d_x && o.x_stride == x_stride && o.T == T && o.N == N) return RSLRL_OK;
+    drop_ops(g);
+    const int H = g->H, D = g->D, G3 = 3 * H;
+    const size_t rows = (size_t)T * N;
+    bool ok = true;
+    o.gi = tf32_op_gemm(d_x, (int)rows, D, x_stride, g->wi_t, G3, g->ld_wi_t, g->gi, G3, g->bi_pad, g->tc_error);
+    ok = ok && o.gi;
+    for (int t = 0; ok && t < T; ++t) {
+        float* gh_t = g->gh + (size_t)t * N * G3;
+        const float* hin_t = g->hin + (size_t)t * N * H;
+        // gh_t = h_in W_h + b_h;  tmp = d gh_t W_h^T (W_h as stored is the operand with the contraction contiguous)
+        o.gh.push_back(tf32_op_gemm(hin_t, N, H, H, g->wh_t, G3, g->ld_wh_t, gh_t, G3, g->bh_pad, g->tc_error));
+        o.dh.push_back(tf32_op_gemm(gh_t, N, G3, G3, g->param + g->off_wh, H, G3, g->tmp, H, nullptr, g->tc_error));
+        ok = o.gh.back() && o.dh.back();
+    }
+    if (ok) {
+        int splits, kchunk;
+        gru_wgrad_split(rows, &splits, &kchunk);
+        const Tf32WgradDesc d[2] = {
+            {d_x, x_stride, D, g->gi, G3, G3, G3, g->partials + g->off_wi, G3},
+            {g->hin, H, H, g->gh, G3, G3, G3, g->partials + g->off_wh, G3}};
+        o.wgrad = tf32_op_wgrad(d, 2, (int)rows, splits, kchunk, (long long)g->P, g->tc_error);
+        ok = o.wgrad != nullptr;
+    }
+    if (!ok) { drop_ops(g); return gfail(g, RSLRL_ERR_CUDA, "could not prepare the tensor-core launches (tensor map encoding)"); }
+    o.x = d_x; o.x_stride = x_stride; o.T = T; o.N = N;
+    return RSLRL_OK;
+}
+
+void drop_ops(rslrl_gru* g) {
+    tf32_op_free(g->ops.gi); tf32_op_free(g->ops.dx_op); tf32_op_free(g->ops.wgrad);
+    for (Tf32Op* o : g->ops.gh) tf32_op_free(o);
+    for (Tf32Op* o : g->ops.dh) tf32_op_free(o);
+    g->ops = rslrl_gru::Ops{};
+}
 
 rslrl_status gfail(rslrl_gru* g, rslrl_status s, const char* fmt, ...) {
     char buf[512];
@@ -150,6 +212,7 @@ bool valid_cfg(const rslrl_gru_cfg* c, std::string* why) {
     if (c->max_steps < 1 || c->max_envs < 1) return bad("max_steps and max_envs must be positive");
     if ((long long)c->max_steps * c->max_envs >= (1ll << 30)) return bad("max_steps * max_envs must be below 2^30");
     if ((long long)c->max_envs * 3 * c->hidden_dim >= (1ll << 31)) return bad("max_envs * 3 * hidden_dim must be below 2^31");
+    if (c->precision < RSLRL_FP32 || c->precision > RSLRL_BF16) return bad("unknown precision");
     return true;
 }
 
@@ -181,6 +244,7 @@ const char* rslrl_gru_last_error(const rslrl_gru* g) { return g ? g->err.c_str()
 rslrl_status rslrl_gru_destroy(rslrl_gru* g) {
     if (!g) return RSLRL_ERR_INVALID_ARG;
     cudaStreamSynchronize(g->stream);
+    drop_ops(g);
     for (void* p : g->allocs) guarded_free(p);
     delete g;
     return RSLRL_OK;
@@ -191,8 +255,14 @@ rslrl_status rslrl_gru_create(const rslrl_gru_cfg* cfg, void* cuda_stream, rslrl
     *out = nullptr;
     std::string why;
     if (!valid_cfg(cfg, &why)) return gfail(nullptr, RSLRL_ERR_INVALID_ARG, "%s", why.c_str());
+    if (cfg->precision == RSLRL_BF16) return gfail(nullptr, RSLRL_ERR_UNSUPPORTED, "the recurrent layer has no BF16 mode");
+    if (cfg->precision == RSLRL_TF32) {
+        std::string terr;
+        if (!tf32_ops_init(&terr)) return gfail(nullptr, RSLRL_ERR_UNSUPPORTED, "tensor-core mode: %s", terr.c_str());
+    }
     rslrl_gru* g = new rslrl_gru();
     g->cfg = *cfg;
+    g->tf32 = cfg->precision == RSLRL_TF32;
     g->stream = (cudaStream_t)cuda_stream;
     g->D = cfg->input_dim; g->H = cfg->hidden_dim; g->max_T = cfg->max_steps; g->max_N = cfg->max_envs;
     const size_t D = g->D, H = g->H;
@@ -200,7 +270,12 @@ rslrl_status rslrl_gru_create(const rslrl_gru_cfg* cfg, void* cuda_stream, rslrl
     g->P = (int)(g->off_bh + 3 * H);
     const size_t rows = (size_t)g->max_T * g->max_N;
     g->max_splits = (int)std::max<size_t>(1, std::min<size_t>(32, rows / 512));
-    const bool ok = dalloc(g, &g->param, (size_t)g->P) && dalloc(g, &g->grad, (size_t)g->P) &&
+    g->ld_wi_t = round_up(g->D, 4); g->ld_wh_t = round_up(g->H, 4);
+    const bool tc_ok = !g->tf32 ||
+                       (dalloc(g, &g->wi_t, 3 * H * g->ld_wi_t) && dalloc(g, &g->wh_t, 3 * H * g->ld_wh_t) &&
+                        dalloc(g, &g->bi_pad, (size_t)round_up((int)(3 * H), 32)) && dalloc(g, &g->bh_pad, (size_t)round_up((int)(3 * H), 32)) &&
+                        dalloc(g, &g->tc_error, 1));
+    const bool ok = tc_ok && dalloc(g, &g->param, (size_t)g->P) && dalloc(g, &g->grad, (size_t)g->P) &&
                     dalloc(g, &g->partials, (size_t)g->P * g->max_splits) && dalloc(g, &g->gi, rows * 3 * H) &&
                     dalloc(g, &g->gh, rows * 3 * H) && dalloc(g, &g->hin, rows * H) &&
                     dalloc(g, &g->dhz, (size_t)g->max_N * H) && dalloc(g, &g->tmp, (size_t)kTmpSplits * g->max_N * H) &&
@@ -218,6 +293,13 @@ rslrl_status rslrl_gru_set_params(rslrl_gru* g, const float* h, size_t n) {
     if (!g || !h) return RSLRL_ERR_INVALID_ARG;
     if (n != (size_t)g->P) return gfail(g, RSLRL_ERR_SHAPE, "expected %d parameters, got %zu", g->P, n);
     GCU(g, cudaMemcpyAsync(g->param, h, sizeof(float) * n, cudaMemcpyHostToDevice, g->stream));
+    if (g->tf32) {
+        const int G3 = 3 * g->H;
+        GCU(g, tf32_transpose(g->param + g->off_wi, g->D, G3, G3, g->wi_t, g->ld_wi_t, g->stream));
+        GCU(g, tf32_transpose(g->param + g->off_wh, g->H, G3, G3, g->wh_t, g->ld_wh_t, g->stream));
+        GCU(g, cudaMemcpyAsync(g->bi_pad, g->param + g->off_bi, sizeof(float) * G3, cudaMemcpyDeviceToDevice, g->stream));
+        GCU(g, cudaMemcpyAsync(g->bh_pad, g->param + g->off_bh, sizeof(float) * G3, cudaMemcpyDeviceToDevice, g->stream));
+    }
     GCU(g, cudaStreamSynchronize(g->stream));
     g->forward_done = false;
     return RSLRL_OK;
@@ -227,7 +309,13 @@ rslrl_status rslrl_gru_get_grads(rslrl_gru* g, float* h, size_t n) {
     if (!g || !h) return RSLRL_ERR_INVALID_ARG;
     if (n != (size_t)g->P) return gfail(g, RSLRL_ERR_SHAPE, "expected %d parameters, got %zu", g->P, n);
     GCU(g, cudaMemcpyAsync(h, g->grad, sizeof(float) * n, cudaMemcpyDeviceToHost, g->stream));
+    int code = 0;
+    if (g->tf32) GCU(g, cudaMemcpyAsync(&code, g->tc_error, sizeof(int), cudaMemcpyDeviceToHost, g->stream));
     GCU(g, cudaStreamSynchronize(g->stream));
+    if (code != 0) {                     // reported once
+        GCU(g, cudaMemsetAsync(g->tc_error, 0, sizeof(int), g->stream));
+        return gfail(g, RSLRL_ERR_TIMEOUT, "a bounded wait in a tensor-core kernel expired (role %d)", code);
+    }
     return RSLRL_OK;
 }
 
@@ -241,8 +329,14 @@ rslrl_status rslrl_gru_forward(rslrl_gru* g, const float* d_x, int32_t x_stride,
     const int H = g->H, D = g->D, G3 = 3 * H;
     const size_t rows = (size_t)T * N;
     g->forward_done = false;
+    if (g->tf32) {
+        const rslrl_status ps = prepare_ops(g, d_x, x_stride, T, N);
+        if (ps != RSLRL_OK) return ps;
+    }
     // input products of all steps at once: gi = x W_i + b_i
-    {
+    if (g->tf32) {
+        GCU(g, tf32_op_launch(g->ops.gi, g->stream));
+    } else {
         GemmBatch b{};
         GemmProblem& p = b.p[b.count++];
         p.A = d_x; p.lda = x_stride; p.B = g->param + g->off_wi; p.ldb = G3; p.C = g->gi; p.ldc = G3;
@@ -259,12 +353,16 @@ rslrl_status rslrl_gru_forward(rslrl_gru* g, const float* d_x, int32_t x_stride,
         float* gi_t = g->gi + (size_t)t * N * G3;
         float* gh_t = g->gh + (size_t)t * N * G3;
         const float* hin_t = g->hin + (size_t)t * N * H;
-        GemmBatch b{};
-        GemmProblem& p = b.p[b.count++];
-        p.A = hin_t; p.lda = H; p.B = g->param + g->off_wh; p.ldb = G3; p.C = gh_t; p.ldc = G3;
-        p.bias = g->param + g->off_bh; p.M = N; p.N = G3; p.K = H; p.Cn = G3;
-        p.splits = 1; p.kchunk = round_up(H, 8); p.split_stride = 0;
-        GCU(g, launch_sgemm(b, false, false, EPI_BIAS, g->stream));
+        if (g->tf32) {
+            GCU(g, tf32_op_launch(g->ops.gh[t], g->stream));
+        } else {
+            GemmBatch b{};
+            GemmProblem& p = b.p[b.count++];
+            p.A = hin_t; p.lda = H; p.B = g->param + g->off_wh; p.ldb = G3; p.C = gh_t; p.ldc = G3;
+            p.bias = g->param + g->off_bh; p.M = N; p.N = G3; p.K = H; p.Cn = G3;
+            p.splits = 1; p.kchunk = round_up(H, 8); p.split_stride = 0;
+            GCU(g, launch_sgemm(b, false, false, EPI_BIAS, g->stream));
+        }
         LaunchScope scope_("gru_gate", g->stream);
         GCU(g, launch_chained(gru_gate_kernel, dim3(blocks), dim3(256), 0, g->stream, gi_t, (const float*)gh_t, hin_t,
                               d_dones + (size_t)t * N, d_h_out + (size_t)t * N * H,
@@ -294,7 +392,12 @@ rslrl_status rslrl_gru_backward(rslrl_gru* g, const float* d_dh, float* d_dx, in
                                   t + 1 < T ? g->dones + (size_t)t * N : (const uint8_t*)nullptr, g->dhz, (const float*)g->tmp,
                                   (size_t)g->max_N * H, N, H));
         }
-        // tmp = d gh W_h^T
+        // tmp = d gh W_h^T (the tensor-core product fills the first of the slices the gate kernel adds up; the
+        // others stay zero)
+        if (g->tf32) {
+            GCU(g, tf32_op_launch(g->ops.dh[t], g->stream));
+            continue;
+        }
         GemmBatch b{};
         GemmProblem& p = b.p[b.count++];
         p.A = gh_t; p.lda = G3; p.B = g->param + g->off_wh; p.ldb = G3; p.C = g->tmp; p.ldc = H;
@@ -306,7 +409,17 @@ rslrl_status rslrl_gru_backward(rslrl_gru* g, const float* d_dh, float* d_dx, in
         LaunchScope scope_("gru_add", g->stream);
         GCU(g, launch_chained(gru_add_kernel, dim3(blocks), dim3(256), 0, g->stream, (const float*)g->dhz, (const float*)g->tmp, (size_t)g->max_N * H, g->h0_reset, d_dh0, N, H));
     }
-    if (d_dx) {
+    if (d_dx && g->tf32) {
+        // dx = d gi W_i^T (W_i as stored is the operand with the contraction contiguous)
+        rslrl_gru::Ops& o = g->ops;
+        if (!o.dx_op || o.dx != d_dx || o.dx_stride != dx_stride) {
+            tf32_op_free(o.dx_op);
+            o.dx_op = tf32_op_gemm(g->gi, (int)rows, G3, G3, g->param + g->off_wi, D, G3, d_dx, dx_stride, nullptr, g->tc_error, round_up(D, 4));
+            if (!o.dx_op) return gfail(g, RSLRL_ERR_CUDA, "could not prepare the tensor-core launch of dx (tensor map encoding)");
+            o.dx = d_dx; o.dx_stride = dx_stride;
+        }
+        GCU(g, tf32_op_launch(o.dx_op, g->stream));
+    } else if (d_dx) {
         GemmBatch b{};
         GemmProblem& p = b.p[b.count++];
         p.A = g->gi; p.lda = G3; p.B = g->param + g->off_wi; p.ldb = G3; p.C = d_dx; p.ldc = dx_stride;
@@ -314,8 +427,9 @@ rslrl_status rslrl_gru_backward(rslrl_gru* g, const float* d_dh, float* d_dx, in
         GCU(g, launch_sgemm(b, false, true, EPI_PLAIN, g->stream));
     }
     // parameter gradients over all steps: dW_i = x^T d gi, dW_h = h_in^T d gh, biases = column sums
-    const int splits = (int)std::max<size_t>(1, std::min<size_t>(32, rows / 512));
-    const int kchunk = round_up((int)((rows + splits - 1) / splits), 8);
+    int splits, kchunk;
+    gru_wgrad_split(rows, &splits, &kchunk);
+    if (g->tf32) GCU(g, tf32_op_launch(g->ops.wgrad, g->stream));
     {
         GemmBatch b{};
         GemmProblem& p = b.p[b.count++];
@@ -324,7 +438,7 @@ rslrl_status rslrl_gru_backward(rslrl_gru* g, const float* d_dh, float* d_dx, in
         GemmProblem& q = b.p[b.count++];
         q.A = g->hin; q.lda = H; q.B = g->gh; q.ldb = G3; q.C = g->partials + g->off_wh; q.ldc = G3;
         q.M = H; q.N = G3; q.K = (int)rows; q.Cn = G3; q.splits = splits; q.kchunk = kchunk; q.split_stride = g->P;
-        GCU(g, launch_sgemm(b, true, false, EPI_PLAIN, g->stream));
+        if (!g->tf32) GCU(g, launch_sgemm(b, true, false, EPI_PLAIN, g->stream));
         ColsumBatch cs{};
         cs.splits = splits; cs.split_stride = g->P; cs.is_bf16 = 0;
         cs.p[cs.count++] = ColsumProblem{g->gi, g->partials + g->off_bi, (int)rows, G3, G3};

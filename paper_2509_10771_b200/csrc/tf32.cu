@@ -30,7 +30,7 @@ constexpr uint32_t kTfStageB = kTfMaxBN * 128;    // 16 KiB
 constexpr uint32_t kTfTile = 32 * 32 * 4;         // 4 KiB result tile per epilogue warp
 constexpr size_t kTfSmem = 1024 + (size_t)kTfStages * (kStageA + kTfStageB) + kEpiWarps * kTfTile + 512;
 
-enum TfMode { TF_FWD = 0, TF_DGRAD = 1 };
+enum TfMode { TF_FWD = 0, TF_DGRAD = 1, TF_BIAS = 2, TF_PLAIN = 3 };   // epilogue: bias + ELU, ELU' from aux, bias, none
 
 struct TfProblem {
     int m_extent, n_extent;        // rows / columns of D that exist (stores are clipped to them)
@@ -240,6 +240,15 @@ __global__ void __launch_bounds__(kThreads, 1) tf32_gemm_kernel(const __grid_con
                         o.y = elu_fast(__uint_as_float(acc[4 * g + 1]) + b.y, P.alpha);
                         o.z = elu_fast(__uint_as_float(acc[4 * g + 2]) + b.z, P.alpha);
                         o.w = elu_fast(__uint_as_float(acc[4 * g + 3]) + b.w, P.alpha);
+                    } else if (MODE == TF_BIAS) {
+                        const float4 b = __ldg(reinterpret_cast<const float4*>(p.bias + col) + g);
+                        o.x = __uint_as_float(acc[4 * g]) + b.x;
+                        o.y = __uint_as_float(acc[4 * g + 1]) + b.y;
+                        o.z = __uint_as_float(acc[4 * g + 2]) + b.z;
+                        o.w = __uint_as_float(acc[4 * g + 3]) + b.w;
+                    } else if (MODE == TF_PLAIN) {
+                        o.x = __uint_as_float(acc[4 * g]); o.y = __uint_as_float(acc[4 * g + 1]);
+                        o.z = __uint_as_float(acc[4 * g + 2]); o.w = __uint_as_float(acc[4 * g + 3]);
                     } else {
                         const float4 h = *piece;
                         o.x = __uint_as_float(acc[4 * g]) * elu_grad_from_h(h.x, P.alpha);
@@ -568,20 +577,22 @@ void finish(TfParams& P, float alpha, int* error) {
 }
 
 // D[rows x n] = A[rows x k] * B[n x k]^T with A [a_rows_total][lda], B [n][ldb], D [rows][ldd]; aux (may be null) like D.
+// n_store (>= n, default n): columns of D that are written; those at and beyond n come out as zero.
 bool add_problem(TfParams& P, const float* A, long long a_rows_total, int rows, int k, int lda, const float* B, int n, int ldb,
-                 float* D, int ldd, const float* aux, const float* bias) {
+                 float* D, int ldd, const float* aux, const float* bias, int n_store = 0) {
     const int i = P.count;
     TfProblem& p = P.p[i];
     memset(&p, 0, sizeof p);
-    p.bn = std::min(kTfMaxBN, round_up(n, 16));
-    p.m_extent = rows; p.n_extent = n;
+    if (n_store < n) n_store = n;
+    p.bn = std::min(kTfMaxBN, round_up(n_store, 16));
+    p.m_extent = rows; p.n_extent = n_store;
     p.m_tiles = (rows + BLOCK_M - 1) / BLOCK_M;
-    p.n_tiles = (n + p.bn - 1) / p.bn;
+    p.n_tiles = (n_store + p.bn - 1) / p.bn;
     p.kblocks = (k + kTfBlockK - 1) / kTfBlockK;
     p.bias = bias;
     if (!make_tmap_f32(&P.tmA[i], A, a_rows_total, k, lda, kTfBlockK, BLOCK_M)) return false;
     if (!make_tmap_f32(&P.tmB[i], B, n, k, ldb, kTfBlockK, p.bn)) return false;
-    if (!make_tmap_f32(&P.tmOut[i], D, rows, n, ldd, 32, 32)) return false;
+    if (!make_tmap_f32(&P.tmOut[i], D, rows, n_store, ldd, 32, 32)) return false;
     if (aux && !make_tmap_f32(&P.tmAux[i], aux, rows, n, ldd, 32, 32)) return false;
     P.count++;
     return true;
@@ -591,7 +602,7 @@ template <int MODE>
 cudaError_t launch_tf(const TfParams& P, int num_sms, cudaStream_t s) {
     if (P.total_items == 0) return cudaSuccess;
     const int grid = std::min(P.total_items, num_sms);
-    LaunchScope scope_(MODE == TF_FWD ? "tc_gemm_fwd" : "tc_gemm_dgrad", s);
+    LaunchScope scope_(MODE == TF_FWD ? "tc_gemm_fwd" : MODE == TF_DGRAD ? "tc_gemm_dgrad" : "tc_gemm_linear", s);
     return launch_chained(tf32_gemm_kernel<MODE>, grid, kThreads, kTfSmem, s, P);
 }
 
@@ -755,6 +766,112 @@ cudaError_t tf32_read_error(Tf32Engine* e, int* host_code) {
     err = cudaStreamSynchronize(e->s.stream);
     if (err != cudaSuccess || *host_code == 0) return err;
     return cudaMemsetAsync(e->error_dev, 0, sizeof(int), e->s.stream);
+}
+
+// ------------------------------------------------------------------ prepared launches for other callers
+struct Tf32Op {
+    int kind = 0;                 // TF_BIAS / TF_PLAIN: P; 100: W
+    TfParams P;
+    TfWgParams W;
+    int num_sms = 148;
+};
+
+namespace {
+
+__global__ void tf32_transpose_one_kernel(TransposeEntry e) {
+    __shared__ float t[32][33];
+    const int i0 = blockIdx.y * 32, o0 = blockIdx.x * 32;
+    for (int r = threadIdx.y; r < 32; r += blockDim.y) {
+        const int i = i0 + r, o = o0 + threadIdx.x;
+        t[r][threadIdx.x] = (i < e.in && o < e.out) ? e.src[(size_t)i * e.ld_src + o] : 0.f;
+    }
+    __syncthreads();
+    for (int r = threadIdx.y; r < 32; r += blockDim.y) {
+        const int o = o0 + r, i = i0 + threadIdx.x;
+        if (o < e.out && i < e.in) e.dst[(size_t)o * e.ld_dst + i] = t[threadIdx.x][r];
+    }
+}
+
+int device_sms() {
+    int sms = 148, dev = 0;
+    if (cudaGetDevice(&dev) == cudaSuccess) cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
+    return sms;
+}
+
+}  // namespace
+
+bool tf32_ops_init(std::string* err) {
+    auto failmsg = [&](const char* m) { if (err) *err = m; return false; };
+    if (!get_encode_fn()) return failmsg("cuTensorMapEncodeTiled is not available from the driver");
+    int dev = 0; cudaDeviceProp prop;
+    if (cudaGetDevice(&dev) != cudaSuccess || cudaGetDeviceProperties(&prop, dev) != cudaSuccess) return failmsg("no CUDA device");
+    if (prop.major != 10) return failmsg("the tensor-core mode needs an sm_100 device");
+    if (cudaFuncSetAttribute(tf32_gemm_kernel<TF_BIAS>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kTfSmem) != cudaSuccess ||
+        cudaFuncSetAttribute(tf32_gemm_kernel<TF_PLAIN>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kTfSmem) != cudaSuccess ||
+        cudaFuncSetAttribute(tf32_wgrad_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kTfWgSmem) != cudaSuccess)
+        return failmsg("could not reserve shared memory for the tensor-core kernels");
+    return true;
+}
+
+Tf32Op* tf32_op_gemm(const float* A, int rows, int k, int lda, const float* B, int n, int ldb, float* D, int ldd,
+                     const float* bias, int* error_dev, int n_store) {
+    Tf32Op* op = new Tf32Op();
+    op->kind = bias ? TF_BIAS : TF_PLAIN;
+    op->num_sms = device_sms();
+    memset(&op->P, 0, sizeof op->P);
+    if (!add_problem(op->P, A, rows, rows, k, lda, B, n, ldb, D, ldd, nullptr, bias, n_store)) { delete op; return nullptr; }
+    finish(op->P, 0.f, error_dev);
+    return op;
+}
+
+Tf32Op* tf32_op_wgrad(const Tf32WgradDesc* d, int count, int rows, int splits, int kchunk, long long split_stride, int* error_dev) {
+    if (count < 1 || count > kTfWgProblems || splits < 1 || kchunk < kTfBlockK || kchunk % kTfBlockK != 0) return nullptr;
+    Tf32Op* op = new Tf32Op();
+    op->kind = 100;
+    op->num_sms = device_sms();
+    TfWgParams& W = op->W;
+    memset(&W, 0, sizeof W);
+    int items = 0;
+    for (int i = 0; i < count; ++i) {
+        TfWgProblem& p = W.p[i];
+        p.m_extent = d[i].m; p.n_store = d[i].n_store;
+        p.bn = std::min(kTfMaxBN, round_up(d[i].n, 32));
+        p.m_tiles = (p.m_extent + BLOCK_M - 1) / BLOCK_M;
+        p.n_tiles = (p.n_store + p.bn - 1) / p.bn;
+        p.kblocks = (rows + kTfBlockK - 1) / kTfBlockK;
+        p.kb_per_split = kchunk / kTfBlockK;
+        p.splits = splits;
+        p.item_begin = items; items += p.m_tiles * p.n_tiles * p.splits;
+        p.out = d[i].out; p.ld_out = d[i].ld_out; p.split_stride = split_stride;
+        if (!make_tmap_f32(&W.tmA[i], d[i].A, rows, d[i].m, d[i].lda, 32, 32, CU_TENSOR_MAP_SWIZZLE_128B_ATOM_32B) ||
+            !make_tmap_f32(&W.tmB[i], d[i].B, rows, d[i].n, d[i].ldb, 32, 32, CU_TENSOR_MAP_SWIZZLE_128B_ATOM_32B)) {
+            delete op;
+            return nullptr;
+        }
+        W.count++;
+    }
+    W.total_items = items; W.error = error_dev;
+    return op;
+}
+
+cudaError_t tf32_op_launch(const Tf32Op* op, cudaStream_t stream) {
+    if (!op) return cudaErrorInvalidValue;
+    if (op->kind == 100) {
+        if (op->W.total_items == 0) return cudaSuccess;
+        LaunchScope scope_("tc_gemm_wgrad", stream);
+        return launch_chained(tf32_wgrad_kernel, std::min(op->W.total_items, op->num_sms), kThreads, kTfWgSmem, stream, op->W);
+    }
+    if (op->kind == TF_BIAS) return launch_tf<TF_BIAS>(op->P, op->num_sms, stream);
+    return launch_tf<TF_PLAIN>(op->P, op->num_sms, stream);
+}
+
+void tf32_op_free(Tf32Op* op) { delete op; }
+
+cudaError_t tf32_transpose(const float* src, int in, int out, int ld_src, float* dst, int ld_dst, cudaStream_t stream) {
+    if (in <= 0 || out <= 0) return cudaSuccess;
+    const TransposeEntry e{src, dst, in, out, ld_src, ld_dst};
+    tf32_transpose_one_kernel<<<dim3((out + 31) / 32, (in + 31) / 32), dim3(32, 8), 0, stream>>>(e);
+    return cudaGetLastError();
 }
 
 }  // namespace rslrl

@@ -48,4 +48,24 @@ cudaError_t tf32_update_wgrad(Tf32Engine* e);
 // Synchronises the stream and returns the device error code (0 = none); a non-zero code is cleared once read.
 cudaError_t tf32_read_error(Tf32Engine* e, int* host_code);
 
+// ------------------------------------------------------------------------------------------------
+// The same kernels for other callers (the recurrent layer): prepared launches on caller-owned buffers.
+struct Tf32Op;
+// Once per process before the first op: shared-memory attributes of the kernels; false (with a reason) on a
+// device without these tensor cores.
+bool tf32_ops_init(std::string* err);
+// D[rows][ldd] = A[rows][k] (row stride lda) * B[n][k]^T (row stride ldb, the contraction contiguous) (+ bias[n],
+// readable up to the next multiple of 32 entries, or null).  Pointers 16-byte aligned, strides multiples of 4 floats.
+// n_store (0: n): columns of D that are written; those from n on come out as zero.
+Tf32Op* tf32_op_gemm(const float* A, int rows, int k, int lda, const float* B, int n, int ldb, float* D, int ldd,
+                     const float* bias, int* error_dev, int n_store = 0);
+// out_i[s][m_i][ld_out_i] (s-th slice at s * split_stride floats) = A_i[rows s][m_i]^T B_i[rows s][n_i] for up to eight
+// pairs, rows s = [s * kchunk, (s + 1) * kchunk) cut at `rows`; kchunk a multiple of 32; n_store_i columns are written.
+struct Tf32WgradDesc { const float* A; int lda, m; const float* B; int ldb, n, n_store; float* out; int ld_out; };
+Tf32Op* tf32_op_wgrad(const Tf32WgradDesc* d, int count, int rows, int splits, int kchunk, long long split_stride, int* error_dev);
+cudaError_t tf32_op_launch(const Tf32Op* op, cudaStream_t stream);
+void tf32_op_free(Tf32Op* op);
+// dst[out][ld_dst] = src[in][ld_src]^T (FP32), on the stream
+cudaError_t tf32_transpose(const float* src, int in, int out, int ld_src, float* dst, int ld_dst, cudaStream_t stream);
+
 }  // namespace rslrl

@@ -85,4 +85,5 @@ def test_rnd_and_gru_configs_without_a_device():
     assert lib.rslrl_gru_num_params(ctypes.byref(g)) == 235 * 768 + 768 + 256 * 768 + 768
     assert lib.rslrl_gru_num_params(ctypes.byref(binding.GruCfg(235, 250, 24, 4096))) == 0     # H not a multiple of 4
     assert lib.rslrl_gru_num_params(ctypes.byref(binding.GruCfg(235, 256, 1 << 15, 1 << 15))) == 0   # T * N too large
-    assert ctypes.sizeof(binding.GruCfg) == 16
+    assert ctypes.sizeof(binding.GruCfg) == 20 and binding.GruCfg.precision.offset == 16
+    assert lib.rslrl_gru_num_params(ctypes.byref(binding.GruCfg(235, 256, 24, 4096, 3))) == 0          # no such precision

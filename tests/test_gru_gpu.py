@@ -25,7 +25,7 @@ CASES = {
 }
 
 
-def _run(case, want_dx=True, want_dh0=True):
+def _run(case, want_dx=True, want_dh0=True, precision=0):
     import torch
     from paper_2509_10771_b200 import binding
     w0, H, pad, dp = CASES[case]
@@ -39,7 +39,7 @@ def _run(case, want_dx=True, want_dh0=True):
     stride = (D + 3) // 4 * 4 + (4 * ((pad + 3) // 4) if pad else 0)
     xp = np.full((T, N, stride), 7.0, dtype=np.float32)        # padding holds junk: it must not be read as data
     xp[..., :D] = x
-    gru = binding.Gru(D, H, T, N)
+    gru = binding.Gru(D, H, T, N, precision=precision)
     gru.set_params(setup["params"])
     dev = "cuda"
     d_x = torch.from_numpy(xp).to(dev)
@@ -72,6 +72,24 @@ def test_states_and_gradients_match_oracle(case):
     for name, a, b in zip(("W_i", "b_i", "W_h", "b_h"), o[:-1], o[1:]):
         assert_close(got["grad"][a:b], ref[a:b], 1e-4, f"{case}.d{name}")
     # columns of dx between D and D rounded up to 4 are written as zero, the rest of the padding is left alone
+    d4 = (D + 3) // 4 * 4
+    assert np.all(got["dx"][..., D:d4] == 0.0) and np.all(got["dx"][..., d4:] == -3.0)
+    gru.destroy()
+
+
+@pytest.mark.parametrize("case", ["tiny", "flat", "rough", "humanoid"])
+def test_states_and_gradients_match_oracle_tf32(case):
+    """RSLRL_TF32: every matrix product of the layer sees TF32 operands (11 significant bits).  States at the mode's
+    tolerance 5e-3; gradients, which back-propagation passes through up to T such products, at twice that."""
+    w, D, H, dones, c, g, got, gru = _run(case, precision=WL.PRECISION_TF32)
+    assert_close(got["h"], c["h"], 5e-3, f"{case}.h")
+    assert not np.array_equal(got["h"], _run(case)[6]["h"])        # the tensor cores did see TF32 operands
+    assert_close(got["dx"][..., :D], g["x"], 1e-2, f"{case}.dx")
+    assert_close(got["dh0"], g["h0"], 1e-2, f"{case}.dh0")
+    ref = G.flat_grads(g)
+    o = np.cumsum([0, D * 3 * H, 3 * H, H * 3 * H, 3 * H])
+    for name, a, b in zip(("W_i", "b_i", "W_h", "b_h"), o[:-1], o[1:]):
+        assert_close(got["grad"][a:b], ref[a:b], 1e-2, f"{case}.d{name}")
     d4 = (D + 3) // 4 * 4
     assert np.all(got["dx"][..., D:d4] == 0.0) and np.all(got["dx"][..., d4:] == -3.0)
     gru.destroy()
