@@ -553,7 +553,8 @@ def run_rnd(args):
     d_obs = torch.from_numpy(obs).to(dev)
     d_rew = torch.zeros(B, device=dev)
     rnd = binding.Rnd(w.actor_obs_dim, setup["idx"], setup["hidden"], setup["embed_dim"], max_rows=B, lr=1e-3,
-                      stream=stream.cuda_stream, max_batch=B, max_epochs=w.epochs, max_minibatches=w.minibatches)
+                      stream=stream.cuda_stream, max_batch=B, max_epochs=w.epochs, max_minibatches=w.minibatches,
+                      precision=WL.PRECISION_TF32 if PRECISION == WL.PRECISION_TF32 else WL.PRECISION_FP32)
     rnd.set_params(setup["predictor"], setup["target"])
     flush_buf = torch.empty(256 << 20, dtype=torch.uint8, device=dev)
     it = [0]
@@ -600,11 +601,11 @@ def run_rnd(args):
     line = {
         "metric": "random network distillation transitions/s", "value": B * args.steps / (ms * 1e-3), "unit": UNIT, "n_gpus": 1,
         "steps": args.steps, "warmup": max(args.warmup, 3), "ms_per_step": ms / args.steps, "higher_is_better": True,
-        "dtype": "f32", "data": "synthetic",
+        "dtype": "tf32" if PRECISION == WL.PRECISION_TF32 else "f32", "data": "synthetic",
         "config": {"workload": w.name, "task": "rnd", "num_envs": N, "num_steps": T, "epochs": w.epochs,
                    "minibatches": w.minibatches, "num_idx": 48, "hidden": [256, 128, 64], "embed_dim": 32,
                    "l2": "256 MiB buffer written between timed steps"},
-        "fp32_tflops": flops / (ms / args.steps * 1e-3) / 1e12,
+        ("tf32_tflops" if PRECISION == WL.PRECISION_TF32 else "fp32_tflops"): flops / (ms / args.steps * 1e-3) / 1e12,
         "kernel_shares": shares,
         "cpu_baseline": {"value": rows_s / cpu_s, "unit": UNIT, "cores": blas_threads(), "kind": "oracle",
                          "sample": f"the oracle's reward and predictor training on {ORACLE_SAMPLE_ENVS} of the {N} environments"},
@@ -765,7 +766,7 @@ def main():
     ap.add_argument("--workload", default=WORKLOAD.name, choices=sorted(WL.WORKLOADS),
                     help="which of the five synthetic workloads to time (default: the one the metric is quoted on)")
     ap.add_argument("--precision", default="bf16", choices=["bf16", "tf32"],
-                    help="operand precision of the products on the tensor cores (ppo task, default bf16; gru task: tf32 selects the tensor-core mode, anything else FP32)")
+                    help="operand precision of the products on the tensor cores (ppo task, default bf16; gru and rnd tasks: tf32 selects the tensor-core mode, anything else FP32)")
     ap.add_argument("--task", default="ppo", choices=["ppo", "distill", "rnd", "gru", "streams"],
                     help="ppo: the learn iteration the metric is quoted on (default); distill: the distillation iteration; "
                          "rnd: random network distillation over one rollout; gru: the recurrent layer over one rollout; "

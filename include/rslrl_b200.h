@@ -312,7 +312,9 @@ rslrl_status rslrl_debug_report(int32_t *h_debug_build, int32_t *h_damaged_guard
  *   r_int = (1/E) sum_j (f_j(s) - g_j(s))^2          (E = embed_dim)
  * rslrl_rnd_reward adds weight * r_int to a reward vector; rslrl_rnd_update regresses f on g
  * (loss = mean over the minibatch rows of r_int) with Adam at a fixed learning rate, over the
- * same kind of keyed minibatches as rslrl_ppo_update.  All arithmetic is FP32.  (Observation
+ * same kind of keyed minibatches as rslrl_ppo_update.  With precision RSLRL_FP32 all arithmetic is FP32; with
+ * RSLRL_TF32 the matrix products of both nets (forward, data and weight gradients) run on the tensor cores with
+ * TF32 operands read from the same FP32 buffers, everything else stays FP32 (tolerance class 5e-3).  (Observation
  * normalisation and reward-weight schedules, which the paper's library offers around this, are
  * left to the caller.)
  *
@@ -336,6 +338,7 @@ typedef struct {
     int32_t max_batch;                  /* largest `batch` of rslrl_rnd_update (>= 1)                */
     int32_t max_epochs;                 /* largest `epochs` of rslrl_rnd_update (>= 1)               */
     int32_t max_minibatches;            /* largest `minibatches` of rslrl_rnd_update (>= 1)          */
+    int32_t precision;                  /* RSLRL_FP32 or RSLRL_TF32 (RSLRL_BF16: RSLRL_ERR_UNSUPPORTED) */
 } rslrl_rnd_cfg;
 
 size_t       rslrl_rnd_num_params(const rslrl_rnd_cfg *cfg);      /* of one net; 0 if cfg is invalid */

@@ -75,7 +75,8 @@ class RndCfg(C.Structure):
     _fields_ = [("obs_dim", C.c_int32), ("num_idx", C.c_int32), ("h_idx", C.c_void_p), ("num_hidden", C.c_int32),
                 ("hidden", C.c_int32 * 8), ("embed_dim", C.c_int32), ("elu_alpha", C.c_float), ("max_rows", C.c_int32),
                 ("lr", C.c_float), ("adam_b1", C.c_float), ("adam_b2", C.c_float), ("adam_eps", C.c_float),
-                ("max_batch", C.c_int32), ("max_epochs", C.c_int32), ("max_minibatches", C.c_int32)]
+                ("max_batch", C.c_int32), ("max_epochs", C.c_int32), ("max_minibatches", C.c_int32),
+                ("precision", C.c_int32)]
 
 
 class GruCfg(C.Structure):
@@ -337,7 +338,7 @@ class Rnd:
 
     def __init__(self, obs_dim: int, idx, hidden, embed_dim: int, max_rows: int, lr: float = 1e-3, elu_alpha: float = 1.0,
                  adam_b1: float = 0.9, adam_b2: float = 0.999, adam_eps: float = 1e-8, stream: int = 0,
-                 max_batch: int = 0, max_epochs: int = 8, max_minibatches: int = 16):
+                 max_batch: int = 0, max_epochs: int = 8, max_minibatches: int = 16, precision: int = 0):
         # max_batch = 0: room for max_minibatches minibatches of max_rows rows
         self.lib = load_library()
         self.handle = None
@@ -351,6 +352,7 @@ class Rnd:
         cfg.lr, cfg.adam_b1, cfg.adam_b2, cfg.adam_eps = lr, adam_b1, adam_b2, adam_eps
         cfg.max_batch = max_batch if max_batch > 0 else max_rows * max_minibatches
         cfg.max_epochs, cfg.max_minibatches = max_epochs, max_minibatches
+        cfg.precision = precision
         self.num_params = int(self.lib.rslrl_rnd_num_params(C.byref(cfg)))
         h = C.c_void_p()
         st = self.lib.rslrl_rnd_create(C.byref(cfg), stream, C.byref(h))

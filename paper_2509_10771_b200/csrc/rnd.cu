@@ -9,6 +9,8 @@
 #include "../../include/rslrl_b200.h"
 #include "common.cuh"
 #include "kernels.h"
+#include "tf32.h"
+#include <map>
 
 #include <algorithm>
 #include <cmath>
@@ -131,6 +133,17 @@ struct rslrl_rnd {
     float* gall = nullptr;                        // [max_batch][ldE] the target's outputs for every row of the batch
     long long adam_step = 0;
     std::string err;
+    // RSLRL_TF32: transposed weight copies of both nets (the forward operands, contraction contiguous; the
+    // predictor's are refreshed after every optimiser step), the device error word of the tensor-core kernels, and
+    // the prepared launches per row count (tensor maps: host work only, built when a row count is first seen)
+    bool tf32 = false;
+    std::vector<float*> wt_f, wt_g; std::vector<int> ld_wt;
+    int* tc_error = nullptr;
+    struct RowsOps {
+        std::vector<rslrl::Tf32Op*> fwd_f, fwd_g, dgrad;     // per layer (dgrad[l] produces dz[l - 1])
+        rslrl::Tf32Op* wgrad = nullptr; int wgrad_splits = 0, wgrad_kchunk = 0;
+    };
+    std::map<int, RowsOps> ops;
 };
 
 namespace {
@@ -163,6 +176,7 @@ bool valid_cfg(const rslrl_rnd_cfg* c, std::string* why) {
         if (c->hidden[l] < 1 || c->hidden[l] > 8192) return bad("a hidden width is out of range");
     if (c->embed_dim < 1 || c->embed_dim > 8192) return bad("embed_dim out of range");
     if (c->max_rows < 1) return bad("max_rows must be positive");
+    if (c->precision < RSLRL_FP32 || c->precision > RSLRL_BF16) return bad("unknown precision");
     if (c->max_batch < 1 || c->max_epochs < 1 || c->max_minibatches < 1) return bad("max_batch, max_epochs and max_minibatches must be positive");
     if ((long long)c->max_epochs * c->max_minibatches > (1 << 20)) return bad("max_epochs * max_minibatches exceeds 2^20 steps");
     if (!(c->lr > 0.f) || !(c->adam_eps > 0.f) || c->adam_b1 < 0.f || c->adam_b1 >= 1.f || c->adam_b2 < 0.f || c->adam_b2 >= 1.f)
@@ -201,8 +215,96 @@ int splits_for(int rows) { return std::max(1, std::min(32, rows / 512)); }
 
 // the predictor (do_f) and / or the target (do_g) through all layers on `rows` rows of r->s; g_last, if not
 // null, receives the target's last layer instead of the work buffer
+// ---- RSLRL_TF32 ------------------------------------------------------------------------------------------
+void drop_ops(rslrl_rnd* r) {
+    for (auto& kv : r->ops) {
+        for (Tf32Op* o : kv.second.fwd_f) tf32_op_free(o);
+        for (Tf32Op* o : kv.second.fwd_g) tf32_op_free(o);
+        for (Tf32Op* o : kv.second.dgrad) tf32_op_free(o);
+        tf32_op_free(kv.second.wgrad);
+    }
+    r->ops.clear();
+}
+
+// Wt[out][in] of one net (0: predictor, 1: target) from its W[in][out_p]
+rslrl_status refresh_transposes(rslrl_rnd* r, int net) {
+    const float* par = net == 0 ? r->pf : r->pg;
+    std::vector<float*>& wt = net == 0 ? r->wt_f : r->wt_g;
+    for (size_t l = 0; l < r->L.size(); ++l)
+        RCU(r, tf32_transpose(par + r->L[l].w_off, r->L[l].in, r->L[l].out, r->L[l].out_p, wt[l], r->ld_wt[l], r->stream));
+    return RSLRL_OK;
+}
+
+// rows per weight-gradient split: a multiple of the tensor-core kernel's k-block in TF32 mode
+int kchunk_for(const rslrl_rnd* r, int rows, int splits) { return round_up((rows + splits - 1) / splits, r->tf32 ? 32 : 8); }
+
+rslrl_status ops_for(rslrl_rnd* r, int rows, rslrl_rnd::RowsOps** out) {
+    auto it = r->ops.find(rows);
+    if (it != r->ops.end()) { *out = &it->second; return RSLRL_OK; }
+    rslrl_rnd::RowsOps o;
+    const int nl = (int)r->L.size();
+    bool ok = true;
+    for (int l = 0; ok && l < nl; ++l) {
+        const RLayer& Ly = r->L[l];
+        for (int net = 0; ok && net < 2; ++net) {
+            const float* par = net == 0 ? r->pf : r->pg;
+            std::vector<float*>& h = net == 0 ? r->hf : r->hg;
+            const float* A = l == 0 ? r->s : h[l - 1];
+            const int lda = l == 0 ? r->lds : r->L[l - 1].ld;
+            const float* B = (net == 0 ? r->wt_f : r->wt_g)[l];
+            Tf32Op* op = l + 1 < nl
+                ? tf32_op_gemm_act(0, A, rows, Ly.in, lda, B, Ly.out, r->ld_wt[l], h[l], Ly.ld, par + Ly.b_off, r->cfg.elu_alpha, r->tc_error, Ly.out_p)
+                : tf32_op_gemm(A, rows, Ly.in, lda, B, Ly.out, r->ld_wt[l], h[l], Ly.ld, par + Ly.b_off, r->tc_error, Ly.out_p);
+            (net == 0 ? o.fwd_f : o.fwd_g).push_back(op);
+            ok = op != nullptr;
+        }
+    }
+    o.dgrad.assign(nl, nullptr);
+    for (int l = nl - 1; ok && l > 0; --l) {
+        const RLayer& Ly = r->L[l];
+        // dz[l-1] = (dz[l] W[l]^T) * ELU'(hf[l-1]); W[l] as stored is the operand with the contraction (out) contiguous
+        o.dgrad[l] = tf32_op_gemm_act(1, r->dz[l], rows, Ly.out, Ly.ld, r->pf + Ly.w_off, Ly.in, Ly.out_p, r->dz[l - 1], r->L[l - 1].ld,
+                                      r->hf[l - 1], r->cfg.elu_alpha, r->tc_error, r->L[l - 1].out_p);
+        ok = o.dgrad[l] != nullptr;
+    }
+    if (ok) {
+        o.wgrad_splits = splits_for(rows);
+        o.wgrad_kchunk = kchunk_for(r, rows, o.wgrad_splits);
+        std::vector<Tf32WgradDesc> d;
+        for (int l = 0; l < nl; ++l) {
+            const RLayer& Ly = r->L[l];
+            d.push_back(Tf32WgradDesc{l == 0 ? r->s : r->hf[l - 1], l == 0 ? r->lds : r->L[l - 1].ld, Ly.in, r->dz[l], Ly.ld, Ly.out,
+                                      Ly.out_p, r->partials + Ly.w_off, Ly.out_p});
+        }
+        o.wgrad = tf32_op_wgrad(d.data(), nl, rows, o.wgrad_splits, o.wgrad_kchunk, (long long)r->P_dev, r->tc_error);
+        ok = o.wgrad != nullptr;
+    }
+    if (!ok) {
+        for (Tf32Op* p : o.fwd_f) tf32_op_free(p);
+        for (Tf32Op* p : o.fwd_g) tf32_op_free(p);
+        for (Tf32Op* p : o.dgrad) tf32_op_free(p);
+        tf32_op_free(o.wgrad);
+        return rfail(r, RSLRL_ERR_CUDA, "could not prepare the tensor-core launches (tensor map encoding)");
+    }
+    *out = &(r->ops[rows] = o);
+    return RSLRL_OK;
+}
+
 rslrl_status forward(rslrl_rnd* r, int rows, bool do_f, bool do_g, float* g_last) {
     const int nl = (int)r->L.size();
+    if (r->tf32) {
+        rslrl_rnd::RowsOps* o = nullptr;
+        const rslrl_status ps = ops_for(r, rows, &o);
+        if (ps != RSLRL_OK) return ps;
+        for (int l = 0; l < nl; ++l) {
+            if (do_f) RCU(r, tf32_op_launch(o->fwd_f[l], r->stream));
+            if (do_g) RCU(r, tf32_op_launch(o->fwd_g[l], r->stream));
+        }
+        // the prepared launches write the target's outputs to its own buffer: copied to where the caller wants them
+        if (do_g && g_last)
+            RCU(r, cudaMemcpyAsync(g_last, r->hg.back(), sizeof(float) * (size_t)rows * r->ldE, cudaMemcpyDeviceToDevice, r->stream));
+        return RSLRL_OK;
+    }
     for (int l = 0; l < nl; ++l) {
         const RLayer& Ly = r->L[l];
         GemmBatch b{};
@@ -237,7 +339,15 @@ rslrl_status subset(rslrl_rnd* r, const float* d_obs, int obs_stride, const int*
 // gradients, then the weight gradients of all layers in one launch and all bias gradients in another
 rslrl_status backward(rslrl_rnd* r, int rows, int splits, int kchunk) {
     const int nl = (int)r->L.size();
-    for (int l = nl - 1; l > 0; --l) {
+    rslrl_rnd::RowsOps* tc = nullptr;
+    if (r->tf32) {
+        const rslrl_status ps = ops_for(r, rows, &tc);
+        if (ps != RSLRL_OK) return ps;
+        if (tc->wgrad_splits != splits || tc->wgrad_kchunk != kchunk) return rfail(r, RSLRL_ERR_STATE, "weight-gradient splits do not match the prepared launch");
+        for (int l = nl - 1; l > 0; --l) RCU(r, tf32_op_launch(tc->dgrad[l], r->stream));
+        RCU(r, tf32_op_launch(tc->wgrad, r->stream));
+    }
+    for (int l = nl - 1; l > 0 && !tc; --l) {
         const RLayer& Ly = r->L[l];
         GemmBatch dg{};
         dg.alpha = r->cfg.elu_alpha;
@@ -250,7 +360,7 @@ rslrl_status backward(rslrl_rnd* r, int rows, int splits, int kchunk) {
         d.splits = 1; d.kchunk = round_up(Ly.out, 8); d.split_stride = 0;
         RCU(r, launch_sgemm(dg, false, true, EPI_DELU, r->stream));
     }
-    for (int l0 = 0; l0 < nl; l0 += kMaxGemmBatch) {
+    for (int l0 = 0; l0 < nl && !tc; l0 += kMaxGemmBatch) {
         GemmBatch wg{};
         for (int l = l0; l < std::min(nl, l0 + kMaxGemmBatch); ++l) {
             const RLayer& Ly = r->L[l];
@@ -290,6 +400,7 @@ const char* rslrl_rnd_last_error(const rslrl_rnd* r) { return r ? r->err.c_str()
 rslrl_status rslrl_rnd_destroy(rslrl_rnd* r) {
     if (!r) return RSLRL_ERR_INVALID_ARG;
     cudaStreamSynchronize(r->stream);
+    drop_ops(r);
     for (void* p : r->allocs) guarded_free(p);
     delete r;
     return RSLRL_OK;
@@ -300,8 +411,14 @@ rslrl_status rslrl_rnd_create(const rslrl_rnd_cfg* cfg, void* cuda_stream, rslrl
     *out = nullptr;
     std::string why;
     if (!valid_cfg(cfg, &why)) return rfail(nullptr, RSLRL_ERR_INVALID_ARG, "%s", why.c_str());
+    if (cfg->precision == RSLRL_BF16) return rfail(nullptr, RSLRL_ERR_UNSUPPORTED, "random network distillation has no BF16 mode");
+    if (cfg->precision == RSLRL_TF32) {
+        std::string terr;
+        if (!tf32_ops_init(&terr)) return rfail(nullptr, RSLRL_ERR_UNSUPPORTED, "tensor-core mode: %s", terr.c_str());
+    }
     rslrl_rnd* r = new rslrl_rnd();
     r->cfg = *cfg; r->cfg.h_idx = nullptr;
+    r->tf32 = cfg->precision == RSLRL_TF32;
     r->stream = (cudaStream_t)cuda_stream;
     layer_dims(cfg, &r->L, &r->P_flat, &r->P_dev);
     r->ns = cfg->num_idx; r->lds = round_up(r->ns, 4);
@@ -309,7 +426,8 @@ rslrl_status rslrl_rnd_create(const rslrl_rnd_cfg* cfg, void* cuda_stream, rslrl
     r->max_rows = cfg->max_rows; r->max_splits = splits_for(cfg->max_rows);
     r->max_loss_blocks = (cfg->max_rows + 7) / 8;
     const size_t rows = (size_t)cfg->max_rows;
-    bool ok = dalloc(r, &r->idx, (size_t)r->ns) && dalloc(r, &r->pf, (size_t)r->P_dev) && dalloc(r, &r->pg, (size_t)r->P_dev) &&
+    // (32 floats of slack behind the parameter vectors: the tensor-core epilogues read biases in groups of 32)
+    bool ok = dalloc(r, &r->idx, (size_t)r->ns) && dalloc(r, &r->pf, (size_t)r->P_dev + 32) && dalloc(r, &r->pg, (size_t)r->P_dev + 32) &&
               dalloc(r, &r->grad, (size_t)r->P_dev) && dalloc(r, &r->m, (size_t)r->P_dev) && dalloc(r, &r->v, (size_t)r->P_dev) &&
               dalloc(r, &r->partials, (size_t)r->P_dev * r->max_splits) && dalloc(r, &r->s, rows * r->lds) &&
               dalloc(r, &r->loss_partials, (size_t)r->max_loss_blocks) &&
@@ -320,6 +438,15 @@ rslrl_status rslrl_rnd_create(const rslrl_rnd_cfg* cfg, void* cuda_stream, rslrl
         float *a = nullptr, *b = nullptr, *c = nullptr;
         ok = dalloc(r, &a, rows * r->L[l].ld) && dalloc(r, &b, rows * r->L[l].ld) && dalloc(r, &c, rows * r->L[l].ld);
         r->hf.push_back(a); r->hg.push_back(b); r->dz.push_back(c);
+    }
+    if (ok && r->tf32) {
+        ok = dalloc(r, &r->tc_error, 1);
+        for (size_t l = 0; ok && l < r->L.size(); ++l) {
+            float *a = nullptr, *b = nullptr;
+            const int ld = round_up(r->L[l].in, 4);
+            ok = dalloc(r, &a, (size_t)r->L[l].out * ld) && dalloc(r, &b, (size_t)r->L[l].out * ld);
+            r->wt_f.push_back(a); r->wt_g.push_back(b); r->ld_wt.push_back(ld);
+        }
     }
     if (ok) ok = cudaMemcpyAsync(r->idx, cfg->h_idx, sizeof(int) * r->ns, cudaMemcpyHostToDevice, r->stream) == cudaSuccess &&
                  cudaStreamSynchronize(r->stream) == cudaSuccess;
@@ -350,6 +477,11 @@ rslrl_status rslrl_rnd_set_params(rslrl_rnd* r, const float* h_predictor, const 
     RCU(r, cudaMemsetAsync(r->m, 0, sizeof(float) * r->P_dev, r->stream));
     RCU(r, cudaMemsetAsync(r->v, 0, sizeof(float) * r->P_dev, r->stream));
     RCU(r, cudaMemsetAsync(r->grad, 0, sizeof(float) * r->P_dev, r->stream));
+    if (r->tf32) {
+        rslrl_status ts = refresh_transposes(r, 0);
+        if (ts == RSLRL_OK) ts = refresh_transposes(r, 1);
+        if (ts != RSLRL_OK) return ts;
+    }
     RCU(r, cudaStreamSynchronize(r->stream));
     r->adam_step = 0;
     return RSLRL_OK;
@@ -360,7 +492,13 @@ static rslrl_status rnd_get_vec(rslrl_rnd* r, const float* d, float* h, size_t n
     if (n != r->P_flat) return rfail(r, RSLRL_ERR_SHAPE, "expected %zu parameters, got %zu", r->P_flat, n);
     std::vector<float> dev((size_t)r->P_dev);
     RCU(r, cudaMemcpyAsync(dev.data(), d, sizeof(float) * dev.size(), cudaMemcpyDeviceToHost, r->stream));
+    int code = 0;
+    if (r->tf32) RCU(r, cudaMemcpyAsync(&code, r->tc_error, sizeof(int), cudaMemcpyDeviceToHost, r->stream));
     RCU(r, cudaStreamSynchronize(r->stream));
+    if (code != 0) {                     // reported once
+        RCU(r, cudaMemsetAsync(r->tc_error, 0, sizeof(int), r->stream));
+        return rfail(r, RSLRL_ERR_TIMEOUT, "a bounded wait in a tensor-core kernel expired (role %d)", code);
+    }
     for (const RLayer& Ly : r->L) {
         for (int i = 0; i < Ly.in; ++i)
             for (int o = 0; o < Ly.out; ++o) h[Ly.w_flat + (size_t)i * Ly.out + o] = dev[Ly.w_off + (size_t)i * Ly.out_p + o];
@@ -412,7 +550,7 @@ rslrl_status rslrl_rnd_update(rslrl_rnd* r, const float* d_obs, int32_t batch, i
         if ((s = forward(r, n, false, true, r->gall + (size_t)r0 * r->ldE)) != RSLRL_OK) return s;
     }
     const int splits = splits_for(rows);
-    const int kchunk = round_up((rows + splits - 1) / splits, 8);
+    const int kchunk = kchunk_for(r, rows, splits);
     const int nloss = (rows + 7) / 8;
     const float scale = 1.0f / ((float)rows * (float)r->E);
     const rslrl_rnd_cfg& c = r->cfg;
@@ -438,6 +576,7 @@ rslrl_status rslrl_rnd_update(rslrl_rnd* r, const float* d_obs, int32_t batch, i
                                   (const float*)r->partials, splits, (size_t)r->P_dev, r->grad, r->pf, r->m, r->v, r->P_dev,
                                   c.lr, c.adam_b1, c.adam_b2, c.adam_eps, c1, c2, (const float*)r->loss_partials, nloss,
                                   1.0f / (float)rows, r->step_loss + done));
+            if (r->tf32 && (s = refresh_transposes(r, 0)) != RSLRL_OK) return s;      // the forward operands of the next step
         }
     }
     if (h_mean_loss || h_first_loss) {

@@ -770,7 +770,7 @@ cudaError_t tf32_read_error(Tf32Engine* e, int* host_code) {
 
 // ------------------------------------------------------------------ prepared launches for other callers
 struct Tf32Op {
-    int kind = 0;                 // TF_BIAS / TF_PLAIN: P; 100: W
+    int kind = 0;                 // a TfMode: P; 100: W
     TfParams P;
     TfWgParams W;
     int num_sms = 148;
@@ -806,7 +806,9 @@ bool tf32_ops_init(std::string* err) {
     int dev = 0; cudaDeviceProp prop;
     if (cudaGetDevice(&dev) != cudaSuccess || cudaGetDeviceProperties(&prop, dev) != cudaSuccess) return failmsg("no CUDA device");
     if (prop.major != 10) return failmsg("the tensor-core mode needs an sm_100 device");
-    if (cudaFuncSetAttribute(tf32_gemm_kernel<TF_BIAS>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kTfSmem) != cudaSuccess ||
+    if (cudaFuncSetAttribute(tf32_gemm_kernel<TF_FWD>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kTfSmem) != cudaSuccess ||
+        cudaFuncSetAttribute(tf32_gemm_kernel<TF_DGRAD>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kTfSmem) != cudaSuccess ||
+        cudaFuncSetAttribute(tf32_gemm_kernel<TF_BIAS>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kTfSmem) != cudaSuccess ||
         cudaFuncSetAttribute(tf32_gemm_kernel<TF_PLAIN>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kTfSmem) != cudaSuccess ||
         cudaFuncSetAttribute(tf32_wgrad_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kTfWgSmem) != cudaSuccess)
         return failmsg("could not reserve shared memory for the tensor-core kernels");
@@ -821,6 +823,19 @@ Tf32Op* tf32_op_gemm(const float* A, int rows, int k, int lda, const float* B, i
     memset(&op->P, 0, sizeof op->P);
     if (!add_problem(op->P, A, rows, rows, k, lda, B, n, ldb, D, ldd, nullptr, bias, n_store)) { delete op; return nullptr; }
     finish(op->P, 0.f, error_dev);
+    return op;
+}
+
+Tf32Op* tf32_op_gemm_act(int kind, const float* A, int rows, int k, int lda, const float* B, int n, int ldb, float* D, int ldd,
+                         const float* bias_or_aux, float alpha, int* error_dev, int n_store) {
+    if (!bias_or_aux || (kind != 0 && kind != 1)) return nullptr;
+    Tf32Op* op = new Tf32Op();
+    op->kind = kind == 0 ? TF_FWD : TF_DGRAD;
+    op->num_sms = device_sms();
+    memset(&op->P, 0, sizeof op->P);
+    if (!add_problem(op->P, A, rows, rows, k, lda, B, n, ldb, D, ldd, kind == 1 ? bias_or_aux : nullptr,
+                     kind == 0 ? bias_or_aux : nullptr, n_store)) { delete op; return nullptr; }
+    finish(op->P, alpha, error_dev);
     return op;
 }
 
@@ -861,6 +876,8 @@ cudaError_t tf32_op_launch(const Tf32Op* op, cudaStream_t stream) {
         LaunchScope scope_("tc_gemm_wgrad", stream);
         return launch_chained(tf32_wgrad_kernel, std::min(op->W.total_items, op->num_sms), kThreads, kTfWgSmem, stream, op->W);
     }
+    if (op->kind == TF_FWD) return launch_tf<TF_FWD>(op->P, op->num_sms, stream);
+    if (op->kind == TF_DGRAD) return launch_tf<TF_DGRAD>(op->P, op->num_sms, stream);
     if (op->kind == TF_BIAS) return launch_tf<TF_BIAS>(op->P, op->num_sms, stream);
     return launch_tf<TF_PLAIN>(op->P, op->num_sms, stream);
 }

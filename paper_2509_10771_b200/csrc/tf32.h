@@ -59,6 +59,10 @@ bool tf32_ops_init(std::string* err);
 // n_store (0: n): columns of D that are written; those from n on come out as zero.
 Tf32Op* tf32_op_gemm(const float* A, int rows, int k, int lda, const float* B, int n, int ldb, float* D, int ldd,
                      const float* bias, int* error_dev, int n_store = 0);
+// The same product with an activation epilogue: kind 0: D = ELU(A B^T + bias) (bias as above); kind 1: D = (A B^T) *
+// ELU'(aux), aux [rows][ldd] holding the stored post-activations.
+Tf32Op* tf32_op_gemm_act(int kind, const float* A, int rows, int k, int lda, const float* B, int n, int ldb, float* D, int ldd,
+                         const float* bias_or_aux, float alpha, int* error_dev, int n_store = 0);
 // out_i[s][m_i][ld_out_i] (s-th slice at s * split_stride floats) = A_i[rows s][m_i]^T B_i[rows s][n_i] for up to eight
 // pairs, rows s = [s * kchunk, (s + 1) * kchunk) cut at `rows`; kchunk a multiple of 32; n_store_i columns are written.
 struct Tf32WgradDesc { const float* A; int lda, m; const float* B; int ldb, n, n_store; float* out; int ld_out; };

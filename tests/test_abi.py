@@ -80,7 +80,9 @@ def test_rnd_and_gru_configs_without_a_device():
     cfg.max_epochs, cfg.max_minibatches = 1 << 11, 1 << 10          # more steps than one call may take
     assert lib.rslrl_rnd_num_params(ctypes.byref(cfg)) == 0
     assert ctypes.sizeof(binding.RndCfg) == 4 + 4 + 8 + 4 + 32 + 4 + 4 + 4 + 16 + 12 + 4 and binding.RndCfg.h_idx.offset == 8
-    assert binding.RndCfg.max_batch.offset == 80
+    assert binding.RndCfg.max_batch.offset == 80 and binding.RndCfg.precision.offset == 92
+    cfg.max_epochs, cfg.max_minibatches, cfg.precision = 5, 4, 7
+    assert lib.rslrl_rnd_num_params(ctypes.byref(cfg)) == 0        # no such precision
     g = binding.GruCfg(235, 256, 24, 4096)
     assert lib.rslrl_gru_num_params(ctypes.byref(g)) == 235 * 768 + 768 + 256 * 768 + 768
     assert lib.rslrl_gru_num_params(ctypes.byref(binding.GruCfg(235, 250, 24, 4096))) == 0     # H not a multiple of 4

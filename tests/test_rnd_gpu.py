@@ -25,7 +25,7 @@ CASES = {
 }
 
 
-def _setup(case, lr=1e-3):
+def _setup(case, lr=1e-3, precision=0):
     import torch
     from paper_2509_10771_b200 import binding
     w, rows, kw, mbs, epochs = CASES[case]
@@ -33,7 +33,8 @@ def _setup(case, lr=1e-3):
     ws = w.scaled(envs)
     obs = WL.make_rollout_inputs(ws)["obs_actor"][:w.num_steps].reshape(rows, w.actor_obs_dim)
     setup = WL.make_rnd_setup(ws, **kw)
-    rnd = binding.Rnd(w.actor_obs_dim, setup["idx"], setup["hidden"], setup["embed_dim"], max_rows=rows, lr=lr, max_batch=rows)
+    rnd = binding.Rnd(w.actor_obs_dim, setup["idx"], setup["hidden"], setup["embed_dim"], max_rows=rows, lr=lr, max_batch=rows,
+                      precision=precision)
     rnd.set_params(setup["predictor"], setup["target"])
     d_obs = torch.from_numpy(obs).to("cuda")
     return w, rows, setup, rnd, obs, d_obs, mbs, epochs
@@ -60,6 +61,37 @@ def test_intrinsic_reward_matches_oracle(case):
     torch.cuda.synchronize()
     assert torch.equal(d_int2[:rows // 3], d_int[:rows // 3])
     assert bool((d_int2[rows // 3:] == -1.0).all())
+    rnd.destroy()
+
+
+@pytest.mark.parametrize("case", ["tiny", "flat", "rough"])
+def test_reward_and_first_step_match_oracle_tf32(case):
+    """RSLRL_TF32: the products of both nets see TF32 operands (11 significant bits).  The reward of untrained nets and
+    the loss at the mode's tolerance 5e-3, the gradient at twice that per element and at 5e-3 in relative L2; the
+    parameters after Adam's first step (lr * sign(g)) as in the FP32 test."""
+    import torch
+    w, rows, setup, rnd, obs, d_obs, mbs, epochs = _setup(case, precision=WL.PRECISION_TF32)
+    ref_r, _, _, _ = O.rnd_reward(setup["predictor"], setup["target"], setup["dims"], obs, setup["idx"], 1.0)
+    d_int = torch.full((rows,), -1.0, device="cuda")
+    rnd.reward(d_obs, rows, w.actor_obs_dim, d_r_int_out=d_int)
+    torch.cuda.synchronize()
+    got_r = d_int.cpu().numpy()
+    assert_close(got_r, ref_r, 5e-3, "r_int")
+    fp32 = _setup(case)
+    d_int32 = torch.full((rows,), -1.0, device="cuda")
+    fp32[3].reward(d_obs, rows, w.actor_obs_dim, d_r_int_out=d_int32)
+    torch.cuda.synchronize()
+    assert not np.array_equal(got_r, d_int32.cpu().numpy())          # the tensor cores did see TF32 operands
+    fp32[3].destroy()
+    hp = SimpleNamespace(epochs=epochs, minibatches=mbs, elu_alpha=1.0, adam_b1=0.9, adam_b2=0.999, adam_eps=1e-8)
+    out = rnd.update(d_obs, rows, w.actor_obs_dim, epochs, mbs, seed=7, iteration=3, max_steps=1)
+    state = O.OptimState(setup["predictor"], 1e-3)
+    ref = O.rnd_update(state, setup["target"], setup["dims"], obs, setup["idx"], hp, seed=7, iteration=3, max_steps=1)
+    assert_close(out["first_loss"], ref[0]["loss"], 5e-3, "loss")
+    g = rnd.get_grads()
+    assert_close(g, ref[0]["grad"], 1e-2, "grad")
+    assert rel_l2(g, ref[0]["grad"]) < 5e-3
+    assert_close(rnd.get_params(), state.theta, 1e-4, "params", max_outlier_frac=2e-2, outlier_abs=2.05e-3)
     rnd.destroy()
 
 
