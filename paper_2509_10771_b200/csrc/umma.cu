@@ -893,8 +893,47 @@ __global__ void __launch_bounds__(kThreads, 1) chain_fwd_kernel(const __grid_con
                     continue;
                 }
                 const bool active = 64 * g < E.ncols;          // uniform across the warp
+                // Nothing still reads the activation buffer: the results go to it as they are formed, 16 accumulator
+                // columns at a time, the next 16 in flight meanwhile.
+                const bool direct = active && E.write_job < 0;
+                if (direct) {
+                    if (P.store) {
+                        if (lane == 0) tma_store_wait_read();   // this warp's last store has read the rows
+                        __syncwarp();
+                    }
+                    const float* bias = sBias + N.bias_off[E.layer] + E.n0 + 64 * g;
+                    const uint32_t t_row = tmem_base + ((uint32_t)(32 * q) << 16) + (((uint32_t)E.tmem_col ^ flip) + (uint32_t)(64 * g));
+                    uint32_t acc[2][16];
+                    tmem_ld16_issue(t_row, acc[0]);
+#pragma unroll
+                    for (int pc = 0; pc < 4; ++pc) {
+                        uint32_t (&cur)[16] = acc[pc & 1];
+                        float bv[16];
+                        const float4* b4 = reinterpret_cast<const float4*>(bias + 16 * pc);
+#pragma unroll
+                        for (int gg = 0; gg < 4; ++gg) {
+                            const float4 t4 = b4[gg];
+                            bv[4 * gg] = t4.x; bv[4 * gg + 1] = t4.y; bv[4 * gg + 2] = t4.z; bv[4 * gg + 3] = t4.w;
+                        }
+                        tmem_ld16_wait(cur);
+                        if (pc < 3) tmem_ld16_issue(t_row + (uint32_t)(16 * (pc + 1)), acc[(pc + 1) & 1]);
+#pragma unroll
+                        for (int gq = 0; gq < 2; ++gq) {
+                            uint32_t o[4];
+#pragma unroll
+                            for (int k = 0; k < 4; ++k) {
+                                const float v0 = elu_fast(__uint_as_float(cur[8 * gq + 2 * k]) + bv[8 * gq + 2 * k], P.alpha);
+                                const float v1 = elu_fast(__uint_as_float(cur[8 * gq + 2 * k + 1]) + bv[8 * gq + 2 * k + 1], P.alpha);
+                                __nv_bfloat162 h2 = __floats2bfloat162_rn(v0, v1);
+                                o[k] = *reinterpret_cast<uint32_t*>(&h2);
+                            }
+                            *reinterpret_cast<uint4*>(tile_row + (((2 * pc + gq) ^ sw) << 4)) = make_uint4(o[0], o[1], o[2], o[3]);
+                        }
+                    }
+                    fence_async_smem();                         // rows -> visible to the MMA and the copy engine
+                }
                 uint4 outv[8];
-                if (active) {
+                if (active && !direct) {
                     const float* bias = sBias + N.bias_off[E.layer] + E.n0 + 64 * g;
 #pragma unroll
                     for (int ci = 0; ci < 2; ++ci) {
@@ -919,7 +958,7 @@ __global__ void __launch_bounds__(kThreads, 1) chain_fwd_kernel(const __grid_con
                 }
                 // the accumulator is in registers; the buffer may still feed a job that runs meanwhile
                 if (E.write_job >= 0 && !mbar_wait(&job_done[E.write_job], t & 1u, abort_flag, P.error, 15)) { ok = false; break; }
-                if (active) {
+                if (active && !direct) {
                     if (P.store) {
                         if (lane == 0) tma_store_wait_read();   // this warp's last store has read the rows
                         __syncwarp();
