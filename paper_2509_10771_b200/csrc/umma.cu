@@ -663,21 +663,26 @@ __global__ void __launch_bounds__(kThreads, 1) chain_fwd_kernel(const __grid_con
     volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-    if (threadIdx.x == 0) {
-        for (int s = 0; s < kSlots; ++s) { mbar_init(&full[s], 1); mbar_init(&empty[s], 1); }
-        for (int j = 0; j < kChainJobs; ++j) mbar_init(&job_done[j], 1);
-        for (int e = 0; e < kChainEpis; ++e) mbar_init(&epi_done[e], kEpiWarps);
-        mbar_init(drain, 1);
-        *abort_flag = 0;
+    // set-up spread over lanes (a single thread pays about five cycles per dependent instruction): warp 0 initialises
+    // the barriers, a lane each; warp 1 allocates tensor memory; warp 2 prefetches the tensor maps, a lane each
+    if (warp == 0) {
+        if (lane < kSlots) { mbar_init(&full[lane], 1); mbar_init(&empty[lane], 1); }
+        if (lane < kChainJobs) mbar_init(&job_done[lane], 1);
+        if (lane < kChainEpis) mbar_init(&epi_done[lane], kEpiWarps);
+        if (lane == 0) { mbar_init(drain, 1); *abort_flag = 0; }
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
         asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
     }
     if (warp == 1) tmem_alloc(tmem_slot, kTmemCols);
-    if (warp == 0 && lane == 0)
-        for (int n = 0; n < P.nnets; ++n) {
-            tma_prefetch_desc(&P.tmX[n]);
-            for (int l = 0; l < P.net[n].nlayers; ++l) { tma_prefetch_desc(&P.tmW[n][l]); tma_prefetch_desc(&P.tmOut[n][l]); }
+    if (warp == 2) {
+        constexpr int per_net = 1 + 2 * kChainLayers;
+        const int n = lane / per_net, r = lane - n * per_net;
+        if (n < P.nnets) {
+            if (r == 0) tma_prefetch_desc(&P.tmX[n]);
+            else if (r - 1 < P.net[n].nlayers) tma_prefetch_desc(&P.tmW[n][r - 1]);
+            else if (r - 1 - kChainLayers >= 0 && r - 1 - kChainLayers < P.net[n].nlayers) tma_prefetch_desc(&P.tmOut[n][r - 1 - kChainLayers]);
         }
+    }
     tc_fence_before();
     __syncthreads();
     tc_fence_after();
