@@ -288,14 +288,15 @@ __global__ void __launch_bounds__(kThreads, 1) tf32_gemm_kernel(const __grid_con
 // dW[features_in x features_out] = X^T dZ over the minibatch rows, both operands as stored ([row][feature], the
 // contraction index outermost: MN-major tiles of 32 features x 32 rows, one 128-byte row per minibatch row, swizzled
 // in units of 32 bytes, the form the tensor cores take for MN-major operands of 32-bit elements).
-// A work item is a 128 x (<= 128) tile of one layer over one split of the row range; its FP32 result is a partial
+// A work item is a 128 x (<= 256) tile of one layer over one split of the row range; its FP32 result is a partial
 // that the gradient reduction sums.  A split without rows (the row range does not always fill the last one) writes
 // zeros.
 constexpr int kTfWgProblems = 2 * kMaxLayers;     // every layer of both nets
 constexpr int kTfWgStages = 4;
 constexpr uint32_t kTfWgBox = 32 * 32 * 4;        // 4 KiB: 32 features x 32 rows
 constexpr uint32_t kTfWgStageA = 4 * kTfWgBox;    // 128 features
-constexpr uint32_t kTfWgStageB = 4 * kTfWgBox;    // up to 128 features
+constexpr int kTfWgMaxBN = 256;                   // output features per tile
+constexpr uint32_t kTfWgStageB = (kTfWgMaxBN / 32) * kTfWgBox;    // up to 256 features
 constexpr size_t kTfWgSmem = 1024 + (size_t)kTfWgStages * (kTfWgStageA + kTfWgStageB) + 512;
 
 struct TfWgProblem {
@@ -383,7 +384,7 @@ __global__ void __launch_bounds__(kThreads, 1) tf32_wgrad_kernel(const __grid_co
 
     if (warp == 0) {
         // ================================ TMA producer =================================
-        // a k-block is up to eight boxes of 32 features x 32 rows (four of A, up to four of B): lane l issues box l
+        // a k-block is up to twelve boxes of 32 features x 32 rows (four of A, up to eight of B): lane l issues box l
         int stage = 0; uint32_t phase = 0;
         uint32_t issued_mask = 0, issued_parity = 0;
         bool ok = true;
@@ -463,7 +464,7 @@ __global__ void __launch_bounds__(kThreads, 1) tf32_wgrad_kernel(const __grid_co
     } else {
         // ================================ epilogue =====================================
         const int q = warp & 3;                    // accumulator lanes 32q .. 32q+31
-        const int group = (warp - 2) >> 2;         // columns [32 group, 32 group + 32) of the tile
+        const int group = (warp - 2) >> 2;         // chunks of 32 columns: group and group + 4
         bool ok = true;
         int local = 0;
         for (int item = blockIdx.x; ok && item < P.total_items; item += gridDim.x, ++local) {
@@ -472,13 +473,16 @@ __global__ void __launch_bounds__(kThreads, 1) tf32_wgrad_kernel(const __grid_co
             const int buf = local & 1;
             const uint32_t use = (uint32_t)(local >> 1);
             const int row = it.m0 + 32 * q + lane;
-            const int col = it.n0 + 32 * group;
-            const bool active = 32 * group < p.bn && col < p.n_store;   // uniform across the warp
             if (!mbar_wait(&tfull[buf], use & 1u, abort_flag, P.error, 24)) { ok = false; break; }
             tc_fence_after();
-            if (active) {
+            // a warp takes the 32-column chunks `group` and `group + 4` of the tile
+#pragma unroll
+            for (int ci = 0; ci < 2; ++ci) {
+                const int chunk = group + 4 * ci;
+                const int col = it.n0 + 32 * chunk;
+                if (32 * chunk >= p.bn || col >= p.n_store) break;          // uniform across the warp
                 uint32_t acc[32];
-                tmem_ld32(tmem_base + ((uint32_t)(32 * q) << 16) + (uint32_t)(buf * kMaxBN + 32 * group), acc);
+                tmem_ld32(tmem_base + ((uint32_t)(32 * q) << 16) + (uint32_t)(buf * kMaxBN + 32 * chunk), acc);
                 if (it.kb0 >= it.kb1) {
 #pragma unroll
                     for (int i = 0; i < 32; ++i) acc[i] = 0u;             // nothing was accumulated
@@ -694,7 +698,7 @@ Tf32Engine* tf32_create(const Tf32Setup& s, std::string* err) {
                 const float* dz = head ? s.dhead[ni] : s.up_dz[ni][l];
                 const int lddz = head ? s.ld_dhead[ni] : s.hid_ld[ni][l];
                 p.m_extent = s.in[ni][l]; p.n_store = s.out_p[ni][l];
-                p.bn = std::min(kTfMaxBN, round_up(s.out[ni][l], 32));
+                p.bn = std::min(kTfWgMaxBN, round_up(s.out[ni][l], 32));
                 p.m_tiles = (p.m_extent + BLOCK_M - 1) / BLOCK_M;
                 p.n_tiles = (p.n_store + p.bn - 1) / p.bn;
                 p.kblocks = (s.R + kTfBlockK - 1) / kTfBlockK;
@@ -850,7 +854,7 @@ Tf32Op* tf32_op_wgrad(const Tf32WgradDesc* d, int count, int rows, int splits, i
     for (int i = 0; i < count; ++i) {
         TfWgProblem& p = W.p[i];
         p.m_extent = d[i].m; p.n_store = d[i].n_store;
-        p.bn = std::min(kTfMaxBN, round_up(d[i].n, 32));
+        p.bn = std::min(kTfWgMaxBN, round_up(d[i].n, 32));
         p.m_tiles = (p.m_extent + BLOCK_M - 1) / BLOCK_M;
         p.n_tiles = (p.n_store + p.bn - 1) / p.bn;
         p.kblocks = (rows + kTfBlockK - 1) / kTfBlockK;
