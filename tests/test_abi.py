@@ -89,3 +89,24 @@ def test_rnd_and_gru_configs_without_a_device():
     assert lib.rslrl_gru_num_params(ctypes.byref(binding.GruCfg(235, 256, 1 << 15, 1 << 15))) == 0   # T * N too large
     assert ctypes.sizeof(binding.GruCfg) == 20 and binding.GruCfg.precision.offset == 16
     assert lib.rslrl_gru_num_params(ctypes.byref(binding.GruCfg(235, 256, 24, 4096, 3))) == 0          # no such precision
+
+
+def test_side_objects_refuse_the_bf16_mode_without_a_device():
+    """The recurrent layer and random network distillation have FP32 and TF32 modes; asking for BF16 is refused by the
+    host code before any device call."""
+    import numpy as np
+    from paper_2509_10771_b200 import binding, build
+    build.build()
+    lib = binding.load_library()
+    h = ctypes.c_void_p()
+    g = binding.GruCfg(16, 8, 4, 32, 2)
+    assert lib.rslrl_gru_create(ctypes.byref(g), None, ctypes.byref(h)) == 5 and not h.value
+    idx = np.array([0, 1], dtype=np.int32)
+    cfg = binding.RndCfg()
+    cfg.obs_dim, cfg.num_idx, cfg.h_idx, cfg.num_hidden = 4, 2, idx.ctypes.data, 1
+    cfg.hidden[0] = 8
+    cfg.embed_dim, cfg.elu_alpha, cfg.max_rows = 4, 1.0, 16
+    cfg.lr, cfg.adam_b1, cfg.adam_b2, cfg.adam_eps = 1e-3, 0.9, 0.999, 1e-8
+    cfg.max_batch, cfg.max_epochs, cfg.max_minibatches, cfg.precision = 16, 1, 1, 2
+    assert lib.rslrl_rnd_create(ctypes.byref(cfg), None, ctypes.byref(h)) == 5 and not h.value
+
