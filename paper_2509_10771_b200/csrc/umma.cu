@@ -659,7 +659,8 @@ __global__ void __launch_bounds__(kThreads, 1) chain_fwd_kernel(const __grid_con
     uint64_t* job_done = empty + kSlots;       // one completion per item each
     uint64_t* epi_done = job_done + kChainJobs;
     uint64_t* drain = epi_done + kChainEpis;
-    uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(drain + 1);
+    uint64_t* head_bar = drain + 1;            // one per lane quarter: the three other warps of a row group have written their partials
+    uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(head_bar + 4);
     volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
@@ -670,6 +671,7 @@ __global__ void __launch_bounds__(kThreads, 1) chain_fwd_kernel(const __grid_con
         if (lane < kChainJobs) mbar_init(&job_done[lane], 1);
         if (lane < kChainEpis) mbar_init(&epi_done[lane], kEpiWarps);
         if (lane == 0) { mbar_init(drain, 1); *abort_flag = 0; }
+        if (lane < 4) mbar_init(&head_bar[lane], 3);
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
         asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
     }
@@ -826,6 +828,7 @@ __global__ void __launch_bounds__(kThreads, 1) chain_fwd_kernel(const __grid_con
         const int sw = lane & 7;
         bool ok = true;
         uint32_t t = 0;
+        uint32_t head_uses = 0;                    // policy-head epilogues this warp has waited for
         for (int item = blockIdx.x; ok && item < P.total_items; item += gridDim.x, ++t) {
             const int ni = item % P.nnets, m0 = (item / P.nnets) * BLOCK_M;
             const ChainNet& N = P.net[ni];
@@ -875,17 +878,25 @@ __global__ void __launch_bounds__(kThreads, 1) chain_fwd_kernel(const __grid_con
                                 if (orow) { orow[c] = av[0]; orow[c + 1] = av[1]; orow[c + 2] = av[2]; orow[c + 3] = av[3]; }   // caller's buffer: 4-byte aligned only
                             }
                         }
-                        // the row's log-probability: the partials of the four warps, added in the order of the actions
+                        // the row's log-probability: the partials of the four warps, added in the order of the actions.
+                        // The three other warps publish theirs and arrive on the row group's barrier; the first warp
+                        // waits for them with the usual bound.  The next item's partials cannot be written before this
+                        // epilogue has been reported done by all of its warps (the item's first job waits for that).
                         float* part = sHead + 256;
-                        part[(4 * q + g) * 32 + lane] = logp;
-                        asm volatile("bar.sync %0, 128;" ::"r"(2 + q) : "memory");
-                        if (g == 0 && live) {
-                            float lp = part[(4 * q) * 32 + lane];
+                        if (g != 0) {
+                            part[(4 * q + g) * 32 + lane] = logp;
+                            __syncwarp();
+                            if (lane == 0) mbar_arrive(&head_bar[q]);
+                        } else {
+                            if (!mbar_wait(&head_bar[q], head_uses & 1u, abort_flag, P.error, 16)) { ok = false; break; }
+                            ++head_uses;
+                            if (live) {
+                                float lp = logp;
 #pragma unroll
-                            for (int gg = 1; gg < 4; ++gg) lp += part[(4 * q + gg) * 32 + lane];
-                            H.logp[n] = lp;
+                                for (int gg = 1; gg < 4; ++gg) lp += part[(4 * q + gg) * 32 + lane];
+                                H.logp[n] = lp;
+                            }
                         }
-                        asm volatile("bar.sync %0, 128;" ::"r"(2 + q) : "memory");      // the partials may be overwritten
                     } else if (g == 0) {
                         uint32_t a4[4], l4[4];
                         tmem_ld4(taddr, a4);
