@@ -702,7 +702,8 @@ def run_streams(args):
     """--task streams: the scan kernels at a bandwidth-shaped size through the stand-alone entry point (rslrl_gae_scan,
     T = 32 steps x 1,048,576 environments, 872 MB of algorithmic traffic per call), one GPU.  The learn iteration's own
     scan moves 2.6 MB and is bound by launch latency; this line is where the scan meets its memory roofline.  Its own
-    JSON line; the gather's and Adam's figures at their own sizes are in the ppo line (roofline.hbm_families)."""
+    JSON line; the gather's and Adam's figures at their own sizes are in the ppo line (roofline.hbm_families).  The line
+    also carries Adam and the gradient reduction at 36 M parameters (the FP32 mode's update of two wide nets)."""
     import torch
     from paper_2509_10771_b200 import binding, build
     if not torch.cuda.is_available():
@@ -735,6 +736,43 @@ def run_streams(args):
         us = 1e3 * sum(a.elapsed_time(b) for a, b in evs) / args.steps
         gbs = nbytes / (us * 1e-6) / 1e9
         out[name] = {"bytes_per_call": nbytes, "us": us, "gbs": gbs, "frac": gbs / peaks["hbm_gbs"], "frac_of_nominal_7700": gbs / 7700.0}
+    # Adam (and the gradient reduction in front of it) at a bandwidth-shaped size: the FP32 mode's update of two
+    # 64-4096-4096-256 nets (36 M parameters, 1 GB of algorithmic traffic per Adam launch) on a 512-transition rollout;
+    # per-launch CUDA events of the library's own accounting
+    del r, v, lv, d, to, ret, adv, scratch
+    from dataclasses import replace
+    w = replace(WL.TINY, name="wide_nets_for_adam", actor_obs_dim=64, critic_obs_dim=64, actor_hidden=(4096, 4096, 256),
+                critic_hidden=(4096, 4096, 256), actor_obs_blocks=((64, "normal"),), critic_obs_blocks=((64, "normal"),))
+    ctx = binding.Context(w, precision=WL.PRECISION_FP32, stream=stream.cuda_stream)
+    ctx.set_params(WL.make_params(w))
+    inp = WL.make_rollout_inputs(w)
+    d_o = torch.from_numpy(inp["obs_actor"]).to(dev)
+    d_r, d_d, d_t = (torch.from_numpy(inp[k]).to(dev) for k in ("rewards", "dones", "timeouts"))
+
+    def wide_iteration():
+        for t in range(w.num_steps):
+            ctx.act(d_o[t]); ctx.record_step(d_r[t], d_d[t], d_t[t])
+        ctx.gae(d_o[w.num_steps])
+        ctx.ppo_update(want_stats=False)
+
+    for _ in range(3):
+        wide_iteration()
+    torch.cuda.synchronize()
+    binding.profile_enable(True)
+    binding.profile_report()
+    for _ in range(max(2, args.steps // 4)):
+        wide_iteration()
+    torch.cuda.synchronize()
+    rep = binding.profile_report()
+    binding.profile_enable(False)
+    P = ctx.num_params
+    for name, per_param in (("adam", 28), ("grad_reduce", 8)):
+        if name in rep and rep[name]["launches"]:
+            us = 1e3 * rep[name]["ms"] / rep[name]["launches"]
+            gbs = per_param * P / (us * 1e-6) / 1e9
+            out[name + "_36M_parameters"] = {"bytes_per_call": per_param * P, "us": us, "gbs": gbs, "frac": gbs / peaks["hbm_gbs"],
+                                             "frac_of_nominal_7700": gbs / 7700.0}
+    ctx.destroy()
     both = out["gae_scan+gae_normalize"]
     line = {
         "metric": "GAE scan + advantage normalisation transitions/s", "value": T * N / (both["us"] * 1e-6), "unit": UNIT, "n_gpus": 1,
