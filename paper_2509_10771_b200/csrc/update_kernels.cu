@@ -40,8 +40,8 @@ __device__ __forceinline__ void store_obs_piece(float* dst, __nv_bfloat16* dst16
 // bandwidth of this kernel is the bytes it keeps in flight, so this loop carries nothing but the rows; the small
 // per-row items are gathered by a second loop with one thread per row.  Storage is read through the read-only path
 // (it does not change while an update runs).
-// Two shapes of the kernel are launched.  The first gather of an update runs alone and is built for bandwidth:
-// eight rows per pass, 256 threads, two blocks per SM.  The others run on a second stream beside the tensor-core
+// Two shapes of the kernel are launched.  The first gather of an update runs alone and, unless rows are mirrored, in
+// the shape built for that: eight rows per pass, 256 threads, two blocks per SM.  The others run on a second stream beside the tensor-core
 // kernels of the minibatch step before, whose CTAs hold an SM's shared memory and 55,296 of its 65,536
 // registers: two rows per pass, 128 threads and at most 80 registers make a block that fits beside such a CTA
 // (10,240 registers, no shared memory), so these gathers really run meanwhile instead of taking SMs in turn.
@@ -813,7 +813,9 @@ cudaError_t launch_gather(const GatherArgs& a, cudaStream_t s, bool alone) {
     // (accounting only) the first gather of an update runs while the caller's stream waits for it, the others beside
     // the kernels of the minibatch step before
     LaunchScope scope_(alone ? "gather_alone" : "gather", s);
-    if (alone) {
+    // (with mirrored copies the small shape is also the faster one alone: 73.7 against 78.9 us at 131,072 rows, its
+    // 24 warps per SM cover the mirror's reads through L1 better than 16 warps with more rows each)
+    if (alone && !a.sym) {
         const int blocks = std::min((a.Bmb + 8 * kGatherRowsAlone - 1) / (8 * kGatherRowsAlone), 148 * 2);   // one resident wave
         return launch_chained(gather_kernel<kGatherRowsAlone, 256, 2>, blocks, 256, 0, s, a);
     }
